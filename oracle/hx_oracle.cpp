@@ -1,0 +1,321 @@
+// CPU oracle for batched placement scoring and workflow horizons.
+//
+// TEST INFRASTRUCTURE ONLY.  This file is the slow, plain, single-threaded
+// definition that the CUDA library is checked against.  It shares no code,
+// header, table or helper with the CUDA path and must never be called from it.
+// Build with:  g++ -O2 -ffp-contract=off -std=c++17 -shared -fPIC
+// (-ffp-contract=off: every rounding below is written out; the compiler must
+// not fuse a multiply and an add on its own).
+//
+// What the paper fixes and what it leaves open
+//   * Horizon H_w(t) = stand-alone completion time of the revealed sub-DAG
+//     (Section 5.1, "Define online workflow horizon").  With one cost per node
+//     this is the longest node-weighted path: orc_longest_path.     [pinned]
+//   * Projected ratio R = ((t - a_w) + Delta) / H_w(t)  (Eq. 2).      [pinned]
+//   * Decode demand m = L_in + L_out and feasibility m <= Cap(d)
+//     (Eq. 3, Eq. 4).                                                [pinned]
+//   * A call goes to the prefill/decode pair with the earliest projected
+//     decode finish (Section 5.3, "Adaptive greedy prefill assignment");
+//     Delta is built from waiting time, prefill time, KV-transfer latency and
+//     the earliest decode finish on the candidate decode instance
+//     (Section 5.1 and 5.3).                                          [pinned]
+//   * The paper names a "roofline-style" latency model (Section 4.2,
+//     Section 6) but prints no formula and no worked example.  The formulas in
+//     latency_terms() are this project's reading of that sentence.  They are
+//     pinned to hand-computed values of that reading, not to the paper:
+//     PARITY UNPINNED for the constants and the exact shape of the prefill,
+//     decode and transfer terms.
+//   * Large queues use a one-pass ordering by the same risk score
+//     (Section 5.3 last sentence, Section 5.4); the top-K list and the
+//     capacity-conflict pass below are this project's reading of that
+//     sentence together with Eq. 4.                    [pinned as defined]
+//
+// All placement arithmetic is IEEE binary32 in the order written here, because
+// a float comparison decides an integer (the chosen pair, the priority order)
+// and both sides must take that decision in the same precision.  The *_f64
+// twin evaluates the same model in double, in textbook form, to measure how far
+// the binary32 sequence is from the real-number value.
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <limits>
+#include <vector>
+#include <algorithm>
+
+extern "C" {
+
+struct OrcCluster {
+    int32_t G, P, D, M;
+    const float* peak_tflops;   // [G]
+    const float* hbm_tbps;      // [G]
+    const uint32_t* typeP;      // [P]
+    const uint32_t* typeD;      // [D]
+    const float* qP;            // [P] seconds until prefill instance p is free
+    const float* qD;            // [D] earliest time decode instance d can admit
+    const float* capD;          // [D] KV capacity in tokens (Eq. 4)
+    const float* link_gbps;     // [P*D] effective bandwidth prefill p -> decode d
+    const float* flops_per_token;   // [M]
+    const float* weight_bytes;      // [M]
+    const float* kv_bytes_per_token;// [M]
+};
+
+struct OrcCall { uint32_t node, model; float prompt_tokens, output_tokens; };
+
+struct OrcDag {                 // results of orc_longest_path, consumed by the scorer
+    const uint32_t* node_wf;    // [N]
+    const float* tail;          // [N]
+    const float* H;             // [W]
+    const float* elapsed;       // [W]
+};
+
+enum { ORC_MODE_COMPLETION = 0, ORC_MODE_SLACK = 1, ORC_MODE_RATIO = 2 };
+enum { ORC_FLAG_NO_DAG = 1, ORC_FLAG_NO_TAIL = 2, ORC_FLAG_UNLOADED = 4 };
+
+}  // extern "C"
+
+namespace {
+
+const float INF = std::numeric_limits<float>::infinity();
+
+// Per-call, per-GPU-class service times (reading of the "roofline-style model",
+// Section 4.2 "Scheduler internals").
+//   prefill  = max(compute time, memory time) of one pass over the prompt
+//   decode   = output tokens x (weights + KV of the average context) / HBM bandwidth
+struct Terms { float kvB, m; std::vector<float> tpre, tdec; };
+
+void latency_terms(const OrcCluster& cl, const OrcCall& c, Terms& t) {
+    const float n = c.prompt_tokens, o = c.output_tokens;
+    const float phi = cl.flops_per_token[c.model];
+    const float omega = cl.weight_bytes[c.model];
+    const float kappa = cl.kv_bytes_per_token[c.model];
+    t.kvB = n * kappa;                                  // KV bytes of the prompt
+    t.m = n + o;                                        // Eq. 3
+    t.tpre.resize(cl.G);
+    t.tdec.resize(cl.G);
+    const float ctx = std::fmaf(0.5f, o - 1.0f, n);     // average context length while decoding
+    const float step = std::fmaf(kappa, ctx, omega);    // bytes read per decode step
+    for (int g = 0; g < cl.G; ++g) {
+        const float invF = 1.0f / (cl.peak_tflops[g] * 1e12f);
+        const float invB = 1.0f / (cl.hbm_tbps[g] * 1e12f);
+        const float pf = (n * phi) * invF;
+        const float pm = (omega + t.kvB) * invB;
+        t.tpre[g] = std::fmax(pf, pm);
+        t.tdec[g] = (o * step) * invB;
+    }
+}
+
+// Projected decode finish of call c on pair (p, d), measured from now
+// (Section 5.3: prefill finish, plus transfer latency, then the earliest decode
+// finish given the decode availability hint; Eq. 4 masks infeasible instances).
+float candidate_fin(const OrcCluster& cl, const Terms& t, int p, int d, bool unloaded) {
+    const float qp = unloaded ? 0.0f : cl.qP[p];
+    const float qd = unloaded ? 0.0f : cl.qD[d];
+    const float invL = 1.0f / (cl.link_gbps[(size_t)p * cl.D + d] * 1e9f);
+    const float A = qp + t.tpre[cl.typeP[p]];                   // prefill finish
+    const float ready = std::fmaf(t.kvB, invL, A);              // KV arrives at d
+    const float start = std::fmax(ready, qd);                   // decode admission
+    const float Dd = (t.m <= cl.capD[d]) ? t.tdec[cl.typeD[d]] : INF;   // Eq. 4
+    return start + Dd;
+}
+
+struct DagView { float elapsed, tail, H; };
+
+DagView dag_view(const OrcDag* dag, const OrcCall& c, int flags) {
+    DagView v{0.0f, 0.0f, 1.0f};
+    if (!(flags & ORC_FLAG_NO_DAG) && dag) {
+        const uint32_t w = dag->node_wf[c.node];
+        v.elapsed = dag->elapsed[w];
+        v.tail = dag->tail[c.node];
+        v.H = dag->H[w];
+    }
+    return v;
+}
+
+}  // namespace
+
+extern "C" {
+
+// fin[c][p][d] for every candidate.
+int orc_fin_all(const OrcCluster* cl, const OrcCall* calls, int C, int flags, float* fin) {
+    Terms t;
+    for (int c = 0; c < C; ++c) {
+        latency_terms(*cl, calls[c], t);
+        for (int p = 0; p < cl->P; ++p)
+            for (int d = 0; d < cl->D; ++d)
+                fin[((size_t)c * cl->P + p) * cl->D + d] =
+                    candidate_fin(*cl, t, p, d, flags & ORC_FLAG_UNLOADED);
+    }
+    return 0;
+}
+
+// Per-class service times of each call: tpre[c][g], tdec[c][g], kvB[c], m[c].
+int orc_terms(const OrcCluster* cl, const OrcCall* calls, int C,
+              float* tpre, float* tdec, float* kvB, float* m) {
+    Terms t;
+    for (int c = 0; c < C; ++c) {
+        latency_terms(*cl, calls[c], t);
+        for (int g = 0; g < cl->G; ++g) { tpre[(size_t)c * cl->G + g] = t.tpre[g]; tdec[(size_t)c * cl->G + g] = t.tdec[g]; }
+        kvB[c] = t.kvB; m[c] = t.m;
+    }
+    return 0;
+}
+
+// Placement of every call against the snapshot: earliest projected decode
+// finish over all pairs, lowest pair index p*D+d on ties; -1 / +inf when no
+// decode instance can hold the call.  out_cost follows the score mode:
+//   completion = (elapsed + Delta) + tail          (projected workflow completion)
+//   slack      = alpha * H - completion
+//   ratio      = completion / H        (Eq. 2 when ORC_FLAG_NO_TAIL drops the tail)
+int orc_schedule(const OrcCluster* cl, const OrcDag* dag, const OrcCall* calls, int C,
+                 int mode, float alpha, int flags,
+                 int32_t* out_assign, float* out_cost, float* out_delta) {
+    Terms t;
+    for (int c = 0; c < C; ++c) {
+        latency_terms(*cl, calls[c], t);
+        float best = INF; int32_t arg = -1;
+        for (int p = 0; p < cl->P; ++p)
+            for (int d = 0; d < cl->D; ++d) {
+                const float f = candidate_fin(*cl, t, p, d, flags & ORC_FLAG_UNLOADED);
+                if (f < best) { best = f; arg = p * cl->D + d; }
+            }
+        const DagView v = dag_view(dag, calls[c], flags);
+        const float tail = (flags & ORC_FLAG_NO_TAIL) ? 0.0f : v.tail;
+        const float comp = (v.elapsed + best) + tail;
+        float score = comp;
+        if (mode == ORC_MODE_SLACK) { const float slo = alpha * v.H; score = slo - comp; }
+        else if (mode == ORC_MODE_RATIO) score = comp / v.H;
+        out_assign[c] = arg;
+        out_cost[c] = score;
+        if (out_delta) out_delta[c] = best;
+    }
+    return 0;
+}
+
+// For every call: its K cheapest distinct decode instances, each with its best
+// prefill partner (lowest p on ties), ordered by (cost, d).  Unused slots hold
+// pair -1, cost +inf.  prio = (elapsed + Delta*) / H (Eq. 2), m = Eq. 3 demand,
+// tpre_sel[c][k] = prefill time of call c on the prefill instance of slot k.
+int orc_topk(const OrcCluster* cl, const OrcDag* dag, const OrcCall* calls, int C, int K, int flags,
+             int32_t* pair, float* cost, float* prio, float* m, float* tpre_sel) {
+    Terms t;
+    std::vector<float> bestd(cl->D);
+    std::vector<int> bestp(cl->D);
+    std::vector<char> used(cl->D);
+    for (int c = 0; c < C; ++c) {
+        latency_terms(*cl, calls[c], t);
+        for (int d = 0; d < cl->D; ++d) {
+            bestd[d] = INF; bestp[d] = -1; used[d] = 0;
+            for (int p = 0; p < cl->P; ++p) {
+                const float f = candidate_fin(*cl, t, p, d, flags & ORC_FLAG_UNLOADED);
+                if (f < bestd[d]) { bestd[d] = f; bestp[d] = p; }
+            }
+        }
+        float delta = INF;
+        for (int k = 0; k < K; ++k) {
+            int arg = -1; float b = INF;
+            for (int d = 0; d < cl->D; ++d)
+                if (!used[d] && bestd[d] < b) { b = bestd[d]; arg = d; }
+            const size_t o = (size_t)c * K + k;
+            if (arg < 0) { pair[o] = -1; cost[o] = INF; tpre_sel[o] = 0.0f; continue; }
+            used[arg] = 1;
+            pair[o] = bestp[arg] * cl->D + arg;
+            cost[o] = b;
+            tpre_sel[o] = t.tpre[cl->typeP[bestp[arg]]];
+            if (k == 0) delta = b;
+        }
+        const DagView v = dag_view(dag, calls[c], flags);
+        prio[c] = (v.elapsed + delta) / v.H;
+        m[c] = t.m;
+    }
+    return 0;
+}
+
+// Capacity-conflict pass over one chunk.  Calls are visited by decreasing prio
+// (lower call index first among equals).  A call takes the first of its K
+// candidates whose decode instance still has free KV tokens for it; that
+// consumes the tokens and lengthens the chosen prefill queue by the call's
+// prefill time.  A call none of whose candidates fits stays unplaced (-1).
+// freeD[D] and qP[P] are updated in place.
+int orc_conflict(int C, int K, int D, const int32_t* pair, const float* prio, const float* m,
+                 const float* tpre_sel, float* freeD, float* qP, int32_t* assign) {
+    std::vector<int> order(C);
+    for (int c = 0; c < C; ++c) order[c] = c;
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return prio[a] > prio[b]; });
+    for (int i = 0; i < C; ++i) {
+        const int c = order[i];
+        assign[c] = -1;
+        for (int k = 0; k < K; ++k) {
+            const int32_t j = pair[(size_t)c * K + k];
+            if (j < 0) continue;
+            const int d = j % D, p = j / D;
+            if (freeD[d] >= m[c]) {
+                freeD[d] = freeD[d] - m[c];
+                qP[p] = qP[p] + tpre_sel[(size_t)c * K + k];
+                assign[c] = j;
+                break;
+            }
+        }
+    }
+    return 0;
+}
+
+// Longest node-weighted path to a sink, per node, over a successor-CSR DAG:
+//   tail[v] = max over successors u of cp[u]   (0 without successors)
+//   cp[v]   = cost[v] + tail[v]
+//   H[w]    = max over nodes v of workflow w of cp[v]
+// Nodes are visited in reverse topological order (Kahn), so every sum runs from
+// the sink towards the source.  Returns -1 if the graph has a cycle.
+int orc_longest_path(const uint32_t* row_ptr, const uint32_t* col, const float* cost,
+                     const uint32_t* node_wf, uint32_t N, uint32_t W,
+                     float* cp, float* tail, float* H) {
+    std::vector<uint32_t> indeg(N, 0), topo;
+    topo.reserve(N);
+    for (uint32_t v = 0; v < N; ++v)
+        for (uint32_t e = row_ptr[v]; e < row_ptr[v + 1]; ++e) ++indeg[col[e]];
+    for (uint32_t v = 0; v < N; ++v) if (indeg[v] == 0) topo.push_back(v);
+    for (size_t i = 0; i < topo.size(); ++i) {
+        const uint32_t v = topo[i];
+        for (uint32_t e = row_ptr[v]; e < row_ptr[v + 1]; ++e)
+            if (--indeg[col[e]] == 0) topo.push_back(col[e]);
+    }
+    if (topo.size() != N) return -1;
+    for (uint32_t w = 0; w < W; ++w) H[w] = 0.0f;
+    for (size_t i = N; i-- > 0;) {
+        const uint32_t v = topo[i];
+        float t = 0.0f;
+        for (uint32_t e = row_ptr[v]; e < row_ptr[v + 1]; ++e) t = std::fmax(t, cp[col[e]]);
+        tail[v] = t;
+        cp[v] = cost[v] + t;
+        H[node_wf[v]] = std::fmax(H[node_wf[v]], cp[v]);
+    }
+    return 0;
+}
+
+// Double-precision twin of orc_fin_all in textbook form (units converted first,
+// plain divisions), to measure the rounding error of the binary32 sequence.
+int orc_fin_all_f64(const OrcCluster* cl, const OrcCall* calls, int C, int flags, double* fin) {
+    for (int c = 0; c < C; ++c) {
+        const double n = calls[c].prompt_tokens, o = calls[c].output_tokens;
+        const double phi = cl->flops_per_token[calls[c].model];
+        const double omega = cl->weight_bytes[calls[c].model];
+        const double kappa = cl->kv_bytes_per_token[calls[c].model];
+        for (int p = 0; p < cl->P; ++p)
+            for (int d = 0; d < cl->D; ++d) {
+                const int gp = cl->typeP[p], gd = cl->typeD[d];
+                const double F = cl->peak_tflops[gp] * 1e12, Bp = cl->hbm_tbps[gp] * 1e12;
+                const double Bd = cl->hbm_tbps[gd] * 1e12;
+                const double L = cl->link_gbps[(size_t)p * cl->D + d] * 1e9;
+                const double qp = (flags & ORC_FLAG_UNLOADED) ? 0.0 : cl->qP[p];
+                const double qd = (flags & ORC_FLAG_UNLOADED) ? 0.0 : cl->qD[d];
+                const double tpre = std::max(n * phi / F, (omega + n * kappa) / Bp);
+                const double tdec = o * (omega + kappa * (n + 0.5 * (o - 1.0))) / Bd;
+                const double ready = qp + tpre + n * kappa / L;
+                const double start = std::max(ready, qd);
+                fin[((size_t)c * cl->P + p) * cl->D + d] =
+                    (n + o <= cl->capD[d]) ? start + tdec : std::numeric_limits<double>::infinity();
+            }
+    }
+    return 0;
+}
+
+}  // extern "C"
