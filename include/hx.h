@@ -1,0 +1,203 @@
+/* hx.h - C ABI of the batched placement-scoring library for workflow-aware
+ * scheduling on heterogeneous prefill/decode (P-D) disaggregated clusters.
+ *
+ * The library evaluates, on one CUDA device, every ready LLM call against every
+ * (prefill instance, decode instance) pair of the cluster and picks, per call,
+ * the pair with the earliest projected decode finish (paper Section 5.3); it
+ * also computes the workflow horizons H_w(t) (Section 5.1) that turn a finish
+ * time into the projected ratio of Eq. 2.
+ *
+ * Conventions
+ *   - Every function returns HX_OK (0) or a negative HX_ERR_* code and never
+ *     throws or aborts; hx_last_error() gives a message for the last failure.
+ *   - "host" pointers are ordinary CPU memory, read or written during the call
+ *     and not retained.  "device" pointers are CUDA global memory of the device
+ *     that was current when the handle was created; buffers passed as device
+ *     pointers stay owned by the caller and must stay alive until the work
+ *     enqueued on `stream` has finished.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *     stream).  Unless stated otherwise a call only enqueues work and returns.
+ *   - All quantities are IEEE binary32.  Times are seconds, token counts are
+ *     integer-valued floats below 2^24, bandwidths and rates use decimal units.
+ *   - A handle is not thread-safe; use one handle per host thread or lock.
+ */
+#ifndef HX_H_
+#define HX_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define HX_OK                0
+#define HX_ERR_INVALID_ARG  (-1)   /* bad size, id out of range, non-finite or non-positive rate ... */
+#define HX_ERR_CUDA         (-2)   /* a CUDA runtime call failed; message holds cudaGetErrorString */
+#define HX_ERR_CYCLE        (-3)   /* the uploaded graph is not acyclic */
+#define HX_ERR_NOT_READY    (-4)   /* scoring needs horizons but hx_critical_path was not enqueued */
+#define HX_ERR_TIMEOUT      (-5)   /* a bounded device-side wait ran out (reported by hx_get_status) */
+#define HX_ERR_OOM          (-6)   /* host or device allocation failed */
+
+/* out_cost of hx_schedule_batch (Delta = earliest projected decode finish of the call) */
+#define HX_MODE_COMPLETION   0     /* (elapsed_w + Delta) + tail(node): projected workflow completion */
+#define HX_MODE_SLACK        1     /* alpha * H_w - completion: slack against the scaled SLO (Eq. 1) */
+#define HX_MODE_RATIO        2     /* completion / H_w; with HX_FLAG_NO_TAIL this is Eq. 2 as printed */
+
+#define HX_FLAG_NO_DAG       1     /* ignore the DAG: elapsed = 0, tail = 0, H = 1 */
+#define HX_FLAG_NO_TAIL      2     /* drop the remaining-critical-path term from the score */
+#define HX_FLAG_UNLOADED     4     /* score against an idle cluster (all queue loads zero) */
+
+#define HX_MAX_TYPES        32     /* GPU classes */
+#define HX_MAX_MODELS       32
+#define HX_MAX_PREFILL    4096     /* prefill instances */
+#define HX_MAX_DECODE      512     /* decode instances */
+#define HX_MAX_TOPK          8
+#define HX_MAX_COMMIT_CALLS 65536  /* largest batch the capacity-conflict pass accepts */
+
+typedef struct hx_cluster hx_cluster;   /* opaque; owns every packed device table */
+
+/* One GPU class ("instance type"): peak dense compute in TFLOP/s and memory
+ * bandwidth in TB/s of one model instance (tensor parallelism folded in).
+ * Inputs of the roofline-style latency estimate of Section 4.2. */
+typedef struct { float peak_tflops, hbm_tbps; } hx_gpu_type;
+
+/* One model instance of the P-D cluster (Section 4.2, "Heterogeneous resource
+ * modelling").  role 0 = prefill (single-server queue), 1 = decode (batched,
+ * KV-capacity bound).  load_s: seconds until a prefill instance has drained
+ * its queue, or earliest time a decode instance can admit a new call.
+ * kv_cap_tokens is Cap(d) of Eq. 4, kv_free_tokens the part of it not in use
+ * (both ignored for prefill instances). */
+typedef struct {
+    uint32_t type;
+    uint32_t role;
+    float load_s;
+    float kv_cap_tokens;
+    float kv_free_tokens;
+} hx_instance;
+
+/* Served model: forward FLOPs per token, bytes of weights read per pass, KV
+ * bytes per token. */
+typedef struct { float flops_per_token, weight_bytes, kv_bytes_per_token; } hx_model;
+
+/* One ready LLM call (Section 7.1: calls carry input length, output length and
+ * workflow identity).  node indexes the uploaded DAG (ignored with
+ * HX_FLAG_NO_DAG), output_tokens is the predicted output length of Eq. 3.
+ * 16 bytes, read with one 128-bit load. */
+typedef struct { uint32_t node, model; float prompt_tokens, output_tokens; } hx_call;
+
+typedef struct {
+    int score_mode;   /* HX_MODE_* */
+    int topk;         /* 0: plain argmin.  1..HX_MAX_TOPK: also build the top-K list and run the
+                         capacity-conflict pass over the batch */
+    int commit;       /* with topk > 0: write the loads consumed by the pass back into the cluster */
+    int flags;        /* HX_FLAG_* */
+    float alpha;      /* SLO scale of Eq. 1, used by HX_MODE_SLACK */
+} hx_options;
+
+/* Cluster-state packing (State Collector snapshot, Section 4.2 and 4.3).
+ * instances: all prefill instances first, then all decode instances.
+ * link_bw_gbps: host, n_instances x n_instances row-major, effective KV-transfer
+ * bandwidth in GB/s from instance i to instance j; only [prefill][decode]
+ * entries are read.  The tables are converted to reciprocal rates and packed
+ * as structure-of-arrays binary32 on the device; the link table is stored
+ * transposed, every row padded to a 16-byte boundary.
+ * Errors: HX_ERR_INVALID_ARG for sizes out of range, ids out of range,
+ * non-finite values, rates or bandwidths <= 0, negative loads, a prefill
+ * instance listed after a decode instance, or a pool that is empty;
+ * HX_ERR_OOM / HX_ERR_CUDA for allocation failures.  *out is set on success. */
+int hx_cluster_create(const hx_gpu_type* gpu_types, int n_types,
+                      const hx_instance* instances, int n_instances,
+                      const float* link_bw_gbps,
+                      const hx_model* models, int n_models,
+                      hx_cluster** out);
+
+/* Replace queue loads and free KV tokens (State Collector refresh between
+ * scheduler invocations).  Each pointer is host memory or NULL (= keep):
+ * qP[n_prefill], qD[n_decode], kv_free[n_decode].  The copies are enqueued on
+ * `stream`; the host arrays may be reused when the call returns. */
+int hx_cluster_update_loads(hx_cluster* h, const float* qP, const float* qD,
+                            const float* kv_free, void* stream);
+
+/* Read the current loads back (after commits).  Synchronises `stream`. */
+int hx_cluster_read_loads(hx_cluster* h, float* qP, float* qD, float* kv_free, void* stream);
+
+int hx_cluster_destroy(hx_cluster* h);
+
+/* Upload the revealed workflow forest (Section 4.1) in successor-CSR form:
+ * row_ptr[n_nodes+1], col_idx[n_edges], one cost per node in seconds, the
+ * workflow of every node, and the elapsed time (t - a_w) of every workflow.
+ * All arrays are host memory.  The graph is validated (monotone row_ptr,
+ * columns in range, edges inside one workflow, finite non-negative costs,
+ * acyclic) and levelised on the host; nodes are regrouped workflow by workflow
+ * and by height for the device pass.  Synchronous.  Errors: HX_ERR_INVALID_ARG,
+ * HX_ERR_CYCLE, HX_ERR_OOM, HX_ERR_CUDA.  Replaces any earlier upload. */
+int hx_dag_upload(hx_cluster* h, const uint32_t* row_ptr, const uint32_t* col_idx,
+                  const float* node_costs, const uint32_t* node_workflow,
+                  const float* workflow_elapsed_s,
+                  uint32_t n_nodes, uint32_t n_edges, uint32_t n_workflows);
+
+/* Workflow horizons (Section 5.1, "Define online workflow horizon"; Algorithm 1,
+ * horizon update): for every node cp = cost + tail, tail = max over successors
+ * of cp (0 for sinks); H[w] = max over the workflow's nodes of cp.  Each sum
+ * runs from the sink towards the source, so results do not depend on the
+ * traversal order.  Enqueues on `stream`. */
+int hx_critical_path(hx_cluster* h, void* stream);
+
+/* Borrowed device pointers to cp[n_nodes], tail[n_nodes] (original node
+ * numbering) and H[n_workflows]; valid until the next upload or destroy.
+ * Any of the three output arguments may be NULL. */
+int hx_get_dag_results(hx_cluster* h, const float** cp, const float** tail, const float** H);
+
+/* Validates and stores the options used by later hx_schedule_batch calls. */
+int hx_set_options(hx_cluster* h, const hx_options* opts);
+
+/* Batched placement scoring (Algorithm 1, inner loop over the waiting calls;
+ * Section 5.3 "Projected-risk prefill ranking" and "Joint prefill-decode
+ * planning"; feasibility by Eq. 3-4).  calls: device, n_calls records, 16-byte
+ * aligned.  out_assign: device int32[n_calls], pair index p * n_decode + d of
+ * the pair with the earliest projected decode finish (lowest index among
+ * equals), or -1 if no decode instance can hold the call.  out_cost: device
+ * float[n_calls], the score selected by hx_options.score_mode.  With topk > 0
+ * the call also fills the top-K list (see hx_get_topk) and runs the
+ * capacity-conflict pass (one-pass ordering by the same risk score for large
+ * queues, Section 5.3 last sentence, with Eq. 4 as the capacity constraint):
+ * out_assign then holds the pair each call obtained, or -1 if none of its K
+ * candidates had room.  The first call with topk > 0, or with a larger batch
+ * than before, allocates the buffers of that pass (and synchronises the
+ * device while doing so).  Needs hx_critical_path to have been enqueued since
+ * the last upload unless HX_FLAG_NO_DAG is set (else HX_ERR_NOT_READY).
+ * A call record whose model or node id is out of range gets assignment -1,
+ * cost +inf, and raises HX_ERR_INVALID_ARG in the status word.
+ * n_calls = 0 is a no-op.  Enqueues on `stream`; does not synchronise. */
+int hx_schedule_batch(hx_cluster* h, const hx_call* calls, int n_calls,
+                      int32_t* out_assign, float* out_cost, void* stream);
+
+/* Same operation with host buffers: copies the calls to the device, runs the
+ * kernels, copies both results back and synchronises `stream`. */
+int hx_schedule_batch_host(hx_cluster* h, const hx_call* calls, int n_calls,
+                           int32_t* out_assign, float* out_cost, void* stream);
+
+/* Borrowed device pointers to the top-K results of the last batch scored with
+ * topk = K > 0: pairs int32[n_calls][K] (-1 = unused slot), costs
+ * float[n_calls][K] (projected decode finish of that pair, +inf if unused),
+ * prio float[n_calls] (Eq. 2 of the best pair; the pass visits calls by
+ * decreasing prio).  The K entries are the K cheapest distinct decode
+ * instances, each with its best prefill partner, ordered by (cost, d).
+ * Any output argument may be NULL. */
+int hx_get_topk(hx_cluster* h, const int32_t** pairs, const float** costs, const float** prio);
+
+/* Device-side status word (0 = fine, else an HX_ERR_* raised inside a kernel,
+ * e.g. HX_ERR_TIMEOUT from a bounded wait).  Synchronises `stream`. */
+int hx_get_status(hx_cluster* h, int* status, void* stream);
+
+/* Message of the last error on this handle ("" if none); with h = NULL, the
+ * message of the last failed hx_cluster_create of the calling thread. */
+const char* hx_last_error(const hx_cluster* h);
+
+/* Number of kernels this library has launched on the handle so far. */
+long long hx_launch_count(const hx_cluster* h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HX_H_ */

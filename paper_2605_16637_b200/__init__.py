@@ -1,0 +1,16 @@
+"""Python binding of libhx.so: batched placement scoring and workflow horizons
+for workflow-aware scheduling on heterogeneous prefill/decode clusters.
+
+The binding only marshals arguments; every step runs in the CUDA library.  It
+raises at import if the library has not been built (python -m
+paper_2605_16637_b200.build); there is no CPU fallback.
+"""
+from .api import (CALL_DTYPE, INSTANCE_DTYPE, HX_FLAG_NO_DAG, HX_FLAG_NO_TAIL, HX_FLAG_UNLOADED,
+                  HX_MODE_COMPLETION, HX_MODE_RATIO, HX_MODE_SLACK, HxError, Cluster,
+                  hx_cluster_create, hx_cluster_destroy, hx_cluster_read_loads,
+                  hx_cluster_update_loads, hx_critical_path, hx_dag_upload, hx_get_dag_results,
+                  hx_get_status, hx_get_topk, hx_last_error, hx_launch_count, hx_schedule_batch,
+                  hx_schedule_batch_host, hx_set_options, lib_path)
+
+__all__ = [n for n in dir() if n.startswith(("hx_", "HX_", "Hx")) or n in
+           ("CALL_DTYPE", "INSTANCE_DTYPE", "Cluster", "lib_path")]

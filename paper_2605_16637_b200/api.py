@@ -1,0 +1,294 @@
+"""ctypes binding of the C ABI declared in include/hx.h.
+
+Module-level functions carry the names of the C entry points and take plain
+pointers / numpy arrays; `Cluster` is a small convenience wrapper that keeps the
+handle and passes torch tensors' data pointers and the current CUDA stream.
+PyTorch is used for device memory and streams only.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+from .build import LIB_PATH
+
+HX_OK = 0
+HX_MODE_COMPLETION, HX_MODE_SLACK, HX_MODE_RATIO = 0, 1, 2
+HX_FLAG_NO_DAG, HX_FLAG_NO_TAIL, HX_FLAG_UNLOADED = 1, 2, 4
+
+CALL_DTYPE = np.dtype([("node", "<u4"), ("model", "<u4"),
+                       ("prompt_tokens", "<f4"), ("output_tokens", "<f4")])
+INSTANCE_DTYPE = np.dtype([("type", "<u4"), ("role", "<u4"), ("load_s", "<f4"),
+                           ("kv_cap_tokens", "<f4"), ("kv_free_tokens", "<f4")])
+
+
+class HxError(RuntimeError):
+    def __init__(self, code, msg):
+        super().__init__("hx error %d: %s" % (code, msg))
+        self.code = code
+
+
+class _Options(C.Structure):
+    _fields_ = [("score_mode", C.c_int), ("topk", C.c_int), ("commit", C.c_int),
+                ("flags", C.c_int), ("alpha", C.c_float)]
+
+
+def lib_path() -> str:
+    return LIB_PATH
+
+
+def _load():
+    if not os.path.exists(LIB_PATH):
+        raise ImportError("libhx.so is not built (run: python paper_2605_16637_b200/build.py); "
+                          "this package has no fallback path")
+    lib = C.CDLL(LIB_PATH)
+    vp, ci, u32 = C.c_void_p, C.c_int, C.c_uint32
+    sig = {
+        "hx_cluster_create": [vp, ci, vp, ci, vp, vp, ci, C.POINTER(vp)],
+        "hx_cluster_update_loads": [vp, vp, vp, vp, vp],
+        "hx_cluster_read_loads": [vp, vp, vp, vp, vp],
+        "hx_cluster_destroy": [vp],
+        "hx_dag_upload": [vp, vp, vp, vp, vp, vp, u32, u32, u32],
+        "hx_critical_path": [vp, vp],
+        "hx_get_dag_results": [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp)],
+        "hx_set_options": [vp, C.POINTER(_Options)],
+        "hx_schedule_batch": [vp, vp, ci, vp, vp, vp],
+        "hx_schedule_batch_host": [vp, vp, ci, vp, vp, vp],
+        "hx_get_topk": [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp)],
+        "hx_get_status": [vp, C.POINTER(ci), vp],
+    }
+    for name, args in sig.items():
+        f = getattr(lib, name)
+        f.argtypes = args
+        f.restype = ci
+    lib.hx_last_error.argtypes = [vp]
+    lib.hx_last_error.restype = C.c_char_p
+    lib.hx_launch_count.argtypes = [vp]
+    lib.hx_launch_count.restype = C.c_longlong
+    return lib
+
+
+_lib = _load()
+
+
+def _check(rc, h=None):
+    if rc != HX_OK:
+        raise HxError(rc, _lib.hx_last_error(h).decode())
+
+
+def _np(a, dtype):
+    return np.ascontiguousarray(a, dtype=dtype)
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+# --- functions named after the C entry points ----------------------------------------------
+
+def hx_cluster_create(gpu_types, instances, link_bw_gbps, models):
+    gpu_types = _np(gpu_types, np.float32).reshape(-1, 2)
+    instances = _np(instances, INSTANCE_DTYPE)
+    n = instances.shape[0]
+    link = _np(link_bw_gbps, np.float32).reshape(n, n)
+    models = _np(models, np.float32).reshape(-1, 3)
+    h = C.c_void_p()
+    _check(_lib.hx_cluster_create(_p(gpu_types), gpu_types.shape[0], _p(instances), n, _p(link),
+                                  _p(models), models.shape[0], C.byref(h)))
+    return h
+
+
+def hx_cluster_update_loads(h, qP=None, qD=None, kv_free=None, stream=0):
+    arrs = [None if a is None else _np(a, np.float32) for a in (qP, qD, kv_free)]
+    _check(_lib.hx_cluster_update_loads(h, _p(arrs[0]), _p(arrs[1]), _p(arrs[2]), stream), h)
+
+
+def hx_cluster_read_loads(h, n_prefill, n_decode, stream=0):
+    qP = np.zeros(n_prefill, np.float32); qD = np.zeros(n_decode, np.float32)
+    free = np.zeros(n_decode, np.float32)
+    _check(_lib.hx_cluster_read_loads(h, _p(qP), _p(qD), _p(free), stream), h)
+    return qP, qD, free
+
+
+def hx_cluster_destroy(h):
+    _check(_lib.hx_cluster_destroy(h))
+
+
+def hx_dag_upload(h, row_ptr, col_idx, node_costs, node_workflow, workflow_elapsed_s):
+    row_ptr = _np(row_ptr, np.uint32); col_idx = _np(col_idx, np.uint32)
+    node_costs = _np(node_costs, np.float32); node_workflow = _np(node_workflow, np.uint32)
+    el = _np(workflow_elapsed_s, np.float32)
+    if row_ptr.shape[0] != node_workflow.shape[0] + 1 or node_costs.shape[0] != node_workflow.shape[0]:
+        raise HxError(-1, "row_ptr, node_costs and node_workflow disagree on the node count")
+    _check(_lib.hx_dag_upload(h, _p(row_ptr), _p(col_idx), _p(node_costs), _p(node_workflow), _p(el),
+                              node_workflow.shape[0], col_idx.shape[0], el.shape[0]), h)
+
+
+def hx_critical_path(h, stream=0):
+    _check(_lib.hx_critical_path(h, stream), h)
+
+
+def hx_get_dag_results(h):
+    """Device addresses (int) of cp, tail, H."""
+    cp, tail, H = C.c_void_p(), C.c_void_p(), C.c_void_p()
+    _check(_lib.hx_get_dag_results(h, C.byref(cp), C.byref(tail), C.byref(H)), h)
+    return cp.value, tail.value, H.value
+
+
+def hx_set_options(h, score_mode=HX_MODE_COMPLETION, topk=0, commit=0, flags=0, alpha=1.5):
+    o = _Options(int(score_mode), int(topk), int(commit), int(flags), float(alpha))
+    _check(_lib.hx_set_options(h, C.byref(o)), h)
+
+
+def hx_schedule_batch(h, calls_ptr, n_calls, out_assign_ptr, out_cost_ptr, stream=0):
+    _check(_lib.hx_schedule_batch(h, calls_ptr, int(n_calls), out_assign_ptr, out_cost_ptr, stream), h)
+
+
+def hx_schedule_batch_host(h, calls, out_assign=None, out_cost=None, stream=0):
+    """calls: host array of CALL_DTYPE (numpy; may be a view of pinned memory)."""
+    calls = _np(calls, CALL_DTYPE)
+    n = calls.shape[0]
+    if out_assign is None:
+        out_assign = np.empty(n, np.int32)
+    if out_cost is None:
+        out_cost = np.empty(n, np.float32)
+    _check(_lib.hx_schedule_batch_host(h, _p(calls), n, _p(out_assign), _p(out_cost), stream), h)
+    return out_assign, out_cost
+
+
+def hx_get_topk(h):
+    """Device addresses (int) of pairs, costs, prio."""
+    a, b, c = C.c_void_p(), C.c_void_p(), C.c_void_p()
+    _check(_lib.hx_get_topk(h, C.byref(a), C.byref(b), C.byref(c)), h)
+    return a.value, b.value, c.value
+
+
+def hx_get_status(h, stream=0):
+    s = C.c_int(0)
+    _check(_lib.hx_get_status(h, C.byref(s), stream), h)
+    return s.value
+
+
+def hx_last_error(h=None):
+    return _lib.hx_last_error(h).decode()
+
+
+def hx_launch_count(h):
+    return int(_lib.hx_launch_count(h))
+
+
+# --- convenience wrapper ----------------------------------------------------------------------
+
+class _Borrowed:
+    """A borrowed device buffer exposed through the CUDA array interface."""
+
+    def __init__(self, ptr, count, typestr):
+        self.__cuda_array_interface__ = {"shape": (count,), "typestr": typestr, "data": (int(ptr), True),
+                                         "version": 2}
+
+
+def _dev_to_numpy(ptr, count, typestr):
+    """Copy `count` items from a borrowed device address into a new numpy array."""
+    import torch
+    if count == 0:
+        return np.zeros(0, dtype=typestr)
+    torch.cuda.current_stream().synchronize()
+    return torch.as_tensor(_Borrowed(ptr, count, typestr), device="cuda").cpu().numpy()
+
+
+class Cluster:
+    """Owns one hx_cluster handle; methods mirror the C entry points."""
+
+    def __init__(self, gpu_types, instances, link_bw_gbps, models):
+        self.h = None
+        self.h = hx_cluster_create(gpu_types, instances, link_bw_gbps, models)
+        inst = _np(instances, INSTANCE_DTYPE)
+        self.P = int((inst["role"] == 0).sum())
+        self.D = int(inst.shape[0] - self.P)
+        self.n_nodes = 0
+        self.n_workflows = 0
+        self.topk = 0
+
+    @classmethod
+    def from_workload(cls, wl):
+        """Build from an object with the attributes of hx_synth.Workload."""
+        I = wl.P + wl.D
+        inst = np.zeros(I, INSTANCE_DTYPE)
+        inst["type"] = wl.inst_type
+        inst["role"][wl.P:] = 1
+        inst["load_s"] = wl.load_s
+        inst["kv_cap_tokens"] = wl.kv_cap
+        inst["kv_free_tokens"] = wl.kv_free
+        return cls(wl.gpu_types, inst, wl.link_gbps, wl.models)
+
+    @staticmethod
+    def _stream():
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+
+    def update_loads(self, qP=None, qD=None, kv_free=None):
+        hx_cluster_update_loads(self.h, qP, qD, kv_free, self._stream())
+
+    def read_loads(self):
+        return hx_cluster_read_loads(self.h, self.P, self.D, self._stream())
+
+    def dag_upload(self, row_ptr, col_idx, node_costs, node_workflow, workflow_elapsed_s):
+        hx_dag_upload(self.h, row_ptr, col_idx, node_costs, node_workflow, workflow_elapsed_s)
+        self.n_nodes = int(np.asarray(node_workflow).shape[0])
+        self.n_workflows = int(np.asarray(workflow_elapsed_s).shape[0])
+
+    def critical_path(self):
+        hx_critical_path(self.h, self._stream())
+
+    def dag_results(self):
+        """cp, tail, H as numpy arrays (synchronises)."""
+        cp, tail, H = hx_get_dag_results(self.h)
+        return (_dev_to_numpy(cp, self.n_nodes, "<f4"), _dev_to_numpy(tail, self.n_nodes, "<f4"),
+                _dev_to_numpy(H, self.n_workflows, "<f4"))
+
+    def set_options(self, score_mode=HX_MODE_COMPLETION, topk=0, commit=0, flags=0, alpha=1.5):
+        hx_set_options(self.h, score_mode, topk, commit, flags, alpha)
+        self.topk = int(topk)
+
+    def schedule_batch(self, calls, out_assign=None, out_cost=None):
+        """calls: CUDA tensor holding n records of 16 bytes, or a numpy CALL_DTYPE array
+        (copied to the device first).  Returns (assign, cost) CUDA tensors."""
+        import torch
+        if isinstance(calls, np.ndarray):
+            calls = torch.from_numpy(_np(calls, CALL_DTYPE).view(np.uint8).copy()).cuda()
+        n = calls.numel() * calls.element_size() // 16
+        if out_assign is None:
+            out_assign = torch.empty(n, dtype=torch.int32, device="cuda")
+        if out_cost is None:
+            out_cost = torch.empty(n, dtype=torch.float32, device="cuda")
+        hx_schedule_batch(self.h, calls.data_ptr(), n, out_assign.data_ptr(), out_cost.data_ptr(), self._stream())
+        return out_assign, out_cost
+
+    def schedule_batch_host(self, calls, out_assign=None, out_cost=None):
+        return hx_schedule_batch_host(self.h, calls, out_assign, out_cost, self._stream())
+
+    def topk_results(self, n_calls):
+        a, b, c = hx_get_topk(self.h)
+        K = self.topk
+        return (_dev_to_numpy(a, n_calls * K, "<i4").reshape(n_calls, K),
+                _dev_to_numpy(b, n_calls * K, "<f4").reshape(n_calls, K),
+                _dev_to_numpy(c, n_calls, "<f4"))
+
+    def status(self):
+        return hx_get_status(self.h, self._stream())
+
+    def launch_count(self):
+        return hx_launch_count(self.h)
+
+    def close(self):
+        if self.h is not None:
+            hx_cluster_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,154 @@
+// Workflow horizons: longest node-weighted path to a sink for every node of the
+// revealed forest (paper Section 5.1, "Define online workflow horizon";
+// Algorithm 1, horizon update).
+//
+//   tail[v] = max over successors u of cp[u]      (0 for a sink)
+//   cp[v]   = cost[v] + tail[v]
+//   H[w]    = max over the nodes of workflow w of cp[v]
+//
+// Workflows are independent components, so no grid-wide level barrier is
+// needed: one group of threads (a warp, or a whole block for big workflows)
+// walks all levels of one workflow.  The host has regrouped the nodes workflow
+// by workflow and by height above the sinks, so the frontier segment of a level
+// is a contiguous index range: the group stages the workflow's slice of the CSR
+// arrays in shared memory with coalesced loads, sweeps the levels there with a
+// group barrier between levels, and writes cp/tail back once.  max is exact and
+// every node does exactly one addition, so the result is independent of the
+// order in which a level is processed.
+#include "hx_internal.h"
+
+namespace {
+
+template <bool WARP>
+__device__ __forceinline__ void group_sync() {
+    if (WARP) __syncwarp(); else __syncthreads();
+}
+
+template <bool WARP>
+__device__ __forceinline__ float group_max(float v, float* red, int t, int tpw) {
+    for (int off = 16; off > 0; off >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, off));
+    if (WARP) return v;
+    __syncthreads();
+    if ((t & 31) == 0) red[t >> 5] = v;
+    __syncthreads();
+    float r = red[0];
+    for (int i = 1; i < (tpw >> 5); ++i) r = fmaxf(r, red[i]);
+    return r;
+}
+
+// One group per workflow, workflow slice staged in shared memory.
+template <bool WARP>
+__global__ void hx_cpath_staged_kernel(HxForestDev f, const uint32_t* __restrict__ wf_ids, uint32_t count,
+                                       int tpw, int wfs_per_block, uint32_t smem_per_wf) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ float red[32];
+    const int g = threadIdx.x / tpw, t = threadIdx.x % tpw;
+    const uint32_t slot = blockIdx.x * wfs_per_block + g;
+    if (slot >= count) return;                // a whole group (warp, or the only group of a block) leaves
+    const uint32_t w = wf_ids[slot];
+    const uint32_t ns = f.wf_node_start[w], n = f.wf_node_start[w + 1] - ns;
+    const uint32_t es = f.wf_edge_start[w], ne = f.wf_edge_start[w + 1] - es;
+    const uint32_t ss = f.wf_seg_start[w], nlev = f.wf_seg_start[w + 1] - ss - 1;
+
+    unsigned char* base = smem_raw + (size_t)g * smem_per_wf;
+    float* cpS = reinterpret_cast<float*>(base);
+    float* costS = cpS + n;                                   // becomes tail once a node is done
+    uint32_t* rowS = reinterpret_cast<uint32_t*>(costS + n);  // n + 1 entries, relative to es
+    uint32_t* segS = rowS + n + 1;                            // nlev + 1 entries
+    uint16_t* colS = reinterpret_cast<uint16_t*>(segS + nlev + 1);
+
+    for (uint32_t i = t; i < n; i += tpw) costS[i] = f.icost[ns + i];
+    for (uint32_t i = t; i <= n; i += tpw) rowS[i] = f.irow[ns + i] - es;
+    for (uint32_t i = t; i <= nlev; i += tpw) segS[i] = f.seg_off[ss + i];
+    for (uint32_t e = t; e < ne; e += tpw) colS[e] = f.icol16[es + e];
+    group_sync<WARP>();
+
+    float hmax = 0.0f;
+    for (uint32_t lev = 0; lev < nlev; ++lev) {
+        const uint32_t hi = segS[lev + 1];
+        for (uint32_t i = segS[lev] + t; i < hi; i += tpw) {
+            float tl = 0.0f;
+            const uint32_t e1 = rowS[i + 1];
+            for (uint32_t e = rowS[i]; e < e1; ++e) tl = fmaxf(tl, cpS[colS[e]]);
+            const float c = __fadd_rn(costS[i], tl);
+            cpS[i] = c;
+            costS[i] = tl;
+            hmax = fmaxf(hmax, c);
+        }
+        group_sync<WARP>();
+    }
+    for (uint32_t i = t; i < n; i += tpw) {
+        const uint32_t v = f.perm[ns + i];
+        f.cp[v] = cpS[i];
+        f.tail[v] = costS[i];
+    }
+    hmax = group_max<WARP>(hmax, red, t, tpw);
+    if (t == 0) f.H[w] = hmax;
+}
+
+// One block per workflow, everything in global memory: for workflows too large
+// to stage.  cp is written and re-read by the same block; the block barrier
+// between levels orders those accesses, and the reads bypass L1.
+__global__ void hx_cpath_global_kernel(HxForestDev f, const uint32_t* __restrict__ wf_ids, uint32_t count) {
+    __shared__ float red[32];
+    const uint32_t w = wf_ids[blockIdx.x];
+    const int t = threadIdx.x, tpw = blockDim.x;
+    const uint32_t ns = f.wf_node_start[w];
+    const uint32_t ss = f.wf_seg_start[w], nlev = f.wf_seg_start[w + 1] - ss - 1;
+    float hmax = 0.0f;
+    for (uint32_t lev = 0; lev < nlev; ++lev) {
+        const uint32_t lo = f.seg_off[ss + lev], hi = f.seg_off[ss + lev + 1];
+        for (uint32_t i = lo + t; i < hi; i += tpw) {
+            float tl = 0.0f;
+            const uint32_t e1 = f.irow[ns + i + 1];
+            for (uint32_t e = f.irow[ns + i]; e < e1; ++e)
+                tl = fmaxf(tl, __ldcg(&f.cp[f.perm[ns + f.icol32[e]]]));
+            const float c = __fadd_rn(f.icost[ns + i], tl);
+            const uint32_t v = f.perm[ns + i];
+            __stcg(&f.cp[v], c);
+            f.tail[v] = tl;
+            hmax = fmaxf(hmax, c);
+        }
+        __syncthreads();
+    }
+    hmax = group_max<false>(hmax, red, t, tpw);
+    if (t == 0) f.H[w] = hmax;
+}
+
+}  // namespace
+
+cudaError_t hx_launch_cpath(const HxForestDev& f, const HxCpClass* classes, int n_classes,
+                            cudaStream_t stream, long long* launches) {
+    for (int k = 0; k < n_classes; ++k) {
+        const HxCpClass& c = classes[k];
+        if (c.count == 0) continue;
+        if (c.smem_per_wf == 0) {
+            hx_cpath_global_kernel<<<c.count, 256, 0, stream>>>(f, c.wf_ids, c.count);
+        } else {
+            const int threads = c.threads_per_wf * c.wfs_per_block;
+            const size_t smem = c.smem_per_wf * c.wfs_per_block;
+            const unsigned grid = (c.count + c.wfs_per_block - 1) / c.wfs_per_block;
+            if (c.threads_per_wf == 32) {
+                {   // static + dynamic shared memory may exceed the 48 KB default
+                    cudaError_t e = cudaFuncSetAttribute(hx_cpath_staged_kernel<true>,
+                                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+                    if (e != cudaSuccess) return e;
+                }
+                hx_cpath_staged_kernel<true><<<grid, threads, smem, stream>>>(
+                    f, c.wf_ids, c.count, 32, c.wfs_per_block, (uint32_t)c.smem_per_wf);
+            } else {
+                {   // static + dynamic shared memory may exceed the 48 KB default
+                    cudaError_t e = cudaFuncSetAttribute(hx_cpath_staged_kernel<false>,
+                                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+                    if (e != cudaSuccess) return e;
+                }
+                hx_cpath_staged_kernel<false><<<grid, threads, smem, stream>>>(
+                    f, c.wf_ids, c.count, c.threads_per_wf, 1, (uint32_t)c.smem_per_wf);
+            }
+        }
+        ++*launches;
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}

@@ -1,0 +1,492 @@
+// Host side of libhx.so: handle, validation, cluster-state packing, forest
+// levelisation and the C ABI declared in hx.h.  No arithmetic of the method
+// runs here except the one-time conversion of rates to reciprocal rates.
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "hx_internal.h"
+
+struct hx_cluster {
+    int device = 0, n_sm = 0;
+    size_t max_smem = 0;
+    int G = 0, P = 0, D = 0, M = 0, Ppad = 0;
+    std::vector<void*> allocs;          // cluster tables, freed at destroy
+    std::vector<void*> dag_allocs;      // forest, freed at the next upload
+    std::vector<void*> tk_allocs;       // top-K / conflict-pass buffers
+    HxTables tab{};
+    int* status = nullptr;
+    // forest
+    bool dag_uploaded = false, cp_ready = false;
+    HxForestDev forest{};
+    uint32_t* d_node_wf = nullptr;
+    float* d_elapsed = nullptr;
+    std::vector<HxCpClass> classes;
+    // top-K
+    HxTopkBufs tk{};
+    size_t counter_bytes = 0;
+    // staging for the host-buffer entry point
+    hx_call* st_calls = nullptr; int32_t* st_assign = nullptr; float* st_cost = nullptr; int st_cap = 0;
+    hx_options opts{HX_MODE_COMPLETION, 0, 0, 0, 1.5f};
+    std::string err;
+    long long launches = 0;
+};
+
+namespace {
+
+thread_local std::string g_create_err;
+
+int fail(hx_cluster* h, int code, const std::string& msg) {
+    if (h) h->err = msg; else g_create_err = msg;
+    return code;
+}
+int fail_cuda(hx_cluster* h, cudaError_t e, const char* what) {
+    return fail(h, e == cudaErrorMemoryAllocation ? HX_ERR_OOM : HX_ERR_CUDA,
+                std::string(what) + ": " + cudaGetErrorString(e));
+}
+
+struct DeviceGuard {
+    int prev = -1; bool changed = false;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) { cudaSetDevice(dev); changed = true; }
+    }
+    ~DeviceGuard() { if (changed) cudaSetDevice(prev); }
+};
+
+template <class T>
+cudaError_t dev_alloc(std::vector<void*>& pool, T** out, size_t count) {
+    void* p = nullptr;
+    cudaError_t e = cudaMalloc(&p, std::max<size_t>(count, 1) * sizeof(T));
+    if (e != cudaSuccess) { *out = nullptr; return e; }
+    pool.push_back(p);
+    *out = static_cast<T*>(p);
+    return cudaSuccess;
+}
+template <class T>
+cudaError_t dev_upload(std::vector<void*>& pool, T** out, const std::vector<T>& src) {
+    cudaError_t e = dev_alloc(pool, out, src.size());
+    if (e != cudaSuccess) return e;
+    if (src.empty()) return cudaSuccess;
+    return cudaMemcpy(*out, src.data(), src.size() * sizeof(T), cudaMemcpyHostToDevice);
+}
+void free_pool(std::vector<void*>& pool) {
+    for (void* p : pool) cudaFree(p);
+    pool.clear();
+}
+
+bool good_rate(float x) { return std::isfinite(x) && x > 0.0f; }
+bool good_load(float x) { return std::isfinite(x) && x >= 0.0f; }
+
+#define HX_TRY(call, what) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return fail_cuda(h, e_, what); } while (0)
+
+int ensure_topk(hx_cluster* h, int n_calls, int K) {
+    if (h->tk.cap_calls >= n_calls && h->tk.K == K) return HX_OK;
+    cudaDeviceSynchronize();
+    free_pool(h->tk_allocs);
+    h->tk = HxTopkBufs{};
+    HxTopkBufs b{};
+    b.K = K;
+    const size_t cap = (size_t)std::max(n_calls, 16384);
+    HX_TRY(dev_alloc(h->tk_allocs, &b.pair, cap * K), "alloc top-K");
+    HX_TRY(dev_alloc(h->tk_allocs, &b.cost, cap * K), "alloc top-K");
+    HX_TRY(dev_alloc(h->tk_allocs, &b.tpre, cap * K), "alloc top-K");
+    HX_TRY(dev_alloc(h->tk_allocs, &b.prio, cap), "alloc top-K");
+    HX_TRY(dev_alloc(h->tk_allocs, &b.mtok, cap), "alloc top-K");
+    const size_t ncnt = 2 * (size_t)h->D + 2 * (size_t)h->P + 1;
+    unsigned int* cnt;
+    HX_TRY(dev_alloc(h->tk_allocs, &cnt, ncnt), "alloc counters");
+    b.dcount = cnt; b.dcursor = cnt + h->D; b.pcount = cnt + 2 * h->D; b.pcursor = b.pcount + h->P;
+    b.n_acc = b.pcursor + h->P;
+    h->counter_bytes = ncnt * sizeof(unsigned int);
+    HX_TRY(dev_alloc(h->tk_allocs, &b.dflat, cap * K), "alloc slots");
+    HX_TRY(dev_alloc(h->tk_allocs, &b.dsorted, cap * K), "alloc slots");
+    HX_TRY(dev_alloc(h->tk_allocs, &b.accflat, cap), "alloc slots");
+    HX_TRY(dev_alloc(h->tk_allocs, &b.pseg, cap), "alloc slots");
+    HX_TRY(dev_alloc(h->tk_allocs, &b.psorted, cap), "alloc slots");
+    b.cap_calls = (int)cap;
+    h->tk = b;
+    return HX_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int hx_cluster_create(const hx_gpu_type* gpu_types, int n_types, const hx_instance* instances,
+                      int n_instances, const float* link_bw_gbps, const hx_model* models,
+                      int n_models, hx_cluster** out) {
+    if (!out) return fail(nullptr, HX_ERR_INVALID_ARG, "out is NULL");
+    *out = nullptr;
+    if (!gpu_types || !instances || !link_bw_gbps || !models)
+        return fail(nullptr, HX_ERR_INVALID_ARG, "NULL table");
+    if (n_types < 1 || n_types > HX_MAX_TYPES) return fail(nullptr, HX_ERR_INVALID_ARG, "n_types out of range");
+    if (n_models < 1 || n_models > HX_MAX_MODELS) return fail(nullptr, HX_ERR_INVALID_ARG, "n_models out of range");
+    if (n_instances < 2) return fail(nullptr, HX_ERR_INVALID_ARG, "need at least one prefill and one decode instance");
+    int P = 0;
+    while (P < n_instances && instances[P].role == 0) ++P;
+    const int D = n_instances - P;
+    for (int i = P; i < n_instances; ++i)
+        if (instances[i].role != 1)
+            return fail(nullptr, HX_ERR_INVALID_ARG, "instances must list all prefill (role 0) then all decode (role 1)");
+    if (P < 1 || D < 1) return fail(nullptr, HX_ERR_INVALID_ARG, "empty prefill or decode pool");
+    if (P > HX_MAX_PREFILL || D > HX_MAX_DECODE) return fail(nullptr, HX_ERR_INVALID_ARG, "pool larger than supported");
+    for (int g = 0; g < n_types; ++g)
+        if (!good_rate(gpu_types[g].peak_tflops) || !good_rate(gpu_types[g].hbm_tbps))
+            return fail(nullptr, HX_ERR_INVALID_ARG, "GPU type rates must be finite and > 0");
+    for (int m = 0; m < n_models; ++m)
+        if (!good_load(models[m].flops_per_token) || !good_load(models[m].weight_bytes) ||
+            !good_load(models[m].kv_bytes_per_token))
+            return fail(nullptr, HX_ERR_INVALID_ARG, "model constants must be finite and >= 0");
+    for (int i = 0; i < n_instances; ++i) {
+        if (instances[i].type >= (uint32_t)n_types) return fail(nullptr, HX_ERR_INVALID_ARG, "instance type out of range");
+        if (!good_load(instances[i].load_s)) return fail(nullptr, HX_ERR_INVALID_ARG, "instance load must be finite and >= 0");
+        if (i >= P && (!good_load(instances[i].kv_cap_tokens) || !good_load(instances[i].kv_free_tokens)))
+            return fail(nullptr, HX_ERR_INVALID_ARG, "KV capacities must be finite and >= 0");
+    }
+    for (int p = 0; p < P; ++p)
+        for (int d = 0; d < D; ++d)
+            if (!good_rate(link_bw_gbps[(size_t)p * n_instances + P + d]))
+                return fail(nullptr, HX_ERR_INVALID_ARG, "link bandwidth must be finite and > 0");
+
+    hx_cluster* h = new (std::nothrow) hx_cluster();
+    if (!h) return fail(nullptr, HX_ERR_OOM, "out of host memory");
+    auto bail = [&](int code) { g_create_err = h->err; free_pool(h->allocs); delete h; return code; };
+    cudaError_t e = cudaGetDevice(&h->device);
+    if (e != cudaSuccess) return bail(fail_cuda(h, e, "cudaGetDevice"));
+    int v = 0;
+    if ((e = cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, h->device)) != cudaSuccess)
+        return bail(fail_cuda(h, e, "cudaDeviceGetAttribute"));
+    h->n_sm = v;
+    if ((e = cudaDeviceGetAttribute(&v, cudaDevAttrMaxSharedMemoryPerBlockOptin, h->device)) != cudaSuccess)
+        return bail(fail_cuda(h, e, "cudaDeviceGetAttribute"));
+    h->max_smem = (size_t)v;
+
+    h->G = n_types; h->P = P; h->D = D; h->M = n_models; h->Ppad = (P + 3) / 4 * 4;
+    std::vector<float> invF(n_types), invB(n_types), qP(h->Ppad, 0.f), qD(D), capD(D), freeD(D);
+    std::vector<float> phi(n_models), omega(n_models), kappa(n_models), invLT((size_t)D * h->Ppad, 0.f);
+    std::vector<int> typeP(h->Ppad, 0), typeD(D);
+    for (int g = 0; g < n_types; ++g) {
+        invF[g] = 1.0f / (gpu_types[g].peak_tflops * 1e12f);
+        invB[g] = 1.0f / (gpu_types[g].hbm_tbps * 1e12f);
+    }
+    for (int p = 0; p < P; ++p) { typeP[p] = (int)instances[p].type; qP[p] = instances[p].load_s; }
+    for (int d = 0; d < D; ++d) {
+        const hx_instance& in = instances[P + d];
+        typeD[d] = (int)in.type; qD[d] = in.load_s; capD[d] = in.kv_cap_tokens; freeD[d] = in.kv_free_tokens;
+    }
+    for (int m = 0; m < n_models; ++m) {
+        phi[m] = models[m].flops_per_token; omega[m] = models[m].weight_bytes; kappa[m] = models[m].kv_bytes_per_token;
+    }
+    for (int p = 0; p < P; ++p)
+        for (int d = 0; d < D; ++d)
+            invLT[(size_t)d * h->Ppad + p] = 1.0f / (link_bw_gbps[(size_t)p * n_instances + P + d] * 1e9f);
+
+    float *d_invF, *d_invB, *d_qP, *d_qD, *d_capD, *d_freeD, *d_invLT, *d_phi, *d_omega, *d_kappa;
+    int *d_typeP, *d_typeD;
+    bool ok = true; cudaError_t first = cudaSuccess;
+    auto up = [&](cudaError_t r) { if (r != cudaSuccess && ok) { ok = false; first = r; } };
+    up(dev_upload(h->allocs, &d_invF, invF)); up(dev_upload(h->allocs, &d_invB, invB));
+    up(dev_upload(h->allocs, &d_qP, qP)); up(dev_upload(h->allocs, &d_qD, qD));
+    up(dev_upload(h->allocs, &d_capD, capD)); up(dev_upload(h->allocs, &d_freeD, freeD));
+    up(dev_upload(h->allocs, &d_invLT, invLT)); up(dev_upload(h->allocs, &d_phi, phi));
+    up(dev_upload(h->allocs, &d_omega, omega)); up(dev_upload(h->allocs, &d_kappa, kappa));
+    up(dev_upload(h->allocs, &d_typeP, typeP)); up(dev_upload(h->allocs, &d_typeD, typeD));
+    up(dev_alloc(h->allocs, &h->status, 1));
+    if (ok) up(cudaMemset(h->status, 0, sizeof(int)));
+    if (!ok) return bail(fail_cuda(h, first, "uploading cluster tables"));
+    h->tab = HxTables{n_types, P, D, n_models, h->Ppad, d_invF, d_invB, d_typeP, d_typeD, d_qP, d_qD,
+                      d_capD, d_freeD, d_invLT, d_phi, d_omega, d_kappa};
+    *out = h;
+    return HX_OK;
+}
+
+int hx_cluster_update_loads(hx_cluster* h, const float* qP, const float* qD, const float* kv_free, void* stream) {
+    if (!h) return HX_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const float* src[3] = {qP, qD, kv_free};
+    float* dst[3] = {h->tab.qP, h->tab.qD, h->tab.freeD};
+    const int n[3] = {h->P, h->D, h->D};
+    for (int k = 0; k < 3; ++k) {
+        if (!src[k]) continue;
+        for (int i = 0; i < n[k]; ++i)
+            if (!good_load(src[k][i])) return fail(h, HX_ERR_INVALID_ARG, "loads must be finite and >= 0");
+    }
+    for (int k = 0; k < 3; ++k)
+        if (src[k])
+            HX_TRY(cudaMemcpyAsync(dst[k], src[k], n[k] * sizeof(float), cudaMemcpyHostToDevice, s), "cudaMemcpyAsync(loads)");
+    return HX_OK;
+}
+
+int hx_cluster_read_loads(hx_cluster* h, float* qP, float* qD, float* kv_free, void* stream) {
+    if (!h) return HX_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (qP) HX_TRY(cudaMemcpyAsync(qP, h->tab.qP, h->P * sizeof(float), cudaMemcpyDeviceToHost, s), "cudaMemcpyAsync(qP)");
+    if (qD) HX_TRY(cudaMemcpyAsync(qD, h->tab.qD, h->D * sizeof(float), cudaMemcpyDeviceToHost, s), "cudaMemcpyAsync(qD)");
+    if (kv_free) HX_TRY(cudaMemcpyAsync(kv_free, h->tab.freeD, h->D * sizeof(float), cudaMemcpyDeviceToHost, s), "cudaMemcpyAsync(kv_free)");
+    HX_TRY(cudaStreamSynchronize(s), "cudaStreamSynchronize");
+    return HX_OK;
+}
+
+int hx_cluster_destroy(hx_cluster* h) {
+    if (!h) return HX_OK;
+    DeviceGuard guard(h->device);
+    cudaDeviceSynchronize();
+    free_pool(h->allocs); free_pool(h->dag_allocs); free_pool(h->tk_allocs);
+    if (h->st_calls) cudaFree(h->st_calls);
+    if (h->st_assign) cudaFree(h->st_assign);
+    if (h->st_cost) cudaFree(h->st_cost);
+    delete h;
+    return HX_OK;
+}
+
+int hx_dag_upload(hx_cluster* h, const uint32_t* row_ptr, const uint32_t* col_idx, const float* node_costs,
+                  const uint32_t* node_workflow, const float* workflow_elapsed_s,
+                  uint32_t n_nodes, uint32_t n_edges, uint32_t n_workflows) {
+    if (!h) return HX_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    const uint32_t N = n_nodes, E = n_edges, W = n_workflows;
+    if (!row_ptr || !node_costs || !node_workflow || !workflow_elapsed_s || (E && !col_idx))
+        return fail(h, HX_ERR_INVALID_ARG, "NULL array");
+    if (W == 0 || N == 0) return fail(h, HX_ERR_INVALID_ARG, "empty forest");
+    if (row_ptr[0] != 0 || row_ptr[N] != E) return fail(h, HX_ERR_INVALID_ARG, "row_ptr does not span the edge array");
+    for (uint32_t v = 0; v < N; ++v) {
+        if (row_ptr[v + 1] < row_ptr[v]) return fail(h, HX_ERR_INVALID_ARG, "row_ptr is not monotone");
+        if (node_workflow[v] >= W) return fail(h, HX_ERR_INVALID_ARG, "workflow id out of range");
+        if (!good_load(node_costs[v])) return fail(h, HX_ERR_INVALID_ARG, "node costs must be finite and >= 0");
+    }
+    for (uint32_t w = 0; w < W; ++w)
+        if (!good_load(workflow_elapsed_s[w])) return fail(h, HX_ERR_INVALID_ARG, "elapsed times must be finite and >= 0");
+    std::vector<uint32_t> indeg(N, 0);
+    for (uint32_t v = 0; v < N; ++v)
+        for (uint32_t e = row_ptr[v]; e < row_ptr[v + 1]; ++e) {
+            const uint32_t u = col_idx[e];
+            if (u >= N) return fail(h, HX_ERR_INVALID_ARG, "edge target out of range");
+            if (node_workflow[u] != node_workflow[v]) return fail(h, HX_ERR_INVALID_ARG, "edge crosses workflows");
+            ++indeg[u];
+        }
+    // topological order (cycle check), then height above the sinks
+    std::vector<uint32_t> topo; topo.reserve(N);
+    for (uint32_t v = 0; v < N; ++v) if (indeg[v] == 0) topo.push_back(v);
+    for (size_t i = 0; i < topo.size(); ++i) {
+        const uint32_t v = topo[i];
+        for (uint32_t e = row_ptr[v]; e < row_ptr[v + 1]; ++e) if (--indeg[col_idx[e]] == 0) topo.push_back(col_idx[e]);
+    }
+    if (topo.size() != N) return fail(h, HX_ERR_CYCLE, "the graph has a cycle");
+    std::vector<uint32_t> height(N, 0);
+    uint32_t max_h = 0;
+    for (size_t i = N; i-- > 0;) {
+        const uint32_t v = topo[i];
+        uint32_t hh = 0;
+        for (uint32_t e = row_ptr[v]; e < row_ptr[v + 1]; ++e) hh = std::max(hh, height[col_idx[e]] + 1);
+        height[v] = hh; max_h = std::max(max_h, hh);
+    }
+    // regroup: workflow by workflow, inside a workflow by height (two stable counting sorts)
+    std::vector<uint32_t> by_h(N), perm(N), inv(N);
+    {
+        std::vector<uint32_t> cnt((size_t)max_h + 2, 0);
+        for (uint32_t v = 0; v < N; ++v) ++cnt[height[v] + 1];
+        for (size_t i = 1; i < cnt.size(); ++i) cnt[i] += cnt[i - 1];
+        for (uint32_t v = 0; v < N; ++v) by_h[cnt[height[v]]++] = v;
+    }
+    std::vector<uint32_t> wf_node_start((size_t)W + 1, 0);
+    for (uint32_t v = 0; v < N; ++v) ++wf_node_start[node_workflow[v] + 1];
+    for (uint32_t w = 0; w < W; ++w) wf_node_start[w + 1] += wf_node_start[w];
+    {
+        std::vector<uint32_t> cur(wf_node_start.begin(), wf_node_start.end() - 1);
+        for (uint32_t i = 0; i < N; ++i) { const uint32_t v = by_h[i]; perm[cur[node_workflow[v]]++] = v; }
+    }
+    for (uint32_t i = 0; i < N; ++i) inv[perm[i]] = i;
+    std::vector<uint32_t> wf_seg_start((size_t)W + 1, 0), seg_off;
+    seg_off.reserve((size_t)N + W);
+    for (uint32_t w = 0; w < W; ++w) {
+        wf_seg_start[w] = (uint32_t)seg_off.size();
+        const uint32_t ns = wf_node_start[w], ne = wf_node_start[w + 1];
+        seg_off.push_back(0);
+        for (uint32_t i = ns; i < ne; ++i)
+            if (i + 1 == ne || height[perm[i + 1]] != height[perm[i]]) seg_off.push_back(i + 1 - ns);
+    }
+    wf_seg_start[W] = (uint32_t)seg_off.size();
+    std::vector<uint32_t> irow((size_t)N + 1, 0), icol32(E), wf_edge_start((size_t)W + 1, 0);
+    std::vector<uint16_t> icol16(E);
+    std::vector<float> icost(N);
+    for (uint32_t i = 0; i < N; ++i) {
+        const uint32_t v = perm[i], ns = wf_node_start[node_workflow[v]];
+        icost[i] = node_costs[v];
+        uint32_t o = irow[i];
+        for (uint32_t e = row_ptr[v]; e < row_ptr[v + 1]; ++e, ++o) {
+            const uint32_t local = inv[col_idx[e]] - ns;
+            icol32[o] = local; icol16[o] = (uint16_t)local;
+        }
+        irow[i + 1] = o;
+    }
+    for (uint32_t w = 0; w <= W; ++w) wf_edge_start[w] = irow[wf_node_start[w]];
+
+    // classes of the horizon pass by staging footprint
+    const size_t kWarpSmall = 3072, kWarpBig = 24576, kBlock = 200 * 1024;
+    std::vector<uint32_t> ids[4];
+    for (uint32_t w = 0; w < W; ++w) {
+        const size_t n = wf_node_start[w + 1] - wf_node_start[w], e = wf_edge_start[w + 1] - wf_edge_start[w];
+        const size_t nlev = wf_seg_start[w + 1] - wf_seg_start[w] - 1;
+        const size_t need = 4 * (3 * n + 1) + 4 * (nlev + 1) + 2 * e + 16;
+        const int k = (n > 65535) ? 3 : need <= kWarpSmall ? 0 : need <= kWarpBig ? 1 : need <= kBlock ? 2 : 3;
+        ids[k].push_back(w);
+    }
+    // largest workflows first inside a class, so that the long ones do not start last
+    for (auto& v : ids)
+        std::stable_sort(v.begin(), v.end(), [&](uint32_t a, uint32_t b) {
+            return wf_node_start[a + 1] - wf_node_start[a] > wf_node_start[b + 1] - wf_node_start[b]; });
+
+    cudaDeviceSynchronize();
+    free_pool(h->dag_allocs);
+    h->dag_uploaded = false; h->cp_ready = false; h->classes.clear();
+    HxForestDev f{};
+    f.n_nodes = N; f.n_edges = E; f.n_workflows = W;
+    uint32_t *d_wns, *d_wes, *d_wss, *d_seg, *d_irow, *d_icol32, *d_perm;
+    uint16_t* d_icol16; float* d_icost;
+    HX_TRY(dev_upload(h->dag_allocs, &d_wns, wf_node_start), "upload forest");
+    HX_TRY(dev_upload(h->dag_allocs, &d_wes, wf_edge_start), "upload forest");
+    HX_TRY(dev_upload(h->dag_allocs, &d_wss, wf_seg_start), "upload forest");
+    HX_TRY(dev_upload(h->dag_allocs, &d_seg, seg_off), "upload forest");
+    HX_TRY(dev_upload(h->dag_allocs, &d_irow, irow), "upload forest");
+    HX_TRY(dev_upload(h->dag_allocs, &d_icol32, icol32), "upload forest");
+    HX_TRY(dev_upload(h->dag_allocs, &d_icol16, icol16), "upload forest");
+    HX_TRY(dev_upload(h->dag_allocs, &d_icost, icost), "upload forest");
+    HX_TRY(dev_upload(h->dag_allocs, &d_perm, perm), "upload forest");
+    f.wf_node_start = d_wns; f.wf_edge_start = d_wes; f.wf_seg_start = d_wss; f.seg_off = d_seg;
+    f.irow = d_irow; f.icol32 = d_icol32; f.icol16 = d_icol16; f.icost = d_icost; f.perm = d_perm;
+    HX_TRY(dev_alloc(h->dag_allocs, &f.cp, N), "alloc cp");
+    HX_TRY(dev_alloc(h->dag_allocs, &f.tail, N), "alloc tail");
+    HX_TRY(dev_alloc(h->dag_allocs, &f.H, W), "alloc H");
+    std::vector<uint32_t> nwf(node_workflow, node_workflow + N);
+    std::vector<float> el(workflow_elapsed_s, workflow_elapsed_s + W);
+    HX_TRY(dev_upload(h->dag_allocs, &h->d_node_wf, nwf), "upload node_workflow");
+    HX_TRY(dev_upload(h->dag_allocs, &h->d_elapsed, el), "upload elapsed");
+    const int tpw[4] = {32, 32, 256, 256}, per_block[4] = {16, 8, 1, 1};
+    const size_t sm[4] = {kWarpSmall, kWarpBig, kBlock, 0};
+    for (int k = 0; k < 4; ++k) {
+        if (ids[k].empty()) continue;
+        uint32_t* d_ids;
+        HX_TRY(dev_upload(h->dag_allocs, &d_ids, ids[k]), "upload workflow classes");
+        h->classes.push_back(HxCpClass{d_ids, (uint32_t)ids[k].size(), tpw[k], per_block[k], sm[k]});
+    }
+    h->forest = f;
+    h->dag_uploaded = true;
+    return HX_OK;
+}
+
+int hx_critical_path(hx_cluster* h, void* stream) {
+    if (!h) return HX_ERR_INVALID_ARG;
+    if (!h->dag_uploaded) return fail(h, HX_ERR_NOT_READY, "no forest uploaded");
+    DeviceGuard guard(h->device);
+    HX_TRY(hx_launch_cpath(h->forest, h->classes.data(), (int)h->classes.size(),
+                           static_cast<cudaStream_t>(stream), &h->launches), "horizon kernels");
+    h->cp_ready = true;
+    return HX_OK;
+}
+
+int hx_get_dag_results(hx_cluster* h, const float** cp, const float** tail, const float** H) {
+    if (!h) return HX_ERR_INVALID_ARG;
+    if (!h->dag_uploaded) return fail(h, HX_ERR_NOT_READY, "no forest uploaded");
+    if (cp) *cp = h->forest.cp;
+    if (tail) *tail = h->forest.tail;
+    if (H) *H = h->forest.H;
+    return HX_OK;
+}
+
+int hx_set_options(hx_cluster* h, const hx_options* o) {
+    if (!h || !o) return HX_ERR_INVALID_ARG;
+    if (o->score_mode < HX_MODE_COMPLETION || o->score_mode > HX_MODE_RATIO) return fail(h, HX_ERR_INVALID_ARG, "unknown score mode");
+    if (o->topk < 0 || o->topk > HX_MAX_TOPK) return fail(h, HX_ERR_INVALID_ARG, "topk out of range");
+    if (o->flags & ~(HX_FLAG_NO_DAG | HX_FLAG_NO_TAIL | HX_FLAG_UNLOADED)) return fail(h, HX_ERR_INVALID_ARG, "unknown flag");
+    if (!std::isfinite(o->alpha) || o->alpha <= 0.f) return fail(h, HX_ERR_INVALID_ARG, "alpha must be finite and > 0");
+    h->opts = *o;
+    return HX_OK;
+}
+
+int hx_schedule_batch(hx_cluster* h, const hx_call* calls, int n_calls, int32_t* out_assign,
+                      float* out_cost, void* stream) {
+    if (!h) return HX_ERR_INVALID_ARG;
+    if (n_calls < 0) return fail(h, HX_ERR_INVALID_ARG, "negative n_calls");
+    if (n_calls == 0) return HX_OK;
+    if (!calls || !out_assign || !out_cost) return fail(h, HX_ERR_INVALID_ARG, "NULL buffer");
+    if (reinterpret_cast<uintptr_t>(calls) % 16) return fail(h, HX_ERR_INVALID_ARG, "calls must be 16-byte aligned");
+    const hx_options& o = h->opts;
+    if (!(o.flags & HX_FLAG_NO_DAG) && !(h->dag_uploaded && h->cp_ready))
+        return fail(h, HX_ERR_NOT_READY, "horizons not computed: call hx_dag_upload and hx_critical_path, or set HX_FLAG_NO_DAG");
+    if (o.topk > 0 && n_calls > HX_MAX_COMMIT_CALLS)
+        return fail(h, HX_ERR_INVALID_ARG, "batch too large for the capacity-conflict pass; split it into chunks");
+    DeviceGuard guard(h->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (o.topk > 0) {
+        int rc = ensure_topk(h, n_calls, o.topk);
+        if (rc != HX_OK) return rc;
+        HX_TRY(cudaMemsetAsync(h->tk.dcount, 0, h->counter_bytes, s), "cudaMemsetAsync(counters)");
+    }
+    HxDagView dag{};
+    if (!(o.flags & HX_FLAG_NO_DAG))
+        dag = HxDagView{h->d_node_wf, h->forest.tail, h->forest.H, h->d_elapsed, h->forest.n_nodes, h->forest.n_workflows};
+    HxTopkBufs tk = h->tk;
+    tk.K = o.topk;
+    ScoreLaunch sl{calls, n_calls, out_assign, out_cost, o.score_mode, o.flags, o.topk, o.alpha};
+    HX_TRY(hx_launch_score(h->tab, dag, tk, sl, h->n_sm, h->max_smem, h->status, s, &h->launches), "scoring kernel");
+    if (o.topk > 0)
+        HX_TRY(hx_launch_conflict(h->tab, tk, n_calls, o.commit, out_assign, h->status, s, &h->launches), "conflict pass");
+    return HX_OK;
+}
+
+int hx_schedule_batch_host(hx_cluster* h, const hx_call* calls, int n_calls, int32_t* out_assign,
+                           float* out_cost, void* stream) {
+    if (!h) return HX_ERR_INVALID_ARG;
+    if (n_calls < 0) return fail(h, HX_ERR_INVALID_ARG, "negative n_calls");
+    if (n_calls == 0) return HX_OK;
+    if (!calls || !out_assign || !out_cost) return fail(h, HX_ERR_INVALID_ARG, "NULL buffer");
+    DeviceGuard guard(h->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (h->st_cap < n_calls) {
+        cudaDeviceSynchronize();
+        if (h->st_calls) cudaFree(h->st_calls);
+        if (h->st_assign) cudaFree(h->st_assign);
+        if (h->st_cost) cudaFree(h->st_cost);
+        h->st_calls = nullptr; h->st_assign = nullptr; h->st_cost = nullptr; h->st_cap = 0;
+        const size_t cap = (size_t)std::max(n_calls, 16384);
+        HX_TRY(cudaMalloc(&h->st_calls, cap * sizeof(hx_call)), "alloc staging");
+        HX_TRY(cudaMalloc(&h->st_assign, cap * sizeof(int32_t)), "alloc staging");
+        HX_TRY(cudaMalloc(&h->st_cost, cap * sizeof(float)), "alloc staging");
+        h->st_cap = (int)cap;
+    }
+    HX_TRY(cudaMemcpyAsync(h->st_calls, calls, (size_t)n_calls * sizeof(hx_call), cudaMemcpyHostToDevice, s), "copy calls");
+    int rc = hx_schedule_batch(h, h->st_calls, n_calls, h->st_assign, h->st_cost, stream);
+    if (rc != HX_OK) return rc;
+    HX_TRY(cudaMemcpyAsync(out_assign, h->st_assign, (size_t)n_calls * sizeof(int32_t), cudaMemcpyDeviceToHost, s), "copy assign");
+    HX_TRY(cudaMemcpyAsync(out_cost, h->st_cost, (size_t)n_calls * sizeof(float), cudaMemcpyDeviceToHost, s), "copy cost");
+    HX_TRY(cudaStreamSynchronize(s), "cudaStreamSynchronize");
+    return HX_OK;
+}
+
+int hx_get_topk(hx_cluster* h, const int32_t** pairs, const float** costs, const float** prio) {
+    if (!h) return HX_ERR_INVALID_ARG;
+    if (h->tk.cap_calls == 0) return fail(h, HX_ERR_NOT_READY, "no batch has been scored with topk > 0");
+    if (pairs) *pairs = h->tk.pair;
+    if (costs) *costs = h->tk.cost;
+    if (prio) *prio = h->tk.prio;
+    return HX_OK;
+}
+
+int hx_get_status(hx_cluster* h, int* status, void* stream) {
+    if (!h || !status) return HX_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    HX_TRY(cudaMemcpyAsync(status, h->status, sizeof(int), cudaMemcpyDeviceToHost, s), "read status");
+    HX_TRY(cudaStreamSynchronize(s), "cudaStreamSynchronize");
+    return HX_OK;
+}
+
+const char* hx_last_error(const hx_cluster* h) { return h ? h->err.c_str() : g_create_err.c_str(); }
+
+long long hx_launch_count(const hx_cluster* h) { return h ? h->launches : 0; }
+
+}  // extern "C"

@@ -1,0 +1,115 @@
+// Internal declarations shared by the translation units of libhx.so.
+#ifndef HX_INTERNAL_H_
+#define HX_INTERNAL_H_
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "hx.h"
+
+// ---------------------------------------------------------------------------
+// Packed cluster snapshot on the device (structure of arrays, binary32).
+// invLT is the link table transposed and inverted: invLT[d * Ppad + p] =
+// 1 / (GB/s of link p->d * 1e9); rows are padded with zeros to Ppad (a
+// multiple of 4) so that every row starts on a 16-byte boundary.
+// ---------------------------------------------------------------------------
+struct HxTables {
+    int G, P, D, M, Ppad;
+    const float* invF;      // [G] 1 / (TFLOP/s * 1e12)
+    const float* invB;      // [G] 1 / (TB/s * 1e12)
+    const int* typeP;       // [Ppad]
+    const int* typeD;       // [D]
+    float* qP;              // [Ppad] seconds
+    float* qD;              // [D]
+    const float* capD;      // [D] tokens
+    float* freeD;           // [D] tokens
+    const float* invLT;     // [D * Ppad]
+    const float* phi;       // [M] flops per token
+    const float* omega;     // [M] weight bytes
+    const float* kappa;     // [M] KV bytes per token
+};
+
+// Device view of the uploaded forest and of the horizon results.
+struct HxDagView {
+    const uint32_t* node_wf;   // [N] original numbering
+    const float* tail;         // [N]
+    const float* H;            // [W]
+    const float* elapsed;      // [W]
+    uint32_t n_nodes, n_workflows;
+};
+
+// Per-batch buffers of the top-K list and of the capacity-conflict pass.  All
+// sizes are linear in the batch: slots are kept in flat arrays segmented by
+// decode (or prefill) instance, segment bounds come from the counters.
+struct HxTopkBufs {
+    int K;
+    int cap_calls;             // capacity (calls) of the per-call arrays
+    int32_t* pair;             // [cap][K]
+    float* cost;               // [cap][K]
+    float* tpre;               // [cap][K] prefill time on the prefill instance of slot k
+    float* prio;               // [cap]
+    float* mtok;               // [cap]
+    // counters, zeroed before every batch (one contiguous allocation)
+    unsigned int* dcount;      // [D] valid slots naming decode instance d
+    unsigned int* dcursor;     // [D]
+    unsigned int* pcount;      // [P] calls that obtained prefill instance p
+    unsigned int* pcursor;     // [P]
+    unsigned int* n_acc;       // [1] calls that obtained a pair
+    uint4* dflat;              // [cap*K] {~prio bits, call, k, m bits}, grouped by decode instance
+    uint2* dsorted;            // [cap*K] {call | k << 24, m bits}, each group in visiting order
+    uint4* accflat;            // [cap]   {~prio bits, call, p, tpre bits} in order of acceptance
+    uint4* pseg;               // [cap]   same entries grouped by prefill instance
+    float* psorted;            // [cap]   prefill times, each group in visiting order
+};
+
+struct ScoreLaunch {
+    const hx_call* calls;
+    int n_calls;
+    int32_t* out_assign;
+    float* out_cost;
+    int mode, flags, K;
+    float alpha;
+};
+
+// Levelised forest on the device (internal numbering: workflow by workflow,
+// inside a workflow by increasing height above the sinks).
+struct HxForestDev {
+    uint32_t n_nodes, n_edges, n_workflows;
+    const uint32_t* wf_node_start;   // [W+1] internal index of the first node of each workflow
+    const uint32_t* wf_edge_start;   // [W+1] first edge of each workflow in icol
+    const uint32_t* wf_seg_start;    // [W+1] first entry of each workflow in seg_off
+    const uint32_t* seg_off;         // per workflow: local offsets of its levels, nlev+1 entries
+    const uint32_t* irow;            // [N+1] edge offsets (global) in internal numbering
+    const uint16_t* icol16;          // [E] successor as local index inside the workflow (16-bit copy)
+    const uint32_t* icol32;          // [E] same, 32-bit
+    const float* icost;              // [N]
+    const uint32_t* perm;            // [N] internal -> original node number
+    float* cp;                       // [N] original numbering
+    float* tail;                     // [N]
+    float* H;                        // [W]
+};
+
+cudaError_t hx_launch_score(const HxTables& t, const HxDagView& dag, const HxTopkBufs& tk,
+                            const ScoreLaunch& s, int n_sm, size_t max_smem, int* status,
+                            cudaStream_t stream, long long* launches);
+
+cudaError_t hx_launch_conflict(const HxTables& t, const HxTopkBufs& tk, int n_calls, int commit,
+                               int32_t* out_assign, int* status, cudaStream_t stream,
+                               long long* launches);
+
+// Workflow classes of the horizon pass: lists of workflow ids handled by one launch each.
+struct HxCpClass {
+    const uint32_t* wf_ids;    // device
+    uint32_t count;
+    int threads_per_wf;        // 32 (one warp) or the block size
+    int wfs_per_block;
+    size_t smem_per_wf;        // bytes of staging per workflow, 0 = work in global memory
+};
+
+cudaError_t hx_launch_cpath(const HxForestDev& f, const HxCpClass* classes, int n_classes,
+                            cudaStream_t stream, long long* launches);
+
+#endif  // HX_INTERNAL_H_

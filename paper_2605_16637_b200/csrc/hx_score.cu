@@ -1,0 +1,413 @@
+// Batched placement scoring (paper Algorithm 1, inner loop over the waiting
+// calls; Section 5.3 "Projected-risk prefill ranking" and "Joint prefill-decode
+// planning"; feasibility by Eq. 3-4; score by Eq. 2).
+//
+// For call c and pair (p, d):
+//   ready(c,p,d) = fma(kvB_c, invL[p][d], A_c[p])        A_c[p] = qP[p] + tpre_c[typeP[p]]
+//   fin(c,p,d)   = max(ready, qD[d]) + Dd_c[d]           Dd_c[d] = m_c <= capD[d] ? tdec_c[typeD[d]] : +inf
+// and the call goes to the pair with the smallest fin, lowest p*D+d among equals.
+//
+// x -> max(x, qD) + Dd is non-decreasing in x also after rounding (max is exact,
+// round-to-nearest addition is monotone), therefore
+//   min_p fin(c,p,d) = max(min_p ready(c,p,d), qD[d]) + Dd_c[d]        bit for bit.
+// The hot loop therefore only does one fused multiply-add and one minimum per
+// candidate: a (calls x decode) register tile of running minima with the prefill
+// index as the reduction dimension, operands staged in shared memory: the link
+// table transposed (rows = decode instances, contiguous in p) and the per-call
+// prefill-finish rows A.  Two consecutive p are processed by one packed
+// fma.rn.f32x2 and folded into the running minimum by one three-input min.
+// The clamp, the decode term, the selection over d and the recovery of the
+// prefill index (a rescan of one row of P candidates for the few selected d)
+// run once per (call, d) or per call.
+#include "hx_internal.h"
+
+namespace {
+
+typedef unsigned long long u64;
+
+struct ScoreParams {
+    HxTables t;
+    HxDagView dag;
+    HxTopkBufs tk;
+    ScoreLaunch s;
+    int* status;
+    int WDn, WCn;        // warps along decode columns / along calls
+    int TCB;             // calls per block tile
+    int nTiles;
+    int Dpad;            // decode columns covered by the block (multiple of 8*LD)
+    int PC;              // prefill chunk length (multiple of 4)
+    int nChunks;
+    int PS;              // shared-memory row stride of LT and A (PC + 4 or PC + 8)
+    int FS;              // row stride of the per-call finish times (Dpad + 4)
+    int offA, offCall, offInst;   // byte offsets into dynamic shared memory (LT at 0)
+};
+
+__device__ __forceinline__ u64 fma2(u64 a, u64 b, u64 c) {
+    u64 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ float min3(float a, float b, float c) {
+    float d;
+    asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ u64 pack2(float lo, float hi) {
+    u64 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(u64 v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+
+#define HX_INF __int_as_float(0x7f800000)
+#define HX_NONE 0x7fffffff
+
+// Smallest (value, column) pair of the row that is lexicographically greater
+// than (pv, pd); (+inf, HX_NONE) if there is none.  Executed by an aligned
+// group of four lanes (gmask); the result is the same on all four.
+__device__ __forceinline__ void group_next(const float* frow, int nq, int t, unsigned gmask,
+                                           float pv, int pd, float& bv, int& bd) {
+    bv = HX_INF; bd = HX_NONE;
+    for (int q = t; q < nq; q += 4) {
+        const float4 f = *reinterpret_cast<const float4*>(frow + 4 * q);
+        const float v[4] = {f.x, f.y, f.z, f.w};
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int d = 4 * q + u;
+            const bool after = (v[u] > pv) || (v[u] == pv && d > pd);
+            if (after && v[u] < bv) { bv = v[u]; bd = d; }
+        }
+    }
+#pragma unroll
+    for (int off = 1; off <= 2; off <<= 1) {
+        const float ov = __shfl_xor_sync(gmask, bv, off);
+        const int od = __shfl_xor_sync(gmask, bd, off);
+        if (ov < bv || (ov == bv && od < bd)) { bv = ov; bd = od; }
+    }
+}
+
+// Lowest prefill index whose candidate on decode column d finishes exactly at v.
+__device__ __forceinline__ int group_rescan(const HxTables& T, const float* qPs, const int* typePs,
+                                            const float* tpre_c, float kvB, float qd, float Dd,
+                                            int d, float v, int t, unsigned gmask) {
+    int best = HX_NONE;
+    const float4* lrow = reinterpret_cast<const float4*>(T.invLT + (size_t)d * T.Ppad);
+    const int nq = T.Ppad >> 2;
+    for (int q = t; q < nq; q += 4) {
+        const float4 l4 = __ldg(lrow + q);
+        const float l[4] = {l4.x, l4.y, l4.z, l4.w};
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int p = 4 * q + u;
+            const float A = __fadd_rn(qPs[p], tpre_c[typePs[p]]);
+            const float r = __fmaf_rn(kvB, l[u], A);
+            const float f = __fadd_rn(fmaxf(r, qd), Dd);
+            if (f == v && p < best) best = p;
+        }
+    }
+#pragma unroll
+    for (int off = 1; off <= 2; off <<= 1) best = min(best, __shfl_xor_sync(gmask, best, off));
+    return best;
+}
+
+template <int TC, int LD>
+__global__ void __launch_bounds__(256, 1) hx_score_kernel(const __grid_constant__ ScoreParams prm) {
+    extern __shared__ __align__(16) unsigned char smem[];
+    constexpr int LC = 32 / LD;
+    const HxTables& T = prm.t;
+    const int G = T.G, P = T.P, D = T.D, Ppad = T.Ppad;
+    const int tid = threadIdx.x, nthr = blockDim.x;
+    const int warp = tid >> 5, lane = tid & 31;
+    const int wd = warp % prm.WDn, wc = warp / prm.WDn;
+    const int dg = lane % LD, cg = lane / LD;
+    const int PS = prm.PS, FS = prm.FS, PC = prm.PC, TCB = prm.TCB, Dpad = prm.Dpad;
+    const bool unloaded = prm.s.flags & HX_FLAG_UNLOADED;
+
+    float* LTs = reinterpret_cast<float*>(smem);                  // [Dpad][PS]
+    float* As = reinterpret_cast<float*>(smem + prm.offA);        // [TCB][PS], later fin [TCB][FS]
+    float* kvBs = reinterpret_cast<float*>(smem + prm.offCall);   // [TCB]
+    float* mtoks = kvBs + TCB;                                    // [TCB]
+    float* tpres = mtoks + TCB;                                   // [TCB][G]
+    float* tdecs = tpres + TCB * G;                               // [TCB][G]
+    float* qPs = reinterpret_cast<float*>(smem + prm.offInst);    // [Ppad]
+    int* typePs = reinterpret_cast<int*>(qPs + Ppad);             // [Ppad]
+    float* qDs = reinterpret_cast<float*>(typePs + Ppad);         // [Dpad]
+    float* capDs = qDs + Dpad;                                    // [Dpad]
+    int* typeDs = reinterpret_cast<int*>(capDs + Dpad);           // [Dpad]
+
+    // instance tables; padded prefill slots can never win, padded decode columns are infeasible
+    for (int p = tid; p < Ppad; p += nthr) {
+        qPs[p] = p < P ? (unloaded ? 0.0f : T.qP[p]) : HX_INF;
+        typePs[p] = p < P ? T.typeP[p] : 0;
+    }
+    for (int d = tid; d < Dpad; d += nthr) {
+        qDs[d] = d < D ? (unloaded ? 0.0f : T.qD[d]) : 0.0f;
+        capDs[d] = d < D ? T.capD[d] : -1.0f;
+        typeDs[d] = d < D ? T.typeD[d] : 0;
+    }
+    auto load_LT = [&](int pc0) {
+        const int nq = PC >> 2;
+        for (int idx = tid; idx < Dpad * nq; idx += nthr) {
+            const int d = idx / nq, q = idx - d * nq;
+            const int p = pc0 + 4 * q;
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (d < D && p < Ppad) v = __ldg(reinterpret_cast<const float4*>(T.invLT + (size_t)d * Ppad + p));
+            *reinterpret_cast<float4*>(LTs + d * PS + 4 * q) = v;
+        }
+    };
+    if (prm.nChunks == 1) load_LT(0);
+    __syncthreads();
+
+    for (int tile = blockIdx.x; tile < prm.nTiles; tile += gridDim.x) {
+        const int c0 = tile * TCB;
+        const int nvalid = min(TCB, prm.s.n_calls - c0);
+
+        // per-call service times on every GPU class (roofline-style estimate, Section 4.2)
+        for (int c = tid; c < TCB; c += nthr) {
+            float n = 1.f, o = 1.f, phi = 0.f, omega = 0.f, kappa = 0.f;
+            if (c < nvalid) {
+                const uint4 raw = __ldg(reinterpret_cast<const uint4*>(prm.s.calls) + c0 + c);
+                n = __uint_as_float(raw.z); o = __uint_as_float(raw.w);
+                if (raw.y < (unsigned)T.M) { phi = T.phi[raw.y]; omega = T.omega[raw.y]; kappa = T.kappa[raw.y]; }
+            }
+            const float kvB = __fmul_rn(n, kappa);
+            const float m = __fadd_rn(n, o);
+            const float ctx = __fmaf_rn(0.5f, __fsub_rn(o, 1.0f), n);
+            const float step = __fmaf_rn(kappa, ctx, omega);
+            const float nphi = __fmul_rn(n, phi), wkv = __fadd_rn(omega, kvB), ostep = __fmul_rn(o, step);
+            for (int g = 0; g < G; ++g) {
+                const float iF = T.invF[g], iB = T.invB[g];
+                tpres[c * G + g] = fmaxf(__fmul_rn(nphi, iF), __fmul_rn(wkv, iB));
+                tdecs[c * G + g] = __fmul_rn(ostep, iB);
+            }
+            kvBs[c] = kvB; mtoks[c] = m;
+        }
+        __syncthreads();
+
+        float acc[TC][8];
+#pragma unroll
+        for (int i = 0; i < TC; ++i)
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc[i][j] = HX_INF;
+        u64 kk[TC];
+#pragma unroll
+        for (int i = 0; i < TC; ++i) {
+            const float k = kvBs[wc * (TC * LC) + cg + LC * i];
+            kk[i] = pack2(k, k);
+        }
+        const float* Arow = As + (wc * (TC * LC) + cg) * PS;       // row i at + i * LC * PS
+        const float* Lrow = LTs + (wd * (8 * LD) + dg) * PS;       // row j at + j * LD * PS
+
+        for (int ch = 0; ch < prm.nChunks; ++ch) {
+            const int pc0 = ch * PC;
+            if (prm.nChunks > 1) load_LT(pc0);
+            {   // prefill finish times A[c][p] of this chunk
+                const int nq = PC >> 2;
+                for (int idx = tid; idx < TCB * nq; idx += nthr) {
+                    const int c = idx / nq, q = idx - c * nq;
+                    const int p = pc0 + 4 * q;
+                    float a[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+                        a[u] = (p + u < Ppad) ? __fadd_rn(qPs[p + u], tpres[c * G + typePs[p + u]]) : HX_INF;
+                    *reinterpret_cast<float4*>(As + c * PS + 4 * q) = make_float4(a[0], a[1], a[2], a[3]);
+                }
+            }
+            __syncthreads();
+#pragma unroll 2
+            for (int q = 0; q < (PC >> 2); ++q) {
+                ulonglong2 a[TC], l[8];
+#pragma unroll
+                for (int i = 0; i < TC; ++i)
+                    a[i] = *reinterpret_cast<const ulonglong2*>(Arow + i * LC * PS + 4 * q);
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    l[j] = *reinterpret_cast<const ulonglong2*>(Lrow + j * LD * PS + 4 * q);
+#pragma unroll
+                for (int i = 0; i < TC; ++i)
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        float r0, r1, r2, r3;
+                        unpack2(fma2(kk[i], l[j].x, a[i].x), r0, r1);
+                        unpack2(fma2(kk[i], l[j].y, a[i].y), r2, r3);
+                        acc[i][j] = min3(min3(acc[i][j], r0, r1), r2, r3);
+                    }
+            }
+            __syncthreads();
+        }
+
+        // clamp to the decode admission time and add the decode term; park the
+        // per-(call, d) finish times in shared memory (over the A tile)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int d = wd * (8 * LD) + dg + LD * j;
+            const float qd = qDs[d], cap = capDs[d];
+            const int ty = typeDs[d];
+#pragma unroll
+            for (int i = 0; i < TC; ++i) {
+                const int c = wc * (TC * LC) + cg + LC * i;
+                const float Dd = (mtoks[c] <= cap) ? tdecs[c * G + ty] : HX_INF;
+                As[c * FS + d] = __fadd_rn(fmaxf(acc[i][j], qd), Dd);
+            }
+        }
+        __syncthreads();
+
+        // selection over d, prefill index recovery and per-call score: four lanes per call
+        const int K = prm.s.K;
+        const int ngroups = nthr >> 2, gid = tid >> 2, t = tid & 3;
+        const unsigned gmask = 0xFu << (lane & 28);       // groups of one warp may leave the loops at different times
+        for (int cb = 0; cb < TCB; cb += ngroups) {
+            const int c = cb + gid;
+            const bool live = c < nvalid;                 // uniform inside the group
+            const int cs = live ? c : 0;
+            const float* frow = As + cs * FS;
+            const float kvB = kvBs[cs], m = mtoks[cs];
+            const float* tpre_c = tpres + cs * G;
+            float pv = -1.0f; int pd = -1;
+            float v0 = HX_INF; int jbest = HX_NONE;
+            int sel_pair[HX_MAX_TOPK]; float sel_cost[HX_MAX_TOPK], sel_tpre[HX_MAX_TOPK];
+#pragma unroll
+            for (int k = 0; k < HX_MAX_TOPK; ++k) { sel_pair[k] = -1; sel_cost[k] = HX_INF; sel_tpre[k] = 0.f; }
+            const int want = K > 0 ? K : 1;
+            for (int k = 0;; ++k) {
+                float v; int d;
+                group_next(frow, Dpad >> 2, t, gmask, pv, pd, v, d);
+                if (d == HX_NONE) break;                  // nothing (feasible) left
+                if (k == 0) v0 = v;
+                const bool tie = (K == 0) && (v == v0);   // the plain argmin orders ties by p first
+                if (k >= want && !tie) break;
+                const float Dd = (m <= capDs[d]) ? tdecs[cs * G + typeDs[d]] : HX_INF;
+                const int p = group_rescan(T, qPs, typePs, tpre_c, kvB, qDs[d], Dd, d, v, t, gmask);
+                if (k < want) {
+#pragma unroll
+                    for (int k2 = 0; k2 < HX_MAX_TOPK; ++k2)
+                        if (k2 == k) { sel_pair[k2] = p * D + d; sel_cost[k2] = v; sel_tpre[k2] = tpre_c[typePs[p]]; }
+                }
+                if (v == v0) jbest = min(jbest, p * D + d);
+                pv = v; pd = d;
+            }
+            if (live && t == 0) {
+                const int gc = c0 + c;
+                const uint4 raw = __ldg(reinterpret_cast<const uint4*>(prm.s.calls) + gc);
+                float elapsed = 0.f, tail = 0.f, H = 1.f;
+                bool bad = raw.y >= (unsigned)T.M;
+                if (!(prm.s.flags & HX_FLAG_NO_DAG)) {
+                    if (raw.x < prm.dag.n_nodes) {
+                        const uint32_t w = prm.dag.node_wf[raw.x];
+                        elapsed = prm.dag.elapsed[w];
+                        H = prm.dag.H[w];
+                        if (!(prm.s.flags & HX_FLAG_NO_TAIL)) tail = prm.dag.tail[raw.x];
+                    } else {
+                        bad = true;
+                    }
+                }
+                if (bad) { atomicExch(prm.status, HX_ERR_INVALID_ARG); v0 = HX_INF; jbest = HX_NONE; }
+                const float comp = __fadd_rn(__fadd_rn(elapsed, v0), tail);
+                float score = comp;
+                if (prm.s.mode == HX_MODE_SLACK) score = __fsub_rn(__fmul_rn(prm.s.alpha, H), comp);
+                else if (prm.s.mode == HX_MODE_RATIO) score = __fdiv_rn(comp, H);
+                if (bad) score = HX_INF;
+                prm.s.out_cost[gc] = score;
+                if (K == 0) {
+                    prm.s.out_assign[gc] = (jbest == HX_NONE) ? -1 : jbest;
+                } else {
+                    prm.s.out_assign[gc] = -1;            // filled in by the capacity-conflict pass
+                    prm.tk.prio[gc] = __fdiv_rn(__fadd_rn(elapsed, v0), H);   // Eq. 2
+                    prm.tk.mtok[gc] = m;
+#pragma unroll
+                    for (int k = 0; k < HX_MAX_TOPK; ++k) {
+                        if (k >= K) break;
+                        const int pr = bad ? -1 : sel_pair[k];
+                        prm.tk.pair[(size_t)gc * K + k] = pr;
+                        prm.tk.cost[(size_t)gc * K + k] = bad ? HX_INF : sel_cost[k];
+                        prm.tk.tpre[(size_t)gc * K + k] = sel_tpre[k];
+                        if (pr >= 0) atomicAdd(&prm.tk.dcount[pr % D], 1u);   // segment sizes of the conflict pass
+                    }
+                }
+            }
+        }
+        __syncthreads();
+    }
+}
+
+template <int TC, int LD>
+cudaError_t launch_one(const ScoreParams& prm, int grid, int threads, size_t smem, cudaStream_t stream) {
+    cudaError_t e = cudaFuncSetAttribute(hx_score_kernel<TC, LD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    hx_score_kernel<TC, LD><<<grid, threads, smem, stream>>>(prm);
+    return cudaGetLastError();
+}
+
+inline int round_up(int a, int b) { return (a + b - 1) / b * b; }
+// row padding (floats) that makes the row stride an odd number of 16-byte units, so that the
+// rows read by the lanes of a warp start in different banks
+inline int pad_of(int pc) { return ((pc >> 2) & 1) ? 8 : 4; }
+
+}  // namespace
+
+cudaError_t hx_launch_score(const HxTables& t, const HxDagView& dag, const HxTopkBufs& tk,
+                            const ScoreLaunch& s, int n_sm, size_t max_smem, int* status,
+                            cudaStream_t stream, long long* launches) {
+    ScoreParams prm;
+    prm.t = t; prm.dag = dag; prm.tk = tk; prm.s = s; prm.status = status;
+    const int D = t.D, C = s.n_calls;
+    const int LD = D > 32 ? 8 : D > 16 ? 4 : D > 8 ? 2 : 1;
+    const int LC = 32 / LD, WD = 8 * LD;
+    prm.WDn = (D + WD - 1) / WD;
+    prm.Dpad = prm.WDn * WD;
+    // warps along calls: up to 8 warps per block, fewer when the batch is too small to fill the SMs
+    const int min_tc = LD == 8 ? 5 : 8;
+    int WCn = prm.WDn >= 8 ? 1 : 8 / prm.WDn;
+    while (WCn > 1 && (C + WCn * min_tc * LC - 1) / (WCn * min_tc * LC) < n_sm) WCn >>= 1;
+    prm.WCn = WCn;
+    // thread tile height: spread the calls evenly over the SMs (a tile of 8 rows per lane
+    // would leave SMs idle whenever the batch is not a multiple of n_sm * WCn * LC * 8 calls)
+    int TC = 8;
+    if (LD == 8) {
+        const int per_sm = (C + n_sm - 1) / n_sm;
+        const int rows = WCn * LC;
+        const int tiles_per_sm = (per_sm + 8 * rows - 1) / (8 * rows);
+        TC = (per_sm + tiles_per_sm * rows - 1) / (tiles_per_sm * rows);
+        TC = TC < 5 ? 5 : (TC > 8 ? 8 : TC);
+    }
+    prm.TCB = WCn * TC * LC;
+    prm.nTiles = (C + prm.TCB - 1) / prm.TCB;
+    prm.FS = prm.Dpad + 4;
+    // prefill chunk: the transposed link tile and the A tile share one row stride
+    const int G = t.G;
+    const size_t callB = (size_t)prm.TCB * (2 + 2 * G) * 4;
+    const size_t instB = (size_t)(2 * t.Ppad + 3 * prm.Dpad) * 4;
+    const size_t fixed = round_up((int)callB, 16) + round_up((int)instB, 16);
+    if (fixed + 4096 > max_smem) return cudaErrorInvalidConfiguration;
+    const size_t budget = max_smem - fixed - 64;
+    int PC = t.Ppad;
+    for (;;) {
+        const size_t a_rows = (size_t)prm.TCB * (PC + pad_of(PC)) * 4;
+        const size_t f_rows = (size_t)prm.TCB * prm.FS * 4;
+        const size_t need = (size_t)prm.Dpad * (PC + pad_of(PC)) * 4 + (a_rows > f_rows ? a_rows : f_rows);
+        if (need <= budget || PC <= 4) break;
+        PC = round_up(PC / 2, 4);
+    }
+    prm.PC = PC;
+    prm.nChunks = (t.Ppad + PC - 1) / PC;
+    prm.PS = PC + pad_of(PC);
+    const size_t ltB = (size_t)prm.Dpad * prm.PS * 4;
+    const size_t aB = (size_t)prm.TCB * (prm.PS > prm.FS ? prm.PS : prm.FS) * 4;
+    prm.offA = round_up((int)ltB, 16);
+    prm.offCall = prm.offA + round_up((int)aB, 16);
+    prm.offInst = prm.offCall + round_up((int)callB, 16);
+    const size_t smem = prm.offInst + round_up((int)instB, 16);
+    if (smem > max_smem) return cudaErrorInvalidConfiguration;
+    const int threads = 32 * prm.WDn * prm.WCn;
+    const int grid = prm.nTiles < n_sm ? prm.nTiles : n_sm;
+    cudaError_t e;
+#define HX_CASE(tc, ld) if (TC == tc && LD == ld) e = launch_one<tc, ld>(prm, grid, threads, smem, stream); else
+    HX_CASE(8, 8) HX_CASE(7, 8) HX_CASE(6, 8) HX_CASE(5, 8)
+    HX_CASE(8, 4) HX_CASE(8, 2) HX_CASE(8, 1)
+    e = cudaErrorInvalidConfiguration;
+#undef HX_CASE
+    if (e == cudaSuccess) ++*launches;
+    return e;
+}
