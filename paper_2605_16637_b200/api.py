@@ -185,7 +185,7 @@ class _Borrowed:
     """A borrowed device buffer exposed through the CUDA array interface."""
 
     def __init__(self, ptr, count, typestr):
-        self.__cuda_array_interface__ = {"shape": (count,), "typestr": typestr, "data": (int(ptr), True),
+        self.__cuda_array_interface__ = {"shape": (count,), "typestr": typestr, "data": (int(ptr), False),
                                          "version": 2}
 
 
