@@ -1,0 +1,336 @@
+#!/usr/bin/env python
+"""Benchmark of the placement-scoring hot path on the throughput-sweep workload.
+
+One step = one pass of the whole path over the sweep configuration: horizon
+kernels over the workflow forest, then 16 scheduler invocations of 16,384 ready
+calls each against 128 x 128 instance pairs (load refresh, scoring with top-4
+lists, capacity-conflict pass with commit).  Prints one JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "placement candidates scored/sec"
+UNIT = "candidates/s"
+FP32_LANES_PER_SM = 128
+
+
+def _peaks():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return json.load(f), "measured"
+    except Exception:
+        return {"hbm_gbs": 6650.0, "sm_max_mhz": 1965.0}, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except Exception:
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------------------------
+# CPU oracle legs (reference arm and cpu_baseline)
+# ----------------------------------------------------------------------------------------------
+
+def oracle_chunks(wl, n_chunks, with_dag):
+    """Runs the oracle, as it stands, on the first n_chunks scheduler invocations of the
+    workload; returns (candidates, seconds)."""
+    from oracle import hx_oracle as ho
+    orc = ho.Oracle()
+    oc = ho.Cluster.from_workload(wl)
+    calls = wl.calls
+    dag = None
+    t0 = time.perf_counter()
+    if with_dag:
+        # horizons from the stand-alone node costs of the workflows touched by these chunks
+        from hx_synth import sub_forest
+        touched = np.unique(wl.node_wf[wl.ready_nodes[: n_chunks * wl.chunk]])
+        rp, col, lwf, ids = sub_forest(wl, touched)
+        cost = orc.schedule(oc, wl.node_calls[ids], flags=ho.FLAG_UNLOADED | ho.FLAG_NO_DAG)[2]
+        sub = orc.longest_path(rp, col, cost, lwf, touched.shape[0])
+        tail = np.zeros(wl.n_nodes, np.float32); tail[ids] = sub.tail
+        H = np.ones(wl.n_workflows, np.float32); H[touched] = sub.H
+        dag = ho.DagResult(None, tail, H)
+    free0 = wl.kv_free[wl.P:].copy()
+    cand = 0
+    for i in range(n_chunks):
+        c = calls[i * wl.chunk:(i + 1) * wl.chunk]
+        pair, cost, prio, m, tsel = orc.topk(oc, c, wl.topk, dag=dag, node_wf=wl.node_wf, elapsed=wl.elapsed)
+        _, _, qP = orc.conflict(pair, prio, m, tsel, free0, oc.qP, wl.D)
+        oc.qP[:] = qP
+        cand += c.shape[0] * wl.P * wl.D
+    return cand, time.perf_counter() - t0
+
+
+def run_reference(args):
+    from hx_synth import make_workload
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    wl = make_workload("sweep")
+    n_chunks = 1                      # bounded sample per step: 1 of the 16 invocations
+    times = []
+    for i in range(args.warmup + args.steps):
+        cand, dt = oracle_chunks(wl, n_chunks, with_dag=False)
+        if i >= args.warmup:
+            times.append(dt)
+    ms = 1e3 * float(np.mean(times))
+    value = cand / (ms * 1e-3)
+    sample = "%d of 16 invocations (%d calls x 16384 pairs, top-4 + conflict pass) per step" % (
+        n_chunks, n_chunks * wl.chunk)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "sweep: 128x128 instances, 262,144 ready calls in chunks of 16,384, top-4 + commit",
+                   "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+# ----------------------------------------------------------------------------------------------
+# CUDA arm
+# ----------------------------------------------------------------------------------------------
+
+def run_cuda(args):
+    import torch
+    import paper_2605_16637_b200 as hx
+    from hx_synth import make_workload
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    # every rank schedules its own, differently seeded, sweep (no data-path exchange)
+    wl = make_workload("sweep", seed=4 + rank)
+    gc = hx.Cluster.from_workload(wl)
+    P, D, chunk = wl.P, wl.D, wl.chunk
+    n_calls = wl.ready_nodes.shape[0]
+    n_chunks = n_calls // chunk
+    cand_per_step = n_calls * P * D
+
+    # stand-alone node costs come from the library itself (unloaded scoring of every node)
+    gc.set_options(score_mode=hx.HX_MODE_COMPLETION, flags=hx.HX_FLAG_UNLOADED | hx.HX_FLAG_NO_DAG)
+    node_cost = gc.schedule_batch(wl.node_calls)[1].cpu().numpy()
+    gc.dag_upload(wl.row_ptr, wl.col, node_cost, wl.node_wf, wl.elapsed)
+    gc.critical_path()
+    gc.set_options(score_mode=hx.HX_MODE_RATIO, topk=wl.topk, commit=1, alpha=wl.alpha)
+
+    calls_host = torch.from_numpy(wl.calls.view(np.uint8).reshape(-1, 16).copy()).pin_memory()
+    calls_dev = calls_host.cuda()
+    out_assign = torch.empty(n_calls, dtype=torch.int32, device="cuda")
+    out_cost = torch.empty(n_calls, dtype=torch.float32, device="cuda")
+    host_assign = torch.empty(n_calls, dtype=torch.int32).pin_memory()
+    host_cost = torch.empty(n_calls, dtype=torch.float32).pin_memory()
+    qP0, qD0, free0 = wl.load_s[:P].copy(), wl.load_s[P:].copy(), wl.kv_free[P:].copy()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")      # larger than the 126 MB L2
+    stream = torch.cuda.current_stream()
+    sptr = stream.cuda_stream
+    h = gc.h
+
+    def step_device(chunk_events=None):
+        hx.hx_critical_path(h, sptr)
+        hx.hx_cluster_update_loads(h, qP0, qD0, free0, sptr)
+        for i in range(n_chunks):
+            if chunk_events is not None:
+                chunk_events[i][0].record(stream)
+            hx.hx_cluster_update_loads(h, None, None, free0, sptr)
+            lo = i * chunk
+            hx.hx_schedule_batch(h, calls_dev[lo:lo + chunk].data_ptr(), chunk,
+                                 out_assign[lo:lo + chunk].data_ptr(), out_cost[lo:lo + chunk].data_ptr(), sptr)
+            if chunk_events is not None:
+                chunk_events[i][1].record(stream)
+
+    ch_np = calls_host.numpy().view(hx.CALL_DTYPE).reshape(-1)
+    ha_np, hc_np = host_assign.numpy(), host_cost.numpy()
+
+    def step_host():
+        hx.hx_critical_path(h, sptr)
+        hx.hx_cluster_update_loads(h, qP0, qD0, free0, sptr)
+        for i in range(n_chunks):
+            hx.hx_cluster_update_loads(h, None, None, free0, sptr)
+            lo = i * chunk
+            hx.hx_schedule_batch_host(h, ch_np[lo:lo + chunk], ha_np[lo:lo + chunk], hc_np[lo:lo + chunk], sptr)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step_device()
+    barrier()
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    gc.enable_kernel_timing(True)
+    gc.read_kernel_timing()
+    launches0 = gc.launch_count()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    cev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_chunks)]
+           for _ in range(args.steps)]
+    barrier()
+    for k in range(args.steps):
+        flush.zero_()                                   # L2 flush between timed iterations (not timed)
+        ev[k][0].record(stream)
+        step_device(cev[k])
+        ev[k][1].record(stream)
+    barrier()
+    launches = gc.launch_count() - launches0
+    kt = gc.read_kernel_timing()
+    gc.enable_kernel_timing(False)
+    step_ms = np.array([a.elapsed_time(b) for a, b in ev])
+    chunk_us = np.array([[a.elapsed_time(b) * 1e3 for a, b in row] for row in cev]).reshape(-1)
+    status = gc.status()
+
+    # end to end through the host-buffer entry point (pinned host memory, copies inside the timed region)
+    for _ in range(2):
+        step_host()
+    barrier()
+    t0 = time.perf_counter()
+    for k in range(args.steps):
+        step_host()
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+
+    total_ms = float(step_ms.sum())
+    tot = torch.tensor([total_ms, e2e_s], dtype=torch.float64, device="cuda")
+    if dist is not None:
+        dist.all_reduce(tot, op=dist.ReduceOp.MAX)
+    total_ms, e2e_s = float(tot[0]), float(tot[1])
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    ms_per_step = total_ms / args.steps
+    value = world * cand_per_step / (ms_per_step * 1e-3)
+    e2e_value = world * cand_per_step * args.steps / e2e_s
+    peaks, which = _peaks()
+    n_sm = torch.cuda.get_device_properties(local).multi_processor_count
+    sm_max_mhz = float(peaks.get("sm_max_mhz", 1965.0))
+    # dominant kernel: scoring.  Algorithmic work: one binary32 fused multiply-add (2 flop) per candidate.
+    score_ms, score_n = kt["scoring"]
+    score_avg_ms = score_ms / max(score_n, 1)
+    achieved = 2.0 * chunk * P * D / (score_avg_ms * 1e-3) / 1e12
+    peak = 2.0 * n_sm * FP32_LANES_PER_SM * sm_max_mhz * 1e6 / 1e12
+    roofline = {"bound": "alu", "kernel": "hx_score_kernel", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                "frac": achieved / peak, "traffic": None,
+                "peak_source": "%d SMs x %d FP32 lanes x %.0f MHz x 2 flop (%s sm_max_mhz)" % (
+                    n_sm, FP32_LANES_PER_SM, sm_max_mhz, which),
+                "avg_launch_us": score_avg_ms * 1e3, "launches_timed": score_n,
+                "flop_per_candidate": 2,
+                "time_share": {k: v[0] / max(total_ms, 1e-9) for k, v in kt.items()}}
+
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        n_b = 8
+        cand, dt = oracle_chunks(make_workload("sweep"), n_b, with_dag=False)
+        cpu = {"value": cand / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+               "sample": "%d of 16 invocations (%d calls x 16384 pairs, top-4 + conflict pass), %.1f s" % (
+                   n_b, n_b * chunk, dt)}
+
+    h2d = n_calls * 16 + (P + 2 * D) * 4 + n_chunks * D * 4
+    d2h = n_calls * 8
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "sweep: %dx%d instances, %d ready calls in %d chunks of %d, top-%d lists + "
+                               "capacity-conflict pass with commit, horizons over %d nodes / %d workflows" % (
+                                   P, D, n_calls, n_chunks, chunk, wl.topk, wl.n_nodes, wl.n_workflows),
+                   "candidates_per_step": cand_per_step, "l2": "flushed between timed steps (256 MB write)",
+                   "seed": wl.seed, "score_mode": "ratio"},
+        "schedule_latency": {"batch_calls": chunk, "p50_us": float(np.percentile(chunk_us, 50)),
+                             "p95_us": float(np.percentile(chunk_us, 95)),
+                             "what": "load refresh + hx_schedule_batch (scoring, top-4, conflict pass, commit) per "
+                                     "ready batch, CUDA events"},
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "what": "hx_schedule_batch_host per chunk from pinned host memory, wall clock"},
+        "gpu_launches": int(launches), "kernel_ms_per_step": {k: v[0] / args.steps for k, v in kt.items()},
+        "device_status": status, "roofline": roofline, "cpu_baseline": cpu, "clocks": clocks,
+    }
+    print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -190,6 +190,16 @@ int hx_get_topk(hx_cluster* h, const int32_t** pairs, const float** costs, const
  * e.g. HX_ERR_TIMEOUT from a bounded wait).  Synchronises `stream`. */
 int hx_get_status(hx_cluster* h, int* status, void* stream);
 
+/* Tracing aid (the paper reports scheduler time per invocation, Section 7.7):
+ * while enabled, each kernel family the library enqueues is bracketed by a pair
+ * of CUDA events on the caller's stream.  Families: 0 = scoring kernel,
+ * 1 = capacity-conflict pass (all its kernels), 2 = horizon kernels.
+ * hx_read_kernel_timing waits for the recorded events, writes the summed
+ * device time in milliseconds and the number of bracketed enqueues per family
+ * (arrays of 3) since the previous read, and resets the record. */
+int hx_enable_kernel_timing(hx_cluster* h, int enable);
+int hx_read_kernel_timing(hx_cluster* h, float* ms, int* launches);
+
 /* Message of the last error on this handle ("" if none); with h = NULL, the
  * message of the last failed hx_cluster_create of the calling thread. */
 const char* hx_last_error(const hx_cluster* h);

@@ -58,6 +58,8 @@ def _load():
         "hx_schedule_batch_host": [vp, vp, ci, vp, vp, vp],
         "hx_get_topk": [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp)],
         "hx_get_status": [vp, C.POINTER(ci), vp],
+        "hx_enable_kernel_timing": [vp, ci],
+        "hx_read_kernel_timing": [vp, C.POINTER(C.c_float), C.POINTER(ci)],
     }
     for name, args in sig.items():
         f = getattr(lib, name)
@@ -171,6 +173,17 @@ def hx_get_status(h, stream=0):
     return s.value
 
 
+def hx_enable_kernel_timing(h, enable=True):
+    _check(_lib.hx_enable_kernel_timing(h, int(bool(enable))), h)
+
+
+def hx_read_kernel_timing(h):
+    """Returns {family: (milliseconds, enqueues)} for scoring, conflict, horizon."""
+    ms = (C.c_float * 3)(); n = (C.c_int * 3)()
+    _check(_lib.hx_read_kernel_timing(h, ms, n), h)
+    return {name: (float(ms[i]), int(n[i])) for i, name in enumerate(("scoring", "conflict", "horizon"))}
+
+
 def hx_last_error(h=None):
     return _lib.hx_last_error(h).decode()
 
@@ -278,6 +291,12 @@ class Cluster:
 
     def status(self):
         return hx_get_status(self.h, self._stream())
+
+    def enable_kernel_timing(self, enable=True):
+        hx_enable_kernel_timing(self.h, enable)
+
+    def read_kernel_timing(self):
+        return hx_read_kernel_timing(self.h)
 
     def launch_count(self):
         return hx_launch_count(self.h)

@@ -32,6 +32,11 @@ struct hx_cluster {
     hx_options opts{HX_MODE_COMPLETION, 0, 0, 0, 1.5f};
     std::string err;
     long long launches = 0;
+    // optional per-kernel-family device timing
+    struct Span { int family; cudaEvent_t a, b; };
+    bool timing = false;
+    std::vector<Span> spans;            // recorded since the last read
+    std::vector<Span> spare;            // events ready for reuse
 };
 
 namespace {
@@ -80,6 +85,23 @@ bool good_rate(float x) { return std::isfinite(x) && x > 0.0f; }
 bool good_load(float x) { return std::isfinite(x) && x >= 0.0f; }
 
 #define HX_TRY(call, what) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return fail_cuda(h, e_, what); } while (0)
+
+// Brackets the launches of one kernel family with events while timing is enabled.
+struct SpanGuard {
+    hx_cluster* h; cudaStream_t s; hx_cluster::Span sp{}; bool on = false;
+    SpanGuard(hx_cluster* h_, int family, cudaStream_t s_) : h(h_), s(s_) {
+        if (!h->timing) return;
+        if (!h->spare.empty()) { sp = h->spare.back(); h->spare.pop_back(); }
+        else if (cudaEventCreate(&sp.a) != cudaSuccess || cudaEventCreate(&sp.b) != cudaSuccess) return;
+        sp.family = family;
+        on = cudaEventRecord(sp.a, s) == cudaSuccess;
+    }
+    ~SpanGuard() {
+        if (!on) return;
+        cudaEventRecord(sp.b, s);
+        h->spans.push_back(sp);
+    }
+};
 
 int ensure_topk(hx_cluster* h, int n_calls, int K) {
     if (h->tk.cap_calls >= n_calls && h->tk.K == K) return HX_OK;
@@ -239,6 +261,8 @@ int hx_cluster_destroy(hx_cluster* h) {
     if (h->st_calls) cudaFree(h->st_calls);
     if (h->st_assign) cudaFree(h->st_assign);
     if (h->st_cost) cudaFree(h->st_cost);
+    for (auto* v : {&h->spans, &h->spare})
+        for (auto& sp : *v) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
     delete h;
     return HX_OK;
 }
@@ -382,8 +406,11 @@ int hx_critical_path(hx_cluster* h, void* stream) {
     if (!h) return HX_ERR_INVALID_ARG;
     if (!h->dag_uploaded) return fail(h, HX_ERR_NOT_READY, "no forest uploaded");
     DeviceGuard guard(h->device);
-    HX_TRY(hx_launch_cpath(h->forest, h->classes.data(), (int)h->classes.size(),
-                           static_cast<cudaStream_t>(stream), &h->launches), "horizon kernels");
+    {
+        SpanGuard span(h, 2, static_cast<cudaStream_t>(stream));
+        HX_TRY(hx_launch_cpath(h->forest, h->classes.data(), (int)h->classes.size(),
+                               static_cast<cudaStream_t>(stream), &h->launches), "horizon kernels");
+    }
     h->cp_ready = true;
     return HX_OK;
 }
@@ -432,9 +459,14 @@ int hx_schedule_batch(hx_cluster* h, const hx_call* calls, int n_calls, int32_t*
     HxTopkBufs tk = h->tk;
     tk.K = o.topk;
     ScoreLaunch sl{calls, n_calls, out_assign, out_cost, o.score_mode, o.flags, o.topk, o.alpha};
-    HX_TRY(hx_launch_score(h->tab, dag, tk, sl, h->n_sm, h->max_smem, h->status, s, &h->launches), "scoring kernel");
-    if (o.topk > 0)
+    {
+        SpanGuard span(h, 0, s);
+        HX_TRY(hx_launch_score(h->tab, dag, tk, sl, h->n_sm, h->max_smem, h->status, s, &h->launches), "scoring kernel");
+    }
+    if (o.topk > 0) {
+        SpanGuard span(h, 1, s);
         HX_TRY(hx_launch_conflict(h->tab, tk, n_calls, o.commit, out_assign, h->status, s, &h->launches), "conflict pass");
+    }
     return HX_OK;
 }
 
@@ -482,6 +514,27 @@ int hx_get_status(hx_cluster* h, int* status, void* stream) {
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     HX_TRY(cudaMemcpyAsync(status, h->status, sizeof(int), cudaMemcpyDeviceToHost, s), "read status");
     HX_TRY(cudaStreamSynchronize(s), "cudaStreamSynchronize");
+    return HX_OK;
+}
+
+int hx_enable_kernel_timing(hx_cluster* h, int enable) {
+    if (!h) return HX_ERR_INVALID_ARG;
+    h->timing = enable != 0;
+    return HX_OK;
+}
+
+int hx_read_kernel_timing(hx_cluster* h, float* ms, int* launches) {
+    if (!h || !ms || !launches) return HX_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    for (int k = 0; k < 3; ++k) { ms[k] = 0.f; launches[k] = 0; }
+    for (auto& sp : h->spans) {
+        HX_TRY(cudaEventSynchronize(sp.b), "cudaEventSynchronize");
+        float t = 0.f;
+        HX_TRY(cudaEventElapsedTime(&t, sp.a, sp.b), "cudaEventElapsedTime");
+        ms[sp.family] += t; ++launches[sp.family];
+        h->spare.push_back(sp);
+    }
+    h->spans.clear();
     return HX_OK;
 }
 
