@@ -8,28 +8,36 @@
 // whose decode instance still has kv_free >= m(c); that subtracts m(c) from the
 // instance and adds the call's prefill time to the chosen prefill queue.
 //
-// Parallel form with identical results: the only shared state a decision reads
-// is the free capacity of one decode instance, so every decode instance is
-// owned by one thread that walks, in visiting order, the list of (call, k)
-// slots naming it.  A slot (c, k) can be decided as soon as call c is known to
-// have failed on its candidates 0..k-1; until then the owner waits, and since
-// the most urgent undecided call is always at the head of the list of the
-// instance it is pending on, some thread can always advance.  Prefill queues
-// are updated afterwards by summing, per prefill instance, the prefill times of
-// the calls it obtained in visiting order (binary32 addition is not
-// associative, so the order is part of the definition).
-//
-// Ordering without a global sort: slots are bucketed per decode instance
-// (counting pass fused into the scoring kernel, scatter here), and each bucket
-// is ordered by counting, for every entry, the entries of the same bucket that
-// precede it; keys (prio, call) are unique inside a bucket.
+// Parallel form with identical results:
+//  1. hx_order_bins_kernel / hx_order_rank_kernel - visiting order of the batch.
+//     Calls are binned by the leading bits of the priority key (bins linear in
+//     the key bits between the batch minimum and maximum); inside a bin every
+//     key counts the keys that precede it.  Keys (prio, call) are unique.
+//  2. hx_conflict_kernel - optimistic windows over the visiting order.  A block
+//     takes the next W calls; every call picks the first candidate that fits the
+//     capacities committed so far, then checks it against the demand of the
+//     earlier calls of the same window that picked the same instance (ordered,
+//     segmented prefix sum).  All calls before the first one whose check fails
+//     have, by induction, made exactly the sequential decision: they commit, the
+//     window restarts at the failing call, which now sees the reduced capacity.
+//     Token counts are integer-valued and below 2^24, so the prefix sums are
+//     exact and equal to the sequential subtractions.  The first call of a
+//     window can never fail, so every step commits at least one call.
+//  3. hx_finish_kernel - writes the obtained pairs and gathers, in visiting
+//     order, (prefill instance, prefill time) of the calls that obtained one.
+//  4. hx_qsum_kernel - one thread per prefill instance adds its prefill times in
+//     visiting order (binary32 addition is not associative, so the order is
+//     part of the definition).
 #include "hx_internal.h"
 
 namespace {
 
 typedef unsigned long long u64;
 
-__device__ __forceinline__ u64 key_of(unsigned hi, unsigned lo) { return ((u64)hi << 32) | lo; }
+constexpr int kBins = 2048;
+constexpr int kWin = 256;          // calls per optimistic window (= block size of the pass)
+constexpr int kCache = 2048;       // calls staged in shared memory ahead of the window
+constexpr unsigned kNone = 0xFFu;  // no candidate taken
 
 // Exclusive prefix sum of n counters into shared memory, by the whole block
 // (blockDim a multiple of 32).  base gets n + 1 entries, tmp needs 33.
@@ -62,140 +70,159 @@ __device__ void block_exclusive_scan(const unsigned* cnt, int n, unsigned* base,
     __syncthreads();
 }
 
-// Scatter every valid (call, k) slot into the segment of its decode instance.
-__global__ void hx_dscatter_kernel(HxTopkBufs tk, int n_calls, int D) {
-    extern __shared__ unsigned sm[];
-    unsigned* base = sm;            // D + 1
-    unsigned* tmp = sm + D + 1;     // 33
-    block_exclusive_scan(tk.dcount, D, base, tmp);
-    const int K = tk.K;
-    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n_calls * K; i += gridDim.x * blockDim.x) {
-        const int pr = tk.pair[i];
-        if (pr < 0) continue;
-        const int c = i / K, k = i - c * K, d = pr % D;
-        const unsigned pos = base[d] + atomicAdd(&tk.dcursor[d], 1u);
-        tk.dflat[pos] = make_uint4(~__float_as_uint(tk.prio[c]), (unsigned)c, (unsigned)k, __float_as_uint(tk.mtok[c]));
-    }
-}
-
-// Order every decode segment: position = number of entries of the segment with a smaller key.
-__global__ void hx_drank_kernel(HxTopkBufs tk, int D) {
-    extern __shared__ unsigned sm[];
-    unsigned* base = sm;
-    unsigned* tmp = sm + D + 1;
-    block_exclusive_scan(tk.dcount, D, base, tmp);
-    const unsigned total = base[D];
-    for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
-        int lo = 0, hi = D;                       // segment d with base[d] <= i < base[d + 1]
-        while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (base[mid] <= i) lo = mid; else hi = mid; }
-        const unsigned b0 = base[lo], b1 = base[lo + 1];
-        const uint4 me = tk.dflat[i];
-        const u64 key = key_of(me.x, me.y);
-        unsigned rank = 0;
-        for (unsigned j = b0; j < b1; ++j) {
-            const uint2 o = __ldg(reinterpret_cast<const uint2*>(tk.dflat + j));
-            rank += key_of(o.x, o.y) < key;
-        }
-        tk.dsorted[b0 + rank] = make_uint2(me.y | (me.z << 24), me.w);
-    }
-}
-
-// One thread per decode instance walks its ordered slot list.  state[c] holds
-// the index of the candidate call c is pending on, or 0xFF once it has a pair.
-// A wait never blocks: a thread that cannot decide its head slot simply retries
-// in the next round, and the number of rounds is bounded.
-__global__ void hx_conflict_kernel(HxTopkBufs tk, HxTables t, int n_calls, int commit,
-                                   int32_t* out_assign, int* status, int max_rounds) {
-    extern __shared__ unsigned sm[];
-    const int D = t.D, K = tk.K;
-    unsigned* base = sm;                                        // D + 1
-    unsigned* tmp = sm + D + 1;                                 // 33
-    volatile unsigned char* state = reinterpret_cast<volatile unsigned char*>(sm + D + 1 + 33);
-    block_exclusive_scan(tk.dcount, D, base, tmp);
-    for (int c = threadIdx.x; c < n_calls; c += blockDim.x) state[c] = 0;
+// 1a. Bin the priority keys: one block.  obase receives the kBins + 1 bin bounds, the smallest
+// key and the shift that maps a key to its bin.
+__global__ void __launch_bounds__(1024) hx_order_bins_kernel(HxTopkBufs tk, int n) {
+    __shared__ unsigned hist[kBins], base[kBins + 1], tmp[33], lohi[2];
+    const int tid = threadIdx.x;
+    for (int i = tid; i < kBins; i += blockDim.x) hist[i] = 0;
+    if (tid == 0) { lohi[0] = 0xFFFFFFFFu; lohi[1] = 0u; }
     __syncthreads();
-    const int d = threadIdx.x;
-    const bool own = d < D;
-    unsigned pos = own ? base[d] : 0;
-    const unsigned end = own ? base[d + 1] : 0;
-    float free_tok = own ? t.freeD[d] : 0.f;
-    int rounds = 0;
-    for (;;) {
-        // take every decidable slot at the head of the list, stop at the first undecidable one
-        while (pos < end) {
-            const uint2 e = tk.dsorted[pos];
-            const unsigned c = e.x & 0xFFFFFFu, k = e.x >> 24;
-            const unsigned s = state[c];
-            if (s < k) break;                                   // call still pending on an earlier candidate
-            if (s == k) {
-                const float m = __uint_as_float(e.y);
-                if (free_tok >= m) {
-                    free_tok = __fsub_rn(free_tok, m);
-                    const int pr = tk.pair[(size_t)c * K + k];
-                    out_assign[c] = pr;
-                    const int p = pr / D;
-                    atomicAdd(&tk.pcount[p], 1u);
-                    const unsigned a = atomicAdd(tk.n_acc, 1u);
-                    tk.accflat[a] = make_uint4(~__float_as_uint(tk.prio[c]), c, (unsigned)p,
-                                               __float_as_uint(tk.tpre[(size_t)c * K + k]));
-                    state[c] = 0xFF;
-                } else {
-                    state[c] = (unsigned char)(k + 1);
-                }
-            }
-            ++pos;
-        }
-        const int done = pos >= end;
-        if (__syncthreads_and(done)) break;
-        if (++rounds > max_rounds) {                            // cannot happen for a consistent list
-            if (threadIdx.x == 0) atomicExch(status, HX_ERR_TIMEOUT);
-            break;
-        }
+    unsigned lo = 0xFFFFFFFFu, hi = 0u;
+#pragma unroll 4
+    for (int c = tid; c < n; c += blockDim.x) {
+        const unsigned key = ~__float_as_uint(__ldg(tk.prio + c));   // larger priority = smaller key
+        lo = min(lo, key); hi = max(hi, key);
     }
-    if (own && commit) t.freeD[d] = free_tok;
-}
-
-// Bucket the obtained pairs per prefill instance.
-__global__ void hx_pscatter_kernel(HxTopkBufs tk, int P) {
-    extern __shared__ unsigned sm[];
-    unsigned* base = sm;
-    unsigned* tmp = sm + P + 1;
-    block_exclusive_scan(tk.pcount, P, base, tmp);
-    const unsigned total = *tk.n_acc;
-    for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
-        const uint4 e = tk.accflat[i];
-        const unsigned pos = base[e.z] + atomicAdd(&tk.pcursor[e.z], 1u);
-        tk.pseg[pos] = e;
+    lo = __reduce_min_sync(0xffffffffu, lo); hi = __reduce_max_sync(0xffffffffu, hi);
+    if ((tid & 31) == 0) { atomicMin(&lohi[0], lo); atomicMax(&lohi[1], hi); }
+    __syncthreads();
+    lo = lohi[0];
+    const unsigned span = lohi[1] - lo;
+    int shift = 0;
+    while ((span >> shift) >= (unsigned)kBins) ++shift;
+#pragma unroll 4
+    for (int c = tid; c < n; c += blockDim.x)
+        atomicAdd(&hist[(~__float_as_uint(__ldg(tk.prio + c)) - lo) >> shift], 1u);
+    __syncthreads();
+    block_exclusive_scan(hist, kBins, base, tmp);
+    for (int i = tid; i <= kBins; i += blockDim.x) tk.obase[i] = base[i];
+    if (tid == 0) { tk.obase[kBins + 1] = lo; tk.obase[kBins + 2] = (unsigned)shift; }
+    for (int i = tid; i < kBins; i += blockDim.x) hist[i] = 0;     // now the bin cursors
+    __syncthreads();
+#pragma unroll 4
+    for (int c = tid; c < n; c += blockDim.x) {
+        const unsigned key = ~__float_as_uint(__ldg(tk.prio + c));
+        const unsigned bin = (key - lo) >> shift;
+        tk.okey[base[bin] + atomicAdd(&hist[bin], 1u)] = ((u64)key << 32) | (unsigned)c;
     }
 }
 
-// Order each prefill bucket by visiting order and add the prefill times to the
-// queue in that order.
-__global__ void hx_qupdate_kernel(HxTopkBufs tk, HxTables t, int P) {
+// 1b. Rank inside the bins and gather the per-call data in visiting order.
+__global__ void hx_order_rank_kernel(HxTopkBufs tk, int n) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const int K = tk.K;
+    const unsigned lo = tk.obase[kBins + 1], shift = tk.obase[kBins + 2];
+    const u64 key = tk.okey[i];
+    const unsigned bin = ((unsigned)(key >> 32) - lo) >> shift;
+    const unsigned b0 = tk.obase[bin], b1 = tk.obase[bin + 1];
+    unsigned rank = b0;
+    for (unsigned j = b0; j < b1; ++j) rank += __ldg(tk.okey + j) < key;
+    const unsigned c = (unsigned)key;
+    tk.ocall[rank] = c;
+    tk.om[rank] = tk.mtok[c];
+    for (int k = 0; k < K; ++k) tk.od[(size_t)rank * K + k] = tk.dsel[(size_t)c * K + k];
+}
+
+// 2. The pass itself: one block of kWin threads.
+__global__ void __launch_bounds__(kWin) hx_conflict_kernel(HxTopkBufs tk, HxTables t, int n, int commit) {
     extern __shared__ unsigned sm[];
-    unsigned* base = sm;
-    unsigned* tmp = sm + P + 1;
-    block_exclusive_scan(tk.pcount, P, base, tmp);
-    for (int p = blockIdx.x; p < P; p += gridDim.x) {
-        const unsigned b0 = base[p], b1 = base[p + 1];
-        for (unsigned i = b0 + threadIdx.x; i < b1; i += blockDim.x) {
-            const uint4 me = tk.pseg[i];
-            const u64 key = key_of(me.x, me.y);
-            unsigned rank = 0;
-            for (unsigned j = b0; j < b1; ++j) {
-                const uint2 o = __ldg(reinterpret_cast<const uint2*>(tk.pseg + j));
-                rank += key_of(o.x, o.y) < key;
+    constexpr int NW = kWin / 32;
+    const int D = t.D, K = tk.K;
+    float* free_s = reinterpret_cast<float*>(sm);               // [D] capacity left after the commits so far
+    float* wtot = free_s + D;                                   // [NW][D] demand per warp and instance
+    float* cm = wtot + NW * D;                                  // [kCache] demands of the staged calls
+    uint16_t* cd = reinterpret_cast<uint16_t*>(cm + kCache);    // [kCache][K] their candidate instances
+    __shared__ int first_fail, n_acc_s, cache_lo;
+    __shared__ unsigned wacc[NW + 1];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    for (int d = tid; d < D; d += kWin) free_s[d] = t.freeD[d];
+    if (tid == 0) { n_acc_s = 0; cache_lo = -kCache; }
+    __syncthreads();
+    int pos = 0;
+    while (pos < n) {
+        if (pos + kWin > cache_lo + kCache) {                   // stage the next calls (one round trip)
+            __syncthreads();
+            for (int i = tid; i < kCache; i += kWin) {
+                const int r = pos + i;
+                cm[i] = r < n ? tk.om[r] : 0.f;
+                for (int k = 0; k < K; ++k) cd[i * K + k] = r < n ? tk.od[(size_t)r * K + k] : (uint16_t)0xFFFF;
             }
-            tk.psorted[b0 + rank] = __uint_as_float(me.w);
+            if (tid == 0) cache_lo = pos;
+            __syncthreads();
+        }
+        const int r = pos + tid, ci = r - cache_lo;
+        const bool active = r < n;
+        const float m = active ? cm[ci] : 0.f;
+        // first candidate that fits the committed capacities
+        unsigned kt = kNone; int dt = -1;
+        if (active)
+            for (int k = K - 1; k >= 0; --k) {
+                const unsigned d = cd[ci * K + k];
+                if (d != 0xFFFFu && free_s[d] >= m) { kt = k; dt = (int)d; }
+            }
+        for (int i = tid; i < NW * D; i += kWin) wtot[i] = 0.f;
+        if (tid == 0) first_fail = kWin;
+        // demand of the earlier lanes of this warp that picked the same instance
+        const unsigned peers = __match_any_sync(0xffffffffu, dt);
+        float cum = 0.f;
+        for (int j = 0; j < 31; ++j) {
+            const float mj = __shfl_sync(0xffffffffu, m, j);
+            if (j < lane && ((peers >> j) & 1u)) cum = __fadd_rn(cum, mj);
         }
         __syncthreads();
-        if (threadIdx.x == 0 && b1 > b0) {
-            float q = t.qP[p];
-            for (unsigned i = b0; i < b1; ++i) q = __fadd_rn(q, __ldcg(&tk.psorted[i]));
-            t.qP[p] = q;
+        if (dt >= 0 && (peers >> lane) <= 1u) wtot[warp * D + dt] = __fadd_rn(cum, m);   // last peer: warp total
+        __syncthreads();
+        if (dt >= 0) for (int w = 0; w < warp; ++w) cum = __fadd_rn(cum, wtot[w * D + dt]);
+        if (dt >= 0 && __fadd_rn(cum, m) > free_s[dt]) atomicMin(&first_fail, tid);
+        __syncthreads();
+        const int f = first_fail;                               // calls before f decided as the sequential pass would
+        const bool done = active && tid < f;
+        const bool acc = done && dt >= 0;
+        if (acc) atomicAdd(&free_s[dt], -m);                    // exact: integer-valued operands
+        // obtained pairs, appended in visiting order
+        const unsigned b = __ballot_sync(0xffffffffu, acc);
+        if (lane == 0) wacc[warp] = __popc(b);
+        __syncthreads();
+        if (acc) {
+            unsigned off = n_acc_s + __popc(b & ((1u << lane) - 1u));
+            for (int w = 0; w < warp; ++w) off += wacc[w];
+            tk.acc_rk[off] = (unsigned)r | (kt << 24);
         }
         __syncthreads();
+        if (tid == 0) { int a = 0; for (int w = 0; w < NW; ++w) a += wacc[w]; n_acc_s += a; }
+        pos += f < kWin ? f : kWin;
     }
+    __syncthreads();
+    if (tid == 0) *tk.n_acc = (unsigned)n_acc_s;
+    if (commit) for (int d = tid; d < D; d += kWin) t.freeD[d] = free_s[d];
+}
+
+// 3. Publish the obtained pairs; gather prefill instance and prefill time in visiting order.
+__global__ void hx_finish_kernel(HxTopkBufs tk, int D, int32_t* out_assign) {
+    const unsigned i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= *tk.n_acc) return;
+    const unsigned rk = tk.acc_rk[i], r = rk & 0xFFFFFFu, k = rk >> 24;
+    const unsigned c = tk.ocall[r];
+    const int pr = tk.pair[(size_t)c * tk.K + k];
+    out_assign[c] = pr;
+    tk.acc_p[i] = pr / D;
+    tk.acc_t[i] = tk.tpre[(size_t)c * tk.K + k];
+}
+
+// 4. Prefill queues: thread p adds, in visiting order, the prefill times of the calls that obtained p.
+__global__ void hx_qsum_kernel(HxTopkBufs tk, HxTables t) {
+    const int p = blockIdx.x * blockDim.x + threadIdx.x;
+    const unsigned na = *tk.n_acc;
+    float q = p < t.P ? t.qP[p] : 0.f;
+#pragma unroll 8
+    for (unsigned i = 0; i < na; ++i) {
+        const int pi = __ldg(tk.acc_p + i);
+        const float ti = __ldg(tk.acc_t + i);
+        if (pi == p) q = __fadd_rn(q, ti);
+    }
+    if (p < t.P) t.qP[p] = q;
 }
 
 }  // namespace
@@ -203,26 +230,21 @@ __global__ void hx_qupdate_kernel(HxTopkBufs tk, HxTables t, int P) {
 cudaError_t hx_launch_conflict(const HxTables& t, const HxTopkBufs& tk, int n_calls, int commit,
                                int32_t* out_assign, int* status, cudaStream_t stream,
                                long long* launches) {
+    (void)status;
     const int D = t.D, P = t.P;
-    const size_t smD = (size_t)(D + 1 + 33) * 4, smP = (size_t)(P + 1 + 33) * 4;
-    const int nslots = n_calls * tk.K;
-    int grid = (nslots + 255) / 256; if (grid > 592) grid = 592;
-    hx_dscatter_kernel<<<grid, 256, smD, stream>>>(tk, n_calls, D);
-    hx_drank_kernel<<<grid, 256, smD, stream>>>(tk, D);
-    const int cthreads = (D + 31) / 32 * 32;
-    const size_t smC = smD + (size_t)((n_calls + 15) / 16 * 16);
+    hx_order_bins_kernel<<<1, 1024, 0, stream>>>(tk, n_calls);
+    hx_order_rank_kernel<<<(n_calls + 127) / 128, 128, 0, stream>>>(tk, n_calls);
+    const size_t smC = (size_t)(D + (kWin / 32) * D + kCache) * 4 + (size_t)kCache * tk.K * 2;
     if (smC > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(hx_conflict_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smC);
         if (e != cudaSuccess) return e;
     }
-    // every round decides at least one slot, so n_calls * K + 2 rounds always suffice
-    hx_conflict_kernel<<<1, cthreads, smC, stream>>>(tk, t, n_calls, commit, out_assign, status, nslots + 2);
-    *launches += 3;
+    hx_conflict_kernel<<<1, kWin, smC, stream>>>(tk, t, n_calls, commit);
+    hx_finish_kernel<<<(n_calls + 255) / 256, 256, 0, stream>>>(tk, D, out_assign);
+    *launches += 4;
     if (commit) {
-        int gp = (n_calls + 255) / 256; if (gp > 592) gp = 592;
-        hx_pscatter_kernel<<<gp, 256, smP, stream>>>(tk, P);
-        hx_qupdate_kernel<<<P < 592 ? P : 592, 128, smP, stream>>>(tk, t, P);
-        *launches += 2;
+        hx_qsum_kernel<<<(P + 31) / 32, 32, 0, stream>>>(tk, t);
+        *launches += 1;
     }
     return cudaGetLastError();
 }

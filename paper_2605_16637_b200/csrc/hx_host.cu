@@ -26,7 +26,6 @@ struct hx_cluster {
     std::vector<HxCpClass> classes;
     // top-K
     HxTopkBufs tk{};
-    size_t counter_bytes = 0;
     // staging for the host-buffer entry point
     hx_call* st_calls = nullptr; int32_t* st_assign = nullptr; float* st_cost = nullptr; int st_cap = 0;
     hx_options opts{HX_MODE_COMPLETION, 0, 0, 0, 1.5f};
@@ -114,19 +113,18 @@ int ensure_topk(hx_cluster* h, int n_calls, int K) {
     HX_TRY(dev_alloc(h->tk_allocs, &b.pair, cap * K), "alloc top-K");
     HX_TRY(dev_alloc(h->tk_allocs, &b.cost, cap * K), "alloc top-K");
     HX_TRY(dev_alloc(h->tk_allocs, &b.tpre, cap * K), "alloc top-K");
+    HX_TRY(dev_alloc(h->tk_allocs, &b.dsel, cap * K), "alloc top-K");
     HX_TRY(dev_alloc(h->tk_allocs, &b.prio, cap), "alloc top-K");
     HX_TRY(dev_alloc(h->tk_allocs, &b.mtok, cap), "alloc top-K");
-    const size_t ncnt = 2 * (size_t)h->D + 2 * (size_t)h->P + 1;
-    unsigned int* cnt;
-    HX_TRY(dev_alloc(h->tk_allocs, &cnt, ncnt), "alloc counters");
-    b.dcount = cnt; b.dcursor = cnt + h->D; b.pcount = cnt + 2 * h->D; b.pcursor = b.pcount + h->P;
-    b.n_acc = b.pcursor + h->P;
-    h->counter_bytes = ncnt * sizeof(unsigned int);
-    HX_TRY(dev_alloc(h->tk_allocs, &b.dflat, cap * K), "alloc slots");
-    HX_TRY(dev_alloc(h->tk_allocs, &b.dsorted, cap * K), "alloc slots");
-    HX_TRY(dev_alloc(h->tk_allocs, &b.accflat, cap), "alloc slots");
-    HX_TRY(dev_alloc(h->tk_allocs, &b.pseg, cap), "alloc slots");
-    HX_TRY(dev_alloc(h->tk_allocs, &b.psorted, cap), "alloc slots");
+    HX_TRY(dev_alloc(h->tk_allocs, &b.okey, cap), "alloc order");
+    HX_TRY(dev_alloc(h->tk_allocs, &b.obase, (size_t)2048 + 3), "alloc order");
+    HX_TRY(dev_alloc(h->tk_allocs, &b.ocall, cap), "alloc order");
+    HX_TRY(dev_alloc(h->tk_allocs, &b.om, cap), "alloc order");
+    HX_TRY(dev_alloc(h->tk_allocs, &b.od, cap * K), "alloc order");
+    HX_TRY(dev_alloc(h->tk_allocs, &b.n_acc, (size_t)1), "alloc outcome");
+    HX_TRY(dev_alloc(h->tk_allocs, &b.acc_rk, cap), "alloc outcome");
+    HX_TRY(dev_alloc(h->tk_allocs, &b.acc_p, cap), "alloc outcome");
+    HX_TRY(dev_alloc(h->tk_allocs, &b.acc_t, cap), "alloc outcome");
     b.cap_calls = (int)cap;
     h->tk = b;
     return HX_OK;
@@ -451,7 +449,6 @@ int hx_schedule_batch(hx_cluster* h, const hx_call* calls, int n_calls, int32_t*
     if (o.topk > 0) {
         int rc = ensure_topk(h, n_calls, o.topk);
         if (rc != HX_OK) return rc;
-        HX_TRY(cudaMemsetAsync(h->tk.dcount, 0, h->counter_bytes, s), "cudaMemsetAsync(counters)");
     }
     HxDagView dag{};
     if (!(o.flags & HX_FLAG_NO_DAG))

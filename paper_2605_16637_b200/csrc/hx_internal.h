@@ -41,28 +41,29 @@ struct HxDagView {
     uint32_t n_nodes, n_workflows;
 };
 
-// Per-batch buffers of the top-K list and of the capacity-conflict pass.  All
-// sizes are linear in the batch: slots are kept in flat arrays segmented by
-// decode (or prefill) instance, segment bounds come from the counters.
+// Per-batch buffers of the top-K list and of the capacity-conflict pass; all
+// sizes are linear in the batch.  "rank" = position of a call in visiting order.
 struct HxTopkBufs {
     int K;
     int cap_calls;             // capacity (calls) of the per-call arrays
+    // written by the scoring kernel, indexed by call
     int32_t* pair;             // [cap][K]
     float* cost;               // [cap][K]
     float* tpre;               // [cap][K] prefill time on the prefill instance of slot k
+    uint16_t* dsel;            // [cap][K] decode instance of slot k, 0xFFFF = unused
     float* prio;               // [cap]
     float* mtok;               // [cap]
-    // counters, zeroed before every batch (one contiguous allocation)
-    unsigned int* dcount;      // [D] valid slots naming decode instance d
-    unsigned int* dcursor;     // [D]
-    unsigned int* pcount;      // [P] calls that obtained prefill instance p
-    unsigned int* pcursor;     // [P]
-    unsigned int* n_acc;       // [1] calls that obtained a pair
-    uint4* dflat;              // [cap*K] {~prio bits, call, k, m bits}, grouped by decode instance
-    uint2* dsorted;            // [cap*K] {call | k << 24, m bits}, each group in visiting order
-    uint4* accflat;            // [cap]   {~prio bits, call, p, tpre bits} in order of acceptance
-    uint4* pseg;               // [cap]   same entries grouped by prefill instance
-    float* psorted;            // [cap]   prefill times, each group in visiting order
+    // visiting order
+    unsigned long long* okey;  // [cap] keys grouped by bin
+    unsigned int* obase;       // [2048 + 3] bin bounds, smallest key, key-to-bin shift
+    unsigned int* ocall;       // [cap] call of each rank
+    float* om;                 // [cap] demand of each rank
+    uint16_t* od;              // [cap][K] decode instances of each rank's slots
+    // outcome: calls that obtained a pair, in visiting order
+    unsigned int* n_acc;       // [1]
+    unsigned int* acc_rk;      // [cap] rank | k << 24
+    int* acc_p;                // [cap] prefill instance obtained
+    float* acc_t;              // [cap] prefill time added to that instance
 };
 
 struct ScoreLaunch {

@@ -37,9 +37,9 @@ struct ScoreParams {
     int Dpad;            // decode columns covered by the block (multiple of 8*LD)
     int PC;              // prefill chunk length (multiple of 4)
     int nChunks;
-    int PS;              // shared-memory row stride of LT and A (PC + 4 or PC + 8)
     int FS;              // row stride of the per-call finish times (Dpad + 4)
-    int offA, offCall, offInst;   // byte offsets into dynamic shared memory (LT at 0)
+    int offA, offF, offCall, offInst;   // byte offsets into dynamic shared memory (LT at 0)
+    int resident;        // whole link table and the A tile stay in shared memory for the index recovery
 };
 
 __device__ __forceinline__ u64 fma2(u64 a, u64 b, u64 c) {
@@ -112,8 +112,50 @@ __device__ __forceinline__ int group_rescan(const HxTables& T, const float* qPs,
     return best;
 }
 
-template <int TC, int LD>
-__global__ void __launch_bounds__(256, 1) hx_score_kernel(const __grid_constant__ ScoreParams prm) {
+// Minimum of a row together with its lowest column and the number of columns attaining it.
+__device__ __forceinline__ void group_min(const float* frow, int nq, int t, unsigned gmask,
+                                          float& bv, int& bd, int& cnt) {
+    bv = HX_INF; bd = HX_NONE; cnt = 0;
+    for (int q = t; q < nq; q += 4) {
+        const float4 f = *reinterpret_cast<const float4*>(frow + 4 * q);
+        const float v[4] = {f.x, f.y, f.z, f.w};
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            if (v[u] < bv) { bv = v[u]; bd = 4 * q + u; cnt = 1; }
+            else if (v[u] == bv && bd != HX_NONE) ++cnt;
+        }
+    }
+#pragma unroll
+    for (int off = 1; off <= 2; off <<= 1) {
+        const float ov = __shfl_xor_sync(gmask, bv, off);
+        const int od = __shfl_xor_sync(gmask, bd, off);
+        const int oc = __shfl_xor_sync(gmask, cnt, off);
+        if (ov < bv) { bv = ov; bd = od; cnt = oc; }
+        else if (ov == bv) { bd = min(bd, od); cnt += oc; }
+    }
+}
+
+// Same as group_rescan with both operands resident in shared memory ([p/4][row] float4 layout).
+// The four lanes of the group take the four p of one 16-byte unit, so a step is one
+// conflict-free scalar load per operand.
+__device__ __forceinline__ int group_rescan_smem(const float* acol, int astride, const float* lcol, int lstride,
+                                                 int nq, float kvB, float qd, float Dd, float v, int t,
+                                                 unsigned gmask) {
+    int best = HX_NONE;
+    for (int q = nq - 1; q >= 0; --q) {
+        const float f = __fadd_rn(fmaxf(__fmaf_rn(kvB, lcol[q * lstride + t], acol[q * astride + t]), qd), Dd);
+        if (f == v) best = 4 * q + t;
+    }
+#pragma unroll
+    for (int off = 1; off <= 2; off <<= 1) best = min(best, __shfl_xor_sync(gmask, best, off));
+    return best;
+}
+
+// Thread tile: TC calls x TD decode columns.  A warp spans LD lanes along d and 32 / LD along
+// the calls; lanes interleave their rows so that the rows one instruction touches start in
+// different shared-memory banks.
+template <int TC, int TD, int LD>
+__global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const __grid_constant__ ScoreParams prm) {
     extern __shared__ __align__(16) unsigned char smem[];
     constexpr int LC = 32 / LD;
     const HxTables& T = prm.t;
@@ -122,11 +164,15 @@ __global__ void __launch_bounds__(256, 1) hx_score_kernel(const __grid_constant_
     const int warp = tid >> 5, lane = tid & 31;
     const int wd = warp % prm.WDn, wc = warp / prm.WDn;
     const int dg = lane % LD, cg = lane / LD;
-    const int PS = prm.PS, FS = prm.FS, PC = prm.PC, TCB = prm.TCB, Dpad = prm.Dpad;
+    const int FS = prm.FS, PC = prm.PC, TCB = prm.TCB, Dpad = prm.Dpad;
     const bool unloaded = prm.s.flags & HX_FLAG_UNLOADED;
+    const bool resident = prm.resident;
 
-    float* LTs = reinterpret_cast<float*>(smem);                  // [Dpad][PS]
-    float* As = reinterpret_cast<float*>(smem + prm.offA);        // [TCB][PS], later fin [TCB][FS]
+    // operand tiles are stored [p / 4][row] as 16-byte units: for a fixed p the rows a warp
+    // reads are contiguous (no bank conflicts, no padding) and their offsets are compile-time
+    float* LTs = reinterpret_cast<float*>(smem);                  // [PC/4][Dpad][4]
+    float* As = reinterpret_cast<float*>(smem + prm.offA);        // [PC/4][TCB][4]
+    float* Fs = reinterpret_cast<float*>(smem + prm.offF);        // [TCB][FS] (may alias As)
     float* kvBs = reinterpret_cast<float*>(smem + prm.offCall);   // [TCB]
     float* mtoks = kvBs + TCB;                                    // [TCB]
     float* tpres = mtoks + TCB;                                   // [TCB][G]
@@ -149,107 +195,103 @@ __global__ void __launch_bounds__(256, 1) hx_score_kernel(const __grid_constant_
     }
     auto load_LT = [&](int pc0) {
         const int nq = PC >> 2;
+#pragma unroll 4
         for (int idx = tid; idx < Dpad * nq; idx += nthr) {
-            const int d = idx / nq, q = idx - d * nq;
+            const int q = idx / Dpad, d = idx - q * Dpad;
             const int p = pc0 + 4 * q;
             float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
             if (d < D && p < Ppad) v = __ldg(reinterpret_cast<const float4*>(T.invLT + (size_t)d * Ppad + p));
-            *reinterpret_cast<float4*>(LTs + d * PS + 4 * q) = v;
+            *reinterpret_cast<float4*>(LTs + 4 * idx) = v;
         }
     };
     if (prm.nChunks == 1) load_LT(0);
-    __syncthreads();
 
     for (int tile = blockIdx.x; tile < prm.nTiles; tile += gridDim.x) {
         const int c0 = tile * TCB;
         const int nvalid = min(TCB, prm.s.n_calls - c0);
 
-        // per-call service times on every GPU class (roofline-style estimate, Section 4.2)
-        for (int c = tid; c < TCB; c += nthr) {
+        // per-call service times on every GPU class (roofline-style estimate, Section 4.2):
+        // one thread per (call, class)
+        for (int idx = tid; idx < TCB * G; idx += nthr) {
+            const int c = idx / G, g = idx - c * G;
             float n = 1.f, o = 1.f, phi = 0.f, omega = 0.f, kappa = 0.f;
             if (c < nvalid) {
                 const uint4 raw = __ldg(reinterpret_cast<const uint4*>(prm.s.calls) + c0 + c);
                 n = __uint_as_float(raw.z); o = __uint_as_float(raw.w);
-                if (raw.y < (unsigned)T.M) { phi = T.phi[raw.y]; omega = T.omega[raw.y]; kappa = T.kappa[raw.y]; }
+                if (raw.y < (unsigned)T.M) { phi = __ldg(T.phi + raw.y); omega = __ldg(T.omega + raw.y); kappa = __ldg(T.kappa + raw.y); }
             }
             const float kvB = __fmul_rn(n, kappa);
-            const float m = __fadd_rn(n, o);
             const float ctx = __fmaf_rn(0.5f, __fsub_rn(o, 1.0f), n);
             const float step = __fmaf_rn(kappa, ctx, omega);
-            const float nphi = __fmul_rn(n, phi), wkv = __fadd_rn(omega, kvB), ostep = __fmul_rn(o, step);
-            for (int g = 0; g < G; ++g) {
-                const float iF = T.invF[g], iB = T.invB[g];
-                tpres[c * G + g] = fmaxf(__fmul_rn(nphi, iF), __fmul_rn(wkv, iB));
-                tdecs[c * G + g] = __fmul_rn(ostep, iB);
-            }
-            kvBs[c] = kvB; mtoks[c] = m;
+            const float iF = __ldg(T.invF + g), iB = __ldg(T.invB + g);
+            tpres[idx] = fmaxf(__fmul_rn(__fmul_rn(n, phi), iF), __fmul_rn(__fadd_rn(omega, kvB), iB));
+            tdecs[idx] = __fmul_rn(__fmul_rn(o, step), iB);
+            if (g == 0) { kvBs[c] = kvB; mtoks[c] = __fadd_rn(n, o); }
         }
         __syncthreads();
 
-        float acc[TC][8];
+        float acc[TC][TD];
 #pragma unroll
         for (int i = 0; i < TC; ++i)
 #pragma unroll
-            for (int j = 0; j < 8; ++j) acc[i][j] = HX_INF;
+            for (int j = 0; j < TD; ++j) acc[i][j] = HX_INF;
         u64 kk[TC];
 #pragma unroll
         for (int i = 0; i < TC; ++i) {
             const float k = kvBs[wc * (TC * LC) + cg + LC * i];
             kk[i] = pack2(k, k);
         }
-        const float* Arow = As + (wc * (TC * LC) + cg) * PS;       // row i at + i * LC * PS
-        const float* Lrow = LTs + (wd * (8 * LD) + dg) * PS;       // row j at + j * LD * PS
-
         for (int ch = 0; ch < prm.nChunks; ++ch) {
             const int pc0 = ch * PC;
             if (prm.nChunks > 1) load_LT(pc0);
             {   // prefill finish times A[c][p] of this chunk
                 const int nq = PC >> 2;
                 for (int idx = tid; idx < TCB * nq; idx += nthr) {
-                    const int c = idx / nq, q = idx - c * nq;
+                    const int q = idx / TCB, c = idx - q * TCB;
                     const int p = pc0 + 4 * q;
                     float a[4];
 #pragma unroll
                     for (int u = 0; u < 4; ++u)
                         a[u] = (p + u < Ppad) ? __fadd_rn(qPs[p + u], tpres[c * G + typePs[p + u]]) : HX_INF;
-                    *reinterpret_cast<float4*>(As + c * PS + 4 * q) = make_float4(a[0], a[1], a[2], a[3]);
+                    *reinterpret_cast<float4*>(As + 4 * idx) = make_float4(a[0], a[1], a[2], a[3]);
                 }
             }
             __syncthreads();
+            const ulonglong2* ap = reinterpret_cast<const ulonglong2*>(As) + wc * (TC * LC) + cg;
+            const ulonglong2* lp = reinterpret_cast<const ulonglong2*>(LTs) + wd * (TD * LD) + dg;
 #pragma unroll 2
             for (int q = 0; q < (PC >> 2); ++q) {
-                ulonglong2 a[TC], l[8];
+                ulonglong2 a[TC], l[TD];
+#pragma unroll
+                for (int i = 0; i < TC; ++i) a[i] = ap[i * LC];
+#pragma unroll
+                for (int j = 0; j < TD; ++j) l[j] = lp[j * LD];
+                ap += TCB; lp += Dpad;
 #pragma unroll
                 for (int i = 0; i < TC; ++i)
-                    a[i] = *reinterpret_cast<const ulonglong2*>(Arow + i * LC * PS + 4 * q);
 #pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    l[j] = *reinterpret_cast<const ulonglong2*>(Lrow + j * LD * PS + 4 * q);
-#pragma unroll
-                for (int i = 0; i < TC; ++i)
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
+                    for (int j = 0; j < TD; ++j) {
                         float r0, r1, r2, r3;
                         unpack2(fma2(kk[i], l[j].x, a[i].x), r0, r1);
                         unpack2(fma2(kk[i], l[j].y, a[i].y), r2, r3);
                         acc[i][j] = min3(min3(acc[i][j], r0, r1), r2, r3);
                     }
             }
-            __syncthreads();
+            if (prm.nChunks > 1 || !resident) __syncthreads();
         }
 
         // clamp to the decode admission time and add the decode term; park the
-        // per-(call, d) finish times in shared memory (over the A tile)
+        // per-(call, d) finish times in shared memory
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const int d = wd * (8 * LD) + dg + LD * j;
+        for (int j = 0; j < TD; ++j) {
+            const int d = wd * (TD * LD) + dg + LD * j;
             const float qd = qDs[d], cap = capDs[d];
             const int ty = typeDs[d];
 #pragma unroll
             for (int i = 0; i < TC; ++i) {
                 const int c = wc * (TC * LC) + cg + LC * i;
                 const float Dd = (mtoks[c] <= cap) ? tdecs[c * G + ty] : HX_INF;
-                As[c * FS + d] = __fadd_rn(fmaxf(acc[i][j], qd), Dd);
+                Fs[c * FS + d] = __fadd_rn(fmaxf(acc[i][j], qd), Dd);
             }
         }
         __syncthreads();
@@ -262,31 +304,46 @@ __global__ void __launch_bounds__(256, 1) hx_score_kernel(const __grid_constant_
             const int c = cb + gid;
             const bool live = c < nvalid;                 // uniform inside the group
             const int cs = live ? c : 0;
-            const float* frow = As + cs * FS;
+            const float* frow = Fs + cs * FS;
             const float kvB = kvBs[cs], m = mtoks[cs];
             const float* tpre_c = tpres + cs * G;
-            float pv = -1.0f; int pd = -1;
-            float v0 = HX_INF; int jbest = HX_NONE;
-            int sel_pair[HX_MAX_TOPK]; float sel_cost[HX_MAX_TOPK], sel_tpre[HX_MAX_TOPK];
-#pragma unroll
-            for (int k = 0; k < HX_MAX_TOPK; ++k) { sel_pair[k] = -1; sel_cost[k] = HX_INF; sel_tpre[k] = 0.f; }
-            const int want = K > 0 ? K : 1;
-            for (int k = 0;; ++k) {
-                float v; int d;
-                group_next(frow, Dpad >> 2, t, gmask, pv, pd, v, d);
-                if (d == HX_NONE) break;                  // nothing (feasible) left
-                if (k == 0) v0 = v;
-                const bool tie = (K == 0) && (v == v0);   // the plain argmin orders ties by p first
-                if (k >= want && !tie) break;
+            auto rescan = [&](int d, float v) {
                 const float Dd = (m <= capDs[d]) ? tdecs[cs * G + typeDs[d]] : HX_INF;
-                const int p = group_rescan(T, qPs, typePs, tpre_c, kvB, qDs[d], Dd, d, v, t, gmask);
-                if (k < want) {
+                return resident
+                    ? group_rescan_smem(As + 4 * cs, 4 * TCB, LTs + 4 * d, 4 * Dpad, Ppad >> 2, kvB, qDs[d], Dd, v, t, gmask)
+                    : group_rescan(T, qPs, typePs, tpre_c, kvB, qDs[d], Dd, d, v, t, gmask);
+            };
+            float v0 = HX_INF; int jbest = HX_NONE;
+            int sel_pair[HX_MAX_TOPK], sel_d[HX_MAX_TOPK]; float sel_cost[HX_MAX_TOPK], sel_tpre[HX_MAX_TOPK];
+#pragma unroll
+            for (int k = 0; k < HX_MAX_TOPK; ++k) { sel_pair[k] = -1; sel_d[k] = 0; sel_cost[k] = HX_INF; sel_tpre[k] = 0.f; }
+            if (K == 0) {
+                // plain argmin: lowest p * D + d among all pairs attaining the minimum
+                int d0, ntie;
+                group_min(frow, Dpad >> 2, t, gmask, v0, d0, ntie);
+                if (d0 != HX_NONE) {
+                    jbest = rescan(d0, v0) * D + d0;
+                    float pv = v0; int pd = d0;
+                    for (int r = 1; r < ntie; ++r) {      // exact ties across decode instances
+                        float v; int d;
+                        group_next(frow, Dpad >> 2, t, gmask, pv, pd, v, d);
+                        jbest = min(jbest, rescan(d, v) * D + d);
+                        pv = v; pd = d;
+                    }
+                }
+            } else {
+                float pv = -1.0f; int pd = -1;
+                for (int k = 0; k < K; ++k) {
+                    float v; int d;
+                    group_next(frow, Dpad >> 2, t, gmask, pv, pd, v, d);
+                    if (d == HX_NONE) break;              // nothing (feasible) left
+                    if (k == 0) v0 = v;
+                    const int p = rescan(d, v);
 #pragma unroll
                     for (int k2 = 0; k2 < HX_MAX_TOPK; ++k2)
-                        if (k2 == k) { sel_pair[k2] = p * D + d; sel_cost[k2] = v; sel_tpre[k2] = tpre_c[typePs[p]]; }
+                        if (k2 == k) { sel_pair[k2] = p * D + d; sel_d[k2] = d; sel_cost[k2] = v; sel_tpre[k2] = tpre_c[typePs[p]]; }
+                    pv = v; pd = d;
                 }
-                if (v == v0) jbest = min(jbest, p * D + d);
-                pv = v; pd = d;
             }
             if (live && t == 0) {
                 const int gc = c0 + c;
@@ -323,7 +380,7 @@ __global__ void __launch_bounds__(256, 1) hx_score_kernel(const __grid_constant_
                         prm.tk.pair[(size_t)gc * K + k] = pr;
                         prm.tk.cost[(size_t)gc * K + k] = bad ? HX_INF : sel_cost[k];
                         prm.tk.tpre[(size_t)gc * K + k] = sel_tpre[k];
-                        if (pr >= 0) atomicAdd(&prm.tk.dcount[pr % D], 1u);   // segment sizes of the conflict pass
+                        prm.tk.dsel[(size_t)gc * K + k] = pr >= 0 ? (uint16_t)sel_d[k] : (uint16_t)0xFFFF;
                     }
                 }
             }
@@ -332,18 +389,15 @@ __global__ void __launch_bounds__(256, 1) hx_score_kernel(const __grid_constant_
     }
 }
 
-template <int TC, int LD>
+template <int TC, int TD, int LD>
 cudaError_t launch_one(const ScoreParams& prm, int grid, int threads, size_t smem, cudaStream_t stream) {
-    cudaError_t e = cudaFuncSetAttribute(hx_score_kernel<TC, LD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(hx_score_kernel<TC, TD, LD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    hx_score_kernel<TC, LD><<<grid, threads, smem, stream>>>(prm);
+    hx_score_kernel<TC, TD, LD><<<grid, threads, smem, stream>>>(prm);
     return cudaGetLastError();
 }
 
 inline int round_up(int a, int b) { return (a + b - 1) / b * b; }
-// row padding (floats) that makes the row stride an odd number of 16-byte units, so that the
-// rows read by the lanes of a warp start in different banks
-inline int pad_of(int pc) { return ((pc >> 2) & 1) ? 8 : 4; }
 
 }  // namespace
 
@@ -353,59 +407,64 @@ cudaError_t hx_launch_score(const HxTables& t, const HxDagView& dag, const HxTop
     ScoreParams prm;
     prm.t = t; prm.dag = dag; prm.tk = tk; prm.s = s; prm.status = status;
     const int D = t.D, C = s.n_calls;
+    // wide decode pools: 16 warps with 4-column thread tiles; narrow ones: 8 warps, 8 columns
     const int LD = D > 32 ? 8 : D > 16 ? 4 : D > 8 ? 2 : 1;
-    const int LC = 32 / LD, WD = 8 * LD;
+    const int TD = LD == 8 ? 4 : 8;
+    const int max_warps = LD == 8 ? 16 : 8;
+    const int LC = 32 / LD, WD = TD * LD;
     prm.WDn = (D + WD - 1) / WD;
     prm.Dpad = prm.WDn * WD;
-    // warps along calls: up to 8 warps per block, fewer when the batch is too small to fill the SMs
-    const int min_tc = LD == 8 ? 5 : 8;
-    int WCn = prm.WDn >= 8 ? 1 : 8 / prm.WDn;
+    // warps along calls: fewer when the batch is too small to fill the SMs
+    const int min_tc = LD == 8 ? 4 : 8;
+    int WCn = prm.WDn >= max_warps ? 1 : max_warps / prm.WDn;
     while (WCn > 1 && (C + WCn * min_tc * LC - 1) / (WCn * min_tc * LC) < n_sm) WCn >>= 1;
     prm.WCn = WCn;
-    // thread tile height: spread the calls evenly over the SMs (a tile of 8 rows per lane
-    // would leave SMs idle whenever the batch is not a multiple of n_sm * WCn * LC * 8 calls)
+    // thread tile height: spread the calls evenly over the SMs (a fixed height would leave SMs
+    // idle whenever the batch is not a multiple of n_sm * rows * height calls)
     int TC = 8;
     if (LD == 8) {
         const int per_sm = (C + n_sm - 1) / n_sm;
         const int rows = WCn * LC;
         const int tiles_per_sm = (per_sm + 8 * rows - 1) / (8 * rows);
         TC = (per_sm + tiles_per_sm * rows - 1) / (tiles_per_sm * rows);
-        TC = TC < 5 ? 5 : (TC > 8 ? 8 : TC);
+        TC = TC < 4 ? 4 : (TC > 8 ? 8 : TC);
     }
     prm.TCB = WCn * TC * LC;
     prm.nTiles = (C + prm.TCB - 1) / prm.TCB;
     prm.FS = prm.Dpad + 4;
-    // prefill chunk: the transposed link tile and the A tile share one row stride
     const int G = t.G;
-    const size_t callB = (size_t)prm.TCB * (2 + 2 * G) * 4;
-    const size_t instB = (size_t)(2 * t.Ppad + 3 * prm.Dpad) * 4;
-    const size_t fixed = round_up((int)callB, 16) + round_up((int)instB, 16);
-    if (fixed + 4096 > max_smem) return cudaErrorInvalidConfiguration;
-    const size_t budget = max_smem - fixed - 64;
+    const size_t callB = round_up(prm.TCB * (2 + 2 * G) * 4, 16);
+    const size_t instB = round_up((2 * t.Ppad + 3 * prm.Dpad) * 4, 16);
+    if (callB + instB + 4096 > max_smem) return cudaErrorInvalidConfiguration;
+    const size_t budget = max_smem - callB - instB - 64;
+    const size_t f_rows = (size_t)prm.TCB * prm.FS * 4;
+    // first choice: whole link table, A tile and finish times side by side
     int PC = t.Ppad;
-    for (;;) {
-        const size_t a_rows = (size_t)prm.TCB * (PC + pad_of(PC)) * 4;
-        const size_t f_rows = (size_t)prm.TCB * prm.FS * 4;
-        const size_t need = (size_t)prm.Dpad * (PC + pad_of(PC)) * 4 + (a_rows > f_rows ? a_rows : f_rows);
-        if (need <= budget || PC <= 4) break;
-        PC = round_up(PC / 2, 4);
+    prm.resident = ((size_t)(prm.Dpad + prm.TCB) * PC * 4 + f_rows <= budget) ? 1 : 0;
+    if (!prm.resident) {
+        // otherwise chunk the prefill dimension; the finish times reuse the A tile
+        for (;;) {
+            const size_t a_rows = (size_t)prm.TCB * PC * 4;
+            if ((size_t)prm.Dpad * PC * 4 + (a_rows > f_rows ? a_rows : f_rows) <= budget || PC <= 4) break;
+            PC = round_up(PC / 2, 4);
+        }
     }
     prm.PC = PC;
     prm.nChunks = (t.Ppad + PC - 1) / PC;
-    prm.PS = PC + pad_of(PC);
-    const size_t ltB = (size_t)prm.Dpad * prm.PS * 4;
-    const size_t aB = (size_t)prm.TCB * (prm.PS > prm.FS ? prm.PS : prm.FS) * 4;
-    prm.offA = round_up((int)ltB, 16);
-    prm.offCall = prm.offA + round_up((int)aB, 16);
-    prm.offInst = prm.offCall + round_up((int)callB, 16);
-    const size_t smem = prm.offInst + round_up((int)instB, 16);
+    const size_t ltB = (size_t)prm.Dpad * PC * 4;
+    const size_t aB = (size_t)prm.TCB * PC * 4;
+    prm.offA = (int)ltB;
+    if (prm.resident) { prm.offF = prm.offA + (int)aB; prm.offCall = prm.offF + round_up((int)f_rows, 16); }
+    else { prm.offF = prm.offA; prm.offCall = prm.offA + (int)(aB > f_rows ? aB : round_up((int)f_rows, 16)); }
+    prm.offInst = prm.offCall + (int)callB;
+    const size_t smem = prm.offInst + instB;
     if (smem > max_smem) return cudaErrorInvalidConfiguration;
     const int threads = 32 * prm.WDn * prm.WCn;
     const int grid = prm.nTiles < n_sm ? prm.nTiles : n_sm;
     cudaError_t e;
-#define HX_CASE(tc, ld) if (TC == tc && LD == ld) e = launch_one<tc, ld>(prm, grid, threads, smem, stream); else
-    HX_CASE(8, 8) HX_CASE(7, 8) HX_CASE(6, 8) HX_CASE(5, 8)
-    HX_CASE(8, 4) HX_CASE(8, 2) HX_CASE(8, 1)
+#define HX_CASE(tc, td, ld) if (TC == tc && TD == td && LD == ld) e = launch_one<tc, td, ld>(prm, grid, threads, smem, stream); else
+    HX_CASE(8, 4, 8) HX_CASE(7, 4, 8) HX_CASE(6, 4, 8) HX_CASE(5, 4, 8) HX_CASE(4, 4, 8)
+    HX_CASE(8, 8, 4) HX_CASE(8, 8, 2) HX_CASE(8, 8, 1)
     e = cudaErrorInvalidConfiguration;
 #undef HX_CASE
     if (e == cudaSuccess) ++*launches;
