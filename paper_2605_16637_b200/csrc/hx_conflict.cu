@@ -36,7 +36,7 @@ typedef unsigned long long u64;
 
 constexpr int kBins = 2048;
 constexpr int kWin = 256;          // calls per optimistic window (= block size of the pass)
-constexpr int kCache = 2048;       // calls staged in shared memory ahead of the window
+constexpr int kCache = 4096;       // calls staged in shared memory ahead of the window
 constexpr unsigned kNone = 0xFFu;  // no candidate taken
 
 // Exclusive prefix sum of n counters into shared memory, by the whole block
@@ -71,19 +71,26 @@ __device__ void block_exclusive_scan(const unsigned* cnt, int n, unsigned* base,
 }
 
 // 1a. Bin the priority keys: one block.  obase receives the kBins + 1 bin bounds, the smallest
-// key and the shift that maps a key to its bin.
+// key and the shift that maps a key to its bin.  Each thread keeps its first kKeep keys in
+// registers (one round trip to memory); the rest of a large batch is read again per pass.
+constexpr int kKeep = 16;
 __global__ void __launch_bounds__(1024) hx_order_bins_kernel(HxTopkBufs tk, int n) {
     __shared__ unsigned hist[kBins], base[kBins + 1], tmp[33], lohi[2];
-    const int tid = threadIdx.x;
-    for (int i = tid; i < kBins; i += blockDim.x) hist[i] = 0;
+    const int tid = threadIdx.x, nthr = blockDim.x;
+    for (int i = tid; i < kBins; i += nthr) hist[i] = 0;
     if (tid == 0) { lohi[0] = 0xFFFFFFFFu; lohi[1] = 0u; }
+    unsigned keep[kKeep];
+#pragma unroll
+    for (int u = 0; u < kKeep; ++u) {
+        const int c = tid + u * nthr;
+        keep[u] = c < n ? ~__float_as_uint(__ldg(tk.prio + c)) : 0u;      // larger priority = smaller key
+    }
+    auto key_of = [&](int u, int c) { return u < kKeep ? keep[u] : ~__float_as_uint(__ldg(tk.prio + c)); };
     __syncthreads();
     unsigned lo = 0xFFFFFFFFu, hi = 0u;
-#pragma unroll 4
-    for (int c = tid; c < n; c += blockDim.x) {
-        const unsigned key = ~__float_as_uint(__ldg(tk.prio + c));   // larger priority = smaller key
-        lo = min(lo, key); hi = max(hi, key);
-    }
+#pragma unroll
+    for (int u = 0; u < kKeep; ++u) if (tid + u * nthr < n) { lo = min(lo, keep[u]); hi = max(hi, keep[u]); }
+    for (int c = tid + kKeep * nthr; c < n; c += nthr) { const unsigned k = key_of(kKeep, c); lo = min(lo, k); hi = max(hi, k); }
     lo = __reduce_min_sync(0xffffffffu, lo); hi = __reduce_max_sync(0xffffffffu, hi);
     if ((tid & 31) == 0) { atomicMin(&lohi[0], lo); atomicMax(&lohi[1], hi); }
     __syncthreads();
@@ -91,18 +98,25 @@ __global__ void __launch_bounds__(1024) hx_order_bins_kernel(HxTopkBufs tk, int 
     const unsigned span = lohi[1] - lo;
     int shift = 0;
     while ((span >> shift) >= (unsigned)kBins) ++shift;
-#pragma unroll 4
-    for (int c = tid; c < n; c += blockDim.x)
-        atomicAdd(&hist[(~__float_as_uint(__ldg(tk.prio + c)) - lo) >> shift], 1u);
+#pragma unroll
+    for (int u = 0; u < kKeep; ++u) if (tid + u * nthr < n) atomicAdd(&hist[(keep[u] - lo) >> shift], 1u);
+    for (int c = tid + kKeep * nthr; c < n; c += nthr) atomicAdd(&hist[(key_of(kKeep, c) - lo) >> shift], 1u);
     __syncthreads();
     block_exclusive_scan(hist, kBins, base, tmp);
-    for (int i = tid; i <= kBins; i += blockDim.x) tk.obase[i] = base[i];
+    for (int i = tid; i <= kBins; i += nthr) tk.obase[i] = base[i];
     if (tid == 0) { tk.obase[kBins + 1] = lo; tk.obase[kBins + 2] = (unsigned)shift; }
-    for (int i = tid; i < kBins; i += blockDim.x) hist[i] = 0;     // now the bin cursors
+    for (int i = tid; i < kBins; i += nthr) hist[i] = 0;           // now the bin cursors
     __syncthreads();
-#pragma unroll 4
-    for (int c = tid; c < n; c += blockDim.x) {
-        const unsigned key = ~__float_as_uint(__ldg(tk.prio + c));
+#pragma unroll
+    for (int u = 0; u < kKeep; ++u) {
+        const int c = tid + u * nthr;
+        if (c < n) {
+            const unsigned bin = (keep[u] - lo) >> shift;
+            tk.okey[base[bin] + atomicAdd(&hist[bin], 1u)] = ((u64)keep[u] << 32) | (unsigned)c;
+        }
+    }
+    for (int c = tid + kKeep * nthr; c < n; c += nthr) {
+        const unsigned key = key_of(kKeep, c);
         const unsigned bin = (key - lo) >> shift;
         tk.okey[base[bin] + atomicAdd(&hist[bin], 1u)] = ((u64)key << 32) | (unsigned)c;
     }
@@ -112,7 +126,6 @@ __global__ void __launch_bounds__(1024) hx_order_bins_kernel(HxTopkBufs tk, int 
 __global__ void hx_order_rank_kernel(HxTopkBufs tk, int n) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
-    const int K = tk.K;
     const unsigned lo = tk.obase[kBins + 1], shift = tk.obase[kBins + 2];
     const u64 key = tk.okey[i];
     const unsigned bin = ((unsigned)(key >> 32) - lo) >> shift;
@@ -122,80 +135,94 @@ __global__ void hx_order_rank_kernel(HxTopkBufs tk, int n) {
     const unsigned c = (unsigned)key;
     tk.ocall[rank] = c;
     tk.om[rank] = tk.mtok[c];
-    for (int k = 0; k < K; ++k) tk.od[(size_t)rank * K + k] = tk.dsel[(size_t)c * K + k];
+    tk.od[rank] = tk.dsel[c];
 }
 
 // 2. The pass itself: one block of kWin threads.
 __global__ void __launch_bounds__(kWin) hx_conflict_kernel(HxTopkBufs tk, HxTables t, int n, int commit) {
-    extern __shared__ unsigned sm[];
+    extern __shared__ __align__(16) unsigned sm[];
     constexpr int NW = kWin / 32;
     const int D = t.D, K = tk.K;
-    float* free_s = reinterpret_cast<float*>(sm);               // [D] capacity left after the commits so far
+    uint4* cd = reinterpret_cast<uint4*>(sm);                   // [kCache] candidate instances of the staged calls
+    float* cm = reinterpret_cast<float*>(cd + kCache);          // [kCache] their demands
+    float* free_s = cm + kCache;                                // [D] capacity left after the commits so far
     float* wtot = free_s + D;                                   // [NW][D] demand per warp and instance
-    float* cm = wtot + NW * D;                                  // [kCache] demands of the staged calls
-    uint16_t* cd = reinterpret_cast<uint16_t*>(cm + kCache);    // [kCache][K] their candidate instances
-    __shared__ int first_fail, n_acc_s, cache_lo;
-    __shared__ unsigned wacc[NW + 1];
+    __shared__ int first_fail;
+    __shared__ unsigned wacc[NW];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     for (int d = tid; d < D; d += kWin) free_s[d] = t.freeD[d];
-    if (tid == 0) { n_acc_s = 0; cache_lo = -kCache; }
-    __syncthreads();
-    int pos = 0;
+    for (int i = tid; i < NW * D; i += kWin) wtot[i] = 0.f;
+    if (tid == 0) first_fail = kWin;
+    int pos = 0, cache_lo = -kCache;
+    unsigned n_acc = 0;                                         // same value in every thread
     while (pos < n) {
-        if (pos + kWin > cache_lo + kCache) {                   // stage the next calls (one round trip)
+        if (pos + kWin > cache_lo + kCache) {                   // stage the next calls: one round trip
             __syncthreads();
-            for (int i = tid; i < kCache; i += kWin) {
-                const int r = pos + i;
-                cm[i] = r < n ? tk.om[r] : 0.f;
-                for (int k = 0; k < K; ++k) cd[i * K + k] = r < n ? tk.od[(size_t)r * K + k] : (uint16_t)0xFFFF;
+            cache_lo = pos;
+#pragma unroll
+            for (int u = 0; u < kCache / kWin; ++u) {
+                const int i = tid + u * kWin, r = pos + i;
+                cd[i] = r < n ? __ldcg(tk.od + r) : make_uint4(~0u, ~0u, ~0u, ~0u);
+                cm[i] = r < n ? __ldcg(tk.om + r) : 0.f;
             }
-            if (tid == 0) cache_lo = pos;
-            __syncthreads();
         }
+        __syncthreads();                                        // S0: staged data, capacities and zeroed totals visible
         const int r = pos + tid, ci = r - cache_lo;
         const bool active = r < n;
-        const float m = active ? cm[ci] : 0.f;
+        const float m = cm[ci];
         // first candidate that fits the committed capacities
         unsigned kt = kNone; int dt = -1;
-        if (active)
-            for (int k = K - 1; k >= 0; --k) {
-                const unsigned d = cd[ci * K + k];
-                if (d != 0xFFFFu && free_s[d] >= m) { kt = k; dt = (int)d; }
+        if (active) {
+            const uint4 row = cd[ci];
+            const unsigned w[4] = {row.x, row.y, row.z, row.w};
+#pragma unroll
+            for (int k = HX_MAX_TOPK - 1; k >= 0; --k) {
+                const unsigned d = (w[k >> 1] >> ((k & 1) * 16)) & 0xFFFFu;
+                if (k < K && d != 0xFFFFu && free_s[d] >= m) { kt = k; dt = (int)d; }
             }
-        for (int i = tid; i < NW * D; i += kWin) wtot[i] = 0.f;
-        if (tid == 0) first_fail = kWin;
-        // demand of the earlier lanes of this warp that picked the same instance
+        }
+        // demand of the earlier lanes of this warp that picked the same instance: one warp scan
+        // per distinct instance
+        float cum = 0.f, incl = 0.f;
+        unsigned rem = __ballot_sync(0xffffffffu, dt >= 0);
+        while (rem) {
+            const int leader = __ffs(rem) - 1;
+            const int dl = __shfl_sync(0xffffffffu, dt, leader);
+            const bool mine = dt == dl;
+            float x = mine ? m : 0.f;
+            for (int off = 1; off < 32; off <<= 1) {
+                const float y = __shfl_up_sync(0xffffffffu, x, off);
+                if (lane >= off) x = __fadd_rn(x, y);
+            }
+            if (mine) { incl = x; cum = __fsub_rn(x, m); }
+            rem &= ~__ballot_sync(0xffffffffu, mine);
+        }
         const unsigned peers = __match_any_sync(0xffffffffu, dt);
-        float cum = 0.f;
-        for (int j = 0; j < 31; ++j) {
-            const float mj = __shfl_sync(0xffffffffu, m, j);
-            if (j < lane && ((peers >> j) & 1u)) cum = __fadd_rn(cum, mj);
-        }
-        __syncthreads();
-        if (dt >= 0 && (peers >> lane) <= 1u) wtot[warp * D + dt] = __fadd_rn(cum, m);   // last peer: warp total
-        __syncthreads();
-        if (dt >= 0) for (int w = 0; w < warp; ++w) cum = __fadd_rn(cum, wtot[w * D + dt]);
-        if (dt >= 0 && __fadd_rn(cum, m) > free_s[dt]) atomicMin(&first_fail, tid);
-        __syncthreads();
+        const bool last_peer = dt >= 0 && (peers >> lane) <= 1u;
+        if (last_peer) wtot[warp * D + dt] = incl;              // demand of this warp on dt
+        __syncthreads();                                        // S1
+        float before = cum;
+        if (dt >= 0) for (int w = 0; w < warp; ++w) before = __fadd_rn(before, wtot[w * D + dt]);
+        if (dt >= 0 && __fadd_rn(before, m) > free_s[dt]) atomicMin(&first_fail, tid);
+        __syncthreads();                                        // S2
         const int f = first_fail;                               // calls before f decided as the sequential pass would
-        const bool done = active && tid < f;
-        const bool acc = done && dt >= 0;
-        if (acc) atomicAdd(&free_s[dt], -m);                    // exact: integer-valued operands
-        // obtained pairs, appended in visiting order
-        const unsigned b = __ballot_sync(0xffffffffu, acc);
-        if (lane == 0) wacc[warp] = __popc(b);
-        __syncthreads();
-        if (acc) {
-            unsigned off = n_acc_s + __popc(b & ((1u << lane) - 1u));
-            for (int w = 0; w < warp; ++w) off += wacc[w];
-            tk.acc_rk[off] = (unsigned)r | (kt << 24);
-        }
-        __syncthreads();
-        if (tid == 0) { int a = 0; for (int w = 0; w < NW; ++w) a += wacc[w]; n_acc_s += a; }
+        const bool acc = active && tid < f && dt >= 0;
+        // the last committing peer of each warp subtracts the demand of its warp's committing peers
+        const unsigned accm = __ballot_sync(0xffffffffu, acc);
+        if (acc && (((peers & accm) >> lane) <= 1u)) atomicAdd(&free_s[dt], -incl);   // exact: integer-valued
+        if (last_peer) wtot[warp * D + dt] = 0.f;
+        if (lane == 0) wacc[warp] = __popc(accm);
+        __syncthreads();                                        // S3
+        if (tid == 0) first_fail = kWin;
+        unsigned off = n_acc + __popc(accm & ((1u << lane) - 1u));
+        unsigned tot = 0;
+        for (int w = 0; w < NW; ++w) { const unsigned a = wacc[w]; tot += a; if (w < warp) off += a; }
+        if (acc) tk.acc_rk[off] = (unsigned)r | (kt << 24);     // obtained pairs, in visiting order
+        n_acc += tot;
         pos += f < kWin ? f : kWin;
     }
     __syncthreads();
-    if (tid == 0) *tk.n_acc = (unsigned)n_acc_s;
+    if (tid == 0) *tk.n_acc = n_acc;
     if (commit) for (int d = tid; d < D; d += kWin) t.freeD[d] = free_s[d];
 }
 
@@ -234,7 +261,7 @@ cudaError_t hx_launch_conflict(const HxTables& t, const HxTopkBufs& tk, int n_ca
     const int D = t.D, P = t.P;
     hx_order_bins_kernel<<<1, 1024, 0, stream>>>(tk, n_calls);
     hx_order_rank_kernel<<<(n_calls + 127) / 128, 128, 0, stream>>>(tk, n_calls);
-    const size_t smC = (size_t)(D + (kWin / 32) * D + kCache) * 4 + (size_t)kCache * tk.K * 2;
+    const size_t smC = (size_t)kCache * 20 + (size_t)(D + (kWin / 32) * D) * 4;
     if (smC > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(hx_conflict_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smC);
         if (e != cudaSuccess) return e;

@@ -113,14 +113,14 @@ int ensure_topk(hx_cluster* h, int n_calls, int K) {
     HX_TRY(dev_alloc(h->tk_allocs, &b.pair, cap * K), "alloc top-K");
     HX_TRY(dev_alloc(h->tk_allocs, &b.cost, cap * K), "alloc top-K");
     HX_TRY(dev_alloc(h->tk_allocs, &b.tpre, cap * K), "alloc top-K");
-    HX_TRY(dev_alloc(h->tk_allocs, &b.dsel, cap * K), "alloc top-K");
+    HX_TRY(dev_alloc(h->tk_allocs, &b.dsel, cap), "alloc top-K");
     HX_TRY(dev_alloc(h->tk_allocs, &b.prio, cap), "alloc top-K");
     HX_TRY(dev_alloc(h->tk_allocs, &b.mtok, cap), "alloc top-K");
     HX_TRY(dev_alloc(h->tk_allocs, &b.okey, cap), "alloc order");
     HX_TRY(dev_alloc(h->tk_allocs, &b.obase, (size_t)2048 + 3), "alloc order");
     HX_TRY(dev_alloc(h->tk_allocs, &b.ocall, cap), "alloc order");
     HX_TRY(dev_alloc(h->tk_allocs, &b.om, cap), "alloc order");
-    HX_TRY(dev_alloc(h->tk_allocs, &b.od, cap * K), "alloc order");
+    HX_TRY(dev_alloc(h->tk_allocs, &b.od, cap), "alloc order");
     HX_TRY(dev_alloc(h->tk_allocs, &b.n_acc, (size_t)1), "alloc outcome");
     HX_TRY(dev_alloc(h->tk_allocs, &b.acc_rk, cap), "alloc outcome");
     HX_TRY(dev_alloc(h->tk_allocs, &b.acc_p, cap), "alloc outcome");

@@ -50,7 +50,7 @@ struct HxTopkBufs {
     int32_t* pair;             // [cap][K]
     float* cost;               // [cap][K]
     float* tpre;               // [cap][K] prefill time on the prefill instance of slot k
-    uint16_t* dsel;            // [cap][K] decode instance of slot k, 0xFFFF = unused
+    uint4* dsel;               // [cap] decode instance of each slot as 8 x 16 bits, 0xFFFF = unused
     float* prio;               // [cap]
     float* mtok;               // [cap]
     // visiting order
@@ -58,7 +58,7 @@ struct HxTopkBufs {
     unsigned int* obase;       // [2048 + 3] bin bounds, smallest key, key-to-bin shift
     unsigned int* ocall;       // [cap] call of each rank
     float* om;                 // [cap] demand of each rank
-    uint16_t* od;              // [cap][K] decode instances of each rank's slots
+    uint4* od;                 // [cap] same rows in visiting order
     // outcome: calls that obtained a pair, in visiting order
     unsigned int* n_acc;       // [1]
     unsigned int* acc_rk;      // [cap] rank | k << 24

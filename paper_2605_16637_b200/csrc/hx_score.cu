@@ -373,6 +373,7 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
                     prm.s.out_assign[gc] = -1;            // filled in by the capacity-conflict pass
                     prm.tk.prio[gc] = __fdiv_rn(__fadd_rn(elapsed, v0), H);   // Eq. 2
                     prm.tk.mtok[gc] = m;
+                    unsigned dw[4] = {~0u, ~0u, ~0u, ~0u};          // decode instances of the slots, 8 x 16 bits
 #pragma unroll
                     for (int k = 0; k < HX_MAX_TOPK; ++k) {
                         if (k >= K) break;
@@ -380,8 +381,9 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
                         prm.tk.pair[(size_t)gc * K + k] = pr;
                         prm.tk.cost[(size_t)gc * K + k] = bad ? HX_INF : sel_cost[k];
                         prm.tk.tpre[(size_t)gc * K + k] = sel_tpre[k];
-                        prm.tk.dsel[(size_t)gc * K + k] = pr >= 0 ? (uint16_t)sel_d[k] : (uint16_t)0xFFFF;
+                        dw[k >> 1] = (dw[k >> 1] & ~(0xFFFFu << ((k & 1) * 16))) | ((pr >= 0 ? (unsigned)sel_d[k] : 0xFFFFu) << ((k & 1) * 16));
                     }
+                    prm.tk.dsel[gc] = make_uint4(dw[0], dw[1], dw[2], dw[3]);
                 }
             }
         }
