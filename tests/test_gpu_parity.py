@@ -1,0 +1,331 @@
+"""GPU-vs-oracle parity through the C ABI binding.
+
+Bars (stated once in hx_helpers): binary32 costs within 1e-5 relative of the oracle,
+placements identical unless the oracle's own cost gap is below that tolerance,
+horizons bit-exact, integer outputs of the capacity pass bit-exact.  The kernels
+are designed to reproduce the oracle's binary32 sequence exactly, so most checks
+also demand identical bits; where they do it is an additional, stricter assertion.
+"""
+import numpy as np
+import pytest
+
+import hx_helpers as hh
+from hx_synth import CALL_DTYPE, make_workload, sub_forest
+from oracle import hx_oracle as ho
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def hx():
+    import __graft_entry__ as entry
+    entry.build()
+    import paper_2605_16637_b200 as mod
+    return mod
+
+
+def _cluster_pair(hx, P, D, G=4, M=2, seed=0, tight=False, qd_round=False):
+    rng = np.random.default_rng(seed)
+    types = np.stack([rng.uniform(50, 2000, G), rng.uniform(0.3, 8, G)], 1).astype(np.float32)
+    models = np.stack([rng.uniform(1e9, 2e11, M), rng.uniform(1e9, 2e11, M),
+                       rng.choice([65536.0, 131072.0, 327680.0], M)], 1).astype(np.float32)
+    inst = np.zeros(P + D, hx.INSTANCE_DTYPE)
+    inst["type"] = rng.integers(0, G, P + D)
+    inst["role"][P:] = 1
+    inst["load_s"] = rng.uniform(0, 2, P + D)
+    if qd_round:
+        inst["load_s"] = np.round(inst["load_s"] * 2) / 2
+    cap = rng.choice([600.0, 3000.0, 1e6], P + D) if tight else np.full(P + D, 1e6)
+    inst["kv_cap_tokens"] = cap
+    inst["kv_free_tokens"] = cap
+    link = rng.uniform(25, 400, (P + D, P + D)).astype(np.float32)
+    gc = hx.Cluster(types, inst, link, models)
+    oc = ho.Cluster(types, inst["type"][:P], inst["type"][P:], inst["load_s"][:P], inst["load_s"][P:],
+                    inst["kv_cap_tokens"][P:], link[:P, P:], models)
+    return gc, oc
+
+
+def _calls(n, M=2, seed=1, lo_mu=7.0):
+    rng = np.random.default_rng(seed)
+    a = np.zeros(n, CALL_DTYPE)
+    a["node"] = np.arange(n)
+    a["model"] = rng.integers(0, M, n)
+    a["prompt_tokens"] = np.clip(np.round(rng.lognormal(lo_mu, 1, n)), 1, 32768)
+    a["output_tokens"] = np.clip(np.round(rng.lognormal(5, 1, n)), 1, 32768)
+    return a
+
+
+def _prepare(hx, oracle, wl):
+    """Cluster on both sides, stand-alone node costs, horizons; returns everything needed to score."""
+    oc, gc = hh.oracle_cluster(wl), hh.gpu_cluster(wl)
+    if wl.node_cost is not None:
+        cost_o = cost_g = wl.node_cost
+    else:
+        cost_o = hh.oracle_node_costs(oracle, oc, wl.node_calls)
+        cost_g = hh.gpu_node_costs(gc, wl.node_calls)
+        hh.assert_costs_close(cost_g, cost_o, "stand-alone node costs")
+        assert np.array_equal(cost_g, cost_o)
+    dag = oracle.longest_path(wl.row_ptr, wl.col, cost_o, wl.node_wf, wl.n_workflows)
+    gc.dag_upload(wl.row_ptr, wl.col, cost_g, wl.node_wf, wl.elapsed)
+    gc.critical_path()
+    return oc, gc, dag
+
+
+CONFIGS = [("tiny", 1.0), ("medium", 1.0), ("large", 1 / 16), ("cp_stress", 1 / 20), ("sweep", 1 / 64)]
+
+
+@pytest.mark.parametrize("name, scale", CONFIGS)
+def test_horizons_bit_exact(hx, oracle, name, scale):
+    wl = make_workload(name, scale=scale)
+    oc, gc, dag = _prepare(hx, oracle, wl)
+    cp, tail, H = gc.dag_results()
+    assert np.array_equal(cp, dag.cp) and np.array_equal(tail, dag.tail) and np.array_equal(H, dag.H)
+    gc.close()
+
+
+@pytest.mark.parametrize("name, scale", CONFIGS)
+def test_scoring_all_modes(hx, oracle, name, scale):
+    wl = make_workload(name, scale=scale)
+    oc, gc, dag = _prepare(hx, oracle, wl)
+    calls = wl.calls
+    kw = dict(dag=dag, node_wf=wl.node_wf, elapsed=wl.elapsed, alpha=wl.alpha)
+    for mode, flags in [(0, 0), (1, 0), (2, 0), (2, hx.HX_FLAG_NO_TAIL), (0, hx.HX_FLAG_UNLOADED)]:
+        gc.set_options(score_mode=mode, flags=flags, alpha=wl.alpha)
+        a, c = gc.schedule_batch(calls)
+        a, c = a.cpu().numpy(), c.cpu().numpy()
+        oa, ocost, _ = oracle.schedule(oc, calls, mode=mode, flags=flags, **kw)
+        hh.assert_costs_close(c, ocost, "%s mode %d flags %d" % (name, mode, flags))
+        hh.assert_assign_matches(oracle, oc, calls, a, oa, flags=flags & hx.HX_FLAG_UNLOADED, what=name)
+        assert np.array_equal(c, ocost) and np.array_equal(a, oa)       # identical bits by construction
+    assert gc.status() == 0
+    gc.close()
+
+
+SHAPES = [(1, 1, 5), (2, 3, 17), (5, 3, 64), (4, 9, 100), (17, 16, 333), (33, 70, 500), (130, 129, 300),
+          (128, 200, 257), (40, 512, 130), (600, 64, 200), (1024, 128, 150)]
+
+
+@pytest.mark.parametrize("P, D, n", SHAPES)
+def test_scoring_ragged_shapes(hx, oracle, P, D, n):
+    """Pool sizes that are not multiples of the tiles, several warps along d, chunked prefill dimension."""
+    gc, oc = _cluster_pair(hx, P, D, seed=P * 1000 + D, tight=True)
+    calls = _calls(n, seed=n)
+    gc.set_options(flags=hx.HX_FLAG_NO_DAG)
+    a, c = gc.schedule_batch(calls)
+    oa, ocost, _ = oracle.schedule(oc, calls)
+    assert np.array_equal(a.cpu().numpy(), oa) and np.array_equal(c.cpu().numpy(), ocost)
+    K = min(4, D)
+    gc.set_options(topk=K, flags=hx.HX_FLAG_NO_DAG)
+    gc.schedule_batch(calls)
+    pair, cost, prio = gc.topk_results(n)
+    op, ocs, opr, _, _ = oracle.topk(oc, calls, K)
+    assert np.array_equal(pair, op) and np.array_equal(cost, ocs) and np.array_equal(prio, opr)
+    gc.close()
+
+
+def test_exact_ties_and_infeasible_calls(hx, oracle):
+    # identical instances, late decode admission: every pair of a decode type ties exactly
+    P, D = 6, 5
+    inst = np.zeros(P + D, hx.INSTANCE_DTYPE)
+    inst["role"][P:] = 1
+    inst["load_s"][:P] = [0.1, 0.0, 0.2, 0.0, 0.3, 0.05]
+    inst["load_s"][P:] = 9.0
+    inst["kv_cap_tokens"] = [0] * P + [1e6, 1e6, 500, 1e6, 1e6]
+    inst["kv_free_tokens"] = inst["kv_cap_tokens"]
+    types = np.array([[1000.0, 1.0]], np.float32)
+    models = np.array([[2e9, 1e9, 1e5]], np.float32)
+    link = np.full((P + D, P + D), 100.0, np.float32)
+    gc = hx.Cluster(types, inst, link, models)
+    oc = ho.Cluster(types, inst["type"][:P], inst["type"][P:], inst["load_s"][:P], inst["load_s"][P:],
+                    inst["kv_cap_tokens"][P:], link[:P, P:], models)
+    calls = np.zeros(4, CALL_DTYPE)
+    calls["prompt_tokens"] = [1000, 200, 3e6, 100]       # the third call fits nowhere
+    calls["output_tokens"] = [11, 50, 10, 100]
+    gc.set_options(flags=hx.HX_FLAG_NO_DAG)
+    a, c = gc.schedule_batch(calls)
+    a, c = a.cpu().numpy(), c.cpu().numpy()
+    oa, ocost, _ = oracle.schedule(oc, calls)
+    assert list(a) == list(oa) == [0, 0, -1, 0]
+    assert np.array_equal(c, ocost) and np.isinf(c[2])
+    gc.set_options(topk=4, flags=hx.HX_FLAG_NO_DAG)
+    a2, _ = gc.schedule_batch(calls)
+    pair, cost, prio = gc.topk_results(4)
+    op, ocs, opr, om, ots = oracle.topk(oc, calls, 4)
+    assert np.array_equal(pair, op) and np.array_equal(cost, ocs) and np.array_equal(prio, opr)
+    assert list(pair[0]) == [0, 1, 3, 4]                 # d = 2 is too small for call 0; ties ordered by d
+    assert list(pair[2]) == [-1] * 4
+    gc.close()
+
+
+def test_single_call_single_pair_closed_form(hx):
+    """P = D = 1, one call: the hand-computed finish of the golden 'hand' case (0.2651055 s)."""
+    inst = np.zeros(2, hx.INSTANCE_DTYPE)
+    inst["role"][1] = 1
+    inst["load_s"] = [0.25, 0.1]
+    inst["kv_cap_tokens"] = inst["kv_free_tokens"] = 1e6
+    gc = hx.Cluster(np.array([[1000.0, 1.0]]), inst, np.full((2, 2), 100.0), np.array([[2e9, 1e9, 1e5]]))
+    calls = np.zeros(1, CALL_DTYPE)
+    calls["prompt_tokens"] = 1000; calls["output_tokens"] = 11
+    gc.set_options(flags=hx.HX_FLAG_NO_DAG)
+    a, c = gc.schedule_batch(calls)
+    assert int(a[0]) == 0 and abs(float(c[0]) - 0.2651055) < 2e-6 * 0.2651055
+    gc.close()
+
+
+def test_empty_batch_not_ready_and_bad_ids(hx, oracle):
+    import torch
+    wl = make_workload("tiny")
+    gc = hh.gpu_cluster(wl)
+    assert hx.hx_schedule_batch(gc.h, None, 0, None, None, 0) is None        # n_calls = 0 is a no-op
+    with pytest.raises(hx.HxError) as e:                                      # horizons not computed yet
+        gc.schedule_batch(wl.calls)
+    assert e.value.code == -4
+    with pytest.raises(hx.HxError):
+        gc.set_options(topk=9)
+    with pytest.raises(hx.HxError) as e:                                      # cycle
+        gc.dag_upload([0, 1, 2], [1, 0], [1.0, 1.0], [0, 0], [0.0])
+    assert e.value.code == -3
+    with pytest.raises(hx.HxError):                                           # edge across workflows
+        gc.dag_upload([0, 1, 1], [1], [1.0, 1.0], [0, 1], [0.0, 0.0])
+    # a record with an unknown model or node is flagged, gets no pair, and does not disturb the others
+    gc.set_options(flags=hx.HX_FLAG_NO_DAG)
+    calls = wl.calls.copy()
+    calls["model"][3] = 77
+    a, c = gc.schedule_batch(calls)
+    a, c = a.cpu().numpy(), c.cpu().numpy()
+    assert a[3] == -1 and np.isinf(c[3]) and gc.status() == -1
+    good = np.arange(len(calls)) != 3
+    oa, ocost, _ = oracle.schedule(hh.oracle_cluster(wl), wl.calls)
+    assert np.array_equal(a[good], oa[good]) and np.array_equal(c[good], ocost[good])
+    gc.close()
+
+
+@pytest.mark.parametrize("kind", ["single", "chain_staged", "chain_block", "chain_global", "mixed"])
+def test_horizon_workflow_classes(hx, oracle, kind):
+    """Workflows small enough for a warp's staging area, for a block's, and too large for either."""
+    rng = np.random.default_rng(5)
+    if kind == "single":
+        n_w = [1]
+    elif kind == "chain_staged":
+        n_w = [900]
+    elif kind == "chain_block":
+        n_w = [6000]
+    elif kind == "chain_global":
+        n_w = [30000]
+    else:
+        n_w = [1, 40, 1500, 3, 9000, 200, 25000, 7]
+    rows, cols, wf = [0], [], []
+    base = 0
+    for w, n in enumerate(n_w):
+        for i in range(n):
+            succ = []
+            if i + 1 < n:
+                succ.append(base + i + 1)
+                if i + 5 < n and rng.random() < 0.3:
+                    succ.append(base + i + 5)
+            cols += succ
+            rows.append(len(cols))
+            wf.append(w)
+        base += n
+    N = base
+    cost = rng.lognormal(0, 1, N).astype(np.float32)
+    wl = make_workload("tiny")
+    gc = hh.gpu_cluster(wl)
+    gc.dag_upload(rows, cols, cost, wf, np.zeros(len(n_w)))
+    gc.critical_path()
+    cp, tail, H = gc.dag_results()
+    r = oracle.longest_path(rows, cols, cost, wf, len(n_w))
+    assert np.array_equal(cp, r.cp) and np.array_equal(tail, r.tail) and np.array_equal(H, r.H)
+    gc.close()
+
+
+@pytest.mark.parametrize("name, scale, K", [("tiny", 1.0, 2), ("medium", 1.0, 4), ("large", 1 / 32, 4),
+                                            ("cp_stress", 1 / 50, 1), ("sweep", 1 / 64, 4), ("sweep", 1 / 64, 8)])
+def test_topk_and_capacity_pass(hx, oracle, name, scale, K):
+    wl = make_workload(name, scale=scale)
+    oc, gc, dag = _prepare(hx, oracle, wl)
+    calls = wl.calls
+    P, D = wl.P, wl.D
+    free0 = wl.kv_free[P:].copy()
+    if name != "sweep":                                   # make capacity scarce so that the pass matters
+        m = calls["prompt_tokens"] + calls["output_tokens"]
+        free0 = np.floor(np.minimum(free0, 0.7 * m.sum() / D)).astype(np.float32)
+    kw = dict(dag=dag, node_wf=wl.node_wf, elapsed=wl.elapsed)
+    n_chunks = 3
+    step = max(1, len(calls) // n_chunks)
+    qP = wl.load_s[:P].copy()
+    gc.set_options(score_mode=hx.HX_MODE_RATIO, topk=K, commit=1, alpha=wl.alpha)
+    for i in range(n_chunks):
+        chunk = calls[i * step:(i + 1) * step]
+        gc.update_loads(kv_free=free0)                    # decode capacity is refreshed between invocations
+        a, c = gc.schedule_batch(chunk)
+        a, c = a.cpu().numpy(), c.cpu().numpy()
+        pair, cost, prio = gc.topk_results(len(chunk))
+        oc.qP[:] = qP
+        op, ocs, opr, om, ots = oracle.topk(oc, chunk, K, **kw)
+        assert np.array_equal(pair, op) and np.array_equal(cost, ocs) and np.array_equal(prio, opr)
+        oa, ofree, oq = oracle.conflict(op, opr, om, ots, free0, qP, D)
+        gq, _, gfree = gc.read_loads()
+        assert np.array_equal(a, oa), "%s chunk %d" % (name, i)
+        assert np.array_equal(gfree, ofree) and np.array_equal(gq, oq)
+        _, ocost, _ = oracle.schedule(oc, chunk, mode=ho.MODE_RATIO, **kw)
+        assert np.array_equal(c, ocost)
+        assert np.all(gfree >= 0)
+        qP = oq
+    assert gc.status() == 0
+    gc.close()
+
+
+def test_capacity_pass_without_commit_leaves_loads(hx, oracle):
+    wl = make_workload("sweep", scale=1 / 64)
+    oc, gc, dag = _prepare(hx, oracle, wl)
+    before = gc.read_loads()
+    gc.set_options(score_mode=hx.HX_MODE_RATIO, topk=4, commit=0)
+    a, _ = gc.schedule_batch(wl.calls)
+    after = gc.read_loads()
+    assert all(np.array_equal(x, y) for x, y in zip(before, after))
+    op, ocs, opr, om, ots = oracle.topk(oc, wl.calls, 4, dag=dag, node_wf=wl.node_wf, elapsed=wl.elapsed)
+    oa, _, _ = oracle.conflict(op, opr, om, ots, wl.kv_free[wl.P:], wl.load_s[:wl.P], wl.D)
+    assert np.array_equal(a.cpu().numpy(), oa)
+    gc.close()
+
+
+def test_equal_priorities_visit_lower_call_first(hx, oracle):
+    """All calls identical: the order of the pass is the call index, capacity runs out part way."""
+    gc, oc = _cluster_pair(hx, 4, 4, seed=3)
+    calls = np.zeros(300, CALL_DTYPE)
+    calls["prompt_tokens"] = 900; calls["output_tokens"] = 100
+    free = np.array([20000, 5000, 7000, 3000], np.float32)
+    gc.update_loads(kv_free=free)
+    gc.set_options(topk=4, commit=1, flags=hx.HX_FLAG_NO_DAG)
+    a, _ = gc.schedule_batch(calls)
+    a = a.cpu().numpy()
+    op, ocs, opr, om, ots = oracle.topk(oc, calls, 4)
+    oa, ofree, oq = oracle.conflict(op, opr, om, ots, free, oc.qP, 4)
+    assert np.array_equal(a, oa) and (a >= 0).sum() == 35 and np.all(a[35:] == -1)
+    gq, _, gfree = gc.read_loads()
+    assert np.array_equal(gfree, ofree) and np.array_equal(gq, oq)
+    gc.close()
+
+
+def test_host_buffer_entry_point_matches_device_path(hx, oracle):
+    wl = make_workload("medium")
+    oc, gc, dag = _prepare(hx, oracle, wl)
+    gc.set_options(score_mode=hx.HX_MODE_SLACK, alpha=wl.alpha)
+    a, c = gc.schedule_batch(wl.calls)
+    ha, hc = gc.schedule_batch_host(wl.calls)
+    assert np.array_equal(a.cpu().numpy(), ha) and np.array_equal(c.cpu().numpy(), hc)
+    gc.close()
+
+
+def test_runs_are_deterministic(hx, oracle):
+    wl = make_workload("sweep", scale=1 / 32)
+    outs = []
+    for _ in range(2):
+        oc, gc, dag = _prepare(hx, oracle, wl)
+        gc.set_options(score_mode=hx.HX_MODE_RATIO, topk=4, commit=1)
+        a, c = gc.schedule_batch(wl.calls)
+        outs.append((a.cpu().numpy().tobytes(), c.cpu().numpy().tobytes(),
+                     b"".join(x.tobytes() for x in gc.read_loads())))
+        gc.close()
+    assert outs[0] == outs[1]
