@@ -177,6 +177,37 @@ int hx_schedule_batch(hx_cluster* h, const hx_call* calls, int n_calls,
 int hx_schedule_batch_host(hx_cluster* h, const hx_call* calls, int n_calls,
                            int32_t* out_assign, float* out_cost, void* stream);
 
+/* hx_schedule_batch for callers that must not allocate.  (The paper has no
+ * counterpart: this entry point exists only because of how the library is
+ * embedded.)  hx_schedule_batch with topk > 0 obtains its intermediate buffers
+ * with cudaMalloc on first use and whenever a batch is larger than any before.
+ * Some hosts of this library cannot tolerate that: a serving process whose
+ * memory pool already owns the whole device, so that a late cudaMalloc fails;
+ * a latency-critical scheduling thread for which the device-wide
+ * synchronisation of an allocation is a stall; code running where the CUDA
+ * allocator may not be entered at all.  This variant computes the same
+ * results but keeps the top-K lists, the visiting order and the bookkeeping of
+ * the capacity pass in one fixed array of about 1.9 MB that is part of the
+ * library image; every device that loads the library holds that array until
+ * the process exits.  It calls no allocating routine.
+ *   Limits: n_calls <= HX_STATIC_MAX_CALLS when topk > 0, topk <=
+ * HX_STATIC_MAX_TOPK; beyond them it returns HX_ERR_INVALID_ARG with a message
+ * naming the limit (with topk = 0 no intermediate buffer is needed and any
+ * batch size is accepted).  Inputs, outputs, options, stream semantics and
+ * error codes are those of hx_schedule_batch; hx_get_topk does not see this
+ * call's lists.
+ *   Set-up: the first call on a device looks up the array's device address
+ * (once per device, under a lock).  Make that first call before starting any
+ * stream capture.
+ *   Sharing: all handles and all calls on a device use the same array, which
+ * keeps whatever the previous call left; every call rewrites all it reads, so
+ * nothing needs clearing, but two calls that overlap on the GPU (different
+ * streams, or different handles) race on it.  Serialise them. */
+#define HX_STATIC_MAX_CALLS 16384
+#define HX_STATIC_MAX_TOPK      4
+int hx_schedule_batch_static(hx_cluster* h, const hx_call* calls, int n_calls,
+                             int32_t* out_assign, float* out_cost, void* stream);
+
 /* Borrowed device pointers to the top-K results of the last batch scored with
  * topk = K > 0: pairs int32[n_calls][K] (-1 = unused slot), costs
  * float[n_calls][K] (projected decode finish of that pair, +inf if unused),

@@ -56,6 +56,7 @@ def _load():
         "hx_set_options": [vp, C.POINTER(_Options)],
         "hx_schedule_batch": [vp, vp, ci, vp, vp, vp],
         "hx_schedule_batch_host": [vp, vp, ci, vp, vp, vp],
+        "hx_schedule_batch_static": [vp, vp, ci, vp, vp, vp],
         "hx_get_topk": [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp)],
         "hx_get_status": [vp, C.POINTER(ci), vp],
         "hx_enable_kernel_timing": [vp, ci],
@@ -146,6 +147,12 @@ def hx_set_options(h, score_mode=HX_MODE_COMPLETION, topk=0, commit=0, flags=0, 
 
 def hx_schedule_batch(h, calls_ptr, n_calls, out_assign_ptr, out_cost_ptr, stream=0):
     _check(_lib.hx_schedule_batch(h, calls_ptr, int(n_calls), out_assign_ptr, out_cost_ptr, stream), h)
+
+
+def hx_schedule_batch_static(h, calls_ptr, n_calls, out_assign_ptr, out_cost_ptr, stream=0):
+    """hx_schedule_batch without any allocation: intermediates live in a fixed device array
+    (at most 16384 calls with topk <= 4); see include/hx.h for who needs this and the rules."""
+    _check(_lib.hx_schedule_batch_static(h, calls_ptr, int(n_calls), out_assign_ptr, out_cost_ptr, stream), h)
 
 
 def hx_schedule_batch_host(h, calls, out_assign=None, out_cost=None, stream=0):

@@ -5,6 +5,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "hx_internal.h"
@@ -493,6 +494,93 @@ int hx_schedule_batch_host(hx_cluster* h, const hx_call* calls, int n_calls, int
     HX_TRY(cudaMemcpyAsync(out_assign, h->st_assign, (size_t)n_calls * sizeof(int32_t), cudaMemcpyDeviceToHost, s), "copy assign");
     HX_TRY(cudaMemcpyAsync(out_cost, h->st_cost, (size_t)n_calls * sizeof(float), cudaMemcpyDeviceToHost, s), "copy cost");
     HX_TRY(cudaStreamSynchronize(s), "cudaStreamSynchronize");
+    return HX_OK;
+}
+
+
+// ---------------------------------------------------------------------------
+// hx_schedule_batch_static: the same batch operation with every intermediate
+// buffer in a fixed device array that is part of the library image.
+// ---------------------------------------------------------------------------
+namespace {
+
+constexpr size_t kStaticAlign = 256;
+constexpr size_t static_round(size_t b) { return (b + kStaticAlign - 1) / kStaticAlign * kStaticAlign; }
+constexpr size_t kSC = HX_STATIC_MAX_CALLS, kSK = HX_STATIC_MAX_TOPK;
+constexpr size_t kStaticBytes =
+    3 * static_round(kSC * kSK * 4) +     // pair, cost, tpre
+    2 * static_round(kSC * 16) +          // dsel, od
+    4 * static_round(kSC * 4) +           // prio, mtok, ocall, om
+    static_round(kSC * 8) +               // okey
+    static_round((2048 + 3) * 4) +        // obase
+    static_round(4) +                     // n_acc
+    3 * static_round(kSC * 4);            // acc_rk, acc_p, acc_t
+
+// Held by every device that loads the library, until the process exits.
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];
+
+std::mutex g_static_mu;
+unsigned char* g_static_base[64] = {};    // device address of the array, per device ordinal
+
+}  // namespace
+
+int hx_schedule_batch_static(hx_cluster* h, const hx_call* calls, int n_calls, int32_t* out_assign,
+                             float* out_cost, void* stream) {
+    if (!h) return HX_ERR_INVALID_ARG;
+    if (n_calls < 0) return fail(h, HX_ERR_INVALID_ARG, "negative n_calls");
+    if (n_calls == 0) return HX_OK;
+    if (!calls || !out_assign || !out_cost) return fail(h, HX_ERR_INVALID_ARG, "NULL buffer");
+    if (reinterpret_cast<uintptr_t>(calls) % 16) return fail(h, HX_ERR_INVALID_ARG, "calls must be 16-byte aligned");
+    const hx_options& o = h->opts;
+    if (!(o.flags & HX_FLAG_NO_DAG) && !(h->dag_uploaded && h->cp_ready))
+        return fail(h, HX_ERR_NOT_READY, "horizons not computed: call hx_dag_upload and hx_critical_path, or set HX_FLAG_NO_DAG");
+    if (o.topk > 0 && n_calls > HX_STATIC_MAX_CALLS)
+        return fail(h, HX_ERR_INVALID_ARG, "hx_schedule_batch_static: more than HX_STATIC_MAX_CALLS (16384) calls in one batch; "
+                                           "split the batch or use hx_schedule_batch");
+    if (o.topk > HX_STATIC_MAX_TOPK)
+        return fail(h, HX_ERR_INVALID_ARG, "hx_schedule_batch_static: topk above HX_STATIC_MAX_TOPK (4); use hx_schedule_batch");
+    if (h->device < 0 || h->device >= 64) return fail(h, HX_ERR_INVALID_ARG, "device ordinal out of range");
+    DeviceGuard guard(h->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    unsigned char* base = nullptr;
+    {
+        // the array's name is only a host-side handle: ask the runtime for its address on this device, once
+        std::lock_guard<std::mutex> lock(g_static_mu);
+        if (!g_static_base[h->device]) {
+            void* p = nullptr;
+            HX_TRY(cudaGetSymbolAddress(&p, g_static_scratch), "cudaGetSymbolAddress(static scratch)");
+            g_static_base[h->device] = static_cast<unsigned char*>(p);
+        }
+        base = g_static_base[h->device];
+    }
+    HxTopkBufs b{};
+    b.K = o.topk;
+    b.cap_calls = HX_STATIC_MAX_CALLS;
+    size_t off = 0;
+    auto carve = [&](size_t bytes) { unsigned char* p = base + off; off += static_round(bytes); return p; };
+    b.pair = reinterpret_cast<int32_t*>(carve(kSC * kSK * 4));
+    b.cost = reinterpret_cast<float*>(carve(kSC * kSK * 4));
+    b.tpre = reinterpret_cast<float*>(carve(kSC * kSK * 4));
+    b.dsel = reinterpret_cast<uint4*>(carve(kSC * 16));
+    b.od = reinterpret_cast<uint4*>(carve(kSC * 16));
+    b.prio = reinterpret_cast<float*>(carve(kSC * 4));
+    b.mtok = reinterpret_cast<float*>(carve(kSC * 4));
+    b.ocall = reinterpret_cast<unsigned int*>(carve(kSC * 4));
+    b.om = reinterpret_cast<float*>(carve(kSC * 4));
+    b.okey = reinterpret_cast<unsigned long long*>(carve(kSC * 8));
+    b.obase = reinterpret_cast<unsigned int*>(carve((2048 + 3) * 4));
+    b.n_acc = reinterpret_cast<unsigned int*>(carve(4));
+    b.acc_rk = reinterpret_cast<unsigned int*>(carve(kSC * 4));
+    b.acc_p = reinterpret_cast<int*>(carve(kSC * 4));
+    b.acc_t = reinterpret_cast<float*>(carve(kSC * 4));
+    if (off != kStaticBytes) return fail(h, HX_ERR_INVALID_ARG, "internal: static scratch layout mismatch");
+    HxDagView dag{};
+    if (!(o.flags & HX_FLAG_NO_DAG))
+        dag = HxDagView{h->d_node_wf, h->forest.tail, h->forest.H, h->d_elapsed, h->forest.n_nodes, h->forest.n_workflows};
+    ScoreLaunch sl{calls, n_calls, out_assign, out_cost, o.score_mode, o.flags, o.topk, o.alpha};
+    HX_TRY(hx_launch_score(h->tab, dag, b, sl, h->n_sm, h->max_smem, h->status, s, &h->launches), "scoring kernel");
+    if (o.topk > 0)
+        HX_TRY(hx_launch_conflict(h->tab, b, n_calls, o.commit, out_assign, h->status, s, &h->launches), "conflict pass");
     return HX_OK;
 }
 
