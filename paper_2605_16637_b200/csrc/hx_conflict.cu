@@ -35,7 +35,7 @@ namespace {
 typedef unsigned long long u64;
 
 constexpr int kBins = 2048;
-constexpr int kWin = 256;          // calls per optimistic window (= block size of the pass)
+constexpr int kWin = 512;          // calls per optimistic window (= block size of the pass)
 constexpr int kCache = 4096;       // calls staged in shared memory ahead of the window
 constexpr unsigned kNone = 0xFFu;  // no candidate taken
 
@@ -74,7 +74,8 @@ __device__ void block_exclusive_scan(const unsigned* cnt, int n, unsigned* base,
 // key and the shift that maps a key to its bin.  Each thread keeps its first kKeep keys in
 // registers (one round trip to memory); the rest of a large batch is read again per pass.
 constexpr int kKeep = 16;
-__global__ void __launch_bounds__(1024) hx_order_bins_kernel(HxTopkBufs tk, int n) {
+__global__ void __launch_bounds__(1024) hx_order_bins_kernel(HxTopkBufs tk, int n, int staged) {
+    extern __shared__ __align__(16) u64 skey[];                   // [n] keys in bin order when they fit (staged)
     __shared__ unsigned hist[kBins], base[kBins + 1], tmp[33], lohi[2];
     const int tid = threadIdx.x, nthr = blockDim.x;
     for (int i = tid; i < kBins; i += nthr) hist[i] = 0;
@@ -98,27 +99,31 @@ __global__ void __launch_bounds__(1024) hx_order_bins_kernel(HxTopkBufs tk, int 
     const unsigned span = lohi[1] - lo;
     int shift = 0;
     while ((span >> shift) >= (unsigned)kBins) ++shift;
+    unsigned slot[kKeep];                                          // arrival number inside the bin
 #pragma unroll
-    for (int u = 0; u < kKeep; ++u) if (tid + u * nthr < n) atomicAdd(&hist[(keep[u] - lo) >> shift], 1u);
-    for (int c = tid + kKeep * nthr; c < n; c += nthr) atomicAdd(&hist[(key_of(kKeep, c) - lo) >> shift], 1u);
+    for (int u = 0; u < kKeep; ++u) slot[u] = tid + u * nthr < n ? atomicAdd(&hist[(keep[u] - lo) >> shift], 1u) : 0u;
+    for (int c = tid + kKeep * nthr; c < n; c += nthr)
+        tk.ocall[c] = atomicAdd(&hist[(key_of(kKeep, c) - lo) >> shift], 1u);   // parked until the bounds are known
     __syncthreads();
     block_exclusive_scan(hist, kBins, base, tmp);
     for (int i = tid; i <= kBins; i += nthr) tk.obase[i] = base[i];
     if (tid == 0) { tk.obase[kBins + 1] = lo; tk.obase[kBins + 2] = (unsigned)shift; }
-    for (int i = tid; i < kBins; i += nthr) hist[i] = 0;           // now the bin cursors
-    __syncthreads();
 #pragma unroll
     for (int u = 0; u < kKeep; ++u) {
         const int c = tid + u * nthr;
         if (c < n) {
-            const unsigned bin = (keep[u] - lo) >> shift;
-            tk.okey[base[bin] + atomicAdd(&hist[bin], 1u)] = ((u64)keep[u] << 32) | (unsigned)c;
+            const unsigned pos = base[(keep[u] - lo) >> shift] + slot[u];
+            const u64 v = ((u64)keep[u] << 32) | (unsigned)c;
+            if (staged) skey[pos] = v; else tk.okey[pos] = v;
         }
     }
     for (int c = tid + kKeep * nthr; c < n; c += nthr) {
         const unsigned key = key_of(kKeep, c);
-        const unsigned bin = (key - lo) >> shift;
-        tk.okey[base[bin] + atomicAdd(&hist[bin], 1u)] = ((u64)key << 32) | (unsigned)c;
+        tk.okey[base[(key - lo) >> shift] + tk.ocall[c]] = ((u64)key << 32) | (unsigned)c;
+    }
+    if (staged) {                                                  // scattered in shared memory, coalesced to global
+        __syncthreads();
+        for (int i = tid; i < n; i += nthr) tk.okey[i] = skey[i];
     }
 }
 
@@ -138,92 +143,135 @@ __global__ void hx_order_rank_kernel(HxTopkBufs tk, int n) {
     tk.od[rank] = tk.dsel[c];
 }
 
-// 2. The pass itself: one block of kWin threads.
+// 2. The pass itself: one block of kWin threads.  Capacities and demands are handled as
+// integers (token counts are integer-valued and below 2^24).  Calls none of whose candidates
+// fits the capacities committed so far can never obtain a pair (capacity only shrinks): they
+// are dropped, in parallel, while the next stretch of the visiting order is staged, so the
+// windows only hold calls that may still be placed.
 __global__ void __launch_bounds__(kWin) hx_conflict_kernel(HxTopkBufs tk, HxTables t, int n, int commit) {
     extern __shared__ __align__(16) unsigned sm[];
     constexpr int NW = kWin / 32;
+    constexpr int kScan = 4 * kWin;                             // ranks examined per staging step
     const int D = t.D, K = tk.K;
-    uint4* cd = reinterpret_cast<uint4*>(sm);                   // [kCache] candidate instances of the staged calls
-    float* cm = reinterpret_cast<float*>(cd + kCache);          // [kCache] their demands
-    float* free_s = cm + kCache;                                // [D] capacity left after the commits so far
-    float* wtot = free_s + D;                                   // [NW][D] demand per warp and instance
-    __shared__ int first_fail;
-    __shared__ unsigned wacc[NW];
+    uint4* cd = reinterpret_cast<uint4*>(sm);                   // [kCache] ring: candidate instances of the live calls
+    int* cm = reinterpret_cast<int*>(cd + kCache);              // [kCache] their demands
+    int* cr = cm + kCache;                                      // [kCache] their ranks
+    int* free_s = cr + kCache;                                  // [D] capacity left after the commits so far
+    int* dtot = free_s + D;                                     // [D] demand of the window per instance
+    __shared__ int first_fail, bad_d, wsum[NW + 1];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    for (int d = tid; d < D; d += kWin) free_s[d] = t.freeD[d];
-    for (int i = tid; i < NW * D; i += kWin) wtot[i] = 0.f;
+    for (int d = tid; d < D; d += kWin) { free_s[d] = __float2int_rd(t.freeD[d]); dtot[d] = 0; }
     if (tid == 0) first_fail = kWin;
-    int pos = 0, cache_lo = -kCache;
-    unsigned n_acc = 0;                                         // same value in every thread
-    while (pos < n) {
-        if (pos + kWin > cache_lo + kCache) {                   // stage the next calls: one round trip
-            __syncthreads();
-            cache_lo = pos;
-#pragma unroll
-            for (int u = 0; u < kCache / kWin; ++u) {
-                const int i = tid + u * kWin, r = pos + i;
-                cd[i] = r < n ? __ldcg(tk.od + r) : make_uint4(~0u, ~0u, ~0u, ~0u);
-                cm[i] = r < n ? __ldcg(tk.om + r) : 0.f;
-            }
-        }
-        __syncthreads();                                        // S0: staged data, capacities and zeroed totals visible
-        const int r = pos + tid, ci = r - cache_lo;
-        const bool active = r < n;
-        const float m = cm[ci];
-        // first candidate that fits the committed capacities
-        unsigned kt = kNone; int dt = -1;
-        if (active) {
-            const uint4 row = cd[ci];
-            const unsigned w[4] = {row.x, row.y, row.z, row.w};
-#pragma unroll
-            for (int k = HX_MAX_TOPK - 1; k >= 0; --k) {
-                const unsigned d = (w[k >> 1] >> ((k & 1) * 16)) & 0xFFFFu;
-                if (k < K && d != 0xFFFFu && free_s[d] >= m) { kt = k; dt = (int)d; }
-            }
-        }
-        // demand of the earlier lanes of this warp that picked the same instance: one warp scan
-        // per distinct instance
-        float cum = 0.f, incl = 0.f;
-        unsigned rem = __ballot_sync(0xffffffffu, dt >= 0);
-        while (rem) {
-            const int leader = __ffs(rem) - 1;
-            const int dl = __shfl_sync(0xffffffffu, dt, leader);
-            const bool mine = dt == dl;
-            float x = mine ? m : 0.f;
-            for (int off = 1; off < 32; off <<= 1) {
-                const float y = __shfl_up_sync(0xffffffffu, x, off);
-                if (lane >= off) x = __fadd_rn(x, y);
-            }
-            if (mine) { incl = x; cum = __fsub_rn(x, m); }
-            rem &= ~__ballot_sync(0xffffffffu, mine);
-        }
-        const unsigned peers = __match_any_sync(0xffffffffu, dt);
-        const bool last_peer = dt >= 0 && (peers >> lane) <= 1u;
-        if (last_peer) wtot[warp * D + dt] = incl;              // demand of this warp on dt
-        __syncthreads();                                        // S1
-        float before = cum;
-        if (dt >= 0) for (int w = 0; w < warp; ++w) before = __fadd_rn(before, wtot[w * D + dt]);
-        if (dt >= 0 && __fadd_rn(before, m) > free_s[dt]) atomicMin(&first_fail, tid);
-        __syncthreads();                                        // S2
-        const int f = first_fail;                               // calls before f decided as the sequential pass would
-        const bool acc = active && tid < f && dt >= 0;
-        // the last committing peer of each warp subtracts the demand of its warp's committing peers
-        const unsigned accm = __ballot_sync(0xffffffffu, acc);
-        if (acc && (((peers & accm) >> lane) <= 1u)) atomicAdd(&free_s[dt], -incl);   // exact: integer-valued
-        if (last_peer) wtot[warp * D + dt] = 0.f;
-        if (lane == 0) wacc[warp] = __popc(accm);
-        __syncthreads();                                        // S3
-        if (tid == 0) first_fail = kWin;
-        unsigned off = n_acc + __popc(accm & ((1u << lane) - 1u));
-        unsigned tot = 0;
-        for (int w = 0; w < NW; ++w) { const unsigned a = wacc[w]; tot += a; if (w < warp) off += a; }
-        if (acc) tk.acc_rk[off] = (unsigned)r | (kt << 24);     // obtained pairs, in visiting order
-        n_acc += tot;
-        pos += f < kWin ? f : kWin;
-    }
     __syncthreads();
+    auto first_fit = [&](const uint4& row, int m, unsigned& kt, int& dt) {
+        const unsigned w[4] = {row.x, row.y, row.z, row.w};
+        int fr[HX_MAX_TOPK]; unsigned dk[HX_MAX_TOPK];
+#pragma unroll
+        for (int k = 0; k < HX_MAX_TOPK; ++k) {
+            dk[k] = (w[k >> 1] >> ((k & 1) * 16)) & 0xFFFFu;
+            fr[k] = k < K ? free_s[min(dk[k], (unsigned)(D - 1))] : 0;
+        }
+        kt = kNone; dt = -1;
+#pragma unroll
+        for (int k = HX_MAX_TOPK - 1; k >= 0; --k)
+            if (k < K && dk[k] != 0xFFFFu && fr[k] >= m) { kt = k; dt = (int)dk[k]; }
+    };
+    int scan = 0;                                               // next rank to examine
+    unsigned head = 0, tail = 0;                                // live calls staged: ring positions [head, tail)
+    unsigned n_acc = 0;                                         // the four values are the same in every thread
+    while (head != tail || scan < n) {
+        while ((int)(tail - head) < kWin && scan < n) {         // stage: keep the calls that may still fit
+            uint4 row[4]; int mm[4]; bool live[4]; unsigned cnt = 0;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int r = scan + 4 * tid + u;
+                row[u] = r < n ? __ldcg(tk.od + r) : make_uint4(~0u, ~0u, ~0u, ~0u);
+                mm[u] = r < n ? __float2int_ru(__ldcg(tk.om + r)) : 0;
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                unsigned kt; int dt;
+                first_fit(row[u], mm[u], kt, dt);
+                live[u] = scan + 4 * tid + u < n && dt >= 0;
+                cnt += live[u];
+            }
+            unsigned x = cnt;                                   // ordered compaction into the ring
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const unsigned y = __shfl_up_sync(0xffffffffu, x, off);
+                if (lane >= off) x += y;
+            }
+            if (lane == 31) wsum[warp] = (int)x;
+            __syncthreads();
+            unsigned before = 0, total = 0;
+#pragma unroll
+            for (int w = 0; w < NW; ++w) { const unsigned a = (unsigned)wsum[w]; total += a; before += w < warp ? a : 0u; }
+            unsigned o = tail + before + x - cnt;
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (live[u]) { const unsigned i = o++ & (kCache - 1); cd[i] = row[u]; cm[i] = mm[u]; cr[i] = scan + 4 * tid + u; }
+            tail += total;
+            scan += kScan;
+            __syncthreads();
+        }
+        const unsigned nwin = min((unsigned)kWin, tail - head);
+        if (nwin == 0) break;
+        const bool active = (unsigned)tid < nwin;
+        const unsigned ci = (head + tid) & (kCache - 1);
+        const int m = active ? cm[ci] : 0;
+        unsigned kt = kNone; int dt = -1;
+        if (active) first_fit(cd[ci], m, kt, dt);               // first candidate that fits the committed capacities
+        if (dt >= 0) atomicAdd(&dtot[dt], m);                   // demand of the window per instance
+        __syncthreads();                                        // S1
+        const bool over = dt >= 0 && dtot[dt] > free_s[dt];
+        int f = kWin;
+        if (__syncthreads_or(over)) {                           // S2: some instance cannot take the whole window
+            // ordered demand ahead of the calls that picked an overflowing instance, one instance at a time
+            int prev = -1;
+            for (;;) {
+                if (tid == 0) bad_d = 0x7fffffff;
+                __syncthreads();
+                if (over && dt > prev) atomicMin(&bad_d, dt);
+                __syncthreads();
+                const int bd = bad_d;
+                if (bd == 0x7fffffff) break;
+                const bool mine = dt == bd;
+                int x = mine ? m : 0;                           // inclusive prefix over the block, in call order
+#pragma unroll
+                for (int off = 1; off < 32; off <<= 1) {
+                    const int y = __shfl_up_sync(0xffffffffu, x, off);
+                    if (lane >= off) x += y;
+                }
+                if (lane == 31) wsum[warp] = x;
+                __syncthreads();
+                int before = 0;
+#pragma unroll
+                for (int w = 0; w < NW; ++w) before += w < warp ? wsum[w] : 0;
+                if (mine && before + x > free_s[bd]) atomicMin(&first_fail, tid);
+                prev = bd;
+            }
+            f = first_fail;                                     // calls before f decided as the sequential pass would
+            __syncthreads();
+            if (tid == 0) first_fail = kWin;
+        }
+        for (int d = tid; d < D; d += kWin) dtot[d] = 0;
+        const bool acc = active && tid < f && dt >= 0;
+        if (acc) atomicSub(&free_s[dt], m);
+        const unsigned accm = __ballot_sync(0xffffffffu, acc);
+        if (lane == 0) wsum[warp] = __popc(accm);
+        const unsigned tot = __syncthreads_count(acc);          // S3
+        if (accm) {
+            unsigned off = n_acc + __popc(accm & ((1u << lane) - 1u));
+#pragma unroll
+            for (int w = 0; w < NW; ++w) off += w < warp ? (unsigned)wsum[w] : 0u;
+            if (acc) tk.acc_rk[off] = (unsigned)cr[ci] | (kt << 24);   // obtained pairs, in visiting order
+        }
+        n_acc += tot;
+        head += (unsigned)f < nwin ? (unsigned)f : nwin;
+        __syncthreads();                                        // S4: capacities and totals settled for the next step
+    }
     if (tid == 0) *tk.n_acc = n_acc;
-    if (commit) for (int d = tid; d < D; d += kWin) t.freeD[d] = free_s[d];
+    if (commit) for (int d = tid; d < D; d += kWin) t.freeD[d] = __int2float_rn(free_s[d]);
 }
 
 // 3. Publish the obtained pairs; gather prefill instance and prefill time in visiting order.
@@ -239,15 +287,21 @@ __global__ void hx_finish_kernel(HxTopkBufs tk, int D, int32_t* out_assign) {
 }
 
 // 4. Prefill queues: thread p adds, in visiting order, the prefill times of the calls that obtained p.
-__global__ void hx_qsum_kernel(HxTopkBufs tk, HxTables t) {
+// The list is staged through shared memory in chunks; every thread scans every chunk.
+constexpr int kQChunk = 2048;
+__global__ void __launch_bounds__(256) hx_qsum_kernel(HxTopkBufs tk, HxTables t) {
+    __shared__ int sp[kQChunk];
+    __shared__ float st[kQChunk];
     const int p = blockIdx.x * blockDim.x + threadIdx.x;
     const unsigned na = *tk.n_acc;
     float q = p < t.P ? t.qP[p] : 0.f;
+    for (unsigned c0 = 0; c0 < na; c0 += kQChunk) {
+        const unsigned len = min((unsigned)kQChunk, na - c0);
+        __syncthreads();
+        for (unsigned i = threadIdx.x; i < len; i += blockDim.x) { sp[i] = tk.acc_p[c0 + i]; st[i] = tk.acc_t[c0 + i]; }
+        __syncthreads();
 #pragma unroll 8
-    for (unsigned i = 0; i < na; ++i) {
-        const int pi = __ldg(tk.acc_p + i);
-        const float ti = __ldg(tk.acc_t + i);
-        if (pi == p) q = __fadd_rn(q, ti);
+        for (unsigned i = 0; i < len; ++i) if (sp[i] == p) q = __fadd_rn(q, st[i]);
     }
     if (p < t.P) t.qP[p] = q;
 }
@@ -259,9 +313,15 @@ cudaError_t hx_launch_conflict(const HxTables& t, const HxTopkBufs& tk, int n_ca
                                long long* launches) {
     (void)status;
     const int D = t.D, P = t.P;
-    hx_order_bins_kernel<<<1, 1024, 0, stream>>>(tk, n_calls);
+    const int staged = n_calls <= 16 * 1024;                       // every key held in registers, list fits shared memory
+    const size_t smB = staged ? (size_t)n_calls * 8 : 0;
+    if (smB > 24 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(hx_order_bins_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smB);
+        if (e != cudaSuccess) return e;
+    }
+    hx_order_bins_kernel<<<1, 1024, smB, stream>>>(tk, n_calls, staged);
     hx_order_rank_kernel<<<(n_calls + 127) / 128, 128, 0, stream>>>(tk, n_calls);
-    const size_t smC = (size_t)kCache * 20 + (size_t)(D + (kWin / 32) * D) * 4;
+    const size_t smC = (size_t)kCache * 24 + (size_t)(2 * D) * 4;
     if (smC > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(hx_conflict_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smC);
         if (e != cudaSuccess) return e;
@@ -270,7 +330,7 @@ cudaError_t hx_launch_conflict(const HxTables& t, const HxTopkBufs& tk, int n_ca
     hx_finish_kernel<<<(n_calls + 255) / 256, 256, 0, stream>>>(tk, D, out_assign);
     *launches += 4;
     if (commit) {
-        hx_qsum_kernel<<<(P + 31) / 32, 32, 0, stream>>>(tk, t);
+        hx_qsum_kernel<<<(P + 255) / 256, 256, 0, stream>>>(tk, t);
         *launches += 1;
     }
     return cudaGetLastError();
