@@ -205,6 +205,9 @@ def run_cuda(args):
     sptr = stream.cuda_stream
     h = gc.h
 
+    ptrs = [(calls_dev[i * chunk:(i + 1) * chunk].data_ptr(), out_assign[i * chunk:(i + 1) * chunk].data_ptr(),
+             out_cost[i * chunk:(i + 1) * chunk].data_ptr()) for i in range(n_chunks)]
+
     def step_device(chunk_events=None):
         hx.hx_critical_path(h, sptr)
         hx.hx_cluster_update_loads(h, qP0, qD0, free0, sptr)
@@ -212,9 +215,7 @@ def run_cuda(args):
             if chunk_events is not None:
                 chunk_events[i][0].record(stream)
             hx.hx_cluster_update_loads(h, None, None, free0, sptr)
-            lo = i * chunk
-            hx.hx_schedule_batch(h, calls_dev[lo:lo + chunk].data_ptr(), chunk,
-                                 out_assign[lo:lo + chunk].data_ptr(), out_cost[lo:lo + chunk].data_ptr(), sptr)
+            hx.hx_schedule_batch(h, ptrs[i][0], chunk, ptrs[i][1], ptrs[i][2], sptr)
             if chunk_events is not None:
                 chunk_events[i][1].record(stream)
 

@@ -148,11 +148,12 @@ __global__ void hx_order_rank_kernel(HxTopkBufs tk, int n) {
 // fits the capacities committed so far can never obtain a pair (capacity only shrinks): they
 // are dropped, in parallel, while the next stretch of the visiting order is staged, so the
 // windows only hold calls that may still be placed.
+template <int KT>   // candidate slots examined per call: K rounded up to 1, 2, 4 or 8
 __global__ void __launch_bounds__(kWin) hx_conflict_kernel(HxTopkBufs tk, HxTables t, int n, int commit) {
     extern __shared__ __align__(16) unsigned sm[];
     constexpr int NW = kWin / 32;
     constexpr int kScan = 4 * kWin;                             // ranks examined per staging step
-    const int D = t.D, K = tk.K;
+    const int D = t.D;
     uint4* cd = reinterpret_cast<uint4*>(sm);                   // [kCache] ring: candidate instances of the live calls
     int* cm = reinterpret_cast<int*>(cd + kCache);              // [kCache] their demands
     int* cr = cm + kCache;                                      // [kCache] their ranks
@@ -165,29 +166,37 @@ __global__ void __launch_bounds__(kWin) hx_conflict_kernel(HxTopkBufs tk, HxTabl
     __syncthreads();
     auto first_fit = [&](const uint4& row, int m, unsigned& kt, int& dt) {
         const unsigned w[4] = {row.x, row.y, row.z, row.w};
-        int fr[HX_MAX_TOPK]; unsigned dk[HX_MAX_TOPK];
+        int fr[KT]; unsigned dk[KT];
 #pragma unroll
-        for (int k = 0; k < HX_MAX_TOPK; ++k) {
-            dk[k] = (w[k >> 1] >> ((k & 1) * 16)) & 0xFFFFu;
-            fr[k] = k < K ? free_s[min(dk[k], (unsigned)(D - 1))] : 0;
+        for (int k = 0; k < KT; ++k) {
+            dk[k] = (w[k >> 1] >> ((k & 1) * 16)) & 0xFFFFu;   // slots beyond K hold 0xFFFF
+            fr[k] = free_s[min(dk[k], (unsigned)(D - 1))];
         }
         kt = kNone; dt = -1;
 #pragma unroll
-        for (int k = HX_MAX_TOPK - 1; k >= 0; --k)
-            if (k < K && dk[k] != 0xFFFFu && fr[k] >= m) { kt = k; dt = (int)dk[k]; }
+        for (int k = KT - 1; k >= 0; --k)
+            if (dk[k] != 0xFFFFu && fr[k] >= m) { kt = k; dt = (int)dk[k]; }
     };
     int scan = 0;                                               // next rank to examine
     unsigned head = 0, tail = 0;                                // live calls staged: ring positions [head, tail)
     unsigned n_acc = 0;                                         // the four values are the same in every thread
+    // the stretch [scan, scan + kScan) is always in flight one step ahead of its use
+    uint4 nrow[4]; float nm[4];
+    auto prefetch = [&](int from) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int r = from + 4 * tid + u;
+            nrow[u] = r < n ? __ldcg(tk.od + r) : make_uint4(~0u, ~0u, ~0u, ~0u);
+            nm[u] = r < n ? __ldcg(tk.om + r) : 0.f;
+        }
+    };
+    prefetch(0);
     while (head != tail || scan < n) {
         while ((int)(tail - head) < kWin && scan < n) {         // stage: keep the calls that may still fit
             uint4 row[4]; int mm[4]; bool live[4]; unsigned cnt = 0;
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int r = scan + 4 * tid + u;
-                row[u] = r < n ? __ldcg(tk.od + r) : make_uint4(~0u, ~0u, ~0u, ~0u);
-                mm[u] = r < n ? __float2int_ru(__ldcg(tk.om + r)) : 0;
-            }
+            for (int u = 0; u < 4; ++u) { row[u] = nrow[u]; mm[u] = __float2int_ru(nm[u]); }
+            prefetch(scan + kScan);
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 unsigned kt; int dt;
@@ -286,24 +295,33 @@ __global__ void hx_finish_kernel(HxTopkBufs tk, int D, int32_t* out_assign) {
     tk.acc_t[i] = tk.tpre[(size_t)c * tk.K + k];
 }
 
-// 4. Prefill queues: thread p adds, in visiting order, the prefill times of the calls that obtained p.
-// The list is staged through shared memory in chunks; every thread scans every chunk.
+// 4. Prefill queues: warp p adds, in visiting order, the prefill times of the calls that obtained p.
+// The block stages the list in shared memory; a warp looks at 32 entries at a time and adds the
+// matching ones in order.
 constexpr int kQChunk = 2048;
 __global__ void __launch_bounds__(256) hx_qsum_kernel(HxTopkBufs tk, HxTables t) {
     __shared__ int sp[kQChunk];
     __shared__ float st[kQChunk];
-    const int p = blockIdx.x * blockDim.x + threadIdx.x;
+    const int p = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     const unsigned na = *tk.n_acc;
     float q = p < t.P ? t.qP[p] : 0.f;
     for (unsigned c0 = 0; c0 < na; c0 += kQChunk) {
         const unsigned len = min((unsigned)kQChunk, na - c0);
         __syncthreads();
-        for (unsigned i = threadIdx.x; i < len; i += blockDim.x) { sp[i] = tk.acc_p[c0 + i]; st[i] = tk.acc_t[c0 + i]; }
+        for (unsigned i = threadIdx.x; i < len; i += blockDim.x) { sp[i] = __ldg(tk.acc_p + c0 + i); st[i] = __ldg(tk.acc_t + c0 + i); }
         __syncthreads();
-#pragma unroll 8
-        for (unsigned i = 0; i < len; ++i) if (sp[i] == p) q = __fadd_rn(q, st[i]);
+        for (unsigned i0 = 0; i0 < len; i0 += 32) {
+            const unsigned i = i0 + lane;
+            const float ti = i < len ? st[i] : 0.f;
+            unsigned hit = __ballot_sync(0xffffffffu, i < len && sp[i] == p);
+            while (hit) {
+                const int j = __ffs(hit) - 1;
+                q = __fadd_rn(q, __shfl_sync(0xffffffffu, ti, j));
+                hit &= hit - 1;
+            }
+        }
     }
-    if (p < t.P) t.qP[p] = q;
+    if (lane == 0 && p < t.P) t.qP[p] = q;
 }
 
 }  // namespace
@@ -315,22 +333,22 @@ cudaError_t hx_launch_conflict(const HxTables& t, const HxTopkBufs& tk, int n_ca
     const int D = t.D, P = t.P;
     const int staged = n_calls <= 16 * 1024;                       // every key held in registers, list fits shared memory
     const size_t smB = staged ? (size_t)n_calls * 8 : 0;
-    if (smB > 24 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(hx_order_bins_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smB);
-        if (e != cudaSuccess) return e;
-    }
+    static size_t allowed_bins[64];
+    cudaError_t e = hx_opt_in_smem(hx_order_bins_kernel, smB, allowed_bins, 24 * 1024);
+    if (e != cudaSuccess) return e;
     hx_order_bins_kernel<<<1, 1024, smB, stream>>>(tk, n_calls, staged);
     hx_order_rank_kernel<<<(n_calls + 127) / 128, 128, 0, stream>>>(tk, n_calls);
     const size_t smC = (size_t)kCache * 24 + (size_t)(2 * D) * 4;
-    if (smC > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(hx_conflict_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smC);
-        if (e != cudaSuccess) return e;
-    }
-    hx_conflict_kernel<<<1, kWin, smC, stream>>>(tk, t, n_calls, commit);
+    auto pass = tk.K <= 1 ? hx_conflict_kernel<1> : tk.K <= 2 ? hx_conflict_kernel<2>
+              : tk.K <= 4 ? hx_conflict_kernel<4> : hx_conflict_kernel<8>;
+    static size_t allowed_pass[4][64];
+    e = hx_opt_in_smem(pass, smC, allowed_pass[tk.K <= 1 ? 0 : tk.K <= 2 ? 1 : tk.K <= 4 ? 2 : 3], 40 * 1024);
+    if (e != cudaSuccess) return e;
+    pass<<<1, kWin, smC, stream>>>(tk, t, n_calls, commit);
     hx_finish_kernel<<<(n_calls + 255) / 256, 256, 0, stream>>>(tk, D, out_assign);
     *launches += 4;
     if (commit) {
-        hx_qsum_kernel<<<(P + 255) / 256, 256, 0, stream>>>(tk, t);
+        hx_qsum_kernel<<<(P + 7) / 8, 256, 0, stream>>>(tk, t);
         *launches += 1;
     }
     return cudaGetLastError();

@@ -130,16 +130,16 @@ cudaError_t hx_launch_cpath(const HxForestDev& f, const HxCpClass* classes, int 
             const unsigned grid = (c.count + c.wfs_per_block - 1) / c.wfs_per_block;
             if (c.threads_per_wf == 32) {
                 {   // static + dynamic shared memory may exceed the 48 KB default
-                    cudaError_t e = cudaFuncSetAttribute(hx_cpath_staged_kernel<true>,
-                                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+                    static size_t allowed[64];
+                    cudaError_t e = hx_opt_in_smem(hx_cpath_staged_kernel<true>, smem, allowed, 40 * 1024);
                     if (e != cudaSuccess) return e;
                 }
                 hx_cpath_staged_kernel<true><<<grid, threads, smem, stream>>>(
                     f, c.wf_ids, c.count, 32, c.wfs_per_block, (uint32_t)c.smem_per_wf);
             } else {
                 {   // static + dynamic shared memory may exceed the 48 KB default
-                    cudaError_t e = cudaFuncSetAttribute(hx_cpath_staged_kernel<false>,
-                                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+                    static size_t allowed[64];
+                    cudaError_t e = hx_opt_in_smem(hx_cpath_staged_kernel<false>, smem, allowed, 40 * 1024);
                     if (e != cudaSuccess) return e;
                 }
                 hx_cpath_staged_kernel<false><<<grid, threads, smem, stream>>>(

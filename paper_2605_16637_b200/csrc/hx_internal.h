@@ -113,4 +113,20 @@ struct HxCpClass {
 cudaError_t hx_launch_cpath(const HxForestDev& f, const HxCpClass* classes, int n_classes,
                             cudaStream_t stream, long long* launches);
 
+// Opt a kernel in to `bytes` of dynamic shared memory, once per device and size: the attribute
+// call is too slow to repeat on every launch.  `allowed` is a per-kernel table of 64 entries
+// that starts at the size the kernel may use without opting in.
+template <class Kernel>
+inline cudaError_t hx_opt_in_smem(Kernel kernel, size_t bytes, size_t* allowed, size_t without_opt_in) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    dev &= 63;
+    if (allowed[dev] < without_opt_in) allowed[dev] = without_opt_in;
+    if (bytes <= allowed[dev]) return cudaSuccess;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (e == cudaSuccess) allowed[dev] = bytes;
+    return e;
+}
+
 #endif  // HX_INTERNAL_H_

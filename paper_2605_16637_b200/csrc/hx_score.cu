@@ -90,7 +90,7 @@ __device__ __forceinline__ void group_next(const float* frow, int nq, int t, uns
 
 // Lowest prefill index whose candidate on decode column d finishes exactly at v.
 __device__ __forceinline__ int group_rescan(const HxTables& T, const float* qPs, const int* typePs,
-                                            const float* tpre_c, float kvB, float qd, float Dd,
+                                            const float* tpre_c, int tstride, float kvB, float qd, float Dd,
                                             int d, float v, int t, unsigned gmask) {
     int best = HX_NONE;
     const float4* lrow = reinterpret_cast<const float4*>(T.invLT + (size_t)d * T.Ppad);
@@ -101,7 +101,7 @@ __device__ __forceinline__ int group_rescan(const HxTables& T, const float* qPs,
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             const int p = 4 * q + u;
-            const float A = __fadd_rn(qPs[p], tpre_c[typePs[p]]);
+            const float A = __fadd_rn(qPs[p], tpre_c[typePs[p] * tstride]);
             const float r = __fmaf_rn(kvB, l[u], A);
             const float f = __fadd_rn(fmaxf(r, qd), Dd);
             if (f == v && p < best) best = p;
@@ -142,6 +142,7 @@ __device__ __forceinline__ int group_rescan_smem(const float* acol, int astride,
                                                  int nq, float kvB, float qd, float Dd, float v, int t,
                                                  unsigned gmask) {
     int best = HX_NONE;
+#pragma unroll 8
     for (int q = nq - 1; q >= 0; --q) {
         const float f = __fadd_rn(fmaxf(__fmaf_rn(kvB, lcol[q * lstride + t], acol[q * astride + t]), qd), Dd);
         if (f == v) best = 4 * q + t;
@@ -175,8 +176,8 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
     float* Fs = reinterpret_cast<float*>(smem + prm.offF);        // [TCB][FS] (may alias As)
     float* kvBs = reinterpret_cast<float*>(smem + prm.offCall);   // [TCB]
     float* mtoks = kvBs + TCB;                                    // [TCB]
-    float* tpres = mtoks + TCB;                                   // [TCB][G]
-    float* tdecs = tpres + TCB * G;                               // [TCB][G]
+    float* tpres = mtoks + TCB;                                   // [G][TCB]
+    float* tdecs = tpres + TCB * G;                               // [G][TCB]
     float* qPs = reinterpret_cast<float*>(smem + prm.offInst);    // [Ppad]
     int* typePs = reinterpret_cast<int*>(qPs + Ppad);             // [Ppad]
     float* qDs = reinterpret_cast<float*>(typePs + Ppad);         // [Dpad]
@@ -193,17 +194,22 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
         capDs[d] = d < D ? T.capD[d] : -1.0f;
         typeDs[d] = d < D ? T.typeD[d] : 0;
     }
+    // asynchronous copies (no register staging): the wait is just before the barrier that precedes the first use
     auto load_LT = [&](int pc0) {
         const int nq = PC >> 2;
-#pragma unroll 4
         for (int idx = tid; idx < Dpad * nq; idx += nthr) {
             const int q = idx / Dpad, d = idx - q * Dpad;
             const int p = pc0 + 4 * q;
-            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (d < D && p < Ppad) v = __ldg(reinterpret_cast<const float4*>(T.invLT + (size_t)d * Ppad + p));
-            *reinterpret_cast<float4*>(LTs + 4 * idx) = v;
+            float* dst = LTs + 4 * idx;
+            if (d < D && p < Ppad) {
+                const unsigned sa = (unsigned)__cvta_generic_to_shared(dst);
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(sa), "l"(T.invLT + (size_t)d * Ppad + p) : "memory");
+            } else {
+                *reinterpret_cast<float4*>(dst) = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
         }
     };
+    auto lt_wait = [] { asm volatile("cp.async.wait_all;" ::: "memory"); };
     if (prm.nChunks == 1) load_LT(0);
 
     for (int tile = blockIdx.x; tile < prm.nTiles; tile += gridDim.x) {
@@ -224,10 +230,11 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
             const float ctx = __fmaf_rn(0.5f, __fsub_rn(o, 1.0f), n);
             const float step = __fmaf_rn(kappa, ctx, omega);
             const float iF = __ldg(T.invF + g), iB = __ldg(T.invB + g);
-            tpres[idx] = fmaxf(__fmul_rn(__fmul_rn(n, phi), iF), __fmul_rn(__fadd_rn(omega, kvB), iB));
-            tdecs[idx] = __fmul_rn(__fmul_rn(o, step), iB);
+            tpres[g * TCB + c] = fmaxf(__fmul_rn(__fmul_rn(n, phi), iF), __fmul_rn(__fadd_rn(omega, kvB), iB));
+            tdecs[g * TCB + c] = __fmul_rn(__fmul_rn(o, step), iB);
             if (g == 0) { kvBs[c] = kvB; mtoks[c] = __fadd_rn(n, o); }
         }
+        lt_wait();
         __syncthreads();
 
         float acc[TC][TD];
@@ -246,16 +253,20 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
             if (prm.nChunks > 1) load_LT(pc0);
             {   // prefill finish times A[c][p] of this chunk
                 const int nq = PC >> 2;
+                const int dq = nthr / TCB, dc = nthr - dq * TCB;
+                int q = tid / TCB, c = tid - q * TCB;
                 for (int idx = tid; idx < TCB * nq; idx += nthr) {
-                    const int q = idx / TCB, c = idx - q * TCB;
                     const int p = pc0 + 4 * q;
                     float a[4];
 #pragma unroll
                     for (int u = 0; u < 4; ++u)
-                        a[u] = (p + u < Ppad) ? __fadd_rn(qPs[p + u], tpres[c * G + typePs[p + u]]) : HX_INF;
+                        a[u] = (p + u < Ppad) ? __fadd_rn(qPs[p + u], tpres[typePs[p + u] * TCB + c]) : HX_INF;
                     *reinterpret_cast<float4*>(As + 4 * idx) = make_float4(a[0], a[1], a[2], a[3]);
+                    q += dq; c += dc;
+                    if (c >= TCB) { c -= TCB; ++q; }
                 }
             }
+            lt_wait();
             __syncthreads();
             const ulonglong2* ap = reinterpret_cast<const ulonglong2*>(As) + wc * (TC * LC) + cg;
             const ulonglong2* lp = reinterpret_cast<const ulonglong2*>(LTs) + wd * (TD * LD) + dg;
@@ -290,7 +301,7 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
 #pragma unroll
             for (int i = 0; i < TC; ++i) {
                 const int c = wc * (TC * LC) + cg + LC * i;
-                const float Dd = (mtoks[c] <= cap) ? tdecs[c * G + ty] : HX_INF;
+                const float Dd = (mtoks[c] <= cap) ? tdecs[ty * TCB + c] : HX_INF;
                 Fs[c * FS + d] = __fadd_rn(fmaxf(acc[i][j], qd), Dd);
             }
         }
@@ -306,12 +317,12 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
             const int cs = live ? c : 0;
             const float* frow = Fs + cs * FS;
             const float kvB = kvBs[cs], m = mtoks[cs];
-            const float* tpre_c = tpres + cs * G;
+            const float* tpre_c = tpres + cs;                 // class g at tpre_c[g * TCB]
             auto rescan = [&](int d, float v) {
-                const float Dd = (m <= capDs[d]) ? tdecs[cs * G + typeDs[d]] : HX_INF;
+                const float Dd = (m <= capDs[d]) ? tdecs[typeDs[d] * TCB + cs] : HX_INF;
                 return resident
                     ? group_rescan_smem(As + 4 * cs, 4 * TCB, LTs + 4 * d, 4 * Dpad, Ppad >> 2, kvB, qDs[d], Dd, v, t, gmask)
-                    : group_rescan(T, qPs, typePs, tpre_c, kvB, qDs[d], Dd, d, v, t, gmask);
+                    : group_rescan(T, qPs, typePs, tpre_c, TCB, kvB, qDs[d], Dd, d, v, t, gmask);
             };
             float v0 = HX_INF; int jbest = HX_NONE;
             int sel_pair[HX_MAX_TOPK], sel_d[HX_MAX_TOPK]; float sel_cost[HX_MAX_TOPK], sel_tpre[HX_MAX_TOPK];
@@ -331,6 +342,39 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
                         pv = v; pd = d;
                     }
                 }
+            } else if (Dpad <= 128) {
+                // the lane's share of the row (every fourth 16-byte unit) is held in registers; each
+                // round takes the smallest (finish, d) not taken yet
+                float vals[32];
+#pragma unroll
+                for (int it = 0; it < 8; ++it) {
+                    const int q = t + 4 * it;
+                    float4 f4 = make_float4(HX_INF, HX_INF, HX_INF, HX_INF);
+                    if (4 * q < Dpad) f4 = *reinterpret_cast<const float4*>(frow + 4 * q);
+                    vals[4 * it] = f4.x; vals[4 * it + 1] = f4.y; vals[4 * it + 2] = f4.z; vals[4 * it + 3] = f4.w;
+                }
+                unsigned taken = 0;
+                for (int k = 0; k < K; ++k) {
+                    float v = HX_INF; int bi = -1;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if (!((taken >> i) & 1u) && vals[i] < v) { v = vals[i]; bi = i; }
+                    int d = bi < 0 ? HX_NONE : 16 * (bi >> 2) + 4 * t + (bi & 3);
+                    const int myd = d;
+#pragma unroll
+                    for (int off = 1; off <= 2; off <<= 1) {
+                        const float ov = __shfl_xor_sync(gmask, v, off);
+                        const int od = __shfl_xor_sync(gmask, d, off);
+                        if (ov < v || (ov == v && od < d)) { v = ov; d = od; }
+                    }
+                    if (d == HX_NONE) break;              // nothing (feasible) left
+                    if (d == myd) taken |= 1u << bi;
+                    if (k == 0) v0 = v;
+                    const int p = rescan(d, v);
+#pragma unroll
+                    for (int k2 = 0; k2 < HX_MAX_TOPK; ++k2)
+                        if (k2 == k) { sel_pair[k2] = p * D + d; sel_d[k2] = d; sel_cost[k2] = v; sel_tpre[k2] = tpre_c[typePs[p] * TCB]; }
+                }
             } else {
                 float pv = -1.0f; int pd = -1;
                 for (int k = 0; k < K; ++k) {
@@ -341,7 +385,7 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
                     const int p = rescan(d, v);
 #pragma unroll
                     for (int k2 = 0; k2 < HX_MAX_TOPK; ++k2)
-                        if (k2 == k) { sel_pair[k2] = p * D + d; sel_d[k2] = d; sel_cost[k2] = v; sel_tpre[k2] = tpre_c[typePs[p]]; }
+                        if (k2 == k) { sel_pair[k2] = p * D + d; sel_d[k2] = d; sel_cost[k2] = v; sel_tpre[k2] = tpre_c[typePs[p] * TCB]; }
                     pv = v; pd = d;
                 }
             }
@@ -393,7 +437,8 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
 
 template <int TC, int TD, int LD>
 cudaError_t launch_one(const ScoreParams& prm, int grid, int threads, size_t smem, cudaStream_t stream) {
-    cudaError_t e = cudaFuncSetAttribute(hx_score_kernel<TC, TD, LD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    static size_t allowed[64];
+    cudaError_t e = hx_opt_in_smem(hx_score_kernel<TC, TD, LD>, smem, allowed, 0);
     if (e != cudaSuccess) return e;
     hx_score_kernel<TC, TD, LD><<<grid, threads, smem, stream>>>(prm);
     return cudaGetLastError();
