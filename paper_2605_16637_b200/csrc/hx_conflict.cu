@@ -35,7 +35,7 @@ namespace {
 typedef unsigned long long u64;
 
 constexpr int kBins = 2048;
-constexpr int kWin = 512;          // calls per optimistic window (= block size of the pass)
+constexpr int kWin = 256;          // calls per optimistic window (= block size of the pass)
 constexpr int kCache = 4096;       // calls staged in shared memory ahead of the window
 constexpr unsigned kNone = 0xFFu;  // no candidate taken
 
@@ -296,13 +296,15 @@ __global__ void hx_finish_kernel(HxTopkBufs tk, int D, int32_t* out_assign) {
 }
 
 // 4. Prefill queues: warp p adds, in visiting order, the prefill times of the calls that obtained p.
-// The block stages the list in shared memory; a warp looks at 32 entries at a time and adds the
-// matching ones in order.
-constexpr int kQChunk = 2048;
-__global__ void __launch_bounds__(256) hx_qsum_kernel(HxTopkBufs tk, HxTables t) {
+// The block stages the list in shared memory chunk by chunk; each warp compacts the entries of
+// its instance (ballot prefix keeps the order) and one lane adds them one after the other.
+constexpr int kQChunk = 1024, kQWarps = 8;
+__global__ void __launch_bounds__(32 * kQWarps) hx_qsum_kernel(HxTopkBufs tk, HxTables t) {
     __shared__ int sp[kQChunk];
     __shared__ float st[kQChunk];
-    const int p = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    __shared__ float mine[kQWarps][kQChunk];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int p = blockIdx.x * kQWarps + warp;
     const unsigned na = *tk.n_acc;
     float q = p < t.P ? t.qP[p] : 0.f;
     for (unsigned c0 = 0; c0 < na; c0 += kQChunk) {
@@ -310,16 +312,20 @@ __global__ void __launch_bounds__(256) hx_qsum_kernel(HxTopkBufs tk, HxTables t)
         __syncthreads();
         for (unsigned i = threadIdx.x; i < len; i += blockDim.x) { sp[i] = __ldg(tk.acc_p + c0 + i); st[i] = __ldg(tk.acc_t + c0 + i); }
         __syncthreads();
+        unsigned cnt = 0;
         for (unsigned i0 = 0; i0 < len; i0 += 32) {
             const unsigned i = i0 + lane;
-            const float ti = i < len ? st[i] : 0.f;
-            unsigned hit = __ballot_sync(0xffffffffu, i < len && sp[i] == p);
-            while (hit) {
-                const int j = __ffs(hit) - 1;
-                q = __fadd_rn(q, __shfl_sync(0xffffffffu, ti, j));
-                hit &= hit - 1;
-            }
+            const bool hit = i < len && sp[i] == p;
+            const unsigned b = __ballot_sync(0xffffffffu, hit);
+            if (hit) mine[warp][cnt + __popc(b & ((1u << lane) - 1u))] = st[i];
+            cnt += __popc(b);
         }
+        __syncwarp();
+        if (lane == 0) {
+#pragma unroll 8
+            for (unsigned i = 0; i < cnt; ++i) q = __fadd_rn(q, mine[warp][i]);
+        }
+        __syncwarp();
     }
     if (lane == 0 && p < t.P) t.qP[p] = q;
 }
@@ -348,7 +354,7 @@ cudaError_t hx_launch_conflict(const HxTables& t, const HxTopkBufs& tk, int n_ca
     hx_finish_kernel<<<(n_calls + 255) / 256, 256, 0, stream>>>(tk, D, out_assign);
     *launches += 4;
     if (commit) {
-        hx_qsum_kernel<<<(P + 7) / 8, 256, 0, stream>>>(tk, t);
+        hx_qsum_kernel<<<(P + kQWarps - 1) / kQWarps, 32 * kQWarps, 0, stream>>>(tk, t);
         *launches += 1;
     }
     return cudaGetLastError();
