@@ -159,7 +159,8 @@ __global__ void __launch_bounds__(kWin) hx_conflict_kernel(HxTopkBufs tk, HxTabl
     int* cr = cm + kCache;                                      // [kCache] their ranks
     int* free_s = cr + kCache;                                  // [D] capacity left after the commits so far
     int* dtot = free_s + D;                                     // [D] demand of the window per instance
-    __shared__ int first_fail, bad_d, wsum[NW + 1];
+    int* wtot = dtot + D;                                       // [NW][D] same per warp (only when an instance overflows)
+    __shared__ int first_fail, wsum[NW + 1];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     for (int d = tid; d < D; d += kWin) { free_s[d] = __float2int_rd(t.freeD[d]); dtot[d] = 0; }
     if (tid == 0) first_fail = kWin;
@@ -235,30 +236,26 @@ __global__ void __launch_bounds__(kWin) hx_conflict_kernel(HxTopkBufs tk, HxTabl
         const bool over = dt >= 0 && dtot[dt] > free_s[dt];
         int f = kWin;
         if (__syncthreads_or(over)) {                           // S2: some instance cannot take the whole window
-            // ordered demand ahead of the calls that picked an overflowing instance, one instance at a time
-            int prev = -1;
-            for (;;) {
-                if (tid == 0) bad_d = 0x7fffffff;
-                __syncthreads();
-                if (over && dt > prev) atomicMin(&bad_d, dt);
-                __syncthreads();
-                const int bd = bad_d;
-                if (bd == 0x7fffffff) break;
-                const bool mine = dt == bd;
-                int x = mine ? m : 0;                           // inclusive prefix over the block, in call order
-#pragma unroll
-                for (int off = 1; off < 32; off <<= 1) {
-                    const int y = __shfl_up_sync(0xffffffffu, x, off);
-                    if (lane >= off) x += y;
-                }
-                if (lane == 31) wsum[warp] = x;
-                __syncthreads();
-                int before = 0;
-#pragma unroll
-                for (int w = 0; w < NW; ++w) before += w < warp ? wsum[w] : 0;
-                if (mine && before + x > free_s[bd]) atomicMin(&first_fail, tid);
-                prev = bd;
+            // ordered demand ahead of every call that picked an overflowing instance: inside the warp by
+            // broadcasting every lane's (instance, demand), across warps through per-warp totals
+            for (int i = tid; i < NW * D; i += kWin) wtot[i] = 0;
+            const int key = over ? dt : -1 - lane;              // calls outside the question match nobody
+            int cum = 0; bool later_peer = false;
+#pragma unroll 8
+            for (int j = 0; j < 32; ++j) {
+                const int kj = __shfl_sync(0xffffffffu, key, j);
+                const int mj = __shfl_sync(0xffffffffu, m, j);
+                if (kj == key) { if (j < lane) cum += mj; else if (j > lane) later_peer = true; }
             }
+            __syncthreads();
+            if (over && !later_peer) wtot[warp * D + dt] = cum + m;     // last of its instance in this warp
+            __syncthreads();
+            if (over) {
+#pragma unroll
+                for (int w = 0; w < NW; ++w) cum += w < warp ? wtot[w * D + dt] : 0;
+                if (cum + m > free_s[dt]) atomicMin(&first_fail, tid);
+            }
+            __syncthreads();
             f = first_fail;                                     // calls before f decided as the sequential pass would
             __syncthreads();
             if (tid == 0) first_fail = kWin;
@@ -344,7 +341,7 @@ cudaError_t hx_launch_conflict(const HxTables& t, const HxTopkBufs& tk, int n_ca
     if (e != cudaSuccess) return e;
     hx_order_bins_kernel<<<1, 1024, smB, stream>>>(tk, n_calls, staged);
     hx_order_rank_kernel<<<(n_calls + 127) / 128, 128, 0, stream>>>(tk, n_calls);
-    const size_t smC = (size_t)kCache * 24 + (size_t)(2 * D) * 4;
+    const size_t smC = (size_t)kCache * 24 + (size_t)(2 * D + (kWin / 32) * D) * 4;
     auto pass = tk.K <= 1 ? hx_conflict_kernel<1> : tk.K <= 2 ? hx_conflict_kernel<2>
               : tk.K <= 4 ? hx_conflict_kernel<4> : hx_conflict_kernel<8>;
     static size_t allowed_pass[4][64];
