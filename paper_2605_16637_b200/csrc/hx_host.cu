@@ -18,6 +18,7 @@ struct hx_cluster {
     std::vector<void*> dag_allocs;      // forest, freed at the next upload
     std::vector<void*> tk_allocs;       // top-K / conflict-pass buffers
     HxTables tab{};
+    HxConstTables ctab{};
     int* status = nullptr;
     // forest
     bool dag_uploaded = false, cp_ready = false;
@@ -204,21 +205,32 @@ int hx_cluster_create(const hx_gpu_type* gpu_types, int n_types, const hx_instan
         for (int d = 0; d < D; ++d)
             invLT[(size_t)d * h->Ppad + p] = 1.0f / (link_bw_gbps[(size_t)p * n_instances + P + d] * 1e9f);
 
-    float *d_invF, *d_invB, *d_qP, *d_qD, *d_capD, *d_freeD, *d_invLT, *d_phi, *d_omega, *d_kappa;
+    // the same reciprocal link table in the tile order of the scoring kernel
+    int ld_, td_, dpadT;
+    hx_score_shape(D, &ld_, &td_, &dpadT);
+    std::vector<float> invLTt((size_t)h->Ppad * dpadT, 0.f);
+    for (int p = 0; p < P; ++p)
+        for (int d = 0; d < D; ++d)
+            invLTt[((size_t)(p >> 2) * dpadT + d) * 4 + (p & 3)] = invLT[(size_t)d * h->Ppad + p];
+    for (int g = 0; g < n_types; ++g) { h->ctab.invF[g] = invF[g]; h->ctab.invB[g] = invB[g]; }
+    for (int m = 0; m < n_models; ++m) { h->ctab.phi[m] = phi[m]; h->ctab.omega[m] = omega[m]; h->ctab.kappa[m] = kappa[m]; }
+
+    float *d_invF, *d_invB, *d_qP, *d_qD, *d_capD, *d_freeD, *d_invLT, *d_invLTt, *d_phi, *d_omega, *d_kappa;
     int *d_typeP, *d_typeD;
     bool ok = true; cudaError_t first = cudaSuccess;
     auto up = [&](cudaError_t r) { if (r != cudaSuccess && ok) { ok = false; first = r; } };
     up(dev_upload(h->allocs, &d_invF, invF)); up(dev_upload(h->allocs, &d_invB, invB));
     up(dev_upload(h->allocs, &d_qP, qP)); up(dev_upload(h->allocs, &d_qD, qD));
     up(dev_upload(h->allocs, &d_capD, capD)); up(dev_upload(h->allocs, &d_freeD, freeD));
-    up(dev_upload(h->allocs, &d_invLT, invLT)); up(dev_upload(h->allocs, &d_phi, phi));
+    up(dev_upload(h->allocs, &d_invLT, invLT)); up(dev_upload(h->allocs, &d_invLTt, invLTt));
+    up(dev_upload(h->allocs, &d_phi, phi));
     up(dev_upload(h->allocs, &d_omega, omega)); up(dev_upload(h->allocs, &d_kappa, kappa));
     up(dev_upload(h->allocs, &d_typeP, typeP)); up(dev_upload(h->allocs, &d_typeD, typeD));
     up(dev_alloc(h->allocs, &h->status, 1));
     if (ok) up(cudaMemset(h->status, 0, sizeof(int)));
     if (!ok) return bail(fail_cuda(h, first, "uploading cluster tables"));
     h->tab = HxTables{n_types, P, D, n_models, h->Ppad, d_invF, d_invB, d_typeP, d_typeD, d_qP, d_qD,
-                      d_capD, d_freeD, d_invLT, d_phi, d_omega, d_kappa};
+                      d_capD, d_freeD, d_invLT, d_invLTt, dpadT, d_phi, d_omega, d_kappa};
     *out = h;
     return HX_OK;
 }
@@ -459,7 +471,7 @@ int hx_schedule_batch(hx_cluster* h, const hx_call* calls, int n_calls, int32_t*
     ScoreLaunch sl{calls, n_calls, out_assign, out_cost, o.score_mode, o.flags, o.topk, o.alpha};
     {
         SpanGuard span(h, 0, s);
-        HX_TRY(hx_launch_score(h->tab, dag, tk, sl, h->n_sm, h->max_smem, h->status, s, &h->launches), "scoring kernel");
+        HX_TRY(hx_launch_score(h->tab, h->ctab, dag, tk, sl, h->n_sm, h->max_smem, h->status, s, &h->launches), "scoring kernel");
     }
     if (o.topk > 0) {
         SpanGuard span(h, 1, s);
@@ -578,7 +590,7 @@ int hx_schedule_batch_static(hx_cluster* h, const hx_call* calls, int n_calls, i
     if (!(o.flags & HX_FLAG_NO_DAG))
         dag = HxDagView{h->d_node_wf, h->forest.tail, h->forest.H, h->d_elapsed, h->forest.n_nodes, h->forest.n_workflows};
     ScoreLaunch sl{calls, n_calls, out_assign, out_cost, o.score_mode, o.flags, o.topk, o.alpha};
-    HX_TRY(hx_launch_score(h->tab, dag, b, sl, h->n_sm, h->max_smem, h->status, s, &h->launches), "scoring kernel");
+    HX_TRY(hx_launch_score(h->tab, h->ctab, dag, b, sl, h->n_sm, h->max_smem, h->status, s, &h->launches), "scoring kernel");
     if (o.topk > 0)
         HX_TRY(hx_launch_conflict(h->tab, b, n_calls, o.commit, out_assign, h->status, s, &h->launches), "conflict pass");
     return HX_OK;

@@ -27,10 +27,27 @@ struct HxTables {
     const float* capD;      // [D] tokens
     float* freeD;           // [D] tokens
     const float* invLT;     // [D * Ppad]
+    const float* invLTt;    // same values tiled for the scoring kernel: [Ppad / 4][DpadT][4], zero padded
+    int DpadT;              // decode columns of the tiled copy (hx_score_dpad(D))
     const float* phi;       // [M] flops per token
     const float* omega;     // [M] weight bytes
     const float* kappa;     // [M] KV bytes per token
 };
+
+// Per-class and per-model constants, small enough to travel with the kernel parameters.
+struct HxConstTables {
+    float invF[HX_MAX_TYPES], invB[HX_MAX_TYPES];
+    float phi[HX_MAX_MODELS], omega[HX_MAX_MODELS], kappa[HX_MAX_MODELS];
+};
+
+// Thread-tile shape of the scoring kernel as a function of the decode pool: LD lanes of a warp
+// along the decode columns, TD columns per thread; the block covers Dpad columns.
+inline void hx_score_shape(int D, int* LD, int* TD, int* Dpad) {
+    const int ld = D > 32 ? 8 : D > 16 ? 4 : D > 8 ? 2 : 1;
+    const int td = ld == 8 ? 4 : 8;
+    const int wd = ld * td;
+    *LD = ld; *TD = td; *Dpad = (D + wd - 1) / wd * wd;
+}
 
 // Device view of the uploaded forest and of the horizon results.
 struct HxDagView {
@@ -93,7 +110,7 @@ struct HxForestDev {
     float* H;                        // [W]
 };
 
-cudaError_t hx_launch_score(const HxTables& t, const HxDagView& dag, const HxTopkBufs& tk,
+cudaError_t hx_launch_score(const HxTables& t, const HxConstTables& ct, const HxDagView& dag, const HxTopkBufs& tk,
                             const ScoreLaunch& s, int n_sm, size_t max_smem, int* status,
                             cudaStream_t stream, long long* launches);
 

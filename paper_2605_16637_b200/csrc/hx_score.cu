@@ -27,6 +27,7 @@ typedef unsigned long long u64;
 
 struct ScoreParams {
     HxTables t;
+    HxConstTables ct;
     HxDagView dag;
     HxTopkBufs tk;
     ScoreLaunch s;
@@ -38,6 +39,7 @@ struct ScoreParams {
     int PC;              // prefill chunk length (multiple of 4)
     int nChunks;
     int FS;              // row stride of the per-call finish times (Dpad + 4)
+    int AS, LS;          // strides, in 16-byte units, between consecutive p / 4 of the A and link tiles
     int offA, offF, offCall, offInst;   // byte offsets into dynamic shared memory (LT at 0)
     int resident;        // whole link table and the A tile stay in shared memory for the index recovery
 };
@@ -135,21 +137,60 @@ __device__ __forceinline__ void group_min(const float* frow, int nq, int t, unsi
     }
 }
 
-// Same as group_rescan with both operands resident in shared memory ([p/4][row] float4 layout).
-// The four lanes of the group take the four p of one 16-byte unit, so a step is one
-// conflict-free scalar load per operand.
-__device__ __forceinline__ int group_rescan_smem(const float* acol, int astride, const float* lcol, int lstride,
-                                                 int nq, float kvB, float qd, float Dd, float v, int t,
-                                                 unsigned gmask) {
-    int best = HX_NONE;
-#pragma unroll 8
-    for (int q = nq - 1; q >= 0; --q) {
-        const float f = __fadd_rn(fmaxf(__fmaf_rn(kvB, lcol[q * lstride + t], acol[q * astride + t]), qd), Dd);
-        if (f == v) best = 4 * q + t;
-    }
+// Lowest prefill index p with fin(c, p, d[k]) == v[k] for up to NK decode columns of one call at
+// once (k < n), both operands resident in shared memory as [p / 4][row] 16-byte units.  The four
+// lanes of the group take the units q = t, t + 4, ... in ascending order and stop as soon as every
+// column is resolved.  A candidate can only reach the minimum v if its ready time is at most
+// v - Dd plus the rounding slack of the final addition (ulp(v) / 2 each for the subtraction here
+// and the addition there, covered by v * 2^-21): that test costs one packed FMA pair, two minima
+// and a compare per unit, and only units passing it are evaluated exactly.
+template <int NK>
+__device__ __forceinline__ void group_rescan_multi(const float* a_c, int astride, const float* lts, int lstride,
+                                                   int nq, float kvB, const int* d, const float* qd,
+                                                   const float* Dd, const float* v, int n, int t,
+                                                   unsigned gmask, int* best) {
+    const u64 kk2 = pack2(kvB, kvB);
+    float thr[NK];
 #pragma unroll
-    for (int off = 1; off <= 2; off <<= 1) best = min(best, __shfl_xor_sync(gmask, best, off));
-    return best;
+    for (int k = 0; k < NK; ++k) {
+        best[k] = HX_NONE;
+        thr[k] = k < n ? __fadd_rn(__fsub_rn(v[k], Dd[k]), __fmul_rn(v[k], 4.76837158203125e-07f)) : -1.0f;
+    }
+    unsigned pending = (1u << n) - 1u;                     // the same in the four lanes
+    const int nsteps = (nq + 3) >> 2;
+    for (int s = 0; s < nsteps && pending; ++s) {
+        const int q = 4 * s + t;
+        const bool valid = q < nq;
+        ulonglong2 a = make_ulonglong2(pack2(HX_INF, HX_INF), pack2(HX_INF, HX_INF));
+        if (valid) a = *reinterpret_cast<const ulonglong2*>(a_c + (size_t)q * astride);
+        int cand[NK];
+        bool any = false;
+#pragma unroll
+        for (int k = 0; k < NK; ++k) {
+            cand[k] = HX_NONE;
+            if (k < n && valid) {
+                const ulonglong2 l = *reinterpret_cast<const ulonglong2*>(lts + (size_t)q * lstride + 4 * d[k]);
+                float r[4];
+                unpack2(fma2(kk2, l.x, a.x), r[0], r[1]);
+                unpack2(fma2(kk2, l.y, a.y), r[2], r[3]);
+                if (fminf(min3(r[0], r[1], r[2]), r[3]) <= thr[k] && ((pending >> k) & 1u)) {
+#pragma unroll
+                    for (int u = 3; u >= 0; --u)
+                        if (__fadd_rn(fmaxf(r[u], qd[k]), Dd[k]) == v[k]) cand[k] = 4 * q + u;
+                    any |= cand[k] != HX_NONE;
+                }
+            }
+        }
+        if (__ballot_sync(gmask, any) & gmask) {
+#pragma unroll
+            for (int k = 0; k < NK; ++k) {
+                int c = cand[k];
+                c = min(c, __shfl_xor_sync(gmask, c, 1));
+                c = min(c, __shfl_xor_sync(gmask, c, 2));
+                if (c != HX_NONE && ((pending >> k) & 1u)) { best[k] = c; pending &= ~(1u << k); }
+            }
+        }
+    }
 }
 
 // Thread tile: TC calls x TD decode columns.  A warp spans LD lanes along d and 32 / LD along
@@ -165,14 +206,14 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
     const int warp = tid >> 5, lane = tid & 31;
     const int wd = warp % prm.WDn, wc = warp / prm.WDn;
     const int dg = lane % LD, cg = lane / LD;
-    const int FS = prm.FS, PC = prm.PC, TCB = prm.TCB, Dpad = prm.Dpad;
+    const int FS = prm.FS, PC = prm.PC, TCB = prm.TCB, Dpad = prm.Dpad, AS = prm.AS, LS = prm.LS;
     const bool unloaded = prm.s.flags & HX_FLAG_UNLOADED;
     const bool resident = prm.resident;
 
     // operand tiles are stored [p / 4][row] as 16-byte units: for a fixed p the rows a warp
     // reads are contiguous (no bank conflicts, no padding) and their offsets are compile-time
-    float* LTs = reinterpret_cast<float*>(smem);                  // [PC/4][Dpad][4]
-    float* As = reinterpret_cast<float*>(smem + prm.offA);        // [PC/4][TCB][4]
+    float* LTs = reinterpret_cast<float*>(smem);                  // [PC/4][LS][4], Dpad of LS used
+    float* As = reinterpret_cast<float*>(smem + prm.offA);        // [PC/4][AS][4], TCB of AS used
     float* Fs = reinterpret_cast<float*>(smem + prm.offF);        // [TCB][FS] (may alias As)
     float* kvBs = reinterpret_cast<float*>(smem + prm.offCall);   // [TCB]
     float* mtoks = kvBs + TCB;                                    // [TCB]
@@ -194,19 +235,22 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
         capDs[d] = d < D ? T.capD[d] : -1.0f;
         typeDs[d] = d < D ? T.typeD[d] : 0;
     }
-    // asynchronous copies (no register staging): the wait is just before the barrier that precedes the first use
+    // asynchronous copies (no register staging) from the tiled copy of the link table: consecutive
+    // threads copy consecutive 16-byte units; the wait is just before the barrier that precedes the first use
     auto load_LT = [&](int pc0) {
-        const int nq = PC >> 2;
+        const int nq = PC >> 2, q0 = pc0 >> 2, nq_all = Ppad >> 2;
+        const int dq = nthr / Dpad, dd = nthr - dq * Dpad;
+        int q = tid / Dpad, d = tid - q * Dpad;
         for (int idx = tid; idx < Dpad * nq; idx += nthr) {
-            const int q = idx / Dpad, d = idx - q * Dpad;
-            const int p = pc0 + 4 * q;
-            float* dst = LTs + 4 * idx;
-            if (d < D && p < Ppad) {
+            float* dst = LTs + 4 * (q * LS + d);
+            if (q0 + q < nq_all) {
                 const unsigned sa = (unsigned)__cvta_generic_to_shared(dst);
-                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(sa), "l"(T.invLT + (size_t)d * Ppad + p) : "memory");
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(sa), "l"(T.invLTt + 4 * ((size_t)(q0 + q) * Dpad + d)) : "memory");
             } else {
                 *reinterpret_cast<float4*>(dst) = make_float4(0.f, 0.f, 0.f, 0.f);
             }
+            q += dq; d += dd;
+            if (d >= Dpad) { d -= Dpad; ++q; }
         }
     };
     auto lt_wait = [] { asm volatile("cp.async.wait_all;" ::: "memory"); };
@@ -224,12 +268,12 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
             if (c < nvalid) {
                 const uint4 raw = __ldg(reinterpret_cast<const uint4*>(prm.s.calls) + c0 + c);
                 n = __uint_as_float(raw.z); o = __uint_as_float(raw.w);
-                if (raw.y < (unsigned)T.M) { phi = __ldg(T.phi + raw.y); omega = __ldg(T.omega + raw.y); kappa = __ldg(T.kappa + raw.y); }
+                if (raw.y < (unsigned)T.M) { phi = prm.ct.phi[raw.y]; omega = prm.ct.omega[raw.y]; kappa = prm.ct.kappa[raw.y]; }
             }
             const float kvB = __fmul_rn(n, kappa);
             const float ctx = __fmaf_rn(0.5f, __fsub_rn(o, 1.0f), n);
             const float step = __fmaf_rn(kappa, ctx, omega);
-            const float iF = __ldg(T.invF + g), iB = __ldg(T.invB + g);
+            const float iF = prm.ct.invF[g], iB = prm.ct.invB[g];
             tpres[g * TCB + c] = fmaxf(__fmul_rn(__fmul_rn(n, phi), iF), __fmul_rn(__fadd_rn(omega, kvB), iB));
             tdecs[g * TCB + c] = __fmul_rn(__fmul_rn(o, step), iB);
             if (g == 0) { kvBs[c] = kvB; mtoks[c] = __fadd_rn(n, o); }
@@ -261,7 +305,7 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
 #pragma unroll
                     for (int u = 0; u < 4; ++u)
                         a[u] = (p + u < Ppad) ? __fadd_rn(qPs[p + u], tpres[typePs[p + u] * TCB + c]) : HX_INF;
-                    *reinterpret_cast<float4*>(As + 4 * idx) = make_float4(a[0], a[1], a[2], a[3]);
+                    *reinterpret_cast<float4*>(As + 4 * (q * AS + c)) = make_float4(a[0], a[1], a[2], a[3]);
                     q += dq; c += dc;
                     if (c >= TCB) { c -= TCB; ++q; }
                 }
@@ -277,7 +321,7 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
                 for (int i = 0; i < TC; ++i) a[i] = ap[i * LC];
 #pragma unroll
                 for (int j = 0; j < TD; ++j) l[j] = lp[j * LD];
-                ap += TCB; lp += Dpad;
+                ap += AS; lp += LS;
 #pragma unroll
                 for (int i = 0; i < TC; ++i)
 #pragma unroll
@@ -318,12 +362,25 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
             const float* frow = Fs + cs * FS;
             const float kvB = kvBs[cs], m = mtoks[cs];
             const float* tpre_c = tpres + cs;                 // class g at tpre_c[g * TCB]
-            auto rescan = [&](int d, float v) {
-                const float Dd = (m <= capDs[d]) ? tdecs[typeDs[d] * TCB + cs] : HX_INF;
-                return resident
-                    ? group_rescan_smem(As + 4 * cs, 4 * TCB, LTs + 4 * d, 4 * Dpad, Ppad >> 2, kvB, qDs[d], Dd, v, t, gmask)
-                    : group_rescan(T, qPs, typePs, tpre_c, TCB, kvB, qDs[d], Dd, d, v, t, gmask);
+            // prefill index of n (<= NK) selected columns: lowest p whose candidate finishes exactly at v[k]
+            auto recover = [&](auto nk_tag, const int* dk, const float* vk, int n, int* pk) {
+                constexpr int NK = decltype(nk_tag)::value;
+                float qd[NK], Dd[NK]; int dd[NK];
+#pragma unroll
+                for (int k = 0; k < NK; ++k) {
+                    dd[k] = k < n ? dk[k] : 0;
+                    qd[k] = qDs[dd[k]];
+                    Dd[k] = (m <= capDs[dd[k]]) ? tdecs[typeDs[dd[k]] * TCB + cs] : HX_INF;
+                }
+                if (resident) {
+                    group_rescan_multi<NK>(As + 4 * cs, 4 * AS, LTs, 4 * LS, Ppad >> 2, kvB, dd, qd, Dd, vk, n, t, gmask, pk);
+                } else {
+#pragma unroll
+                    for (int k = 0; k < NK; ++k)
+                        pk[k] = k < n ? group_rescan(T, qPs, typePs, tpre_c, TCB, kvB, qd[k], Dd[k], dd[k], vk[k], t, gmask) : HX_NONE;
+                }
             };
+            struct One { enum { value = 1 }; }; struct Four { enum { value = 4 }; };
             float v0 = HX_INF; int jbest = HX_NONE;
             int sel_pair[HX_MAX_TOPK], sel_d[HX_MAX_TOPK]; float sel_cost[HX_MAX_TOPK], sel_tpre[HX_MAX_TOPK];
 #pragma unroll
@@ -333,60 +390,75 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
                 int d0, ntie;
                 group_min(frow, Dpad >> 2, t, gmask, v0, d0, ntie);
                 if (d0 != HX_NONE) {
-                    jbest = rescan(d0, v0) * D + d0;
+                    int p0;
+                    recover(One{}, &d0, &v0, 1, &p0);
+                    jbest = p0 * D + d0;
                     float pv = v0; int pd = d0;
                     for (int r = 1; r < ntie; ++r) {      // exact ties across decode instances
                         float v; int d;
                         group_next(frow, Dpad >> 2, t, gmask, pv, pd, v, d);
-                        jbest = min(jbest, rescan(d, v) * D + d);
+                        recover(One{}, &d, &v, 1, &p0);
+                        jbest = min(jbest, p0 * D + d);
                         pv = v; pd = d;
                     }
                 }
-            } else if (Dpad <= 128) {
-                // the lane's share of the row (every fourth 16-byte unit) is held in registers; each
-                // round takes the smallest (finish, d) not taken yet
-                float vals[32];
-#pragma unroll
-                for (int it = 0; it < 8; ++it) {
-                    const int q = t + 4 * it;
-                    float4 f4 = make_float4(HX_INF, HX_INF, HX_INF, HX_INF);
-                    if (4 * q < Dpad) f4 = *reinterpret_cast<const float4*>(frow + 4 * q);
-                    vals[4 * it] = f4.x; vals[4 * it + 1] = f4.y; vals[4 * it + 2] = f4.z; vals[4 * it + 3] = f4.w;
-                }
-                unsigned taken = 0;
-                for (int k = 0; k < K; ++k) {
-                    float v = HX_INF; int bi = -1;
-#pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        if (!((taken >> i) & 1u) && vals[i] < v) { v = vals[i]; bi = i; }
-                    int d = bi < 0 ? HX_NONE : 16 * (bi >> 2) + 4 * t + (bi & 3);
-                    const int myd = d;
-#pragma unroll
-                    for (int off = 1; off <= 2; off <<= 1) {
-                        const float ov = __shfl_xor_sync(gmask, v, off);
-                        const int od = __shfl_xor_sync(gmask, d, off);
-                        if (ov < v || (ov == v && od < d)) { v = ov; d = od; }
-                    }
-                    if (d == HX_NONE) break;              // nothing (feasible) left
-                    if (d == myd) taken |= 1u << bi;
-                    if (k == 0) v0 = v;
-                    const int p = rescan(d, v);
-#pragma unroll
-                    for (int k2 = 0; k2 < HX_MAX_TOPK; ++k2)
-                        if (k2 == k) { sel_pair[k2] = p * D + d; sel_d[k2] = d; sel_cost[k2] = v; sel_tpre[k2] = tpre_c[typePs[p] * TCB]; }
-                }
             } else {
-                float pv = -1.0f; int pd = -1;
-                for (int k = 0; k < K; ++k) {
-                    float v; int d;
-                    group_next(frow, Dpad >> 2, t, gmask, pv, pd, v, d);
-                    if (d == HX_NONE) break;              // nothing (feasible) left
-                    if (k == 0) v0 = v;
-                    const int p = rescan(d, v);
+                int nsel = 0;
+                if (Dpad <= 128) {
+                    // the lane's share of the row (every fourth 16-byte unit) is held in registers; each
+                    // round takes the smallest (finish, d) not taken yet
+                    float vals[32];
 #pragma unroll
-                    for (int k2 = 0; k2 < HX_MAX_TOPK; ++k2)
-                        if (k2 == k) { sel_pair[k2] = p * D + d; sel_d[k2] = d; sel_cost[k2] = v; sel_tpre[k2] = tpre_c[typePs[p] * TCB]; }
-                    pv = v; pd = d;
+                    for (int it = 0; it < 8; ++it) {
+                        const int q = t + 4 * it;
+                        float4 f4 = make_float4(HX_INF, HX_INF, HX_INF, HX_INF);
+                        if (4 * q < Dpad) f4 = *reinterpret_cast<const float4*>(frow + 4 * q);
+                        vals[4 * it] = f4.x; vals[4 * it + 1] = f4.y; vals[4 * it + 2] = f4.z; vals[4 * it + 3] = f4.w;
+                    }
+                    unsigned taken = 0;
+                    for (int k = 0; k < K; ++k) {
+                        float v = HX_INF; int bi = -1;
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (!((taken >> i) & 1u) && vals[i] < v) { v = vals[i]; bi = i; }
+                        int d = bi < 0 ? HX_NONE : 16 * (bi >> 2) + 4 * t + (bi & 3);
+                        const int myd = d;
+#pragma unroll
+                        for (int off = 1; off <= 2; off <<= 1) {
+                            const float ov = __shfl_xor_sync(gmask, v, off);
+                            const int od = __shfl_xor_sync(gmask, d, off);
+                            if (ov < v || (ov == v && od < d)) { v = ov; d = od; }
+                        }
+                        if (d == HX_NONE) break;              // nothing (feasible) left
+                        if (d == myd) taken |= 1u << bi;
+#pragma unroll
+                        for (int k2 = 0; k2 < HX_MAX_TOPK; ++k2)
+                            if (k2 == k) { sel_d[k2] = d; sel_cost[k2] = v; }
+                        nsel = k + 1;
+                    }
+                } else {
+                    float pv = -1.0f; int pd = -1;
+                    for (int k = 0; k < K; ++k) {
+                        float v; int d;
+                        group_next(frow, Dpad >> 2, t, gmask, pv, pd, v, d);
+                        if (d == HX_NONE) break;              // nothing (feasible) left
+#pragma unroll
+                        for (int k2 = 0; k2 < HX_MAX_TOPK; ++k2)
+                            if (k2 == k) { sel_d[k2] = d; sel_cost[k2] = v; }
+                        nsel = k + 1;
+                        pv = v; pd = d;
+                    }
+                }
+                if (nsel > 0) v0 = sel_cost[0];
+#pragma unroll
+                for (int k0 = 0; k0 < HX_MAX_TOPK; k0 += 4) {
+                    if (k0 < nsel) {                          // uniform inside the group
+                        int pk[4];
+                        recover(Four{}, &sel_d[k0], &sel_cost[k0], min(4, nsel - k0), pk);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            if (k0 + k < nsel) { sel_pair[k0 + k] = pk[k] * D + sel_d[k0 + k]; sel_tpre[k0 + k] = tpre_c[typePs[pk[k]] * TCB]; }
+                    }
                 }
             }
             if (live && t == 0) {
@@ -448,19 +520,20 @@ inline int round_up(int a, int b) { return (a + b - 1) / b * b; }
 
 }  // namespace
 
-cudaError_t hx_launch_score(const HxTables& t, const HxDagView& dag, const HxTopkBufs& tk,
+cudaError_t hx_launch_score(const HxTables& t, const HxConstTables& ct, const HxDagView& dag, const HxTopkBufs& tk,
                             const ScoreLaunch& s, int n_sm, size_t max_smem, int* status,
                             cudaStream_t stream, long long* launches) {
     ScoreParams prm;
-    prm.t = t; prm.dag = dag; prm.tk = tk; prm.s = s; prm.status = status;
+    prm.t = t; prm.ct = ct; prm.dag = dag; prm.tk = tk; prm.s = s; prm.status = status;
     const int D = t.D, C = s.n_calls;
     // wide decode pools: 16 warps with 4-column thread tiles; narrow ones: 8 warps, 8 columns
-    const int LD = D > 32 ? 8 : D > 16 ? 4 : D > 8 ? 2 : 1;
-    const int TD = LD == 8 ? 4 : 8;
+    int LD, TD, Dpad;
+    hx_score_shape(D, &LD, &TD, &Dpad);
+    if (Dpad != t.DpadT) return cudaErrorInvalidConfiguration;     // the tiled link table was packed for this shape
     const int max_warps = LD == 8 ? 16 : 8;
     const int LC = 32 / LD, WD = TD * LD;
-    prm.WDn = (D + WD - 1) / WD;
-    prm.Dpad = prm.WDn * WD;
+    prm.WDn = Dpad / WD;
+    prm.Dpad = Dpad;
     // warps along calls: fewer when the batch is too small to fill the SMs
     const int min_tc = LD == 8 ? 4 : 8;
     int WCn = prm.WDn >= max_warps ? 1 : max_warps / prm.WDn;
@@ -479,6 +552,11 @@ cudaError_t hx_launch_score(const HxTables& t, const HxDagView& dag, const HxTop
     prm.TCB = WCn * TC * LC;
     prm.nTiles = (C + prm.TCB - 1) / prm.TCB;
     prm.FS = prm.Dpad + 4;
+    // strides of the operand tiles: 2 (mod 8) 16-byte units, so that the four lanes of a selection
+    // group, which read four consecutive p / 4 of one row, fall into different bank groups
+    auto pad_stride = [](int n) { return n + ((2 - n) % 8 + 8) % 8; };
+    prm.AS = pad_stride(prm.TCB);
+    prm.LS = pad_stride(prm.Dpad);
     const int G = t.G;
     const size_t callB = round_up(prm.TCB * (2 + 2 * G) * 4, 16);
     const size_t instB = round_up((2 * t.Ppad + 3 * prm.Dpad) * 4, 16);
@@ -487,19 +565,19 @@ cudaError_t hx_launch_score(const HxTables& t, const HxDagView& dag, const HxTop
     const size_t f_rows = (size_t)prm.TCB * prm.FS * 4;
     // first choice: whole link table, A tile and finish times side by side
     int PC = t.Ppad;
-    prm.resident = ((size_t)(prm.Dpad + prm.TCB) * PC * 4 + f_rows <= budget) ? 1 : 0;
+    prm.resident = ((size_t)(prm.LS + prm.AS) * PC * 4 + f_rows <= budget) ? 1 : 0;
     if (!prm.resident) {
         // otherwise chunk the prefill dimension; the finish times reuse the A tile
         for (;;) {
-            const size_t a_rows = (size_t)prm.TCB * PC * 4;
-            if ((size_t)prm.Dpad * PC * 4 + (a_rows > f_rows ? a_rows : f_rows) <= budget || PC <= 4) break;
+            const size_t a_rows = (size_t)prm.AS * PC * 4;
+            if ((size_t)prm.LS * PC * 4 + (a_rows > f_rows ? a_rows : f_rows) <= budget || PC <= 4) break;
             PC = round_up(PC / 2, 4);
         }
     }
     prm.PC = PC;
     prm.nChunks = (t.Ppad + PC - 1) / PC;
-    const size_t ltB = (size_t)prm.Dpad * PC * 4;
-    const size_t aB = (size_t)prm.TCB * PC * 4;
+    const size_t ltB = (size_t)prm.LS * PC * 4;
+    const size_t aB = (size_t)prm.AS * PC * 4;
     prm.offA = (int)ltB;
     if (prm.resident) { prm.offF = prm.offA + (int)aB; prm.offCall = prm.offF + round_up((int)f_rows, 16); }
     else { prm.offF = prm.offA; prm.offCall = prm.offA + (int)(aB > f_rows ? aB : round_up((int)f_rows, 16)); }
