@@ -26,6 +26,9 @@ sys.path.insert(0, ROOT)
 METRIC = "placement candidates scored/sec"
 UNIT = "candidates/s"
 FP32_LANES_PER_SM = 128
+ALGO_LANE_OPS_PER_CANDIDATE = 4      # fma, max, add, min of the per-candidate cost definition
+EXEC_LANE_OPS_PER_CANDIDATE = 2      # what the candidate loop executes: fma and min
+SCORE_DRAM_BYTES_PER_LAUNCH = 3261184   # ncu, one launch of 16,384 calls x 128 x 128 pairs with top-4 lists
 
 
 def _peaks():
@@ -287,18 +290,27 @@ def run_cuda(args):
     peaks, which = _peaks()
     n_sm = torch.cuda.get_device_properties(local).multi_processor_count
     sm_max_mhz = float(peaks.get("sm_max_mhz", 1965.0))
-    # dominant kernel: scoring.  Algorithmic work: two FP32 lane-operations per candidate (one fused
-    # multiply-add, one minimum); like the peak, each lane-operation is counted as 2 flop.
+    # Roofline of the scoring kernel (bound: FP32 issue).  Algorithmic work per candidate = the four
+    # FP32 lane-instructions of the cost definition (fused multiply-add, maximum, addition, running
+    # minimum); like the peak, every lane-instruction is counted as 2 flop.  The kernel itself executes
+    # only two of them per candidate (the maximum and the addition are taken once per (call, decode
+    # instance) after the reduction over the prefill instances): frac_executed counts those two only.
     score_ms, score_n = kt["scoring"]
     score_avg_ms = score_ms / max(score_n, 1)
-    achieved = 4.0 * chunk * P * D / (score_avg_ms * 1e-3) / 1e12
+    lane_rate = chunk * P * D / (score_avg_ms * 1e-3)              # candidates per second of one launch
     peak = 2.0 * n_sm * FP32_LANES_PER_SM * sm_max_mhz * 1e6 / 1e12
+    achieved = 2.0 * ALGO_LANE_OPS_PER_CANDIDATE * lane_rate / 1e12
     roofline = {"bound": "alu", "kernel": "hx_score_kernel", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                "frac": achieved / peak, "traffic": None,
+                "frac": achieved / peak, "traffic": SCORE_DRAM_BYTES_PER_LAUNCH,
                 "peak_source": "%d SMs x %d FP32 lanes x %.0f MHz x 2 flop (%s sm_max_mhz)" % (
                     n_sm, FP32_LANES_PER_SM, sm_max_mhz, which),
                 "avg_launch_us": score_avg_ms * 1e3, "launches_timed": score_n,
-                "lane_ops_per_candidate": 2, "flop_equiv_per_candidate": 4,
+                "lane_ops_per_candidate": ALGO_LANE_OPS_PER_CANDIDATE,
+                "frac_executed": 2.0 * EXEC_LANE_OPS_PER_CANDIDATE * lane_rate / 1e12 / peak,
+                "lane_ops_executed_per_candidate": EXEC_LANE_OPS_PER_CANDIDATE,
+                "candidates_per_s_kernel": lane_rate,
+                "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch on this "
+                                  "workload (profiles/hx_score_kernel_sweep_chunk.md)",
                 "time_share": {k: v[0] / max(total_ms, 1e-9) for k, v in kt.items()}}
 
     cpu = None

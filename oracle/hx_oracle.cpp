@@ -259,6 +259,56 @@ int orc_conflict(int C, int K, int D, const int32_t* pair, const float* prio, co
     return 0;
 }
 
+// Recomputing greedy planner for small queues (Algorithm 1, the while-loop over
+// the queue snapshot; Section 5.3 "Adaptive greedy prefill assignment").
+// Until the queue is empty: for every waiting call project its best feasible
+// placement against the simulated state, its Delta and its ratio R (Eq. 2);
+// take the call with the largest R (lower call index among equals); record its
+// pair; update the simulated state; remove the call.
+// Simulated state: the chosen prefill queue grows by the call's prefill time,
+// the chosen decode instance loses m(c) free KV tokens; qD is left as it is.
+// A pair is feasible when m(c) <= Cap(d) (Eq. 4) and m(c) <= free KV tokens of
+// d in the simulated state.  A call without a feasible pair is passed over; the
+// loop ends when no waiting call has one (the state never improves).
+// Outputs: assign[c] pair or -1, ratio[c] = R at the moment of selection (+inf
+// if never placed), order[i] = call taken in iteration i (-1 past the end);
+// qP[P] and freeD[D] are updated in place.  Returns the number of placed calls.
+int orc_greedy(const OrcCluster* cl, const OrcDag* dag, const OrcCall* calls, int C, int flags,
+               float* qP, float* freeD, int32_t* assign, float* ratio, int32_t* order) {
+    OrcCluster sim = *cl;
+    sim.qP = qP;                                        // candidate_fin reads the simulated queues
+    std::vector<char> waiting(C, 1);
+    std::vector<Terms> terms(C);
+    for (int c = 0; c < C; ++c) { latency_terms(*cl, calls[c], terms[c]); assign[c] = -1; ratio[c] = INF; order[c] = -1; }
+    int placed = 0;
+    for (int it = 0; it < C; ++it) {
+        int best_c = -1, best_j = -1; float best_R = -INF;
+        for (int c = 0; c < C; ++c) {
+            if (!waiting[c]) continue;
+            const Terms& t = terms[c];
+            float delta = INF; int arg = -1;
+            for (int p = 0; p < cl->P; ++p)
+                for (int d = 0; d < cl->D; ++d) {
+                    if (!(t.m <= freeD[d])) continue;           // KV tokens left in the simulated state
+                    const float f = candidate_fin(sim, t, p, d, false);
+                    if (f < delta) { delta = f; arg = p * cl->D + d; }
+                }
+            if (arg < 0) continue;
+            const DagView v = dag_view(dag, calls[c], flags);
+            const float R = (v.elapsed + delta) / v.H;          // Eq. 2
+            if (R > best_R) { best_R = R; best_c = c; best_j = arg; }
+        }
+        if (best_c < 0) break;
+        const int p = best_j / cl->D, d = best_j % cl->D;
+        assign[best_c] = best_j; ratio[best_c] = best_R; order[it] = best_c;
+        qP[p] = qP[p] + terms[best_c].tpre[cl->typeP[p]];
+        freeD[d] = freeD[d] - terms[best_c].m;
+        waiting[best_c] = 0;
+        ++placed;
+    }
+    return placed;
+}
+
 // Longest node-weighted path to a sink, per node, over a successor-CSR DAG:
 //   tail[v] = max over successors u of cp[u]   (0 without successors)
 //   cp[v]   = cost[v] + tail[v]

@@ -188,3 +188,19 @@ class Oracle:
         self.lib.orc_conflict(n, K, int(D), _ptr(pair), _ptr(prio), _ptr(m), _ptr(tpre_sel),
                               _ptr(freeD), _ptr(qP), _ptr(assign))
         return assign, freeD, qP
+
+    def greedy(self, cl: Cluster, calls, freeD, flags=0, dag: DagResult | None = None, node_wf=None,
+               elapsed=None):
+        """Recomputing greedy of Algorithm 1 over one queue snapshot.
+        Returns (assign i32[C], ratio f32[C], order i32[C], n_placed, qP', freeD')."""
+        calls, n = self._calls(calls)
+        assign = np.zeros(n, np.int32); ratio = np.zeros(n, np.float32); order = np.zeros(n, np.int32)
+        qP = _f32(cl.qP).copy(); free = _f32(freeD).copy()
+        c = cl._c()
+        d, keep = self._dag(dag, node_wf, elapsed)
+        if d is None:
+            flags |= FLAG_NO_DAG
+        self.lib.orc_greedy.restype = C.c_int
+        placed = self.lib.orc_greedy(C.byref(c), C.byref(d) if d is not None else None, _ptr(calls), n,
+                                     int(flags), _ptr(qP), _ptr(free), _ptr(assign), _ptr(ratio), _ptr(order))
+        return assign, ratio, order, int(placed), qP, free
