@@ -208,6 +208,32 @@ int hx_schedule_batch_host(hx_cluster* h, const hx_call* calls, int n_calls,
 int hx_schedule_batch_static(hx_cluster* h, const hx_call* calls, int n_calls,
                              int32_t* out_assign, float* out_cost, void* stream);
 
+/* Recomputing greedy planner for small queues (Algorithm 1, the while-loop over
+ * the queue snapshot; Section 5.3 "Adaptive greedy prefill assignment"): until
+ * the queue is empty, every waiting call's best feasible pair, its Delta and its
+ * ratio R = (elapsed_w + Delta) / H_w (Eq. 2) are projected against the simulated
+ * state; the call with the largest R is taken (lower call index among equals),
+ * its pair is recorded, its prefill time is added to the chosen prefill queue
+ * and its m(c) = L_in + L_out tokens (Eq. 3) are taken from the free KV tokens of
+ * the chosen decode instance; then it leaves the queue.  A pair is feasible when
+ * m(c) <= Cap(d) (Eq. 4) and m(c) fits the free KV tokens the simulated state has
+ * left on d.  A call that fits nowhere is passed over; the loop ends when no
+ * waiting call fits anywhere.
+ *   calls: device, n_calls records, 16-byte aligned, 1 <= n_calls <=
+ * HX_GREEDY_MAX_CALLS and small enough for the whole state to fit the shared
+ * memory of one SM (HX_ERR_INVALID_ARG otherwise).  out_assign: device
+ * int32[n_calls], pair p * n_decode + d or -1.  out_ratio: device
+ * float[n_calls], R at the moment the call was taken, +inf if never taken.
+ * out_order: device int32[n_calls], out_order[i] = call taken in iteration i,
+ * -1 after the last one.  Uses hx_options.flags (HX_FLAG_NO_DAG: elapsed = 0,
+ * H = 1; HX_FLAG_UNLOADED is rejected) and hx_options.commit (write the
+ * simulated queues and free KV tokens back into the cluster).  Needs
+ * hx_critical_path unless HX_FLAG_NO_DAG is set.  Invalid model or node ids:
+ * as for hx_schedule_batch.  Enqueues one kernel on `stream`. */
+#define HX_GREEDY_MAX_CALLS 4096
+int hx_schedule_greedy(hx_cluster* h, const hx_call* calls, int n_calls,
+                       int32_t* out_assign, float* out_ratio, int32_t* out_order, void* stream);
+
 /* Borrowed device pointers to the top-K results of the last batch scored with
  * topk = K > 0: pairs int32[n_calls][K] (-1 = unused slot), costs
  * float[n_calls][K] (projected decode finish of that pair, +inf if unused),

@@ -57,6 +57,7 @@ def _load():
         "hx_schedule_batch": [vp, vp, ci, vp, vp, vp],
         "hx_schedule_batch_host": [vp, vp, ci, vp, vp, vp],
         "hx_schedule_batch_static": [vp, vp, ci, vp, vp, vp],
+        "hx_schedule_greedy": [vp, vp, ci, vp, vp, vp, vp],
         "hx_get_topk": [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp)],
         "hx_get_status": [vp, C.POINTER(ci), vp],
         "hx_enable_kernel_timing": [vp, ci],
@@ -153,6 +154,12 @@ def hx_schedule_batch_static(h, calls_ptr, n_calls, out_assign_ptr, out_cost_ptr
     """hx_schedule_batch without any allocation: intermediates live in a fixed device array
     (at most 16384 calls with topk <= 4); see include/hx.h for who needs this and the rules."""
     _check(_lib.hx_schedule_batch_static(h, calls_ptr, int(n_calls), out_assign_ptr, out_cost_ptr, stream), h)
+
+
+def hx_schedule_greedy(h, calls_ptr, n_calls, out_assign_ptr, out_ratio_ptr, out_order_ptr, stream=0):
+    """Recomputing greedy planner for small queues (Algorithm 1); device pointers."""
+    _check(_lib.hx_schedule_greedy(h, calls_ptr, int(n_calls), out_assign_ptr, out_ratio_ptr, out_order_ptr,
+                                   stream), h)
 
 
 def hx_schedule_batch_host(h, calls, out_assign=None, out_cost=None, stream=0):
@@ -285,6 +292,19 @@ class Cluster:
             out_cost = torch.empty(n, dtype=torch.float32, device="cuda")
         hx_schedule_batch(self.h, calls.data_ptr(), n, out_assign.data_ptr(), out_cost.data_ptr(), self._stream())
         return out_assign, out_cost
+
+    def schedule_greedy(self, calls):
+        """calls as for schedule_batch.  Returns (assign, ratio, order) CUDA tensors."""
+        import torch
+        if isinstance(calls, np.ndarray):
+            calls = torch.from_numpy(_np(calls, CALL_DTYPE).view(np.uint8).copy()).cuda()
+        n = calls.numel() * calls.element_size() // 16
+        assign = torch.empty(n, dtype=torch.int32, device="cuda")
+        ratio = torch.empty(n, dtype=torch.float32, device="cuda")
+        order = torch.empty(n, dtype=torch.int32, device="cuda")
+        hx_schedule_greedy(self.h, calls.data_ptr(), n, assign.data_ptr(), ratio.data_ptr(), order.data_ptr(),
+                           self._stream())
+        return assign, ratio, order
 
     def schedule_batch_host(self, calls, out_assign=None, out_cost=None):
         return hx_schedule_batch_host(self.h, calls, out_assign, out_cost, self._stream())

@@ -1,0 +1,224 @@
+// Recomputing greedy planner for small queues (paper Algorithm 1, the while-loop
+// over the queue snapshot; Section 5.3 "Adaptive greedy prefill assignment").
+//
+// Until the queue is empty: project every waiting call's best feasible pair
+// against the simulated state, its Delta and its ratio R = (elapsed + Delta) / H
+// (Eq. 2); take the call with the largest R (lower call index among equals);
+// record its pair; add its prefill time to the chosen prefill queue and take its
+// m(c) = L_in + L_out KV tokens (Eq. 3) from the chosen decode instance; remove
+// it.  A pair is feasible when m(c) <= Cap(d) (Eq. 4) and m(c) fits the KV tokens
+// the simulated state has left on d.
+//
+// One persistent block holds the whole state in shared memory.  A commit touches
+// one prefill queue p* and one decode instance d*, and every candidate only gets
+// later or disappears; so the projection of a waiting call changes only if its
+// own best pair uses p*, or uses d* and no longer fits.  Per iteration the block
+// (1) re-projects exactly those calls, one warp per call with the lanes over the
+// pairs, (2) reduces the largest ratio, (3) commits and lists the calls to
+// re-project.  The arithmetic of a candidate is the canonical binary32 sequence
+// of the scoring kernel, so the results equal the definition bit for bit.
+#include "hx_internal.h"
+
+namespace {
+
+constexpr int kThreads = 1024;
+constexpr int kWarps = kThreads / 32;
+#define HX_INF __int_as_float(0x7f800000)
+#define HX_NEG_INF __int_as_float(0xff800000)
+constexpr int kDead = -2;          // call already taken (or rejected as invalid)
+constexpr int kNoPair = -1;        // waiting, but no feasible pair: can never be taken any more
+
+struct GreedyParams {
+    HxTables t;
+    HxConstTables ct;
+    HxDagView dag;
+    const hx_call* calls;
+    int n, flags, commit;
+    int32_t* out_assign;
+    float* out_ratio;
+    int32_t* out_order;
+    int* status;
+};
+
+__global__ void __launch_bounds__(kThreads, 1) hx_greedy_kernel(const __grid_constant__ GreedyParams prm) {
+    extern __shared__ __align__(16) unsigned char smem[];
+    __shared__ float red_v[kWarps];
+    __shared__ int red_c[kWarps];
+    __shared__ int s_call, s_p, s_d, s_ndirty;
+    const HxTables& T = prm.t;
+    const int P = T.P, D = T.D, G = T.G, n = prm.n;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    float* invL = reinterpret_cast<float*>(smem);              // [P][D]
+    float* qPs = invL + (size_t)P * D;                         // [P]
+    float* qDs = qPs + P;                                      // [D]
+    float* capDs = qDs + D;                                    // [D]
+    float* frees = capDs + D;                                  // [D]
+    int* typePs = reinterpret_cast<int*>(frees + D);           // [P]
+    int* typeDs = typePs + P;                                  // [D]
+    float* scratch = reinterpret_cast<float*>(typeDs + D);     // [kWarps][64] per-class times of the call a warp works on
+    float* cn = scratch + kWarps * 64;                         // [n] prompt tokens
+    float* co = cn + n;                                        // [n] output tokens
+    float* cel = co + n;                                       // [n] elapsed time of the workflow
+    float* cH = cel + n;                                       // [n] horizon of the workflow
+    float* cR = cH + n;                                        // [n] projected ratio, -inf if it cannot be taken
+    int* cpair = reinterpret_cast<int*>(cR + n);               // [n] best pair as p << 16 | d, kNoPair, kDead
+    int* cmodel = cpair + n;                                   // [n]
+    unsigned short* dirty = reinterpret_cast<unsigned short*>(cmodel + n);   // [n] calls to re-project
+
+    for (int i = tid; i < P * D; i += kThreads) { const int p = i / D, d = i - p * D; invL[i] = T.invLT[(size_t)d * T.Ppad + p]; }
+    for (int p = tid; p < P; p += kThreads) { qPs[p] = T.qP[p]; typePs[p] = T.typeP[p]; }
+    for (int d = tid; d < D; d += kThreads) { qDs[d] = T.qD[d]; capDs[d] = T.capD[d]; frees[d] = T.freeD[d]; typeDs[d] = T.typeD[d]; }
+    for (int c = tid; c < n; c += kThreads) {
+        const uint4 raw = __ldg(reinterpret_cast<const uint4*>(prm.calls) + c);
+        bool bad = raw.y >= (unsigned)T.M;
+        float el = 0.f, H = 1.f;
+        if (!(prm.flags & HX_FLAG_NO_DAG)) {
+            if (raw.x < prm.dag.n_nodes) { const uint32_t w = prm.dag.node_wf[raw.x]; el = prm.dag.elapsed[w]; H = prm.dag.H[w]; }
+            else bad = true;
+        }
+        if (bad) atomicExch(prm.status, HX_ERR_INVALID_ARG);
+        cn[c] = __uint_as_float(raw.z); co[c] = __uint_as_float(raw.w);
+        cmodel[c] = bad ? 0 : (int)raw.y;
+        cel[c] = el; cH[c] = H;
+        cR[c] = HX_NEG_INF;
+        cpair[c] = bad ? kDead : kNoPair;
+        dirty[c] = (unsigned short)c;
+        prm.out_assign[c] = -1; prm.out_ratio[c] = HX_INF; prm.out_order[c] = -1;
+    }
+    if (tid == 0) s_ndirty = n;
+    __syncthreads();
+
+    for (int it = 0; it < n; ++it) {
+        // (1) re-project the listed calls: one warp per call, lanes over the pairs
+        const int nd = s_ndirty;
+        float* tpre = scratch + warp * 64;
+        float* tdec = tpre + 32;
+        for (int i = warp; i < nd; i += kWarps) {
+            const int c = dirty[i];
+            if (cpair[c] == kDead) continue;                   // rejected at load time (warp-uniform)
+            const float nt = cn[c], ot = co[c];
+            const int mdl = cmodel[c];
+            const float phi = prm.ct.phi[mdl], omega = prm.ct.omega[mdl], kappa = prm.ct.kappa[mdl];
+            const float kvB = __fmul_rn(nt, kappa);
+            const float ctx = __fmaf_rn(0.5f, __fsub_rn(ot, 1.0f), nt);
+            const float step = __fmaf_rn(kappa, ctx, omega);
+            const float m = __fadd_rn(nt, ot);
+            if (lane < G) {
+                const float iF = prm.ct.invF[lane], iB = prm.ct.invB[lane];
+                tpre[lane] = fmaxf(__fmul_rn(__fmul_rn(nt, phi), iF), __fmul_rn(__fadd_rn(omega, kvB), iB));
+                tdec[lane] = __fmul_rn(__fmul_rn(ot, step), iB);
+            }
+            __syncwarp();
+            float best = HX_INF; int bj = 0x7fffffff;
+            int p = lane / D, d = lane - p * D;
+            while (p < P) {
+                const bool fits = m <= capDs[d] && m <= frees[d];
+                const float Dd = fits ? tdec[typeDs[d]] : HX_INF;
+                const float A = __fadd_rn(qPs[p], tpre[typePs[p]]);
+                const float ready = __fmaf_rn(kvB, invL[p * D + d], A);
+                const float fin = __fadd_rn(fmaxf(ready, qDs[d]), Dd);
+                if (fin < best) { best = fin; bj = (p << 16) | d; }
+                d += 32;
+                while (d >= D) { d -= D; ++p; }
+            }
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) {
+                const float ov = __shfl_xor_sync(0xffffffffu, best, off);
+                const int oj = __shfl_xor_sync(0xffffffffu, bj, off);
+                if (ov < best || (ov == best && oj < bj)) { best = ov; bj = oj; }
+            }
+            if (lane == 0) {
+                if (best < HX_INF) { cpair[c] = bj; cR[c] = __fdiv_rn(__fadd_rn(cel[c], best), cH[c]); }
+                else { cpair[c] = kNoPair; cR[c] = HX_NEG_INF; }
+            }
+            __syncwarp();
+        }
+        __syncthreads();
+        // (2) most urgent waiting call: largest ratio, lower call index among equals
+        float rv = HX_NEG_INF; int rc = 0x7fffffff;
+        for (int c = tid; c < n; c += kThreads) {
+            const float r = cR[c];
+            if (r > rv) { rv = r; rc = c; }                    // ascending c: keeps the lowest index
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, rv, off);
+            const int oc = __shfl_xor_sync(0xffffffffu, rc, off);
+            if (ov > rv || (ov == rv && oc < rc)) { rv = ov; rc = oc; }
+        }
+        if (lane == 0) { red_v[warp] = rv; red_c[warp] = rc; }
+        __syncthreads();
+        if (warp == 0) {
+            rv = red_v[lane]; rc = red_c[lane];
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) {
+                const float ov = __shfl_xor_sync(0xffffffffu, rv, off);
+                const int oc = __shfl_xor_sync(0xffffffffu, rc, off);
+                if (ov > rv || (ov == rv && oc < rc)) { rv = ov; rc = oc; }
+            }
+            if (lane == 0) {
+                if (rc == 0x7fffffff) {
+                    s_call = -1;                               // nobody left that fits anywhere
+                } else {
+                    // (3) commit: update the simulated state
+                    const int bj = cpair[rc], p = bj >> 16, d = bj & 0xFFFF;
+                    const float nt = cn[rc], ot = co[rc];
+                    const int mdl = cmodel[rc];
+                    const float phi = prm.ct.phi[mdl], omega = prm.ct.omega[mdl], kappa = prm.ct.kappa[mdl];
+                    const float kvB = __fmul_rn(nt, kappa);
+                    const int g = typePs[p];
+                    const float tp = fmaxf(__fmul_rn(__fmul_rn(nt, phi), prm.ct.invF[g]), __fmul_rn(__fadd_rn(omega, kvB), prm.ct.invB[g]));
+                    qPs[p] = __fadd_rn(qPs[p], tp);
+                    frees[d] = __fsub_rn(frees[d], __fadd_rn(nt, ot));
+                    prm.out_assign[rc] = p * D + d;
+                    prm.out_ratio[rc] = rv;
+                    prm.out_order[it] = rc;
+                    cpair[rc] = kDead; cR[rc] = HX_NEG_INF;
+                    s_call = rc; s_p = p; s_d = d;
+                }
+                s_ndirty = 0;
+            }
+        }
+        __syncthreads();
+        if (s_call < 0) break;
+        // calls whose projection the commit can have changed
+        const int ps = s_p, ds = s_d;
+        const float left = frees[ds];
+        for (int c = tid; c < n; c += kThreads) {
+            const int bj = cpair[c];
+            if (bj < 0) continue;
+            const bool hit = (bj >> 16) == ps || ((bj & 0xFFFF) == ds && __fadd_rn(cn[c], co[c]) > left);
+            if (hit) dirty[atomicAdd(&s_ndirty, 1)] = (unsigned short)c;
+        }
+        __syncthreads();
+    }
+    if (prm.commit) {
+        for (int p = tid; p < P; p += kThreads) T.qP[p] = qPs[p];
+        for (int d = tid; d < D; d += kThreads) T.freeD[d] = frees[d];
+    }
+}
+
+}  // namespace
+
+size_t hx_greedy_smem_bytes(const HxTables& t, int n_calls) {
+    return ((size_t)t.P * t.D + 2 * (size_t)t.P + 5 * (size_t)t.D + kWarps * 64 + 7 * (size_t)n_calls) * 4 +
+           (size_t)n_calls * 2 + 16;
+}
+
+cudaError_t hx_launch_greedy(const HxTables& t, const HxConstTables& ct, const HxDagView& dag,
+                             const hx_call* calls, int n_calls, int flags, int commit,
+                             int32_t* out_assign, float* out_ratio, int32_t* out_order, int* status,
+                             cudaStream_t stream, long long* launches) {
+    GreedyParams prm;
+    prm.t = t; prm.ct = ct; prm.dag = dag; prm.calls = calls; prm.n = n_calls; prm.flags = flags; prm.commit = commit;
+    prm.out_assign = out_assign; prm.out_ratio = out_ratio; prm.out_order = out_order; prm.status = status;
+    const size_t smem = hx_greedy_smem_bytes(t, n_calls);
+    static size_t allowed[64];
+    cudaError_t e = hx_opt_in_smem(hx_greedy_kernel, smem, allowed, 40 * 1024);
+    if (e != cudaSuccess) return e;
+    hx_greedy_kernel<<<1, kThreads, smem, stream>>>(prm);
+    e = cudaGetLastError();
+    if (e == cudaSuccess) ++*launches;
+    return e;
+}

@@ -596,6 +596,34 @@ int hx_schedule_batch_static(hx_cluster* h, const hx_call* calls, int n_calls, i
     return HX_OK;
 }
 
+int hx_schedule_greedy(hx_cluster* h, const hx_call* calls, int n_calls, int32_t* out_assign,
+                       float* out_ratio, int32_t* out_order, void* stream) {
+    if (!h) return HX_ERR_INVALID_ARG;
+    if (n_calls < 0) return fail(h, HX_ERR_INVALID_ARG, "negative n_calls");
+    if (n_calls == 0) return HX_OK;
+    if (!calls || !out_assign || !out_ratio || !out_order) return fail(h, HX_ERR_INVALID_ARG, "NULL buffer");
+    if (reinterpret_cast<uintptr_t>(calls) % 16) return fail(h, HX_ERR_INVALID_ARG, "calls must be 16-byte aligned");
+    const hx_options& o = h->opts;
+    if (o.flags & HX_FLAG_UNLOADED) return fail(h, HX_ERR_INVALID_ARG, "hx_schedule_greedy plans against the loaded cluster: clear HX_FLAG_UNLOADED");
+    if (!(o.flags & HX_FLAG_NO_DAG) && !(h->dag_uploaded && h->cp_ready))
+        return fail(h, HX_ERR_NOT_READY, "horizons not computed: call hx_dag_upload and hx_critical_path, or set HX_FLAG_NO_DAG");
+    if (n_calls > HX_GREEDY_MAX_CALLS)
+        return fail(h, HX_ERR_INVALID_ARG, "hx_schedule_greedy: more than HX_GREEDY_MAX_CALLS (4096) calls; use hx_schedule_batch with topk > 0 for large queues");
+    if (hx_greedy_smem_bytes(h->tab, n_calls) > h->max_smem)
+        return fail(h, HX_ERR_INVALID_ARG, "hx_schedule_greedy: cluster tables and queue do not fit the shared memory of one SM");
+    DeviceGuard guard(h->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    HxDagView dag{};
+    if (!(o.flags & HX_FLAG_NO_DAG))
+        dag = HxDagView{h->d_node_wf, h->forest.tail, h->forest.H, h->d_elapsed, h->forest.n_nodes, h->forest.n_workflows};
+    {
+        SpanGuard span(h, 0, s);
+        HX_TRY(hx_launch_greedy(h->tab, h->ctab, dag, calls, n_calls, o.flags, o.commit, out_assign, out_ratio,
+                                out_order, h->status, s, &h->launches), "greedy planner kernel");
+    }
+    return HX_OK;
+}
+
 int hx_get_topk(hx_cluster* h, const int32_t** pairs, const float** costs, const float** prio) {
     if (!h) return HX_ERR_INVALID_ARG;
     if (h->tk.cap_calls == 0) return fail(h, HX_ERR_NOT_READY, "no batch has been scored with topk > 0");

@@ -118,6 +118,12 @@ cudaError_t hx_launch_conflict(const HxTables& t, const HxTopkBufs& tk, int n_ca
                                int32_t* out_assign, int* status, cudaStream_t stream,
                                long long* launches);
 
+size_t hx_greedy_smem_bytes(const HxTables& t, int n_calls);
+cudaError_t hx_launch_greedy(const HxTables& t, const HxConstTables& ct, const HxDagView& dag,
+                             const hx_call* calls, int n_calls, int flags, int commit,
+                             int32_t* out_assign, float* out_ratio, int32_t* out_order, int* status,
+                             cudaStream_t stream, long long* launches);
+
 // Workflow classes of the horizon pass: lists of workflow ids handled by one launch each.
 struct HxCpClass {
     const uint32_t* wf_ids;    // device
