@@ -321,6 +321,7 @@ def run_cuda(args):
                "sample": "%d of 16 invocations (%d calls x 16384 pairs, top-4 + conflict pass), %.1f s" % (
                    n_b, n_b * chunk, dt)}
 
+    greedy = greedy_leg(with_cpu=not args.no_cpu_baseline) if world == 1 else None
     h2d = n_calls * 16 + (P + 2 * D) * 4 + n_chunks * D * 4
     d2h = n_calls * 8
     out = {
@@ -340,10 +341,48 @@ def run_cuda(args):
                 "what": "hx_schedule_batch_host per chunk from pinned host memory, wall clock"},
         "gpu_launches": int(launches), "kernel_ms_per_step": {k: v[0] / args.steps for k, v in kt.items()},
         "device_status": status, "roofline": roofline, "cpu_baseline": cpu, "clocks": clocks,
+        "greedy_planner": greedy,
     }
     print(json.dumps(out))
     if dist is not None:
         dist.destroy_process_group()
+
+
+def greedy_leg(with_cpu):
+    """Side measurement, outside the timed region: the recomputing greedy planner (Algorithm 1,
+    small queues) on the medium configuration, 4,096 ready calls x 16 x 16 pairs."""
+    import torch
+    import paper_2605_16637_b200 as hx
+    from hx_synth import make_workload
+    out = {}
+    for label, scale in (("medium", 1.0), ("medium_quarter", 0.25)):
+        wl = make_workload("medium", scale=scale)
+        gc = hx.Cluster.from_workload(wl)
+        gc.set_options(score_mode=hx.HX_MODE_COMPLETION, flags=hx.HX_FLAG_UNLOADED | hx.HX_FLAG_NO_DAG)
+        cost = gc.schedule_batch(wl.node_calls)[1].cpu().numpy()
+        gc.dag_upload(wl.row_ptr, wl.col, cost, wl.node_wf, wl.elapsed)
+        gc.critical_path()
+        gc.set_options(score_mode=hx.HX_MODE_RATIO, commit=0)
+        calls = torch.from_numpy(wl.calls.view(np.uint8).reshape(-1, 16).copy()).cuda()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(5)]
+        for _ in range(2):
+            gc.schedule_greedy(calls)
+        for a, b in ev:
+            a.record(); res = gc.schedule_greedy(calls); b.record()
+        torch.cuda.synchronize()
+        ms = float(np.median([a.elapsed_time(b) for a, b in ev]))
+        n = len(wl.calls)
+        out[label] = {"calls": n, "pairs": wl.P * wl.D, "ms": ms, "placed": int((res[0] >= 0).sum().item()),
+                      "us_per_iteration": 1e3 * ms / n}
+        if with_cpu and label == "medium_quarter":
+            from oracle import hx_oracle as ho
+            orc, oc = ho.Oracle(), ho.Cluster.from_workload(wl)
+            dag = orc.longest_path(wl.row_ptr, wl.col, cost, wl.node_wf, wl.n_workflows)
+            t0 = time.perf_counter()
+            orc.greedy(oc, wl.calls, wl.kv_free[wl.P:], dag=dag, node_wf=wl.node_wf, elapsed=wl.elapsed)
+            out[label]["oracle_ms_1_core"] = 1e3 * (time.perf_counter() - t0)
+        gc.close()
+    return out
 
 
 def main():

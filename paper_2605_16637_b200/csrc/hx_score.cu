@@ -295,19 +295,23 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
         for (int ch = 0; ch < prm.nChunks; ++ch) {
             const int pc0 = ch * PC;
             if (prm.nChunks > 1) load_LT(pc0);
-            {   // prefill finish times A[c][p] of this chunk
+            {   // prefill finish times A[c][p] of this chunk: a thread keeps the queue loads and classes
+                // of one p / 4 in registers and walks over the calls, 16 lanes along the calls
                 const int nq = PC >> 2;
-                const int dq = nthr / TCB, dc = nthr - dq * TCB;
-                int q = tid / TCB, c = tid - q * TCB;
-                for (int idx = tid; idx < TCB * nq; idx += nthr) {
+                const int cl = tid & 15, qs = tid >> 4, nqs = nthr >> 4;
+                for (int q = qs; q < nq; q += nqs) {
                     const int p = pc0 + 4 * q;
-                    float a[4];
-#pragma unroll
-                    for (int u = 0; u < 4; ++u)
-                        a[u] = (p + u < Ppad) ? __fadd_rn(qPs[p + u], tpres[typePs[p + u] * TCB + c]) : HX_INF;
-                    *reinterpret_cast<float4*>(As + 4 * (q * AS + c)) = make_float4(a[0], a[1], a[2], a[3]);
-                    q += dq; c += dc;
-                    if (c >= TCB) { c -= TCB; ++q; }
+                    float4 qp = make_float4(HX_INF, HX_INF, HX_INF, HX_INF);
+                    int4 ty = make_int4(0, 0, 0, 0);
+                    if (p < Ppad) {                           // Ppad is a multiple of 4: whole unit or nothing
+                        qp = *reinterpret_cast<const float4*>(qPs + p);
+                        ty = *reinterpret_cast<const int4*>(typePs + p);
+                    }
+                    const float* t0 = tpres + ty.x * TCB; const float* t1 = tpres + ty.y * TCB;
+                    const float* t2 = tpres + ty.z * TCB; const float* t3 = tpres + ty.w * TCB;
+                    for (int c = cl; c < TCB; c += 16)
+                        *reinterpret_cast<float4*>(As + 4 * (q * AS + c)) =
+                            make_float4(__fadd_rn(qp.x, t0[c]), __fadd_rn(qp.y, t1[c]), __fadd_rn(qp.z, t2[c]), __fadd_rn(qp.w, t3[c]));
                 }
             }
             lt_wait();
@@ -405,23 +409,29 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
             } else {
                 int nsel = 0;
                 if (Dpad <= 128) {
-                    // the lane's share of the row (every fourth 16-byte unit) is held in registers; each
-                    // round takes the smallest (finish, d) not taken yet
-                    float vals[32];
+                    // a lane owns every fourth 16-byte unit of the row and keeps the minimum of each unit in
+                    // a register; a round takes the smallest (finish, d) left, and only its owner re-reads
+                    // that unit (the taken entry is overwritten with +inf in shared memory)
+                    float um[8];
+                    float* fr = Fs + cs * FS;
 #pragma unroll
                     for (int it = 0; it < 8; ++it) {
                         const int q = t + 4 * it;
                         float4 f4 = make_float4(HX_INF, HX_INF, HX_INF, HX_INF);
-                        if (4 * q < Dpad) f4 = *reinterpret_cast<const float4*>(frow + 4 * q);
-                        vals[4 * it] = f4.x; vals[4 * it + 1] = f4.y; vals[4 * it + 2] = f4.z; vals[4 * it + 3] = f4.w;
+                        if (4 * q < Dpad) f4 = *reinterpret_cast<const float4*>(fr + 4 * q);
+                        um[it] = fminf(min3(f4.x, f4.y, f4.z), f4.w);
                     }
-                    unsigned taken = 0;
-                    for (int k = 0; k < K; ++k) {
-                        float v = HX_INF; int bi = -1;
+                    for (int k = 0; k < (live ? K : 0); ++k) {     // a group without a call must not write the row
+                        float v = um[0]; int bi = 0;
 #pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            if (!((taken >> i) & 1u) && vals[i] < v) { v = vals[i]; bi = i; }
-                        int d = bi < 0 ? HX_NONE : 16 * (bi >> 2) + 4 * t + (bi & 3);
+                        for (int it = 1; it < 8; ++it)
+                            if (um[it] < v) { v = um[it]; bi = it; }
+                        // position inside the unit: lowest of its four columns holding v
+                        const int qb = t + 4 * bi;            // a unit beyond Dpad has minimum +inf and is never read
+                        float4 f4 = make_float4(HX_INF, HX_INF, HX_INF, HX_INF);
+                        if (v < HX_INF) f4 = *reinterpret_cast<const float4*>(fr + 4 * qb);
+                        const int u = f4.x == v ? 0 : f4.y == v ? 1 : f4.z == v ? 2 : 3;
+                        int d = v < HX_INF ? 4 * qb + u : HX_NONE;
                         const int myd = d;
 #pragma unroll
                         for (int off = 1; off <= 2; off <<= 1) {
@@ -430,7 +440,14 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
                             if (ov < v || (ov == v && od < d)) { v = ov; d = od; }
                         }
                         if (d == HX_NONE) break;              // nothing (feasible) left
-                        if (d == myd) taken |= 1u << bi;
+                        if (d == myd) {                       // owner: retire the entry, refresh the unit minimum
+                            fr[d] = HX_INF;
+                            const float a = u == 0 ? HX_INF : f4.x, b = u == 1 ? HX_INF : f4.y;
+                            const float c2 = u == 2 ? HX_INF : f4.z, e = u == 3 ? HX_INF : f4.w;
+                            const float nu = fminf(min3(a, b, c2), e);
+#pragma unroll
+                            for (int it = 0; it < 8; ++it) um[it] = it == bi ? nu : um[it];
+                        }
 #pragma unroll
                         for (int k2 = 0; k2 < HX_MAX_TOPK; ++k2)
                             if (k2 == k) { sel_d[k2] = d; sel_cost[k2] = v; }
