@@ -168,12 +168,12 @@ __device__ __forceinline__ void group_rescan_multi(const float* a_c, int astride
 #pragma unroll
         for (int k = 0; k < NK; ++k) {
             cand[k] = HX_NONE;
-            if (k < n && valid) {
+            if (valid && ((pending >> k) & 1u)) {            // pending only has bits below n
                 const ulonglong2 l = *reinterpret_cast<const ulonglong2*>(lts + (size_t)q * lstride + 4 * d[k]);
                 float r[4];
                 unpack2(fma2(kk2, l.x, a.x), r[0], r[1]);
                 unpack2(fma2(kk2, l.y, a.y), r[2], r[3]);
-                if (fminf(min3(r[0], r[1], r[2]), r[3]) <= thr[k] && ((pending >> k) & 1u)) {
+                if (fminf(min3(r[0], r[1], r[2]), r[3]) <= thr[k]) {
 #pragma unroll
                     for (int u = 3; u >= 0; --u)
                         if (__fadd_rn(fmaxf(r[u], qd[k]), Dd[k]) == v[k]) cand[k] = 4 * q + u;
@@ -219,12 +219,24 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
     float* mtoks = kvBs + TCB;                                    // [TCB]
     float* tpres = mtoks + TCB;                                   // [G][TCB]
     float* tdecs = tpres + TCB * G;                               // [G][TCB]
+    unsigned* nodeS = reinterpret_cast<unsigned*>(tdecs + TCB * G);   // [TCB] DAG node of the call
+    unsigned* wfS = nodeS + TCB;                                  // [TCB] its workflow
     float* qPs = reinterpret_cast<float*>(smem + prm.offInst);    // [Ppad]
     int* typePs = reinterpret_cast<int*>(qPs + Ppad);             // [Ppad]
     float* qDs = reinterpret_cast<float*>(typePs + Ppad);         // [Dpad]
     float* capDs = qDs + Dpad;                                    // [Dpad]
     int* typeDs = reinterpret_cast<int*>(capDs + Dpad);           // [Dpad]
 
+    // the call records of the first tile come from DRAM: request them before anything else
+    const bool with_dag = !(prm.s.flags & HX_FLAG_NO_DAG);
+    uint4 pre[2];
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+        const int idx = tid + k * nthr, c = idx / G;
+        const int gc = blockIdx.x * TCB + c;
+        pre[k] = make_uint4(0u, 0u, 0u, 0u);
+        if (idx < TCB * G && gc < prm.s.n_calls) pre[k] = __ldg(reinterpret_cast<const uint4*>(prm.s.calls) + gc);
+    }
     // instance tables; padded prefill slots can never win, padded decode columns are infeasible
     for (int p = tid; p < Ppad; p += nthr) {
         qPs[p] = p < P ? (unloaded ? 0.0f : T.qP[p]) : HX_INF;
@@ -262,11 +274,15 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
 
         // per-call service times on every GPU class (roofline-style estimate, Section 4.2):
         // one thread per (call, class)
-        for (int idx = tid; idx < TCB * G; idx += nthr) {
+        int k_it = 0;
+        for (int idx = tid; idx < TCB * G; idx += nthr, ++k_it) {
             const int c = idx / G, g = idx - c * G;
             float n = 1.f, o = 1.f, phi = 0.f, omega = 0.f, kappa = 0.f;
             if (c < nvalid) {
-                const uint4 raw = __ldg(reinterpret_cast<const uint4*>(prm.s.calls) + c0 + c);
+                uint4 raw;
+                if (tile == (int)blockIdx.x && k_it < 2) raw = k_it == 0 ? pre[0] : pre[1];
+                else raw = __ldg(reinterpret_cast<const uint4*>(prm.s.calls) + c0 + c);
+                if (g == 0) nodeS[c] = raw.x;
                 n = __uint_as_float(raw.z); o = __uint_as_float(raw.w);
                 if (raw.y < (unsigned)T.M) { phi = prm.ct.phi[raw.y]; omega = prm.ct.omega[raw.y]; kappa = prm.ct.kappa[raw.y]; }
             }
@@ -280,6 +296,20 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
         }
         lt_wait();
         __syncthreads();
+
+        // workflow of the call: requested now, parked behind the A tile, so that the score at the end
+        // of the tile finds it in shared memory and its three gathers in L2
+        unsigned my_node = 0xFFFFFFFFu, my_wf = 0xFFFFFFFFu;
+        const bool one_pass = TCB <= nthr;                    // one call per thread; else a plain loop
+        if (with_dag && one_pass && tid < nvalid) {
+            my_node = nodeS[tid];
+            if (my_node < prm.dag.n_nodes) my_wf = __ldg(prm.dag.node_wf + my_node);
+        }
+        if (with_dag && !one_pass)
+            for (int c = tid; c < nvalid; c += nthr) {
+                const unsigned nd = nodeS[c];
+                wfS[c] = nd < prm.dag.n_nodes ? __ldg(prm.dag.node_wf + nd) : 0xFFFFFFFFu;
+            }
 
         float acc[TC][TD];
 #pragma unroll
@@ -314,6 +344,14 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
                             make_float4(__fadd_rn(qp.x, t0[c]), __fadd_rn(qp.y, t1[c]), __fadd_rn(qp.z, t2[c]), __fadd_rn(qp.w, t3[c]));
                 }
             }
+            if (ch == 0 && with_dag && one_pass && tid < nvalid) {
+                wfS[tid] = my_wf;
+                if (my_wf != 0xFFFFFFFFu) {
+                    asm volatile("prefetch.global.L2 [%0];" :: "l"(prm.dag.elapsed + my_wf));
+                    asm volatile("prefetch.global.L2 [%0];" :: "l"(prm.dag.H + my_wf));
+                    asm volatile("prefetch.global.L2 [%0];" :: "l"(prm.dag.tail + my_node));
+                }
+            }
             lt_wait();
             __syncthreads();
             const ulonglong2* ap = reinterpret_cast<const ulonglong2*>(As) + wc * (TC * LC) + cg;
@@ -341,6 +379,9 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
 
         // clamp to the decode admission time and add the decode term; park the
         // per-(call, d) finish times in shared memory
+        float mt[TC];
+#pragma unroll
+        for (int i = 0; i < TC; ++i) mt[i] = mtoks[wc * (TC * LC) + cg + LC * i];
 #pragma unroll
         for (int j = 0; j < TD; ++j) {
             const int d = wd * (TD * LD) + dg + LD * j;
@@ -349,7 +390,7 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
 #pragma unroll
             for (int i = 0; i < TC; ++i) {
                 const int c = wc * (TC * LC) + cg + LC * i;
-                const float Dd = (mtoks[c] <= cap) ? tdecs[ty * TCB + c] : HX_INF;
+                const float Dd = (mt[i] <= cap) ? tdecs[ty * TCB + c] : HX_INF;
                 Fs[c * FS + d] = __fadd_rn(fmaxf(acc[i][j], qd), Dd);
             }
         }
@@ -485,7 +526,7 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
                 bool bad = raw.y >= (unsigned)T.M;
                 if (!(prm.s.flags & HX_FLAG_NO_DAG)) {
                     if (raw.x < prm.dag.n_nodes) {
-                        const uint32_t w = prm.dag.node_wf[raw.x];
+                        const uint32_t w = wfS[c];
                         elapsed = prm.dag.elapsed[w];
                         H = prm.dag.H[w];
                         if (!(prm.s.flags & HX_FLAG_NO_TAIL)) tail = prm.dag.tail[raw.x];
@@ -568,14 +609,14 @@ cudaError_t hx_launch_score(const HxTables& t, const HxConstTables& ct, const Hx
     }
     prm.TCB = WCn * TC * LC;
     prm.nTiles = (C + prm.TCB - 1) / prm.TCB;
-    prm.FS = prm.Dpad + 4;
+    prm.FS = prm.Dpad + 8;     // rows 8 banks apart: the clamp phase stores four rows x eight columns per warp
     // strides of the operand tiles: 2 (mod 8) 16-byte units, so that the four lanes of a selection
     // group, which read four consecutive p / 4 of one row, fall into different bank groups
     auto pad_stride = [](int n) { return n + ((2 - n) % 8 + 8) % 8; };
     prm.AS = pad_stride(prm.TCB);
     prm.LS = pad_stride(prm.Dpad);
     const int G = t.G;
-    const size_t callB = round_up(prm.TCB * (2 + 2 * G) * 4, 16);
+    const size_t callB = round_up(prm.TCB * (4 + 2 * G) * 4, 16);
     const size_t instB = round_up((2 * t.Ppad + 3 * prm.Dpad) * 4, 16);
     if (callB + instB + 4096 > max_smem) return cudaErrorInvalidConfiguration;
     const size_t budget = max_smem - callB - instB - 64;
