@@ -143,6 +143,27 @@ int hx_dag_upload(hx_cluster* h, const uint32_t* row_ptr, const uint32_t* col_id
  * traversal order.  Enqueues on `stream`. */
 int hx_critical_path(hx_cluster* h, void* stream);
 
+/* Online horizon refinement (Section 5.1, "Define online workflow horizon": the
+ * horizon is kept up to date as the workflow proceeds and cost estimates are
+ * replaced by observed latencies; Algorithm 1, horizon update).
+ * hx_dag_update_costs replaces the cost of n_updates nodes (host arrays: node
+ * ids in the numbering of the upload, new costs in seconds; if a node is listed
+ * more than once its last value counts) and recomputes cp, tail and H of the
+ * workflows these nodes belong to, and of no other; the result equals a full
+ * hx_critical_path over the updated costs bit for bit.  If hx_critical_path has
+ * not run since the upload, only the costs are replaced.  The host arrays may
+ * be reused on return; the work is enqueued on `stream`.  The first call (and
+ * a call larger than any before) allocates scratch for the update lists and
+ * synchronises the device while doing so.  Errors: HX_ERR_NOT_READY without an
+ * upload, HX_ERR_INVALID_ARG for ids out of range or costs that are negative
+ * or not finite (nothing is changed then).
+ * hx_dag_update_elapsed replaces the elapsed time (t - a_w) of every workflow
+ * (host array of n_workflows values), which Eq. 2 needs afresh at every
+ * scheduler invocation; the structure and the horizons stay as they are. */
+int hx_dag_update_costs(hx_cluster* h, const uint32_t* node_ids, const float* new_costs,
+                        uint32_t n_updates, void* stream);
+int hx_dag_update_elapsed(hx_cluster* h, const float* workflow_elapsed_s, void* stream);
+
 /* Borrowed device pointers to cp[n_nodes], tail[n_nodes] (original node
  * numbering) and H[n_workflows]; valid until the next upload or destroy.
  * Any of the three output arguments may be NULL. */

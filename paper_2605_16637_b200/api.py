@@ -52,6 +52,8 @@ def _load():
         "hx_cluster_destroy": [vp],
         "hx_dag_upload": [vp, vp, vp, vp, vp, vp, u32, u32, u32],
         "hx_critical_path": [vp, vp],
+        "hx_dag_update_costs": [vp, vp, vp, u32, vp],
+        "hx_dag_update_elapsed": [vp, vp, vp],
         "hx_get_dag_results": [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp)],
         "hx_set_options": [vp, C.POINTER(_Options)],
         "hx_schedule_batch": [vp, vp, ci, vp, vp, vp],
@@ -132,6 +134,20 @@ def hx_dag_upload(h, row_ptr, col_idx, node_costs, node_workflow, workflow_elaps
 
 def hx_critical_path(h, stream=0):
     _check(_lib.hx_critical_path(h, stream), h)
+
+
+def hx_dag_update_costs(h, node_ids, new_costs, stream=0):
+    """Replace node cost estimates (e.g. by observed latencies) and refresh the horizons of the
+    workflows they belong to."""
+    node_ids = _np(node_ids, np.uint32); new_costs = _np(new_costs, np.float32)
+    if node_ids.shape[0] != new_costs.shape[0]:
+        raise HxError(-1, "node_ids and new_costs differ in length")
+    _check(_lib.hx_dag_update_costs(h, _p(node_ids), _p(new_costs), node_ids.shape[0], stream), h)
+
+
+def hx_dag_update_elapsed(h, workflow_elapsed_s, stream=0):
+    el = _np(workflow_elapsed_s, np.float32)
+    _check(_lib.hx_dag_update_elapsed(h, _p(el), stream), h)
 
 
 def hx_get_dag_results(h):
@@ -268,6 +284,15 @@ class Cluster:
 
     def critical_path(self):
         hx_critical_path(self.h, self._stream())
+
+    def update_costs(self, node_ids, new_costs):
+        hx_dag_update_costs(self.h, node_ids, new_costs, self._stream())
+
+    def update_elapsed(self, workflow_elapsed_s):
+        el = _np(workflow_elapsed_s, np.float32)
+        if el.shape[0] != self.n_workflows:
+            raise HxError(-1, "one elapsed time per workflow is needed")
+        hx_dag_update_elapsed(self.h, el, self._stream())
 
     def dag_results(self):
         """cp, tail, H as numpy arrays (synchronises)."""

@@ -115,7 +115,23 @@ __global__ void hx_cpath_global_kernel(HxForestDev f, const uint32_t* __restrict
     if (t == 0) f.H[w] = hmax;
 }
 
+// Replaces the cost estimates of some nodes (internal numbering) by newer values, e.g. observed
+// latencies (Section 5.1, "Define online workflow horizon").
+__global__ void hx_cost_update_kernel(float* __restrict__ icost, const uint32_t* __restrict__ idx,
+                                      const float* __restrict__ cost, uint32_t n) {
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) icost[idx[i]] = cost[i];
+}
+
 }  // namespace
+
+cudaError_t hx_launch_cost_update(const HxForestDev& f, const uint32_t* idx, const float* cost, uint32_t n,
+                                  cudaStream_t stream, long long* launches) {
+    if (n == 0) return cudaSuccess;
+    hx_cost_update_kernel<<<(n + 255) / 256, 256, 0, stream>>>(const_cast<float*>(f.icost), idx, cost, n);
+    ++*launches;
+    return cudaGetLastError();
+}
 
 cudaError_t hx_launch_cpath(const HxForestDev& f, const HxCpClass* classes, int n_classes,
                             cudaStream_t stream, long long* launches) {

@@ -26,6 +26,12 @@ struct hx_cluster {
     uint32_t* d_node_wf = nullptr;
     float* d_elapsed = nullptr;
     std::vector<HxCpClass> classes;
+    // host copies for incremental refinement: node -> internal index, node -> workflow, workflow -> class
+    std::vector<uint32_t> h_inv, h_node_wf;
+    std::vector<uint8_t> h_wf_class;
+    std::vector<void*> upd_allocs;      // scratch of hx_dag_update_costs, grown on demand
+    uint32_t* d_upd_idx = nullptr; float* d_upd_cost = nullptr; uint32_t* d_upd_wf = nullptr;
+    size_t upd_cap = 0, upd_wf_cap = 0;
     // top-K
     HxTopkBufs tk{};
     // staging for the host-buffer entry point
@@ -268,7 +274,7 @@ int hx_cluster_destroy(hx_cluster* h) {
     if (!h) return HX_OK;
     DeviceGuard guard(h->device);
     cudaDeviceSynchronize();
-    free_pool(h->allocs); free_pool(h->dag_allocs); free_pool(h->tk_allocs);
+    free_pool(h->allocs); free_pool(h->dag_allocs); free_pool(h->tk_allocs); free_pool(h->upd_allocs);
     if (h->st_calls) cudaFree(h->st_calls);
     if (h->st_assign) cudaFree(h->st_assign);
     if (h->st_cost) cudaFree(h->st_cost);
@@ -361,14 +367,17 @@ int hx_dag_upload(hx_cluster* h, const uint32_t* row_ptr, const uint32_t* col_id
     for (uint32_t w = 0; w <= W; ++w) wf_edge_start[w] = irow[wf_node_start[w]];
 
     // classes of the horizon pass by staging footprint
-    const size_t kWarpSmall = 3072, kWarpBig = 24576, kBlock = 200 * 1024;
+    const size_t kWarpSmall = hx_cpath_class_shape(0).smem_per_wf, kWarpBig = hx_cpath_class_shape(1).smem_per_wf,
+                 kBlock = hx_cpath_class_shape(2).smem_per_wf;
     std::vector<uint32_t> ids[4];
+    std::vector<uint8_t> wf_class(W);
     for (uint32_t w = 0; w < W; ++w) {
         const size_t n = wf_node_start[w + 1] - wf_node_start[w], e = wf_edge_start[w + 1] - wf_edge_start[w];
         const size_t nlev = wf_seg_start[w + 1] - wf_seg_start[w] - 1;
         const size_t need = 4 * (3 * n + 1) + 4 * (nlev + 1) + 2 * e + 16;
         const int k = (n > 65535) ? 3 : need <= kWarpSmall ? 0 : need <= kWarpBig ? 1 : need <= kBlock ? 2 : 3;
         ids[k].push_back(w);
+        wf_class[w] = (uint8_t)k;
     }
     // largest workflows first inside a class, so that the long ones do not start last
     for (auto& v : ids)
@@ -400,15 +409,18 @@ int hx_dag_upload(hx_cluster* h, const uint32_t* row_ptr, const uint32_t* col_id
     std::vector<float> el(workflow_elapsed_s, workflow_elapsed_s + W);
     HX_TRY(dev_upload(h->dag_allocs, &h->d_node_wf, nwf), "upload node_workflow");
     HX_TRY(dev_upload(h->dag_allocs, &h->d_elapsed, el), "upload elapsed");
-    const int tpw[4] = {32, 32, 256, 256}, per_block[4] = {16, 8, 1, 1};
-    const size_t sm[4] = {kWarpSmall, kWarpBig, kBlock, 0};
     for (int k = 0; k < 4; ++k) {
         if (ids[k].empty()) continue;
         uint32_t* d_ids;
         HX_TRY(dev_upload(h->dag_allocs, &d_ids, ids[k]), "upload workflow classes");
-        h->classes.push_back(HxCpClass{d_ids, (uint32_t)ids[k].size(), tpw[k], per_block[k], sm[k]});
+        HxCpClass c = hx_cpath_class_shape(k);
+        c.wf_ids = d_ids; c.count = (uint32_t)ids[k].size();
+        h->classes.push_back(c);
     }
     h->forest = f;
+    h->h_inv = inv;
+    h->h_node_wf.assign(node_workflow, node_workflow + N);
+    h->h_wf_class = wf_class;
     h->dag_uploaded = true;
     return HX_OK;
 }
@@ -423,6 +435,85 @@ int hx_critical_path(hx_cluster* h, void* stream) {
                                static_cast<cudaStream_t>(stream), &h->launches), "horizon kernels");
     }
     h->cp_ready = true;
+    return HX_OK;
+}
+
+int hx_dag_update_elapsed(hx_cluster* h, const float* workflow_elapsed_s, void* stream) {
+    if (!h) return HX_ERR_INVALID_ARG;
+    if (!h->dag_uploaded) return fail(h, HX_ERR_NOT_READY, "no forest uploaded");
+    if (!workflow_elapsed_s) return fail(h, HX_ERR_INVALID_ARG, "NULL array");
+    const uint32_t W = h->forest.n_workflows;
+    for (uint32_t w = 0; w < W; ++w)
+        if (!good_load(workflow_elapsed_s[w])) return fail(h, HX_ERR_INVALID_ARG, "elapsed times must be finite and >= 0");
+    DeviceGuard guard(h->device);
+    HX_TRY(cudaMemcpyAsync(h->d_elapsed, workflow_elapsed_s, (size_t)W * sizeof(float), cudaMemcpyHostToDevice,
+                           static_cast<cudaStream_t>(stream)), "cudaMemcpyAsync(elapsed)");
+    return HX_OK;
+}
+
+int hx_dag_update_costs(hx_cluster* h, const uint32_t* node_ids, const float* new_costs, uint32_t n_updates,
+                        void* stream) {
+    if (!h) return HX_ERR_INVALID_ARG;
+    if (!h->dag_uploaded) return fail(h, HX_ERR_NOT_READY, "no forest uploaded");
+    if (n_updates == 0) return HX_OK;
+    if (!node_ids || !new_costs) return fail(h, HX_ERR_INVALID_ARG, "NULL array");
+    const uint32_t N = h->forest.n_nodes, W = h->forest.n_workflows;
+    for (uint32_t i = 0; i < n_updates; ++i) {
+        if (node_ids[i] >= N) return fail(h, HX_ERR_INVALID_ARG, "node id out of range");
+        if (!good_load(new_costs[i])) return fail(h, HX_ERR_INVALID_ARG, "node costs must be finite and >= 0");
+    }
+    // the last value given for a node wins; the workflows touched are recomputed, nothing else
+    std::vector<uint32_t> idx; std::vector<float> val;
+    idx.reserve(n_updates); val.reserve(n_updates);
+    std::vector<uint32_t> dirty[4];
+    {
+        std::vector<uint32_t> order(n_updates);
+        for (uint32_t i = 0; i < n_updates; ++i) order[i] = i;
+        std::stable_sort(order.begin(), order.end(), [&](uint32_t a, uint32_t b) { return node_ids[a] < node_ids[b]; });
+        std::vector<uint32_t> wfs;
+        for (uint32_t i = 0; i < n_updates; ++i) {
+            if (i + 1 < n_updates && node_ids[order[i + 1]] == node_ids[order[i]]) continue;
+            const uint32_t v = node_ids[order[i]];
+            idx.push_back(h->h_inv[v]); val.push_back(new_costs[order[i]]);
+            wfs.push_back(h->h_node_wf[v]);
+        }
+        std::sort(wfs.begin(), wfs.end());
+        wfs.erase(std::unique(wfs.begin(), wfs.end()), wfs.end());
+        for (uint32_t w : wfs) dirty[h->h_wf_class[w]].push_back(w);
+    }
+    DeviceGuard guard(h->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    size_t n_wf = 0;
+    for (auto& v : dirty) n_wf += v.size();
+    if (idx.size() > h->upd_cap || n_wf > h->upd_wf_cap) {
+        cudaDeviceSynchronize();
+        free_pool(h->upd_allocs);
+        h->upd_cap = std::max<size_t>(idx.size(), 4096); h->upd_wf_cap = std::max<size_t>(n_wf, 4096);
+        HX_TRY(dev_alloc(h->upd_allocs, &h->d_upd_idx, h->upd_cap), "alloc update scratch");
+        HX_TRY(dev_alloc(h->upd_allocs, &h->d_upd_cost, h->upd_cap), "alloc update scratch");
+        HX_TRY(dev_alloc(h->upd_allocs, &h->d_upd_wf, h->upd_wf_cap), "alloc update scratch");
+    }
+    HX_TRY(cudaMemcpyAsync(h->d_upd_idx, idx.data(), idx.size() * sizeof(uint32_t), cudaMemcpyHostToDevice, s), "copy updates");
+    HX_TRY(cudaMemcpyAsync(h->d_upd_cost, val.data(), val.size() * sizeof(float), cudaMemcpyHostToDevice, s), "copy updates");
+    std::vector<HxCpClass> part;
+    size_t off = 0;
+    for (int k = 0; k < 4; ++k) {
+        if (dirty[k].empty()) continue;
+        HX_TRY(cudaMemcpyAsync(h->d_upd_wf + off, dirty[k].data(), dirty[k].size() * sizeof(uint32_t),
+                               cudaMemcpyHostToDevice, s), "copy dirty workflows");
+        HxCpClass c = hx_cpath_class_shape(k);
+        c.wf_ids = h->d_upd_wf + off; c.count = (uint32_t)dirty[k].size();
+        part.push_back(c);
+        off += dirty[k].size();
+    }
+    // pageable host memory: the copies above have read the vectors by the time they return
+    {
+        SpanGuard span(h, 2, s);
+        HX_TRY(hx_launch_cost_update(h->forest, h->d_upd_idx, h->d_upd_cost, (uint32_t)idx.size(), s, &h->launches), "cost update kernel");
+        if (h->cp_ready)
+            HX_TRY(hx_launch_cpath(h->forest, part.data(), (int)part.size(), s, &h->launches), "horizon kernels");
+    }
+    (void)W;
     return HX_OK;
 }
 

@@ -136,6 +136,18 @@ struct HxCpClass {
 cudaError_t hx_launch_cpath(const HxForestDev& f, const HxCpClass* classes, int n_classes,
                             cudaStream_t stream, long long* launches);
 
+// Launch shape of workflow class k (by staging footprint): 0 = one warp, <= 3 KB; 1 = one warp,
+// <= 24 KB; 2 = one block, <= 200 KB; 3 = one block working in global memory.
+inline HxCpClass hx_cpath_class_shape(int k) {
+    const int tpw[4] = {32, 32, 256, 256}, per_block[4] = {16, 8, 1, 1};
+    const size_t sm[4] = {3072, 24576, 200 * 1024, 0};
+    return HxCpClass{nullptr, 0, tpw[k], per_block[k], sm[k]};
+}
+
+// icost[idx[i]] = cost[i] (internal node numbering), ahead of a partial horizon pass.
+cudaError_t hx_launch_cost_update(const HxForestDev& f, const uint32_t* idx, const float* cost, uint32_t n,
+                                  cudaStream_t stream, long long* launches);
+
 // Opt a kernel in to `bytes` of dynamic shared memory, once per device and size: the attribute
 // call is too slow to repeat on every launch.  `allowed` is a per-kernel table of 64 entries
 // that starts at the size the kernel may use without opting in.

@@ -383,3 +383,22 @@ def test_oracle_runs_on_generated_configs(oracle):
         a, score, delta = oracle.schedule(cl, wl.calls, mode=ho.MODE_SLACK, alpha=wl.alpha, dag=dag,
                                           node_wf=wl.node_wf, elapsed=wl.elapsed)
         assert np.all(a >= 0) and np.all(a < wl.P * wl.D) and np.all(np.isfinite(score))
+
+
+def test_cost_change_stays_inside_its_workflow_and_is_monotone(oracle):
+    """Workflows are independent components: replacing a node's cost estimate by an observed latency
+    (Section 5.1) can only change the nodes of that workflow that reach the node, a larger cost never
+    shortens any path, and the node's own tail is untouched."""
+    wl = make_workload("medium", scale=0.25)
+    rng = np.random.default_rng(3)
+    cost = rng.lognormal(0, 1, wl.n_nodes).astype(np.float32)
+    base = oracle.longest_path(wl.row_ptr, wl.col, cost, wl.node_wf, wl.n_workflows)
+    v = int(rng.integers(0, wl.n_nodes))
+    up = cost.copy(); up[v] = cost[v] * np.float32(3.0)
+    new = oracle.longest_path(wl.row_ptr, wl.col, up, wl.node_wf, wl.n_workflows)
+    other = wl.node_wf != wl.node_wf[v]
+    assert np.array_equal(new.cp[other], base.cp[other]) and np.array_equal(new.tail[other], base.tail[other])
+    keep = np.ones(wl.n_workflows, bool); keep[wl.node_wf[v]] = False
+    assert np.array_equal(new.H[keep], base.H[keep])
+    assert np.all(new.cp >= base.cp) and np.all(new.H >= base.H)
+    assert new.tail[v] == base.tail[v] and new.cp[v] == np.float32(up[v] + base.tail[v])
