@@ -309,6 +309,96 @@ int orc_greedy(const OrcCluster* cl, const OrcDag* dag, const OrcCall* calls, in
     return placed;
 }
 
+// Decode-stage scheduler (Section 5.4): calls whose KV cache has arrived wait for
+// decode admission.  Ranking by the projected ratio (Eq. 2), feasibility by the
+// decode KV capacity (Eq. 3-4), now over time: every decode instance carries its
+// token-capacity intervals (Section 6: "decode token-capacity intervals"), i.e.
+// which calls hold how many KV tokens until when.
+// "Adaptive greedy decode assignment": repeatedly take the most urgent waiting
+// call, find the earliest capacity-feasible start on every legal instance,
+// assign it to the instance with the earliest projected finish, and add its
+// interval to the simulated state.  A call locked to an instance (chosen during
+// prefill planning) may only go there; a free call may go to any instance that
+// can ever hold it (m <= Cap).
+//
+// Usage of instance d over time is a step function: breakpoints t[0] = 0 < t[1] <
+// ... and tokens in use u[k] on [t[k], t[k+1]) (the last segment runs to +inf).
+// Earliest feasible start of a call with demand m, duration tau, ready at r:
+// walk the segments from the one holding r; a segment with u[k] + m > Cap pushes
+// the candidate start to its end; the candidate is accepted as soon as a segment
+// ends at or after candidate + tau (binary32 addition) without such a push.
+struct StepFn { std::vector<float> t, u; };     // t.size() == u.size() >= 1, t[0] == 0
+
+static float earliest_start(const StepFn& f, float cap, float m, float tau, float ready, float* finish) {
+    size_t k = 0;
+    while (k + 1 < f.t.size() && f.t[k + 1] <= ready) ++k;      // segment that holds the ready time
+    float cand = ready;
+    for (;; ++k) {
+        const float seg_end = (k + 1 < f.t.size()) ? f.t[k + 1] : INF;
+        if (f.u[k] + m > cap) { cand = seg_end; continue; }       // no room here: not before this segment ends
+        const float fin = cand + tau;
+        if (seg_end >= fin) { *finish = fin; return cand; }
+    }
+}
+
+static void add_interval(StepFn& f, float s, float e, float m) {
+    auto cut = [&](float x) {                                     // make x a breakpoint; returns its index
+        size_t k = 0;
+        while (k + 1 < f.t.size() && f.t[k + 1] <= x) ++k;
+        if (f.t[k] == x) return k;
+        f.t.insert(f.t.begin() + k + 1, x);
+        f.u.insert(f.u.begin() + k + 1, f.u[k]);
+        return k + 1;
+    };
+    const size_t a = cut(s), b = cut(e);
+    for (size_t k = a; k < b; ++k) f.u[k] = f.u[k] + m;
+}
+
+// run_ptr[D+1], run_end[], run_tok[]: calls decoding now on each instance (each holds run_tok
+// tokens until run_end seconds from now).  lock[c] = -1 or a decode instance; ready[c] = time the
+// KV cache of c is on the decode side.  Outputs: inst[c] (-1 if it fits nowhere), start[c],
+// ratio[c] = R at selection, order[i]; returns the number of placed calls.
+int orc_decode_greedy(const OrcCluster* cl, const OrcDag* dag, const OrcCall* calls, int C, int flags,
+                      const uint32_t* run_ptr, const float* run_end, const float* run_tok,
+                      const int32_t* lock, const float* ready,
+                      int32_t* inst, float* start, float* ratio, int32_t* order) {
+    const int D = cl->D;
+    std::vector<StepFn> fn(D);
+    for (int d = 0; d < D; ++d) {
+        fn[d].t.assign(1, 0.0f); fn[d].u.assign(1, 0.0f);
+        for (uint32_t i = run_ptr[d]; i < run_ptr[d + 1]; ++i) add_interval(fn[d], 0.0f, run_end[i], run_tok[i]);
+    }
+    std::vector<Terms> terms(C);
+    std::vector<char> waiting(C, 1);
+    for (int c = 0; c < C; ++c) { latency_terms(*cl, calls[c], terms[c]); inst[c] = -1; start[c] = INF; ratio[c] = INF; order[c] = -1; }
+    int placed = 0;
+    for (int it = 0; it < C; ++it) {
+        int best_c = -1, best_d = -1; float best_R = -INF, best_s = 0.0f, best_f = 0.0f;
+        for (int c = 0; c < C; ++c) {
+            if (!waiting[c]) continue;
+            const Terms& t = terms[c];
+            float fin = INF, st = 0.0f; int arg = -1;
+            for (int d = 0; d < D; ++d) {
+                if (lock[c] >= 0 && lock[c] != d) continue;     // locked calls do not migrate
+                if (!(t.m <= cl->capD[d])) continue;            // Eq. 4
+                float f;
+                const float s = earliest_start(fn[d], cl->capD[d], t.m, t.tdec[cl->typeD[d]], ready[c], &f);
+                if (f < fin) { fin = f; st = s; arg = d; }
+            }
+            if (arg < 0) continue;
+            const DagView v = dag_view(dag, calls[c], flags);
+            const float R = (v.elapsed + fin) / v.H;            // Eq. 2 with Delta_D = projected decode finish
+            if (R > best_R) { best_R = R; best_c = c; best_d = arg; best_s = st; best_f = fin; }
+        }
+        if (best_c < 0) break;
+        add_interval(fn[best_d], best_s, best_f, terms[best_c].m);
+        inst[best_c] = best_d; start[best_c] = best_s; ratio[best_c] = best_R; order[it] = best_c;
+        waiting[best_c] = 0;
+        ++placed;
+    }
+    return placed;
+}
+
 // Longest node-weighted path to a sink, per node, over a successor-CSR DAG:
 //   tail[v] = max over successors u of cp[u]   (0 without successors)
 //   cp[v]   = cost[v] + tail[v]

@@ -204,3 +204,22 @@ class Oracle:
         placed = self.lib.orc_greedy(C.byref(c), C.byref(d) if d is not None else None, _ptr(calls), n,
                                      int(flags), _ptr(qP), _ptr(free), _ptr(assign), _ptr(ratio), _ptr(order))
         return assign, ratio, order, int(placed), qP, free
+
+    def decode_greedy(self, cl: Cluster, calls, run_ptr, run_end, run_tok, lock, ready, flags=0,
+                      dag: DagResult | None = None, node_wf=None, elapsed=None):
+        """Decode-stage greedy over capacity intervals (Section 5.4).
+        Returns (inst i32[C], start f32[C], ratio f32[C], order i32[C], n_placed)."""
+        calls, n = self._calls(calls)
+        run_ptr = _u32(run_ptr); run_end = _f32(run_end); run_tok = _f32(run_tok)
+        lock = np.ascontiguousarray(lock, np.int32); ready = _f32(ready)
+        inst = np.zeros(n, np.int32); start = np.zeros(n, np.float32); ratio = np.zeros(n, np.float32)
+        order = np.zeros(n, np.int32)
+        c = cl._c()
+        d, keep = self._dag(dag, node_wf, elapsed)
+        if d is None:
+            flags |= FLAG_NO_DAG
+        self.lib.orc_decode_greedy.restype = C.c_int
+        placed = self.lib.orc_decode_greedy(C.byref(c), C.byref(d) if d is not None else None, _ptr(calls), n,
+                                            int(flags), _ptr(run_ptr), _ptr(run_end), _ptr(run_tok), _ptr(lock),
+                                            _ptr(ready), _ptr(inst), _ptr(start), _ptr(ratio), _ptr(order))
+        return inst, start, ratio, order, int(placed)
