@@ -255,6 +255,48 @@ int hx_schedule_batch_static(hx_cluster* h, const hx_call* calls, int n_calls,
 int hx_schedule_greedy(hx_cluster* h, const hx_call* calls, int n_calls,
                        int32_t* out_assign, float* out_ratio, int32_t* out_order, void* stream);
 
+/* Decode-stage scheduler (Section 5.4, "Decode scheduling with instance locks",
+ * "Decode KV-capacity feasibility check", "Adaptive greedy decode assignment").
+ * State: the decode token-capacity intervals of every decode instance
+ * (Section 6), i.e. which calls hold how many KV tokens until when.
+ *
+ * hx_decode_set_running loads the snapshot: inst_ptr[n_decode + 1] (host, CSR
+ * offsets into `running`) and one hx_kv_interval per call that is decoding now
+ * (end_s: seconds from now until it finishes, finite and > 0; tokens: the KV
+ * tokens it holds, a whole number; the tokens in use on one instance must stay
+ * below 2^24).  An instance may have no running call.  Enqueues copies on
+ * `stream`; the host arrays may be reused on return; may (re)allocate, which
+ * synchronises the device.
+ *
+ * hx_schedule_decode plans the queue of calls whose KV cache is (or will be) on
+ * the decode side.  calls: device, n_calls records (1..HX_DECODE_MAX_CALLS).
+ * lock: device int32[n_calls] or NULL: -1 = free call, else the decode instance
+ * the call was planned on during prefill scheduling (it cannot migrate).
+ * ready_s: device float[n_calls] or NULL (= 0): time from now at which the
+ * call's KV cache is on the decode side.  Until the queue is empty the most
+ * urgent waiting call (largest R = (elapsed_w + Delta_D) / H_w, Eq. 2; lower index
+ * among equals) is assigned: on every legal instance (its lock, or every
+ * instance with m(c) <= Cap(d), Eq. 3-4) the earliest start >= ready_s is found
+ * at which m(c) tokens are free for the whole decode time of the call on that
+ * instance's GPU class; Delta_D is the earliest finish over those instances
+ * (lower instance index among equals); the interval is added to the simulated
+ * state.  out_inst: device int32[n_calls], decode instance or -1 (the call
+ * exceeds Cap of every legal instance).  out_start: planned decode start.
+ * out_ratio: R when taken (+inf if never).  out_order: out_order[i] = call
+ * taken in iteration i, -1 after the last.  With hx_options.commit the simulated
+ * intervals become the snapshot of the next call; otherwise the snapshot is
+ * left as it was.  Uses HX_FLAG_NO_DAG like hx_schedule_batch.  Errors:
+ * HX_ERR_NOT_READY without a snapshot or horizons; HX_ERR_INVALID_ARG for sizes
+ * out of range; a record with an id out of range, a lock >= n_decode or a
+ * ready time that is negative or not finite is left unassigned and raises
+ * HX_ERR_INVALID_ARG in the status word.  Enqueues one kernel on `stream`. */
+typedef struct { float end_s; float tokens; } hx_kv_interval;
+#define HX_DECODE_MAX_CALLS 2048
+int hx_decode_set_running(hx_cluster* h, const uint32_t* inst_ptr, const hx_kv_interval* running, void* stream);
+int hx_schedule_decode(hx_cluster* h, const hx_call* calls, const int32_t* lock, const float* ready_s,
+                       int n_calls, int32_t* out_inst, float* out_start, float* out_ratio,
+                       int32_t* out_order, void* stream);
+
 /* Borrowed device pointers to the top-K results of the last batch scored with
  * topk = K > 0: pairs int32[n_calls][K] (-1 = unused slot), costs
  * float[n_calls][K] (projected decode finish of that pair, +inf if unused),

@@ -354,19 +354,21 @@ static void add_interval(StepFn& f, float s, float e, float m) {
     for (size_t k = a; k < b; ++k) f.u[k] = f.u[k] + m;
 }
 
-// run_ptr[D+1], run_end[], run_tok[]: calls decoding now on each instance (each holds run_tok
-// tokens until run_end seconds from now).  lock[c] = -1 or a decode instance; ready[c] = time the
+// run_ptr[D+1], run_start[] (NULL = all 0), run_end[], run_tok[]: intervals already on each instance
+// (calls decoding now hold run_tok tokens from 0 until run_end seconds from now; intervals planned
+// earlier may start later).  lock[c] = -1 or a decode instance; ready[c] = time the
 // KV cache of c is on the decode side.  Outputs: inst[c] (-1 if it fits nowhere), start[c],
 // ratio[c] = R at selection, order[i]; returns the number of placed calls.
 int orc_decode_greedy(const OrcCluster* cl, const OrcDag* dag, const OrcCall* calls, int C, int flags,
-                      const uint32_t* run_ptr, const float* run_end, const float* run_tok,
+                      const uint32_t* run_ptr, const float* run_start, const float* run_end, const float* run_tok,
                       const int32_t* lock, const float* ready,
                       int32_t* inst, float* start, float* ratio, int32_t* order) {
     const int D = cl->D;
     std::vector<StepFn> fn(D);
     for (int d = 0; d < D; ++d) {
         fn[d].t.assign(1, 0.0f); fn[d].u.assign(1, 0.0f);
-        for (uint32_t i = run_ptr[d]; i < run_ptr[d + 1]; ++i) add_interval(fn[d], 0.0f, run_end[i], run_tok[i]);
+        for (uint32_t i = run_ptr[d]; i < run_ptr[d + 1]; ++i)
+            add_interval(fn[d], run_start ? run_start[i] : 0.0f, run_end[i], run_tok[i]);
     }
     std::vector<Terms> terms(C);
     std::vector<char> waiting(C, 1);

@@ -206,11 +206,12 @@ class Oracle:
         return assign, ratio, order, int(placed), qP, free
 
     def decode_greedy(self, cl: Cluster, calls, run_ptr, run_end, run_tok, lock, ready, flags=0,
-                      dag: DagResult | None = None, node_wf=None, elapsed=None):
+                      dag: DagResult | None = None, node_wf=None, elapsed=None, run_start=None):
         """Decode-stage greedy over capacity intervals (Section 5.4).
         Returns (inst i32[C], start f32[C], ratio f32[C], order i32[C], n_placed)."""
         calls, n = self._calls(calls)
         run_ptr = _u32(run_ptr); run_end = _f32(run_end); run_tok = _f32(run_tok)
+        run_start = None if run_start is None else _f32(run_start)
         lock = np.ascontiguousarray(lock, np.int32); ready = _f32(ready)
         inst = np.zeros(n, np.int32); start = np.zeros(n, np.float32); ratio = np.zeros(n, np.float32)
         order = np.zeros(n, np.int32)
@@ -220,6 +221,7 @@ class Oracle:
             flags |= FLAG_NO_DAG
         self.lib.orc_decode_greedy.restype = C.c_int
         placed = self.lib.orc_decode_greedy(C.byref(c), C.byref(d) if d is not None else None, _ptr(calls), n,
-                                            int(flags), _ptr(run_ptr), _ptr(run_end), _ptr(run_tok), _ptr(lock),
+                                            int(flags), _ptr(run_ptr), None if run_start is None else _ptr(run_start),
+                                            _ptr(run_end), _ptr(run_tok), _ptr(lock),
                                             _ptr(ready), _ptr(inst), _ptr(start), _ptr(ratio), _ptr(order))
         return inst, start, ratio, order, int(placed)

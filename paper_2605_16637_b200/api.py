@@ -60,6 +60,8 @@ def _load():
         "hx_schedule_batch_host": [vp, vp, ci, vp, vp, vp],
         "hx_schedule_batch_static": [vp, vp, ci, vp, vp, vp],
         "hx_schedule_greedy": [vp, vp, ci, vp, vp, vp, vp],
+        "hx_decode_set_running": [vp, vp, vp, vp],
+        "hx_schedule_decode": [vp, vp, vp, vp, ci, vp, vp, vp, vp, vp],
         "hx_get_topk": [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp)],
         "hx_get_status": [vp, C.POINTER(ci), vp],
         "hx_enable_kernel_timing": [vp, ci],
@@ -176,6 +178,24 @@ def hx_schedule_greedy(h, calls_ptr, n_calls, out_assign_ptr, out_ratio_ptr, out
     """Recomputing greedy planner for small queues (Algorithm 1); device pointers."""
     _check(_lib.hx_schedule_greedy(h, calls_ptr, int(n_calls), out_assign_ptr, out_ratio_ptr, out_order_ptr,
                                    stream), h)
+
+
+KV_INTERVAL_DTYPE = np.dtype([("end_s", "<f4"), ("tokens", "<f4")])
+
+
+def hx_decode_set_running(h, inst_ptr, running, stream=0):
+    """inst_ptr: CSR offsets per decode instance; running: KV_INTERVAL_DTYPE records (host)."""
+    inst_ptr = _np(inst_ptr, np.uint32); running = _np(running, KV_INTERVAL_DTYPE)
+    if inst_ptr.shape[0] < 1 or inst_ptr[-1] != running.shape[0]:
+        raise HxError(-1, "inst_ptr does not span the running calls")
+    _check(_lib.hx_decode_set_running(h, _p(inst_ptr), _p(running), stream), h)
+
+
+def hx_schedule_decode(h, calls_ptr, lock_ptr, ready_ptr, n_calls, out_inst_ptr, out_start_ptr, out_ratio_ptr,
+                       out_order_ptr, stream=0):
+    """Decode-stage scheduler over token-capacity intervals (Section 5.4); device pointers."""
+    _check(_lib.hx_schedule_decode(h, calls_ptr, lock_ptr, ready_ptr, int(n_calls), out_inst_ptr, out_start_ptr,
+                                   out_ratio_ptr, out_order_ptr, stream), h)
 
 
 def hx_schedule_batch_host(h, calls, out_assign=None, out_cost=None, stream=0):
@@ -330,6 +350,29 @@ class Cluster:
         hx_schedule_greedy(self.h, calls.data_ptr(), n, assign.data_ptr(), ratio.data_ptr(), order.data_ptr(),
                            self._stream())
         return assign, ratio, order
+
+    def decode_set_running(self, inst_ptr, end_s, tokens):
+        run = np.zeros(len(end_s), KV_INTERVAL_DTYPE)
+        run["end_s"] = end_s; run["tokens"] = tokens
+        hx_decode_set_running(self.h, inst_ptr, run, self._stream())
+
+    def schedule_decode(self, calls, lock=None, ready_s=None):
+        """Returns (inst, start, ratio, order) CUDA tensors."""
+        import torch
+        if isinstance(calls, np.ndarray):
+            calls = torch.from_numpy(_np(calls, CALL_DTYPE).view(np.uint8).copy()).cuda()
+        n = calls.numel() * calls.element_size() // 16
+        lk = None if lock is None else torch.as_tensor(np.ascontiguousarray(lock, np.int32)).cuda()
+        rd = None if ready_s is None else torch.as_tensor(np.ascontiguousarray(ready_s, np.float32)).cuda()
+        inst = torch.empty(n, dtype=torch.int32, device="cuda")
+        start = torch.empty(n, dtype=torch.float32, device="cuda")
+        ratio = torch.empty(n, dtype=torch.float32, device="cuda")
+        order = torch.empty(n, dtype=torch.int32, device="cuda")
+        hx_schedule_decode(self.h, calls.data_ptr(), None if lk is None else lk.data_ptr(),
+                           None if rd is None else rd.data_ptr(), n, inst.data_ptr(), start.data_ptr(),
+                           ratio.data_ptr(), order.data_ptr(), self._stream())
+        torch.cuda.current_stream().synchronize()      # lk / rd are temporaries of this call
+        return inst, start, ratio, order
 
     def schedule_batch_host(self, calls, out_assign=None, out_cost=None):
         return hx_schedule_batch_host(self.h, calls, out_assign, out_cost, self._stream())

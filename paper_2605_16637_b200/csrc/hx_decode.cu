@@ -1,0 +1,276 @@
+// Decode-stage scheduler (paper Section 5.4, "Decode scheduling with instance
+// locks", "Adaptive greedy decode assignment"; Section 6 names the state it
+// works on: decode token-capacity intervals).
+//
+// Calls whose KV cache has arrived wait for decode admission.  Until the queue
+// is empty: for every waiting call find, on each legal decode instance (its
+// lock if it has one, else every instance with m(c) <= Cap(d), Eq. 3-4), the
+// earliest start >= ready at which m(c) tokens are free for the whole decode;
+// its Delta_D is the earliest projected finish over those instances, its ratio
+// R = (elapsed + Delta_D) / H (Eq. 2); the call with the largest R (lower index
+// among equals) is assigned, its interval is added to the chosen instance.
+//
+// Tokens in use on an instance are a step function of time: breakpoints
+// t[0] = 0 < t[1] < ... and usage u[k] on [t[k], t[k+1]); the last segment runs
+// to infinity.  A search walks the segments from the one that holds the ready
+// time: a segment without room moves the candidate start to its end, and the
+// candidate is accepted once a segment ends at or after candidate + duration.
+// One persistent block; one warp projects one call with the lanes over the
+// instances; adding an interval only delays starts on that instance, so only
+// calls whose best instance it was are projected again.
+#include "hx_internal.h"
+
+namespace {
+
+constexpr int kThreads = 1024;
+constexpr int kWarps = kThreads / 32;
+#define HX_INF __int_as_float(0x7f800000)
+#define HX_NEG_INF __int_as_float(0xff800000)
+constexpr int kDead = -2, kNoInst = -1;
+
+struct DecodeParams {
+    HxTables t;
+    HxConstTables ct;
+    HxDagView dag;
+    HxStepFns base, work;      // usage step functions: snapshot and simulated state
+    const hx_call* calls;
+    const int32_t* lock;
+    const float* ready;
+    int n, flags, commit;
+    int32_t* out_inst;
+    float* out_start;
+    float* out_ratio;
+    int32_t* out_order;
+    int* status;
+};
+
+// Segment index holding x in t[0..K): the largest k with t[k] <= x.  Executed by one warp.
+__device__ __forceinline__ int warp_find_segment(const float* t, int K, float x, int lane) {
+    int cnt = 0;
+    for (int i0 = 0; i0 < K; i0 += 32) {
+        const int i = i0 + lane;
+        cnt += __popc(__ballot_sync(0xffffffffu, i < K && t[i] <= x));
+    }
+    return cnt - 1;                                     // t[0] = 0 <= x always
+}
+
+// Make x a breakpoint of instance arrays (t, u, K); returns its index.  One warp.
+__device__ int warp_cut(float* t, float* u, int& K, float x, int lane) {
+    const int k = warp_find_segment(t, K, x, lane);
+    if (t[k] == x) return k;
+    // shift (k, K) up by one, from the top, a warp-wide chunk at a time
+    for (int hi = K; hi > k + 1; hi -= 32) {
+        const int i = hi - 1 - lane;                    // hi-1, hi-2, ... > k
+        float tv = 0.f, uv = 0.f;
+        const bool mv = i > k;
+        if (mv) { tv = t[i]; uv = u[i]; }
+        __syncwarp();
+        if (mv) { t[i + 1] = tv; u[i + 1] = uv; }
+        __syncwarp();
+    }
+    if (lane == 0) { t[k + 1] = x; u[k + 1] = u[k]; }
+    __syncwarp();
+    ++K;
+    return k + 1;
+}
+
+__global__ void __launch_bounds__(kThreads, 1) hx_decode_kernel(const __grid_constant__ DecodeParams prm) {
+    extern __shared__ __align__(16) unsigned char smem[];
+    __shared__ float red_v[kWarps];
+    __shared__ int red_c[kWarps];
+    __shared__ int s_call, s_d, s_ndirty;
+    const HxTables& T = prm.t;
+    const int D = T.D, G = T.G, n = prm.n;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int cap = prm.work.cap;
+
+    float* capDs = reinterpret_cast<float*>(smem);              // [D]
+    int* typeDs = reinterpret_cast<int*>(capDs + D);            // [D]
+    int* Ks = typeDs + D;                                       // [D] breakpoints per instance
+    float* cn = reinterpret_cast<float*>(Ks + D);               // [n]
+    float* co = cn + n;
+    float* cel = co + n;
+    float* cH = cel + n;
+    float* cready = cH + n;
+    float* cR = cready + n;                                     // projected ratio, -inf if it cannot be taken
+    float* cstart = cR + n;
+    float* cfin = cstart + n;
+    int* cbest = reinterpret_cast<int*>(cfin + n);              // best instance, kNoInst, kDead
+    int* clock_ = cbest + n;                                    // lock (-1 = free)
+    int* cmodel = clock_ + n;
+    unsigned short* dirty = reinterpret_cast<unsigned short*>(cmodel + n);
+
+    for (int d = tid; d < D; d += kThreads) {
+        capDs[d] = T.capD[d]; typeDs[d] = T.typeD[d];
+        Ks[d] = prm.base.K[d];
+    }
+    __syncthreads();
+    for (int d = warp; d < D; d += kWarps)                      // simulated state starts as the snapshot
+        for (int i = lane; i < Ks[d]; i += 32) {
+            prm.work.t[(size_t)d * cap + i] = prm.base.t[(size_t)d * prm.base.cap + i];
+            prm.work.u[(size_t)d * cap + i] = prm.base.u[(size_t)d * prm.base.cap + i];
+        }
+    for (int c = tid; c < n; c += kThreads) {
+        const uint4 raw = __ldg(reinterpret_cast<const uint4*>(prm.calls) + c);
+        bool bad = raw.y >= (unsigned)T.M;
+        float el = 0.f, H = 1.f;
+        if (!(prm.flags & HX_FLAG_NO_DAG)) {
+            if (raw.x < prm.dag.n_nodes) { const uint32_t w = prm.dag.node_wf[raw.x]; el = prm.dag.elapsed[w]; H = prm.dag.H[w]; }
+            else bad = true;
+        }
+        const int lk = prm.lock ? prm.lock[c] : -1;
+        const float rd = prm.ready ? prm.ready[c] : 0.f;
+        if (lk >= D || !(rd >= 0.f) || rd == HX_INF) bad = true;
+        if (bad) atomicExch(prm.status, HX_ERR_INVALID_ARG);
+        cn[c] = __uint_as_float(raw.z); co[c] = __uint_as_float(raw.w);
+        cmodel[c] = bad ? 0 : (int)raw.y;
+        cel[c] = el; cH[c] = H; cready[c] = rd; clock_[c] = lk < 0 ? -1 : lk;
+        cR[c] = HX_NEG_INF; cstart[c] = HX_INF; cfin[c] = HX_INF;
+        cbest[c] = bad ? kDead : kNoInst;
+        dirty[c] = (unsigned short)c;
+        prm.out_inst[c] = -1; prm.out_start[c] = HX_INF; prm.out_ratio[c] = HX_INF; prm.out_order[c] = -1;
+    }
+    if (tid == 0) s_ndirty = n;
+    __syncthreads();
+
+    for (int it = 0; it < n; ++it) {
+        // (1) project the listed calls: one warp per call, lanes over the decode instances
+        const int nd = s_ndirty;
+        for (int i = warp; i < nd; i += kWarps) {
+            const int c = dirty[i];
+            if (cbest[c] == kDead) continue;
+            const float nt = cn[c], ot = co[c];
+            const int mdl = cmodel[c];
+            const float omega = prm.ct.omega[mdl], kappa = prm.ct.kappa[mdl];
+            const float ctx = __fmaf_rn(0.5f, __fsub_rn(ot, 1.0f), nt);
+            const float step = __fmaf_rn(kappa, ctx, omega);
+            const float m = __fadd_rn(nt, ot);
+            const float rd = cready[c];
+            const int lk = clock_[c];
+            float best = HX_INF, bs = 0.f; int bd = 0x7fffffff;
+            for (int d = lane; d < D; d += 32) {
+                if ((lk >= 0 && lk != d) || !(m <= capDs[d])) continue;
+                const float tau = __fmul_rn(__fmul_rn(ot, step), prm.ct.invB[typeDs[d]]);
+                const float* tt = prm.work.t + (size_t)d * cap;
+                const float* uu = prm.work.u + (size_t)d * cap;
+                const int K = Ks[d];
+                int k = 0;
+                while (k + 1 < K && tt[k + 1] <= rd) ++k;       // segment that holds the ready time
+                float cand = rd, fin;
+                for (;; ++k) {
+                    const float seg_end = (k + 1 < K) ? tt[k + 1] : HX_INF;
+                    if (__fadd_rn(uu[k], m) > capDs[d]) {
+                        if (k + 1 >= K) { fin = HX_INF; break; }   // last segment is empty on a valid state: not reached
+                        cand = seg_end; continue;
+                    }
+                    fin = __fadd_rn(cand, tau);
+                    if (seg_end >= fin) break;
+                }
+                if (fin < best) { best = fin; bs = cand; bd = d; }   // ascending d per lane: lowest d kept
+            }
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) {
+                const float ov = __shfl_xor_sync(0xffffffffu, best, off);
+                const float os = __shfl_xor_sync(0xffffffffu, bs, off);
+                const int od = __shfl_xor_sync(0xffffffffu, bd, off);
+                if (ov < best || (ov == best && od < bd)) { best = ov; bs = os; bd = od; }
+            }
+            if (lane == 0) {
+                if (bd != 0x7fffffff) {
+                    cbest[c] = bd; cstart[c] = bs; cfin[c] = best;
+                    cR[c] = __fdiv_rn(__fadd_rn(cel[c], best), cH[c]);
+                } else { cbest[c] = kNoInst; cR[c] = HX_NEG_INF; }
+            }
+        }
+        __syncthreads();
+        // (2) most urgent waiting call
+        float rv = HX_NEG_INF; int rc = 0x7fffffff;
+        for (int c = tid; c < n; c += kThreads) {
+            const float r = cR[c];
+            if (r > rv) { rv = r; rc = c; }
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, rv, off);
+            const int oc = __shfl_xor_sync(0xffffffffu, rc, off);
+            if (ov > rv || (ov == rv && oc < rc)) { rv = ov; rc = oc; }
+        }
+        if (lane == 0) { red_v[warp] = rv; red_c[warp] = rc; }
+        __syncthreads();
+        if (warp == 0) {
+            rv = red_v[lane]; rc = red_c[lane];
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) {
+                const float ov = __shfl_xor_sync(0xffffffffu, rv, off);
+                const int oc = __shfl_xor_sync(0xffffffffu, rc, off);
+                if (ov > rv || (ov == rv && oc < rc)) { rv = ov; rc = oc; }
+            }
+            // (3) commit (warp 0): add the interval [start, finish) with m tokens to the step function
+            if (rc == 0x7fffffff) {
+                if (lane == 0) { s_call = -1; s_ndirty = 0; }
+            } else {
+                const int d = cbest[rc];
+                const float s = cstart[rc], e = cfin[rc], m = __fadd_rn(cn[rc], co[rc]);
+                float* tt = prm.work.t + (size_t)d * cap;
+                float* uu = prm.work.u + (size_t)d * cap;
+                int K = Ks[d];
+                if (K + 2 > cap) {                              // cannot happen with the capacity the host sizes
+                    if (lane == 0) { atomicExch(prm.status, HX_ERR_INVALID_ARG); s_call = -1; s_ndirty = 0; }
+                } else {
+                    const int a = warp_cut(tt, uu, K, s, lane);
+                    const int b = warp_cut(tt, uu, K, e, lane);
+                    for (int k = a + lane; k < b; k += 32) uu[k] = __fadd_rn(uu[k], m);
+                    if (lane == 0) {
+                        Ks[d] = K;
+                        prm.out_inst[rc] = d; prm.out_start[rc] = s; prm.out_ratio[rc] = rv; prm.out_order[it] = rc;
+                        cbest[rc] = kDead; cR[rc] = HX_NEG_INF;
+                        s_call = rc; s_d = d; s_ndirty = 0;
+                    }
+                }
+            }
+        }
+        __syncthreads();
+        if (s_call < 0) break;
+        const int ds = s_d;
+        for (int c = tid; c < n; c += kThreads)
+            if (cbest[c] == ds) dirty[atomicAdd(&s_ndirty, 1)] = (unsigned short)c;
+        __syncthreads();
+    }
+    if (prm.commit) {                                           // the simulated state becomes the snapshot
+        __syncthreads();
+        for (int d = warp; d < D; d += kWarps) {
+            const int K = min(Ks[d], prm.base.cap);
+            for (int i = lane; i < K; i += 32) {
+                prm.base.t[(size_t)d * prm.base.cap + i] = prm.work.t[(size_t)d * cap + i];
+                prm.base.u[(size_t)d * prm.base.cap + i] = prm.work.u[(size_t)d * cap + i];
+            }
+            if (lane == 0) prm.base.K[d] = K;
+        }
+    }
+}
+
+}  // namespace
+
+size_t hx_decode_smem_bytes(const HxTables& t, int n_calls) {
+    return (3 * (size_t)t.D + 11 * (size_t)n_calls) * 4 + (size_t)n_calls * 2 + 16;
+}
+
+cudaError_t hx_launch_decode(const HxTables& t, const HxConstTables& ct, const HxDagView& dag,
+                             const HxStepFns& base, const HxStepFns& work,
+                             const hx_call* calls, const int32_t* lock, const float* ready, int n_calls,
+                             int flags, int commit, int32_t* out_inst, float* out_start, float* out_ratio,
+                             int32_t* out_order, int* status, cudaStream_t stream, long long* launches) {
+    DecodeParams prm;
+    prm.t = t; prm.ct = ct; prm.dag = dag; prm.base = base; prm.work = work;
+    prm.calls = calls; prm.lock = lock; prm.ready = ready; prm.n = n_calls; prm.flags = flags; prm.commit = commit;
+    prm.out_inst = out_inst; prm.out_start = out_start; prm.out_ratio = out_ratio; prm.out_order = out_order;
+    prm.status = status;
+    const size_t smem = hx_decode_smem_bytes(t, n_calls);
+    static size_t allowed[64];
+    cudaError_t e = hx_opt_in_smem(hx_decode_kernel, smem, allowed, 40 * 1024);
+    if (e != cudaSuccess) return e;
+    hx_decode_kernel<<<1, kThreads, smem, stream>>>(prm);
+    e = cudaGetLastError();
+    if (e == cudaSuccess) ++*launches;
+    return e;
+}

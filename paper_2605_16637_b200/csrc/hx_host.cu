@@ -32,6 +32,11 @@ struct hx_cluster {
     std::vector<void*> upd_allocs;      // scratch of hx_dag_update_costs, grown on demand
     uint32_t* d_upd_idx = nullptr; float* d_upd_cost = nullptr; uint32_t* d_upd_wf = nullptr;
     size_t upd_cap = 0, upd_wf_cap = 0;
+    // decode-stage scheduler: usage step functions (snapshot and simulated state)
+    std::vector<void*> dec_allocs;
+    HxStepFns dec_base{}, dec_work{};
+    int dec_k_bound = 0;                // upper bound on the breakpoints of any instance in the snapshot
+    bool dec_ready = false;
     // top-K
     HxTopkBufs tk{};
     // staging for the host-buffer entry point
@@ -274,7 +279,7 @@ int hx_cluster_destroy(hx_cluster* h) {
     if (!h) return HX_OK;
     DeviceGuard guard(h->device);
     cudaDeviceSynchronize();
-    free_pool(h->allocs); free_pool(h->dag_allocs); free_pool(h->tk_allocs); free_pool(h->upd_allocs);
+    free_pool(h->allocs); free_pool(h->dag_allocs); free_pool(h->tk_allocs); free_pool(h->upd_allocs); free_pool(h->dec_allocs);
     if (h->st_calls) cudaFree(h->st_calls);
     if (h->st_assign) cudaFree(h->st_assign);
     if (h->st_cost) cudaFree(h->st_cost);
@@ -712,6 +717,120 @@ int hx_schedule_greedy(hx_cluster* h, const hx_call* calls, int n_calls, int32_t
         HX_TRY(hx_launch_greedy(h->tab, h->ctab, dag, calls, n_calls, o.flags, o.commit, out_assign, out_ratio,
                                 out_order, h->status, s, &h->launches), "greedy planner kernel");
     }
+    return HX_OK;
+}
+
+namespace {
+
+// (Re)allocates the step-function arrays with room for `cap` breakpoints per instance; the
+// snapshot is carried over when keep is set.
+int decode_reserve(hx_cluster* h, int cap, bool keep) {
+    if (h->dec_base.cap >= cap) return HX_OK;
+    const int D = h->D;
+    cudaDeviceSynchronize();
+    std::vector<void*> fresh;
+    HxStepFns b{}, w{};
+    b.cap = w.cap = cap;
+    HX_TRY(dev_alloc(fresh, &b.t, (size_t)D * cap), "alloc decode intervals");
+    HX_TRY(dev_alloc(fresh, &b.u, (size_t)D * cap), "alloc decode intervals");
+    HX_TRY(dev_alloc(fresh, &b.K, (size_t)D), "alloc decode intervals");
+    HX_TRY(dev_alloc(fresh, &w.t, (size_t)D * cap), "alloc decode intervals");
+    HX_TRY(dev_alloc(fresh, &w.u, (size_t)D * cap), "alloc decode intervals");
+    w.K = b.K;
+    if (keep && h->dec_base.cap > 0) {
+        const size_t ow = (size_t)h->dec_base.cap * sizeof(float);
+        HX_TRY(cudaMemcpy2D(b.t, (size_t)cap * sizeof(float), h->dec_base.t, ow, ow, D, cudaMemcpyDeviceToDevice), "copy decode intervals");
+        HX_TRY(cudaMemcpy2D(b.u, (size_t)cap * sizeof(float), h->dec_base.u, ow, ow, D, cudaMemcpyDeviceToDevice), "copy decode intervals");
+        HX_TRY(cudaMemcpy(b.K, h->dec_base.K, (size_t)D * sizeof(int), cudaMemcpyDeviceToDevice), "copy decode intervals");
+    }
+    free_pool(h->dec_allocs);
+    h->dec_allocs = fresh;
+    h->dec_base = b; h->dec_work = w;
+    return HX_OK;
+}
+
+}  // namespace
+
+int hx_decode_set_running(hx_cluster* h, const uint32_t* inst_ptr, const hx_kv_interval* running, void* stream) {
+    if (!h) return HX_ERR_INVALID_ARG;
+    if (!inst_ptr) return fail(h, HX_ERR_INVALID_ARG, "NULL array");
+    const int D = h->D;
+    if (inst_ptr[0] != 0) return fail(h, HX_ERR_INVALID_ARG, "inst_ptr must start at 0");
+    for (int d = 0; d < D; ++d)
+        if (inst_ptr[d + 1] < inst_ptr[d]) return fail(h, HX_ERR_INVALID_ARG, "inst_ptr is not monotone");
+    const uint32_t total = inst_ptr[D];
+    if (total && !running) return fail(h, HX_ERR_INVALID_ARG, "NULL array");
+    int maxK = 1;
+    for (uint32_t i = 0; i < total; ++i) {
+        if (!(std::isfinite(running[i].end_s) && running[i].end_s > 0.0f))
+            return fail(h, HX_ERR_INVALID_ARG, "a running call must end at a finite time > 0");
+        if (!good_load(running[i].tokens) || running[i].tokens >= 16777216.0f || running[i].tokens != std::floor(running[i].tokens))
+            return fail(h, HX_ERR_INVALID_ARG, "tokens of a running call must be a whole number below 2^24");
+    }
+    for (int d = 0; d < D; ++d) maxK = std::max<int>(maxK, (int)(inst_ptr[d + 1] - inst_ptr[d]) + 1);
+    DeviceGuard guard(h->device);
+    int rc = decode_reserve(h, std::max(maxK + 2, 64), false);
+    if (rc != HX_OK) return rc;
+    // step function of every instance: usage until the next call ends (token counts are whole
+    // numbers, so the sums are exact in any order)
+    const int cap = h->dec_base.cap;
+    std::vector<float> t((size_t)D * cap, 0.f), u((size_t)D * cap, 0.f);
+    std::vector<int> K(D, 1);
+    for (int d = 0; d < D; ++d) {
+        std::vector<std::pair<float, float>> ev;
+        for (uint32_t i = inst_ptr[d]; i < inst_ptr[d + 1]; ++i) ev.emplace_back(running[i].end_s, running[i].tokens);
+        std::sort(ev.begin(), ev.end());
+        float held = 0.f;
+        for (auto& e : ev) held += e.second;
+        if (held >= 16777216.0f) return fail(h, HX_ERR_INVALID_ARG, "tokens in use on an instance must stay below 2^24");
+        float* td = &t[(size_t)d * cap]; float* ud = &u[(size_t)d * cap];
+        int k = 0;
+        td[0] = 0.f; ud[0] = held;
+        for (size_t i = 0; i < ev.size(); ++i) {
+            held -= ev[i].second;
+            if (i + 1 < ev.size() && ev[i + 1].first == ev[i].first) continue;     // calls ending together
+            ++k; td[k] = ev[i].first; ud[k] = held;
+        }
+        K[d] = k + 1;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    HX_TRY(cudaMemcpyAsync(h->dec_base.t, t.data(), t.size() * sizeof(float), cudaMemcpyHostToDevice, s), "copy decode intervals");
+    HX_TRY(cudaMemcpyAsync(h->dec_base.u, u.data(), u.size() * sizeof(float), cudaMemcpyHostToDevice, s), "copy decode intervals");
+    HX_TRY(cudaMemcpyAsync(h->dec_base.K, K.data(), K.size() * sizeof(int), cudaMemcpyHostToDevice, s), "copy decode intervals");
+    h->dec_k_bound = maxK;
+    h->dec_ready = true;
+    return HX_OK;
+}
+
+int hx_schedule_decode(hx_cluster* h, const hx_call* calls, const int32_t* lock, const float* ready_s, int n_calls,
+                       int32_t* out_inst, float* out_start, float* out_ratio, int32_t* out_order, void* stream) {
+    if (!h) return HX_ERR_INVALID_ARG;
+    if (n_calls < 0) return fail(h, HX_ERR_INVALID_ARG, "negative n_calls");
+    if (n_calls == 0) return HX_OK;
+    if (!calls || !out_inst || !out_start || !out_ratio || !out_order) return fail(h, HX_ERR_INVALID_ARG, "NULL buffer");
+    if (reinterpret_cast<uintptr_t>(calls) % 16) return fail(h, HX_ERR_INVALID_ARG, "calls must be 16-byte aligned");
+    if (!h->dec_ready) return fail(h, HX_ERR_NOT_READY, "no decode intervals: call hx_decode_set_running first (it may list no running call)");
+    const hx_options& o = h->opts;
+    if (!(o.flags & HX_FLAG_NO_DAG) && !(h->dag_uploaded && h->cp_ready))
+        return fail(h, HX_ERR_NOT_READY, "horizons not computed: call hx_dag_upload and hx_critical_path, or set HX_FLAG_NO_DAG");
+    if (n_calls > HX_DECODE_MAX_CALLS)
+        return fail(h, HX_ERR_INVALID_ARG, "hx_schedule_decode: more than HX_DECODE_MAX_CALLS (2048) calls in the decode queue");
+    if (hx_decode_smem_bytes(h->tab, n_calls) > h->max_smem)
+        return fail(h, HX_ERR_INVALID_ARG, "hx_schedule_decode: queue does not fit the shared memory of one SM");
+    DeviceGuard guard(h->device);
+    int rc = decode_reserve(h, h->dec_k_bound + 2 * n_calls + 2, true);
+    if (rc != HX_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    HxDagView dag{};
+    if (!(o.flags & HX_FLAG_NO_DAG))
+        dag = HxDagView{h->d_node_wf, h->forest.tail, h->forest.H, h->d_elapsed, h->forest.n_nodes, h->forest.n_workflows};
+    {
+        SpanGuard span(h, 0, s);
+        HX_TRY(hx_launch_decode(h->tab, h->ctab, dag, h->dec_base, h->dec_work, calls, lock, ready_s, n_calls, o.flags,
+                                o.commit, out_inst, out_start, out_ratio, out_order, h->status, s, &h->launches),
+               "decode scheduler kernel");
+    }
+    if (o.commit) h->dec_k_bound += 2 * n_calls;
     return HX_OK;
 }
 

@@ -124,6 +124,23 @@ cudaError_t hx_launch_greedy(const HxTables& t, const HxConstTables& ct, const H
                              int32_t* out_assign, float* out_ratio, int32_t* out_order, int* status,
                              cudaStream_t stream, long long* launches);
 
+// Tokens in use on every decode instance as step functions of time (decode token-capacity
+// intervals): instance d has K[d] breakpoints t[d * cap + k] (t = 0 first, ascending) and usage
+// u[d * cap + k] on [t[k], t[k + 1]); the last segment runs to infinity.
+struct HxStepFns {
+    float* t;
+    float* u;
+    int* K;
+    int cap;
+};
+
+size_t hx_decode_smem_bytes(const HxTables& t, int n_calls);
+cudaError_t hx_launch_decode(const HxTables& t, const HxConstTables& ct, const HxDagView& dag,
+                             const HxStepFns& base, const HxStepFns& work,
+                             const hx_call* calls, const int32_t* lock, const float* ready, int n_calls,
+                             int flags, int commit, int32_t* out_inst, float* out_start, float* out_ratio,
+                             int32_t* out_order, int* status, cudaStream_t stream, long long* launches);
+
 // Workflow classes of the horizon pass: lists of workflow ids handled by one launch each.
 struct HxCpClass {
     const uint32_t* wf_ids;    // device
