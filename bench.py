@@ -343,6 +343,7 @@ def run_cuda(args):
         "gpu_launches": int(launches), "kernel_ms_per_step": {k: v[0] / args.steps for k, v in kt.items()},
         "device_status": status, "roofline": roofline, "cpu_baseline": cpu, "clocks": clocks,
         "greedy_planner": greedy,
+        "decode_scheduler": decode_leg() if world == 1 and not args.no_cpu_baseline else None,
     }
     print(json.dumps(out))
     if dist is not None:
@@ -384,6 +385,32 @@ def greedy_leg(with_cpu):
             out[label]["oracle_ms_1_core"] = 1e3 * (time.perf_counter() - t0)
         gc.close()
     return out
+
+
+def decode_leg():
+    """Side measurement, outside the timed region: the decode-stage scheduler (Section 5.4) on the decode
+    pool of the medium configuration (16 instances), queue of 1,024 calls, four running calls per instance."""
+    import paper_2605_16637_b200 as hx
+    from hx_synth import make_decode_queue, make_workload
+    from oracle import hx_oracle as ho
+    wl = make_workload("medium")
+    calls, lock, ready, ptr, end, tok = make_decode_queue(wl, 1024)
+    gc = hx.Cluster.from_workload(wl)
+    gc.set_options(score_mode=hx.HX_MODE_RATIO, flags=hx.HX_FLAG_NO_DAG, commit=0)
+    gc.decode_set_running(ptr, end, tok)
+    times = []
+    for i in range(6):
+        t0 = time.perf_counter()
+        res = gc.schedule_decode(calls, lock, ready)         # synchronises
+        times.append(time.perf_counter() - t0)
+    orc, oc = ho.Oracle(), ho.Cluster.from_workload(wl)
+    t0 = time.perf_counter()
+    want = orc.decode_greedy(oc, calls, ptr, end, tok, lock, ready)
+    cpu_ms = 1e3 * (time.perf_counter() - t0)
+    same = bool(np.array_equal(res[0].cpu().numpy(), want[0]) and np.array_equal(res[3].cpu().numpy(), want[3]))
+    gc.close()
+    return {"calls": 1024, "decode_instances": wl.D, "ms_wall_incl_copies": 1e3 * float(np.median(times[1:])),
+            "oracle_ms_1_core": cpu_ms, "identical_to_oracle": same}
 
 
 def main():

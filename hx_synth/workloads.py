@@ -341,3 +341,25 @@ def sub_forest(wl: Workload, workflows: np.ndarray):
     assert np.all(col >= 0)
     local_wf = np.repeat(np.arange(workflows.shape[0]), ends - starts)
     return (row_ptr.astype(np.uint32), col.astype(np.uint32), local_wf.astype(np.uint32), node_ids)
+
+
+def make_decode_queue(wl: Workload, n_calls: int, seed: int = 0, running_per_instance: int = 4,
+                      load: float = 0.6, locked: float = 0.3):
+    """Seeded decode-side snapshot for the decode-stage scheduler (Section 5.4), drawn for the decode
+    pool of `wl`: the first n_calls ready calls as the decode queue, a lock for a share of them, the time
+    their KV cache is on the decode side, and per decode instance a few calls decoding now that together
+    hold about `load` of the instance's KV capacity until some time within the next two seconds.
+    Returns (calls, lock i32, ready_s f32, run_ptr u32[D+1], run_end f32, run_tok f32)."""
+    rng = np.random.default_rng([seed, 17, n_calls])
+    D = wl.D
+    calls = wl.calls[:n_calls].copy()
+    lock = np.where(rng.random(n_calls) < locked, rng.integers(0, D, n_calls), -1).astype(np.int32)
+    ready = np.where(rng.random(n_calls) < 0.5, 0.0, rng.uniform(0.0, 0.5, n_calls)).astype(np.float32)
+    cap = wl.kv_cap[wl.P:]
+    ptr, end, tok = [0], [], []
+    for d in range(D):
+        share = rng.dirichlet(np.ones(running_per_instance)) * load * cap[d]
+        for s in share:
+            end.append(rng.uniform(0.05, 2.0)); tok.append(np.floor(s))
+        ptr.append(len(end))
+    return (calls, lock, ready, np.array(ptr, np.uint32), np.array(end, np.float32), np.array(tok, np.float32))
