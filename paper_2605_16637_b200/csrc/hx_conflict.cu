@@ -38,6 +38,8 @@ constexpr int kBins = 2048;
 constexpr int kWin = 256;          // calls per optimistic window (= block size of the pass)
 constexpr int kCache = 4096;       // calls staged in shared memory ahead of the window
 constexpr unsigned kNone = 0xFFu;  // no candidate taken
+constexpr int kTailLen = 8192;     // obtained pairs handled per round of the fused tail
+constexpr int kTailMaxP = 512;     // largest prefill pool the fused tail handles
 
 // Exclusive prefix sum of n counters into shared memory, by the whole block
 // (blockDim a multiple of 32).  base gets n + 1 entries, tmp needs 33.
@@ -149,7 +151,8 @@ __global__ void hx_order_rank_kernel(HxTopkBufs tk, int n) {
 // are dropped, in parallel, while the next stretch of the visiting order is staged, so the
 // windows only hold calls that may still be placed.
 template <int KT>   // candidate slots examined per call: K rounded up to 1, 2, 4 or 8
-__global__ void __launch_bounds__(kWin) hx_conflict_kernel(HxTopkBufs tk, HxTables t, int n, int commit) {
+__global__ void __launch_bounds__(kWin) hx_conflict_kernel(HxTopkBufs tk, HxTables t, int n, int commit,
+                                                           int fused_tail, int32_t* out_assign) {
     extern __shared__ __align__(16) unsigned sm[];
     constexpr int NW = kWin / 32;
     constexpr int kScan = 4 * kWin;                             // ranks examined per staging step
@@ -278,6 +281,103 @@ __global__ void __launch_bounds__(kWin) hx_conflict_kernel(HxTopkBufs tk, HxTabl
     }
     if (tid == 0) *tk.n_acc = n_acc;
     if (commit) for (int d = tid; d < D; d += kWin) t.freeD[d] = __int2float_rn(free_s[d]);
+    if (!fused_tail) return;
+
+    // ---- tail (prefill pools of up to kTailMaxP instances): publish the obtained pairs and add the
+    // prefill times to the prefill queues in visiting order, without leaving the block.  The list of
+    // obtained pairs is taken in rounds of kTailLen entries; a round is split by prefill instance with
+    // a stable counting sort (per-warp groups by match, per-warp counts, offsets), then one thread per
+    // instance adds its run one after the other (binary32 addition is not associative: the order is
+    // part of the definition).
+    const int P = t.P;
+    __syncthreads();                                            // the ring is free, acc_rk is visible
+    unsigned short* pbuf = reinterpret_cast<unsigned short*>(sm);           // [kTailLen]
+    float* tbuf = reinterpret_cast<float*>(pbuf + kTailLen);                // [kTailLen]
+    float* sorted = tbuf + kTailLen;                                        // [kTailLen]
+    int* tail_i = wtot + NW * D;                                            // behind the pass's own arrays
+    float* qsum = reinterpret_cast<float*>(tail_i);                         // [P]
+    int* hist = tail_i + P;                                                 // [P]
+    int* off0 = hist + P;                                                   // [P] start of the run of p in `sorted`
+    int* off = off0 + P;                                                    // [P] next free slot of the run
+    int* wcnt = off + P;                                                    // [NW][P], zero between uses
+    for (int p = tid; p < P; p += kWin) qsum[p] = t.qP[p];
+    for (int i = tid; i < NW * P; i += kWin) wcnt[i] = 0;
+    for (unsigned r0 = 0; r0 < n_acc; r0 += kTailLen) {
+        const int len = (int)min((unsigned)kTailLen, n_acc - r0);
+        for (int p = tid; p < P; p += kWin) hist[p] = 0;
+        __syncthreads();
+        // three dependent gathers per entry (list -> call -> pair, prefill time): eight entries in flight per thread
+        for (int i0 = tid; i0 < len; i0 += 8 * kWin) {
+            unsigned rk[8], c[8]; int pr[8]; float tp[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) rk[u] = i0 + u * kWin < len ? __ldcg(tk.acc_rk + r0 + i0 + u * kWin) : 0u;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) c[u] = i0 + u * kWin < len ? __ldcg(tk.ocall + (rk[u] & 0xFFFFFFu)) : 0u;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const size_t o = (size_t)c[u] * tk.K + (rk[u] >> 24);
+                const bool ok = i0 + u * kWin < len;
+                pr[u] = ok ? __ldcg(tk.pair + o) : 0;
+                tp[u] = ok ? __ldcg(tk.tpre + o) : 0.f;
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int i = i0 + u * kWin;
+                if (i < len) {
+                    out_assign[c[u]] = pr[u];
+                    const int p = pr[u] / D;
+                    pbuf[i] = (unsigned short)p;
+                    tbuf[i] = tp[u];
+                    atomicAdd(&hist[p], 1);
+                }
+            }
+        }
+        __syncthreads();
+        if (warp == 0) {                                        // exclusive prefix of the histogram
+            int run = 0;
+            for (int p0 = 0; p0 < P; p0 += 32) {
+                const int p = p0 + lane;
+                const int h = p < P ? hist[p] : 0;
+                int x = h;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, x, o); if (lane >= o) x += y; }
+                if (p < P) { off0[p] = run + x - h; off[p] = run + x - h; }
+                run += __shfl_sync(0xffffffffu, x, 31);
+            }
+        }
+        __syncthreads();
+        for (int ch = 0; ch < len; ch += kWin) {
+            const int i = ch + tid;
+            const bool valid = i < len;
+            const int p = valid ? (int)pbuf[i] : -1 - lane;
+            const unsigned peers = __match_any_sync(0xffffffffu, p);
+            const int rank = __popc(peers & ((1u << lane) - 1u));
+            const bool leader = valid && rank == 0;
+            if (leader) wcnt[warp * P + p] = __popc(peers);
+            __syncthreads();
+            int before = 0, total = 0;
+            if (valid) {
+#pragma unroll
+                for (int w = 0; w < NW; ++w) { const int cw = wcnt[w * P + p]; total += cw; before += w < warp ? cw : 0; }
+                sorted[off[p] + before + rank] = tbuf[i];
+            }
+            __syncthreads();
+            if (leader) {
+                if (before == 0) off[p] += total;               // first warp of this chunk that holds p
+                wcnt[warp * P + p] = 0;
+            }
+            __syncthreads();
+        }
+        for (int p = tid; p < P; p += kWin) {
+            const int a = off0[p], b = a + hist[p];
+            float q = qsum[p];
+#pragma unroll 8
+            for (int j = a; j < b; ++j) q = __fadd_rn(q, sorted[j]);
+            qsum[p] = q;
+        }
+        __syncthreads();
+    }
+    if (commit) for (int p = tid; p < P; p += kWin) t.qP[p] = qsum[p];
 }
 
 // 3. Publish the obtained pairs; gather prefill instance and prefill time in visiting order.
@@ -341,18 +441,23 @@ cudaError_t hx_launch_conflict(const HxTables& t, const HxTopkBufs& tk, int n_ca
     if (e != cudaSuccess) return e;
     hx_order_bins_kernel<<<1, 1024, smB, stream>>>(tk, n_calls, staged);
     hx_order_rank_kernel<<<(n_calls + 127) / 128, 128, 0, stream>>>(tk, n_calls);
-    const size_t smC = (size_t)kCache * 24 + (size_t)(2 * D + (kWin / 32) * D) * 4;
+    const int fused = P <= kTailMaxP;                               // pairs published and queues summed inside the pass
+    const size_t smC = (size_t)kCache * 24 + (size_t)(2 * D + (kWin / 32) * D) * 4 +
+                       (fused ? (size_t)(4 * P + (kWin / 32) * P) * 4 : 0);
     auto pass = tk.K <= 1 ? hx_conflict_kernel<1> : tk.K <= 2 ? hx_conflict_kernel<2>
               : tk.K <= 4 ? hx_conflict_kernel<4> : hx_conflict_kernel<8>;
     static size_t allowed_pass[4][64];
     e = hx_opt_in_smem(pass, smC, allowed_pass[tk.K <= 1 ? 0 : tk.K <= 2 ? 1 : tk.K <= 4 ? 2 : 3], 40 * 1024);
     if (e != cudaSuccess) return e;
-    pass<<<1, kWin, smC, stream>>>(tk, t, n_calls, commit);
-    hx_finish_kernel<<<(n_calls + 255) / 256, 256, 0, stream>>>(tk, D, out_assign);
-    *launches += 4;
-    if (commit) {
-        hx_qsum_kernel<<<(P + kQWarps - 1) / kQWarps, 32 * kQWarps, 0, stream>>>(tk, t);
+    pass<<<1, kWin, smC, stream>>>(tk, t, n_calls, commit, fused, out_assign);
+    *launches += 3;
+    if (!fused) {
+        hx_finish_kernel<<<(n_calls + 255) / 256, 256, 0, stream>>>(tk, D, out_assign);
         *launches += 1;
+        if (commit) {
+            hx_qsum_kernel<<<(P + kQWarps - 1) / kQWarps, 32 * kQWarps, 0, stream>>>(tk, t);
+            *launches += 1;
+        }
     }
     return cudaGetLastError();
 }
