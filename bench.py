@@ -413,6 +413,67 @@ def decode_leg():
             "oracle_ms_1_core": cpu_ms, "identical_to_oracle": same}
 
 
+def run_configs(args):
+    """`--configs`: ready-batch schedule latency and horizon time on the four smaller configurations
+    (the default run times the sweep).  Prints one JSON object; plain argmin, slack score, whole batch in
+    one hx_schedule_batch call; CUDA events per call plus host wall clock enqueue -> synchronise."""
+    import torch
+    import paper_2605_16637_b200 as hx
+    from hx_synth import make_workload
+    from oracle import hx_oracle as ho
+    torch.cuda.set_device(0)
+    out = {}
+    reps, warm = 200, 20
+    for name in ("tiny", "medium", "large", "cp_stress"):
+        wl = make_workload(name)
+        gc = hx.Cluster.from_workload(wl)
+        if wl.node_cost is not None:
+            cost = np.asarray(wl.node_cost, np.float32)
+        else:
+            gc.set_options(score_mode=hx.HX_MODE_COMPLETION, flags=hx.HX_FLAG_UNLOADED | hx.HX_FLAG_NO_DAG)
+            cost = gc.schedule_batch(wl.node_calls)[1].cpu().numpy()
+        gc.dag_upload(wl.row_ptr, wl.col, cost, wl.node_wf, wl.elapsed)
+        gc.critical_path()
+        gc.set_options(score_mode=hx.HX_MODE_SLACK, alpha=wl.alpha)
+        calls = torch.from_numpy(wl.calls.view(np.uint8).reshape(-1, 16).copy()).cuda()
+        n = len(wl.calls)
+        a = torch.empty(n, dtype=torch.int32, device="cuda"); c = torch.empty(n, dtype=torch.float32, device="cuda")
+        stream = torch.cuda.current_stream(); sp = stream.cuda_stream
+        def timed(fn):
+            for _ in range(warm):
+                fn()
+            torch.cuda.synchronize()
+            ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+            wall = []
+            for e0, e1 in ev:
+                t0 = time.perf_counter()
+                e0.record(stream); fn(); e1.record(stream)
+                stream.synchronize()
+                wall.append(1e6 * (time.perf_counter() - t0))
+            us = np.array([1e3 * e0.elapsed_time(e1) for e0, e1 in ev])
+            return {"p50_us": float(np.percentile(us, 50)), "p95_us": float(np.percentile(us, 95)),
+                    "wall_p50_us": float(np.percentile(wall, 50))}
+        sched = timed(lambda: hx.hx_schedule_batch(gc.h, calls.data_ptr(), n, a.data_ptr(), c.data_ptr(), sp))
+        cpath = timed(lambda: hx.hx_critical_path(gc.h, sp))
+        cand = n * wl.P * wl.D
+        m = min(n, 4096)                                   # bounded oracle sample
+        orc, oc = ho.Oracle(), ho.Cluster.from_workload(wl)
+        t0 = time.perf_counter()
+        dag = orc.longest_path(wl.row_ptr, wl.col, cost, wl.node_wf, wl.n_workflows)
+        t_dag = time.perf_counter() - t0
+        t0 = time.perf_counter()
+        orc.schedule(oc, wl.calls[:m], mode=ho.MODE_SLACK, alpha=wl.alpha, dag=dag, node_wf=wl.node_wf, elapsed=wl.elapsed)
+        t_or = time.perf_counter() - t0
+        out[name] = {"instances": "%dx%d" % (wl.P, wl.D), "calls": n, "candidates": cand, "nodes": int(wl.n_nodes),
+                     "workflows": int(wl.n_workflows), "schedule_batch": sched,
+                     "candidates_per_s": cand / (sched["p50_us"] * 1e-6), "critical_path": cpath,
+                     "nodes_per_s": wl.n_nodes / (cpath["p50_us"] * 1e-6),
+                     "oracle": {"schedule_candidates_per_s_1_core": m * wl.P * wl.D / t_or, "sample_calls": m,
+                                "longest_path_ms_1_core": 1e3 * t_dag}}
+        gc.close()
+    print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -421,8 +482,12 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true",
                     help="skip the side legs outside the timed region (oracle sample, greedy planner)")
+    ap.add_argument("--configs", action="store_true",
+                    help="time the four smaller configurations instead (one JSON object)")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.configs:
+        run_configs(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_cuda(args)

@@ -592,21 +592,25 @@ cudaError_t hx_launch_score(const HxTables& t, const HxConstTables& ct, const Hx
     const int LC = 32 / LD, WD = TD * LD;
     prm.WDn = Dpad / WD;
     prm.Dpad = Dpad;
-    // warps along calls: fewer when the batch is too small to fill the SMs
-    const int min_tc = LD == 8 ? 4 : 8;
     int WCn = prm.WDn >= max_warps ? 1 : max_warps / prm.WDn;
-    while (WCn > 1 && (C + WCn * min_tc * LC - 1) / (WCn * min_tc * LC) < n_sm) WCn >>= 1;
-    prm.WCn = WCn;
-    // thread tile height: spread the calls evenly over the SMs (a fixed height would leave SMs
-    // idle whenever the batch is not a multiple of n_sm * rows * height calls)
     int TC = 8;
     if (LD == 8) {
+        // warps along calls: fewer when the batch is too small to fill the SMs
+        while (WCn > 1 && (C + WCn * 4 * LC - 1) / (WCn * 4 * LC) < n_sm) WCn >>= 1;
+        // thread tile height: spread the calls evenly over the SMs (a fixed height would leave SMs
+        // idle whenever the batch is not a multiple of n_sm * rows * height calls)
         const int per_sm = (C + n_sm - 1) / n_sm;
         const int rows = WCn * LC;
         const int tiles_per_sm = (per_sm + 8 * rows - 1) / (8 * rows);
         TC = (per_sm + tiles_per_sm * rows - 1) / (tiles_per_sm * rows);
         TC = TC < 4 ? 4 : (TC > 8 ? 8 : TC);
+    } else {
+        // narrow decode pools: the candidate loop is short, latency decides.  Keep all warps of the
+        // block (they hide the latency of the prologue and of the selection) and shrink the thread
+        // tile instead, until the batch gives every SM a block or the tile is one call high.
+        while (TC > 1 && (C + WCn * TC * LC - 1) / (WCn * TC * LC) < n_sm) TC >>= 1;
     }
+    prm.WCn = WCn;
     prm.TCB = WCn * TC * LC;
     prm.nTiles = (C + prm.TCB - 1) / prm.TCB;
     prm.FS = prm.Dpad + 8;     // rows 8 banks apart: the clamp phase stores four rows x eight columns per warp
@@ -647,7 +651,8 @@ cudaError_t hx_launch_score(const HxTables& t, const HxConstTables& ct, const Hx
     cudaError_t e;
 #define HX_CASE(tc, td, ld) if (TC == tc && TD == td && LD == ld) e = launch_one<tc, td, ld>(prm, grid, threads, smem, stream); else
     HX_CASE(8, 4, 8) HX_CASE(7, 4, 8) HX_CASE(6, 4, 8) HX_CASE(5, 4, 8) HX_CASE(4, 4, 8)
-    HX_CASE(8, 8, 4) HX_CASE(8, 8, 2) HX_CASE(8, 8, 1)
+    HX_CASE(8, 8, 4) HX_CASE(8, 8, 2) HX_CASE(8, 8, 1) HX_CASE(4, 8, 4) HX_CASE(4, 8, 2) HX_CASE(4, 8, 1)
+    HX_CASE(2, 8, 4) HX_CASE(2, 8, 2) HX_CASE(2, 8, 1) HX_CASE(1, 8, 4) HX_CASE(1, 8, 2) HX_CASE(1, 8, 1)
     e = cudaErrorInvalidConfiguration;
 #undef HX_CASE
     if (e == cudaSuccess) ++*launches;
