@@ -69,7 +69,13 @@ __global__ void hx_cpath_staged_kernel(HxForestDev f, const uint32_t* __restrict
         for (uint32_t i = segS[lev] + t; i < hi; i += tpw) {
             float tl = 0.0f;
             const uint32_t e1 = rowS[i + 1];
-            for (uint32_t e = rowS[i]; e < e1; ++e) tl = fmaxf(tl, cpS[colS[e]]);
+            uint32_t e = rowS[i];
+            for (; e + 4 <= e1; e += 4) {                     // four successors in flight (max is exact: any order)
+                const uint32_t c0 = colS[e], c1 = colS[e + 1], c2 = colS[e + 2], c3 = colS[e + 3];
+                const float v0 = cpS[c0], v1 = cpS[c1], v2 = cpS[c2], v3 = cpS[c3];
+                tl = fmaxf(fmaxf(tl, fmaxf(v0, v1)), fmaxf(v2, v3));
+            }
+            for (; e < e1; ++e) tl = fmaxf(tl, cpS[colS[e]]);
             const float c = __fadd_rn(costS[i], tl);
             cpS[i] = c;
             costS[i] = tl;
@@ -134,12 +140,32 @@ cudaError_t hx_launch_cost_update(const HxForestDev& f, const uint32_t* idx, con
 }
 
 cudaError_t hx_launch_cpath(const HxForestDev& f, const HxCpClass* classes, int n_classes,
-                            cudaStream_t stream, long long* launches) {
+                            cudaStream_t stream, long long* launches, const HxForkJoin* fj) {
+    // the classes touch disjoint workflows: with side streams the second and later classes run
+    // beside the first one and join the caller's stream afterwards
+    int n_live = 0;
+    for (int k = 0; k < n_classes; ++k) n_live += classes[k].count != 0;
+    const bool fork = fj && fj->ready && n_live > 1;
+    if (fork) {
+        cudaError_t e = cudaEventRecord(fj->fork, stream);
+        if (e != cudaSuccess) return e;
+    }
+    int side = 0;
+    bool first = true;
     for (int k = 0; k < n_classes; ++k) {
         const HxCpClass& c = classes[k];
         if (c.count == 0) continue;
+        cudaStream_t s = stream;
+        int my_side = -1;
+        if (fork && !first && side < 3) {
+            my_side = side++;
+            s = fj->aux[my_side];
+            cudaError_t e = cudaStreamWaitEvent(s, fj->fork, 0);
+            if (e != cudaSuccess) return e;
+        }
+        first = false;
         if (c.smem_per_wf == 0) {
-            hx_cpath_global_kernel<<<c.count, 256, 0, stream>>>(f, c.wf_ids, c.count);
+            hx_cpath_global_kernel<<<c.count, 256, 0, s>>>(f, c.wf_ids, c.count);
         } else {
             const int threads = c.threads_per_wf * c.wfs_per_block;
             const size_t smem = c.smem_per_wf * c.wfs_per_block;
@@ -150,7 +176,7 @@ cudaError_t hx_launch_cpath(const HxForestDev& f, const HxCpClass* classes, int 
                     cudaError_t e = hx_opt_in_smem(hx_cpath_staged_kernel<true>, smem, allowed, 40 * 1024);
                     if (e != cudaSuccess) return e;
                 }
-                hx_cpath_staged_kernel<true><<<grid, threads, smem, stream>>>(
+                hx_cpath_staged_kernel<true><<<grid, threads, smem, s>>>(
                     f, c.wf_ids, c.count, 32, c.wfs_per_block, (uint32_t)c.smem_per_wf);
             } else {
                 {   // static + dynamic shared memory may exceed the 48 KB default
@@ -158,13 +184,17 @@ cudaError_t hx_launch_cpath(const HxForestDev& f, const HxCpClass* classes, int 
                     cudaError_t e = hx_opt_in_smem(hx_cpath_staged_kernel<false>, smem, allowed, 40 * 1024);
                     if (e != cudaSuccess) return e;
                 }
-                hx_cpath_staged_kernel<false><<<grid, threads, smem, stream>>>(
+                hx_cpath_staged_kernel<false><<<grid, threads, smem, s>>>(
                     f, c.wf_ids, c.count, c.threads_per_wf, 1, (uint32_t)c.smem_per_wf);
             }
         }
         ++*launches;
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
+        if (my_side >= 0) {
+            if ((e = cudaEventRecord(fj->join[my_side], s)) != cudaSuccess) return e;
+            if ((e = cudaStreamWaitEvent(stream, fj->join[my_side], 0)) != cudaSuccess) return e;
+        }
     }
     return cudaSuccess;
 }

@@ -26,6 +26,7 @@ struct hx_cluster {
     uint32_t* d_node_wf = nullptr;
     float* d_elapsed = nullptr;
     std::vector<HxCpClass> classes;
+    HxForkJoin fj{};                    // side streams of the horizon pass, created with the first upload
     // host copies for incremental refinement: node -> internal index, node -> workflow, workflow -> class
     std::vector<uint32_t> h_inv, h_node_wf;
     std::vector<uint8_t> h_wf_class;
@@ -283,6 +284,10 @@ int hx_cluster_destroy(hx_cluster* h) {
     if (h->st_calls) cudaFree(h->st_calls);
     if (h->st_assign) cudaFree(h->st_assign);
     if (h->st_cost) cudaFree(h->st_cost);
+    if (h->fj.ready) {
+        for (int i = 0; i < 3; ++i) { cudaStreamDestroy(h->fj.aux[i]); cudaEventDestroy(h->fj.join[i]); }
+        cudaEventDestroy(h->fj.fork);
+    }
     for (auto* v : {&h->spans, &h->spare})
         for (auto& sp : *v) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
     delete h;
@@ -422,6 +427,14 @@ int hx_dag_upload(hx_cluster* h, const uint32_t* row_ptr, const uint32_t* col_id
         c.wf_ids = d_ids; c.count = (uint32_t)ids[k].size();
         h->classes.push_back(c);
     }
+    if (!h->fj.ready) {
+        bool ok = cudaEventCreateWithFlags(&h->fj.fork, cudaEventDisableTiming) == cudaSuccess;
+        for (int i = 0; i < 3 && ok; ++i)
+            ok = cudaStreamCreateWithFlags(&h->fj.aux[i], cudaStreamNonBlocking) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&h->fj.join[i], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) return fail(h, HX_ERR_CUDA, "creating the side streams of the horizon pass");
+        h->fj.ready = 1;
+    }
     h->forest = f;
     h->h_inv = inv;
     h->h_node_wf.assign(node_workflow, node_workflow + N);
@@ -437,7 +450,7 @@ int hx_critical_path(hx_cluster* h, void* stream) {
     {
         SpanGuard span(h, 2, static_cast<cudaStream_t>(stream));
         HX_TRY(hx_launch_cpath(h->forest, h->classes.data(), (int)h->classes.size(),
-                               static_cast<cudaStream_t>(stream), &h->launches), "horizon kernels");
+                               static_cast<cudaStream_t>(stream), &h->launches, &h->fj), "horizon kernels");
     }
     h->cp_ready = true;
     return HX_OK;
@@ -516,7 +529,7 @@ int hx_dag_update_costs(hx_cluster* h, const uint32_t* node_ids, const float* ne
         SpanGuard span(h, 2, s);
         HX_TRY(hx_launch_cost_update(h->forest, h->d_upd_idx, h->d_upd_cost, (uint32_t)idx.size(), s, &h->launches), "cost update kernel");
         if (h->cp_ready)
-            HX_TRY(hx_launch_cpath(h->forest, part.data(), (int)part.size(), s, &h->launches), "horizon kernels");
+            HX_TRY(hx_launch_cpath(h->forest, part.data(), (int)part.size(), s, &h->launches, &h->fj), "horizon kernels");
     }
     (void)W;
     return HX_OK;

@@ -150,8 +150,16 @@ struct HxCpClass {
     size_t smem_per_wf;        // bytes of staging per workflow, 0 = work in global memory
 };
 
+// Side streams and events for running the independent workflow classes of one horizon pass
+// next to each other (fork from / join into the caller's stream).  Zero-initialised = serial.
+struct HxForkJoin {
+    cudaStream_t aux[3];
+    cudaEvent_t fork, join[3];
+    int ready;
+};
+
 cudaError_t hx_launch_cpath(const HxForestDev& f, const HxCpClass* classes, int n_classes,
-                            cudaStream_t stream, long long* launches);
+                            cudaStream_t stream, long long* launches, const HxForkJoin* fj = nullptr);
 
 // Launch shape of workflow class k (by staging footprint): 0 = one warp, <= 3 KB; 1 = one warp,
 // <= 24 KB; 2 = one block, <= 200 KB; 3 = one block working in global memory.
