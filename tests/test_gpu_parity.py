@@ -123,6 +123,32 @@ def test_scoring_ragged_shapes(hx, oracle, P, D, n):
     gc.close()
 
 
+@pytest.mark.parametrize("D, LD", [(5, 1), (12, 2), (24, 4)])
+@pytest.mark.parametrize("TC", [1, 2, 4, 8])
+def test_scoring_thread_tile_heights_of_narrow_pools(hx, oracle, D, LD, TC):
+    """For decode pools of at most 32 instances the kernel keeps eight warps per block and picks the thread
+    tile height (1, 2, 4 or 8 calls) from the batch size: a batch of 148 tiles of that height selects it on
+    a 148-SM device.  Every height of every lane layout is compared with the oracle, plain argmin and top-2."""
+    import torch
+    n_sm = torch.cuda.get_device_properties(0).multi_processor_count
+    rows = 8 * (32 // LD)                        # calls per block and unit of tile height
+    n = n_sm * rows * TC - 3                     # ragged last tile
+    P = 3
+    gc, oc = _cluster_pair(hx, P, D, seed=D * 10 + TC, tight=True)
+    calls = _calls(n, seed=n % 1000)
+    gc.set_options(flags=hx.HX_FLAG_NO_DAG)
+    a, c = gc.schedule_batch(calls)
+    oa, ocost, _ = oracle.schedule(oc, calls)
+    assert np.array_equal(a.cpu().numpy(), oa) and np.array_equal(c.cpu().numpy(), ocost)
+    m = min(n, 16000)                            # the capacity pass takes at most 65,536 calls
+    gc.set_options(topk=2, flags=hx.HX_FLAG_NO_DAG)
+    gc.schedule_batch(calls[:m])
+    pair, cost, prio = gc.topk_results(m)
+    op, ocs, opr, _, _ = oracle.topk(oc, calls[:m], 2)
+    assert np.array_equal(pair, op) and np.array_equal(cost, ocs) and np.array_equal(prio, opr)
+    gc.close()
+
+
 def test_exact_ties_and_infeasible_calls(hx, oracle):
     # identical instances, late decode admission: every pair of a decode type ties exactly
     P, D = 6, 5
