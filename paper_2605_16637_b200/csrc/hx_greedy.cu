@@ -17,7 +17,17 @@
 // pairs, (2) reduces the largest ratio, (3) commits and lists the calls to
 // re-project.  The arithmetic of a candidate is the canonical binary32 sequence
 // of the scoring kernel, so the results equal the definition bit for bit.
+//
+// Long queues run on a thread-block cluster of kCluster blocks (one SM each): call c belongs to
+// block c mod kCluster, every block keeps its own copy of the small simulated state, and per
+// iteration the blocks exchange their most urgent call and the winner's commit through
+// distributed shared memory with two cluster barriers.  All blocks reduce the same candidates and
+// apply the same commit, so their copies stay identical and every exit is taken by all of them.
+#include <cooperative_groups.h>
+
 #include "hx_internal.h"
+
+namespace cg = cooperative_groups;
 
 namespace {
 
@@ -40,14 +50,22 @@ struct GreedyParams {
     int* status;
 };
 
+template <int NC>   // blocks of the cluster (1 = a plain single block)
 __global__ void __launch_bounds__(kThreads, 1) hx_greedy_kernel(const __grid_constant__ GreedyParams prm) {
     extern __shared__ __align__(16) unsigned char smem[];
     __shared__ float red_v[kWarps];
     __shared__ int red_c[kWarps];
     __shared__ int s_call, s_p, s_d, s_ndirty;
+    __shared__ float x_v[NC];                  // most urgent call of every block (written by its owner block)
+    __shared__ int x_c[NC];
+    __shared__ float x_commit[4];              // p, d (as int bits), prefill time, demand of the committed call
     const HxTables& T = prm.t;
-    const int P = T.P, D = T.D, G = T.G, n = prm.n;
+    const int P = T.P, D = T.D, G = T.G;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    int rank = 0;
+    if (NC > 1) rank = (int)cg::this_cluster().block_rank();
+    const int n_all = prm.n;
+    const int n = (n_all - rank + NC - 1) / NC;                // calls of this block: c = li * NC + rank
 
     float* invL = reinterpret_cast<float*>(smem);              // [P][D]
     float* qPs = invL + (size_t)P * D;                         // [P]
@@ -70,7 +88,8 @@ __global__ void __launch_bounds__(kThreads, 1) hx_greedy_kernel(const __grid_con
     for (int p = tid; p < P; p += kThreads) { qPs[p] = T.qP[p]; typePs[p] = T.typeP[p]; }
     for (int d = tid; d < D; d += kThreads) { qDs[d] = T.qD[d]; capDs[d] = T.capD[d]; frees[d] = T.freeD[d]; typeDs[d] = T.typeD[d]; }
     for (int c = tid; c < n; c += kThreads) {
-        const uint4 raw = __ldg(reinterpret_cast<const uint4*>(prm.calls) + c);
+        const int gcall = c * NC + rank;
+        const uint4 raw = __ldg(reinterpret_cast<const uint4*>(prm.calls) + gcall);
         bool bad = raw.y >= (unsigned)T.M;
         float el = 0.f, H = 1.f;
         if (!(prm.flags & HX_FLAG_NO_DAG)) {
@@ -84,12 +103,12 @@ __global__ void __launch_bounds__(kThreads, 1) hx_greedy_kernel(const __grid_con
         cR[c] = HX_NEG_INF;
         cpair[c] = bad ? kDead : kNoPair;
         dirty[c] = (unsigned short)c;
-        prm.out_assign[c] = -1; prm.out_ratio[c] = HX_INF; prm.out_order[c] = -1;
+        prm.out_assign[gcall] = -1; prm.out_ratio[gcall] = HX_INF; prm.out_order[gcall] = -1;
     }
     if (tid == 0) s_ndirty = n;
     __syncthreads();
 
-    for (int it = 0; it < n; ++it) {
+    for (int it = 0; it < n_all; ++it) {
         // (1) re-project the listed calls: one warp per call, lanes over the pairs
         const int nd = s_ndirty;
         float* tpre = scratch + warp * 64;
@@ -139,7 +158,7 @@ __global__ void __launch_bounds__(kThreads, 1) hx_greedy_kernel(const __grid_con
         float rv = HX_NEG_INF; int rc = 0x7fffffff;
         for (int c = tid; c < n; c += kThreads) {
             const float r = cR[c];
-            if (r > rv) { rv = r; rc = c; }                    // ascending c: keeps the lowest index
+            if (r > rv) { rv = r; rc = c * NC + rank; }        // ascending c: keeps the lowest index
         }
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) {
@@ -158,27 +177,64 @@ __global__ void __launch_bounds__(kThreads, 1) hx_greedy_kernel(const __grid_con
                 if (ov > rv || (ov == rv && oc < rc)) { rv = ov; rc = oc; }
             }
             if (lane == 0) {
-                if (rc == 0x7fffffff) {
-                    s_call = -1;                               // nobody left that fits anywhere
+                if (NC > 1) {                                  // publish the block's candidate in every block
+                    cg::cluster_group cl = cg::this_cluster();
+                    for (int r = 0; r < NC; ++r) {
+                        *cl.map_shared_rank(&x_v[rank], r) = rv;
+                        *cl.map_shared_rank(&x_c[rank], r) = rc;
+                    }
                 } else {
-                    // (3) commit: update the simulated state
-                    const int bj = cpair[rc], p = bj >> 16, d = bj & 0xFFFF;
-                    const float nt = cn[rc], ot = co[rc];
-                    const int mdl = cmodel[rc];
-                    const float phi = prm.ct.phi[mdl], omega = prm.ct.omega[mdl], kappa = prm.ct.kappa[mdl];
-                    const float kvB = __fmul_rn(nt, kappa);
-                    const int g = typePs[p];
-                    const float tp = fmaxf(__fmul_rn(__fmul_rn(nt, phi), prm.ct.invF[g]), __fmul_rn(__fadd_rn(omega, kvB), prm.ct.invB[g]));
-                    qPs[p] = __fadd_rn(qPs[p], tp);
-                    frees[d] = __fsub_rn(frees[d], __fadd_rn(nt, ot));
-                    prm.out_assign[rc] = p * D + d;
-                    prm.out_ratio[rc] = rv;
-                    prm.out_order[it] = rc;
-                    cpair[rc] = kDead; cR[rc] = HX_NEG_INF;
-                    s_call = rc; s_p = p; s_d = d;
+                    x_v[0] = rv; x_c[0] = rc;
                 }
-                s_ndirty = 0;
             }
+        }
+        if (NC > 1) cg::this_cluster().sync(); else __syncthreads();      // every thread of every block
+        if (warp == 0) {
+            rv = lane < NC ? x_v[lane] : HX_NEG_INF;           // all blocks reduce the same list
+            rc = lane < NC ? x_c[lane] : 0x7fffffff;
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) {
+                const float ov = __shfl_xor_sync(0xffffffffu, rv, off);
+                const int oc = __shfl_xor_sync(0xffffffffu, rc, off);
+                if (ov > rv || (ov == rv && oc < rc)) { rv = ov; rc = oc; }
+            }
+            const bool none = rc == 0x7fffffff;
+            if (lane == 0) s_call = none ? -1 : rc;            // -1: nobody left that fits anywhere
+            if (lane == 0 && !none && rc % NC == rank) {
+                // (3) commit by the block that owns the call
+                const int li = rc / NC;
+                const int bj = cpair[li], p = bj >> 16, d = bj & 0xFFFF;
+                const float nt = cn[li], ot = co[li];
+                const int mdl = cmodel[li];
+                const float phi = prm.ct.phi[mdl], omega = prm.ct.omega[mdl], kappa = prm.ct.kappa[mdl];
+                const float kvB = __fmul_rn(nt, kappa);
+                const int g = typePs[p];
+                const float tp = fmaxf(__fmul_rn(__fmul_rn(nt, phi), prm.ct.invF[g]), __fmul_rn(__fadd_rn(omega, kvB), prm.ct.invB[g]));
+                const float m = __fadd_rn(nt, ot);
+                prm.out_assign[rc] = p * D + d;
+                prm.out_ratio[rc] = rv;
+                prm.out_order[it] = rc;
+                cpair[li] = kDead; cR[li] = HX_NEG_INF;
+                if (NC > 1) {
+                    cg::cluster_group cl = cg::this_cluster();
+                    for (int r = 0; r < NC; ++r) {
+                        float* xc = cl.map_shared_rank(x_commit, r);
+                        xc[0] = __int_as_float(p); xc[1] = __int_as_float(d); xc[2] = tp; xc[3] = m;
+                    }
+                } else {
+                    x_commit[0] = __int_as_float(p); x_commit[1] = __int_as_float(d); x_commit[2] = tp; x_commit[3] = m;
+                }
+            }
+        }
+        if (NC > 1) cg::this_cluster().sync(); else __syncthreads();      // the commit has reached every block
+        if (tid == 0) {
+            if (s_call >= 0) {                                 // the same update in every block
+                const int p = __float_as_int(x_commit[0]), d = __float_as_int(x_commit[1]);
+                qPs[p] = __fadd_rn(qPs[p], x_commit[2]);
+                frees[d] = __fsub_rn(frees[d], x_commit[3]);
+                s_p = p; s_d = d;
+            }
+            s_ndirty = 0;
         }
         __syncthreads();
         if (s_call < 0) break;
@@ -193,17 +249,27 @@ __global__ void __launch_bounds__(kThreads, 1) hx_greedy_kernel(const __grid_con
         }
         __syncthreads();
     }
-    if (prm.commit) {
+    if (prm.commit && rank == 0) {
         for (int p = tid; p < P; p += kThreads) T.qP[p] = qPs[p];
         for (int d = tid; d < D; d += kThreads) T.freeD[d] = frees[d];
     }
+    if (NC > 1) cg::this_cluster().sync();     // no block leaves while another may still write into it
 }
 
 }  // namespace
 
+constexpr int kCluster = 8;                    // blocks of the cluster used for long queues (portable maximum)
+constexpr int kClusterFrom = 512;              // queues longer than this use the cluster
+
+static size_t greedy_smem(const HxTables& t, int calls_per_block) {
+    return ((size_t)t.P * t.D + 2 * (size_t)t.P + 5 * (size_t)t.D + kWarps * 64 + 7 * (size_t)calls_per_block) * 4 +
+           (size_t)calls_per_block * 2 + 16;
+}
+
+// Shared memory of one block for a queue of n_calls (the longest queue a single block must be able
+// to take is kClusterFrom calls; longer ones are split over the cluster when the device can run it).
 size_t hx_greedy_smem_bytes(const HxTables& t, int n_calls) {
-    return ((size_t)t.P * t.D + 2 * (size_t)t.P + 5 * (size_t)t.D + kWarps * 64 + 7 * (size_t)n_calls) * 4 +
-           (size_t)n_calls * 2 + 16;
+    return greedy_smem(t, n_calls > kClusterFrom ? (n_calls + kCluster - 1) / kCluster : n_calls);
 }
 
 cudaError_t hx_launch_greedy(const HxTables& t, const HxConstTables& ct, const HxDagView& dag,
@@ -213,11 +279,30 @@ cudaError_t hx_launch_greedy(const HxTables& t, const HxConstTables& ct, const H
     GreedyParams prm;
     prm.t = t; prm.ct = ct; prm.dag = dag; prm.calls = calls; prm.n = n_calls; prm.flags = flags; prm.commit = commit;
     prm.out_assign = out_assign; prm.out_ratio = out_ratio; prm.out_order = out_order; prm.status = status;
-    const size_t smem = hx_greedy_smem_bytes(t, n_calls);
-    static size_t allowed[64];
-    cudaError_t e = hx_opt_in_smem(hx_greedy_kernel, smem, allowed, 40 * 1024);
-    if (e != cudaSuccess) return e;
-    hx_greedy_kernel<<<1, kThreads, smem, stream>>>(prm);
+    cudaError_t e;
+    if (n_calls > kClusterFrom) {
+        const size_t smem = greedy_smem(t, (n_calls + kCluster - 1) / kCluster);
+        static size_t allowed[64];
+        if ((e = hx_opt_in_smem(hx_greedy_kernel<kCluster>, smem, allowed, 40 * 1024)) != cudaSuccess) return e;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(kCluster); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = kCluster; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        int n_clusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&n_clusters, hx_greedy_kernel<kCluster>, &cfg) == cudaSuccess && n_clusters >= 1) {
+            e = cudaLaunchKernelEx(&cfg, hx_greedy_kernel<kCluster>, prm);
+            if (e == cudaSuccess) ++*launches;
+            return e;
+        }
+        (void)cudaGetLastError();              // the device cannot host the cluster: one block, if the queue fits
+        if (greedy_smem(t, n_calls) > (size_t)227 * 1024) return cudaErrorInvalidConfiguration;
+    }
+    const size_t smem = greedy_smem(t, n_calls);
+    static size_t allowed1[64];
+    if ((e = hx_opt_in_smem(hx_greedy_kernel<1>, smem, allowed1, 40 * 1024)) != cudaSuccess) return e;
+    hx_greedy_kernel<1><<<1, kThreads, smem, stream>>>(prm);
     e = cudaGetLastError();
     if (e == cudaSuccess) ++*launches;
     return e;
