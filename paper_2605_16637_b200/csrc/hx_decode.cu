@@ -18,7 +18,17 @@
 // One persistent block; one warp projects one call with the lanes over the
 // instances; adding an interval only delays starts on that instance, so only
 // calls whose best instance it was are projected again.
+//
+// Long queues run on a thread-block cluster: call c belongs to block c mod kCluster, every block
+// keeps its own copy of the step functions, and per iteration the blocks exchange their most urgent
+// call and the winner's interval through distributed shared memory with two cluster barriers; all
+// blocks reduce the same candidates and insert the same interval, so the copies stay identical and
+// every exit is taken by all blocks.
+#include <cooperative_groups.h>
+
 #include "hx_internal.h"
+
+namespace cg = cooperative_groups;
 
 namespace {
 
@@ -74,15 +84,25 @@ __device__ int warp_cut(float* t, float* u, int& K, float x, int lane) {
     return k + 1;
 }
 
+template <int NC>   // blocks of the cluster (1 = a plain single block)
 __global__ void __launch_bounds__(kThreads, 1) hx_decode_kernel(const __grid_constant__ DecodeParams prm) {
     extern __shared__ __align__(16) unsigned char smem[];
     __shared__ float red_v[kWarps];
     __shared__ int red_c[kWarps];
     __shared__ int s_call, s_d, s_ndirty;
+    __shared__ float x_v[NC];                  // most urgent call of every block (written by its owner block)
+    __shared__ int x_c[NC];
+    __shared__ float x_commit[4];              // instance (int bits), start, finish, demand of the committed call
     const HxTables& T = prm.t;
-    const int D = T.D, G = T.G, n = prm.n;
+    const int D = T.D, G = T.G;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int cap = prm.work.cap;
+    int rank = 0;
+    if (NC > 1) rank = (int)cg::this_cluster().block_rank();
+    const int n_all = prm.n;
+    const int n = (n_all - rank + NC - 1) / NC;                // calls of this block: c = li * NC + rank
+    float* const wt = prm.work.t + (size_t)rank * D * cap;      // this block's copy of the step functions
+    float* const wu = prm.work.u + (size_t)rank * D * cap;
 
     float* capDs = reinterpret_cast<float*>(smem);              // [D]
     int* typeDs = reinterpret_cast<int*>(capDs + D);            // [D]
@@ -107,19 +127,20 @@ __global__ void __launch_bounds__(kThreads, 1) hx_decode_kernel(const __grid_con
     __syncthreads();
     for (int d = warp; d < D; d += kWarps)                      // simulated state starts as the snapshot
         for (int i = lane; i < Ks[d]; i += 32) {
-            prm.work.t[(size_t)d * cap + i] = prm.base.t[(size_t)d * prm.base.cap + i];
-            prm.work.u[(size_t)d * cap + i] = prm.base.u[(size_t)d * prm.base.cap + i];
+            wt[(size_t)d * cap + i] = prm.base.t[(size_t)d * prm.base.cap + i];
+            wu[(size_t)d * cap + i] = prm.base.u[(size_t)d * prm.base.cap + i];
         }
     for (int c = tid; c < n; c += kThreads) {
-        const uint4 raw = __ldg(reinterpret_cast<const uint4*>(prm.calls) + c);
+        const int gcall = c * NC + rank;
+        const uint4 raw = __ldg(reinterpret_cast<const uint4*>(prm.calls) + gcall);
         bool bad = raw.y >= (unsigned)T.M;
         float el = 0.f, H = 1.f;
         if (!(prm.flags & HX_FLAG_NO_DAG)) {
             if (raw.x < prm.dag.n_nodes) { const uint32_t w = prm.dag.node_wf[raw.x]; el = prm.dag.elapsed[w]; H = prm.dag.H[w]; }
             else bad = true;
         }
-        const int lk = prm.lock ? prm.lock[c] : -1;
-        const float rd = prm.ready ? prm.ready[c] : 0.f;
+        const int lk = prm.lock ? prm.lock[gcall] : -1;
+        const float rd = prm.ready ? prm.ready[gcall] : 0.f;
         if (lk >= D || !(rd >= 0.f) || rd == HX_INF) bad = true;
         if (bad) atomicExch(prm.status, HX_ERR_INVALID_ARG);
         cn[c] = __uint_as_float(raw.z); co[c] = __uint_as_float(raw.w);
@@ -128,12 +149,12 @@ __global__ void __launch_bounds__(kThreads, 1) hx_decode_kernel(const __grid_con
         cR[c] = HX_NEG_INF; cstart[c] = HX_INF; cfin[c] = HX_INF;
         cbest[c] = bad ? kDead : kNoInst;
         dirty[c] = (unsigned short)c;
-        prm.out_inst[c] = -1; prm.out_start[c] = HX_INF; prm.out_ratio[c] = HX_INF; prm.out_order[c] = -1;
+        prm.out_inst[gcall] = -1; prm.out_start[gcall] = HX_INF; prm.out_ratio[gcall] = HX_INF; prm.out_order[gcall] = -1;
     }
     if (tid == 0) s_ndirty = n;
     __syncthreads();
 
-    for (int it = 0; it < n; ++it) {
+    for (int it = 0; it < n_all; ++it) {
         // (1) project the listed calls: one warp per call, lanes over the decode instances
         const int nd = s_ndirty;
         for (int i = warp; i < nd; i += kWarps) {
@@ -151,8 +172,8 @@ __global__ void __launch_bounds__(kThreads, 1) hx_decode_kernel(const __grid_con
             for (int d = lane; d < D; d += 32) {
                 if ((lk >= 0 && lk != d) || !(m <= capDs[d])) continue;
                 const float tau = __fmul_rn(__fmul_rn(ot, step), prm.ct.invB[typeDs[d]]);
-                const float* tt = prm.work.t + (size_t)d * cap;
-                const float* uu = prm.work.u + (size_t)d * cap;
+                const float* tt = wt + (size_t)d * cap;
+                const float* uu = wu + (size_t)d * cap;
                 const int K = Ks[d];
                 int k = 0;
                 while (k + 1 < K && tt[k + 1] <= rd) ++k;       // segment that holds the ready time
@@ -187,7 +208,7 @@ __global__ void __launch_bounds__(kThreads, 1) hx_decode_kernel(const __grid_con
         float rv = HX_NEG_INF; int rc = 0x7fffffff;
         for (int c = tid; c < n; c += kThreads) {
             const float r = cR[c];
-            if (r > rv) { rv = r; rc = c; }
+            if (r > rv) { rv = r; rc = c * NC + rank; }
         }
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) {
@@ -205,29 +226,67 @@ __global__ void __launch_bounds__(kThreads, 1) hx_decode_kernel(const __grid_con
                 const int oc = __shfl_xor_sync(0xffffffffu, rc, off);
                 if (ov > rv || (ov == rv && oc < rc)) { rv = ov; rc = oc; }
             }
-            // (3) commit (warp 0): add the interval [start, finish) with m tokens to the step function
-            if (rc == 0x7fffffff) {
-                if (lane == 0) { s_call = -1; s_ndirty = 0; }
-            } else {
-                const int d = cbest[rc];
-                const float s = cstart[rc], e = cfin[rc], m = __fadd_rn(cn[rc], co[rc]);
-                float* tt = prm.work.t + (size_t)d * cap;
-                float* uu = prm.work.u + (size_t)d * cap;
-                int K = Ks[d];
-                if (K + 2 > cap) {                              // cannot happen with the capacity the host sizes
-                    if (lane == 0) { atomicExch(prm.status, HX_ERR_INVALID_ARG); s_call = -1; s_ndirty = 0; }
-                } else {
-                    const int a = warp_cut(tt, uu, K, s, lane);
-                    const int b = warp_cut(tt, uu, K, e, lane);
-                    for (int k = a + lane; k < b; k += 32) uu[k] = __fadd_rn(uu[k], m);
-                    if (lane == 0) {
-                        Ks[d] = K;
-                        prm.out_inst[rc] = d; prm.out_start[rc] = s; prm.out_ratio[rc] = rv; prm.out_order[it] = rc;
-                        cbest[rc] = kDead; cR[rc] = HX_NEG_INF;
-                        s_call = rc; s_d = d; s_ndirty = 0;
+            if (lane == 0) {
+                if (NC > 1) {                                  // publish the block's candidate in every block
+                    cg::cluster_group cl = cg::this_cluster();
+                    for (int r = 0; r < NC; ++r) {
+                        *cl.map_shared_rank(&x_v[rank], r) = rv;
+                        *cl.map_shared_rank(&x_c[rank], r) = rc;
                     }
+                } else {
+                    x_v[0] = rv; x_c[0] = rc;
                 }
             }
+        }
+        if (NC > 1) cg::this_cluster().sync(); else __syncthreads();      // every thread of every block
+        if (warp == 0) {
+            rv = lane < NC ? x_v[lane] : HX_NEG_INF;           // all blocks reduce the same list
+            rc = lane < NC ? x_c[lane] : 0x7fffffff;
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) {
+                const float ov = __shfl_xor_sync(0xffffffffu, rv, off);
+                const int oc = __shfl_xor_sync(0xffffffffu, rc, off);
+                if (ov > rv || (ov == rv && oc < rc)) { rv = ov; rc = oc; }
+            }
+            if (lane == 0) s_call = rc == 0x7fffffff ? -1 : rc;
+            if (lane == 0 && rc != 0x7fffffff && rc % NC == rank) {
+                // the block that owns the call publishes its interval and records the result
+                const int li = rc / NC;
+                const int d = cbest[li];
+                const float st = cstart[li], en = cfin[li], m = __fadd_rn(cn[li], co[li]);
+                prm.out_inst[rc] = d; prm.out_start[rc] = st; prm.out_ratio[rc] = rv; prm.out_order[it] = rc;
+                cbest[li] = kDead; cR[li] = HX_NEG_INF;
+                if (NC > 1) {
+                    cg::cluster_group cl = cg::this_cluster();
+                    for (int r = 0; r < NC; ++r) {
+                        float* xc = cl.map_shared_rank(x_commit, r);
+                        xc[0] = __int_as_float(d); xc[1] = st; xc[2] = en; xc[3] = m;
+                    }
+                } else {
+                    x_commit[0] = __int_as_float(d); x_commit[1] = st; x_commit[2] = en; x_commit[3] = m;
+                }
+            }
+        }
+        if (NC > 1) cg::this_cluster().sync(); else __syncthreads();      // the interval has reached every block
+        if (warp == 0) {
+            // (3) commit (warp 0 of every block): add the interval [start, finish) with m tokens to the block's copy
+            if (s_call >= 0) {
+                const int d = __float_as_int(x_commit[0]);
+                const float st = x_commit[1], en = x_commit[2], m = x_commit[3];
+                float* tt = wt + (size_t)d * cap;
+                float* uu = wu + (size_t)d * cap;
+                int K = Ks[d];
+                __syncwarp();
+                if (K + 2 > cap) {                              // cannot happen with the capacity the host sizes
+                    if (lane == 0) { atomicExch(prm.status, HX_ERR_INVALID_ARG); s_call = -1; }
+                } else {
+                    const int a = warp_cut(tt, uu, K, st, lane);
+                    const int b = warp_cut(tt, uu, K, en, lane);
+                    for (int k = a + lane; k < b; k += 32) uu[k] = __fadd_rn(uu[k], m);
+                    if (lane == 0) { Ks[d] = K; s_d = d; }
+                }
+            }
+            if (lane == 0) s_ndirty = 0;
         }
         __syncthreads();
         if (s_call < 0) break;
@@ -236,24 +295,32 @@ __global__ void __launch_bounds__(kThreads, 1) hx_decode_kernel(const __grid_con
             if (cbest[c] == ds) dirty[atomicAdd(&s_ndirty, 1)] = (unsigned short)c;
         __syncthreads();
     }
-    if (prm.commit) {                                           // the simulated state becomes the snapshot
+    if (prm.commit && rank == 0) {                              // the simulated state becomes the snapshot
         __syncthreads();
         for (int d = warp; d < D; d += kWarps) {
             const int K = min(Ks[d], prm.base.cap);
             for (int i = lane; i < K; i += 32) {
-                prm.base.t[(size_t)d * prm.base.cap + i] = prm.work.t[(size_t)d * cap + i];
-                prm.base.u[(size_t)d * prm.base.cap + i] = prm.work.u[(size_t)d * cap + i];
+                prm.base.t[(size_t)d * prm.base.cap + i] = wt[(size_t)d * cap + i];
+                prm.base.u[(size_t)d * prm.base.cap + i] = wu[(size_t)d * cap + i];
             }
             if (lane == 0) prm.base.K[d] = K;
         }
     }
+    if (NC > 1) cg::this_cluster().sync();     // no block leaves while another may still write into it
 }
 
 }  // namespace
 
-size_t hx_decode_smem_bytes(const HxTables& t, int n_calls) {
-    return (3 * (size_t)t.D + 11 * (size_t)n_calls) * 4 + (size_t)n_calls * 2 + 16;
+constexpr int kCluster = 8;                    // blocks of the cluster used for long queues
+constexpr int kClusterFrom = 256;              // queues longer than this use the cluster
+
+static size_t decode_smem(const HxTables& t, int calls_per_block) {
+    return (3 * (size_t)t.D + 11 * (size_t)calls_per_block) * 4 + (size_t)calls_per_block * 2 + 16;
 }
+
+size_t hx_decode_smem_bytes(const HxTables& t, int n_calls) { return decode_smem(t, n_calls); }
+
+int hx_decode_replicas() { return kCluster; }
 
 cudaError_t hx_launch_decode(const HxTables& t, const HxConstTables& ct, const HxDagView& dag,
                              const HxStepFns& base, const HxStepFns& work,
@@ -265,11 +332,29 @@ cudaError_t hx_launch_decode(const HxTables& t, const HxConstTables& ct, const H
     prm.calls = calls; prm.lock = lock; prm.ready = ready; prm.n = n_calls; prm.flags = flags; prm.commit = commit;
     prm.out_inst = out_inst; prm.out_start = out_start; prm.out_ratio = out_ratio; prm.out_order = out_order;
     prm.status = status;
-    const size_t smem = hx_decode_smem_bytes(t, n_calls);
-    static size_t allowed[64];
-    cudaError_t e = hx_opt_in_smem(hx_decode_kernel, smem, allowed, 40 * 1024);
-    if (e != cudaSuccess) return e;
-    hx_decode_kernel<<<1, kThreads, smem, stream>>>(prm);
+    cudaError_t e;
+    if (n_calls > kClusterFrom) {
+        const size_t smem = decode_smem(t, (n_calls + kCluster - 1) / kCluster);
+        static size_t allowed[64];
+        if ((e = hx_opt_in_smem(hx_decode_kernel<kCluster>, smem, allowed, 40 * 1024)) != cudaSuccess) return e;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(kCluster); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = kCluster; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        int n_clusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&n_clusters, hx_decode_kernel<kCluster>, &cfg) == cudaSuccess && n_clusters >= 1) {
+            e = cudaLaunchKernelEx(&cfg, hx_decode_kernel<kCluster>, prm);
+            if (e == cudaSuccess) ++*launches;
+            return e;
+        }
+        (void)cudaGetLastError();              // the device cannot host the cluster: one block
+    }
+    const size_t smem = decode_smem(t, n_calls);
+    static size_t allowed1[64];
+    if ((e = hx_opt_in_smem(hx_decode_kernel<1>, smem, allowed1, 40 * 1024)) != cudaSuccess) return e;
+    hx_decode_kernel<1><<<1, kThreads, smem, stream>>>(prm);
     e = cudaGetLastError();
     if (e == cudaSuccess) ++*launches;
     return e;

@@ -747,8 +747,8 @@ int decode_reserve(hx_cluster* h, int cap, bool keep) {
     HX_TRY(dev_alloc(fresh, &b.t, (size_t)D * cap), "alloc decode intervals");
     HX_TRY(dev_alloc(fresh, &b.u, (size_t)D * cap), "alloc decode intervals");
     HX_TRY(dev_alloc(fresh, &b.K, (size_t)D), "alloc decode intervals");
-    HX_TRY(dev_alloc(fresh, &w.t, (size_t)D * cap), "alloc decode intervals");
-    HX_TRY(dev_alloc(fresh, &w.u, (size_t)D * cap), "alloc decode intervals");
+    HX_TRY(dev_alloc(fresh, &w.t, (size_t)hx_decode_replicas() * D * cap), "alloc decode intervals");
+    HX_TRY(dev_alloc(fresh, &w.u, (size_t)hx_decode_replicas() * D * cap), "alloc decode intervals");
     w.K = b.K;
     if (keep && h->dec_base.cap > 0) {
         const size_t ow = (size_t)h->dec_base.cap * sizeof(float);
