@@ -202,7 +202,9 @@ def run_cuda(args):
     out_cost = torch.empty(n_calls, dtype=torch.float32, device="cuda")
     host_assign = torch.empty(n_calls, dtype=torch.int32).pin_memory()
     host_cost = torch.empty(n_calls, dtype=torch.float32).pin_memory()
-    qP0, qD0, free0 = wl.load_s[:P].copy(), wl.load_s[P:].copy(), wl.kv_free[P:].copy()
+    # refreshed loads come from pinned host memory (also what a captured copy needs)
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a, np.float32).copy()).pin_memory().numpy()
+    qP0, qD0, free0 = pin(wl.load_s[:P]), pin(wl.load_s[P:]), pin(wl.kv_free[P:])
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")      # larger than the 126 MB L2
     stream = torch.cuda.current_stream()
     sptr = stream.cuda_stream
@@ -211,16 +213,16 @@ def run_cuda(args):
     ptrs = [(calls_dev[i * chunk:(i + 1) * chunk].data_ptr(), out_assign[i * chunk:(i + 1) * chunk].data_ptr(),
              out_cost[i * chunk:(i + 1) * chunk].data_ptr()) for i in range(n_chunks)]
 
-    def step_device(chunk_events=None):
-        hx.hx_critical_path(h, sptr)
-        hx.hx_cluster_update_loads(h, qP0, qD0, free0, sptr)
+    def step_device(sp, strm=None, chunk_events=None):
+        hx.hx_critical_path(h, sp)
+        hx.hx_cluster_update_loads(h, qP0, qD0, free0, sp)
         for i in range(n_chunks):
             if chunk_events is not None:
-                chunk_events[i][0].record(stream)
-            hx.hx_cluster_update_loads(h, None, None, free0, sptr)
-            hx.hx_schedule_batch(h, ptrs[i][0], chunk, ptrs[i][1], ptrs[i][2], sptr)
+                chunk_events[i][0].record(strm)
+            hx.hx_cluster_update_loads(h, None, None, free0, sp)
+            hx.hx_schedule_batch(h, ptrs[i][0], chunk, ptrs[i][1], ptrs[i][2], sp)
             if chunk_events is not None:
-                chunk_events[i][1].record(stream)
+                chunk_events[i][1].record(strm)
 
     ch_np = calls_host.numpy().view(hx.CALL_DTYPE).reshape(-1)
     ha_np, hc_np = host_assign.numpy(), host_cost.numpy()
@@ -239,32 +241,75 @@ def run_cuda(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(max(args.warmup, 3)):
-        step_device()
+    launches0 = gc.launch_count()
+    step_device(sptr)
+    launches_per_step = gc.launch_count() - launches0
+    for _ in range(max(args.warmup, 3) - 1):
+        step_device(sptr)
+    barrier()
+
+    # One step = 16 scheduler invocations of three short kernels each: launch-bound.  The whole step is
+    # captured once into a CUDA graph through the same C entry points and replayed (every pointer and
+    # size is the same in every step); if the capture is refused the step is enqueued call by call.
+    graph, mode = None, "eager"
+    if not args.no_graph:
+        try:
+            cap = torch.cuda.Stream()
+            cap.wait_stream(stream)
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=cap):
+                step_device(torch.cuda.current_stream().cuda_stream)
+            stream.wait_stream(cap)
+            g.replay(); g.replay()
+            torch.cuda.synchronize()
+            graph, mode = g, "cuda graph replay"
+        except Exception as exc:                          # keep measuring, say why
+            mode = "eager (capture refused: %s)" % str(exc).splitlines()[0][:80]
+            torch.cuda.synchronize()
     barrier()
 
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    gc.enable_kernel_timing(True)
-    gc.read_kernel_timing()
-    launches0 = gc.launch_count()
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    cev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_chunks)]
-           for _ in range(args.steps)]
     barrier()
     for k in range(args.steps):
         flush.zero_()                                   # L2 flush between timed iterations (not timed)
         ev[k][0].record(stream)
-        step_device(cev[k])
+        if graph is not None:
+            graph.replay()
+        else:
+            step_device(sptr)
         ev[k][1].record(stream)
     barrier()
-    launches = gc.launch_count() - launches0
+    launches = launches_per_step * args.steps
+    step_ms = np.array([a.elapsed_time(b) for a, b in ev])
+    status = gc.status()
+    replay_ok = None
+    if graph is not None:                               # a replayed step leaves the same placements as one enqueued call by call
+        got_a, got_c = out_assign.clone(), out_cost.clone()
+        step_device(sptr)
+        torch.cuda.synchronize()
+        replay_ok = bool(torch.equal(got_a, out_assign) and torch.equal(got_c, out_cost))
+
+    # second timed region, call by call with event pairs around every kernel family and every ready
+    # batch: per-kernel times (roofline of the scoring kernel, shares) and the ready-batch latency
+    n_inst = min(args.steps, 10)
+    gc.enable_kernel_timing(True)
+    gc.read_kernel_timing()
+    ev2 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_inst)]
+    cev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_chunks)]
+           for _ in range(n_inst)]
+    for k in range(n_inst):
+        flush.zero_()
+        ev2[k][0].record(stream)
+        step_device(sptr, stream, cev[k])
+        ev2[k][1].record(stream)
+    barrier()
     kt = gc.read_kernel_timing()
     gc.enable_kernel_timing(False)
-    step_ms = np.array([a.elapsed_time(b) for a, b in ev])
+    inst_ms = float(np.sum([a.elapsed_time(b) for a, b in ev2]))
     chunk_us = np.array([[a.elapsed_time(b) * 1e3 for a, b in row] for row in cev]).reshape(-1)
-    status = gc.status()
 
     # end to end through the host-buffer entry point (pinned host memory, copies inside the timed region)
     for _ in range(2):
@@ -311,7 +356,8 @@ def run_cuda(args):
                 "candidates_per_s_kernel": lane_rate,
                 "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch on this "
                                   "workload (profiles/hx_score_kernel_sweep_chunk.md)",
-                "time_share": {k: v[0] / max(total_ms, 1e-9) for k, v in kt.items()}}
+                "time_share": {k: v[0] / max(inst_ms, 1e-9) for k, v in kt.items()},
+                "timed_with": "%d steps enqueued call by call with event pairs around every kernel family" % n_inst}
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
@@ -340,7 +386,9 @@ def run_cuda(args):
                                      "ready batch, CUDA events"},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "what": "hx_schedule_batch_host per chunk from pinned host memory, wall clock"},
-        "gpu_launches": int(launches), "kernel_ms_per_step": {k: v[0] / args.steps for k, v in kt.items()},
+        "gpu_launches": int(launches), "launch_mode": mode, "replay_matches_call_by_call": replay_ok,
+        "ms_per_step_call_by_call_instrumented": inst_ms / n_inst,
+        "kernel_ms_per_step": {k: v[0] / n_inst for k, v in kt.items()},
         "device_status": status, "roofline": roofline, "cpu_baseline": cpu, "clocks": clocks,
         "greedy_planner": greedy,
         "decode_scheduler": decode_leg() if world == 1 and not args.no_cpu_baseline else None,
@@ -482,6 +530,7 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true",
                     help="skip the side legs outside the timed region (oracle sample, greedy planner)")
+    ap.add_argument("--no-graph", action="store_true", help="enqueue every step call by call instead of replaying a CUDA graph")
     ap.add_argument("--configs", action="store_true",
                     help="time the four smaller configurations instead (one JSON object)")
     args = ap.parse_args()
