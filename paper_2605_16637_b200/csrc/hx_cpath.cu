@@ -53,14 +53,27 @@ __global__ void hx_cpath_staged_kernel(HxForestDev f, const uint32_t* __restrict
     unsigned char* base = smem_raw + (size_t)g * smem_per_wf;
     float* cpS = reinterpret_cast<float*>(base);
     float* costS = cpS + n;                                   // becomes tail once a node is done
-    uint32_t* rowS = reinterpret_cast<uint32_t*>(costS + n);  // n + 1 entries, relative to es
+    uint32_t* rowS = reinterpret_cast<uint32_t*>(costS + n);  // n + 1 entries, absolute edge offsets
     uint32_t* segS = rowS + n + 1;                            // nlev + 1 entries
-    uint16_t* colS = reinterpret_cast<uint16_t*>(segS + nlev + 1);
+    uint16_t* colW = reinterpret_cast<uint16_t*>(segS + nlev + 1);   // copied as 32-bit words from an even edge offset
+    const uint32_t eodd = es & 1u;
+    uint16_t* colS = colW + eodd;                             // colS[e - es] = successor of edge e
 
-    for (uint32_t i = t; i < n; i += tpw) costS[i] = f.icost[ns + i];
-    for (uint32_t i = t; i <= n; i += tpw) rowS[i] = f.irow[ns + i] - es;
-    for (uint32_t i = t; i <= nlev; i += tpw) segS[i] = f.seg_off[ss + i];
-    for (uint32_t e = t; e < ne; e += tpw) colS[e] = f.icol16[es + e];
+    // the slice goes to shared memory with asynchronous 4-byte copies: all of them are in flight at once,
+    // where a load-then-store loop of one warp would pay one memory latency per iteration
+    auto cp4 = [](void* dst, const void* src) {
+        const unsigned sa = (unsigned)__cvta_generic_to_shared(dst);
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" :: "r"(sa), "l"(src) : "memory");
+    };
+    for (uint32_t i = t; i < n; i += tpw) cp4(costS + i, f.icost + ns + i);
+    for (uint32_t i = t; i <= n; i += tpw) cp4(rowS + i, f.irow + ns + i);
+    for (uint32_t i = t; i <= nlev; i += tpw) cp4(segS + i, f.seg_off + ss + i);
+    {
+        const uint32_t* src = reinterpret_cast<const uint32_t*>(f.icol16 + (es - eodd));
+        const uint32_t nw = (ne + eodd + 1) >> 1;             // the last word may reach one entry past the slice (padded array)
+        for (uint32_t i = t; i < nw; i += tpw) cp4(reinterpret_cast<uint32_t*>(colW) + i, src + i);
+    }
+    asm volatile("cp.async.wait_all;" ::: "memory");
     group_sync<WARP>();
 
     float hmax = 0.0f;
@@ -68,8 +81,8 @@ __global__ void hx_cpath_staged_kernel(HxForestDev f, const uint32_t* __restrict
         const uint32_t hi = segS[lev + 1];
         for (uint32_t i = segS[lev] + t; i < hi; i += tpw) {
             float tl = 0.0f;
-            const uint32_t e1 = rowS[i + 1];
-            uint32_t e = rowS[i];
+            const uint32_t e1 = rowS[i + 1] - es;
+            uint32_t e = rowS[i] - es;
             for (; e + 4 <= e1; e += 4) {                     // four successors in flight (max is exact: any order)
                 const uint32_t c0 = colS[e], c1 = colS[e + 1], c2 = colS[e + 2], c3 = colS[e + 3];
                 const float v0 = cpS[c0], v1 = cpS[c1], v2 = cpS[c2], v3 = cpS[c3];
@@ -83,10 +96,15 @@ __global__ void hx_cpath_staged_kernel(HxForestDev f, const uint32_t* __restrict
         }
         group_sync<WARP>();
     }
-    for (uint32_t i = t; i < n; i += tpw) {
-        const uint32_t v = f.perm[ns + i];
-        f.cp[v] = cpS[i];
-        f.tail[v] = costS[i];
+    for (uint32_t i0 = t; i0 < n; i0 += 4 * tpw) {            // four node numbers in flight per thread
+        uint32_t v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) v[u] = i0 + u * tpw < n ? __ldg(f.perm + ns + i0 + u * tpw) : 0u;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const uint32_t i = i0 + u * tpw;
+            if (i < n) { f.cp[v[u]] = cpS[i]; f.tail[v[u]] = costS[i]; }
+        }
     }
     hmax = group_max<WARP>(hmax, red, t, tpw);
     if (t == 0) f.H[w] = hmax;
@@ -157,7 +175,7 @@ cudaError_t hx_launch_cpath(const HxForestDev& f, const HxCpClass* classes, int 
         if (c.count == 0) continue;
         cudaStream_t s = stream;
         int my_side = -1;
-        if (fork && !first && side < 3) {
+        if (fork && !first && side < HX_CP_SIDE) {
             my_side = side++;
             s = fj->aux[my_side];
             cudaError_t e = cudaStreamWaitEvent(s, fj->fork, 0);

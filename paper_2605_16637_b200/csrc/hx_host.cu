@@ -285,7 +285,7 @@ int hx_cluster_destroy(hx_cluster* h) {
     if (h->st_assign) cudaFree(h->st_assign);
     if (h->st_cost) cudaFree(h->st_cost);
     if (h->fj.ready) {
-        for (int i = 0; i < 3; ++i) { cudaStreamDestroy(h->fj.aux[i]); cudaEventDestroy(h->fj.join[i]); }
+        for (int i = 0; i < HX_CP_SIDE; ++i) { cudaStreamDestroy(h->fj.aux[i]); cudaEventDestroy(h->fj.join[i]); }
         cudaEventDestroy(h->fj.fork);
     }
     for (auto* v : {&h->spans, &h->spare})
@@ -362,7 +362,7 @@ int hx_dag_upload(hx_cluster* h, const uint32_t* row_ptr, const uint32_t* col_id
     }
     wf_seg_start[W] = (uint32_t)seg_off.size();
     std::vector<uint32_t> irow((size_t)N + 1, 0), icol32(E), wf_edge_start((size_t)W + 1, 0);
-    std::vector<uint16_t> icol16(E);
+    std::vector<uint16_t> icol16((size_t)E + 2);       // two spare entries: slices are copied as 32-bit words
     std::vector<float> icost(N);
     for (uint32_t i = 0; i < N; ++i) {
         const uint32_t v = perm[i], ns = wf_node_start[node_workflow[v]];
@@ -377,15 +377,13 @@ int hx_dag_upload(hx_cluster* h, const uint32_t* row_ptr, const uint32_t* col_id
     for (uint32_t w = 0; w <= W; ++w) wf_edge_start[w] = irow[wf_node_start[w]];
 
     // classes of the horizon pass by staging footprint
-    const size_t kWarpSmall = hx_cpath_class_shape(0).smem_per_wf, kWarpBig = hx_cpath_class_shape(1).smem_per_wf,
-                 kBlock = hx_cpath_class_shape(2).smem_per_wf;
-    std::vector<uint32_t> ids[4];
+    std::vector<uint32_t> ids[HX_CP_CLASSES];
     std::vector<uint8_t> wf_class(W);
     for (uint32_t w = 0; w < W; ++w) {
         const size_t n = wf_node_start[w + 1] - wf_node_start[w], e = wf_edge_start[w + 1] - wf_edge_start[w];
         const size_t nlev = wf_seg_start[w + 1] - wf_seg_start[w] - 1;
         const size_t need = 4 * (3 * n + 1) + 4 * (nlev + 1) + 2 * e + 16;
-        const int k = (n > 65535) ? 3 : need <= kWarpSmall ? 0 : need <= kWarpBig ? 1 : need <= kBlock ? 2 : 3;
+        const int k = hx_cpath_class_of(need, n);
         ids[k].push_back(w);
         wf_class[w] = (uint8_t)k;
     }
@@ -419,7 +417,7 @@ int hx_dag_upload(hx_cluster* h, const uint32_t* row_ptr, const uint32_t* col_id
     std::vector<float> el(workflow_elapsed_s, workflow_elapsed_s + W);
     HX_TRY(dev_upload(h->dag_allocs, &h->d_node_wf, nwf), "upload node_workflow");
     HX_TRY(dev_upload(h->dag_allocs, &h->d_elapsed, el), "upload elapsed");
-    for (int k = 0; k < 4; ++k) {
+    for (int k = 0; k < HX_CP_CLASSES; ++k) {
         if (ids[k].empty()) continue;
         uint32_t* d_ids;
         HX_TRY(dev_upload(h->dag_allocs, &d_ids, ids[k]), "upload workflow classes");
@@ -429,7 +427,7 @@ int hx_dag_upload(hx_cluster* h, const uint32_t* row_ptr, const uint32_t* col_id
     }
     if (!h->fj.ready) {
         bool ok = cudaEventCreateWithFlags(&h->fj.fork, cudaEventDisableTiming) == cudaSuccess;
-        for (int i = 0; i < 3 && ok; ++i)
+        for (int i = 0; i < HX_CP_SIDE && ok; ++i)
             ok = cudaStreamCreateWithFlags(&h->fj.aux[i], cudaStreamNonBlocking) == cudaSuccess &&
                  cudaEventCreateWithFlags(&h->fj.join[i], cudaEventDisableTiming) == cudaSuccess;
         if (!ok) return fail(h, HX_ERR_CUDA, "creating the side streams of the horizon pass");
@@ -483,7 +481,7 @@ int hx_dag_update_costs(hx_cluster* h, const uint32_t* node_ids, const float* ne
     // the last value given for a node wins; the workflows touched are recomputed, nothing else
     std::vector<uint32_t> idx; std::vector<float> val;
     idx.reserve(n_updates); val.reserve(n_updates);
-    std::vector<uint32_t> dirty[4];
+    std::vector<uint32_t> dirty[HX_CP_CLASSES];
     {
         std::vector<uint32_t> order(n_updates);
         for (uint32_t i = 0; i < n_updates; ++i) order[i] = i;
@@ -515,7 +513,7 @@ int hx_dag_update_costs(hx_cluster* h, const uint32_t* node_ids, const float* ne
     HX_TRY(cudaMemcpyAsync(h->d_upd_cost, val.data(), val.size() * sizeof(float), cudaMemcpyHostToDevice, s), "copy updates");
     std::vector<HxCpClass> part;
     size_t off = 0;
-    for (int k = 0; k < 4; ++k) {
+    for (int k = 0; k < HX_CP_CLASSES; ++k) {
         if (dirty[k].empty()) continue;
         HX_TRY(cudaMemcpyAsync(h->d_upd_wf + off, dirty[k].data(), dirty[k].size() * sizeof(uint32_t),
                                cudaMemcpyHostToDevice, s), "copy dirty workflows");
