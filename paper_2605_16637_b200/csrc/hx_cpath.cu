@@ -19,15 +19,23 @@
 
 namespace {
 
-template <bool WARP>
+// GW = lanes of the group that owns one workflow: 8 (a quarter of a warp), 32 (a warp) or 0 (the
+// whole block).  Small workflows have one to eight nodes per level: with a quarter warp per workflow
+// a warp instruction serves four workflows instead of one.
+template <int GW>
+__device__ __forceinline__ unsigned group_mask() {
+    return GW == 8 ? 0xFFu << (threadIdx.x & 24) : 0xffffffffu;
+}
+template <int GW>
 __device__ __forceinline__ void group_sync() {
-    if (WARP) __syncwarp(); else __syncthreads();
+    if (GW == 0) __syncthreads(); else __syncwarp(group_mask<GW>());
 }
 
-template <bool WARP>
+template <int GW>
 __device__ __forceinline__ float group_max(float v, float* red, int t, int tpw) {
-    for (int off = 16; off > 0; off >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, off));
-    if (WARP) return v;
+    const unsigned mask = group_mask<GW>();
+    for (int off = (GW == 8 ? 4 : 16); off > 0; off >>= 1) v = fmaxf(v, __shfl_xor_sync(mask, v, off));
+    if (GW != 0) return v;
     __syncthreads();
     if ((t & 31) == 0) red[t >> 5] = v;
     __syncthreads();
@@ -37,7 +45,7 @@ __device__ __forceinline__ float group_max(float v, float* red, int t, int tpw) 
 }
 
 // One group per workflow, workflow slice staged in shared memory.
-template <bool WARP>
+template <int GW>
 __global__ void hx_cpath_staged_kernel(HxForestDev f, const uint32_t* __restrict__ wf_ids, uint32_t count,
                                        int tpw, int wfs_per_block, uint32_t smem_per_wf) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -74,7 +82,7 @@ __global__ void hx_cpath_staged_kernel(HxForestDev f, const uint32_t* __restrict
         for (uint32_t i = t; i < nw; i += tpw) cp4(reinterpret_cast<uint32_t*>(colW) + i, src + i);
     }
     asm volatile("cp.async.wait_all;" ::: "memory");
-    group_sync<WARP>();
+    group_sync<GW>();
 
     float hmax = 0.0f;
     for (uint32_t lev = 0; lev < nlev; ++lev) {
@@ -94,7 +102,7 @@ __global__ void hx_cpath_staged_kernel(HxForestDev f, const uint32_t* __restrict
             costS[i] = tl;
             hmax = fmaxf(hmax, c);
         }
-        group_sync<WARP>();
+        group_sync<GW>();
     }
     for (uint32_t i0 = t; i0 < n; i0 += 4 * tpw) {            // four node numbers in flight per thread
         uint32_t v[4];
@@ -106,7 +114,7 @@ __global__ void hx_cpath_staged_kernel(HxForestDev f, const uint32_t* __restrict
             if (i < n) { f.cp[v[u]] = cpS[i]; f.tail[v[u]] = costS[i]; }
         }
     }
-    hmax = group_max<WARP>(hmax, red, t, tpw);
+    hmax = group_max<GW>(hmax, red, t, tpw);
     if (t == 0) f.H[w] = hmax;
 }
 
@@ -188,21 +196,21 @@ cudaError_t hx_launch_cpath(const HxForestDev& f, const HxCpClass* classes, int 
             const int threads = c.threads_per_wf * c.wfs_per_block;
             const size_t smem = c.smem_per_wf * c.wfs_per_block;
             const unsigned grid = (c.count + c.wfs_per_block - 1) / c.wfs_per_block;
-            if (c.threads_per_wf == 32) {
-                {   // static + dynamic shared memory may exceed the 48 KB default
-                    static size_t allowed[64];
-                    cudaError_t e = hx_opt_in_smem(hx_cpath_staged_kernel<true>, smem, allowed, 40 * 1024);
-                    if (e != cudaSuccess) return e;
-                }
-                hx_cpath_staged_kernel<true><<<grid, threads, smem, s>>>(
+            cudaError_t e = cudaSuccess;
+            if (c.threads_per_wf == 8) {
+                static size_t allowed[64];
+                if ((e = hx_opt_in_smem(hx_cpath_staged_kernel<8>, smem, allowed, 40 * 1024)) != cudaSuccess) return e;
+                hx_cpath_staged_kernel<8><<<grid, threads, smem, s>>>(
+                    f, c.wf_ids, c.count, 8, c.wfs_per_block, (uint32_t)c.smem_per_wf);
+            } else if (c.threads_per_wf == 32) {
+                static size_t allowed[64];     // static + dynamic shared memory may exceed the 48 KB default
+                if ((e = hx_opt_in_smem(hx_cpath_staged_kernel<32>, smem, allowed, 40 * 1024)) != cudaSuccess) return e;
+                hx_cpath_staged_kernel<32><<<grid, threads, smem, s>>>(
                     f, c.wf_ids, c.count, 32, c.wfs_per_block, (uint32_t)c.smem_per_wf);
             } else {
-                {   // static + dynamic shared memory may exceed the 48 KB default
-                    static size_t allowed[64];
-                    cudaError_t e = hx_opt_in_smem(hx_cpath_staged_kernel<false>, smem, allowed, 40 * 1024);
-                    if (e != cudaSuccess) return e;
-                }
-                hx_cpath_staged_kernel<false><<<grid, threads, smem, s>>>(
+                static size_t allowed[64];
+                if ((e = hx_opt_in_smem(hx_cpath_staged_kernel<0>, smem, allowed, 40 * 1024)) != cudaSuccess) return e;
+                hx_cpath_staged_kernel<0><<<grid, threads, smem, s>>>(
                     f, c.wf_ids, c.count, c.threads_per_wf, 1, (uint32_t)c.smem_per_wf);
             }
         }

@@ -151,8 +151,8 @@ struct HxCpClass {
     size_t smem_per_wf;        // bytes of staging per workflow, 0 = work in global memory
 };
 
-#define HX_CP_CLASSES 5      // workflow classes of the horizon pass
-#define HX_CP_SIDE 4         // side streams: every class after the first
+#define HX_CP_CLASSES 6      // workflow classes of the horizon pass
+#define HX_CP_SIDE 5         // side streams: every class after the first
 
 // Side streams and events for running the independent workflow classes of one horizon pass
 // next to each other (fork from / join into the caller's stream).  Zero-initialised = serial.
@@ -165,13 +165,13 @@ struct HxForkJoin {
 cudaError_t hx_launch_cpath(const HxForestDev& f, const HxCpClass* classes, int n_classes,
                             cudaStream_t stream, long long* launches, const HxForkJoin* fj = nullptr);
 
-// Launch shape of workflow class k, by staging footprint: 0 = one warp, <= 3 KB, 16 per block;
-// 1 = one warp, <= 12 KB, 8 per block; 2 = one warp, <= 48 KB, 2 per block (blocks of 96 KB or less
-// can share an SM with blocks of other classes); 3 = one block, <= 200 KB; 4 = one block working in
-// global memory.
+// Launch shape of workflow class k, by staging footprint: 0 = a quarter warp, <= 768 B, 64 per block;
+// 1 = one warp, <= 3 KB, 16 per block; 2 = one warp, <= 12 KB, 8 per block; 3 = one warp, <= 48 KB, 2 per
+// block (blocks of 96 KB or less can share an SM with blocks of other classes); 4 = one block,
+// <= 200 KB; 5 = one block working in global memory.
 inline HxCpClass hx_cpath_class_shape(int k) {
-    const int tpw[HX_CP_CLASSES] = {32, 32, 32, 256, 256}, per_block[HX_CP_CLASSES] = {16, 8, 2, 1, 1};
-    const size_t sm[HX_CP_CLASSES] = {3072, 12288, 49152, 200 * 1024, 0};
+    const int tpw[HX_CP_CLASSES] = {8, 32, 32, 32, 256, 256}, per_block[HX_CP_CLASSES] = {64, 16, 8, 2, 1, 1};
+    const size_t sm[HX_CP_CLASSES] = {768, 3072, 12288, 49152, 200 * 1024, 0};
     return HxCpClass{nullptr, 0, tpw[k], per_block[k], sm[k]};
 }
 inline int hx_cpath_class_of(size_t need_bytes, size_t n_nodes) {
