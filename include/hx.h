@@ -198,6 +198,17 @@ int hx_schedule_batch(hx_cluster* h, const hx_call* calls, int n_calls,
 int hx_schedule_batch_host(hx_cluster* h, const hx_call* calls, int n_calls,
                            int32_t* out_assign, float* out_cost, void* stream);
 
+/* The same without the final synchronisation: the copies and kernels are only
+ * enqueued on `stream`, and out_assign / out_cost hold the results once the
+ * stream has reached the end of this call's work.  For successive ready batches
+ * whose loads depend on one another (the commits of one batch are the snapshot
+ * of the next) this lets the caller enqueue all of them and synchronise once.
+ * calls, out_assign and out_cost must be page-locked host memory and stay alive
+ * and untouched until then; the device staging buffers are shared by all calls
+ * on the handle, so use one stream per handle. */
+int hx_schedule_batch_host_async(hx_cluster* h, const hx_call* calls, int n_calls,
+                                 int32_t* out_assign, float* out_cost, void* stream);
+
 /* hx_schedule_batch for callers that must not allocate.  (The paper has no
  * counterpart: this entry point exists only because of how the library is
  * embedded.)  hx_schedule_batch with topk > 0 obtains its intermediate buffers

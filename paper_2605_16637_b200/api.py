@@ -58,6 +58,7 @@ def _load():
         "hx_set_options": [vp, C.POINTER(_Options)],
         "hx_schedule_batch": [vp, vp, ci, vp, vp, vp],
         "hx_schedule_batch_host": [vp, vp, ci, vp, vp, vp],
+        "hx_schedule_batch_host_async": [vp, vp, ci, vp, vp, vp],
         "hx_schedule_batch_static": [vp, vp, ci, vp, vp, vp],
         "hx_schedule_greedy": [vp, vp, ci, vp, vp, vp, vp],
         "hx_decode_set_running": [vp, vp, vp, vp],
@@ -208,6 +209,16 @@ def hx_schedule_batch_host(h, calls, out_assign=None, out_cost=None, stream=0):
         out_cost = np.empty(n, np.float32)
     _check(_lib.hx_schedule_batch_host(h, _p(calls), n, _p(out_assign), _p(out_cost), stream), h)
     return out_assign, out_cost
+
+
+def hx_schedule_batch_host_async(h, calls, out_assign, out_cost, stream=0):
+    """Enqueue only: calls / out_assign / out_cost are numpy views of page-locked memory that the
+    caller keeps alive until the stream has been synchronised."""
+    if calls.dtype != CALL_DTYPE or out_assign.dtype != np.int32 or out_cost.dtype != np.float32:
+        raise HxError(-1, "hx_schedule_batch_host_async takes CALL_DTYPE, int32 and float32 arrays as they are")
+    if not (calls.flags.c_contiguous and out_assign.flags.c_contiguous and out_cost.flags.c_contiguous):
+        raise HxError(-1, "hx_schedule_batch_host_async needs contiguous arrays")
+    _check(_lib.hx_schedule_batch_host_async(h, _p(calls), calls.shape[0], _p(out_assign), _p(out_cost), stream), h)
 
 
 def hx_get_topk(h):

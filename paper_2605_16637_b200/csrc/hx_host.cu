@@ -587,8 +587,8 @@ int hx_schedule_batch(hx_cluster* h, const hx_call* calls, int n_calls, int32_t*
     return HX_OK;
 }
 
-int hx_schedule_batch_host(hx_cluster* h, const hx_call* calls, int n_calls, int32_t* out_assign,
-                           float* out_cost, void* stream) {
+static int schedule_batch_host_impl(hx_cluster* h, const hx_call* calls, int n_calls, int32_t* out_assign,
+                                    float* out_cost, void* stream, bool sync) {
     if (!h) return HX_ERR_INVALID_ARG;
     if (n_calls < 0) return fail(h, HX_ERR_INVALID_ARG, "negative n_calls");
     if (n_calls == 0) return HX_OK;
@@ -612,8 +612,18 @@ int hx_schedule_batch_host(hx_cluster* h, const hx_call* calls, int n_calls, int
     if (rc != HX_OK) return rc;
     HX_TRY(cudaMemcpyAsync(out_assign, h->st_assign, (size_t)n_calls * sizeof(int32_t), cudaMemcpyDeviceToHost, s), "copy assign");
     HX_TRY(cudaMemcpyAsync(out_cost, h->st_cost, (size_t)n_calls * sizeof(float), cudaMemcpyDeviceToHost, s), "copy cost");
-    HX_TRY(cudaStreamSynchronize(s), "cudaStreamSynchronize");
+    if (sync) HX_TRY(cudaStreamSynchronize(s), "cudaStreamSynchronize");
     return HX_OK;
+}
+
+int hx_schedule_batch_host(hx_cluster* h, const hx_call* calls, int n_calls, int32_t* out_assign,
+                           float* out_cost, void* stream) {
+    return schedule_batch_host_impl(h, calls, n_calls, out_assign, out_cost, stream, true);
+}
+
+int hx_schedule_batch_host_async(hx_cluster* h, const hx_call* calls, int n_calls, int32_t* out_assign,
+                                 float* out_cost, void* stream) {
+    return schedule_batch_host_impl(h, calls, n_calls, out_assign, out_cost, stream, false);
 }
 
 

@@ -344,6 +344,38 @@ def test_host_buffer_entry_point_matches_device_path(hx, oracle):
     gc.close()
 
 
+def test_async_host_entry_point_chains_dependent_batches(hx, oracle):
+    """Four ready batches whose commits feed the next one, enqueued from page-locked memory without a
+    synchronisation in between, equal the same batches run one by one through the device entry point."""
+    import torch
+    wl = make_workload("sweep", scale=1 / 32)
+    oc, gc, dag = _prepare(hx, oracle, wl)
+    gc.set_options(score_mode=hx.HX_MODE_RATIO, topk=4, commit=1, alpha=wl.alpha)
+    n = len(wl.calls) // 4
+    qP0, free0 = wl.load_s[:wl.P].copy(), wl.kv_free[wl.P:].copy()
+    want = []
+    for i in range(4):
+        a, c = gc.schedule_batch(wl.calls[i * n:(i + 1) * n])
+        want.append((a.cpu().numpy(), c.cpu().numpy()))
+    loads_want = gc.read_loads()
+    gc.update_loads(qP=qP0, kv_free=free0)
+    calls_pin = torch.from_numpy(wl.calls[:4 * n].view(np.uint8).reshape(-1, 16).copy()).pin_memory()
+    a_pin = torch.empty(4 * n, dtype=torch.int32).pin_memory()
+    c_pin = torch.empty(4 * n, dtype=torch.float32).pin_memory()
+    cn = calls_pin.numpy().view(hx.CALL_DTYPE).reshape(-1)
+    sp = torch.cuda.current_stream().cuda_stream
+    for i in range(4):
+        hx.hx_schedule_batch_host_async(gc.h, cn[i * n:(i + 1) * n], a_pin.numpy()[i * n:(i + 1) * n],
+                                        c_pin.numpy()[i * n:(i + 1) * n], sp)
+    torch.cuda.current_stream().synchronize()
+    for i in range(4):
+        assert np.array_equal(a_pin.numpy()[i * n:(i + 1) * n], want[i][0])
+        assert np.array_equal(c_pin.numpy()[i * n:(i + 1) * n], want[i][1])
+    for x, y in zip(gc.read_loads(), loads_want):
+        assert np.array_equal(x, y)
+    gc.close()
+
+
 def test_runs_are_deterministic(hx, oracle):
     wl = make_workload("sweep", scale=1 / 32)
     outs = []
