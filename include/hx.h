@@ -140,7 +140,10 @@ int hx_dag_upload(hx_cluster* h, const uint32_t* row_ptr, const uint32_t* col_id
  * horizon update): for every node cp = cost + tail, tail = max over successors
  * of cp (0 for sinks); H[w] = max over the workflow's nodes of cp.  Each sum
  * runs from the sink towards the source, so results do not depend on the
- * traversal order.  Enqueues on `stream`. */
+ * traversal order.  Enqueues on `stream`; independent groups of workflows may
+ * run on side streams owned by the handle that fork from `stream` and join it
+ * again with events before the call returns, so later work on `stream` sees
+ * the results. */
 int hx_critical_path(hx_cluster* h, void* stream);
 
 /* Online horizon refinement (Section 5.1, "Define online workflow horizon": the
