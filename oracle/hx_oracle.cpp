@@ -57,6 +57,7 @@ struct OrcCluster {
     const float* flops_per_token;   // [M]
     const float* weight_bytes;      // [M]
     const float* kv_bytes_per_token;// [M]
+    const float* attn_flops_per_token2;   // [M] or NULL: attention FLOPs per pair of prompt tokens (prefill variant)
 };
 
 struct OrcCall { uint32_t node, model; float prompt_tokens, output_tokens; };
@@ -88,6 +89,7 @@ void latency_terms(const OrcCluster& cl, const OrcCall& c, Terms& t) {
     const float phi = cl.flops_per_token[c.model];
     const float omega = cl.weight_bytes[c.model];
     const float kappa = cl.kv_bytes_per_token[c.model];
+    const float psi = cl.attn_flops_per_token2 ? cl.attn_flops_per_token2[c.model] : 0.0f;
     t.kvB = n * kappa;                                  // KV bytes of the prompt
     t.m = n + o;                                        // Eq. 3
     t.tpre.resize(cl.G);
@@ -97,7 +99,9 @@ void latency_terms(const OrcCluster& cl, const OrcCall& c, Terms& t) {
     for (int g = 0; g < cl.G; ++g) {
         const float invF = 1.0f / (cl.peak_tflops[g] * 1e12f);
         const float invB = 1.0f / (cl.hbm_tbps[g] * 1e12f);
-        const float pf = (n * phi) * invF;
+        // variant with a quadratic attention term: prefill FLOPs = n * phi + n * n * psi (psi = 0 without it)
+        const float flops = std::fmaf(n * psi, n, n * phi);         // exactly n * phi when psi = 0
+        const float pf = flops * invF;
         const float pm = (omega + t.kvB) * invB;
         t.tpre[g] = std::fmax(pf, pm);
         t.tdec[g] = (o * step) * invB;
@@ -449,7 +453,8 @@ int orc_fin_all_f64(const OrcCluster* cl, const OrcCall* calls, int C, int flags
                 const double L = cl->link_gbps[(size_t)p * cl->D + d] * 1e9;
                 const double qp = (flags & ORC_FLAG_UNLOADED) ? 0.0 : cl->qP[p];
                 const double qd = (flags & ORC_FLAG_UNLOADED) ? 0.0 : cl->qD[d];
-                const double tpre = std::max(n * phi / F, (omega + n * kappa) / Bp);
+                const double psi = cl->attn_flops_per_token2 ? cl->attn_flops_per_token2[calls[c].model] : 0.0;
+                const double tpre = std::max((n * phi + n * n * psi) / F, (omega + n * kappa) / Bp);
                 const double tdec = o * (omega + kappa * (n + 0.5 * (o - 1.0))) / Bd;
                 const double ready = qp + tpre + n * kappa / L;
                 const double start = std::max(ready, qd);

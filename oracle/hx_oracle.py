@@ -43,7 +43,7 @@ class _Cluster(C.Structure):
                 ("qP", C.c_void_p), ("qD", C.c_void_p), ("capD", C.c_void_p),
                 ("link_gbps", C.c_void_p),
                 ("flops_per_token", C.c_void_p), ("weight_bytes", C.c_void_p),
-                ("kv_bytes_per_token", C.c_void_p)]
+                ("kv_bytes_per_token", C.c_void_p), ("attn_flops_per_token2", C.c_void_p)]
 
 
 class _Dag(C.Structure):
@@ -83,6 +83,11 @@ class Cluster:
         self.link = _f32(link_pd_gbps).reshape(self.P, self.D)
         self.phi = _f32(models[:, 0]); self.omega = _f32(models[:, 1]); self.kappa = _f32(models[:, 2])
         self.G, self.M = self.tflops.shape[0], self.phi.shape[0]
+        self.psi = None                 # optional attention FLOPs per token pair, one per model (set_attention)
+
+    def set_attention(self, psi):
+        self.psi = _f32(psi)
+        assert self.psi.shape[0] == self.M
 
     @classmethod
     def from_workload(cls, wl):
@@ -94,7 +99,7 @@ class Cluster:
         return _Cluster(self.G, self.P, self.D, self.M, _ptr(self.tflops), _ptr(self.tbps),
                         _ptr(self.typeP), _ptr(self.typeD), _ptr(self.qP), _ptr(self.qD),
                         _ptr(self.capD), _ptr(self.link), _ptr(self.phi), _ptr(self.omega),
-                        _ptr(self.kappa))
+                        _ptr(self.kappa), None if self.psi is None else _ptr(self.psi))
 
 
 class Oracle:

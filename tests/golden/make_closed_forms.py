@@ -23,11 +23,12 @@ from fractions import Fraction as Fr
 
 
 def terms(types, model, n, o):
-    phi, omega, kappa = (Fr(x) for x in model)
+    phi, omega, kappa = (Fr(x) for x in model[:3])
+    psi = Fr(model[3]) if len(model) > 3 else Fr(0)      # attention FLOPs per pair of prompt tokens (variant)
     out = []
     for tflops, tbps in types:
         F, B = Fr(tflops) * 10**12, Fr(tbps) * 10**12
-        pf = Fr(n) * phi / F
+        pf = (Fr(n) * phi + Fr(n) * Fr(n) * psi) / F
         pm = (omega + Fr(n) * kappa) / B
         tdec = Fr(o) * (omega + kappa * (Fr(n) + Fr(o - 1) / 2)) / B
         out.append(dict(pf=pf, pm=pm, tpre=max(pf, pm), tdec=tdec))
@@ -56,7 +57,8 @@ def case(name, types, model, n, o, typeP, typeD, qP, qD, capD, bw, elapsed, tail
                    ratio_eq2=float((Fr(elapsed) + best) / Fr(H)),
                    slack=float(Fr(alpha) * Fr(H) - comp))
     return dict(name=name, note=note,
-                inputs=dict(gpu_types=[[float(a), float(b)] for a, b in types], model=[float(x) for x in model],
+                inputs=dict(gpu_types=[[float(a), float(b)] for a, b in types], model=[float(x) for x in model[:3]],
+                            attn_flops_per_token2=float(model[3]) if len(model) > 3 else 0.0,
                             prompt_tokens=n, output_tokens=o, typeP=typeP, typeD=typeD,
                             qP=[float(x) for x in qP], qD=[float(x) for x in qD], capD=capD, link_gbps=bw,
                             elapsed=float(elapsed), tail=float(tail), H=float(H), alpha=float(alpha)),
@@ -81,6 +83,10 @@ def main():
              [0], [0, 5], [1010, 1011], [[100, 100]], 1, 0, 2, Fr(3, 2),
              "demand 1011 tokens: instance 0 (capacity 1010) is infeasible by Eq. 4, instance 1 "
              "(capacity 1011, equality allowed) is taken although it admits five seconds later"),
+        case("quadratic_prefill", [(1000, Fr(1))], (2 * 10**9, 10**9, 10**5, 4 * 10**5), 8000, 11, [0], [0],
+             [0], [0], [10**6], [[100]], 0, 0, 1, Fr(3, 2),
+             "prefill variant with a quadratic attention term: 8000 tokens, 4e5 FLOPs per token pair: "
+             "compute = (8000*2e9 + 8000^2*4e5)/1e15 = 0.016 + 0.0256 = 0.0416 s, above the memory term 0.0018 s"),
         case("all_infeasible", [(1000, Fr(1))], (2 * 10**9, 10**9, 10**5), 1000, 11, [0], [0],
              [0], [0], [100], [[100]], 0, 0, 1, Fr(3, 2),
              "no decode instance can hold the call: assignment -1"),

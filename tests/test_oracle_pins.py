@@ -29,6 +29,8 @@ def _golden_case(c):
     i = c["inputs"]
     cl = ho.Cluster(i["gpu_types"], i["typeP"], i["typeD"], i["qP"], i["qD"], i["capD"],
                     i["link_gbps"], [i["model"]])
+    if i.get("attn_flops_per_token2"):
+        cl.set_attention([i["attn_flops_per_token2"]])       # prefill variant with a quadratic attention term
     calls = _calls([(0, 0, i["prompt_tokens"], i["output_tokens"])])
     dag = ho.DagResult(cp=None, tail=np.array([i["tail"]], np.float32), H=np.array([i["H"]], np.float32))
     return cl, calls, dag, i
@@ -402,3 +404,27 @@ def test_cost_change_stays_inside_its_workflow_and_is_monotone(oracle):
     assert np.array_equal(new.H[keep], base.H[keep])
     assert np.all(new.cp >= base.cp) and np.all(new.H >= base.H)
     assert new.tail[v] == base.tail[v] and new.cp[v] == np.float32(up[v] + base.tail[v])
+
+
+def test_quadratic_prefill_variant(oracle):
+    """psi = 0 is the linear model bit for bit; psi > 0 only lengthens the prefill, by n^2 * psi / F on a
+    compute-bound class, and leaves decode time, demand and transfer alone."""
+    rng = np.random.default_rng(41)
+    cl = _random_cluster(rng, 3, 3)
+    calls = _random_calls(rng, 50)
+    base = oracle.fin_all(cl, calls)
+    t0 = oracle.terms(cl, calls)
+    cl.set_attention(np.zeros(cl.M, np.float32))
+    assert np.array_equal(oracle.fin_all(cl, calls), base)
+    psi = np.array([3e5, 7e5], np.float32)
+    cl.set_attention(psi)
+    t1 = oracle.terms(cl, calls)
+    assert np.array_equal(t1[1], t0[1]) and np.array_equal(t1[2], t0[2]) and np.array_equal(t1[3], t0[3])
+    assert np.all(t1[0] >= t0[0]) and np.all(oracle.fin_all(cl, calls) >= base)
+    n = calls["prompt_tokens"].astype(np.float64)
+    F = cl.tflops.astype(np.float64) * 1e12
+    B = cl.tbps.astype(np.float64) * 1e12
+    phi, om, ka = (x.astype(np.float64)[calls["model"]] for x in (cl.phi, cl.omega, cl.kappa))
+    want = np.maximum((n * phi + n * n * psi.astype(np.float64)[calls["model"]])[:, None] / F[None, :],
+                      (om + n * ka)[:, None] / B[None, :])
+    assert np.max(np.abs(t1[0] - want) / want) < 1e-6
