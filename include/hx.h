@@ -172,6 +172,15 @@ int hx_dag_update_elapsed(hx_cluster* h, const float* workflow_elapsed_s, void* 
  * Any of the three output arguments may be NULL. */
 int hx_get_dag_results(hx_cluster* h, const float** cp, const float** tail, const float** H);
 
+/* Prefill variant with a quadratic attention term (the roofline-style estimate of
+ * Section 4.2 leaves the shape of the compute term open): with per_model[m] =
+ * attention FLOPs per pair of prompt tokens of model m, the compute time of a
+ * prefill becomes (n * flops_per_token + n * n * per_model[m]) / peak instead of
+ * n * flops_per_token / peak.  per_model: host, n_models values, finite and
+ * >= 0; all zero (the state after hx_cluster_create) is the linear model bit for
+ * bit.  Takes effect for every later scoring, greedy and stand-alone-cost call. */
+int hx_set_attention_flops(hx_cluster* h, const float* per_model);
+
 /* Validates and stores the options used by later hx_schedule_batch calls. */
 int hx_set_options(hx_cluster* h, const hx_options* opts);
 

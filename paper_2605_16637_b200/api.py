@@ -56,6 +56,7 @@ def _load():
         "hx_dag_update_elapsed": [vp, vp, vp],
         "hx_get_dag_results": [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp)],
         "hx_set_options": [vp, C.POINTER(_Options)],
+        "hx_set_attention_flops": [vp, vp],
         "hx_schedule_batch": [vp, vp, ci, vp, vp, vp],
         "hx_schedule_batch_host": [vp, vp, ci, vp, vp, vp],
         "hx_schedule_batch_host_async": [vp, vp, ci, vp, vp, vp],
@@ -163,6 +164,12 @@ def hx_get_dag_results(h):
 def hx_set_options(h, score_mode=HX_MODE_COMPLETION, topk=0, commit=0, flags=0, alpha=1.5):
     o = _Options(int(score_mode), int(topk), int(commit), int(flags), float(alpha))
     _check(_lib.hx_set_options(h, C.byref(o)), h)
+
+
+def hx_set_attention_flops(h, per_model):
+    """Attention FLOPs per pair of prompt tokens, one value per model (quadratic prefill variant)."""
+    a = _np(per_model, np.float32)
+    _check(_lib.hx_set_attention_flops(h, _p(a)), h)
 
 
 def hx_schedule_batch(h, calls_ptr, n_calls, out_assign_ptr, out_cost_ptr, stream=0):
@@ -281,6 +288,7 @@ class Cluster:
         inst = _np(instances, INSTANCE_DTYPE)
         self.P = int((inst["role"] == 0).sum())
         self.D = int(inst.shape[0] - self.P)
+        self.M = int(_np(models, np.float32).reshape(-1, 3).shape[0])
         self.n_nodes = 0
         self.n_workflows = 0
         self.topk = 0
@@ -334,6 +342,12 @@ class Cluster:
     def set_options(self, score_mode=HX_MODE_COMPLETION, topk=0, commit=0, flags=0, alpha=1.5):
         hx_set_options(self.h, score_mode, topk, commit, flags, alpha)
         self.topk = int(topk)
+
+    def set_attention_flops(self, per_model):
+        a = _np(per_model, np.float32)
+        if a.shape[0] != self.M:
+            raise HxError(-1, "one value per model is needed")
+        hx_set_attention_flops(self.h, a)
 
     def schedule_batch(self, calls, out_assign=None, out_cost=None):
         """calls: CUDA tensor holding n records of 16 bytes, or a numpy CALL_DTYPE array

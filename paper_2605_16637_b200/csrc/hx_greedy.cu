@@ -125,7 +125,7 @@ __global__ void __launch_bounds__(kThreads, 1) hx_greedy_kernel(const __grid_con
             const float m = __fadd_rn(nt, ot);
             if (lane < G) {
                 const float iF = prm.ct.invF[lane], iB = prm.ct.invB[lane];
-                tpre[lane] = fmaxf(__fmul_rn(__fmul_rn(nt, phi), iF), __fmul_rn(__fadd_rn(omega, kvB), iB));
+                tpre[lane] = fmaxf(__fmul_rn(__fmaf_rn(__fmul_rn(nt, prm.ct.psi[mdl]), nt, __fmul_rn(nt, phi)), iF), __fmul_rn(__fadd_rn(omega, kvB), iB));
                 tdec[lane] = __fmul_rn(__fmul_rn(ot, step), iB);
             }
             __syncwarp();
@@ -209,7 +209,7 @@ __global__ void __launch_bounds__(kThreads, 1) hx_greedy_kernel(const __grid_con
                 const float phi = prm.ct.phi[mdl], omega = prm.ct.omega[mdl], kappa = prm.ct.kappa[mdl];
                 const float kvB = __fmul_rn(nt, kappa);
                 const int g = typePs[p];
-                const float tp = fmaxf(__fmul_rn(__fmul_rn(nt, phi), prm.ct.invF[g]), __fmul_rn(__fadd_rn(omega, kvB), prm.ct.invB[g]));
+                const float tp = fmaxf(__fmul_rn(__fmaf_rn(__fmul_rn(nt, prm.ct.psi[mdl]), nt, __fmul_rn(nt, phi)), prm.ct.invF[g]), __fmul_rn(__fadd_rn(omega, kvB), prm.ct.invB[g]));
                 const float m = __fadd_rn(nt, ot);
                 prm.out_assign[rc] = p * D + d;
                 prm.out_ratio[rc] = rv;

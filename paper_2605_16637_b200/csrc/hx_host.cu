@@ -542,6 +542,15 @@ int hx_get_dag_results(hx_cluster* h, const float** cp, const float** tail, cons
     return HX_OK;
 }
 
+int hx_set_attention_flops(hx_cluster* h, const float* per_model) {
+    if (!h) return HX_ERR_INVALID_ARG;
+    if (!per_model) return fail(h, HX_ERR_INVALID_ARG, "NULL array");
+    for (int m = 0; m < h->M; ++m)
+        if (!good_load(per_model[m])) return fail(h, HX_ERR_INVALID_ARG, "attention FLOPs must be finite and >= 0");
+    for (int m = 0; m < h->M; ++m) h->ctab.psi[m] = per_model[m];     // travels with the kernel parameters
+    return HX_OK;
+}
+
 int hx_set_options(hx_cluster* h, const hx_options* o) {
     if (!h || !o) return HX_ERR_INVALID_ARG;
     if (o->score_mode < HX_MODE_COMPLETION || o->score_mode > HX_MODE_RATIO) return fail(h, HX_ERR_INVALID_ARG, "unknown score mode");

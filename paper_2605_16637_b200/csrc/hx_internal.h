@@ -38,6 +38,7 @@ struct HxTables {
 struct HxConstTables {
     float invF[HX_MAX_TYPES], invB[HX_MAX_TYPES];
     float phi[HX_MAX_MODELS], omega[HX_MAX_MODELS], kappa[HX_MAX_MODELS];
+    float psi[HX_MAX_MODELS];       // attention FLOPs per pair of prompt tokens (0 = linear prefill model)
 };
 
 // Thread-tile shape of the scoring kernel as a function of the decode pool: LD lanes of a warp

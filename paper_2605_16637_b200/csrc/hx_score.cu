@@ -277,20 +277,21 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
         int k_it = 0;
         for (int idx = tid; idx < TCB * G; idx += nthr, ++k_it) {
             const int c = idx / G, g = idx - c * G;
-            float n = 1.f, o = 1.f, phi = 0.f, omega = 0.f, kappa = 0.f;
+            float n = 1.f, o = 1.f, phi = 0.f, omega = 0.f, kappa = 0.f, psi = 0.f;
             if (c < nvalid) {
                 uint4 raw;
                 if (tile == (int)blockIdx.x && k_it < 2) raw = k_it == 0 ? pre[0] : pre[1];
                 else raw = __ldg(reinterpret_cast<const uint4*>(prm.s.calls) + c0 + c);
                 if (g == 0) nodeS[c] = raw.x;
                 n = __uint_as_float(raw.z); o = __uint_as_float(raw.w);
-                if (raw.y < (unsigned)T.M) { phi = prm.ct.phi[raw.y]; omega = prm.ct.omega[raw.y]; kappa = prm.ct.kappa[raw.y]; }
+                if (raw.y < (unsigned)T.M) { phi = prm.ct.phi[raw.y]; omega = prm.ct.omega[raw.y]; kappa = prm.ct.kappa[raw.y]; psi = prm.ct.psi[raw.y]; }
             }
             const float kvB = __fmul_rn(n, kappa);
             const float ctx = __fmaf_rn(0.5f, __fsub_rn(o, 1.0f), n);
             const float step = __fmaf_rn(kappa, ctx, omega);
             const float iF = prm.ct.invF[g], iB = prm.ct.invB[g];
-            tpres[g * TCB + c] = fmaxf(__fmul_rn(__fmul_rn(n, phi), iF), __fmul_rn(__fadd_rn(omega, kvB), iB));
+            const float flops = __fmaf_rn(__fmul_rn(n, psi), n, __fmul_rn(n, phi));   // exactly n * phi when psi = 0
+            tpres[g * TCB + c] = fmaxf(__fmul_rn(flops, iF), __fmul_rn(__fadd_rn(omega, kvB), iB));
             tdecs[g * TCB + c] = __fmul_rn(__fmul_rn(o, step), iB);
             if (g == 0) { kvBs[c] = kvB; mtoks[c] = __fadd_rn(n, o); }
         }

@@ -376,6 +376,38 @@ def test_async_host_entry_point_chains_dependent_batches(hx, oracle):
     gc.close()
 
 
+@pytest.mark.parametrize("P, D, n", [(4, 9, 300), (70, 130, 700)])
+def test_quadratic_prefill_variant(hx, oracle, P, D, n):
+    """Attention FLOPs per token pair set on both sides: scoring, top-K lists and the greedy planner agree
+    bit for bit; with zeros the results are those of the linear model."""
+    gc, oc = _cluster_pair(hx, P, D, seed=P + D)
+    calls = _calls(n, seed=P)
+    gc.set_options(flags=hx.HX_FLAG_NO_DAG)
+    base_a, base_c = (x.cpu().numpy() for x in gc.schedule_batch(calls))
+    gc.set_attention_flops([0.0, 0.0])
+    a, c = (x.cpu().numpy() for x in gc.schedule_batch(calls))
+    assert np.array_equal(a, base_a) and np.array_equal(c, base_c)
+    psi = np.array([2.5e5, 9e5], np.float32)
+    gc.set_attention_flops(psi)
+    oc.set_attention(psi)
+    a, c = (x.cpu().numpy() for x in gc.schedule_batch(calls))
+    oa, ocost, _ = oracle.schedule(oc, calls)
+    assert np.array_equal(a, oa) and np.array_equal(c, ocost) and np.all(c >= base_c) and (c > base_c).any()
+    gc.set_options(topk=3, flags=hx.HX_FLAG_NO_DAG)
+    gc.schedule_batch(calls)
+    pair, cost, prio = gc.topk_results(n)
+    op, ocs, opr, _, _ = oracle.topk(oc, calls, 3)
+    assert np.array_equal(pair, op) and np.array_equal(cost, ocs) and np.array_equal(prio, opr)
+    gc.set_options(score_mode=hx.HX_MODE_RATIO, flags=hx.HX_FLAG_NO_DAG, commit=0)
+    m = min(n, 200)
+    ga, gr, go = (x.cpu().numpy() for x in gc.schedule_greedy(calls[:m]))
+    ea, er, eo, _, _, _ = oracle.greedy(oc, calls[:m], np.full(D, 1e6, np.float32))
+    assert np.array_equal(ga, ea) and np.array_equal(gr, er) and np.array_equal(go, eo)
+    with pytest.raises(hx.HxError):
+        gc.set_attention_flops([-1.0, 0.0])
+    gc.close()
+
+
 def test_runs_are_deterministic(hx, oracle):
     wl = make_workload("sweep", scale=1 / 32)
     outs = []
