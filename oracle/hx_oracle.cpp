@@ -437,6 +437,33 @@ int orc_longest_path(const uint32_t* row_ptr, const uint32_t* col, const float* 
     return 0;
 }
 
+// Earliest start and finish of every node when each node takes its cost and
+// starts as soon as all its predecessors have finished (Section 4.1: a node is
+// ready when all predecessors have completed):
+//   est[v] = max over predecessors u of eft[u]   (0 without predecessors)
+//   eft[v] = est[v] + cost[v]
+// Nodes are visited in topological order (Kahn) and each finished node pushes
+// its finish time to its successors, so every sum runs from the source towards
+// the sink.  Returns -1 if the graph has a cycle.
+int orc_earliest_start(const uint32_t* row_ptr, const uint32_t* col, const float* cost,
+                       uint32_t N, float* est, float* eft) {
+    std::vector<uint32_t> indeg(N, 0), ready;
+    ready.reserve(N);
+    for (uint32_t v = 0; v < N; ++v)
+        for (uint32_t e = row_ptr[v]; e < row_ptr[v + 1]; ++e) ++indeg[col[e]];
+    for (uint32_t v = 0; v < N; ++v) { est[v] = 0.0f; if (indeg[v] == 0) ready.push_back(v); }
+    for (size_t i = 0; i < ready.size(); ++i) {
+        const uint32_t v = ready[i];
+        eft[v] = est[v] + cost[v];
+        for (uint32_t e = row_ptr[v]; e < row_ptr[v + 1]; ++e) {
+            const uint32_t u = col[e];
+            est[u] = std::fmax(est[u], eft[v]);
+            if (--indeg[u] == 0) ready.push_back(u);
+        }
+    }
+    return ready.size() == N ? 0 : -1;
+}
+
 // Double-precision twin of orc_fin_all in textbook form (units converted first,
 // plain divisions), to measure the rounding error of the binary32 sequence.
 int orc_fin_all_f64(const OrcCluster* cl, const OrcCall* calls, int C, int flags, double* fin) {

@@ -119,6 +119,16 @@ class Oracle:
             raise ValueError("graph has a cycle")
         return DagResult(cp, tail, H)
 
+    def earliest_start(self, row_ptr, col, cost):
+        """est, eft of every node (forward pass over the same DAG)."""
+        row_ptr, col, cost = _u32(row_ptr), _u32(col), _f32(cost)
+        N = cost.shape[0]
+        est = np.zeros(N, np.float32); eft = np.zeros(N, np.float32)
+        rc = self.lib.orc_earliest_start(_ptr(row_ptr), _ptr(col), _ptr(cost), C.c_uint32(N), _ptr(est), _ptr(eft))
+        if rc != 0:
+            raise ValueError("graph has a cycle")
+        return est, eft
+
     # -- scoring ----------------------------------------------------------
     @staticmethod
     def _calls(calls):
