@@ -172,6 +172,24 @@ int hx_dag_update_elapsed(hx_cluster* h, const float* workflow_elapsed_s, void* 
  * Any of the three output arguments may be NULL. */
 int hx_get_dag_results(hx_cluster* h, const float** cp, const float** tail, const float** H);
 
+/* Forward pass over the same forest (Section 4.1: a node becomes ready when
+ * all its predecessors have completed): for every node v
+ *   est[v] = max over predecessors u of eft[u]      (0 for a source)
+ *   eft[v] = est[v] + cost[v]
+ * the earliest start and finish of v measured from the start of its workflow
+ * when every node takes its stand-alone cost; est[v] + cp[v] is the longest
+ * path through v, so H_w - (est[v] + cp[v]) is the slack of v.  Binary32, one
+ * rounded add per node, max exact.  The first call after an upload builds the
+ * transposed forest on the host (O(N + E)), allocates and synchronises the
+ * device; later calls only enqueue on `stream`.  hx_dag_update_costs keeps the
+ * forward results current once this has been called.  Scheduling does not
+ * read them.  Errors: HX_ERR_NOT_READY without an upload.
+ * hx_get_earliest_results: borrowed device pointers est[n_nodes],
+ * eft[n_nodes] (original node numbering), valid until the next upload or
+ * destroy; either argument may be NULL. */
+int hx_earliest_start(hx_cluster* h, void* stream);
+int hx_get_earliest_results(hx_cluster* h, const float** est, const float** eft);
+
 /* Prefill variant with a quadratic attention term (the roofline-style estimate of
  * Section 4.2 leaves the shape of the compute term open): with per_model[m] =
  * attention FLOPs per pair of prompt tokens of model m, the compute time of a

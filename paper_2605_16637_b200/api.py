@@ -55,6 +55,8 @@ def _load():
         "hx_dag_update_costs": [vp, vp, vp, u32, vp],
         "hx_dag_update_elapsed": [vp, vp, vp],
         "hx_get_dag_results": [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp)],
+        "hx_earliest_start": [vp, vp],
+        "hx_get_earliest_results": [vp, C.POINTER(vp), C.POINTER(vp)],
         "hx_set_options": [vp, C.POINTER(_Options)],
         "hx_set_attention_flops": [vp, vp],
         "hx_schedule_batch": [vp, vp, ci, vp, vp, vp],
@@ -159,6 +161,17 @@ def hx_get_dag_results(h):
     cp, tail, H = C.c_void_p(), C.c_void_p(), C.c_void_p()
     _check(_lib.hx_get_dag_results(h, C.byref(cp), C.byref(tail), C.byref(H)), h)
     return cp.value, tail.value, H.value
+
+
+def hx_earliest_start(h, stream=0):
+    _check(_lib.hx_earliest_start(h, stream), h)
+
+
+def hx_get_earliest_results(h):
+    """Device addresses (int) of est, eft."""
+    est, eft = C.c_void_p(), C.c_void_p()
+    _check(_lib.hx_get_earliest_results(h, C.byref(est), C.byref(eft)), h)
+    return est.value, eft.value
 
 
 def hx_set_options(h, score_mode=HX_MODE_COMPLETION, topk=0, commit=0, flags=0, alpha=1.5):
@@ -338,6 +351,14 @@ class Cluster:
         cp, tail, H = hx_get_dag_results(self.h)
         return (_dev_to_numpy(cp, self.n_nodes, "<f4"), _dev_to_numpy(tail, self.n_nodes, "<f4"),
                 _dev_to_numpy(H, self.n_workflows, "<f4"))
+
+    def earliest_start(self):
+        hx_earliest_start(self.h, self._stream())
+
+    def earliest_results(self):
+        """est, eft as numpy arrays (synchronises)."""
+        est, eft = hx_get_earliest_results(self.h)
+        return _dev_to_numpy(est, self.n_nodes, "<f4"), _dev_to_numpy(eft, self.n_nodes, "<f4")
 
     def set_options(self, score_mode=HX_MODE_COMPLETION, topk=0, commit=0, flags=0, alpha=1.5):
         hx_set_options(self.h, score_mode, topk, commit, flags, alpha)

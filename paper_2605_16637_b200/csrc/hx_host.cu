@@ -30,6 +30,13 @@ struct hx_cluster {
     // host copies for incremental refinement: node -> internal index, node -> workflow, workflow -> class
     std::vector<uint32_t> h_inv, h_node_wf;
     std::vector<uint8_t> h_wf_class;
+    // forward pass (earliest start): the same kernels on the transposed forest, built on first use
+    std::vector<uint32_t> h_row, h_col; std::vector<float> h_cost;
+    std::vector<void*> fwd_allocs;
+    HxForestDev fwd{};
+    std::vector<HxCpClass> fwd_classes;
+    std::vector<uint32_t> h_fwd_inv; std::vector<uint8_t> h_fwd_wf_class;
+    bool fwd_built = false, est_ready = false;
     std::vector<void*> upd_allocs;      // scratch of hx_dag_update_costs, grown on demand
     uint32_t* d_upd_idx = nullptr; float* d_upd_cost = nullptr; uint32_t* d_upd_wf = nullptr;
     size_t upd_cap = 0, upd_wf_cap = 0;
@@ -141,6 +148,136 @@ int ensure_topk(hx_cluster* h, int n_calls, int K) {
     HX_TRY(dev_alloc(h->tk_allocs, &b.acc_t, cap), "alloc outcome");
     b.cap_calls = (int)cap;
     h->tk = b;
+    return HX_OK;
+}
+
+
+// A forest regrouped for the horizon kernels: workflow by workflow, inside a workflow level by level
+// (level = height above the sinks), successors as local indices.
+struct HostForest {
+    uint32_t N = 0, E = 0, W = 0;
+    std::vector<uint32_t> perm, inv, wf_node_start, wf_edge_start, wf_seg_start, seg_off, irow, icol32;
+    std::vector<uint16_t> icol16;
+    std::vector<float> icost;
+    std::vector<uint32_t> ids[HX_CP_CLASSES];
+    std::vector<uint8_t> wf_class;
+};
+
+// Host part of an upload; false when the graph has a cycle.  The arrays were validated by the caller.
+bool prepare_forest(const uint32_t* row_ptr, const uint32_t* col_idx, const float* node_costs,
+                    const uint32_t* node_workflow, uint32_t N, uint32_t E, uint32_t W, HostForest* out) {
+    HostForest& hf = *out;
+    hf.N = N; hf.E = E; hf.W = W;
+    std::vector<uint32_t> indeg(N, 0);
+    for (uint32_t e = 0; e < E; ++e) ++indeg[col_idx[e]];
+    // topological order (cycle check), then height above the sinks
+    std::vector<uint32_t> topo; topo.reserve(N);
+    for (uint32_t v = 0; v < N; ++v) if (indeg[v] == 0) topo.push_back(v);
+    for (size_t i = 0; i < topo.size(); ++i) {
+        const uint32_t v = topo[i];
+        for (uint32_t e = row_ptr[v]; e < row_ptr[v + 1]; ++e) if (--indeg[col_idx[e]] == 0) topo.push_back(col_idx[e]);
+    }
+    if (topo.size() != N) return false;
+    std::vector<uint32_t> height(N, 0);
+    uint32_t max_h = 0;
+    for (size_t i = N; i-- > 0;) {
+        const uint32_t v = topo[i];
+        uint32_t hh = 0;
+        for (uint32_t e = row_ptr[v]; e < row_ptr[v + 1]; ++e) hh = std::max(hh, height[col_idx[e]] + 1);
+        height[v] = hh; max_h = std::max(max_h, hh);
+    }
+    // regroup: workflow by workflow, inside a workflow by height (two stable counting sorts)
+    std::vector<uint32_t> by_h(N);
+    auto& perm = hf.perm; auto& inv = hf.inv;
+    perm.assign(N, 0); inv.assign(N, 0);
+    {
+        std::vector<uint32_t> cnt((size_t)max_h + 2, 0);
+        for (uint32_t v = 0; v < N; ++v) ++cnt[height[v] + 1];
+        for (size_t i = 1; i < cnt.size(); ++i) cnt[i] += cnt[i - 1];
+        for (uint32_t v = 0; v < N; ++v) by_h[cnt[height[v]]++] = v;
+    }
+    auto& wf_node_start = hf.wf_node_start;
+    wf_node_start.assign((size_t)W + 1, 0);
+    for (uint32_t v = 0; v < N; ++v) ++wf_node_start[node_workflow[v] + 1];
+    for (uint32_t w = 0; w < W; ++w) wf_node_start[w + 1] += wf_node_start[w];
+    {
+        std::vector<uint32_t> cur(wf_node_start.begin(), wf_node_start.end() - 1);
+        for (uint32_t i = 0; i < N; ++i) { const uint32_t v = by_h[i]; perm[cur[node_workflow[v]]++] = v; }
+    }
+    for (uint32_t i = 0; i < N; ++i) inv[perm[i]] = i;
+    auto& wf_seg_start = hf.wf_seg_start; auto& seg_off = hf.seg_off;
+    wf_seg_start.assign((size_t)W + 1, 0); seg_off.clear();
+    seg_off.reserve((size_t)N + W);
+    for (uint32_t w = 0; w < W; ++w) {
+        wf_seg_start[w] = (uint32_t)seg_off.size();
+        const uint32_t ns = wf_node_start[w], ne = wf_node_start[w + 1];
+        seg_off.push_back(0);
+        for (uint32_t i = ns; i < ne; ++i)
+            if (i + 1 == ne || height[perm[i + 1]] != height[perm[i]]) seg_off.push_back(i + 1 - ns);
+    }
+    wf_seg_start[W] = (uint32_t)seg_off.size();
+    auto& irow = hf.irow; auto& icol32 = hf.icol32; auto& wf_edge_start = hf.wf_edge_start;
+    irow.assign((size_t)N + 1, 0); icol32.assign(E, 0); wf_edge_start.assign((size_t)W + 1, 0);
+    auto& icol16 = hf.icol16; auto& icost = hf.icost;
+    icol16.assign((size_t)E + 2, 0);                   // two spare entries: slices are copied as 32-bit words
+    icost.assign(N, 0.0f);
+    for (uint32_t i = 0; i < N; ++i) {
+        const uint32_t v = perm[i], ns = wf_node_start[node_workflow[v]];
+        icost[i] = node_costs[v];
+        uint32_t o = irow[i];
+        for (uint32_t e = row_ptr[v]; e < row_ptr[v + 1]; ++e, ++o) {
+            const uint32_t local = inv[col_idx[e]] - ns;
+            icol32[o] = local; icol16[o] = (uint16_t)local;
+        }
+        irow[i + 1] = o;
+    }
+    for (uint32_t w = 0; w <= W; ++w) wf_edge_start[w] = irow[wf_node_start[w]];
+
+    // classes of the horizon pass by staging footprint
+    auto& ids = hf.ids; auto& wf_class = hf.wf_class;
+    wf_class.assign(W, 0);
+    for (uint32_t w = 0; w < W; ++w) {
+        const size_t n = wf_node_start[w + 1] - wf_node_start[w], e = wf_edge_start[w + 1] - wf_edge_start[w];
+        const size_t nlev = wf_seg_start[w + 1] - wf_seg_start[w] - 1;
+        const size_t need = 4 * (3 * n + 1) + 4 * (nlev + 1) + 2 * e + 16;
+        const int k = hx_cpath_class_of(need, n);
+        ids[k].push_back(w);
+        wf_class[w] = (uint8_t)k;
+    }
+    // largest workflows first inside a class, so that the long ones do not start last
+    for (auto& v : ids)
+        std::stable_sort(v.begin(), v.end(), [&](uint32_t a, uint32_t b) {
+            return wf_node_start[a + 1] - wf_node_start[a] > wf_node_start[b + 1] - wf_node_start[b]; });
+
+    return true;
+}
+
+// Device part of an upload.  f->cp, f->tail and f->H are set by the caller.
+int upload_forest(hx_cluster* h, std::vector<void*>& pool, const HostForest& hf, HxForestDev* f,
+                  std::vector<HxCpClass>* classes) {
+    f->n_nodes = hf.N; f->n_edges = hf.E; f->n_workflows = hf.W;
+    uint32_t *d_wns, *d_wes, *d_wss, *d_seg, *d_irow, *d_icol32, *d_perm;
+    uint16_t* d_icol16; float* d_icost;
+    HX_TRY(dev_upload(pool, &d_wns, hf.wf_node_start), "upload forest");
+    HX_TRY(dev_upload(pool, &d_wes, hf.wf_edge_start), "upload forest");
+    HX_TRY(dev_upload(pool, &d_wss, hf.wf_seg_start), "upload forest");
+    HX_TRY(dev_upload(pool, &d_seg, hf.seg_off), "upload forest");
+    HX_TRY(dev_upload(pool, &d_irow, hf.irow), "upload forest");
+    HX_TRY(dev_upload(pool, &d_icol32, hf.icol32), "upload forest");
+    HX_TRY(dev_upload(pool, &d_icol16, hf.icol16), "upload forest");
+    HX_TRY(dev_upload(pool, &d_icost, hf.icost), "upload forest");
+    HX_TRY(dev_upload(pool, &d_perm, hf.perm), "upload forest");
+    f->wf_node_start = d_wns; f->wf_edge_start = d_wes; f->wf_seg_start = d_wss; f->seg_off = d_seg;
+    f->irow = d_irow; f->icol32 = d_icol32; f->icol16 = d_icol16; f->icost = d_icost; f->perm = d_perm;
+    classes->clear();
+    for (int k = 0; k < HX_CP_CLASSES; ++k) {
+        if (hf.ids[k].empty()) continue;
+        uint32_t* d_ids;
+        HX_TRY(dev_upload(pool, &d_ids, hf.ids[k]), "upload workflow classes");
+        HxCpClass c = hx_cpath_class_shape(k);
+        c.wf_ids = d_ids; c.count = (uint32_t)hf.ids[k].size();
+        classes->push_back(c);
+    }
     return HX_OK;
 }
 
@@ -280,7 +417,7 @@ int hx_cluster_destroy(hx_cluster* h) {
     if (!h) return HX_OK;
     DeviceGuard guard(h->device);
     cudaDeviceSynchronize();
-    free_pool(h->allocs); free_pool(h->dag_allocs); free_pool(h->tk_allocs); free_pool(h->upd_allocs); free_pool(h->dec_allocs);
+    free_pool(h->allocs); free_pool(h->dag_allocs); free_pool(h->fwd_allocs); free_pool(h->tk_allocs); free_pool(h->upd_allocs); free_pool(h->dec_allocs);
     if (h->st_calls) cudaFree(h->st_calls);
     if (h->st_assign) cudaFree(h->st_assign);
     if (h->st_cost) cudaFree(h->st_cost);
@@ -311,120 +448,30 @@ int hx_dag_upload(hx_cluster* h, const uint32_t* row_ptr, const uint32_t* col_id
     }
     for (uint32_t w = 0; w < W; ++w)
         if (!good_load(workflow_elapsed_s[w])) return fail(h, HX_ERR_INVALID_ARG, "elapsed times must be finite and >= 0");
-    std::vector<uint32_t> indeg(N, 0);
     for (uint32_t v = 0; v < N; ++v)
         for (uint32_t e = row_ptr[v]; e < row_ptr[v + 1]; ++e) {
             const uint32_t u = col_idx[e];
             if (u >= N) return fail(h, HX_ERR_INVALID_ARG, "edge target out of range");
             if (node_workflow[u] != node_workflow[v]) return fail(h, HX_ERR_INVALID_ARG, "edge crosses workflows");
-            ++indeg[u];
         }
-    // topological order (cycle check), then height above the sinks
-    std::vector<uint32_t> topo; topo.reserve(N);
-    for (uint32_t v = 0; v < N; ++v) if (indeg[v] == 0) topo.push_back(v);
-    for (size_t i = 0; i < topo.size(); ++i) {
-        const uint32_t v = topo[i];
-        for (uint32_t e = row_ptr[v]; e < row_ptr[v + 1]; ++e) if (--indeg[col_idx[e]] == 0) topo.push_back(col_idx[e]);
-    }
-    if (topo.size() != N) return fail(h, HX_ERR_CYCLE, "the graph has a cycle");
-    std::vector<uint32_t> height(N, 0);
-    uint32_t max_h = 0;
-    for (size_t i = N; i-- > 0;) {
-        const uint32_t v = topo[i];
-        uint32_t hh = 0;
-        for (uint32_t e = row_ptr[v]; e < row_ptr[v + 1]; ++e) hh = std::max(hh, height[col_idx[e]] + 1);
-        height[v] = hh; max_h = std::max(max_h, hh);
-    }
-    // regroup: workflow by workflow, inside a workflow by height (two stable counting sorts)
-    std::vector<uint32_t> by_h(N), perm(N), inv(N);
-    {
-        std::vector<uint32_t> cnt((size_t)max_h + 2, 0);
-        for (uint32_t v = 0; v < N; ++v) ++cnt[height[v] + 1];
-        for (size_t i = 1; i < cnt.size(); ++i) cnt[i] += cnt[i - 1];
-        for (uint32_t v = 0; v < N; ++v) by_h[cnt[height[v]]++] = v;
-    }
-    std::vector<uint32_t> wf_node_start((size_t)W + 1, 0);
-    for (uint32_t v = 0; v < N; ++v) ++wf_node_start[node_workflow[v] + 1];
-    for (uint32_t w = 0; w < W; ++w) wf_node_start[w + 1] += wf_node_start[w];
-    {
-        std::vector<uint32_t> cur(wf_node_start.begin(), wf_node_start.end() - 1);
-        for (uint32_t i = 0; i < N; ++i) { const uint32_t v = by_h[i]; perm[cur[node_workflow[v]]++] = v; }
-    }
-    for (uint32_t i = 0; i < N; ++i) inv[perm[i]] = i;
-    std::vector<uint32_t> wf_seg_start((size_t)W + 1, 0), seg_off;
-    seg_off.reserve((size_t)N + W);
-    for (uint32_t w = 0; w < W; ++w) {
-        wf_seg_start[w] = (uint32_t)seg_off.size();
-        const uint32_t ns = wf_node_start[w], ne = wf_node_start[w + 1];
-        seg_off.push_back(0);
-        for (uint32_t i = ns; i < ne; ++i)
-            if (i + 1 == ne || height[perm[i + 1]] != height[perm[i]]) seg_off.push_back(i + 1 - ns);
-    }
-    wf_seg_start[W] = (uint32_t)seg_off.size();
-    std::vector<uint32_t> irow((size_t)N + 1, 0), icol32(E), wf_edge_start((size_t)W + 1, 0);
-    std::vector<uint16_t> icol16((size_t)E + 2);       // two spare entries: slices are copied as 32-bit words
-    std::vector<float> icost(N);
-    for (uint32_t i = 0; i < N; ++i) {
-        const uint32_t v = perm[i], ns = wf_node_start[node_workflow[v]];
-        icost[i] = node_costs[v];
-        uint32_t o = irow[i];
-        for (uint32_t e = row_ptr[v]; e < row_ptr[v + 1]; ++e, ++o) {
-            const uint32_t local = inv[col_idx[e]] - ns;
-            icol32[o] = local; icol16[o] = (uint16_t)local;
-        }
-        irow[i + 1] = o;
-    }
-    for (uint32_t w = 0; w <= W; ++w) wf_edge_start[w] = irow[wf_node_start[w]];
-
-    // classes of the horizon pass by staging footprint
-    std::vector<uint32_t> ids[HX_CP_CLASSES];
-    std::vector<uint8_t> wf_class(W);
-    for (uint32_t w = 0; w < W; ++w) {
-        const size_t n = wf_node_start[w + 1] - wf_node_start[w], e = wf_edge_start[w + 1] - wf_edge_start[w];
-        const size_t nlev = wf_seg_start[w + 1] - wf_seg_start[w] - 1;
-        const size_t need = 4 * (3 * n + 1) + 4 * (nlev + 1) + 2 * e + 16;
-        const int k = hx_cpath_class_of(need, n);
-        ids[k].push_back(w);
-        wf_class[w] = (uint8_t)k;
-    }
-    // largest workflows first inside a class, so that the long ones do not start last
-    for (auto& v : ids)
-        std::stable_sort(v.begin(), v.end(), [&](uint32_t a, uint32_t b) {
-            return wf_node_start[a + 1] - wf_node_start[a] > wf_node_start[b + 1] - wf_node_start[b]; });
+    HostForest hf;
+    if (!prepare_forest(row_ptr, col_idx, node_costs, node_workflow, N, E, W, &hf))
+        return fail(h, HX_ERR_CYCLE, "the graph has a cycle");
 
     cudaDeviceSynchronize();
     free_pool(h->dag_allocs);
+    free_pool(h->fwd_allocs);
     h->dag_uploaded = false; h->cp_ready = false; h->classes.clear();
+    h->fwd_built = false; h->est_ready = false; h->fwd_classes.clear();
     HxForestDev f{};
-    f.n_nodes = N; f.n_edges = E; f.n_workflows = W;
-    uint32_t *d_wns, *d_wes, *d_wss, *d_seg, *d_irow, *d_icol32, *d_perm;
-    uint16_t* d_icol16; float* d_icost;
-    HX_TRY(dev_upload(h->dag_allocs, &d_wns, wf_node_start), "upload forest");
-    HX_TRY(dev_upload(h->dag_allocs, &d_wes, wf_edge_start), "upload forest");
-    HX_TRY(dev_upload(h->dag_allocs, &d_wss, wf_seg_start), "upload forest");
-    HX_TRY(dev_upload(h->dag_allocs, &d_seg, seg_off), "upload forest");
-    HX_TRY(dev_upload(h->dag_allocs, &d_irow, irow), "upload forest");
-    HX_TRY(dev_upload(h->dag_allocs, &d_icol32, icol32), "upload forest");
-    HX_TRY(dev_upload(h->dag_allocs, &d_icol16, icol16), "upload forest");
-    HX_TRY(dev_upload(h->dag_allocs, &d_icost, icost), "upload forest");
-    HX_TRY(dev_upload(h->dag_allocs, &d_perm, perm), "upload forest");
-    f.wf_node_start = d_wns; f.wf_edge_start = d_wes; f.wf_seg_start = d_wss; f.seg_off = d_seg;
-    f.irow = d_irow; f.icol32 = d_icol32; f.icol16 = d_icol16; f.icost = d_icost; f.perm = d_perm;
     HX_TRY(dev_alloc(h->dag_allocs, &f.cp, N), "alloc cp");
     HX_TRY(dev_alloc(h->dag_allocs, &f.tail, N), "alloc tail");
     HX_TRY(dev_alloc(h->dag_allocs, &f.H, W), "alloc H");
+    if (int rc = upload_forest(h, h->dag_allocs, hf, &f, &h->classes)) return rc;
     std::vector<uint32_t> nwf(node_workflow, node_workflow + N);
     std::vector<float> el(workflow_elapsed_s, workflow_elapsed_s + W);
     HX_TRY(dev_upload(h->dag_allocs, &h->d_node_wf, nwf), "upload node_workflow");
     HX_TRY(dev_upload(h->dag_allocs, &h->d_elapsed, el), "upload elapsed");
-    for (int k = 0; k < HX_CP_CLASSES; ++k) {
-        if (ids[k].empty()) continue;
-        uint32_t* d_ids;
-        HX_TRY(dev_upload(h->dag_allocs, &d_ids, ids[k]), "upload workflow classes");
-        HxCpClass c = hx_cpath_class_shape(k);
-        c.wf_ids = d_ids; c.count = (uint32_t)ids[k].size();
-        h->classes.push_back(c);
-    }
     if (!h->fj.ready) {
         bool ok = cudaEventCreateWithFlags(&h->fj.fork, cudaEventDisableTiming) == cudaSuccess;
         for (int i = 0; i < HX_CP_SIDE && ok; ++i)
@@ -434,9 +481,13 @@ int hx_dag_upload(hx_cluster* h, const uint32_t* row_ptr, const uint32_t* col_id
         h->fj.ready = 1;
     }
     h->forest = f;
-    h->h_inv = inv;
+    h->h_inv = std::move(hf.inv);
     h->h_node_wf.assign(node_workflow, node_workflow + N);
-    h->h_wf_class = wf_class;
+    h->h_wf_class = std::move(hf.wf_class);
+    // host copy of the graph: the forward pass builds its transposed forest from it on first use
+    h->h_row.assign(row_ptr, row_ptr + N + 1);
+    h->h_col.assign(col_idx, col_idx + E);
+    h->h_cost.assign(node_costs, node_costs + N);
     h->dag_uploaded = true;
     return HX_OK;
 }
@@ -479,9 +530,10 @@ int hx_dag_update_costs(hx_cluster* h, const uint32_t* node_ids, const float* ne
         if (!good_load(new_costs[i])) return fail(h, HX_ERR_INVALID_ARG, "node costs must be finite and >= 0");
     }
     // the last value given for a node wins; the workflows touched are recomputed, nothing else
+    const bool fwd = h->fwd_built;
     std::vector<uint32_t> idx; std::vector<float> val;
-    idx.reserve(n_updates); val.reserve(n_updates);
-    std::vector<uint32_t> dirty[HX_CP_CLASSES];
+    idx.reserve((fwd ? 2 : 1) * (size_t)n_updates); val.reserve(n_updates);
+    std::vector<uint32_t> dirty[HX_CP_CLASSES], fdirty[HX_CP_CLASSES];
     {
         std::vector<uint32_t> order(n_updates);
         for (uint32_t i = 0; i < n_updates; ++i) order[i] = i;
@@ -492,15 +544,26 @@ int hx_dag_update_costs(hx_cluster* h, const uint32_t* node_ids, const float* ne
             const uint32_t v = node_ids[order[i]];
             idx.push_back(h->h_inv[v]); val.push_back(new_costs[order[i]]);
             wfs.push_back(h->h_node_wf[v]);
+            h->h_cost[v] = new_costs[order[i]];
         }
         std::sort(wfs.begin(), wfs.end());
         wfs.erase(std::unique(wfs.begin(), wfs.end()), wfs.end());
         for (uint32_t w : wfs) dirty[h->h_wf_class[w]].push_back(w);
+        if (fwd) {
+            // second half of idx: the same nodes in the numbering of the transposed forest
+            for (uint32_t i = 0; i < n_updates; ++i) {
+                if (i + 1 < n_updates && node_ids[order[i + 1]] == node_ids[order[i]]) continue;
+                idx.push_back(h->h_fwd_inv[node_ids[order[i]]]);
+            }
+            for (uint32_t w : wfs) fdirty[h->h_fwd_wf_class[w]].push_back(w);
+        }
     }
+    const size_t n_set = val.size();
     DeviceGuard guard(h->device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     size_t n_wf = 0;
     for (auto& v : dirty) n_wf += v.size();
+    for (auto& v : fdirty) n_wf += v.size();
     if (idx.size() > h->upd_cap || n_wf > h->upd_wf_cap) {
         cudaDeviceSynchronize();
         free_pool(h->upd_allocs);
@@ -511,23 +574,30 @@ int hx_dag_update_costs(hx_cluster* h, const uint32_t* node_ids, const float* ne
     }
     HX_TRY(cudaMemcpyAsync(h->d_upd_idx, idx.data(), idx.size() * sizeof(uint32_t), cudaMemcpyHostToDevice, s), "copy updates");
     HX_TRY(cudaMemcpyAsync(h->d_upd_cost, val.data(), val.size() * sizeof(float), cudaMemcpyHostToDevice, s), "copy updates");
-    std::vector<HxCpClass> part;
+    std::vector<HxCpClass> part, fpart;
     size_t off = 0;
-    for (int k = 0; k < HX_CP_CLASSES; ++k) {
-        if (dirty[k].empty()) continue;
-        HX_TRY(cudaMemcpyAsync(h->d_upd_wf + off, dirty[k].data(), dirty[k].size() * sizeof(uint32_t),
-                               cudaMemcpyHostToDevice, s), "copy dirty workflows");
-        HxCpClass c = hx_cpath_class_shape(k);
-        c.wf_ids = h->d_upd_wf + off; c.count = (uint32_t)dirty[k].size();
-        part.push_back(c);
-        off += dirty[k].size();
-    }
+    for (int pass = 0; pass < 2; ++pass)
+        for (int k = 0; k < HX_CP_CLASSES; ++k) {
+            const std::vector<uint32_t>& dk = pass ? fdirty[k] : dirty[k];
+            if (dk.empty()) continue;
+            HX_TRY(cudaMemcpyAsync(h->d_upd_wf + off, dk.data(), dk.size() * sizeof(uint32_t),
+                                   cudaMemcpyHostToDevice, s), "copy dirty workflows");
+            HxCpClass c = hx_cpath_class_shape(k);
+            c.wf_ids = h->d_upd_wf + off; c.count = (uint32_t)dk.size();
+            (pass ? fpart : part).push_back(c);
+            off += dk.size();
+        }
     // pageable host memory: the copies above have read the vectors by the time they return
     {
         SpanGuard span(h, 2, s);
-        HX_TRY(hx_launch_cost_update(h->forest, h->d_upd_idx, h->d_upd_cost, (uint32_t)idx.size(), s, &h->launches), "cost update kernel");
+        HX_TRY(hx_launch_cost_update(h->forest, h->d_upd_idx, h->d_upd_cost, (uint32_t)n_set, s, &h->launches), "cost update kernel");
         if (h->cp_ready)
             HX_TRY(hx_launch_cpath(h->forest, part.data(), (int)part.size(), s, &h->launches, &h->fj), "horizon kernels");
+        if (fwd) {
+            HX_TRY(hx_launch_cost_update(h->fwd, h->d_upd_idx + n_set, h->d_upd_cost, (uint32_t)n_set, s, &h->launches), "cost update kernel");
+            if (h->est_ready)
+                HX_TRY(hx_launch_cpath(h->fwd, fpart.data(), (int)fpart.size(), s, &h->launches, &h->fj), "forward pass kernels");
+        }
     }
     (void)W;
     return HX_OK;
@@ -539,6 +609,58 @@ int hx_get_dag_results(hx_cluster* h, const float** cp, const float** tail, cons
     if (cp) *cp = h->forest.cp;
     if (tail) *tail = h->forest.tail;
     if (H) *H = h->forest.H;
+    return HX_OK;
+}
+
+// Builds the transposed forest (every edge reversed) for the forward pass.
+static int build_forward_forest(hx_cluster* h) {
+    const uint32_t N = h->forest.n_nodes, E = h->forest.n_edges, W = h->forest.n_workflows;
+    std::vector<uint32_t> trow((size_t)N + 1, 0), tcol(E);
+    for (uint32_t e = 0; e < E; ++e) ++trow[h->h_col[e] + 1];
+    for (uint32_t v = 0; v < N; ++v) trow[v + 1] += trow[v];
+    {
+        std::vector<uint32_t> cur(trow.begin(), trow.end() - 1);
+        for (uint32_t v = 0; v < N; ++v)
+            for (uint32_t e = h->h_row[v]; e < h->h_row[v + 1]; ++e) tcol[cur[h->h_col[e]]++] = v;
+    }
+    HostForest hf;
+    if (!prepare_forest(trow.data(), tcol.data(), h->h_cost.data(), h->h_node_wf.data(), N, E, W, &hf))
+        return fail(h, HX_ERR_CYCLE, "the graph has a cycle");
+    cudaDeviceSynchronize();
+    free_pool(h->fwd_allocs);
+    h->fwd_built = false; h->est_ready = false;
+    HxForestDev f{};
+    HX_TRY(dev_alloc(h->fwd_allocs, &f.cp, N), "alloc earliest finish");
+    HX_TRY(dev_alloc(h->fwd_allocs, &f.tail, N), "alloc earliest start");
+    HX_TRY(dev_alloc(h->fwd_allocs, &f.H, W), "alloc forward horizon");
+    if (int rc = upload_forest(h, h->fwd_allocs, hf, &f, &h->fwd_classes)) return rc;
+    h->fwd = f;
+    h->h_fwd_inv = std::move(hf.inv);
+    h->h_fwd_wf_class = std::move(hf.wf_class);
+    h->fwd_built = true;
+    return HX_OK;
+}
+
+int hx_earliest_start(hx_cluster* h, void* stream) {
+    if (!h) return HX_ERR_INVALID_ARG;
+    if (!h->dag_uploaded) return fail(h, HX_ERR_NOT_READY, "no forest uploaded");
+    DeviceGuard guard(h->device);
+    if (!h->fwd_built)
+        if (int rc = build_forward_forest(h)) return rc;
+    {
+        SpanGuard span(h, 2, static_cast<cudaStream_t>(stream));
+        HX_TRY(hx_launch_cpath(h->fwd, h->fwd_classes.data(), (int)h->fwd_classes.size(),
+                               static_cast<cudaStream_t>(stream), &h->launches, &h->fj), "forward pass kernels");
+    }
+    h->est_ready = true;
+    return HX_OK;
+}
+
+int hx_get_earliest_results(hx_cluster* h, const float** est, const float** eft) {
+    if (!h) return HX_ERR_INVALID_ARG;
+    if (!h->fwd_built) return fail(h, HX_ERR_NOT_READY, "no forward pass yet: call hx_earliest_start");
+    if (est) *est = h->fwd.tail;
+    if (eft) *eft = h->fwd.cp;
     return HX_OK;
 }
 

@@ -97,3 +97,64 @@ def test_elapsed_refresh_feeds_the_ratio(hx, oracle):
     with pytest.raises(hx.HxError):
         gc.update_elapsed(later[:-1])
     gc.close()
+
+
+@pytest.mark.parametrize("name, scale, frac", [("tiny", 1.0, 0.3), ("medium", 1.0, 0.02), ("cp_stress", 1 / 20, 0.001),
+                                               ("large", 1 / 16, 0.2), ("sweep", 1 / 8, 0.01)])
+def test_forward_pass_equals_oracle_and_follows_cost_updates(hx, oracle, name, scale, frac):
+    wl = make_workload(name, scale=scale)
+    oc, gc = hh.oracle_cluster(wl), hh.gpu_cluster(wl)
+    cost = _costs(wl, oracle, oc, gc)
+    gc.dag_upload(wl.row_ptr, wl.col, cost, wl.node_wf, wl.elapsed)
+    with pytest.raises(hx.HxError) as e:
+        gc.earliest_results()
+    assert e.value.code == -4
+    gc.critical_path()
+    gc.earliest_start()
+    est, eft = gc.earliest_results()
+    w_est, w_eft = oracle.earliest_start(wl.row_ptr, wl.col, cost)
+    assert np.array_equal(est, w_est) and np.array_equal(eft, w_eft)
+    cp, tail, H = gc.dag_results()
+    want = oracle.longest_path(wl.row_ptr, wl.col, cost, wl.node_wf, wl.n_workflows)
+    assert np.array_equal(cp, want.cp) and np.array_equal(H, want.H)       # the backward results are untouched
+    # longest path through a node never exceeds the horizon by more than the rounding of two sums
+    assert np.all(est + cp <= H[wl.node_wf] * (1 + 1e-4))
+    rng = np.random.default_rng(17)
+    for rnd in range(2):
+        k = max(1, int(frac * wl.n_nodes))
+        ids = rng.integers(0, wl.n_nodes, k).astype(np.uint32)
+        new = (cost[ids] * rng.uniform(0.5, 2.0, k)).astype(np.float32)
+        gc.update_costs(ids, new)
+        for i, v in zip(ids, new):
+            cost[i] = v
+        est, eft = gc.earliest_results()
+        w_est, w_eft = oracle.earliest_start(wl.row_ptr, wl.col, cost)
+        assert np.array_equal(est, w_est) and np.array_equal(eft, w_eft)
+        cp, tail, H = gc.dag_results()
+        want = oracle.longest_path(wl.row_ptr, wl.col, cost, wl.node_wf, wl.n_workflows)
+        assert np.array_equal(cp, want.cp) and np.array_equal(tail, want.tail) and np.array_equal(H, want.H)
+    assert gc.status() == 0
+    gc.close()
+
+
+def test_forward_pass_built_after_cost_updates_and_rebuilt_after_upload(hx, oracle):
+    wl = make_workload("medium", scale=0.25)
+    oc, gc = hh.oracle_cluster(wl), hh.gpu_cluster(wl)
+    cost = _costs(wl, oracle, oc, gc)
+    gc.dag_upload(wl.row_ptr, wl.col, cost, wl.node_wf, wl.elapsed)
+    gc.update_costs([3, 5, 3], [0.25, 0.5, 0.75])              # before the transposed forest exists
+    cost[3], cost[5] = 0.75, 0.5
+    gc.earliest_start()                                        # without hx_critical_path: independent of it
+    est, eft = gc.earliest_results()
+    w_est, w_eft = oracle.earliest_start(wl.row_ptr, wl.col, cost)
+    assert np.array_equal(est, w_est) and np.array_equal(eft, w_eft)
+    wl2 = make_workload("tiny")
+    cost2 = _costs(wl2, oracle, hh.oracle_cluster(wl2), hh.gpu_cluster(wl2))
+    gc.dag_upload(wl2.row_ptr, wl2.col, cost2, wl2.node_wf, wl2.elapsed)
+    with pytest.raises(hx.HxError):
+        gc.earliest_results()                                  # the old forward results went with the old forest
+    gc.earliest_start()
+    est, eft = gc.earliest_results()
+    w_est, w_eft = oracle.earliest_start(wl2.row_ptr, wl2.col, cost2)
+    assert np.array_equal(est, w_est) and np.array_equal(eft, w_eft)
+    gc.close()
