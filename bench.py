@@ -394,6 +394,7 @@ def run_cuda(args):
         "device_status": status, "roofline": roofline, "cpu_baseline": cpu, "clocks": clocks,
         "greedy_planner": greedy,
         "decode_scheduler": decode_leg() if world == 1 and not args.no_cpu_baseline else None,
+        "horizon_refinement": refine_leg() if world == 1 and not args.no_cpu_baseline else None,
     }
     print(json.dumps(out))
     if dist is not None:
@@ -461,6 +462,54 @@ def decode_leg():
     gc.close()
     return {"calls": 1024, "decode_instances": wl.D, "ms_wall_incl_copies": 1e3 * float(np.median(times[1:])),
             "oracle_ms_1_core": cpu_ms, "identical_to_oracle": same}
+
+
+def refine_leg():
+    """Side measurement, outside the timed region: online refinement of the horizons on the forest of the
+    sweep (Section 5.1).  Wall clock per call including host work and a synchronisation, median of 5;
+    the oracle's full pass on one core beside it."""
+    import torch
+    import paper_2605_16637_b200 as hx
+    from hx_synth import make_workload
+    from oracle import hx_oracle as ho
+    wl = make_workload("sweep")
+    rng = np.random.default_rng(5)
+    cost = rng.lognormal(0, 1, wl.n_nodes).astype(np.float32)
+    gc = hx.Cluster.from_workload(wl)
+
+    def wall(fn, reps=5):
+        ts = []
+        for _ in range(reps):
+            torch.cuda.synchronize(); t0 = time.perf_counter(); fn(); torch.cuda.synchronize()
+            ts.append(time.perf_counter() - t0)
+        return 1e3 * float(np.median(ts))
+
+    out = {"nodes": wl.n_nodes, "workflows": wl.n_workflows}
+    out["upload_ms"] = wall(lambda: gc.dag_upload(wl.row_ptr, wl.col, cost, wl.node_wf, wl.elapsed), reps=3)
+    out["full_pass_ms"] = wall(gc.critical_path)
+    k = 1000
+    ids = rng.choice(wl.n_nodes, k, replace=False).astype(np.uint32)
+    out["update_1000_costs_ms"] = wall(lambda: gc.update_costs(ids, (cost[ids] * rng.uniform(0.5, 2, k)).astype(np.float32)))
+    def forward():
+        gc.earliest_start()
+    out["forward_pass_first_ms"] = wall(forward, reps=1)
+    out["forward_pass_ms"] = wall(forward)
+    # 1,000 newly revealed nodes, one behind a random node of each of 1,000 workflows
+    order = np.argsort(wl.node_wf, kind="stable")
+    first_of = order[np.searchsorted(wl.node_wf[order], np.arange(wl.n_workflows))].astype(np.uint32)
+    batches = []
+    for i in range(5):
+        wfs = rng.choice(wl.n_workflows, k, replace=False).astype(np.uint32)
+        new = np.arange(wl.n_nodes + i * k, wl.n_nodes + (i + 1) * k, dtype=np.uint32)
+        batches.append((rng.lognormal(0, 1, k).astype(np.float32), wfs, first_of[wfs], new))
+    out["append_1000_nodes_ms"] = wall(lambda: gc.dag_append(*batches.pop(0)))
+    orc = ho.Oracle()
+    t0 = time.perf_counter()
+    orc.longest_path(wl.row_ptr, wl.col, cost, wl.node_wf, wl.n_workflows)
+    out["oracle_full_pass_ms_1_core"] = 1e3 * (time.perf_counter() - t0)
+    out["device_status"] = gc.status()
+    gc.close()
+    return out
 
 
 def run_configs(args):

@@ -172,6 +172,29 @@ int hx_dag_update_elapsed(hx_cluster* h, const float* workflow_elapsed_s, void* 
  * Any of the three output arguments may be NULL. */
 int hx_get_dag_results(hx_cluster* h, const float** cp, const float** tail, const float** H);
 
+/* Appends newly revealed nodes and edges to the uploaded forest (Section 5.1:
+ * the horizon is refined as the workflow reveals more of its DAG).  The new
+ * nodes take the numbers n_nodes .. n_nodes + n_new_nodes - 1 (n_nodes = the
+ * count before the call); new_costs[i] and new_node_workflow[i] (an existing
+ * workflow) describe node n_nodes + i.  Edge e runs from edge_src[e] to
+ * edge_dst[e]; either end may be an old or a new node of the same workflow.
+ * All arrays are host arrays, read before the call returns.  The workflows
+ * touched are levelised again as a group of their own and, once horizons
+ * exist, recomputed on `stream`; all other workflows keep their results
+ * untouched, and the outcome equals a fresh upload of the grown graph followed
+ * by hx_critical_path, bit for bit.  The call allocates device memory for the
+ * regrouped workflows; when the node arrays outgrow their reserve (a quarter
+ * of the uploaded size) they are reallocated, which synchronises the device
+ * and moves the arrays: fetch hx_get_dag_results again after an append.  The
+ * forward results are dropped; call hx_earliest_start again.
+ * Errors, all leaving the forest as it was: HX_ERR_NOT_READY without an
+ * upload; HX_ERR_INVALID_ARG for a NULL array, a workflow or endpoint out of
+ * range, an edge across workflows, a cost that is negative or not finite;
+ * HX_ERR_CYCLE when the new edges close a cycle. */
+int hx_dag_append(hx_cluster* h, uint32_t n_new_nodes, const float* new_costs,
+                  const uint32_t* new_node_workflow, uint32_t n_new_edges,
+                  const uint32_t* edge_src, const uint32_t* edge_dst, void* stream);
+
 /* Forward pass over the same forest (Section 4.1: a node becomes ready when
  * all its predecessors have completed): for every node v
  *   est[v] = max over predecessors u of eft[u]      (0 for a source)

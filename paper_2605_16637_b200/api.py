@@ -55,6 +55,7 @@ def _load():
         "hx_dag_update_costs": [vp, vp, vp, u32, vp],
         "hx_dag_update_elapsed": [vp, vp, vp],
         "hx_get_dag_results": [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp)],
+        "hx_dag_append": [vp, C.c_uint32, vp, vp, C.c_uint32, vp, vp, vp],
         "hx_earliest_start": [vp, vp],
         "hx_get_earliest_results": [vp, C.POINTER(vp), C.POINTER(vp)],
         "hx_set_options": [vp, C.POINTER(_Options)],
@@ -161,6 +162,15 @@ def hx_get_dag_results(h):
     cp, tail, H = C.c_void_p(), C.c_void_p(), C.c_void_p()
     _check(_lib.hx_get_dag_results(h, C.byref(cp), C.byref(tail), C.byref(H)), h)
     return cp.value, tail.value, H.value
+
+
+def hx_dag_append(h, new_costs, new_node_workflow, edge_src, edge_dst, stream=0):
+    """Appends nodes (costs, workflows) and edges (src, dst); the new nodes are numbered on from the old count."""
+    c, w = _np(new_costs, np.float32), _np(new_node_workflow, np.uint32)
+    es, ed = _np(edge_src, np.uint32), _np(edge_dst, np.uint32)
+    if c.shape[0] != w.shape[0] or es.shape[0] != ed.shape[0]:
+        raise HxError(-1, "array lengths differ")
+    _check(_lib.hx_dag_append(h, c.shape[0], _p(c), _p(w), es.shape[0], _p(es), _p(ed), stream), h)
 
 
 def hx_earliest_start(h, stream=0):
@@ -351,6 +361,10 @@ class Cluster:
         cp, tail, H = hx_get_dag_results(self.h)
         return (_dev_to_numpy(cp, self.n_nodes, "<f4"), _dev_to_numpy(tail, self.n_nodes, "<f4"),
                 _dev_to_numpy(H, self.n_workflows, "<f4"))
+
+    def dag_append(self, new_costs, new_node_workflow, edge_src, edge_dst):
+        hx_dag_append(self.h, new_costs, new_node_workflow, edge_src, edge_dst, self._stream())
+        self.n_nodes += int(np.asarray(new_costs).shape[0])
 
     def earliest_start(self):
         hx_earliest_start(self.h, self._stream())

@@ -115,7 +115,7 @@ __global__ void hx_cpath_staged_kernel(HxForestDev f, const uint32_t* __restrict
         }
     }
     hmax = group_max<GW>(hmax, red, t, tpw);
-    if (t == 0) f.H[w] = hmax;
+    if (t == 0) f.H[f.wf_gid ? f.wf_gid[w] : w] = hmax;
 }
 
 // One block per workflow, everything in global memory: for workflows too large
@@ -144,7 +144,7 @@ __global__ void hx_cpath_global_kernel(HxForestDev f, const uint32_t* __restrict
         __syncthreads();
     }
     hmax = group_max<false>(hmax, red, t, tpw);
-    if (t == 0) f.H[w] = hmax;
+    if (t == 0) f.H[f.wf_gid ? f.wf_gid[w] : w] = hmax;
 }
 
 // Replaces the cost estimates of some nodes (internal numbering) by newer values, e.g. observed

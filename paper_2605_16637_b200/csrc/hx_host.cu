@@ -7,8 +7,56 @@
 #include <cstring>
 #include <mutex>
 #include <new>
+#include <unordered_map>
 
 #include "hx_internal.h"
+
+// A group of workflows levelised together: the upload is part 0, every append adds one that takes
+// over the workflows it touched.  The class lists on the device are mirrored here so that a workflow
+// can be taken out of its list with one 4-byte copy.
+struct ForestPart {
+    HxForestDev f{};
+    std::vector<void*> allocs;
+    std::vector<uint32_t> ids[HX_CP_CLASSES];   // workflows (numbering of this part) per class
+    uint32_t* d_ids[HX_CP_CLASSES] = {};
+    std::vector<uint32_t> pos;                  // workflow -> position in its class list
+    std::vector<uint8_t> wf_class;              // workflow -> class
+    uint32_t live = 0;                          // workflows this part still owns
+    void classes(std::vector<HxCpClass>* out) const {
+        out->clear();
+        for (int k = 0; k < HX_CP_CLASSES; ++k) {
+            if (ids[k].empty()) continue;
+            HxCpClass c = hx_cpath_class_shape(k);
+            c.wf_ids = d_ids[k]; c.count = (uint32_t)ids[k].size();
+            out->push_back(c);
+        }
+    }
+    // Workflow l now belongs to another part: the last entry of its list takes its place.  The device
+    // lists follow at the next flush().
+    std::vector<uint32_t> changed[HX_CP_CLASSES];
+    void drop(uint32_t l) {
+        const int k = wf_class[l];
+        std::vector<uint32_t>& v = ids[k];
+        const uint32_t p = pos[l], last = v.back();
+        v[p] = last; pos[last] = p; v.pop_back(); pos[l] = ~0u; --live;
+        changed[k].push_back(p);
+    }
+    cudaError_t flush(cudaStream_t s) {
+        cudaError_t e = cudaSuccess;
+        for (int k = 0; k < HX_CP_CLASSES && e == cudaSuccess; ++k) {
+            const std::vector<uint32_t>& v = ids[k];
+            if (changed[k].size() > 8) {             // one copy of the whole list beats many 4-byte copies
+                if (!v.empty()) e = cudaMemcpyAsync(d_ids[k], v.data(), v.size() * sizeof(uint32_t), cudaMemcpyHostToDevice, s);
+            } else {
+                for (uint32_t p : changed[k])
+                    if (p < v.size() && e == cudaSuccess)
+                        e = cudaMemcpyAsync(d_ids[k] + p, &v[p], sizeof(uint32_t), cudaMemcpyHostToDevice, s);
+            }
+            changed[k].clear();
+        }
+        return e;
+    }
+};
 
 struct hx_cluster {
     int device = 0, n_sm = 0;
@@ -22,14 +70,19 @@ struct hx_cluster {
     int* status = nullptr;
     // forest
     bool dag_uploaded = false, cp_ready = false;
-    HxForestDev forest{};
+    std::vector<ForestPart> parts;      // part 0: the upload; later ones: workflows rebuilt by hx_dag_append
+    uint32_t N = 0, E = 0, W = 0;       // current size of the forest
+    size_t capN = 0;                    // room in cp, tail and node_wf
+    std::vector<void*> node_allocs;     // cp, tail, node_wf: regrown when appended nodes outgrow them
+    float *g_cp = nullptr, *g_tail = nullptr, *g_H = nullptr;
     uint32_t* d_node_wf = nullptr;
     float* d_elapsed = nullptr;
-    std::vector<HxCpClass> classes;
     HxForkJoin fj{};                    // side streams of the horizon pass, created with the first upload
-    // host copies for incremental refinement: node -> internal index, node -> workflow, workflow -> class
-    std::vector<uint32_t> h_inv, h_node_wf;
-    std::vector<uint8_t> h_wf_class;
+    // host state for incremental refinement: node -> index inside the owning part, node -> workflow,
+    // workflow -> owning part and its number there; appended nodes and edges on top of the uploaded CSR
+    std::vector<uint32_t> h_inv, h_node_wf, h_wf_part, h_wf_local, h_base_perm, h_base_wns, h_local;
+    std::vector<float> h_elapsed;
+    std::unordered_map<uint32_t, std::vector<uint32_t>> extra_succ, extra_nodes;
     // forward pass (earliest start): the same kernels on the transposed forest, built on first use
     std::vector<uint32_t> h_row, h_col; std::vector<float> h_cost;
     std::vector<void*> fwd_allocs;
@@ -252,33 +305,64 @@ bool prepare_forest(const uint32_t* row_ptr, const uint32_t* col_idx, const floa
     return true;
 }
 
-// Device part of an upload.  f->cp, f->tail and f->H are set by the caller.
-int upload_forest(hx_cluster* h, std::vector<void*>& pool, const HostForest& hf, HxForestDev* f,
-                  std::vector<HxCpClass>* classes) {
+// Device part of an upload into part->allocs.  part->f.cp, .tail and .H are set by the caller.  With
+// `node_gid` / `wf_gid` the forest is a slice of a larger one: results go to those node and workflow numbers.
+int upload_forest(hx_cluster* h, const HostForest& hf, ForestPart* part,
+                  const std::vector<uint32_t>* node_gid = nullptr, const std::vector<uint32_t>* wf_gid = nullptr) {
+    HxForestDev* f = &part->f;
     f->n_nodes = hf.N; f->n_edges = hf.E; f->n_workflows = hf.W;
-    uint32_t *d_wns, *d_wes, *d_wss, *d_seg, *d_irow, *d_icol32, *d_perm;
-    uint16_t* d_icol16; float* d_icost;
-    HX_TRY(dev_upload(pool, &d_wns, hf.wf_node_start), "upload forest");
-    HX_TRY(dev_upload(pool, &d_wes, hf.wf_edge_start), "upload forest");
-    HX_TRY(dev_upload(pool, &d_wss, hf.wf_seg_start), "upload forest");
-    HX_TRY(dev_upload(pool, &d_seg, hf.seg_off), "upload forest");
-    HX_TRY(dev_upload(pool, &d_irow, hf.irow), "upload forest");
-    HX_TRY(dev_upload(pool, &d_icol32, hf.icol32), "upload forest");
-    HX_TRY(dev_upload(pool, &d_icol16, hf.icol16), "upload forest");
-    HX_TRY(dev_upload(pool, &d_icost, hf.icost), "upload forest");
-    HX_TRY(dev_upload(pool, &d_perm, hf.perm), "upload forest");
-    f->wf_node_start = d_wns; f->wf_edge_start = d_wes; f->wf_seg_start = d_wss; f->seg_off = d_seg;
-    f->irow = d_irow; f->icol32 = d_icol32; f->icol16 = d_icol16; f->icost = d_icost; f->perm = d_perm;
-    classes->clear();
+    // one allocation and one copy for the whole part: sections packed on 256-byte boundaries
+    std::vector<unsigned char> blob;
+    auto put = [&](const void* src, size_t bytes) {
+        const size_t off = (blob.size() + 255) & ~size_t(255);
+        blob.resize(off + bytes);
+        if (bytes) std::memcpy(blob.data() + off, src, bytes);
+        return off;
+    };
+    auto put_u32 = [&](const std::vector<uint32_t>& v) { return put(v.data(), v.size() * sizeof(uint32_t)); };
+    const size_t o_wns = put_u32(hf.wf_node_start), o_wes = put_u32(hf.wf_edge_start), o_wss = put_u32(hf.wf_seg_start);
+    const size_t o_seg = put_u32(hf.seg_off), o_irow = put_u32(hf.irow), o_icol32 = put_u32(hf.icol32);
+    const size_t o_icol16 = put(hf.icol16.data(), hf.icol16.size() * sizeof(uint16_t));
+    const size_t o_icost = put(hf.icost.data(), hf.icost.size() * sizeof(float));
+    size_t o_perm;
+    if (node_gid) {
+        std::vector<uint32_t> perm(hf.perm.size());
+        for (size_t i = 0; i < perm.size(); ++i) perm[i] = (*node_gid)[hf.perm[i]];
+        o_perm = put_u32(perm);
+    } else {
+        o_perm = put_u32(hf.perm);
+    }
+    const size_t o_gid = wf_gid ? put_u32(*wf_gid) : 0;
+    size_t o_ids[HX_CP_CLASSES];
+    for (int k = 0; k < HX_CP_CLASSES; ++k) o_ids[k] = put_u32(hf.ids[k]);
+    unsigned char* base = nullptr;
+    HX_TRY(dev_alloc(part->allocs, &base, blob.size()), "alloc forest");
+    HX_TRY(cudaMemcpy(base, blob.data(), blob.size(), cudaMemcpyHostToDevice), "upload forest");
+    auto u32 = [&](size_t off) { return reinterpret_cast<uint32_t*>(base + off); };
+    f->wf_node_start = u32(o_wns); f->wf_edge_start = u32(o_wes); f->wf_seg_start = u32(o_wss);
+    f->seg_off = u32(o_seg); f->irow = u32(o_irow); f->icol32 = u32(o_icol32);
+    f->icol16 = reinterpret_cast<uint16_t*>(base + o_icol16);
+    f->icost = reinterpret_cast<float*>(base + o_icost);
+    f->perm = u32(o_perm);
+    f->wf_gid = wf_gid ? u32(o_gid) : nullptr;
+    part->wf_class = hf.wf_class;
+    part->pos.assign(hf.W, 0);
+    part->live = hf.W;
     for (int k = 0; k < HX_CP_CLASSES; ++k) {
-        if (hf.ids[k].empty()) continue;
-        uint32_t* d_ids;
-        HX_TRY(dev_upload(pool, &d_ids, hf.ids[k]), "upload workflow classes");
-        HxCpClass c = hx_cpath_class_shape(k);
-        c.wf_ids = d_ids; c.count = (uint32_t)hf.ids[k].size();
-        classes->push_back(c);
+        part->ids[k] = hf.ids[k];
+        part->d_ids[k] = hf.ids[k].empty() ? nullptr : u32(o_ids[k]);
+        for (size_t i = 0; i < hf.ids[k].size(); ++i) part->pos[hf.ids[k][i]] = (uint32_t)i;
     }
     return HX_OK;
+}
+
+// Successors of node v in the current graph: its row of the uploaded CSR plus appended edges.
+template <class Fn>
+void for_each_successor(const hx_cluster* h, uint32_t v, Fn fn) {
+    if ((size_t)v + 1 < h->h_row.size())
+        for (uint32_t e = h->h_row[v]; e < h->h_row[v + 1]; ++e) fn(h->h_col[e]);
+    auto it = h->extra_succ.find(v);
+    if (it != h->extra_succ.end()) for (uint32_t u : it->second) fn(u);
 }
 
 }  // namespace
@@ -417,6 +501,8 @@ int hx_cluster_destroy(hx_cluster* h) {
     if (!h) return HX_OK;
     DeviceGuard guard(h->device);
     cudaDeviceSynchronize();
+    for (auto& p : h->parts) free_pool(p.allocs);
+    free_pool(h->node_allocs);
     free_pool(h->allocs); free_pool(h->dag_allocs); free_pool(h->fwd_allocs); free_pool(h->tk_allocs); free_pool(h->upd_allocs); free_pool(h->dec_allocs);
     if (h->st_calls) cudaFree(h->st_calls);
     if (h->st_assign) cudaFree(h->st_assign);
@@ -459,19 +545,27 @@ int hx_dag_upload(hx_cluster* h, const uint32_t* row_ptr, const uint32_t* col_id
         return fail(h, HX_ERR_CYCLE, "the graph has a cycle");
 
     cudaDeviceSynchronize();
+    for (auto& p : h->parts) free_pool(p.allocs);
+    h->parts.clear();
     free_pool(h->dag_allocs);
+    free_pool(h->node_allocs);
     free_pool(h->fwd_allocs);
-    h->dag_uploaded = false; h->cp_ready = false; h->classes.clear();
+    h->dag_uploaded = false; h->cp_ready = false;
     h->fwd_built = false; h->est_ready = false; h->fwd_classes.clear();
-    HxForestDev f{};
-    HX_TRY(dev_alloc(h->dag_allocs, &f.cp, N), "alloc cp");
-    HX_TRY(dev_alloc(h->dag_allocs, &f.tail, N), "alloc tail");
-    HX_TRY(dev_alloc(h->dag_allocs, &f.H, W), "alloc H");
-    if (int rc = upload_forest(h, h->dag_allocs, hf, &f, &h->classes)) return rc;
-    std::vector<uint32_t> nwf(node_workflow, node_workflow + N);
+    h->N = h->E = h->W = 0; h->capN = 0;
+    // results and the node -> workflow map keep room for nodes appended later
+    const size_t cap = (size_t)N + std::max<size_t>(N / 4, 4096);
+    HX_TRY(dev_alloc(h->node_allocs, &h->g_cp, cap), "alloc cp");
+    HX_TRY(dev_alloc(h->node_allocs, &h->g_tail, cap), "alloc tail");
+    HX_TRY(dev_alloc(h->node_allocs, &h->d_node_wf, cap), "alloc node_workflow");
+    HX_TRY(dev_alloc(h->dag_allocs, &h->g_H, W), "alloc H");
+    HX_TRY(cudaMemcpy(h->d_node_wf, node_workflow, (size_t)N * sizeof(uint32_t), cudaMemcpyHostToDevice), "upload node_workflow");
     std::vector<float> el(workflow_elapsed_s, workflow_elapsed_s + W);
-    HX_TRY(dev_upload(h->dag_allocs, &h->d_node_wf, nwf), "upload node_workflow");
     HX_TRY(dev_upload(h->dag_allocs, &h->d_elapsed, el), "upload elapsed");
+    h->parts.emplace_back();
+    ForestPart& base = h->parts.back();
+    base.f.cp = h->g_cp; base.f.tail = h->g_tail; base.f.H = h->g_H;
+    if (int rc = upload_forest(h, hf, &base)) return rc;
     if (!h->fj.ready) {
         bool ok = cudaEventCreateWithFlags(&h->fj.fork, cudaEventDisableTiming) == cudaSuccess;
         for (int i = 0; i < HX_CP_SIDE && ok; ++i)
@@ -480,15 +574,33 @@ int hx_dag_upload(hx_cluster* h, const uint32_t* row_ptr, const uint32_t* col_id
         if (!ok) return fail(h, HX_ERR_CUDA, "creating the side streams of the horizon pass");
         h->fj.ready = 1;
     }
-    h->forest = f;
+    h->N = N; h->E = E; h->W = W; h->capN = cap;
     h->h_inv = std::move(hf.inv);
     h->h_node_wf.assign(node_workflow, node_workflow + N);
-    h->h_wf_class = std::move(hf.wf_class);
-    // host copy of the graph: the forward pass builds its transposed forest from it on first use
+    h->h_wf_part.assign(W, 0);
+    h->h_wf_local.resize(W);
+    for (uint32_t w = 0; w < W; ++w) h->h_wf_local[w] = w;
+    // host copy of the graph: appended nodes and the forward pass rebuild slices of it
     h->h_row.assign(row_ptr, row_ptr + N + 1);
     h->h_col.assign(col_idx, col_idx + E);
     h->h_cost.assign(node_costs, node_costs + N);
+    h->h_elapsed = std::move(el);
+    h->h_base_perm = std::move(hf.perm);
+    h->h_base_wns = std::move(hf.wf_node_start);
+    h->extra_succ.clear(); h->extra_nodes.clear();
+    h->h_local.assign(N, ~0u);
     h->dag_uploaded = true;
+    return HX_OK;
+}
+
+// One horizon pass over every live workflow of every part.
+static int launch_all_parts(hx_cluster* h, cudaStream_t s) {
+    std::vector<HxCpClass> cls;
+    for (auto& p : h->parts) {
+        if (!p.live) continue;
+        p.classes(&cls);
+        HX_TRY(hx_launch_cpath(p.f, cls.data(), (int)cls.size(), s, &h->launches, &h->fj), "horizon kernels");
+    }
     return HX_OK;
 }
 
@@ -498,8 +610,7 @@ int hx_critical_path(hx_cluster* h, void* stream) {
     DeviceGuard guard(h->device);
     {
         SpanGuard span(h, 2, static_cast<cudaStream_t>(stream));
-        HX_TRY(hx_launch_cpath(h->forest, h->classes.data(), (int)h->classes.size(),
-                               static_cast<cudaStream_t>(stream), &h->launches, &h->fj), "horizon kernels");
+        if (int rc = launch_all_parts(h, static_cast<cudaStream_t>(stream))) return rc;
     }
     h->cp_ready = true;
     return HX_OK;
@@ -509,12 +620,13 @@ int hx_dag_update_elapsed(hx_cluster* h, const float* workflow_elapsed_s, void* 
     if (!h) return HX_ERR_INVALID_ARG;
     if (!h->dag_uploaded) return fail(h, HX_ERR_NOT_READY, "no forest uploaded");
     if (!workflow_elapsed_s) return fail(h, HX_ERR_INVALID_ARG, "NULL array");
-    const uint32_t W = h->forest.n_workflows;
+    const uint32_t W = h->W;
     for (uint32_t w = 0; w < W; ++w)
         if (!good_load(workflow_elapsed_s[w])) return fail(h, HX_ERR_INVALID_ARG, "elapsed times must be finite and >= 0");
     DeviceGuard guard(h->device);
     HX_TRY(cudaMemcpyAsync(h->d_elapsed, workflow_elapsed_s, (size_t)W * sizeof(float), cudaMemcpyHostToDevice,
                            static_cast<cudaStream_t>(stream)), "cudaMemcpyAsync(elapsed)");
+    h->h_elapsed.assign(workflow_elapsed_s, workflow_elapsed_s + W);
     return HX_OK;
 }
 
@@ -524,16 +636,19 @@ int hx_dag_update_costs(hx_cluster* h, const uint32_t* node_ids, const float* ne
     if (!h->dag_uploaded) return fail(h, HX_ERR_NOT_READY, "no forest uploaded");
     if (n_updates == 0) return HX_OK;
     if (!node_ids || !new_costs) return fail(h, HX_ERR_INVALID_ARG, "NULL array");
-    const uint32_t N = h->forest.n_nodes, W = h->forest.n_workflows;
+    const uint32_t N = h->N;
     for (uint32_t i = 0; i < n_updates; ++i) {
         if (node_ids[i] >= N) return fail(h, HX_ERR_INVALID_ARG, "node id out of range");
         if (!good_load(new_costs[i])) return fail(h, HX_ERR_INVALID_ARG, "node costs must be finite and >= 0");
     }
-    // the last value given for a node wins; the workflows touched are recomputed, nothing else
+    // the last value given for a node wins; the workflows touched are recomputed, nothing else.
+    // Nodes are grouped by the part that owns their workflow; the transposed forest is one more group.
+    struct Group { const HxForestDev* f; std::vector<uint32_t> idx; std::vector<float> val; std::vector<uint32_t> dirty[HX_CP_CLASSES]; };
     const bool fwd = h->fwd_built;
-    std::vector<uint32_t> idx; std::vector<float> val;
-    idx.reserve((fwd ? 2 : 1) * (size_t)n_updates); val.reserve(n_updates);
-    std::vector<uint32_t> dirty[HX_CP_CLASSES], fdirty[HX_CP_CLASSES];
+    std::vector<Group> groups(h->parts.size() + 1);
+    for (size_t q = 0; q < h->parts.size(); ++q) groups[q].f = &h->parts[q].f;
+    Group& gf = groups.back();
+    gf.f = &h->fwd;
     {
         std::vector<uint32_t> order(n_updates);
         for (uint32_t i = 0; i < n_updates; ++i) order[i] = i;
@@ -541,87 +656,80 @@ int hx_dag_update_costs(hx_cluster* h, const uint32_t* node_ids, const float* ne
         std::vector<uint32_t> wfs;
         for (uint32_t i = 0; i < n_updates; ++i) {
             if (i + 1 < n_updates && node_ids[order[i + 1]] == node_ids[order[i]]) continue;
-            const uint32_t v = node_ids[order[i]];
-            idx.push_back(h->h_inv[v]); val.push_back(new_costs[order[i]]);
-            wfs.push_back(h->h_node_wf[v]);
-            h->h_cost[v] = new_costs[order[i]];
+            const uint32_t v = node_ids[order[i]], w = h->h_node_wf[v];
+            const float c = new_costs[order[i]];
+            Group& g = groups[h->h_wf_part[w]];
+            g.idx.push_back(h->h_inv[v]); g.val.push_back(c);
+            if (fwd) { gf.idx.push_back(h->h_fwd_inv[v]); gf.val.push_back(c); }
+            wfs.push_back(w);
+            h->h_cost[v] = c;
         }
         std::sort(wfs.begin(), wfs.end());
         wfs.erase(std::unique(wfs.begin(), wfs.end()), wfs.end());
-        for (uint32_t w : wfs) dirty[h->h_wf_class[w]].push_back(w);
-        if (fwd) {
-            // second half of idx: the same nodes in the numbering of the transposed forest
-            for (uint32_t i = 0; i < n_updates; ++i) {
-                if (i + 1 < n_updates && node_ids[order[i + 1]] == node_ids[order[i]]) continue;
-                idx.push_back(h->h_fwd_inv[node_ids[order[i]]]);
-            }
-            for (uint32_t w : wfs) fdirty[h->h_fwd_wf_class[w]].push_back(w);
+        for (uint32_t w : wfs) {
+            const uint32_t q = h->h_wf_part[w], l = h->h_wf_local[w];
+            groups[q].dirty[h->parts[q].wf_class[l]].push_back(l);
+            if (fwd) gf.dirty[h->h_fwd_wf_class[w]].push_back(w);
         }
     }
-    const size_t n_set = val.size();
     DeviceGuard guard(h->device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    size_t n_wf = 0;
-    for (auto& v : dirty) n_wf += v.size();
-    for (auto& v : fdirty) n_wf += v.size();
-    if (idx.size() > h->upd_cap || n_wf > h->upd_wf_cap) {
+    size_t n_idx = 0, n_wf = 0;
+    for (auto& g : groups) { n_idx += g.idx.size(); for (auto& v : g.dirty) n_wf += v.size(); }
+    if (n_idx > h->upd_cap || n_wf > h->upd_wf_cap) {
         cudaDeviceSynchronize();
         free_pool(h->upd_allocs);
-        h->upd_cap = std::max<size_t>(idx.size(), 4096); h->upd_wf_cap = std::max<size_t>(n_wf, 4096);
+        h->upd_cap = std::max<size_t>(n_idx, 4096); h->upd_wf_cap = std::max<size_t>(n_wf, 4096);
         HX_TRY(dev_alloc(h->upd_allocs, &h->d_upd_idx, h->upd_cap), "alloc update scratch");
         HX_TRY(dev_alloc(h->upd_allocs, &h->d_upd_cost, h->upd_cap), "alloc update scratch");
         HX_TRY(dev_alloc(h->upd_allocs, &h->d_upd_wf, h->upd_wf_cap), "alloc update scratch");
     }
-    HX_TRY(cudaMemcpyAsync(h->d_upd_idx, idx.data(), idx.size() * sizeof(uint32_t), cudaMemcpyHostToDevice, s), "copy updates");
-    HX_TRY(cudaMemcpyAsync(h->d_upd_cost, val.data(), val.size() * sizeof(float), cudaMemcpyHostToDevice, s), "copy updates");
-    std::vector<HxCpClass> part, fpart;
-    size_t off = 0;
-    for (int pass = 0; pass < 2; ++pass)
+    // pageable host memory: every copy below has read its vector by the time it returns
+    SpanGuard span(h, 2, s);
+    size_t off = 0, woff = 0;
+    std::vector<HxCpClass> part;
+    for (size_t q = 0; q < groups.size(); ++q) {
+        Group& g = groups[q];
+        if (g.idx.empty()) continue;
+        const bool is_fwd = q + 1 == groups.size();
+        HX_TRY(cudaMemcpyAsync(h->d_upd_idx + off, g.idx.data(), g.idx.size() * sizeof(uint32_t), cudaMemcpyHostToDevice, s), "copy updates");
+        HX_TRY(cudaMemcpyAsync(h->d_upd_cost + off, g.val.data(), g.val.size() * sizeof(float), cudaMemcpyHostToDevice, s), "copy updates");
+        HX_TRY(hx_launch_cost_update(*g.f, h->d_upd_idx + off, h->d_upd_cost + off, (uint32_t)g.idx.size(), s, &h->launches), "cost update kernel");
+        off += g.idx.size();
+        part.clear();
         for (int k = 0; k < HX_CP_CLASSES; ++k) {
-            const std::vector<uint32_t>& dk = pass ? fdirty[k] : dirty[k];
-            if (dk.empty()) continue;
-            HX_TRY(cudaMemcpyAsync(h->d_upd_wf + off, dk.data(), dk.size() * sizeof(uint32_t),
+            if (g.dirty[k].empty()) continue;
+            HX_TRY(cudaMemcpyAsync(h->d_upd_wf + woff, g.dirty[k].data(), g.dirty[k].size() * sizeof(uint32_t),
                                    cudaMemcpyHostToDevice, s), "copy dirty workflows");
             HxCpClass c = hx_cpath_class_shape(k);
-            c.wf_ids = h->d_upd_wf + off; c.count = (uint32_t)dk.size();
-            (pass ? fpart : part).push_back(c);
-            off += dk.size();
+            c.wf_ids = h->d_upd_wf + woff; c.count = (uint32_t)g.dirty[k].size();
+            part.push_back(c);
+            woff += g.dirty[k].size();
         }
-    // pageable host memory: the copies above have read the vectors by the time they return
-    {
-        SpanGuard span(h, 2, s);
-        HX_TRY(hx_launch_cost_update(h->forest, h->d_upd_idx, h->d_upd_cost, (uint32_t)n_set, s, &h->launches), "cost update kernel");
-        if (h->cp_ready)
-            HX_TRY(hx_launch_cpath(h->forest, part.data(), (int)part.size(), s, &h->launches, &h->fj), "horizon kernels");
-        if (fwd) {
-            HX_TRY(hx_launch_cost_update(h->fwd, h->d_upd_idx + n_set, h->d_upd_cost, (uint32_t)n_set, s, &h->launches), "cost update kernel");
-            if (h->est_ready)
-                HX_TRY(hx_launch_cpath(h->fwd, fpart.data(), (int)fpart.size(), s, &h->launches, &h->fj), "forward pass kernels");
-        }
+        if (is_fwd ? h->est_ready : h->cp_ready)
+            HX_TRY(hx_launch_cpath(*g.f, part.data(), (int)part.size(), s, &h->launches, &h->fj), "horizon kernels");
     }
-    (void)W;
     return HX_OK;
 }
 
 int hx_get_dag_results(hx_cluster* h, const float** cp, const float** tail, const float** H) {
     if (!h) return HX_ERR_INVALID_ARG;
     if (!h->dag_uploaded) return fail(h, HX_ERR_NOT_READY, "no forest uploaded");
-    if (cp) *cp = h->forest.cp;
-    if (tail) *tail = h->forest.tail;
-    if (H) *H = h->forest.H;
+    if (cp) *cp = h->g_cp;
+    if (tail) *tail = h->g_tail;
+    if (H) *H = h->g_H;
     return HX_OK;
 }
 
 // Builds the transposed forest (every edge reversed) for the forward pass.
 static int build_forward_forest(hx_cluster* h) {
-    const uint32_t N = h->forest.n_nodes, E = h->forest.n_edges, W = h->forest.n_workflows;
+    const uint32_t N = h->N, E = h->E, W = h->W;
     std::vector<uint32_t> trow((size_t)N + 1, 0), tcol(E);
-    for (uint32_t e = 0; e < E; ++e) ++trow[h->h_col[e] + 1];
+    for (uint32_t v = 0; v < N; ++v) for_each_successor(h, v, [&](uint32_t u) { ++trow[u + 1]; });
     for (uint32_t v = 0; v < N; ++v) trow[v + 1] += trow[v];
     {
         std::vector<uint32_t> cur(trow.begin(), trow.end() - 1);
-        for (uint32_t v = 0; v < N; ++v)
-            for (uint32_t e = h->h_row[v]; e < h->h_row[v + 1]; ++e) tcol[cur[h->h_col[e]]++] = v;
+        for (uint32_t v = 0; v < N; ++v) for_each_successor(h, v, [&](uint32_t u) { tcol[cur[u]++] = v; });
     }
     HostForest hf;
     if (!prepare_forest(trow.data(), tcol.data(), h->h_cost.data(), h->h_node_wf.data(), N, E, W, &hf))
@@ -629,12 +737,16 @@ static int build_forward_forest(hx_cluster* h) {
     cudaDeviceSynchronize();
     free_pool(h->fwd_allocs);
     h->fwd_built = false; h->est_ready = false;
-    HxForestDev f{};
-    HX_TRY(dev_alloc(h->fwd_allocs, &f.cp, N), "alloc earliest finish");
-    HX_TRY(dev_alloc(h->fwd_allocs, &f.tail, N), "alloc earliest start");
-    HX_TRY(dev_alloc(h->fwd_allocs, &f.H, W), "alloc forward horizon");
-    if (int rc = upload_forest(h, h->fwd_allocs, hf, &f, &h->fwd_classes)) return rc;
-    h->fwd = f;
+    ForestPart tmp;
+    HX_TRY(dev_alloc(h->fwd_allocs, &tmp.f.cp, N), "alloc earliest finish");
+    HX_TRY(dev_alloc(h->fwd_allocs, &tmp.f.tail, N), "alloc earliest start");
+    HX_TRY(dev_alloc(h->fwd_allocs, &tmp.f.H, W), "alloc forward horizon");
+    const int rc = upload_forest(h, hf, &tmp);
+    h->fwd_allocs.insert(h->fwd_allocs.end(), tmp.allocs.begin(), tmp.allocs.end());
+    tmp.allocs.clear();
+    if (rc) return rc;
+    h->fwd = tmp.f;
+    tmp.classes(&h->fwd_classes);
     h->h_fwd_inv = std::move(hf.inv);
     h->h_fwd_wf_class = std::move(hf.wf_class);
     h->fwd_built = true;
@@ -661,6 +773,165 @@ int hx_get_earliest_results(hx_cluster* h, const float** est, const float** eft)
     if (!h->fwd_built) return fail(h, HX_ERR_NOT_READY, "no forward pass yet: call hx_earliest_start");
     if (est) *est = h->fwd.tail;
     if (eft) *eft = h->fwd.cp;
+    return HX_OK;
+}
+
+// Too many parts make a full pass a long chain of small launches: regroup the whole graph as one upload.
+static const size_t kMaxParts = 64;
+static int rebuild_as_one_part(hx_cluster* h, cudaStream_t s) {
+    const uint32_t N = h->N, E = h->E, W = h->W;
+    std::vector<uint32_t> row((size_t)N + 1, 0), col;
+    col.reserve(E);
+    for (uint32_t v = 0; v < N; ++v) {
+        for_each_successor(h, v, [&](uint32_t u) { col.push_back(u); });
+        row[v + 1] = (uint32_t)col.size();
+    }
+    const std::vector<float> cost = h->h_cost, el = h->h_elapsed;      // the upload replaces the members
+    const std::vector<uint32_t> nwf = h->h_node_wf;
+    const bool had_cp = h->cp_ready;
+    int rc = hx_dag_upload(h, row.data(), col.data(), cost.data(), nwf.data(), el.data(), N, E, W);
+    if (rc == HX_OK && had_cp) rc = hx_critical_path(h, s);
+    return rc;
+}
+
+// Room for `need` nodes in cp, tail and the node -> workflow map; the arrays move when they grow.
+static int reserve_nodes(hx_cluster* h, size_t need) {
+    if (need <= h->capN) return HX_OK;
+    const size_t cap = std::max(need, 2 * h->capN);
+    std::vector<void*> fresh;
+    float *cp, *tail; uint32_t* nwf;
+    cudaError_t e = dev_alloc(fresh, &cp, cap);
+    if (e == cudaSuccess) e = dev_alloc(fresh, &tail, cap);
+    if (e == cudaSuccess) e = dev_alloc(fresh, &nwf, cap);
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e == cudaSuccess) e = cudaMemcpy(cp, h->g_cp, (size_t)h->N * sizeof(float), cudaMemcpyDeviceToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(tail, h->g_tail, (size_t)h->N * sizeof(float), cudaMemcpyDeviceToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(nwf, h->d_node_wf, (size_t)h->N * sizeof(uint32_t), cudaMemcpyDeviceToDevice);
+    if (e != cudaSuccess) { free_pool(fresh); return fail_cuda(h, e, "growing the node arrays"); }
+    free_pool(h->node_allocs);
+    h->node_allocs = fresh;
+    h->g_cp = cp; h->g_tail = tail; h->d_node_wf = nwf; h->capN = cap;
+    for (auto& p : h->parts) { p.f.cp = cp; p.f.tail = tail; }
+    return HX_OK;
+}
+
+int hx_dag_append(hx_cluster* h, uint32_t n_new_nodes, const float* new_costs, const uint32_t* new_node_workflow,
+                  uint32_t n_new_edges, const uint32_t* edge_src, const uint32_t* edge_dst, void* stream) {
+    if (!h) return HX_ERR_INVALID_ARG;
+    if (!h->dag_uploaded) return fail(h, HX_ERR_NOT_READY, "no forest uploaded");
+    if (n_new_nodes == 0 && n_new_edges == 0) return HX_OK;
+    if ((n_new_nodes && (!new_costs || !new_node_workflow)) || (n_new_edges && (!edge_src || !edge_dst)))
+        return fail(h, HX_ERR_INVALID_ARG, "NULL array");
+    const uint32_t N0 = h->N, W = h->W;
+    if ((uint64_t)N0 + n_new_nodes > 0xFFFFFFF0ull || (uint64_t)h->E + n_new_edges > 0xFFFFFFF0ull)
+        return fail(h, HX_ERR_INVALID_ARG, "more than 2^32 nodes or edges");
+    const uint32_t N1 = N0 + n_new_nodes;
+    auto wf_of = [&](uint32_t v) { return v < N0 ? h->h_node_wf[v] : new_node_workflow[v - N0]; };
+    for (uint32_t i = 0; i < n_new_nodes; ++i) {
+        if (new_node_workflow[i] >= W) return fail(h, HX_ERR_INVALID_ARG, "workflow id out of range");
+        if (!good_load(new_costs[i])) return fail(h, HX_ERR_INVALID_ARG, "node costs must be finite and >= 0");
+    }
+    for (uint32_t e = 0; e < n_new_edges; ++e) {
+        if (edge_src[e] >= N1 || edge_dst[e] >= N1) return fail(h, HX_ERR_INVALID_ARG, "edge endpoint out of range");
+        if (wf_of(edge_src[e]) != wf_of(edge_dst[e])) return fail(h, HX_ERR_INVALID_ARG, "edge crosses workflows");
+    }
+    // workflows touched, in increasing order: they are rebuilt as one new part
+    std::vector<uint32_t> touched;
+    for (uint32_t i = 0; i < n_new_nodes; ++i) touched.push_back(new_node_workflow[i]);
+    for (uint32_t e = 0; e < n_new_edges; ++e) touched.push_back(wf_of(edge_src[e]));
+    std::sort(touched.begin(), touched.end());
+    touched.erase(std::unique(touched.begin(), touched.end()), touched.end());
+    // nodes of those workflows: uploaded ones, ones appended earlier, new ones
+    std::vector<uint32_t> gid, lwf;                      // local node -> node number, local node -> local workflow
+    // node number -> local node: a table over all nodes that is kept between calls; the entries set
+    // here are cleared again on every way out
+    struct LocalTable {
+        std::vector<uint32_t>& t; const std::vector<uint32_t>& used;
+        ~LocalTable() { for (uint32_t v : used) t[v] = ~0u; }
+        uint32_t at(uint32_t v) const { return t[v]; }
+    };
+    h->h_local.resize(N1, ~0u);
+    LocalTable local{h->h_local, gid};
+    std::vector<std::vector<uint32_t>> fresh(touched.size());
+    for (uint32_t i = 0; i < n_new_nodes; ++i) {
+        const size_t j = std::lower_bound(touched.begin(), touched.end(), new_node_workflow[i]) - touched.begin();
+        fresh[j].push_back(N0 + i);
+    }
+    for (size_t j = 0; j < touched.size(); ++j) {
+        const uint32_t w = touched[j];
+        auto add = [&](uint32_t v) { h->h_local[v] = (uint32_t)gid.size(); gid.push_back(v); lwf.push_back((uint32_t)j); };
+        for (uint32_t i = h->h_base_wns[w]; i < h->h_base_wns[w + 1]; ++i) add(h->h_base_perm[i]);
+        auto it = h->extra_nodes.find(w);
+        if (it != h->extra_nodes.end()) for (uint32_t v : it->second) add(v);
+        for (uint32_t v : fresh[j]) add(v);
+    }
+    const uint32_t n = (uint32_t)gid.size();
+    // their edges: old ones, then the new ones
+    std::vector<std::vector<uint32_t>> extra(n);
+    for (uint32_t e = 0; e < n_new_edges; ++e) extra[local.at(edge_src[e])].push_back(local.at(edge_dst[e]));
+    std::vector<uint32_t> row((size_t)n + 1, 0), col;
+    std::vector<float> cost(n);
+    for (uint32_t i = 0; i < n; ++i) {
+        const uint32_t v = gid[i];
+        cost[i] = v < N0 ? h->h_cost[v] : new_costs[v - N0];
+        if (v < N0) for_each_successor(h, v, [&](uint32_t u) { col.push_back(local.at(u)); });
+        for (uint32_t u : extra[i]) col.push_back(u);
+        row[i + 1] = (uint32_t)col.size();
+    }
+    HostForest hf;
+    if (!prepare_forest(row.data(), col.data(), cost.data(), lwf.data(), n, (uint32_t)col.size(), (uint32_t)touched.size(), &hf))
+        return fail(h, HX_ERR_CYCLE, "the new edges close a cycle");     // nothing has changed so far
+
+    DeviceGuard guard(h->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (int rc = reserve_nodes(h, N1)) return rc;
+    // a free slot, else a new one
+    size_t q = 1;
+    while (q < h->parts.size() && (h->parts[q].live || !h->parts[q].allocs.empty())) ++q;
+    if (q >= h->parts.size()) h->parts.emplace_back();
+    {
+        ForestPart fresh_part;
+        fresh_part.f.cp = h->g_cp; fresh_part.f.tail = h->g_tail; fresh_part.f.H = h->g_H;
+        int rc = upload_forest(h, hf, &fresh_part, &gid, &touched);
+        if (!rc && n_new_nodes) {
+            const cudaError_t e = cudaMemcpyAsync(h->d_node_wf + N0, new_node_workflow, (size_t)n_new_nodes * sizeof(uint32_t),
+                                                  cudaMemcpyHostToDevice, s);
+            if (e != cudaSuccess) rc = fail_cuda(h, e, "copy node_workflow");
+        }
+        if (rc) { free_pool(fresh_part.allocs); return rc; }
+        h->parts[q] = std::move(fresh_part);
+    }
+    // from here on nothing fails: commit the host state
+    h->h_node_wf.insert(h->h_node_wf.end(), new_node_workflow, new_node_workflow + n_new_nodes);
+    h->h_cost.insert(h->h_cost.end(), new_costs, new_costs + n_new_nodes);
+    h->h_inv.resize(N1);
+    for (uint32_t i = 0; i < n; ++i) h->h_inv[gid[i]] = hf.inv[i];
+    for (size_t j = 0; j < touched.size(); ++j) {
+        const uint32_t w = touched[j];
+        h->parts[h->h_wf_part[w]].drop(h->h_wf_local[w]);
+        h->h_wf_part[w] = (uint32_t)q; h->h_wf_local[w] = (uint32_t)j;
+        if (!fresh[j].empty()) {
+            auto& v = h->extra_nodes[w];
+            v.insert(v.end(), fresh[j].begin(), fresh[j].end());
+        }
+    }
+    for (uint32_t e = 0; e < n_new_edges; ++e) h->extra_succ[edge_src[e]].push_back(edge_dst[e]);
+    h->N = N1; h->E += n_new_edges;
+    for (auto& p : h->parts)
+        if (p.live) HX_TRY(p.flush(s), "updating the class lists");
+    // parts that own nothing any more give their memory back (cudaFree waits for the work in flight)
+    for (size_t i = 1; i < h->parts.size(); ++i)
+        if (!h->parts[i].live && !h->parts[i].allocs.empty()) { free_pool(h->parts[i].allocs); h->parts[i] = ForestPart{}; }
+    h->fwd_built = false; h->est_ready = false;          // the transposed forest is rebuilt at the next forward pass
+    size_t n_live = 0;
+    for (auto& p : h->parts) n_live += p.live != 0;
+    if (n_live > kMaxParts) return rebuild_as_one_part(h, s);
+    if (h->cp_ready) {
+        SpanGuard span(h, 2, s);
+        std::vector<HxCpClass> cls;
+        h->parts[q].classes(&cls);
+        HX_TRY(hx_launch_cpath(h->parts[q].f, cls.data(), (int)cls.size(), s, &h->launches, &h->fj), "horizon kernels");
+    }
     return HX_OK;
 }
 
@@ -703,7 +974,7 @@ int hx_schedule_batch(hx_cluster* h, const hx_call* calls, int n_calls, int32_t*
     }
     HxDagView dag{};
     if (!(o.flags & HX_FLAG_NO_DAG))
-        dag = HxDagView{h->d_node_wf, h->forest.tail, h->forest.H, h->d_elapsed, h->forest.n_nodes, h->forest.n_workflows};
+        dag = HxDagView{h->d_node_wf, h->g_tail, h->g_H, h->d_elapsed, h->N, h->W};
     HxTopkBufs tk = h->tk;
     tk.K = o.topk;
     ScoreLaunch sl{calls, n_calls, out_assign, out_cost, o.score_mode, o.flags, o.topk, o.alpha};
@@ -836,7 +1107,7 @@ int hx_schedule_batch_static(hx_cluster* h, const hx_call* calls, int n_calls, i
     if (off != kStaticBytes) return fail(h, HX_ERR_INVALID_ARG, "internal: static scratch layout mismatch");
     HxDagView dag{};
     if (!(o.flags & HX_FLAG_NO_DAG))
-        dag = HxDagView{h->d_node_wf, h->forest.tail, h->forest.H, h->d_elapsed, h->forest.n_nodes, h->forest.n_workflows};
+        dag = HxDagView{h->d_node_wf, h->g_tail, h->g_H, h->d_elapsed, h->N, h->W};
     ScoreLaunch sl{calls, n_calls, out_assign, out_cost, o.score_mode, o.flags, o.topk, o.alpha};
     HX_TRY(hx_launch_score(h->tab, h->ctab, dag, b, sl, h->n_sm, h->max_smem, h->status, s, &h->launches), "scoring kernel");
     if (o.topk > 0)
@@ -863,7 +1134,7 @@ int hx_schedule_greedy(hx_cluster* h, const hx_call* calls, int n_calls, int32_t
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     HxDagView dag{};
     if (!(o.flags & HX_FLAG_NO_DAG))
-        dag = HxDagView{h->d_node_wf, h->forest.tail, h->forest.H, h->d_elapsed, h->forest.n_nodes, h->forest.n_workflows};
+        dag = HxDagView{h->d_node_wf, h->g_tail, h->g_H, h->d_elapsed, h->N, h->W};
     {
         SpanGuard span(h, 0, s);
         HX_TRY(hx_launch_greedy(h->tab, h->ctab, dag, calls, n_calls, o.flags, o.commit, out_assign, out_ratio,
@@ -975,7 +1246,7 @@ int hx_schedule_decode(hx_cluster* h, const hx_call* calls, const int32_t* lock,
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     HxDagView dag{};
     if (!(o.flags & HX_FLAG_NO_DAG))
-        dag = HxDagView{h->d_node_wf, h->forest.tail, h->forest.H, h->d_elapsed, h->forest.n_nodes, h->forest.n_workflows};
+        dag = HxDagView{h->d_node_wf, h->g_tail, h->g_H, h->d_elapsed, h->N, h->W};
     {
         SpanGuard span(h, 0, s);
         HX_TRY(hx_launch_decode(h->tab, h->ctab, dag, h->dec_base, h->dec_work, calls, lock, ready_s, n_calls, o.flags,

@@ -106,6 +106,7 @@ struct HxForestDev {
     const uint32_t* icol32;          // [E] same, 32-bit
     const float* icost;              // [N]
     const uint32_t* perm;            // [N] internal -> original node number
+    const uint32_t* wf_gid;          // [W] workflow number of the caller for H, or NULL when it is w itself
     float* cp;                       // [N] original numbering
     float* tail;                     // [N]
     float* H;                        // [W]
