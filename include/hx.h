@@ -319,6 +319,15 @@ int hx_schedule_batch_static(hx_cluster* h, const hx_call* calls, int n_calls,
 int hx_schedule_greedy(hx_cluster* h, const hx_call* calls, int n_calls,
                        int32_t* out_assign, float* out_ratio, int32_t* out_order, void* stream);
 
+/* hx_schedule_greedy with one more output: out_delta, device float[n_calls], the
+ * projected completion Delta (seconds from now) of each call on the pair it was
+ * given, i.e. the Delta inside its ratio (Eq. 2), projected against the
+ * simulated state at the moment the call was taken; +inf if never taken.  May
+ * be NULL, which makes the call hx_schedule_greedy. */
+int hx_schedule_greedy_plan(hx_cluster* h, const hx_call* calls, int n_calls,
+                            int32_t* out_assign, float* out_ratio, int32_t* out_order,
+                            float* out_delta, void* stream);
+
 /* Decode-stage scheduler (Section 5.4, "Decode scheduling with instance locks",
  * "Decode KV-capacity feasibility check", "Adaptive greedy decode assignment").
  * State: the decode token-capacity intervals of every decode instance

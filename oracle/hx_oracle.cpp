@@ -276,17 +276,21 @@ int orc_conflict(int C, int K, int D, const int32_t* pair, const float* prio, co
 // loop ends when no waiting call has one (the state never improves).
 // Outputs: assign[c] pair or -1, ratio[c] = R at the moment of selection (+inf
 // if never placed), order[i] = call taken in iteration i (-1 past the end);
-// qP[P] and freeD[D] are updated in place.  Returns the number of placed calls.
+// qP[P] and freeD[D] are updated in place; delta[c] (may be NULL) = the Delta
+// inside ratio[c], +inf if never placed.  Returns the number of placed calls.
 int orc_greedy(const OrcCluster* cl, const OrcDag* dag, const OrcCall* calls, int C, int flags,
-               float* qP, float* freeD, int32_t* assign, float* ratio, int32_t* order) {
+               float* qP, float* freeD, int32_t* assign, float* ratio, int32_t* order, float* delta_out) {
     OrcCluster sim = *cl;
     sim.qP = qP;                                        // candidate_fin reads the simulated queues
     std::vector<char> waiting(C, 1);
     std::vector<Terms> terms(C);
-    for (int c = 0; c < C; ++c) { latency_terms(*cl, calls[c], terms[c]); assign[c] = -1; ratio[c] = INF; order[c] = -1; }
+    for (int c = 0; c < C; ++c) {
+        latency_terms(*cl, calls[c], terms[c]); assign[c] = -1; ratio[c] = INF; order[c] = -1;
+        if (delta_out) delta_out[c] = INF;
+    }
     int placed = 0;
     for (int it = 0; it < C; ++it) {
-        int best_c = -1, best_j = -1; float best_R = -INF;
+        int best_c = -1, best_j = -1; float best_R = -INF, best_delta = INF;
         for (int c = 0; c < C; ++c) {
             if (!waiting[c]) continue;
             const Terms& t = terms[c];
@@ -300,11 +304,12 @@ int orc_greedy(const OrcCluster* cl, const OrcDag* dag, const OrcCall* calls, in
             if (arg < 0) continue;
             const DagView v = dag_view(dag, calls[c], flags);
             const float R = (v.elapsed + delta) / v.H;          // Eq. 2
-            if (R > best_R) { best_R = R; best_c = c; best_j = arg; }
+            if (R > best_R) { best_R = R; best_c = c; best_j = arg; best_delta = delta; }
         }
         if (best_c < 0) break;
         const int p = best_j / cl->D, d = best_j % cl->D;
         assign[best_c] = best_j; ratio[best_c] = best_R; order[it] = best_c;
+        if (delta_out) delta_out[best_c] = best_delta;
         qP[p] = qP[p] + terms[best_c].tpre[cl->typeP[p]];
         freeD[d] = freeD[d] - terms[best_c].m;
         waiting[best_c] = 0;

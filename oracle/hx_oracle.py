@@ -205,11 +205,13 @@ class Oracle:
         return assign, freeD, qP
 
     def greedy(self, cl: Cluster, calls, freeD, flags=0, dag: DagResult | None = None, node_wf=None,
-               elapsed=None):
+               elapsed=None, with_delta=False):
         """Recomputing greedy of Algorithm 1 over one queue snapshot.
-        Returns (assign i32[C], ratio f32[C], order i32[C], n_placed, qP', freeD')."""
+        Returns (assign i32[C], ratio f32[C], order i32[C], n_placed, qP', freeD'), plus delta f32[C] with
+        with_delta."""
         calls, n = self._calls(calls)
         assign = np.zeros(n, np.int32); ratio = np.zeros(n, np.float32); order = np.zeros(n, np.int32)
+        delta = np.zeros(n, np.float32)
         qP = _f32(cl.qP).copy(); free = _f32(freeD).copy()
         c = cl._c()
         d, keep = self._dag(dag, node_wf, elapsed)
@@ -217,7 +219,10 @@ class Oracle:
             flags |= FLAG_NO_DAG
         self.lib.orc_greedy.restype = C.c_int
         placed = self.lib.orc_greedy(C.byref(c), C.byref(d) if d is not None else None, _ptr(calls), n,
-                                     int(flags), _ptr(qP), _ptr(free), _ptr(assign), _ptr(ratio), _ptr(order))
+                                     int(flags), _ptr(qP), _ptr(free), _ptr(assign), _ptr(ratio), _ptr(order),
+                                     _ptr(delta) if with_delta else None)
+        if with_delta:
+            return assign, ratio, order, int(placed), qP, free, delta
         return assign, ratio, order, int(placed), qP, free
 
     def decode_greedy(self, cl: Cluster, calls, run_ptr, run_end, run_tok, lock, ready, flags=0,

@@ -65,6 +65,7 @@ def _load():
         "hx_schedule_batch_host_async": [vp, vp, ci, vp, vp, vp],
         "hx_schedule_batch_static": [vp, vp, ci, vp, vp, vp],
         "hx_schedule_greedy": [vp, vp, ci, vp, vp, vp, vp],
+        "hx_schedule_greedy_plan": [vp, vp, ci, vp, vp, vp, vp, vp],
         "hx_decode_set_running": [vp, vp, vp, vp],
         "hx_schedule_decode": [vp, vp, vp, vp, ci, vp, vp, vp, vp, vp],
         "hx_get_topk": [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp)],
@@ -209,6 +210,13 @@ def hx_schedule_greedy(h, calls_ptr, n_calls, out_assign_ptr, out_ratio_ptr, out
     """Recomputing greedy planner for small queues (Algorithm 1); device pointers."""
     _check(_lib.hx_schedule_greedy(h, calls_ptr, int(n_calls), out_assign_ptr, out_ratio_ptr, out_order_ptr,
                                    stream), h)
+
+
+def hx_schedule_greedy_plan(h, calls_ptr, n_calls, out_assign_ptr, out_ratio_ptr, out_order_ptr, out_delta_ptr,
+                            stream=0):
+    """hx_schedule_greedy plus the projected completion Delta of every call; device pointers."""
+    _check(_lib.hx_schedule_greedy_plan(h, calls_ptr, int(n_calls), out_assign_ptr, out_ratio_ptr, out_order_ptr,
+                                        out_delta_ptr, stream), h)
 
 
 KV_INTERVAL_DTYPE = np.dtype([("end_s", "<f4"), ("tokens", "<f4")])
@@ -398,8 +406,8 @@ class Cluster:
         hx_schedule_batch(self.h, calls.data_ptr(), n, out_assign.data_ptr(), out_cost.data_ptr(), self._stream())
         return out_assign, out_cost
 
-    def schedule_greedy(self, calls):
-        """calls as for schedule_batch.  Returns (assign, ratio, order) CUDA tensors."""
+    def schedule_greedy(self, calls, with_delta=False):
+        """calls as for schedule_batch.  Returns (assign, ratio, order) CUDA tensors, plus delta on request."""
         import torch
         if isinstance(calls, np.ndarray):
             calls = torch.from_numpy(_np(calls, CALL_DTYPE).view(np.uint8).copy()).cuda()
@@ -407,9 +415,14 @@ class Cluster:
         assign = torch.empty(n, dtype=torch.int32, device="cuda")
         ratio = torch.empty(n, dtype=torch.float32, device="cuda")
         order = torch.empty(n, dtype=torch.int32, device="cuda")
-        hx_schedule_greedy(self.h, calls.data_ptr(), n, assign.data_ptr(), ratio.data_ptr(), order.data_ptr(),
-                           self._stream())
-        return assign, ratio, order
+        if not with_delta:
+            hx_schedule_greedy(self.h, calls.data_ptr(), n, assign.data_ptr(), ratio.data_ptr(), order.data_ptr(),
+                               self._stream())
+            return assign, ratio, order
+        delta = torch.empty(n, dtype=torch.float32, device="cuda")
+        hx_schedule_greedy_plan(self.h, calls.data_ptr(), n, assign.data_ptr(), ratio.data_ptr(), order.data_ptr(),
+                                delta.data_ptr(), self._stream())
+        return assign, ratio, order, delta
 
     def decode_set_running(self, inst_ptr, end_s, tokens):
         run = np.zeros(len(end_s), KV_INTERVAL_DTYPE)

@@ -47,6 +47,7 @@ struct GreedyParams {
     int32_t* out_assign;
     float* out_ratio;
     int32_t* out_order;
+    float* out_delta;          // may be NULL
     int* status;
 };
 
@@ -104,6 +105,7 @@ __global__ void __launch_bounds__(kThreads, 1) hx_greedy_kernel(const __grid_con
         cpair[c] = bad ? kDead : kNoPair;
         dirty[c] = (unsigned short)c;
         prm.out_assign[gcall] = -1; prm.out_ratio[gcall] = HX_INF; prm.out_order[gcall] = -1;
+        if (prm.out_delta) prm.out_delta[gcall] = HX_INF;
     }
     if (tid == 0) s_ndirty = n;
     __syncthreads();
@@ -214,6 +216,13 @@ __global__ void __launch_bounds__(kThreads, 1) hx_greedy_kernel(const __grid_con
                 prm.out_assign[rc] = p * D + d;
                 prm.out_ratio[rc] = rv;
                 prm.out_order[it] = rc;
+                if (prm.out_delta) {
+                    // Delta of the chosen pair: the projection that made the ratio, from the same state
+                    const float ctx = __fmaf_rn(0.5f, __fsub_rn(ot, 1.0f), nt);
+                    const float td = __fmul_rn(__fmul_rn(ot, __fmaf_rn(kappa, ctx, omega)), prm.ct.invB[typeDs[d]]);
+                    const float ready = __fmaf_rn(kvB, invL[p * D + d], __fadd_rn(qPs[p], tp));
+                    prm.out_delta[rc] = __fadd_rn(fmaxf(ready, qDs[d]), td);
+                }
                 cpair[li] = kDead; cR[li] = HX_NEG_INF;
                 if (NC > 1) {
                     cg::cluster_group cl = cg::this_cluster();
@@ -274,11 +283,12 @@ size_t hx_greedy_smem_bytes(const HxTables& t, int n_calls) {
 
 cudaError_t hx_launch_greedy(const HxTables& t, const HxConstTables& ct, const HxDagView& dag,
                              const hx_call* calls, int n_calls, int flags, int commit,
-                             int32_t* out_assign, float* out_ratio, int32_t* out_order, int* status,
+                             int32_t* out_assign, float* out_ratio, int32_t* out_order, float* out_delta, int* status,
                              cudaStream_t stream, long long* launches) {
     GreedyParams prm;
     prm.t = t; prm.ct = ct; prm.dag = dag; prm.calls = calls; prm.n = n_calls; prm.flags = flags; prm.commit = commit;
-    prm.out_assign = out_assign; prm.out_ratio = out_ratio; prm.out_order = out_order; prm.status = status;
+    prm.out_assign = out_assign; prm.out_ratio = out_ratio; prm.out_order = out_order; prm.out_delta = out_delta;
+    prm.status = status;
     cudaError_t e;
     if (n_calls > kClusterFrom) {
         const size_t smem = greedy_smem(t, (n_calls + kCluster - 1) / kCluster);

@@ -1117,6 +1117,11 @@ int hx_schedule_batch_static(hx_cluster* h, const hx_call* calls, int n_calls, i
 
 int hx_schedule_greedy(hx_cluster* h, const hx_call* calls, int n_calls, int32_t* out_assign,
                        float* out_ratio, int32_t* out_order, void* stream) {
+    return hx_schedule_greedy_plan(h, calls, n_calls, out_assign, out_ratio, out_order, nullptr, stream);
+}
+
+int hx_schedule_greedy_plan(hx_cluster* h, const hx_call* calls, int n_calls, int32_t* out_assign,
+                            float* out_ratio, int32_t* out_order, float* out_delta, void* stream) {
     if (!h) return HX_ERR_INVALID_ARG;
     if (n_calls < 0) return fail(h, HX_ERR_INVALID_ARG, "negative n_calls");
     if (n_calls == 0) return HX_OK;
@@ -1138,7 +1143,7 @@ int hx_schedule_greedy(hx_cluster* h, const hx_call* calls, int n_calls, int32_t
     {
         SpanGuard span(h, 0, s);
         HX_TRY(hx_launch_greedy(h->tab, h->ctab, dag, calls, n_calls, o.flags, o.commit, out_assign, out_ratio,
-                                out_order, h->status, s, &h->launches), "greedy planner kernel");
+                                out_order, out_delta, h->status, s, &h->launches), "greedy planner kernel");
     }
     return HX_OK;
 }

@@ -123,7 +123,7 @@ cudaError_t hx_launch_conflict(const HxTables& t, const HxTopkBufs& tk, int n_ca
 size_t hx_greedy_smem_bytes(const HxTables& t, int n_calls);
 cudaError_t hx_launch_greedy(const HxTables& t, const HxConstTables& ct, const HxDagView& dag,
                              const hx_call* calls, int n_calls, int flags, int commit,
-                             int32_t* out_assign, float* out_ratio, int32_t* out_order, int* status,
+                             int32_t* out_assign, float* out_ratio, int32_t* out_order, float* out_delta, int* status,
                              cudaStream_t stream, long long* launches);
 
 // Tokens in use on every decode instance as step functions of time (decode token-capacity

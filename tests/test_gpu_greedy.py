@@ -25,9 +25,11 @@ def hx():
 
 def _compare(hx, gc, oc, oracle, calls, free0, P, D, dag=None, node_wf=None, elapsed=None, flags=0):
     gc.set_options(score_mode=hx.HX_MODE_RATIO, commit=1, flags=flags)
-    a, r, o = (t.cpu().numpy() for t in gc.schedule_greedy(calls))
-    ea, er, eo, placed, eq, ef = oracle.greedy(oc, calls, free0, dag=dag, node_wf=node_wf, elapsed=elapsed)
+    a, r, o, dl = (t.cpu().numpy() for t in gc.schedule_greedy(calls, with_delta=True))
+    ea, er, eo, placed, eq, ef, ed = oracle.greedy(oc, calls, free0, dag=dag, node_wf=node_wf, elapsed=elapsed,
+                                                   with_delta=True)
     assert np.array_equal(o, eo), "order differs"
+    assert np.array_equal(dl, ed), "projected completions differ"
     assert np.array_equal(a, ea), "pairs differ"
     hh.assert_costs_close(r, er, "ratios")
     assert np.array_equal(r, er)

@@ -78,11 +78,12 @@ def _python_loop(orc, cl, calls, freeD, dag, node_wf, el):
     tpre, _, _, m = orc.terms(cl, calls)
     waiting = list(range(C))
     assign = np.full(C, -1, np.int32); ratio = np.full(C, np.inf, np.float32); order = []
+    delta = np.full(C, np.inf, np.float32)
     while waiting:
         sim = _clone(cl, qP=qP, capD=np.minimum(cl.capD, free))
         idx = np.array(waiting)
-        a, r, _ = orc.schedule(sim, calls[idx], mode=ho.MODE_RATIO, flags=ho.FLAG_NO_TAIL, dag=dag,
-                               node_wf=node_wf, elapsed=el)
+        a, r, dl = orc.schedule(sim, calls[idx], mode=ho.MODE_RATIO, flags=ho.FLAG_NO_TAIL, dag=dag,
+                                node_wf=node_wf, elapsed=el)
         ok = np.flatnonzero(a >= 0)
         if ok.size == 0:
             break
@@ -91,10 +92,10 @@ def _python_loop(orc, cl, calls, freeD, dag, node_wf, el):
         p, d = divmod(j, cl.D)
         qP[p] = np.float32(qP[p] + tpre[c, cl.typeP[p]])
         free[d] = np.float32(free[d] - m[c])
-        assign[c], ratio[c] = j, r[k]
+        assign[c], ratio[c], delta[c] = j, r[k], dl[k]
         order.append(c)
         waiting.remove(c)
-    return assign, ratio, order, qP, free
+    return assign, ratio, order, qP, free, delta
 
 
 def test_greedy_equals_loop_around_the_one_shot_scorer(oracle):
@@ -105,10 +106,14 @@ def test_greedy_equals_loop_around_the_one_shot_scorer(oracle):
         dag, nwf, el = _dag(rng, C)
         _, _, _, m = oracle.terms(cl, calls)
         freeD = np.floor(rng.uniform(0.5, 1.5, D) * frac * m.sum() / D).astype(np.float32)
-        a, ratio, order, placed, qP, free = oracle.greedy(cl, calls, freeD, dag=dag, node_wf=nwf, elapsed=el)
-        ea, er, eo, eq, ef = _python_loop(oracle, cl, calls, freeD, dag, nwf, el)
+        a, ratio, order, placed, qP, free, delta = oracle.greedy(cl, calls, freeD, dag=dag, node_wf=nwf, elapsed=el,
+                                                                 with_delta=True)
+        ea, er, eo, eq, ef, ed = _python_loop(oracle, cl, calls, freeD, dag, nwf, el)
         assert placed == len(eo) and list(order[:placed]) == eo
         assert np.array_equal(a, ea) and np.array_equal(ratio, er)
+        assert np.array_equal(delta, ed)                      # the Delta inside the ratio, +inf when passed over
+        took = a >= 0
+        assert np.array_equal(ratio[took], ((el[nwf[calls["node"][took]]] + delta[took]) / dag.H[nwf[calls["node"][took]]]).astype(np.float32))
         assert np.array_equal(qP, eq) and np.array_equal(free, ef)
         if frac < 1:
             assert (a == -1).any() and (a >= 0).any()        # capacity really binds
