@@ -328,6 +328,42 @@ int hx_schedule_greedy_plan(hx_cluster* h, const hx_call* calls, int n_calls,
                             int32_t* out_assign, float* out_ratio, int32_t* out_order,
                             float* out_delta, void* stream);
 
+/* Minimal event-driven replay around the greedy planner (Section 6: the
+ * stand-alone simulator tracks every call from waiting for prefill to
+ * completion; Section 7.2: Req95 / Req99).  Workflows arrive at arrival_s[w]; a
+ * call becomes ready when all its predecessors have completed (Section 4.1); at
+ * every event time (an arrival or a completion; equal time stamps are taken
+ * together) all ready calls are planned by hx_schedule_greedy_plan in ratio mode
+ * against the state of the cluster at that time, at most qmax calls per run in
+ * increasing node number, run after run until every ready call was offered once.
+ * State shown to the planner at time t: prefill queue max(0, busy_p - t), free KV
+ * tokens Cap(d) minus the tokens (Eq. 3) of the calls planned onto d and not yet
+ * complete, decode hint 0, elapsed time t - a_w.  The planner's projection is
+ * taken as what happens: a planned call completes Delta after t and its prefill
+ * instance is busy until t + (simulated queue after the run); the six stages of
+ * a call's life are the terms inside Delta.  A call the planner passes over
+ * stays ready until the next event.  Time is binary64 on the host and rounded to
+ * binary32 for the planner.  The paper prints no pseudo-code of its simulator:
+ * these rules are this library's reading.
+ *   The forest must have been uploaded with the same row_ptr / col_idx /
+ * node_workflow (host arrays, given again here) and hx_critical_path enqueued;
+ * node_calls[v] (host, n_nodes records) describes node v.  Outputs (host):
+ * out_fin[n_nodes] completion time of every call (+inf if never planned),
+ * out_ratio[n_workflows] = (completion of the last call - arrival) / H_w,
+ * out_req[2] = Req95, Req99 (the smallest scale alpha such that at least 95 % /
+ * 99 % of the workflows have ratio <= alpha), out_stats[2] = planner runs, calls
+ * left unplanned.  The call overwrites the cluster's loads and elapsed times,
+ * uses `stream`, synchronises it once per planner run, allocates and frees its
+ * device scratch, and restores hx_options on return.  Errors:
+ * HX_ERR_INVALID_ARG (NULL array, qmax outside 1 .. HX_GREEDY_MAX_CALLS, sizes
+ * that differ from the upload, node_calls[v].node != v, a negative or non-finite
+ * arrival), HX_ERR_NOT_READY without horizons, and those of the calls it makes. */
+int hx_replay(hx_cluster* h, const uint32_t* row_ptr, const uint32_t* col_idx,
+              const uint32_t* node_workflow, uint32_t n_nodes, uint32_t n_workflows,
+              const hx_call* node_calls, const double* arrival_s, int qmax,
+              double* out_fin, double* out_ratio, double* out_req, int* out_stats,
+              void* stream);
+
 /* Decode-stage scheduler (Section 5.4, "Decode scheduling with instance locks",
  * "Decode KV-capacity feasibility check", "Adaptive greedy decode assignment").
  * State: the decode token-capacity intervals of every decode instance

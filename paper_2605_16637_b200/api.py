@@ -66,6 +66,7 @@ def _load():
         "hx_schedule_batch_static": [vp, vp, ci, vp, vp, vp],
         "hx_schedule_greedy": [vp, vp, ci, vp, vp, vp, vp],
         "hx_schedule_greedy_plan": [vp, vp, ci, vp, vp, vp, vp, vp],
+        "hx_replay": [vp, vp, vp, vp, C.c_uint32, C.c_uint32, vp, vp, ci, vp, vp, vp, vp, vp],
         "hx_decode_set_running": [vp, vp, vp, vp],
         "hx_schedule_decode": [vp, vp, vp, vp, ci, vp, vp, vp, vp, vp],
         "hx_get_topk": [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp)],
@@ -217,6 +218,21 @@ def hx_schedule_greedy_plan(h, calls_ptr, n_calls, out_assign_ptr, out_ratio_ptr
     """hx_schedule_greedy plus the projected completion Delta of every call; device pointers."""
     _check(_lib.hx_schedule_greedy_plan(h, calls_ptr, int(n_calls), out_assign_ptr, out_ratio_ptr, out_order_ptr,
                                         out_delta_ptr, stream), h)
+
+
+def hx_replay(h, row_ptr, col_idx, node_workflow, n_workflows, node_calls, arrival_s, qmax=4096, stream=0):
+    """Event-driven replay; host arrays in, dict(fin, ratio, req95, req99, runs, stuck) out."""
+    row, col, nwf = _np(row_ptr, np.uint32), _np(col_idx, np.uint32), _np(node_workflow, np.uint32)
+    calls, arr = _np(node_calls, CALL_DTYPE), _np(arrival_s, np.float64)
+    n, w = nwf.shape[0], int(n_workflows)
+    if row.shape[0] != n + 1 or calls.shape[0] != n or arr.shape[0] != w:
+        raise HxError(-1, "array lengths differ")
+    fin, ratio = np.zeros(n, np.float64), np.zeros(w, np.float64)
+    req, stats = np.zeros(2, np.float64), np.zeros(2, np.int32)
+    _check(_lib.hx_replay(h, _p(row), _p(col), _p(nwf), n, w, _p(calls), _p(arr), int(qmax), _p(fin), _p(ratio),
+                          _p(req), _p(stats), stream), h)
+    return dict(fin=fin, ratio=ratio, req95=float(req[0]), req99=float(req[1]), runs=int(stats[0]),
+                stuck=int(stats[1]))
 
 
 KV_INTERVAL_DTYPE = np.dtype([("end_s", "<f4"), ("tokens", "<f4")])
@@ -423,6 +439,10 @@ class Cluster:
         hx_schedule_greedy_plan(self.h, calls.data_ptr(), n, assign.data_ptr(), ratio.data_ptr(), order.data_ptr(),
                                 delta.data_ptr(), self._stream())
         return assign, ratio, order, delta
+
+    def replay(self, row_ptr, col_idx, node_workflow, node_calls, arrival_s, qmax=4096):
+        return hx_replay(self.h, row_ptr, col_idx, node_workflow, self.n_workflows, node_calls, arrival_s, qmax,
+                         self._stream())
 
     def decode_set_running(self, inst_ptr, end_s, tokens):
         run = np.zeros(len(end_s), KV_INTERVAL_DTYPE)

@@ -367,6 +367,13 @@ void for_each_successor(const hx_cluster* h, uint32_t v, Fn fn) {
 
 }  // namespace
 
+int hx_fail(hx_cluster* h, int code, const char* msg) { return fail(h, code, msg); }
+void hx_cluster_shape(const hx_cluster* h, int* P, int* D, const float** capD_dev, uint32_t* n_nodes, uint32_t* n_workflows) {
+    *P = h->P; *D = h->D; *capD_dev = h->tab.capD;
+    *n_nodes = h->dag_uploaded ? h->N : 0; *n_workflows = h->dag_uploaded ? h->W : 0;
+}
+hx_options hx_current_options(const hx_cluster* h) { return h->opts; }
+
 extern "C" {
 
 int hx_cluster_create(const hx_gpu_type* gpu_types, int n_types, const hx_instance* instances,

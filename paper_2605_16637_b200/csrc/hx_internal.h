@@ -187,6 +187,11 @@ inline int hx_cpath_class_of(size_t need_bytes, size_t n_nodes) {
 cudaError_t hx_launch_cost_update(const HxForestDev& f, const uint32_t* idx, const float* cost, uint32_t n,
                                   cudaStream_t stream, long long* launches);
 
+// Accessors for host code outside the file that defines the handle.
+int hx_fail(hx_cluster* h, int code, const char* msg);            // records msg as the last error, returns code
+void hx_cluster_shape(const hx_cluster* h, int* P, int* D, const float** capD_dev, uint32_t* n_nodes, uint32_t* n_workflows);
+hx_options hx_current_options(const hx_cluster* h);
+
 // Opt a kernel in to `bytes` of dynamic shared memory, once per device and size: the attribute
 // call is too slow to repeat on every launch.  `allowed` is a per-kernel table of 64 entries
 // that starts at the size the kernel may use without opting in.
