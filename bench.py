@@ -395,6 +395,7 @@ def run_cuda(args):
         "greedy_planner": greedy,
         "decode_scheduler": decode_leg() if world == 1 and not args.no_cpu_baseline else None,
         "horizon_refinement": refine_leg() if world == 1 and not args.no_cpu_baseline else None,
+        "replay": replay_leg() if world == 1 and not args.no_cpu_baseline else None,
     }
     print(json.dumps(out))
     if dist is not None:
@@ -507,6 +508,47 @@ def refine_leg():
     t0 = time.perf_counter()
     orc.longest_path(wl.row_ptr, wl.col, cost, wl.node_wf, wl.n_workflows)
     out["oracle_full_pass_ms_1_core"] = 1e3 * (time.perf_counter() - t0)
+    out["device_status"] = gc.status()
+    gc.close()
+    return out
+
+
+LOADS = (4.0, 32.0, 256.0)       # offered stand-alone work per second and prefill instance (replay leg)
+
+
+def replay_leg():
+    """Side measurement, outside the timed region: the event-driven replay (Section 6, Section 7.2) of the
+    medium configuration (512 workflows, 16 x 16 instances) at three offered loads; Req95 / Req99 and wall
+    clock, and the oracle's replay of the middle load on one core beside it."""
+    import paper_2605_16637_b200 as hx
+    from hx_synth import make_workload
+    from oracle import hx_oracle as ho
+    from oracle import hx_replay as hr
+    wl = make_workload("medium")
+    gc = hx.Cluster.from_workload(wl)
+    gc.set_options(score_mode=hx.HX_MODE_COMPLETION, flags=hx.HX_FLAG_UNLOADED | hx.HX_FLAG_NO_DAG)
+    cost = gc.schedule_batch(wl.node_calls)[1].cpu().numpy()
+    gc.dag_upload(wl.row_ptr, wl.col, cost, wl.node_wf, wl.elapsed)
+    gc.critical_path()
+    gc.set_options(score_mode=hx.HX_MODE_RATIO)
+    out = {"workflows": wl.n_workflows, "calls": wl.n_nodes, "pairs": wl.P * wl.D, "loads": {}}
+    rng = np.random.default_rng(6)
+    u = np.sort(rng.uniform(0, 1, wl.n_workflows))
+    for load in LOADS:
+        arrival = u * float(cost.sum()) / (wl.P * load)
+        t0 = time.perf_counter()
+        r = gc.replay(wl.row_ptr, wl.col, wl.node_wf, wl.node_calls, arrival)
+        dt = time.perf_counter() - t0
+        out["loads"]["%.1f" % load] = {"req95": r["req95"], "req99": r["req99"], "planner_runs": r["runs"],
+                                       "unplanned": r["stuck"], "wall_ms": 1e3 * dt,
+                                       "us_per_planner_run": 1e6 * dt / max(r["runs"], 1)}
+        if load == LOADS[1]:
+            orc, oc = ho.Oracle(), ho.Cluster.from_workload(wl)
+            dag = orc.longest_path(wl.row_ptr, wl.col, cost, wl.node_wf, wl.n_workflows)
+            t0 = time.perf_counter()
+            w = hr.replay(orc, oc, wl.row_ptr, wl.col, wl.node_wf, wl.n_workflows, wl.node_calls, arrival, dag)
+            out["oracle_wall_ms_1_core_middle_load"] = 1e3 * (time.perf_counter() - t0)
+            out["identical_to_oracle"] = bool(np.array_equal(r["fin"], w["fin"]) and r["req99"] == w["req99"])
     out["device_status"] = gc.status()
     gc.close()
     return out
