@@ -19,10 +19,14 @@ struct Event {
 
 struct Hold { double end; int d; double tokens; };
 
-struct Buffers {                               // device scratch of one replay, freed on every way out
+struct Buffers {                               // device scratch and page-locked staging of one replay, freed on every way out
     hx_call* calls = nullptr; int32_t* assign = nullptr; float* ratio = nullptr; int32_t* order = nullptr;
     float* delta = nullptr;
-    ~Buffers() { cudaFree(calls); cudaFree(assign); cudaFree(ratio); cudaFree(order); cudaFree(delta); }
+    unsigned char* pinned = nullptr;
+    ~Buffers() {
+        cudaFree(calls); cudaFree(assign); cudaFree(ratio); cudaFree(order); cudaFree(delta);
+        cudaFreeHost(pinned);
+    }
 };
 
 double order_statistic(std::vector<double> r, double q) {
@@ -77,9 +81,15 @@ extern "C" int hx_replay(hx_cluster* h, const uint32_t* row_ptr, const uint32_t*
     std::vector<double> busy(P, 0.0), used(D);
     std::vector<Hold> holds;
     std::set<uint32_t> ready;                   // ordered: calls are offered in increasing node number
-    std::vector<float> qP(P), qP2(P), qD(D, 0.0f), kv_free(D), elapsed(W), delta(qmax);
-    std::vector<int32_t> assign(qmax);
-    std::vector<hx_call> chunk(qmax);
+    // staging in page-locked memory: the copies of a planner run are asynchronous and cost one synchronisation
+    const size_t n_f32 = 2 * (size_t)P + 2 * (size_t)D + W + qmax;
+    if (cudaHostAlloc(&b.pinned, (size_t)qmax * sizeof(hx_call) + n_f32 * 4 + (size_t)qmax * 4, cudaHostAllocDefault) != cudaSuccess)
+        return hx_fail(h, HX_ERR_OOM, "replay staging");
+    hx_call* chunk = reinterpret_cast<hx_call*>(b.pinned);
+    float* qP = reinterpret_cast<float*>(chunk + qmax);
+    float *qP2 = qP + P, *qD = qP2 + P, *kv_free = qD + D, *elapsed = kv_free + D, *delta = elapsed + W;
+    int32_t* assign = reinterpret_cast<int32_t*>(delta + qmax);
+    for (int d = 0; d < D; ++d) qD[d] = 0.0f;
     std::vector<uint32_t> offered;
     std::vector<char> touched(P);
     for (uint32_t v = 0; v < N; ++v) out_fin[v] = INFINITY;
@@ -112,15 +122,15 @@ extern "C" int hx_replay(hx_cluster* h, const uint32_t* row_ptr, const uint32_t*
             for (int d = 0; d < D; ++d) kv_free[d] = (float)((double)cap[d] - used[d]);
             for (uint32_t w = 0; w < W; ++w) elapsed[w] = (float)std::max(0.0, t - arrival_s[w]);
             for (int i = 0; i < n; ++i) chunk[i] = node_calls[offered[o + i]];
-            if ((rc = hx_cluster_update_loads(h, qP.data(), qD.data(), kv_free.data(), stream)) != HX_OK) return leave(rc);
-            if ((rc = hx_dag_update_elapsed(h, elapsed.data(), stream)) != HX_OK) return leave(rc);
-            if (cudaMemcpyAsync(b.calls, chunk.data(), (size_t)n * sizeof(hx_call), cudaMemcpyHostToDevice, s) != cudaSuccess)
+            if ((rc = hx_cluster_update_loads(h, qP, qD, kv_free, stream)) != HX_OK) return leave(rc);
+            if ((rc = hx_dag_update_elapsed(h, elapsed, stream)) != HX_OK) return leave(rc);
+            if (cudaMemcpyAsync(b.calls, chunk, (size_t)n * sizeof(hx_call), cudaMemcpyHostToDevice, s) != cudaSuccess)
                 return leave(hx_fail(h, HX_ERR_CUDA, "copying the ready calls"));
             if ((rc = hx_schedule_greedy_plan(h, b.calls, n, b.assign, b.ratio, b.order, b.delta, stream)) != HX_OK) return leave(rc);
-            if (cudaMemcpyAsync(assign.data(), b.assign, (size_t)n * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
-                cudaMemcpyAsync(delta.data(), b.delta, (size_t)n * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+            if (cudaMemcpyAsync(assign, b.assign, (size_t)n * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+                cudaMemcpyAsync(delta, b.delta, (size_t)n * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess)
                 return leave(hx_fail(h, HX_ERR_CUDA, "reading the plan"));
-            if ((rc = hx_cluster_read_loads(h, qP2.data(), nullptr, nullptr, stream)) != HX_OK) return leave(rc);   // synchronises
+            if ((rc = hx_cluster_read_loads(h, qP2, nullptr, nullptr, stream)) != HX_OK) return leave(rc);   // synchronises
             ++runs;
             std::fill(touched.begin(), touched.end(), 0);
             for (int i = 0; i < n; ++i) {
