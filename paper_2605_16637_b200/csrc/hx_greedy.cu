@@ -132,23 +132,28 @@ __global__ void __launch_bounds__(kThreads, 1) hx_greedy_kernel(const __grid_con
             }
             __syncwarp();
             float best = HX_INF; int bj = 0x7fffffff;
-            int p = lane / D, d = lane - p * D;
-            while (p < P) {
+            // a lane keeps its decode instance and walks the prefill instances, so that everything that
+            // depends on d alone (room, decode time, availability) is read once per call: with D lanes per
+            // prefill row when D divides 32, else with the lanes over d and every lane over all rows
+            const int dlanes = (D < 32 && 32 % D == 0) ? D : 32;
+            const int prow = lane / dlanes, pstep = 32 / dlanes;
+            for (int d = lane - prow * dlanes; d < D; d += dlanes) {
                 const bool fits = m <= capDs[d] && m <= frees[d];
-                const float Dd = fits ? tdec[typeDs[d]] : HX_INF;
-                const float A = __fadd_rn(qPs[p], tpre[typePs[p]]);
-                const float ready = __fmaf_rn(kvB, invL[p * D + d], A);
-                const float fin = __fadd_rn(fmaxf(ready, qDs[d]), Dd);
-                if (fin < best) { best = fin; bj = (p << 16) | d; }
-                d += 32;
-                while (d >= D) { d -= D; ++p; }
+                if (!fits) continue;                           // every pair on d is +inf: cannot be the minimum
+                const float Dd = tdec[typeDs[d]], qd = qDs[d];
+                for (int p = prow; p < P; p += pstep) {
+                    const float A = __fadd_rn(qPs[p], tpre[typePs[p]]);
+                    const float ready = __fmaf_rn(kvB, invL[p * D + d], A);
+                    const float fin = __fadd_rn(fmaxf(ready, qd), Dd);
+                    const int j = (p << 16) | d;
+                    if (fin < best || (fin == best && j < bj)) { best = fin; bj = j; }
+                }
             }
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) {
-                const float ov = __shfl_xor_sync(0xffffffffu, best, off);
-                const int oj = __shfl_xor_sync(0xffffffffu, bj, off);
-                if (ov < best || (ov == best && oj < bj)) { best = ov; bj = oj; }
-            }
+            // finish times are >= 0 or +inf, so their bit patterns order like the values: two warp-wide
+            // integer minima give the smallest value and the lowest pair among the lanes that hold it
+            const unsigned vmin = __reduce_min_sync(0xffffffffu, __float_as_uint(best));
+            bj = (int)__reduce_min_sync(0xffffffffu, __float_as_uint(best) == vmin ? (unsigned)bj : 0x7fffffffu);
+            best = __uint_as_float(vmin);
             if (lane == 0) {
                 if (best < HX_INF) { cpair[c] = bj; cR[c] = __fdiv_rn(__fadd_rn(cel[c], best), cH[c]); }
                 else { cpair[c] = kNoPair; cR[c] = HX_NEG_INF; }
