@@ -47,6 +47,7 @@ struct DecodeParams {
     const int32_t* lock;
     const float* ready;
     int n, flags, commit;
+    int pool_T;                // entries of the shared-memory pool of breakpoints (POOL variant)
     int32_t* out_inst;
     float* out_start;
     float* out_ratio;
@@ -84,17 +85,21 @@ __device__ int warp_cut(float* t, float* u, int& K, float x, int lane) {
     return k + 1;
 }
 
-template <int NC>   // blocks of the cluster (1 = a plain single block)
+// POOL: the step functions of all instances live in one shared-memory pool (their total length is bounded by
+// the snapshot plus two breakpoints per queued call, whatever the split between instances); an instance whose
+// region is full makes warp 0 lay the regions out again in the second half of the pool.  Without POOL every
+// block works on its own copy in global memory, each instance with room for the worst case.
+template <int NC, bool POOL>   // NC: blocks of the cluster (1 = a plain single block)
 __global__ void __launch_bounds__(kThreads, 1) hx_decode_kernel(const __grid_constant__ DecodeParams prm) {
     extern __shared__ __align__(16) unsigned char smem[];
     __shared__ float red_v[kWarps];
     __shared__ int red_c[kWarps];
-    __shared__ int s_call, s_d, s_ndirty;
+    __shared__ int s_call, s_d, s_ndirty, s_cur;
     __shared__ float x_v[NC];                  // most urgent call of every block (written by its owner block)
     __shared__ int x_c[NC];
     __shared__ float x_commit[4];              // instance (int bits), start, finish, demand of the committed call
     const HxTables& T = prm.t;
-    const int D = T.D, G = T.G;
+    const int D = T.D;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int cap = prm.work.cap;
     int rank = 0;
@@ -119,17 +124,37 @@ __global__ void __launch_bounds__(kThreads, 1) hx_decode_kernel(const __grid_con
     int* clock_ = cbest + n;                                    // lock (-1 = free)
     int* cmodel = clock_ + n;
     unsigned short* dirty = reinterpret_cast<unsigned short*>(cmodel + n);
+    const int PT = prm.pool_T;
+    int* roff = reinterpret_cast<int*>(dirty + ((n + 1) & ~1));  // [D+1] regions of the pool (POOL)
+    int* roff2 = roff + D + 1;                                    // [D+1] the next layout while regions move
+    float* pool_t = reinterpret_cast<float*>(roff2 + D + 1);     // [2][PT] breakpoints, two halves
+    float* pool_u = pool_t + 2 * (size_t)PT;                    // [2][PT] usage
+    // step function of instance d in the simulated state
+    auto seg_t = [&](int d) -> float* { return POOL ? pool_t + (size_t)s_cur * PT + roff[d] : wt + (size_t)d * cap; };
+    auto seg_u = [&](int d) -> float* { return POOL ? pool_u + (size_t)s_cur * PT + roff[d] : wu + (size_t)d * cap; };
 
     for (int d = tid; d < D; d += kThreads) {
         capDs[d] = T.capD[d]; typeDs[d] = T.typeD[d];
         Ks[d] = prm.base.K[d];
     }
+    if (tid == 0) s_cur = 0;
     __syncthreads();
-    for (int d = warp; d < D; d += kWarps)                      // simulated state starts as the snapshot
+    if (POOL && tid == 0) {                                     // every instance its breakpoints plus an equal share of the rest
+        int sum = 0;
+        for (int d = 0; d < D; ++d) sum += Ks[d];
+        const int share = max(0, (PT - sum) / D);
+        int o = 0;
+        for (int d = 0; d < D; ++d) { roff[d] = o; o += Ks[d] + share; }
+        roff[D] = o;
+    }
+    __syncthreads();
+    for (int d = warp; d < D; d += kWarps) {                    // simulated state starts as the snapshot
+        float* tt = seg_t(d); float* uu = seg_u(d);
         for (int i = lane; i < Ks[d]; i += 32) {
-            wt[(size_t)d * cap + i] = prm.base.t[(size_t)d * prm.base.cap + i];
-            wu[(size_t)d * cap + i] = prm.base.u[(size_t)d * prm.base.cap + i];
+            tt[i] = prm.base.t[(size_t)d * prm.base.cap + i];
+            uu[i] = prm.base.u[(size_t)d * prm.base.cap + i];
         }
+    }
     for (int c = tid; c < n; c += kThreads) {
         const int gcall = c * NC + rank;
         const uint4 raw = __ldg(reinterpret_cast<const uint4*>(prm.calls) + gcall);
@@ -172,11 +197,14 @@ __global__ void __launch_bounds__(kThreads, 1) hx_decode_kernel(const __grid_con
             for (int d = lane; d < D; d += 32) {
                 if ((lk >= 0 && lk != d) || !(m <= capDs[d])) continue;
                 const float tau = __fmul_rn(__fmul_rn(ot, step), prm.ct.invB[typeDs[d]]);
-                const float* tt = wt + (size_t)d * cap;
-                const float* uu = wu + (size_t)d * cap;
+                const float* tt = seg_t(d);
+                const float* uu = seg_u(d);
                 const int K = Ks[d];
-                int k = 0;
-                while (k + 1 < K && tt[k + 1] <= rd) ++k;       // segment that holds the ready time
+                int k = 0, hi = K - 1;                          // segment that holds the ready time: largest k with
+                while (k < hi) {                                // t[k] <= ready (t[0] = 0), by bisection
+                    const int mid = (k + hi + 1) >> 1;
+                    if (tt[mid] <= rd) k = mid; else hi = mid - 1;
+                }
                 float cand = rd, fin;
                 for (;; ++k) {
                     const float seg_end = (k + 1 < K) ? tt[k + 1] : HX_INF;
@@ -273,11 +301,45 @@ __global__ void __launch_bounds__(kThreads, 1) hx_decode_kernel(const __grid_con
             if (s_call >= 0) {
                 const int d = __float_as_int(x_commit[0]);
                 const float st = x_commit[1], en = x_commit[2], m = x_commit[3];
-                float* tt = wt + (size_t)d * cap;
-                float* uu = wu + (size_t)d * cap;
                 int K = Ks[d];
+                bool room = POOL ? K + 2 <= roff[d + 1] - roff[d] : K + 2 <= cap;
+                if (POOL && !room) {
+                    // lay the regions out again in the other half: every instance its breakpoints plus an equal
+                    // share of what is free, after two entries set aside for this commit
+                    if (lane == 0) {
+                        int sum = 0;
+                        for (int e = 0; e < D; ++e) sum += Ks[e];
+                        const int free_now = PT - sum - 2;
+                        if (free_now >= 0) {
+                            const int share = free_now / D;
+                            int o = 0;
+                            for (int e = 0; e < D; ++e) { roff2[e] = o; o += Ks[e] + share + (e == d ? 2 : 0); }
+                            roff2[D] = o;
+                        } else {
+                            roff2[D] = -1;                       // the pool itself is full: the host sized it too small
+                        }
+                    }
+                    __syncwarp();
+                    if (roff2[D] >= 0) {
+                        const int cur = s_cur;
+                        for (int e = 0; e < D; ++e) {
+                            const float* ot = pool_t + (size_t)cur * PT + roff[e];
+                            const float* ou = pool_u + (size_t)cur * PT + roff[e];
+                            float* nt2 = pool_t + (size_t)(cur ^ 1) * PT + roff2[e];
+                            float* nu2 = pool_u + (size_t)(cur ^ 1) * PT + roff2[e];
+                            for (int i = lane; i < Ks[e]; i += 32) { nt2[i] = ot[i]; nu2[i] = ou[i]; }
+                        }
+                        __syncwarp();
+                        for (int e = lane; e <= D; e += 32) roff[e] = roff2[e];
+                        if (lane == 0) s_cur = cur ^ 1;
+                        __syncwarp();
+                        room = true;
+                    }
+                }
+                float* tt = seg_t(d);
+                float* uu = seg_u(d);
                 __syncwarp();
-                if (K + 2 > cap) {                              // cannot happen with the capacity the host sizes
+                if (!room) {                                    // cannot happen with the capacity the host sizes
                     if (lane == 0) { atomicExch(prm.status, HX_ERR_INVALID_ARG); s_call = -1; }
                 } else {
                     const int a = warp_cut(tt, uu, K, st, lane);
@@ -299,9 +361,10 @@ __global__ void __launch_bounds__(kThreads, 1) hx_decode_kernel(const __grid_con
         __syncthreads();
         for (int d = warp; d < D; d += kWarps) {
             const int K = min(Ks[d], prm.base.cap);
+            const float* tt = seg_t(d); const float* uu = seg_u(d);
             for (int i = lane; i < K; i += 32) {
-                prm.base.t[(size_t)d * prm.base.cap + i] = wt[(size_t)d * cap + i];
-                prm.base.u[(size_t)d * prm.base.cap + i] = wu[(size_t)d * cap + i];
+                prm.base.t[(size_t)d * prm.base.cap + i] = tt[i];
+                prm.base.u[(size_t)d * prm.base.cap + i] = uu[i];
             }
             if (lane == 0) prm.base.K[d] = K;
         }
@@ -317,13 +380,43 @@ constexpr int kClusterFrom = 256;              // queues longer than this use th
 static size_t decode_smem(const HxTables& t, int calls_per_block) {
     return (3 * (size_t)t.D + 11 * (size_t)calls_per_block) * 4 + (size_t)calls_per_block * 2 + 16;
 }
+// With the pool of breakpoints behind the per-call state: two layouts of pool_T entries, times and usage.
+static size_t decode_pool_smem(const HxTables& t, int calls_per_block, int pool_T) {
+    return decode_smem(t, calls_per_block) + 4 + 2 * ((size_t)t.D + 1) * 4 + 4 * (size_t)pool_T * 4;
+}
 
 size_t hx_decode_smem_bytes(const HxTables& t, int n_calls) { return decode_smem(t, n_calls); }
 
 int hx_decode_replicas() { return kCluster; }
 
+template <int NC, bool POOL>
+static cudaError_t launch_variant(const DecodeParams& prm, size_t smem, cudaStream_t stream, bool* launched) {
+    static size_t allowed[64];
+    *launched = false;
+    cudaError_t e = hx_opt_in_smem(hx_decode_kernel<NC, POOL>, smem, allowed, 40 * 1024);
+    if (e != cudaSuccess) return e;
+    if (NC == 1) {
+        hx_decode_kernel<NC, POOL><<<1, kThreads, smem, stream>>>(prm);
+        *launched = true;
+        return cudaGetLastError();
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(NC); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = NC; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    int n_clusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&n_clusters, hx_decode_kernel<NC, POOL>, &cfg) != cudaSuccess || n_clusters < 1) {
+        (void)cudaGetLastError();              // the device cannot host the cluster: the caller falls back to one block
+        return cudaSuccess;
+    }
+    *launched = true;
+    return cudaLaunchKernelEx(&cfg, hx_decode_kernel<NC, POOL>, prm);
+}
+
 cudaError_t hx_launch_decode(const HxTables& t, const HxConstTables& ct, const HxDagView& dag,
-                             const HxStepFns& base, const HxStepFns& work,
+                             const HxStepFns& base, const HxStepFns& work, int k_total,
                              const hx_call* calls, const int32_t* lock, const float* ready, int n_calls,
                              int flags, int commit, int32_t* out_inst, float* out_start, float* out_ratio,
                              int32_t* out_order, int* status, cudaStream_t stream, long long* launches) {
@@ -332,30 +425,30 @@ cudaError_t hx_launch_decode(const HxTables& t, const HxConstTables& ct, const H
     prm.calls = calls; prm.lock = lock; prm.ready = ready; prm.n = n_calls; prm.flags = flags; prm.commit = commit;
     prm.out_inst = out_inst; prm.out_start = out_start; prm.out_ratio = out_ratio; prm.out_order = out_order;
     prm.status = status;
+    // all breakpoints the run can create: those of the snapshot, two per queued call, some slack per instance
+    const long long pool = (long long)k_total + 2LL * n_calls + 4LL * t.D;
+    const size_t kPoolLimit = 200 * 1024;
     cudaError_t e;
+    bool launched = false;
     if (n_calls > kClusterFrom) {
-        const size_t smem = decode_smem(t, (n_calls + kCluster - 1) / kCluster);
-        static size_t allowed[64];
-        if ((e = hx_opt_in_smem(hx_decode_kernel<kCluster>, smem, allowed, 40 * 1024)) != cudaSuccess) return e;
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(kCluster); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = smem; cfg.stream = stream;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = kCluster; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-        cfg.attrs = attr; cfg.numAttrs = 1;
-        int n_clusters = 0;
-        if (cudaOccupancyMaxActiveClusters(&n_clusters, hx_decode_kernel<kCluster>, &cfg) == cudaSuccess && n_clusters >= 1) {
-            e = cudaLaunchKernelEx(&cfg, hx_decode_kernel<kCluster>, prm);
-            if (e == cudaSuccess) ++*launches;
-            return e;
+        const int cpb = (n_calls + kCluster - 1) / kCluster;
+        if (pool < (1 << 24) && decode_pool_smem(t, cpb, (int)pool) <= kPoolLimit) {
+            prm.pool_T = (int)pool;
+            e = launch_variant<kCluster, true>(prm, decode_pool_smem(t, cpb, (int)pool), stream, &launched);
+        } else {
+            prm.pool_T = 0;
+            e = launch_variant<kCluster, false>(prm, decode_smem(t, cpb), stream, &launched);
         }
-        (void)cudaGetLastError();              // the device cannot host the cluster: one block
+        if (e != cudaSuccess) return e;
+        if (launched) { ++*launches; return cudaSuccess; }
     }
-    const size_t smem = decode_smem(t, n_calls);
-    static size_t allowed1[64];
-    if ((e = hx_opt_in_smem(hx_decode_kernel<1>, smem, allowed1, 40 * 1024)) != cudaSuccess) return e;
-    hx_decode_kernel<1><<<1, kThreads, smem, stream>>>(prm);
-    e = cudaGetLastError();
+    if (pool < (1 << 24) && decode_pool_smem(t, n_calls, (int)pool) <= kPoolLimit) {
+        prm.pool_T = (int)pool;
+        e = launch_variant<1, true>(prm, decode_pool_smem(t, n_calls, (int)pool), stream, &launched);
+    } else {
+        prm.pool_T = 0;
+        e = launch_variant<1, false>(prm, decode_smem(t, n_calls), stream, &launched);
+    }
     if (e == cudaSuccess) ++*launches;
     return e;
 }

@@ -97,6 +97,7 @@ struct hx_cluster {
     std::vector<void*> dec_allocs;
     HxStepFns dec_base{}, dec_work{};
     int dec_k_bound = 0;                // upper bound on the breakpoints of any instance in the snapshot
+    long long dec_k_total = 0;          // upper bound on the breakpoints of all instances together
     bool dec_ready = false;
     // top-K
     HxTopkBufs tk{};
@@ -1233,6 +1234,8 @@ int hx_decode_set_running(hx_cluster* h, const uint32_t* inst_ptr, const hx_kv_i
     HX_TRY(cudaMemcpyAsync(h->dec_base.u, u.data(), u.size() * sizeof(float), cudaMemcpyHostToDevice, s), "copy decode intervals");
     HX_TRY(cudaMemcpyAsync(h->dec_base.K, K.data(), K.size() * sizeof(int), cudaMemcpyHostToDevice, s), "copy decode intervals");
     h->dec_k_bound = maxK;
+    h->dec_k_total = 0;
+    for (int d = 0; d < D; ++d) h->dec_k_total += K[d];
     h->dec_ready = true;
     return HX_OK;
 }
@@ -1261,11 +1264,12 @@ int hx_schedule_decode(hx_cluster* h, const hx_call* calls, const int32_t* lock,
         dag = HxDagView{h->d_node_wf, h->g_tail, h->g_H, h->d_elapsed, h->N, h->W};
     {
         SpanGuard span(h, 0, s);
-        HX_TRY(hx_launch_decode(h->tab, h->ctab, dag, h->dec_base, h->dec_work, calls, lock, ready_s, n_calls, o.flags,
+        HX_TRY(hx_launch_decode(h->tab, h->ctab, dag, h->dec_base, h->dec_work,
+                                (int)std::min<long long>(h->dec_k_total, 1 << 30), calls, lock, ready_s, n_calls, o.flags,
                                 o.commit, out_inst, out_start, out_ratio, out_order, h->status, s, &h->launches),
                "decode scheduler kernel");
     }
-    if (o.commit) h->dec_k_bound += 2 * n_calls;
+    if (o.commit) { h->dec_k_bound += 2 * n_calls; h->dec_k_total += 2LL * n_calls; }
     return HX_OK;
 }
 

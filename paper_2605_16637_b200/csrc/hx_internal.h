@@ -139,7 +139,7 @@ struct HxStepFns {
 size_t hx_decode_smem_bytes(const HxTables& t, int n_calls);
 int hx_decode_replicas();      // copies of the simulated step functions the kernel may use (one per cluster block)
 cudaError_t hx_launch_decode(const HxTables& t, const HxConstTables& ct, const HxDagView& dag,
-                             const HxStepFns& base, const HxStepFns& work,
+                             const HxStepFns& base, const HxStepFns& work, int k_total,
                              const hx_call* calls, const int32_t* lock, const float* ready, int n_calls,
                              int flags, int commit, int32_t* out_inst, float* out_start, float* out_ratio,
                              int32_t* out_order, int* status, cudaStream_t stream, long long* launches);

@@ -88,6 +88,26 @@ def test_decode_scheduler_matches_oracle(hx, oracle, D, C, per, caps):
     gc.close()
 
 
+@pytest.mark.parametrize("C", [100, 300])
+def test_decode_scheduler_with_a_snapshot_too_long_for_shared_memory(hx, oracle, C):
+    # 40 instances x 700 running calls: the step functions do not fit the shared-memory pool, so every block works
+    # on its copy in global memory (one block for 100 calls, the cluster for 300)
+    rng = np.random.default_rng(300 + C)
+    D = 40
+    gc, oc = _pair(hx, rng, D, (1.0e6,))
+    calls, lock, ready = _queue(rng, C, D, hi=20000)
+    ptr, end, tok = [0], [], []
+    for d in range(D):
+        share = rng.dirichlet(np.ones(701))[:700] * 0.995 * oc.capD[d]
+        end += list(rng.uniform(0.01, 3.0, 700).astype(F32)); tok += list(np.floor(share))
+        ptr.append(len(end))
+    ptr, end, tok = np.array(ptr, np.uint32), np.array(end, F32), np.array(tok, F32)
+    gc.decode_set_running(ptr, end, tok)
+    inst, start, ratio, order, placed = _check(hx, gc, oc, oracle, calls, lock, ready, ptr, end, tok)
+    assert placed == C and (start > ready).any()
+    gc.close()
+
+
 def test_decode_commit_carries_the_plan_into_the_next_invocation(hx, oracle):
     rng = np.random.default_rng(77)
     D = 6
