@@ -230,10 +230,7 @@ def run_cuda(args):
     def step_host():
         hx.hx_critical_path(h, sptr)
         hx.hx_cluster_update_loads(h, qP0, qD0, free0, sptr)
-        for i in range(n_chunks):
-            hx.hx_cluster_update_loads(h, None, None, free0, sptr)
-            lo = i * chunk
-            hx.hx_schedule_batch_host_async(h, ch_np[lo:lo + chunk], ha_np[lo:lo + chunk], hc_np[lo:lo + chunk], sptr)
+        hx.hx_schedule_sweep_host(h, ch_np, chunk, free0, ha_np, hc_np, sptr)
         torch.cuda.current_stream().synchronize()        # results of all 16 batches are in host memory
 
     def barrier():
@@ -386,8 +383,8 @@ def run_cuda(args):
                              "what": "load refresh + hx_schedule_batch (scoring, top-4, conflict pass, commit) per "
                                      "ready batch, CUDA events"},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "what": "hx_schedule_batch_host_async per chunk from pinned host memory into pinned host memory, one "
-                        "synchronisation per step, wall clock"},
+                "what": "hx_schedule_sweep_host (all 16 chunks, copies on their own streams) from pinned host memory into "
+                        "pinned host memory, one synchronisation per step, wall clock"},
         "gpu_launches": int(launches), "launch_mode": mode, "replay_matches_call_by_call": replay_ok,
         "ms_per_step_call_by_call_instrumented": inst_ms / n_inst,
         "kernel_ms_per_step": {k: v[0] / n_inst for k, v in kt.items()},

@@ -262,6 +262,27 @@ int hx_schedule_batch_host(hx_cluster* h, const hx_call* calls, int n_calls,
 int hx_schedule_batch_host_async(hx_cluster* h, const hx_call* calls, int n_calls,
                                  int32_t* out_assign, float* out_cost, void* stream);
 
+/* A whole sweep of successive ready batches from host buffers: the n_calls
+ * records are handled in chunks of chunk_calls (the last one may be shorter),
+ * in order, each chunk exactly as hx_schedule_batch_host_async would handle it
+ * (the commits of a chunk are the snapshot of the next).  When kv_free_reset is
+ * not NULL (host, n_decode values) the free KV tokens of the decode instances
+ * are set to it ahead of every chunk (decode completions between two scheduler
+ * invocations), as hx_cluster_update_loads(h, NULL, NULL, kv_free_reset) would.
+ * Unlike a loop over the per-chunk call, the records of all chunks go up on a
+ * copy stream of the handle ahead of the kernels, and the results of a chunk
+ * come down on a second copy stream while the next chunk is being scored; the
+ * caller's `stream` carries the kernels, waits for what was on it before, and
+ * ends after the last copy, so one synchronisation of `stream` covers
+ * everything.  calls, out_assign, out_cost (and kv_free_reset) should be
+ * page-locked for the copies to overlap, and must stay alive and untouched until
+ * then.  Device staging grows to n_calls records (a synchronising allocation the
+ * first time).  Errors: those of hx_schedule_batch; HX_ERR_INVALID_ARG for
+ * chunk_calls < 1 or, with topk > 0, > HX_MAX_COMMIT_CALLS. */
+int hx_schedule_sweep_host(hx_cluster* h, const hx_call* calls, int n_calls, int chunk_calls,
+                           const float* kv_free_reset, int32_t* out_assign, float* out_cost,
+                           void* stream);
+
 /* hx_schedule_batch for callers that must not allocate.  (The paper has no
  * counterpart: this entry point exists only because of how the library is
  * embedded.)  hx_schedule_batch with topk > 0 obtains its intermediate buffers

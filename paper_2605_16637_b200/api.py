@@ -63,6 +63,7 @@ def _load():
         "hx_schedule_batch": [vp, vp, ci, vp, vp, vp],
         "hx_schedule_batch_host": [vp, vp, ci, vp, vp, vp],
         "hx_schedule_batch_host_async": [vp, vp, ci, vp, vp, vp],
+        "hx_schedule_sweep_host": [vp, vp, ci, ci, vp, vp, vp, vp],
         "hx_schedule_batch_static": [vp, vp, ci, vp, vp, vp],
         "hx_schedule_greedy": [vp, vp, ci, vp, vp, vp, vp],
         "hx_schedule_greedy_plan": [vp, vp, ci, vp, vp, vp, vp, vp],
@@ -273,6 +274,19 @@ def hx_schedule_batch_host_async(h, calls, out_assign, out_cost, stream=0):
     if not (calls.flags.c_contiguous and out_assign.flags.c_contiguous and out_cost.flags.c_contiguous):
         raise HxError(-1, "hx_schedule_batch_host_async needs contiguous arrays")
     _check(_lib.hx_schedule_batch_host_async(h, _p(calls), calls.shape[0], _p(out_assign), _p(out_cost), stream), h)
+
+
+def hx_schedule_sweep_host(h, calls, chunk_calls, kv_free_reset, out_assign, out_cost, stream=0):
+    """Enqueue a whole sweep (chunks of chunk_calls, copies overlapped with the kernels); arrays as for
+    hx_schedule_batch_host_async, kv_free_reset a float32 array (page-locked for overlap) or None."""
+    if calls.dtype != CALL_DTYPE or out_assign.dtype != np.int32 or out_cost.dtype != np.float32:
+        raise HxError(-1, "hx_schedule_sweep_host takes CALL_DTYPE, int32 and float32 arrays as they are")
+    if not (calls.flags.c_contiguous and out_assign.flags.c_contiguous and out_cost.flags.c_contiguous):
+        raise HxError(-1, "hx_schedule_sweep_host needs contiguous arrays")
+    if kv_free_reset is not None and (kv_free_reset.dtype != np.float32 or not kv_free_reset.flags.c_contiguous):
+        raise HxError(-1, "kv_free_reset must be a contiguous float32 array")
+    _check(_lib.hx_schedule_sweep_host(h, _p(calls), calls.shape[0], int(chunk_calls), _p(kv_free_reset),
+                                       _p(out_assign), _p(out_cost), stream), h)
 
 
 def hx_get_topk(h):

@@ -103,6 +103,9 @@ struct hx_cluster {
     HxTopkBufs tk{};
     // staging for the host-buffer entry point
     hx_call* st_calls = nullptr; int32_t* st_assign = nullptr; float* st_cost = nullptr; int st_cap = 0;
+    // copy streams and events of hx_schedule_sweep_host, created on first use
+    cudaStream_t sw_in = nullptr, sw_out = nullptr;
+    std::vector<cudaEvent_t> sw_ev;
     hx_options opts{HX_MODE_COMPLETION, 0, 0, 0, 1.5f};
     std::string err;
     long long launches = 0;
@@ -519,6 +522,9 @@ int hx_cluster_destroy(hx_cluster* h) {
         for (int i = 0; i < HX_CP_SIDE; ++i) { cudaStreamDestroy(h->fj.aux[i]); cudaEventDestroy(h->fj.join[i]); }
         cudaEventDestroy(h->fj.fork);
     }
+    for (cudaEvent_t e : h->sw_ev) cudaEventDestroy(e);
+    if (h->sw_in) cudaStreamDestroy(h->sw_in);
+    if (h->sw_out) cudaStreamDestroy(h->sw_out);
     for (auto* v : {&h->spans, &h->spare})
         for (auto& sp : *v) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
     delete h;
@@ -997,6 +1003,22 @@ int hx_schedule_batch(hx_cluster* h, const hx_call* calls, int n_calls, int32_t*
     return HX_OK;
 }
 
+// Device staging of the host-buffer entry points: room for n_calls records and results.
+static int reserve_staging(hx_cluster* h, int n_calls) {
+    if (h->st_cap >= n_calls) return HX_OK;
+    cudaDeviceSynchronize();
+    if (h->st_calls) cudaFree(h->st_calls);
+    if (h->st_assign) cudaFree(h->st_assign);
+    if (h->st_cost) cudaFree(h->st_cost);
+    h->st_calls = nullptr; h->st_assign = nullptr; h->st_cost = nullptr; h->st_cap = 0;
+    const size_t cap = (size_t)std::max(n_calls, 16384);
+    HX_TRY(cudaMalloc(&h->st_calls, cap * sizeof(hx_call)), "alloc staging");
+    HX_TRY(cudaMalloc(&h->st_assign, cap * sizeof(int32_t)), "alloc staging");
+    HX_TRY(cudaMalloc(&h->st_cost, cap * sizeof(float)), "alloc staging");
+    h->st_cap = (int)cap;
+    return HX_OK;
+}
+
 static int schedule_batch_host_impl(hx_cluster* h, const hx_call* calls, int n_calls, int32_t* out_assign,
                                     float* out_cost, void* stream, bool sync) {
     if (!h) return HX_ERR_INVALID_ARG;
@@ -1005,18 +1027,7 @@ static int schedule_batch_host_impl(hx_cluster* h, const hx_call* calls, int n_c
     if (!calls || !out_assign || !out_cost) return fail(h, HX_ERR_INVALID_ARG, "NULL buffer");
     DeviceGuard guard(h->device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (h->st_cap < n_calls) {
-        cudaDeviceSynchronize();
-        if (h->st_calls) cudaFree(h->st_calls);
-        if (h->st_assign) cudaFree(h->st_assign);
-        if (h->st_cost) cudaFree(h->st_cost);
-        h->st_calls = nullptr; h->st_assign = nullptr; h->st_cost = nullptr; h->st_cap = 0;
-        const size_t cap = (size_t)std::max(n_calls, 16384);
-        HX_TRY(cudaMalloc(&h->st_calls, cap * sizeof(hx_call)), "alloc staging");
-        HX_TRY(cudaMalloc(&h->st_assign, cap * sizeof(int32_t)), "alloc staging");
-        HX_TRY(cudaMalloc(&h->st_cost, cap * sizeof(float)), "alloc staging");
-        h->st_cap = (int)cap;
-    }
+    if (int rc = reserve_staging(h, n_calls)) return rc;
     HX_TRY(cudaMemcpyAsync(h->st_calls, calls, (size_t)n_calls * sizeof(hx_call), cudaMemcpyHostToDevice, s), "copy calls");
     int rc = hx_schedule_batch(h, h->st_calls, n_calls, h->st_assign, h->st_cost, stream);
     if (rc != HX_OK) return rc;
@@ -1034,6 +1045,63 @@ int hx_schedule_batch_host(hx_cluster* h, const hx_call* calls, int n_calls, int
 int hx_schedule_batch_host_async(hx_cluster* h, const hx_call* calls, int n_calls, int32_t* out_assign,
                                  float* out_cost, void* stream) {
     return schedule_batch_host_impl(h, calls, n_calls, out_assign, out_cost, stream, false);
+}
+
+int hx_schedule_sweep_host(hx_cluster* h, const hx_call* calls, int n_calls, int chunk_calls,
+                           const float* kv_free_reset, int32_t* out_assign, float* out_cost, void* stream) {
+    if (!h) return HX_ERR_INVALID_ARG;
+    if (n_calls < 0 || chunk_calls < 1) return fail(h, HX_ERR_INVALID_ARG, "n_calls must be >= 0 and chunk_calls >= 1");
+    if (n_calls == 0) return HX_OK;
+    if (!calls || !out_assign || !out_cost) return fail(h, HX_ERR_INVALID_ARG, "NULL buffer");
+    if (h->opts.topk > 0 && chunk_calls > HX_MAX_COMMIT_CALLS)
+        return fail(h, HX_ERR_INVALID_ARG, "chunk too large for the capacity-conflict pass");
+    if (kv_free_reset)
+        for (int d = 0; d < h->D; ++d)
+            if (!good_load(kv_free_reset[d])) return fail(h, HX_ERR_INVALID_ARG, "loads must be finite and >= 0");
+    DeviceGuard guard(h->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (int rc = reserve_staging(h, n_calls)) return rc;
+    const int n_chunks = (n_calls + chunk_calls - 1) / chunk_calls;
+    if (!h->sw_in) {
+        HX_TRY(cudaStreamCreateWithFlags(&h->sw_in, cudaStreamNonBlocking), "creating the copy streams");
+        HX_TRY(cudaStreamCreateWithFlags(&h->sw_out, cudaStreamNonBlocking), "creating the copy streams");
+    }
+    while (h->sw_ev.size() < 2 * (size_t)n_chunks + 2) {
+        cudaEvent_t e;
+        HX_TRY(cudaEventCreateWithFlags(&e, cudaEventDisableTiming), "creating events");
+        h->sw_ev.push_back(e);
+    }
+    cudaEvent_t ev_start = h->sw_ev[0], ev_done = h->sw_ev[1];
+    // whatever is already on the caller's stream comes first
+    HX_TRY(cudaEventRecord(ev_start, s), "event");
+    HX_TRY(cudaStreamWaitEvent(h->sw_in, ev_start, 0), "event");
+    HX_TRY(cudaStreamWaitEvent(h->sw_out, ev_start, 0), "event");
+    // every chunk's records go up on their own stream, ahead of the kernels that need them
+    for (int c = 0; c < n_chunks; ++c) {
+        const size_t o = (size_t)c * chunk_calls, n = std::min<size_t>(chunk_calls, (size_t)n_calls - o);
+        HX_TRY(cudaMemcpyAsync(h->st_calls + o, calls + o, n * sizeof(hx_call), cudaMemcpyHostToDevice, h->sw_in), "copy calls");
+        HX_TRY(cudaEventRecord(h->sw_ev[2 + c], h->sw_in), "event");
+    }
+    for (int c = 0; c < n_chunks; ++c) {
+        const size_t o = (size_t)c * chunk_calls, n = std::min<size_t>(chunk_calls, (size_t)n_calls - o);
+        HX_TRY(cudaStreamWaitEvent(s, h->sw_ev[2 + c], 0), "event");
+        if (kv_free_reset)
+            HX_TRY(cudaMemcpyAsync(h->tab.freeD, kv_free_reset, h->D * sizeof(float), cudaMemcpyHostToDevice, s), "cudaMemcpyAsync(loads)");
+        const int rc = hx_schedule_batch(h, h->st_calls + o, (int)n, h->st_assign + o, h->st_cost + o, stream);
+        if (rc != HX_OK) {                               // leave no stream waiting on work that will never come
+            cudaEventRecord(ev_done, h->sw_out); cudaStreamWaitEvent(s, ev_done, 0);
+            return rc;
+        }
+        // results go down on their own stream as soon as the chunk's kernels are through
+        cudaEvent_t ev_k = h->sw_ev[2 + n_chunks + c];
+        HX_TRY(cudaEventRecord(ev_k, s), "event");
+        HX_TRY(cudaStreamWaitEvent(h->sw_out, ev_k, 0), "event");
+        HX_TRY(cudaMemcpyAsync(out_assign + o, h->st_assign + o, n * sizeof(int32_t), cudaMemcpyDeviceToHost, h->sw_out), "copy assign");
+        HX_TRY(cudaMemcpyAsync(out_cost + o, h->st_cost + o, n * sizeof(float), cudaMemcpyDeviceToHost, h->sw_out), "copy cost");
+    }
+    HX_TRY(cudaEventRecord(ev_done, h->sw_out), "event");
+    HX_TRY(cudaStreamWaitEvent(s, ev_done, 0), "event");         // the caller's stream ends after the last copy
+    return HX_OK;
 }
 
 

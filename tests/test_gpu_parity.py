@@ -376,6 +376,46 @@ def test_async_host_entry_point_chains_dependent_batches(hx, oracle):
     gc.close()
 
 
+@pytest.mark.parametrize("reset", [False, True])
+def test_sweep_entry_point_equals_the_batches_one_by_one(hx, oracle, reset):
+    """hx_schedule_sweep_host (copies on their own streams, overlapped with the kernels) against the same chunks
+    run one by one through the device entry point, with and without the reset of the free KV tokens ahead of
+    every chunk; a ragged last chunk; twice in a row on the same handle."""
+    import torch
+    wl = make_workload("sweep", scale=1 / 32)
+    oc, gc, dag = _prepare(hx, oracle, wl)
+    gc.set_options(score_mode=hx.HX_MODE_RATIO, topk=4, commit=1, alpha=wl.alpha)
+    total = len(wl.calls) - 37
+    n = 1500                                               # 6 chunks, the last one shorter
+    qP0, free0 = wl.load_s[:wl.P].copy(), wl.kv_free[wl.P:].copy()
+    want_a, want_c = [], []
+    for lo in range(0, total, n):
+        if reset:
+            gc.update_loads(kv_free=free0)
+        a, c = gc.schedule_batch(wl.calls[lo:min(total, lo + n)])
+        want_a.append(a.cpu().numpy()); want_c.append(c.cpu().numpy())
+    want_a, want_c = np.concatenate(want_a), np.concatenate(want_c)
+    loads_want = gc.read_loads()
+    calls_pin = torch.from_numpy(wl.calls[:total].view(np.uint8).reshape(-1, 16).copy()).pin_memory()
+    a_pin = torch.empty(total, dtype=torch.int32).pin_memory()
+    c_pin = torch.empty(total, dtype=torch.float32).pin_memory()
+    free_pin = torch.from_numpy(free0.astype(np.float32)).pin_memory()
+    cn = calls_pin.numpy().view(hx.CALL_DTYPE).reshape(-1)
+    sp = torch.cuda.current_stream().cuda_stream
+    for rep in range(2):
+        a_pin.fill_(-7); c_pin.fill_(-7.0)
+        gc.update_loads(qP=qP0, kv_free=free0)
+        hx.hx_schedule_sweep_host(gc.h, cn, n, free_pin.numpy() if reset else None, a_pin.numpy(), c_pin.numpy(), sp)
+        torch.cuda.current_stream().synchronize()
+        assert np.array_equal(a_pin.numpy(), want_a) and np.array_equal(c_pin.numpy(), want_c)
+        for x, y in zip(gc.read_loads(), loads_want):
+            assert np.array_equal(x, y)
+    with pytest.raises(hx.HxError):
+        hx.hx_schedule_sweep_host(gc.h, cn, 0, None, a_pin.numpy(), c_pin.numpy(), sp)
+    assert gc.status() == 0
+    gc.close()
+
+
 @pytest.mark.parametrize("P, D, n", [(4, 9, 300), (70, 130, 700)])
 def test_quadratic_prefill_variant(hx, oracle, P, D, n):
     """Attention FLOPs per token pair set on both sides: scoring, top-K lists and the greedy planner agree
