@@ -112,7 +112,8 @@ __global__ void __launch_bounds__(kThreads, 1) hx_decode_kernel(const __grid_con
     float* capDs = reinterpret_cast<float*>(smem);              // [D]
     int* typeDs = reinterpret_cast<int*>(capDs + D);            // [D]
     int* Ks = typeDs + D;                                       // [D] breakpoints per instance
-    float* cn = reinterpret_cast<float*>(Ks + D);               // [n]
+    float* umax = reinterpret_cast<float*>(Ks + D);             // [D] largest usage of any segment of the instance
+    float* cn = umax + D;                                       // [n]
     float* co = cn + n;
     float* cel = co + n;
     float* cH = cel + n;
@@ -150,10 +151,15 @@ __global__ void __launch_bounds__(kThreads, 1) hx_decode_kernel(const __grid_con
     __syncthreads();
     for (int d = warp; d < D; d += kWarps) {                    // simulated state starts as the snapshot
         float* tt = seg_t(d); float* uu = seg_u(d);
+        float mx = 0.f;
         for (int i = lane; i < Ks[d]; i += 32) {
             tt[i] = prm.base.t[(size_t)d * prm.base.cap + i];
-            uu[i] = prm.base.u[(size_t)d * prm.base.cap + i];
+            const float uv = prm.base.u[(size_t)d * prm.base.cap + i];
+            uu[i] = uv; mx = fmaxf(mx, uv);
         }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        if (lane == 0) umax[d] = mx;
     }
     for (int c = tid; c < n; c += kThreads) {
         const int gcall = c * NC + rank;
@@ -197,6 +203,13 @@ __global__ void __launch_bounds__(kThreads, 1) hx_decode_kernel(const __grid_con
             for (int d = lane; d < D; d += 32) {
                 if ((lk >= 0 && lk != d) || !(m <= capDs[d])) continue;
                 const float tau = __fmul_rn(__fmul_rn(ot, step), prm.ct.invB[typeDs[d]]);
+                if (__fadd_rn(umax[d], m) <= capDs[d]) {
+                    // room in every segment (token counts are whole numbers, so the sum is exact): the walk below
+                    // would accept the ready time itself
+                    const float fin = __fadd_rn(rd, tau);
+                    if (fin < best) { best = fin; bs = rd; bd = d; }
+                    continue;
+                }
                 const float* tt = seg_t(d);
                 const float* uu = seg_u(d);
                 const int K = Ks[d];
@@ -344,8 +357,11 @@ __global__ void __launch_bounds__(kThreads, 1) hx_decode_kernel(const __grid_con
                 } else {
                     const int a = warp_cut(tt, uu, K, st, lane);
                     const int b = warp_cut(tt, uu, K, en, lane);
-                    for (int k = a + lane; k < b; k += 32) uu[k] = __fadd_rn(uu[k], m);
-                    if (lane == 0) { Ks[d] = K; s_d = d; }
+                    float mx = 0.f;
+                    for (int k = a + lane; k < b; k += 32) { const float uv = __fadd_rn(uu[k], m); uu[k] = uv; mx = fmaxf(mx, uv); }
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+                    if (lane == 0) { Ks[d] = K; s_d = d; umax[d] = fmaxf(umax[d], mx); }
                 }
             }
             if (lane == 0) s_ndirty = 0;
@@ -378,7 +394,7 @@ constexpr int kCluster = 8;                    // blocks of the cluster used for
 constexpr int kClusterFrom = 256;              // queues longer than this use the cluster
 
 static size_t decode_smem(const HxTables& t, int calls_per_block) {
-    return (3 * (size_t)t.D + 11 * (size_t)calls_per_block) * 4 + (size_t)calls_per_block * 2 + 16;
+    return (4 * (size_t)t.D + 11 * (size_t)calls_per_block) * 4 + (size_t)calls_per_block * 2 + 16;
 }
 // With the pool of breakpoints behind the per-call state: two layouts of pool_T entries, times and usage.
 static size_t decode_pool_smem(const HxTables& t, int calls_per_block, int pool_T) {
