@@ -200,35 +200,59 @@ __global__ void __launch_bounds__(kThreads, 1) hx_decode_kernel(const __grid_con
             const float rd = cready[c];
             const int lk = clock_[c];
             float best = HX_INF, bs = 0.f; int bd = 0x7fffffff;
-            for (int d = lane; d < D; d += 32) {
-                if ((lk >= 0 && lk != d) || !(m <= capDs[d])) continue;
-                const float tau = __fmul_rn(__fmul_rn(ot, step), prm.ct.invB[typeDs[d]]);
-                if (__fadd_rn(umax[d], m) <= capDs[d]) {
-                    // room in every segment (token counts are whole numbers, so the sum is exact): the walk below
-                    // would accept the ready time itself
-                    const float fin = __fadd_rn(rd, tau);
-                    if (fin < best) { best = fin; bs = rd; bd = d; }
-                    continue;
-                }
-                const float* tt = seg_t(d);
-                const float* uu = seg_u(d);
-                const int K = Ks[d];
-                int k = 0, hi = K - 1;                          // segment that holds the ready time: largest k with
-                while (k < hi) {                                // t[k] <= ready (t[0] = 0), by bisection
-                    const int mid = (k + hi + 1) >> 1;
-                    if (tt[mid] <= rd) k = mid; else hi = mid - 1;
-                }
-                float cand = rd, fin;
-                for (;; ++k) {
-                    const float seg_end = (k + 1 < K) ? tt[k + 1] : HX_INF;
-                    if (__fadd_rn(uu[k], m) > capDs[d]) {
-                        if (k + 1 >= K) { fin = HX_INF; break; }   // last segment is empty on a valid state: not reached
-                        cand = seg_end; continue;
+            for (int d0 = 0; d0 < D; d0 += 32) {
+                const int d = d0 + lane;
+                bool walk = false; float tau = 0.f;
+                if (d < D && !((lk >= 0 && lk != d) || !(m <= capDs[d]))) {
+                    tau = __fmul_rn(__fmul_rn(ot, step), prm.ct.invB[typeDs[d]]);
+                    if (__fadd_rn(umax[d], m) <= capDs[d]) {
+                        // room in every segment (token counts are whole numbers, so the sum is exact): the walk
+                        // would accept the ready time itself
+                        const float fin = __fadd_rn(rd, tau);
+                        if (fin < best) { best = fin; bs = rd; bd = d; }
+                    } else {
+                        walk = true;
                     }
-                    fin = __fadd_rn(cand, tau);
-                    if (seg_end >= fin) break;
                 }
-                if (fin < best) { best = fin; bs = cand; bd = d; }   // ascending d per lane: lowest d kept
+                // the instances that have to be walked, one after the other, the warp on 32 segments at a time:
+                // the sequential walk stops at the first segment that either has no room (the candidate start moves
+                // to the end of the run of such segments) or ends at or after candidate + duration (accepted)
+                unsigned todo = __ballot_sync(0xffffffffu, walk);
+                while (todo) {
+                    const int src = __ffs(todo) - 1;
+                    todo &= todo - 1;
+                    const int dd = d0 + src;
+                    const float tau_d = __shfl_sync(0xffffffffu, tau, src);
+                    const float* tt = seg_t(dd);
+                    const float* uu = seg_u(dd);
+                    const int K = Ks[dd];
+                    const float capd = capDs[dd];
+                    int k = warp_find_segment(tt, K, rd, lane);           // segment that holds the ready time
+                    float cand = rd, fin = HX_INF;
+                    for (;;) {
+                        const int i = k + lane;
+                        const bool in = i < K;
+                        const float end_i = (in && i + 1 < K) ? tt[i + 1] : HX_INF;
+                        const bool viol = in && __fadd_rn(uu[i], m) > capd;
+                        const float f = __fadd_rn(cand, tau_d);
+                        const bool acc = in && !viol && end_i >= f;
+                        const unsigned mv = __ballot_sync(0xffffffffu, viol), ma = __ballot_sync(0xffffffffu, acc);
+                        const int fv = mv ? __ffs(mv) - 1 : 32, fa = ma ? __ffs(ma) - 1 : 32;
+                        if (fa < fv) { fin = f; break; }
+                        if (fv == 32) {                                   // no decision among these 32 segments
+                            k += 32;
+                            if (k >= K) break;                            // not reached: the last segment ends at +inf
+                            continue;
+                        }
+                        const unsigned rest = ~(mv >> fv);                // zero bits: the run of full segments goes on
+                        const int len = rest ? __ffs(rest) - 1 : 32 - fv;
+                        const int last = fv + len - 1;
+                        if (k + last + 1 >= K) break;                     // the last segment has no room: no start at all
+                        cand = __shfl_sync(0xffffffffu, end_i, last);
+                        k += last + 1;
+                    }
+                    if (lane == src && fin < best) { best = fin; bs = cand; bd = dd; }   // ascending d per lane: lowest d kept
+                }
             }
 #pragma unroll
             for (int off = 16; off > 0; off >>= 1) {
