@@ -51,7 +51,9 @@ struct GreedyParams {
     int* status;
 };
 
-template <int NC>   // blocks of the cluster (1 = a plain single block)
+// CACHE: the per-class prefill and decode times, the KV bytes and the demand of every call are computed once and kept
+// in shared memory ([class][call]); without it a warp recomputes them whenever it re-projects a call.
+template <int NC, bool CACHE>   // NC: blocks of the cluster (1 = a plain single block)
 __global__ void __launch_bounds__(kThreads, 1) hx_greedy_kernel(const __grid_constant__ GreedyParams prm) {
     extern __shared__ __align__(16) unsigned char smem[];
     __shared__ float red_v[kWarps];
@@ -83,7 +85,11 @@ __global__ void __launch_bounds__(kThreads, 1) hx_greedy_kernel(const __grid_con
     float* cR = cH + n;                                        // [n] projected ratio, -inf if it cannot be taken
     int* cpair = reinterpret_cast<int*>(cR + n);               // [n] best pair as p << 16 | d, kNoPair, kDead
     int* cmodel = cpair + n;                                   // [n]
-    unsigned short* dirty = reinterpret_cast<unsigned short*>(cmodel + n);   // [n] calls to re-project
+    float* ckv = reinterpret_cast<float*>(cmodel + n);         // [n] KV bytes of the prompt (CACHE)
+    float* cmm = ckv + (CACHE ? n : 0);                        // [n] demand in tokens (CACHE)
+    float* tpreC = cmm + (CACHE ? n : 0);                      // [G][n] prefill time per GPU class (CACHE)
+    float* tdecC = tpreC + (CACHE ? (size_t)G * n : 0);        // [G][n] decode time per GPU class (CACHE)
+    unsigned short* dirty = reinterpret_cast<unsigned short*>(tdecC + (CACHE ? (size_t)G * n : 0));   // [n] calls to re-project
 
     for (int i = tid; i < P * D; i += kThreads) { const int p = i / D, d = i - p * D; invL[i] = T.invLT[(size_t)d * T.Ppad + p]; }
     for (int p = tid; p < P; p += kThreads) { qPs[p] = T.qP[p]; typePs[p] = T.typeP[p]; }
@@ -104,6 +110,20 @@ __global__ void __launch_bounds__(kThreads, 1) hx_greedy_kernel(const __grid_con
         cR[c] = HX_NEG_INF;
         cpair[c] = bad ? kDead : kNoPair;
         dirty[c] = (unsigned short)c;
+        if (CACHE) {
+            const float nt = cn[c], ot = co[c];
+            const int mdl = cmodel[c];
+            const float phi = prm.ct.phi[mdl], omega = prm.ct.omega[mdl], kappa = prm.ct.kappa[mdl];
+            const float kvB = __fmul_rn(nt, kappa);
+            const float ctx = __fmaf_rn(0.5f, __fsub_rn(ot, 1.0f), nt);
+            const float step = __fmaf_rn(kappa, ctx, omega);
+            ckv[c] = kvB; cmm[c] = __fadd_rn(nt, ot);
+            for (int g = 0; g < G; ++g) {
+                const float iF = prm.ct.invF[g], iB = prm.ct.invB[g];
+                tpreC[g * n + c] = fmaxf(__fmul_rn(__fmaf_rn(__fmul_rn(nt, prm.ct.psi[mdl]), nt, __fmul_rn(nt, phi)), iF), __fmul_rn(__fadd_rn(omega, kvB), iB));
+                tdecC[g * n + c] = __fmul_rn(__fmul_rn(ot, step), iB);
+            }
+        }
         prm.out_assign[gcall] = -1; prm.out_ratio[gcall] = HX_INF; prm.out_order[gcall] = -1;
         if (prm.out_delta) prm.out_delta[gcall] = HX_INF;
     }
@@ -113,24 +133,33 @@ __global__ void __launch_bounds__(kThreads, 1) hx_greedy_kernel(const __grid_con
     for (int it = 0; it < n_all; ++it) {
         // (1) re-project the listed calls: one warp per call, lanes over the pairs
         const int nd = s_ndirty;
-        float* tpre = scratch + warp * 64;
-        float* tdec = tpre + 32;
         for (int i = warp; i < nd; i += kWarps) {
             const int c = dirty[i];
             if (cpair[c] == kDead) continue;                   // rejected at load time (warp-uniform)
-            const float nt = cn[c], ot = co[c];
-            const int mdl = cmodel[c];
-            const float phi = prm.ct.phi[mdl], omega = prm.ct.omega[mdl], kappa = prm.ct.kappa[mdl];
-            const float kvB = __fmul_rn(nt, kappa);
-            const float ctx = __fmaf_rn(0.5f, __fsub_rn(ot, 1.0f), nt);
-            const float step = __fmaf_rn(kappa, ctx, omega);
-            const float m = __fadd_rn(nt, ot);
-            if (lane < G) {
-                const float iF = prm.ct.invF[lane], iB = prm.ct.invB[lane];
-                tpre[lane] = fmaxf(__fmul_rn(__fmaf_rn(__fmul_rn(nt, prm.ct.psi[mdl]), nt, __fmul_rn(nt, phi)), iF), __fmul_rn(__fadd_rn(omega, kvB), iB));
-                tdec[lane] = __fmul_rn(__fmul_rn(ot, step), iB);
+            // per-class times of this call: tpre[g * ts], tdec[g * ts]
+            const float* tpre; const float* tdec; int ts;
+            float kvB, m;
+            if (CACHE) {
+                tpre = tpreC + c; tdec = tdecC + c; ts = n;
+                kvB = ckv[c]; m = cmm[c];
+            } else {
+                float* wpre = scratch + warp * 64;
+                float* wdec = wpre + 32;
+                const float nt = cn[c], ot = co[c];
+                const int mdl = cmodel[c];
+                const float phi = prm.ct.phi[mdl], omega = prm.ct.omega[mdl], kappa = prm.ct.kappa[mdl];
+                kvB = __fmul_rn(nt, kappa);
+                const float ctx = __fmaf_rn(0.5f, __fsub_rn(ot, 1.0f), nt);
+                const float step = __fmaf_rn(kappa, ctx, omega);
+                m = __fadd_rn(nt, ot);
+                if (lane < G) {
+                    const float iF = prm.ct.invF[lane], iB = prm.ct.invB[lane];
+                    wpre[lane] = fmaxf(__fmul_rn(__fmaf_rn(__fmul_rn(nt, prm.ct.psi[mdl]), nt, __fmul_rn(nt, phi)), iF), __fmul_rn(__fadd_rn(omega, kvB), iB));
+                    wdec[lane] = __fmul_rn(__fmul_rn(ot, step), iB);
+                }
+                __syncwarp();
+                tpre = wpre; tdec = wdec; ts = 1;
             }
-            __syncwarp();
             float best = HX_INF; int bj = 0x7fffffff;
             // a lane keeps its decode instance and walks the prefill instances, so that everything that
             // depends on d alone (room, decode time, availability) is read once per call: with D lanes per
@@ -140,9 +169,9 @@ __global__ void __launch_bounds__(kThreads, 1) hx_greedy_kernel(const __grid_con
             for (int d = lane - prow * dlanes; d < D; d += dlanes) {
                 const bool fits = m <= capDs[d] && m <= frees[d];
                 if (!fits) continue;                           // every pair on d is +inf: cannot be the minimum
-                const float Dd = tdec[typeDs[d]], qd = qDs[d];
+                const float Dd = tdec[typeDs[d] * ts], qd = qDs[d];
                 for (int p = prow; p < P; p += pstep) {
-                    const float A = __fadd_rn(qPs[p], tpre[typePs[p]]);
+                    const float A = __fadd_rn(qPs[p], tpre[typePs[p] * ts]);
                     const float ready = __fmaf_rn(kvB, invL[p * D + d], A);
                     const float fin = __fadd_rn(fmaxf(ready, qd), Dd);
                     const int j = (p << 16) | d;
@@ -279,6 +308,13 @@ static size_t greedy_smem(const HxTables& t, int calls_per_block) {
     return ((size_t)t.P * t.D + 2 * (size_t)t.P + 5 * (size_t)t.D + kWarps * 64 + 7 * (size_t)calls_per_block) * 4 +
            (size_t)calls_per_block * 2 + 16;
 }
+// With the per-class times of every call kept in shared memory.
+static size_t greedy_cache_smem(const HxTables& t, int calls_per_block) {
+    return greedy_smem(t, calls_per_block) + (size_t)calls_per_block * (2 + 2 * (size_t)t.G) * 4;
+}
+static bool greedy_cache_ok(const HxTables& t, int calls_per_block) {
+    return greedy_cache_smem(t, calls_per_block) <= (size_t)200 * 1024;
+}
 
 // Shared memory of one block for a queue of n_calls (the longest queue a single block must be able
 // to take is kClusterFrom calls; longer ones are split over the cluster when the device can run it).
@@ -296,9 +332,12 @@ cudaError_t hx_launch_greedy(const HxTables& t, const HxConstTables& ct, const H
     prm.status = status;
     cudaError_t e;
     if (n_calls > kClusterFrom) {
-        const size_t smem = greedy_smem(t, (n_calls + kCluster - 1) / kCluster);
-        static size_t allowed[64];
-        if ((e = hx_opt_in_smem(hx_greedy_kernel<kCluster>, smem, allowed, 40 * 1024)) != cudaSuccess) return e;
+        const int cpb = (n_calls + kCluster - 1) / kCluster;
+        const bool cache = greedy_cache_ok(t, cpb);
+        const size_t smem = cache ? greedy_cache_smem(t, cpb) : greedy_smem(t, cpb);
+        static size_t allowed[64], allowed_c[64];
+        void (*kern)(GreedyParams) = cache ? hx_greedy_kernel<kCluster, true> : hx_greedy_kernel<kCluster, false>;
+        if ((e = hx_opt_in_smem(kern, smem, cache ? allowed_c : allowed, 40 * 1024)) != cudaSuccess) return e;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(kCluster); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = smem; cfg.stream = stream;
         cudaLaunchAttribute attr[1];
@@ -306,18 +345,24 @@ cudaError_t hx_launch_greedy(const HxTables& t, const HxConstTables& ct, const H
         attr[0].val.clusterDim.x = kCluster; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr; cfg.numAttrs = 1;
         int n_clusters = 0;
-        if (cudaOccupancyMaxActiveClusters(&n_clusters, hx_greedy_kernel<kCluster>, &cfg) == cudaSuccess && n_clusters >= 1) {
-            e = cudaLaunchKernelEx(&cfg, hx_greedy_kernel<kCluster>, prm);
+        if (cudaOccupancyMaxActiveClusters(&n_clusters, kern, &cfg) == cudaSuccess && n_clusters >= 1) {
+            e = cudaLaunchKernelEx(&cfg, kern, prm);
             if (e == cudaSuccess) ++*launches;
             return e;
         }
         (void)cudaGetLastError();              // the device cannot host the cluster: one block, if the queue fits
         if (greedy_smem(t, n_calls) > (size_t)227 * 1024) return cudaErrorInvalidConfiguration;
     }
-    const size_t smem = greedy_smem(t, n_calls);
-    static size_t allowed1[64];
-    if ((e = hx_opt_in_smem(hx_greedy_kernel<1>, smem, allowed1, 40 * 1024)) != cudaSuccess) return e;
-    hx_greedy_kernel<1><<<1, kThreads, smem, stream>>>(prm);
+    const bool cache = greedy_cache_ok(t, n_calls);
+    const size_t smem = cache ? greedy_cache_smem(t, n_calls) : greedy_smem(t, n_calls);
+    static size_t allowed1[64], allowed1_c[64];
+    if (cache) {
+        if ((e = hx_opt_in_smem(hx_greedy_kernel<1, true>, smem, allowed1_c, 40 * 1024)) != cudaSuccess) return e;
+        hx_greedy_kernel<1, true><<<1, kThreads, smem, stream>>>(prm);
+    } else {
+        if ((e = hx_opt_in_smem(hx_greedy_kernel<1, false>, smem, allowed1, 40 * 1024)) != cudaSuccess) return e;
+        hx_greedy_kernel<1, false><<<1, kThreads, smem, stream>>>(prm);
+    }
     e = cudaGetLastError();
     if (e == cudaSuccess) ++*launches;
     return e;
