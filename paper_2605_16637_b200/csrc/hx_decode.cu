@@ -341,16 +341,17 @@ __global__ void __launch_bounds__(kThreads, 1) hx_decode_kernel(const __grid_con
                 int K = Ks[d];
                 bool room = POOL ? K + 2 <= roff[d + 1] - roff[d] : K + 2 <= cap;
                 if (POOL && !room) {
-                    // lay the regions out again in the other half: every instance its breakpoints plus an equal
-                    // share of what is free, after two entries set aside for this commit
+                    // lay the regions out again in the other half, after two entries set aside for this commit
                     if (lane == 0) {
                         int sum = 0;
                         for (int e = 0; e < D; ++e) sum += Ks[e];
                         const int free_now = PT - sum - 2;
                         if (free_now >= 0) {
-                            const int share = free_now / D;
+                            // half of what is free goes to the instance that ran full (it is the popular one and
+                            // would be back soon with an equal share), the rest is split evenly
+                            const int mine = free_now / 2, share = (free_now - mine) / D;
                             int o = 0;
-                            for (int e = 0; e < D; ++e) { roff2[e] = o; o += Ks[e] + share + (e == d ? 2 : 0); }
+                            for (int e = 0; e < D; ++e) { roff2[e] = o; o += Ks[e] + share + (e == d ? 2 + mine : 0); }
                             roff2[D] = o;
                         } else {
                             roff2[D] = -1;                       // the pool itself is full: the host sized it too small
