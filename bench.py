@@ -514,7 +514,7 @@ LOADS = (4.0, 32.0, 256.0)       # offered stand-alone work per second and prefi
 
 
 def replay_leg():
-    """Side measurement, outside the timed region: the event-driven replay (Section 6, Section 7.2) of the
+    """Side measurement, outside the timed region: the event-driven replay (Section 6, Section 7.3) of the
     medium configuration (512 workflows, 16 x 16 instances) at three offered loads; Req95 / Req99 and wall
     clock, and the oracle's replay of the middle load on one core beside it."""
     import paper_2605_16637_b200 as hx

@@ -35,7 +35,8 @@ extern "C" {
 #define HX_ERR_CUDA         (-2)   /* a CUDA runtime call failed; message holds cudaGetErrorString */
 #define HX_ERR_CYCLE        (-3)   /* the uploaded graph is not acyclic */
 #define HX_ERR_NOT_READY    (-4)   /* scoring needs horizons but hx_critical_path was not enqueued */
-#define HX_ERR_TIMEOUT      (-5)   /* a bounded device-side wait ran out (reported by hx_get_status) */
+#define HX_ERR_TIMEOUT      (-5)   /* reserved for a bounded device-side wait that runs out; no entry point of
+                                      this version waits on the device, so the code is never returned */
 #define HX_ERR_OOM          (-6)   /* host or device allocation failed */
 
 /* out_cost of hx_schedule_batch (Delta = earliest projected decode finish of the call) */
@@ -66,7 +67,8 @@ typedef struct { float peak_tflops, hbm_tbps; } hx_gpu_type;
  * KV-capacity bound).  load_s: seconds until a prefill instance has drained
  * its queue, or earliest time a decode instance can admit a new call.
  * kv_cap_tokens is Cap(d) of Eq. 4, kv_free_tokens the part of it not in use
- * (both ignored for prefill instances). */
+ * (both ignored for prefill instances; whole numbers in [0, 2^24) for decode
+ * instances, HX_ERR_INVALID_ARG otherwise). */
 typedef struct {
     uint32_t type;
     uint32_t role;
@@ -113,8 +115,10 @@ int hx_cluster_create(const hx_gpu_type* gpu_types, int n_types,
 
 /* Replace queue loads and free KV tokens (State Collector refresh between
  * scheduler invocations).  Each pointer is host memory or NULL (= keep):
- * qP[n_prefill], qD[n_decode], kv_free[n_decode].  The copies are enqueued on
- * `stream`; the host arrays may be reused when the call returns. */
+ * qP[n_prefill], qD[n_decode], kv_free[n_decode] (finite and >= 0; kv_free
+ * whole numbers below 2^24; HX_ERR_INVALID_ARG otherwise, nothing changed).
+ * The copies are enqueued on `stream`; the host arrays may be reused when the
+ * call returns. */
 int hx_cluster_update_loads(hx_cluster* h, const float* qP, const float* qD,
                             const float* kv_free, void* stream);
 
@@ -241,7 +245,10 @@ int hx_set_options(hx_cluster* h, const hx_options* opts);
  * device while doing so).  Needs hx_critical_path to have been enqueued since
  * the last upload unless HX_FLAG_NO_DAG is set (else HX_ERR_NOT_READY).
  * A call record whose model or node id is out of range gets assignment -1,
- * cost +inf, and raises HX_ERR_INVALID_ARG in the status word.
+ * cost +inf, and raises HX_ERR_INVALID_ARG in the status word; with topk > 0
+ * the same happens to a record whose prompt or output length is negative, not
+ * a whole number, or sums to 2^24 or more (the capacity pass takes its decisions
+ * on integer token counts).
  * n_calls = 0 is a no-op.  Enqueues on `stream`; does not synchronise. */
 int hx_schedule_batch(hx_cluster* h, const hx_call* calls, int n_calls,
                       int32_t* out_assign, float* out_cost, void* stream);
@@ -351,7 +358,7 @@ int hx_schedule_greedy_plan(hx_cluster* h, const hx_call* calls, int n_calls,
 
 /* Minimal event-driven replay around the greedy planner (Section 6: the
  * stand-alone simulator tracks every call from waiting for prefill to
- * completion; Section 7.2: Req95 / Req99).  Workflows arrive at arrival_s[w]; a
+ * completion; Section 7.3: Req95 / Req99).  Workflows arrive at arrival_s[w]; a
  * call becomes ready when all its predecessors have completed (Section 4.1); at
  * every event time (an arrival or a completion; equal time stamps are taken
  * together) all ready calls are planned by hx_schedule_greedy_plan in ratio mode
@@ -436,8 +443,10 @@ int hx_schedule_decode(hx_cluster* h, const hx_call* calls, const int32_t* lock,
  * Any output argument may be NULL. */
 int hx_get_topk(hx_cluster* h, const int32_t** pairs, const float** costs, const float** prio);
 
-/* Device-side status word (0 = fine, else an HX_ERR_* raised inside a kernel,
- * e.g. HX_ERR_TIMEOUT from a bounded wait).  Synchronises `stream`. */
+/* Device-side status word: 0 = fine, else the HX_ERR_* code a kernel raised
+ * (HX_ERR_INVALID_ARG for a bad call record) in work enqueued on `stream` since
+ * the previous hx_get_status.  Reads the word, clears it, and synchronises
+ * `stream`, so each call reports on the batches since the one before. */
 int hx_get_status(hx_cluster* h, int* status, void* stream);
 
 /* Tracing aid (the paper reports scheduler time per invocation, Section 7.7):

@@ -3,7 +3,7 @@
 TEST INFRASTRUCTURE ONLY: the plain definition that the library's replay is checked
 against.  It shares no code with the CUDA path and is never called from it.
 
-What it models (Section 6, the stand-alone simulator; Section 7.2, Req95 / Req99):
+What it models (Section 6, the stand-alone simulator; Section 7.3, Req95 / Req99):
 workflows arrive over time, a call becomes ready when all its predecessors have
 completed (Section 4.1), and at every event time the scheduler plans all ready
 calls with the recomputing greedy of Algorithm 1 (projected ratio of Eq. 2) against

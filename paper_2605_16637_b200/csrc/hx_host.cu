@@ -160,6 +160,9 @@ void free_pool(std::vector<void*>& pool) {
 
 bool good_rate(float x) { return std::isfinite(x) && x > 0.0f; }
 bool good_load(float x) { return std::isfinite(x) && x >= 0.0f; }
+// KV token counts are whole numbers below 2^24: sums and differences of such values are exact in
+// binary32, which the capacity pass relies on when it takes its decisions on integers.
+bool good_tokens(float x) { return std::isfinite(x) && x >= 0.0f && x < 16777216.0f && x == std::floor(x); }
 
 #define HX_TRY(call, what) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return fail_cuda(h, e_, what); } while (0)
 
@@ -408,8 +411,8 @@ int hx_cluster_create(const hx_gpu_type* gpu_types, int n_types, const hx_instan
     for (int i = 0; i < n_instances; ++i) {
         if (instances[i].type >= (uint32_t)n_types) return fail(nullptr, HX_ERR_INVALID_ARG, "instance type out of range");
         if (!good_load(instances[i].load_s)) return fail(nullptr, HX_ERR_INVALID_ARG, "instance load must be finite and >= 0");
-        if (i >= P && (!good_load(instances[i].kv_cap_tokens) || !good_load(instances[i].kv_free_tokens)))
-            return fail(nullptr, HX_ERR_INVALID_ARG, "KV capacities must be finite and >= 0");
+        if (i >= P && (!good_tokens(instances[i].kv_cap_tokens) || !good_tokens(instances[i].kv_free_tokens)))
+            return fail(nullptr, HX_ERR_INVALID_ARG, "KV capacities and free KV tokens must be whole numbers in [0, 2^24)");
     }
     for (int p = 0; p < P; ++p)
         for (int d = 0; d < D; ++d)
@@ -488,8 +491,11 @@ int hx_cluster_update_loads(hx_cluster* h, const float* qP, const float* qD, con
     const int n[3] = {h->P, h->D, h->D};
     for (int k = 0; k < 3; ++k) {
         if (!src[k]) continue;
-        for (int i = 0; i < n[k]; ++i)
+        for (int i = 0; i < n[k]; ++i) {
             if (!good_load(src[k][i])) return fail(h, HX_ERR_INVALID_ARG, "loads must be finite and >= 0");
+            if (k == 2 && !good_tokens(src[k][i]))
+                return fail(h, HX_ERR_INVALID_ARG, "free KV tokens must be whole numbers in [0, 2^24)");
+        }
     }
     for (int k = 0; k < 3; ++k)
         if (src[k])
@@ -1057,7 +1063,8 @@ int hx_schedule_sweep_host(hx_cluster* h, const hx_call* calls, int n_calls, int
         return fail(h, HX_ERR_INVALID_ARG, "chunk too large for the capacity-conflict pass");
     if (kv_free_reset)
         for (int d = 0; d < h->D; ++d)
-            if (!good_load(kv_free_reset[d])) return fail(h, HX_ERR_INVALID_ARG, "loads must be finite and >= 0");
+            if (!good_tokens(kv_free_reset[d]))
+                return fail(h, HX_ERR_INVALID_ARG, "free KV tokens must be whole numbers in [0, 2^24)");
     DeviceGuard guard(h->device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (int rc = reserve_staging(h, n_calls)) return rc;
@@ -1355,6 +1362,7 @@ int hx_get_status(hx_cluster* h, int* status, void* stream) {
     DeviceGuard guard(h->device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     HX_TRY(cudaMemcpyAsync(status, h->status, sizeof(int), cudaMemcpyDeviceToHost, s), "read status");
+    HX_TRY(cudaMemsetAsync(h->status, 0, sizeof(int), s), "clear status");      // read and clear: the next read covers later work only
     HX_TRY(cudaStreamSynchronize(s), "cudaStreamSynchronize");
     return HX_OK;
 }

@@ -525,6 +525,11 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
                 const uint4 raw = __ldg(reinterpret_cast<const uint4*>(prm.s.calls) + gc);
                 float elapsed = 0.f, tail = 0.f, H = 1.f;
                 bool bad = raw.y >= (unsigned)T.M;
+                if (K > 0) {
+                    // the capacity pass decides on integers: token counts must be whole and their sum below 2^24
+                    const float n = __uint_as_float(raw.z), o = __uint_as_float(raw.w);
+                    bad |= !(n >= 0.f && o >= 0.f && n == floorf(n) && o == floorf(o) && __fadd_rn(n, o) < 16777216.0f);
+                }
                 if (!(prm.s.flags & HX_FLAG_NO_DAG)) {
                     if (raw.x < prm.dag.n_nodes) {
                         const uint32_t w = wfS[c];

@@ -74,7 +74,8 @@ def _check(hx, gc, oc, oracle, calls, lock, ready, ptr, end, tok, commit=0, run_
 
 @pytest.mark.parametrize("D, C, per, caps", [(1, 10, 2, (4000.0,)), (2, 40, 3, (3000.0, 6000.0)),
                                              (5, 150, 4, (3000.0, 6000.0, 20000.0)), (16, 400, 6, (4000.0, 8000.0)),
-                                             (40, 700, 3, (6000.0,)), (64, 1024, 2, (5000.0, 9000.0))])
+                                             (40, 700, 3, (6000.0,)), (64, 1024, 2, (5000.0, 9000.0)),
+                                             (16, 2048, 4, (4000.0, 8000.0))])     # the longest queue accepted
 def test_decode_scheduler_matches_oracle(hx, oracle, D, C, per, caps):
     rng = np.random.default_rng(200 + D)
     gc, oc = _pair(hx, rng, D, caps)

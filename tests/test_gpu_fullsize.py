@@ -1,16 +1,23 @@
 """Parity at the full sizes of the evaluation configurations, in the launch configuration the
-benchmark times.  The oracle is too slow to redo everything, so it recomputes sampled outputs
-one by one (with the horizons of exactly the workflows those calls belong to) and, for the
-capacity pass, the complete first scheduler invocation; the rest is checked through properties
-that hold at any size."""
+benchmark times.  Every output is compared with the oracle: all 65,536 calls of the large
+configuration, the 1,000,000-node forest and all 50,000 calls of the critical-path stress, and all
+16 scheduler invocations of the sweep, chained through the prefill queues exactly as the benchmark
+chains them.  The oracle is single-threaded; the test spreads independent slices of calls over the
+host's cores (the oracle's functions are pure, and ctypes releases the interpreter lock), which
+changes no result."""
+import os
+from concurrent.futures import ThreadPoolExecutor
+
 import numpy as np
 import pytest
 
 import hx_helpers as hh
-from hx_synth import make_workload, sub_forest
+from hx_synth import make_workload
 from oracle import hx_oracle as ho
 
-pytestmark = [pytest.mark.gpu, pytest.mark.timeout(900)]
+pytestmark = [pytest.mark.gpu, pytest.mark.timeout(1500)]
+
+N_THREADS = max(1, min(16, (os.cpu_count() or 2) - 1))
 
 
 @pytest.fixture(scope="module")
@@ -21,16 +28,24 @@ def hx():
     return mod
 
 
-def _oracle_dag_for(oracle, oc, wl, workflows):
-    """Oracle horizons of the given workflows only, scattered into full-size arrays."""
-    workflows = np.unique(workflows)
-    rp, col, lwf, ids = sub_forest(wl, workflows)
-    cost = wl.node_cost[ids] if wl.node_cost is not None else hh.oracle_node_costs(oracle, oc, wl.node_calls[ids])
-    sub = oracle.longest_path(rp, col, cost, lwf, workflows.shape[0])
-    tail = np.zeros(wl.n_nodes, np.float32); tail[ids] = sub.tail
-    cp = np.zeros(wl.n_nodes, np.float32); cp[ids] = sub.cp
-    H = np.ones(wl.n_workflows, np.float32); H[workflows] = sub.H
-    return ho.DagResult(cp, tail, H), ids, workflows, cost
+def _sliced(fn, calls, n_out):
+    """fn(calls[lo:hi]) over slices of the batch on several host threads; fn returns a tuple of arrays
+    with one row per call, of which the first n_out are concatenated again."""
+    n = len(calls)
+    step = max(256, -(-n // (4 * N_THREADS)))
+    bounds = [(lo, min(n, lo + step)) for lo in range(0, n, step)]
+    with ThreadPoolExecutor(N_THREADS) as ex:
+        parts = list(ex.map(lambda b: fn(calls[b[0]:b[1]]), bounds))
+    return tuple(np.concatenate([p[k] for p in parts]) for k in range(n_out))
+
+
+def _oracle_forest(oracle, oc, wl):
+    """Stand-alone node costs and horizons of the whole forest from the oracle."""
+    if wl.node_cost is not None:
+        cost = wl.node_cost
+    else:
+        cost = _sliced(lambda c: oracle.schedule(oc, c, flags=ho.FLAG_UNLOADED | ho.FLAG_NO_DAG), wl.node_calls, 3)[2]
+    return cost, oracle.longest_path(wl.row_ptr, wl.col, cost, wl.node_wf, wl.n_workflows)
 
 
 def _gpu_setup(hx, wl):
@@ -41,26 +56,29 @@ def _gpu_setup(hx, wl):
     return gc, cost
 
 
-def test_large_full_sampled(hx, oracle):
+def _check_forest(gc, gcost, ocost, dag):
+    assert np.array_equal(gcost, ocost), "stand-alone node costs differ"
+    cp, tail, H = gc.dag_results()
+    assert np.array_equal(cp, dag.cp) and np.array_equal(tail, dag.tail) and np.array_equal(H, dag.H), "horizons differ"
+
+
+def test_large_full(hx, oracle):
     wl = make_workload("large")
     gc, gcost = _gpu_setup(hx, wl)
-    calls = wl.calls
-    gc.set_options(score_mode=hx.HX_MODE_SLACK, alpha=wl.alpha)
-    a, c = gc.schedule_batch(calls)
-    a, c = a.cpu().numpy(), c.cpu().numpy()
-    assert a.min() >= -1 and a.max() < wl.P * wl.D and gc.status() == 0
-    pick = np.random.default_rng(0).choice(len(calls), 400, replace=False)
     oc = hh.oracle_cluster(wl)
-    dag, ids, wfs, ocost = _oracle_dag_for(oracle, oc, wl, wl.node_wf[calls["node"][pick]])
-    assert np.array_equal(gcost[ids], ocost)
-    cp, tail, H = gc.dag_results()
-    assert np.array_equal(cp[ids], dag.cp[ids]) and np.array_equal(tail[ids], dag.tail[ids])
-    assert np.array_equal(H[wfs], dag.H[wfs])
-    oa, ocst, _ = oracle.schedule(oc, calls[pick], mode=ho.MODE_SLACK, alpha=wl.alpha, dag=dag,
-                                  node_wf=wl.node_wf, elapsed=wl.elapsed)
-    hh.assert_costs_close(c[pick], ocst, "large")
-    hh.assert_assign_matches(oracle, oc, calls[pick], a[pick], oa, what="large")
-    assert np.array_equal(c[pick], ocst) and np.array_equal(a[pick], oa)
+    ocost, dag = _oracle_forest(oracle, oc, wl)
+    _check_forest(gc, gcost, ocost, dag)
+    calls = wl.calls
+    kw = dict(dag=dag, node_wf=wl.node_wf, elapsed=wl.elapsed)
+    for mode_g, mode_o in ((hx.HX_MODE_SLACK, ho.MODE_SLACK), (hx.HX_MODE_RATIO, ho.MODE_RATIO)):
+        gc.set_options(score_mode=mode_g, alpha=wl.alpha)
+        a, c = gc.schedule_batch(calls)
+        a, c = a.cpu().numpy(), c.cpu().numpy()
+        oa, ocst, _ = _sliced(lambda s: oracle.schedule(oc, s, mode=mode_o, alpha=wl.alpha, **kw), calls, 3)
+        hh.assert_costs_close(c, ocst, "large")
+        hh.assert_assign_matches(oracle, oc, calls, a, oa, what="large")
+        assert np.array_equal(c, ocst) and np.array_equal(a, oa)
+    assert gc.status() == 0
     gc.close()
 
 
@@ -77,20 +95,26 @@ def test_cp_stress_full(hx, oracle):
     gc.set_options(score_mode=hx.HX_MODE_RATIO, alpha=wl.alpha)
     a, c = gc.schedule_batch(calls)
     a, c = a.cpu().numpy(), c.cpu().numpy()
-    pick = np.random.default_rng(1).choice(len(calls), 2000, replace=False)
     oc = hh.oracle_cluster(wl)
-    oa, ocst, _ = oracle.schedule(oc, calls[pick], mode=ho.MODE_RATIO, dag=r, node_wf=wl.node_wf, elapsed=wl.elapsed)
-    assert np.array_equal(c[pick], ocst) and np.array_equal(a[pick], oa)
+    oa, ocst, _ = _sliced(lambda s: oracle.schedule(oc, s, mode=ho.MODE_RATIO, dag=r, node_wf=wl.node_wf,
+                                                    elapsed=wl.elapsed), calls, 3)
+    assert np.array_equal(c, ocst) and np.array_equal(a, oa)
+    assert gc.status() == 0
     gc.close()
 
 
 def test_sweep_full_as_benchmarked(hx, oracle):
+    """All 16 scheduler invocations of the sweep, as the benchmark runs them: the free KV tokens are
+    restored ahead of every invocation, the prefill queues carry the commits of the one before."""
+    import torch
     wl = make_workload("sweep")
     P, D, chunk, K = wl.P, wl.D, wl.chunk, wl.topk
     gc, gcost = _gpu_setup(hx, wl)
     calls = wl.calls
     n_chunks = len(calls) // chunk
+    assert n_chunks == 16 and n_chunks * chunk == len(calls)
     free0 = wl.kv_free[P:].copy()
+    qP0 = wl.load_s[:P].copy()
     gc.set_options(score_mode=hx.HX_MODE_RATIO, topk=K, commit=1, alpha=wl.alpha)
     results = []
     for i in range(n_chunks):
@@ -100,25 +124,49 @@ def test_sweep_full_as_benchmarked(hx, oracle):
         qP, _, free = gc.read_loads()
         results.append((a.cpu().numpy(), c.cpu().numpy(), pair, cost, prio, qP, free))
     assert gc.status() == 0
-    m = calls["prompt_tokens"] + calls["output_tokens"]
-    for i, (a, c, pair, cost, prio, qP, free) in enumerate(results):
-        mi = m[i * chunk:(i + 1) * chunk]
-        placed = a >= 0
-        assert np.all(free >= 0) and np.all(free <= free0)                  # never over-committed
-        used = np.zeros(D); np.add.at(used, a[placed] % D, mi[placed])
-        assert np.array_equal((free0 - free).astype(np.float64), used)       # tokens are conserved
-        assert np.all((pair == a[:, None]).any(axis=1) | ~placed)            # a call only gets one of its candidates
-        assert np.all(np.diff(cost, axis=1)[np.isfinite(cost[:, 1:])] >= 0)  # lists ordered by finish time
-        if i:
-            assert np.all(qP >= results[i - 1][5])                           # prefill queues only grow
-    # the first scheduler invocation, completely, against the oracle
+
+    # the same 16 invocations through the host-buffer entry point (what the end-to-end figure times)
+    calls_pin = torch.from_numpy(calls.view(np.uint8).reshape(-1, 16).copy()).pin_memory()
+    a_pin = torch.full((len(calls),), -7, dtype=torch.int32).pin_memory()
+    c_pin = torch.full((len(calls),), -7.0, dtype=torch.float32).pin_memory()
+    free_pin = torch.from_numpy(free0.astype(np.float32)).pin_memory()
+    gc.update_loads(qP=qP0, kv_free=free0)
+    sp = torch.cuda.current_stream().cuda_stream
+    hx.hx_schedule_sweep_host(gc.h, calls_pin.numpy().view(hx.CALL_DTYPE).reshape(-1), chunk, free_pin.numpy(),
+                              a_pin.numpy(), c_pin.numpy(), sp)
+    torch.cuda.current_stream().synchronize()
+    assert np.array_equal(a_pin.numpy(), np.concatenate([r[0] for r in results]))
+    assert np.array_equal(c_pin.numpy(), np.concatenate([r[1] for r in results]))
+    sw_qP, _, sw_free = gc.read_loads()
+    assert np.array_equal(sw_qP, results[-1][5]) and np.array_equal(sw_free, results[-1][6])
+
+    # the oracle, invocation by invocation
     oc = hh.oracle_cluster(wl)
-    c0 = calls[:chunk]
-    dag, ids, wfs, ocost = _oracle_dag_for(oracle, oc, wl, wl.node_wf[c0["node"]])
-    assert np.array_equal(gcost[ids], ocost)
-    a, c, pair, cost, prio, qP, free = results[0]
-    op, ocs, opr, om, ots = oracle.topk(oc, c0, K, dag=dag, node_wf=wl.node_wf, elapsed=wl.elapsed)
-    assert np.array_equal(pair, op) and np.array_equal(cost, ocs) and np.array_equal(prio, opr)
-    oa, ofree, oq = oracle.conflict(op, opr, om, ots, free0, wl.load_s[:P], D)
-    assert np.array_equal(a, oa) and np.array_equal(free, ofree) and np.array_equal(qP, oq)
+    ocost, dag = _oracle_forest(oracle, oc, wl)
+    _check_forest(gc, gcost, ocost, dag)
+    kw = dict(dag=dag, node_wf=wl.node_wf, elapsed=wl.elapsed)
+    qP = qP0.copy()
+    m = calls["prompt_tokens"] + calls["output_tokens"]
+    placed_total = 0
+    for i, (a, c, pair, cost, prio, gq, gfree) in enumerate(results):
+        ci = calls[i * chunk:(i + 1) * chunk]
+        oc.qP[:] = qP
+        op, ocs, opr, om, ots = _sliced(lambda s: oracle.topk(oc, s, K, **kw), ci, 5)
+        what = "sweep invocation %d" % i
+        assert np.array_equal(pair, op), what
+        assert np.array_equal(cost, ocs) and np.array_equal(prio, opr), what
+        oa, ofree, oq = oracle.conflict(op, opr, om, ots, free0, qP, D)
+        assert np.array_equal(a, oa), what
+        assert np.array_equal(gfree, ofree) and np.array_equal(gq, oq), what
+        _, ocost_i, _ = _sliced(lambda s: oracle.schedule(oc, s, mode=ho.MODE_RATIO, **kw), ci, 3)
+        assert np.array_equal(c, ocost_i), what
+        # properties that hold at any size
+        placed = a >= 0
+        assert np.all(gfree >= 0) and np.all(gfree <= free0)
+        used = np.zeros(D); np.add.at(used, a[placed] % D, m[i * chunk:(i + 1) * chunk][placed])
+        assert np.array_equal((free0 - gfree).astype(np.float64), used)
+        assert np.all(gq >= qP)
+        placed_total += int(placed.sum())
+        qP = oq
+    assert 0 < placed_total < len(calls)
     gc.close()

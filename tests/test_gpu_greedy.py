@@ -39,7 +39,8 @@ def _compare(hx, gc, oc, oracle, calls, free0, P, D, dag=None, node_wf=None, ela
     return placed, a
 
 
-@pytest.mark.parametrize("name, scale", [("tiny", 1.0), ("medium", 1 / 8), ("medium", 1 / 2)])
+# the last case is the whole medium configuration: 4,096 calls (the largest queue the planner takes) x 16 x 16 pairs
+@pytest.mark.parametrize("name, scale", [("tiny", 1.0), ("medium", 1 / 8), ("medium", 1 / 2), ("medium", 1.0)])
 def test_greedy_on_generated_queues(hx, oracle, name, scale):
     wl = make_workload(name, scale=scale)
     oc, gc = hh.oracle_cluster(wl), hh.gpu_cluster(wl)

@@ -223,6 +223,41 @@ def test_empty_batch_not_ready_and_bad_ids(hx, oracle):
     good = np.arange(len(calls)) != 3
     oa, ocost, _ = oracle.schedule(hh.oracle_cluster(wl), wl.calls)
     assert np.array_equal(a[good], oa[good]) and np.array_equal(c[good], ocost[good])
+    assert gc.status() == 0                               # reading the status word clears it
+    a, _ = gc.schedule_batch(wl.calls)
+    assert gc.status() == 0                               # a clean batch after a bad one reports clean
+    gc.close()
+
+
+def test_fractional_token_counts_are_refused_by_the_capacity_pass(hx, oracle):
+    """The capacity pass takes its decisions on whole token counts.  A record with a fractional prompt or
+    output length is flagged (status word, no pair) when the pass is on, while the plain argmin, which
+    compares in binary32 like the oracle, scores it; free KV tokens that are not whole numbers are
+    refused by the host."""
+    gc, oc = _cluster_pair(hx, 5, 6, seed=11)
+    calls = _calls(200, seed=12)
+    calls["prompt_tokens"][17] += 0.5
+    calls["output_tokens"][90] += 0.25
+    gc.set_options(flags=hx.HX_FLAG_NO_DAG)
+    a, c = gc.schedule_batch(calls)
+    oa, ocost, _ = oracle.schedule(oc, calls)
+    assert np.array_equal(a.cpu().numpy(), oa) and np.array_equal(c.cpu().numpy(), ocost) and gc.status() == 0
+    gc.set_options(topk=3, commit=1, flags=hx.HX_FLAG_NO_DAG)
+    a, c = gc.schedule_batch(calls)
+    a, c = a.cpu().numpy(), c.cpu().numpy()
+    assert gc.status() == -1
+    assert a[17] == -1 and a[90] == -1 and np.isinf(c[17]) and np.isinf(c[90])
+    good = np.ones(200, bool); good[[17, 90]] = False
+    op, ocs, opr, om, ots = oracle.topk(oc, calls[good], 3)
+    oa, ofree, oq = oracle.conflict(op, opr, om, ots, np.full(6, 1e6, np.float32), oc.qP, 6)
+    assert np.array_equal(a[good], oa)
+    gq, _, gfree = gc.read_loads()
+    assert np.array_equal(gfree, ofree) and np.array_equal(gq, oq)
+    with pytest.raises(hx.HxError) as e:
+        gc.update_loads(kv_free=np.full(6, 1000.5, np.float32))
+    assert e.value.code == -1
+    with pytest.raises(hx.HxError):
+        gc.update_loads(kv_free=np.full(6, 2.0 ** 24, np.float32))
     gc.close()
 
 

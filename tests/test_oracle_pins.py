@@ -359,6 +359,44 @@ def test_conflict_pass_vs_plain_python(oracle):
             assert a[first] == pair[first, 0]                 # the most urgent call gets its best pair
 
 
+def test_conflict_pass_hand_worked_case(oracle):
+    """Eight calls, K = 3, worked by hand (tests/golden/make_conflict_case.py): an exact priority tie that
+    decides who gets the last room, a first candidate that is full, a call that takes its third candidate,
+    calls left unplaced, an equality fit, and prefill-queue sums whose binary32 value depends on the
+    order of the additions."""
+    with open(os.path.join(GOLD, "conflict_hand.json")) as f:
+        g = json.load(f)
+    prio = np.array([np.inf if x == "inf" else x for x in g["prio"]], np.float32)
+    pair = np.array(g["pair"], np.int32)
+    tpre = np.array(g["tpre"], np.float32)
+    assert np.array_equal(tpre.astype(np.float64), np.array(g["tpre"]))      # inputs are binary32 values
+    a, free, qP = oracle.conflict(pair, prio, np.array(g["m"], np.float32), tpre, g["free"], g["qP"], g["D"])
+    e = g["expect"]
+    assert a.tolist() == e["assign"]
+    assert free.tolist() == e["free"]
+    assert [float(x).hex() for x in qP] == e["qP_hex"]
+    # the hand-derived visiting order really is the one the rule states
+    order = sorted(range(len(prio)), key=lambda c: (-float(prio[c]), c))
+    assert order == e["order"]
+
+
+def test_conflict_pass_equal_calls_are_visited_by_index(oracle):
+    """300 identical calls of 1,000 tokens, four decode instances with room for 20 + 5 + 7 + 3 of them,
+    every call listing all four instances: all priorities are equal, so the calls are visited by index
+    and exactly the first 35 obtain a pair."""
+    rng = np.random.default_rng(3)
+    cl = _random_cluster(rng, 4, 4)
+    calls = np.zeros(300, CALL_DTYPE)
+    calls["prompt_tokens"] = 900; calls["output_tokens"] = 100
+    pair, cost, prio, m, tsel = oracle.topk(cl, calls, 4)
+    assert np.all(prio == prio[0]) and np.all(m == 1000) and np.all(pair >= 0)
+    free = np.array([20000, 5000, 7000, 3000], np.float32)
+    a, f2, _ = oracle.conflict(pair, prio, m, tsel, free, cl.qP, 4)
+    assert (a[:35] >= 0).all() and (a[35:] == -1).all()
+    assert f2.tolist() == [0, 0, 0, 0]
+    assert np.bincount(a[:35] % 4, minlength=4).tolist() == [20, 5, 7, 3]
+
+
 def test_conflict_pass_without_contention_is_the_argmin(oracle):
     rng = np.random.default_rng(13)
     cl = _random_cluster(rng, 4, 4)

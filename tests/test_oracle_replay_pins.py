@@ -1,6 +1,6 @@
 """Pins of the oracle's event-driven replay (oracle/hx_replay.py).  The paper gives no worked example of its
 simulator; these pin the replay to what its definition and the paper's metric fix: a workflow alone on the
-cluster reproduces its stand-alone horizon (that is how Section 7.2 defines H_w), a two-call hand case with a
+cluster reproduces its stand-alone horizon (that is how Section 7.3 defines H_w), a two-call hand case with a
 closed form built from the pinned service times, causality and capacity invariants, and Req95 / Req99 on a
 known list."""
 import numpy as np
