@@ -13,7 +13,7 @@
 //     Calls are binned by the leading bits of the priority key (bins linear in
 //     the key bits between the batch minimum and maximum); inside a bin every
 //     key counts the keys that precede it.  Keys (prio, call) are unique.
-//  2. hx_conflict_kernel - optimistic windows over the visiting order.  A block
+//  2. hx_conflict_kernel - optimistic windows over the visiting order.  A warp
 //     takes the next W calls; every call picks the first candidate that fits the
 //     capacities committed so far, then checks it against the demand of the
 //     earlier calls of the same window that picked the same instance (ordered,
@@ -28,6 +28,9 @@
 //  4. hx_qsum_kernel - one thread per prefill instance adds its prefill times in
 //     visiting order (binary32 addition is not associative, so the order is
 //     part of the definition).
+//
+#include <type_traits>
+
 #include "hx_internal.h"
 
 namespace {
@@ -35,8 +38,6 @@ namespace {
 typedef unsigned long long u64;
 
 constexpr int kBins = 2048;
-constexpr int kWin = 256;          // calls per optimistic window (= block size of the pass)
-constexpr int kCache = 4096;       // calls staged in shared memory ahead of the window
 constexpr unsigned kNone = 0xFFu;  // no candidate taken
 constexpr int kTailLen = 8192;     // obtained pairs handled per round of the fused tail
 constexpr int kTailMaxP = 512;     // largest prefill pool the fused tail handles
@@ -145,184 +146,47 @@ __global__ void hx_order_rank_kernel(HxTopkBufs tk, int n) {
     tk.od[rank] = tk.dsel[c];
 }
 
-// 2. The pass itself: one block of kWin threads.  Capacities and demands are handled as
-// integers (token counts are integer-valued and below 2^24).  Calls none of whose candidates
-// fits the capacities committed so far can never obtain a pair (capacity only shrinks): they
-// are dropped, in parallel, while the next stretch of the visiting order is staged, so the
-// windows only hold calls that may still be placed.
-template <int KT>   // candidate slots examined per call: K rounded up to 1, 2, 4 or 8
-__global__ void __launch_bounds__(kWin) hx_conflict_kernel(HxTopkBufs tk, HxTables t, int n, int commit,
-                                                           int fused_tail, int32_t* out_assign) {
-    extern __shared__ __align__(16) unsigned sm[];
-    constexpr int NW = kWin / 32;
-    constexpr int kScan = 4 * kWin;                             // ranks examined per staging step
-    const int D = t.D;
-    uint4* cd = reinterpret_cast<uint4*>(sm);                   // [kCache] ring: candidate instances of the live calls
-    int* cm = reinterpret_cast<int*>(cd + kCache);              // [kCache] their demands
-    int* cr = cm + kCache;                                      // [kCache] their ranks
-    int* free_s = cr + kCache;                                  // [D] capacity left after the commits so far
-    int* dtot = free_s + D;                                     // [D] demand of the window per instance
-    int* wtot = dtot + D;                                       // [NW][D] same per warp (only when an instance overflows)
-    __shared__ int first_fail, wsum[NW + 1];
+// Publishes the obtained pairs and adds the prefill times to the prefill queues in visiting order (NT
+// threads).  The list of obtained pairs holds call | k << 24.  It is taken in rounds of kTailLen entries; a
+// round is split by prefill instance with a stable counting sort (per-warp groups by match, per-warp
+// counts, offsets), then one thread per instance adds its run one after the other (binary32 addition is
+// not associative: the order is part of the definition).  pbuf [kTailLen] u16, tbuf and sorted [kTailLen]
+// f32, tail_i [(4 + NT / 32) * P] ints.
+template <int NT>
+__device__ __forceinline__ void publish_and_sum(const HxTopkBufs& tk, const HxTables& t, unsigned n_acc, int commit,
+                                                int32_t* out_assign, unsigned short* pbuf, float* tbuf,
+                                                float* sorted, int* tail_i) {
+    constexpr int NW = NT / 32;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    for (int d = tid; d < D; d += kWin) { free_s[d] = __float2int_rd(t.freeD[d]); dtot[d] = 0; }
-    if (tid == 0) first_fail = kWin;
-    __syncthreads();
-    auto first_fit = [&](const uint4& row, int m, unsigned& kt, int& dt) {
-        const unsigned w[4] = {row.x, row.y, row.z, row.w};
-        int fr[KT]; unsigned dk[KT];
-#pragma unroll
-        for (int k = 0; k < KT; ++k) {
-            dk[k] = (w[k >> 1] >> ((k & 1) * 16)) & 0xFFFFu;   // slots beyond K hold 0xFFFF
-            fr[k] = free_s[min(dk[k], (unsigned)(D - 1))];
-        }
-        kt = kNone; dt = -1;
-#pragma unroll
-        for (int k = KT - 1; k >= 0; --k)
-            if (dk[k] != 0xFFFFu && fr[k] >= m) { kt = k; dt = (int)dk[k]; }
-    };
-    int scan = 0;                                               // next rank to examine
-    unsigned head = 0, tail = 0;                                // live calls staged: ring positions [head, tail)
-    unsigned n_acc = 0;                                         // the four values are the same in every thread
-    // the stretch [scan, scan + kScan) is always in flight one step ahead of its use
-    uint4 nrow[4]; float nm[4];
-    auto prefetch = [&](int from) {
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int r = from + 4 * tid + u;
-            nrow[u] = r < n ? __ldcg(tk.od + r) : make_uint4(~0u, ~0u, ~0u, ~0u);
-            nm[u] = r < n ? __ldcg(tk.om + r) : 0.f;
-        }
-    };
-    prefetch(0);
-    while (head != tail || scan < n) {
-        while ((int)(tail - head) < kWin && scan < n) {         // stage: keep the calls that may still fit
-            uint4 row[4]; int mm[4]; bool live[4]; unsigned cnt = 0;
-#pragma unroll
-            for (int u = 0; u < 4; ++u) { row[u] = nrow[u]; mm[u] = __float2int_ru(nm[u]); }
-            prefetch(scan + kScan);
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                unsigned kt; int dt;
-                first_fit(row[u], mm[u], kt, dt);
-                live[u] = scan + 4 * tid + u < n && dt >= 0;
-                cnt += live[u];
-            }
-            unsigned x = cnt;                                   // ordered compaction into the ring
-#pragma unroll
-            for (int off = 1; off < 32; off <<= 1) {
-                const unsigned y = __shfl_up_sync(0xffffffffu, x, off);
-                if (lane >= off) x += y;
-            }
-            if (lane == 31) wsum[warp] = (int)x;
-            __syncthreads();
-            unsigned before = 0, total = 0;
-#pragma unroll
-            for (int w = 0; w < NW; ++w) { const unsigned a = (unsigned)wsum[w]; total += a; before += w < warp ? a : 0u; }
-            unsigned o = tail + before + x - cnt;
-#pragma unroll
-            for (int u = 0; u < 4; ++u)
-                if (live[u]) { const unsigned i = o++ & (kCache - 1); cd[i] = row[u]; cm[i] = mm[u]; cr[i] = scan + 4 * tid + u; }
-            tail += total;
-            scan += kScan;
-            __syncthreads();
-        }
-        const unsigned nwin = min((unsigned)kWin, tail - head);
-        if (nwin == 0) break;
-        const bool active = (unsigned)tid < nwin;
-        const unsigned ci = (head + tid) & (kCache - 1);
-        const int m = active ? cm[ci] : 0;
-        unsigned kt = kNone; int dt = -1;
-        if (active) first_fit(cd[ci], m, kt, dt);               // first candidate that fits the committed capacities
-        if (dt >= 0) atomicAdd(&dtot[dt], m);                   // demand of the window per instance
-        __syncthreads();                                        // S1
-        const bool over = dt >= 0 && dtot[dt] > free_s[dt];
-        int f = kWin;
-        if (__syncthreads_or(over)) {                           // S2: some instance cannot take the whole window
-            // ordered demand ahead of every call that picked an overflowing instance: inside the warp by
-            // broadcasting every lane's (instance, demand), across warps through per-warp totals
-            for (int i = tid; i < NW * D; i += kWin) wtot[i] = 0;
-            const int key = over ? dt : -1 - lane;              // calls outside the question match nobody
-            int cum = 0; bool later_peer = false;
-#pragma unroll 8
-            for (int j = 0; j < 32; ++j) {
-                const int kj = __shfl_sync(0xffffffffu, key, j);
-                const int mj = __shfl_sync(0xffffffffu, m, j);
-                if (kj == key) { if (j < lane) cum += mj; else if (j > lane) later_peer = true; }
-            }
-            __syncthreads();
-            if (over && !later_peer) wtot[warp * D + dt] = cum + m;     // last of its instance in this warp
-            __syncthreads();
-            if (over) {
-#pragma unroll
-                for (int w = 0; w < NW; ++w) cum += w < warp ? wtot[w * D + dt] : 0;
-                if (cum + m > free_s[dt]) atomicMin(&first_fail, tid);
-            }
-            __syncthreads();
-            f = first_fail;                                     // calls before f decided as the sequential pass would
-            __syncthreads();
-            if (tid == 0) first_fail = kWin;
-        }
-        for (int d = tid; d < D; d += kWin) dtot[d] = 0;
-        const bool acc = active && tid < f && dt >= 0;
-        if (acc) atomicSub(&free_s[dt], m);
-        const unsigned accm = __ballot_sync(0xffffffffu, acc);
-        if (lane == 0) wsum[warp] = __popc(accm);
-        const unsigned tot = __syncthreads_count(acc);          // S3
-        if (accm) {
-            unsigned off = n_acc + __popc(accm & ((1u << lane) - 1u));
-#pragma unroll
-            for (int w = 0; w < NW; ++w) off += w < warp ? (unsigned)wsum[w] : 0u;
-            if (acc) tk.acc_rk[off] = (unsigned)cr[ci] | (kt << 24);   // obtained pairs, in visiting order
-        }
-        n_acc += tot;
-        head += (unsigned)f < nwin ? (unsigned)f : nwin;
-        __syncthreads();                                        // S4: capacities and totals settled for the next step
-    }
-    if (tid == 0) *tk.n_acc = n_acc;
-    if (commit) for (int d = tid; d < D; d += kWin) t.freeD[d] = __int2float_rn(free_s[d]);
-    if (!fused_tail) return;
-
-    // ---- tail (prefill pools of up to kTailMaxP instances): publish the obtained pairs and add the
-    // prefill times to the prefill queues in visiting order, without leaving the block.  The list of
-    // obtained pairs is taken in rounds of kTailLen entries; a round is split by prefill instance with
-    // a stable counting sort (per-warp groups by match, per-warp counts, offsets), then one thread per
-    // instance adds its run one after the other (binary32 addition is not associative: the order is
-    // part of the definition).
-    const int P = t.P;
-    __syncthreads();                                            // the ring is free, acc_rk is visible
-    unsigned short* pbuf = reinterpret_cast<unsigned short*>(sm);           // [kTailLen]
-    float* tbuf = reinterpret_cast<float*>(pbuf + kTailLen);                // [kTailLen]
-    float* sorted = tbuf + kTailLen;                                        // [kTailLen]
-    int* tail_i = wtot + NW * D;                                            // behind the pass's own arrays
+    const int P = t.P, D = t.D;
     float* qsum = reinterpret_cast<float*>(tail_i);                         // [P]
     int* hist = tail_i + P;                                                 // [P]
     int* off0 = hist + P;                                                   // [P] start of the run of p in `sorted`
     int* off = off0 + P;                                                    // [P] next free slot of the run
     int* wcnt = off + P;                                                    // [NW][P], zero between uses
-    for (int p = tid; p < P; p += kWin) qsum[p] = t.qP[p];
-    for (int i = tid; i < NW * P; i += kWin) wcnt[i] = 0;
+    for (int p = tid; p < P; p += NT) qsum[p] = t.qP[p];
+    for (int i = tid; i < NW * P; i += NT) wcnt[i] = 0;
     for (unsigned r0 = 0; r0 < n_acc; r0 += kTailLen) {
         const int len = (int)min((unsigned)kTailLen, n_acc - r0);
-        for (int p = tid; p < P; p += kWin) hist[p] = 0;
+        for (int p = tid; p < P; p += NT) hist[p] = 0;
         __syncthreads();
-        // three dependent gathers per entry (list -> call -> pair, prefill time): eight entries in flight per thread
-        for (int i0 = tid; i0 < len; i0 += 8 * kWin) {
+        // dependent gathers per entry (list -> [call ->] pair, prefill time): eight entries in flight per thread
+        for (int i0 = tid; i0 < len; i0 += 8 * NT) {
             unsigned rk[8], c[8]; int pr[8]; float tp[8];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) rk[u] = i0 + u * kWin < len ? __ldcg(tk.acc_rk + r0 + i0 + u * kWin) : 0u;
+            for (int u = 0; u < 8; ++u) rk[u] = i0 + u * NT < len ? __ldcg(tk.acc_rk + r0 + i0 + u * NT) : 0u;
 #pragma unroll
-            for (int u = 0; u < 8; ++u) c[u] = i0 + u * kWin < len ? __ldcg(tk.ocall + (rk[u] & 0xFFFFFFu)) : 0u;
+            for (int u = 0; u < 8; ++u) c[u] = rk[u] & 0xFFFFFFu;
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
                 const size_t o = (size_t)c[u] * tk.K + (rk[u] >> 24);
-                const bool ok = i0 + u * kWin < len;
+                const bool ok = i0 + u * NT < len;
                 pr[u] = ok ? __ldcg(tk.pair + o) : 0;
                 tp[u] = ok ? __ldcg(tk.tpre + o) : 0.f;
             }
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
-                const int i = i0 + u * kWin;
+                const int i = i0 + u * NT;
                 if (i < len) {
                     out_assign[c[u]] = pr[u];
                     const int p = pr[u] / D;
@@ -346,7 +210,7 @@ __global__ void __launch_bounds__(kWin) hx_conflict_kernel(HxTopkBufs tk, HxTabl
             }
         }
         __syncthreads();
-        for (int ch = 0; ch < len; ch += kWin) {
+        for (int ch = 0; ch < len; ch += NT) {
             const int i = ch + tid;
             const bool valid = i < len;
             const int p = valid ? (int)pbuf[i] : -1 - lane;
@@ -357,7 +221,7 @@ __global__ void __launch_bounds__(kWin) hx_conflict_kernel(HxTopkBufs tk, HxTabl
             __syncthreads();
             int before = 0, total = 0;
             if (valid) {
-#pragma unroll
+#pragma unroll 8
                 for (int w = 0; w < NW; ++w) { const int cw = wcnt[w * P + p]; total += cw; before += w < warp ? cw : 0; }
                 sorted[off[p] + before + rank] = tbuf[i];
             }
@@ -368,7 +232,7 @@ __global__ void __launch_bounds__(kWin) hx_conflict_kernel(HxTopkBufs tk, HxTabl
             }
             __syncthreads();
         }
-        for (int p = tid; p < P; p += kWin) {
+        for (int p = tid; p < P; p += NT) {
             const int a = off0[p], b = a + hist[p];
             float q = qsum[p];
 #pragma unroll 8
@@ -377,15 +241,174 @@ __global__ void __launch_bounds__(kWin) hx_conflict_kernel(HxTopkBufs tk, HxTabl
         }
         __syncthreads();
     }
-    if (commit) for (int p = tid; p < P; p += kWin) t.qP[p] = qsum[p];
+    if (commit) for (int p = tid; p < P; p += NT) t.qP[p] = qsum[p];
+}
+
+// 2. The pass itself: one block of kPassThreads threads.  Capacities and demands are handled as
+// integers (token counts are whole numbers below 2^24).  The visiting order is staged kPassThreads
+// ranks at a time by the whole block: calls none of whose candidates fits the capacities committed
+// so far can never obtain a pair (capacity only shrinks) and are dropped, in parallel, so that only
+// calls that may still be placed reach the sequential part.  That part is run by ONE warp, in
+// optimistic windows of 32 staged calls, with warp shuffles and votes only: a window step costs a
+// few hundred cycles, where a step of a block-wide window costs a chain of block barriers.
+constexpr int kPassThreads = 1024;
+constexpr int kRing = 2048;        // staged calls waiting for the window warp (at most kDrain + kPassThreads)
+constexpr int kDrain = 96;         // the windows run once this many calls are staged (or the order is exhausted)
+template <int KT>   // candidate slots examined per call: K rounded up to 1, 2, 4 or 8
+__global__ void __launch_bounds__(kPassThreads, 1) hx_conflict_kernel(HxTopkBufs tk, HxTables t, int n, int commit,
+                                                                      int fused_tail, int32_t* out_assign) {
+    extern __shared__ __align__(16) unsigned sm[];
+    constexpr int NW = kPassThreads / 32;
+    static_assert(NW == 32, "the staging step keeps one warp total per lane");
+    const int D = t.D;
+    // candidate instances of a staged call, 16 bits each; an unused slot points at instance D, which never has room
+    using Row = typename std::conditional<(KT > 4), uint4, uint2>::type;
+    Row* cd = reinterpret_cast<Row*>(sm);                       // [kRing] candidate instances of the staged calls
+    int* cm = reinterpret_cast<int*>(cd + kRing);               // [kRing] their demands
+    int* cr = cm + kRing;                                       // [kRing] their call numbers
+    int* free_s = cr + kRing;                                   // [D + 1] capacity left after the commits so far
+    __shared__ int wsum[NW];
+    __shared__ unsigned n_acc_s;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const unsigned lt = (1u << lane) - 1u;
+    for (int d = tid; d <= D; d += kPassThreads) free_s[d] = d < D ? __float2int_rd(t.freeD[d]) : -1;
+    __syncthreads();
+    auto remap = [&](const uint4& r) {                          // 0xFFFF (no candidate) -> D
+        const unsigned w[4] = {r.x, r.y, r.z, r.w};
+        unsigned o[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) o[q] = min(w[q] & 0xFFFFu, (unsigned)D) | (min(w[q] >> 16, (unsigned)D) << 16);
+        Row out;
+        out.x = o[0]; out.y = o[1];
+        if constexpr (KT > 4) { out.z = o[2]; out.w = o[3]; }
+        return out;
+    };
+    auto first_fit = [&](const Row& row, int m, unsigned& kt, int& dt, int& fr_t) {
+        unsigned w[4] = {row.x, row.y, 0u, 0u};
+        if constexpr (KT > 4) { w[2] = row.z; w[3] = row.w; }
+        int fr[KT]; unsigned dk[KT];
+#pragma unroll
+        for (int k = 0; k < KT; ++k) {
+            dk[k] = (k & 1) ? w[k >> 1] >> 16 : w[k >> 1] & 0xFFFFu;
+            fr[k] = free_s[dk[k]];
+        }
+        kt = kNone; dt = -1; fr_t = 0;
+#pragma unroll
+        for (int k = KT - 1; k >= 0; --k)
+            if (fr[k] >= m) { kt = k; dt = (int)dk[k]; fr_t = fr[k]; }
+    };
+    // rank scan + tid is in flight one staging step ahead of its use
+    uint4 nrow; float nm; unsigned ncall;
+    auto prefetch = [&](int from) {
+        const int r = from + tid;
+        nrow = r < n ? __ldcg(tk.od + r) : make_uint4(~0u, ~0u, ~0u, ~0u);
+        nm = r < n ? __ldcg(tk.om + r) : 0.f;
+        ncall = r < n ? __ldcg(tk.ocall + r) : 0u;
+    };
+    prefetch(0);
+    unsigned n_acc = 0;                                         // kept by warp 0 (the same in its 32 lanes)
+    unsigned count = 0;                                         // staged calls, the same in every thread
+    for (int scan = 0; scan < n; scan += kPassThreads) {
+        const Row row = remap(nrow);
+        const int mm = __float2int_ru(nm);
+        const unsigned call = ncall;
+        prefetch(scan + kPassThreads);
+        unsigned kt0; int dt0, fr0;
+        first_fit(row, mm, kt0, dt0, fr0);
+        const bool live = scan + tid < n && dt0 >= 0;
+        const unsigned lm = __ballot_sync(0xffffffffu, live);   // ordered compaction behind the staged calls
+        if (lane == 0) wsum[warp] = __popc(lm);
+        __syncthreads();
+        unsigned wx = (unsigned)wsum[lane];
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const unsigned y = __shfl_up_sync(0xffffffffu, wx, off);
+            if (lane >= off) wx += y;
+        }
+        const unsigned total = __shfl_sync(0xffffffffu, wx, 31);
+        const unsigned before = __shfl_sync(0xffffffffu, wx, warp) - (unsigned)__popc(lm);
+        if (live) {
+            const unsigned o = count + before + __popc(lm & lt);
+            cd[o] = row; cm[o] = mm; cr[o] = (int)call;
+        }
+        count += total;
+        const bool drain = count >= (unsigned)kDrain || scan + kPassThreads >= n;
+        __syncthreads();
+        if (!drain) continue;
+        // One warp walks the staged calls in windows of 32: every lane picks the first candidate that fits the
+        // committed capacities.  A lane whose pick no longer fits after the lower lanes that picked the same
+        // instance has failed; every lane before the lowest failing lane has taken the decision of the
+        // sequential pass and commits; the window restarts at the failing lane, which then sees the reduced
+        // capacity.  Lane 0 always fits its pick, so every step advances.
+        if (warp == 0) {
+            unsigned pos = 0;
+            while (pos < count) {
+                const unsigned i = pos + lane;
+                int m = 0, dt = -1, fr = 0; unsigned kt = kNone;
+                if (i < count) { m = cm[i]; first_fit(cd[i], m, kt, dt, fr); }
+                const unsigned picked = __ballot_sync(0xffffffffu, dt >= 0);
+                if (picked == 0u) { pos += 32; continue; }      // nothing here fits any more
+                // A pick can only fail if its instance has less room than the whole window asks for (S): all other
+                // picks are safe whatever the lower lanes took.  Instances short of S are resolved one by one: total
+                // demand of the lanes that picked it and, if that overflows, an ordered prefix sum to find the
+                // first lane that no longer fits.
+                const int S = __reduce_add_sync(0xffffffffu, dt >= 0 ? m : 0);
+                unsigned f = 32, gm = 0; int v = 0;
+                for (unsigned rem = __ballot_sync(0xffffffffu, dt >= 0 && fr < S); rem;) {
+                    const int leader = __ffs(rem) - 1;
+                    const int d0 = __shfl_sync(0xffffffffu, dt, leader);
+                    const int room = __shfl_sync(0xffffffffu, fr, leader);
+                    const bool mine = dt == d0;
+                    const unsigned g = __ballot_sync(0xffffffffu, mine);
+                    if (__reduce_add_sync(0xffffffffu, mine ? m : 0) > room) {
+                        int x = mine ? m : 0;
+#pragma unroll
+                        for (int off = 1; off < 32; off <<= 1) {
+                            const int y = __shfl_up_sync(0xffffffffu, x, off);
+                            if (lane >= off) x += y;
+                        }
+                        if (mine) { v = x; gm = g; }
+                        const unsigned fail = __ballot_sync(0xffffffffu, mine && x > room);
+                        f = min(f, (unsigned)(__ffs(fail) - 1));     // lane 0 never fails
+                    }
+                    rem &= ~g;
+                }
+                const bool acc = dt >= 0 && (unsigned)lane < f;
+                const unsigned accm = __ballot_sync(0xffffffffu, acc);
+                if (acc) {
+                    if (gm == 0u) atomicSub(&free_s[dt], m);                              // the whole group fits
+                    else if (((gm & accm) >> lane) == 1u) free_s[dt] = fr - v;            // last committing lane of an overflowing group
+                }
+                if (acc) tk.acc_rk[n_acc + __popc(accm & lt)] = (unsigned)cr[i] | (kt << 24);   // obtained pairs, in visiting order
+                n_acc += __popc(accm);
+                pos += f;
+                __syncwarp();
+            }
+        }
+        count = 0;
+        __syncthreads();
+    }
+    if (tid == 0) { *tk.n_acc = n_acc; n_acc_s = n_acc; }
+    __syncthreads();
+    n_acc = n_acc_s;
+    if (commit) for (int d = tid; d < D; d += kPassThreads) t.freeD[d] = __int2float_rn(free_s[d]);
+    if (!fused_tail) return;
+
+    // ---- tail (prefill pools of up to kTailMaxP instances): publish the obtained pairs and add the
+    // prefill times to the prefill queues in visiting order, without leaving the block (acc_rk was
+    // written by this block: visible after the barrier above).
+    unsigned short* pbuf = reinterpret_cast<unsigned short*>(sm);           // [kTailLen]
+    float* tbuf = reinterpret_cast<float*>(pbuf + kTailLen);                // [kTailLen]
+    float* sorted = tbuf + kTailLen;                                        // [kTailLen]
+    publish_and_sum<kPassThreads>(tk, t, n_acc, commit, out_assign, pbuf, tbuf, sorted,
+                                         reinterpret_cast<int*>(sorted + kTailLen));
 }
 
 // 3. Publish the obtained pairs; gather prefill instance and prefill time in visiting order.
 __global__ void hx_finish_kernel(HxTopkBufs tk, int D, int32_t* out_assign) {
     const unsigned i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= *tk.n_acc) return;
-    const unsigned rk = tk.acc_rk[i], r = rk & 0xFFFFFFu, k = rk >> 24;
-    const unsigned c = tk.ocall[r];
+    const unsigned rk = tk.acc_rk[i], c = rk & 0xFFFFFFu, k = rk >> 24;
     const int pr = tk.pair[(size_t)c * tk.K + k];
     out_assign[c] = pr;
     tk.acc_p[i] = pr / D;
@@ -427,6 +450,7 @@ __global__ void __launch_bounds__(32 * kQWarps) hx_qsum_kernel(HxTopkBufs tk, Hx
     if (lane == 0 && p < t.P) t.qP[p] = q;
 }
 
+
 }  // namespace
 
 cudaError_t hx_launch_conflict(const HxTables& t, const HxTopkBufs& tk, int n_calls, int commit,
@@ -442,14 +466,15 @@ cudaError_t hx_launch_conflict(const HxTables& t, const HxTopkBufs& tk, int n_ca
     hx_order_bins_kernel<<<1, 1024, smB, stream>>>(tk, n_calls, staged);
     hx_order_rank_kernel<<<(n_calls + 127) / 128, 128, 0, stream>>>(tk, n_calls);
     const int fused = P <= kTailMaxP;                               // pairs published and queues summed inside the pass
-    const size_t smC = (size_t)kCache * 24 + (size_t)(2 * D + (kWin / 32) * D) * 4 +
-                       (fused ? (size_t)(4 * P + (kWin / 32) * P) * 4 : 0);
+    const size_t smRing = (size_t)kRing * 24 + (size_t)(D + 1) * 4;
+    const size_t smTail = fused ? (size_t)kTailLen * 10 + (size_t)(4 + kPassThreads / 32) * P * 4 : 0;
+    const size_t smC = smRing > smTail ? smRing : smTail;
     auto pass = tk.K <= 1 ? hx_conflict_kernel<1> : tk.K <= 2 ? hx_conflict_kernel<2>
               : tk.K <= 4 ? hx_conflict_kernel<4> : hx_conflict_kernel<8>;
     static size_t allowed_pass[4][64];
     e = hx_opt_in_smem(pass, smC, allowed_pass[tk.K <= 1 ? 0 : tk.K <= 2 ? 1 : tk.K <= 4 ? 2 : 3], 40 * 1024);
     if (e != cudaSuccess) return e;
-    pass<<<1, kWin, smC, stream>>>(tk, t, n_calls, commit, fused, out_assign);
+    pass<<<1, kPassThreads, smC, stream>>>(tk, t, n_calls, commit, fused, out_assign);
     *launches += 3;
     if (!fused) {
         hx_finish_kernel<<<(n_calls + 255) / 256, 256, 0, stream>>>(tk, D, out_assign);

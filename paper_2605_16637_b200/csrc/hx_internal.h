@@ -79,7 +79,7 @@ struct HxTopkBufs {
     uint4* od;                 // [cap] same rows in visiting order
     // outcome: calls that obtained a pair, in visiting order
     unsigned int* n_acc;       // [1]
-    unsigned int* acc_rk;      // [cap] rank | k << 24
+    unsigned int* acc_rk;      // [cap] call | k << 24
     int* acc_p;                // [cap] prefill instance obtained
     float* acc_t;              // [cap] prefill time added to that instance
 };

@@ -369,6 +369,42 @@ def test_equal_priorities_visit_lower_call_first(hx, oracle):
     gc.close()
 
 
+@pytest.mark.parametrize("n, K, P, D", [(20000, 4, 8, 12), (16384, 4, 8, 12), (16385, 2, 5, 40), (5000, 8, 300, 9),
+                                       (33, 3, 2, 5), (1, 1, 1, 1)])
+def test_capacity_pass_batch_sizes_and_pool_shapes(hx, oracle, n, K, P, D):
+    """Batches on both sides of the size up to which the pass runs as one block-resident kernel, a prefill
+    pool too wide for the fused queue sums, and the smallest shapes; a tenth of the calls fits no decode
+    instance at all (priority +inf: visited first, placed nowhere) and a fifth are exact duplicates of one
+    another (equal priorities: visited by call number)."""
+    gc, oc = _cluster_pair(hx, P, D, seed=n + K, tight=True)
+    calls = _calls(n, seed=n)
+    rng = np.random.default_rng(n)
+    dup = rng.random(n) < 0.2
+    calls["model"][dup] = 0; calls["prompt_tokens"][dup] = 777; calls["output_tokens"][dup] = 33
+    calls["prompt_tokens"][rng.random(n) < 0.1] = 2.0e6
+    m = calls["prompt_tokens"] + calls["output_tokens"]
+    free = np.floor(rng.uniform(0.05, 0.6, D) * np.minimum(m, 40000).sum() / D).astype(np.float32)
+    free = np.minimum(free, 2.0 ** 24 - 1).astype(np.float32)
+    qP = oc.qP.copy()
+    gc.set_options(score_mode=hx.HX_MODE_RATIO, topk=K, commit=1, flags=hx.HX_FLAG_NO_DAG)
+    for rep in range(2):                                  # the second batch sees the committed queues
+        gc.update_loads(kv_free=free)
+        a, _ = gc.schedule_batch(calls)
+        oc.qP[:] = qP
+        op, ocs, opr, om, ots = oracle.topk(oc, calls, K)
+        pair, cost, prio = gc.topk_results(n)
+        assert np.array_equal(pair, op) and np.array_equal(cost, ocs) and np.array_equal(prio, opr)
+        oa, ofree, oq = oracle.conflict(op, opr, om, ots, free, qP, D)
+        gq, _, gfree = gc.read_loads()
+        assert np.array_equal(a.cpu().numpy(), oa), "placements differ"
+        assert np.array_equal(gfree, ofree) and np.array_equal(gq, oq), "committed loads differ"
+        qP = oq
+    if n > 100:
+        assert np.isinf(opr).any() and (oa >= 0).any() and (oa < 0).any()
+    assert gc.status() == 0
+    gc.close()
+
+
 def test_host_buffer_entry_point_matches_device_path(hx, oracle):
     wl = make_workload("medium")
     oc, gc, dag = _prepare(hx, oracle, wl)
