@@ -9,10 +9,13 @@
 // instance and adds the call's prefill time to the chosen prefill queue.
 //
 // Parallel form with identical results:
-//  1. hx_order_bins_kernel / hx_order_rank_kernel - visiting order of the batch.
-//     Calls are binned by the leading bits of the priority key (bins linear in
-//     the key bits between the batch minimum and maximum); inside a bin every
-//     key counts the keys that precede it.  Keys (prio, call) are unique.
+//  1. hx_order_hist_kernel / hx_order_scatter_kernel / hx_order_rank_kernel -
+//     visiting order of the batch, three short grids.  Calls are binned by the
+//     leading bits of the priority key (bins linear in the key bits between the
+//     batch minimum and maximum, which the scoring kernel left behind per block;
+//     priorities of +inf have a bin of their own, so that calls that fit nowhere
+//     do not stretch the range); inside a bin every key counts the keys that
+//     precede it.  Keys (prio, call) are unique.
 //  2. hx_conflict_kernel - optimistic windows over the visiting order.  A warp
 //     takes the next W calls; every call picks the first candidate that fits the
 //     capacities committed so far, then checks it against the demand of the
@@ -37,7 +40,7 @@ namespace {
 
 typedef unsigned long long u64;
 
-constexpr int kBins = 2048;
+constexpr int kBins = HX_ORDER_BINS;
 constexpr unsigned kNone = 0xFFu;  // no candidate taken
 constexpr int kTailLen = 8192;     // obtained pairs handled per round of the fused tail
 constexpr int kTailMaxP = 512;     // largest prefill pool the fused tail handles
@@ -73,77 +76,72 @@ __device__ void block_exclusive_scan(const unsigned* cnt, int n, unsigned* base,
     __syncthreads();
 }
 
-// 1a. Bin the priority keys: one block.  obase receives the kBins + 1 bin bounds, the smallest
-// key and the shift that maps a key to its bin.  Each thread keeps its first kKeep keys in
-// registers (one round trip to memory); the rest of a large batch is read again per pass.
-constexpr int kKeep = 16;
-__global__ void __launch_bounds__(1024) hx_order_bins_kernel(HxTopkBufs tk, int n, int staged) {
-    extern __shared__ __align__(16) u64 skey[];                   // [n] keys in bin order when they fit (staged)
-    __shared__ unsigned hist[kBins], base[kBins + 1], tmp[33], lohi[2];
-    const int tid = threadIdx.x, nthr = blockDim.x;
-    for (int i = tid; i < kBins; i += nthr) hist[i] = 0;
+// 1a. Bin the priority keys (grid of 256-thread blocks, one call per thread).  The scoring kernel left the
+// key range of each of its blocks behind and cleared the bin counters; every block here reduces those ranges
+// to the range of the batch, and every call draws its arrival number inside its bin from the global counter.
+constexpr int kOrdThreads = 256;
+__device__ __forceinline__ unsigned bin_of(unsigned key, unsigned lo, unsigned shift) {
+    return key == HX_FIRST_KEY ? 0u : 1u + ((key - lo) >> shift);
+}
+__global__ void __launch_bounds__(kOrdThreads) hx_order_hist_kernel(HxTopkBufs tk, int n) {
+    __shared__ unsigned lohi[2];
+    const int tid = threadIdx.x;
     if (tid == 0) { lohi[0] = 0xFFFFFFFFu; lohi[1] = 0u; }
-    unsigned keep[kKeep];
-#pragma unroll
-    for (int u = 0; u < kKeep; ++u) {
-        const int c = tid + u * nthr;
-        keep[u] = c < n ? ~__float_as_uint(__ldg(tk.prio + c)) : 0u;      // larger priority = smaller key
-    }
-    auto key_of = [&](int u, int c) { return u < kKeep ? keep[u] : ~__float_as_uint(__ldg(tk.prio + c)); };
     __syncthreads();
     unsigned lo = 0xFFFFFFFFu, hi = 0u;
-#pragma unroll
-    for (int u = 0; u < kKeep; ++u) if (tid + u * nthr < n) { lo = min(lo, keep[u]); hi = max(hi, keep[u]); }
-    for (int c = tid + kKeep * nthr; c < n; c += nthr) { const unsigned k = key_of(kKeep, c); lo = min(lo, k); hi = max(hi, k); }
+    for (int b = tid; b < HX_ORDER_MAXBLK; b += kOrdThreads) {
+        lo = min(lo, __ldcg(tk.blk_lohi + b)); hi = max(hi, __ldcg(tk.blk_lohi + HX_ORDER_MAXBLK + b));
+    }
     lo = __reduce_min_sync(0xffffffffu, lo); hi = __reduce_max_sync(0xffffffffu, hi);
     if ((tid & 31) == 0) { atomicMin(&lohi[0], lo); atomicMax(&lohi[1], hi); }
     __syncthreads();
     lo = lohi[0];
-    const unsigned span = lohi[1] - lo;
-    int shift = 0;
-    while ((span >> shift) >= (unsigned)kBins) ++shift;
-    unsigned slot[kKeep];                                          // arrival number inside the bin
-#pragma unroll
-    for (int u = 0; u < kKeep; ++u) slot[u] = tid + u * nthr < n ? atomicAdd(&hist[(keep[u] - lo) >> shift], 1u) : 0u;
-    for (int c = tid + kKeep * nthr; c < n; c += nthr)
-        tk.ocall[c] = atomicAdd(&hist[(key_of(kKeep, c) - lo) >> shift], 1u);   // parked until the bounds are known
-    __syncthreads();
-    block_exclusive_scan(hist, kBins, base, tmp);
-    for (int i = tid; i <= kBins; i += nthr) tk.obase[i] = base[i];
-    if (tid == 0) { tk.obase[kBins + 1] = lo; tk.obase[kBins + 2] = (unsigned)shift; }
-#pragma unroll
-    for (int u = 0; u < kKeep; ++u) {
-        const int c = tid + u * nthr;
-        if (c < n) {
-            const unsigned pos = base[(keep[u] - lo) >> shift] + slot[u];
-            const u64 v = ((u64)keep[u] << 32) | (unsigned)c;
-            if (staged) skey[pos] = v; else tk.okey[pos] = v;
-        }
-    }
-    for (int c = tid + kKeep * nthr; c < n; c += nthr) {
-        const unsigned key = key_of(kKeep, c);
-        tk.okey[base[(key - lo) >> shift] + tk.ocall[c]] = ((u64)key << 32) | (unsigned)c;
-    }
-    if (staged) {                                                  // scattered in shared memory, coalesced to global
-        __syncthreads();
-        for (int i = tid; i < n; i += nthr) tk.okey[i] = skey[i];
-    }
+    const unsigned span = lohi[1] >= lo ? lohi[1] - lo : 0u;      // no finite key at all: nothing lands in bins 1 ..
+    unsigned shift = 0;
+    while ((span >> shift) >= (unsigned)(kBins - 1)) ++shift;
+    if (blockIdx.x == 0 && tid == 0) { tk.obase[kBins + 1] = lo; tk.obase[kBins + 2] = shift; }
+    const int c = blockIdx.x * kOrdThreads + tid;
+    if (c >= n) return;
+    const unsigned bin = bin_of(hx_order_key(__float_as_uint(__ldcg(tk.prio + c))), lo, shift);
+    tk.oslot[c] = (bin << 16) | atomicAdd(tk.ghist + bin, 1u);
 }
 
-// 1b. Rank inside the bins and gather the per-call data in visiting order.
-__global__ void hx_order_rank_kernel(HxTopkBufs tk, int n) {
+// 1b. Every block turns the bin counters into bin bounds (the same 2,048-entry scan in every block is cheaper
+// than one more launch) and moves its calls' keys to their place in bin order.
+__global__ void __launch_bounds__(kOrdThreads) hx_order_scatter_kernel(HxTopkBufs tk, int n) {
+    __shared__ unsigned hist[kBins], base[kBins + 1], tmp[33];
+    const int tid = threadIdx.x;
+    for (int i = tid; i < kBins; i += kOrdThreads) hist[i] = __ldcg(tk.ghist + i);
+    __syncthreads();
+    block_exclusive_scan(hist, kBins, base, tmp);
+    if (blockIdx.x == 0) for (int i = tid; i <= kBins; i += kOrdThreads) tk.obase[i] = base[i];
+    const int c = blockIdx.x * kOrdThreads + tid;
+    if (c >= n) return;
+    const unsigned bs = __ldcg(tk.oslot + c);
+    const unsigned key = hx_order_key(__float_as_uint(__ldcg(tk.prio + c)));
+    tk.okey[base[bs >> 16] + (bs & 0xFFFFu)] = ((u64)key << 32) | (unsigned)c;
+}
+
+// 1c. Rank inside the bins and gather the per-call data in visiting order.
+__global__ void hx_order_rank_kernel(HxTopkBufs tk, int n, unsigned D) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
     const unsigned lo = tk.obase[kBins + 1], shift = tk.obase[kBins + 2];
     const u64 key = tk.okey[i];
-    const unsigned bin = ((unsigned)(key >> 32) - lo) >> shift;
+    const unsigned bin = bin_of((unsigned)(key >> 32), lo, shift);
     const unsigned b0 = tk.obase[bin], b1 = tk.obase[bin + 1];
     unsigned rank = b0;
     for (unsigned j = b0; j < b1; ++j) rank += __ldg(tk.okey + j) < key;
     const unsigned c = (unsigned)key;
     tk.ocall[rank] = c;
-    tk.om[rank] = tk.mtok[c];
-    tk.od[rank] = tk.dsel[c];
+    tk.om[rank] = __float2int_ru(tk.mtok[c]);                   // token counts are whole numbers below 2^24
+    // candidate instances, 16 bits each; an unused slot (0xFFFF) points at instance D, which never has room
+    const uint4 r = tk.dsel[c];
+    const unsigned w[4] = {r.x, r.y, r.z, r.w};
+    unsigned o[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) o[q] = min(w[q] & 0xFFFFu, D) | (min(w[q] >> 16, D) << 16);
+    tk.od[rank] = make_uint4(o[0], o[1], o[2], o[3]);
 }
 
 // Publishes the obtained pairs and adds the prefill times to the prefill queues in visiting order (NT
@@ -273,15 +271,19 @@ __global__ void __launch_bounds__(kPassThreads, 1) hx_conflict_kernel(HxTopkBufs
     const unsigned lt = (1u << lane) - 1u;
     for (int d = tid; d <= D; d += kPassThreads) free_s[d] = d < D ? __float2int_rd(t.freeD[d]) : -1;
     __syncthreads();
-    auto remap = [&](const uint4& r) {                          // 0xFFFF (no candidate) -> D
-        const unsigned w[4] = {r.x, r.y, r.z, r.w};
-        unsigned o[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) o[q] = min(w[q] & 0xFFFFu, (unsigned)D) | (min(w[q] >> 16, (unsigned)D) << 16);
+    auto narrow = [&](const uint4& r) {                         // the slots this instantiation examines
         Row out;
-        out.x = o[0]; out.y = o[1];
-        if constexpr (KT > 4) { out.z = o[2]; out.w = o[3]; }
+        out.x = r.x; out.y = r.y;
+        if constexpr (KT > 4) { out.z = r.z; out.w = r.w; }
         return out;
+    };
+    auto any_fit = [&](const Row& row, int m) {                  // does any candidate still have room?
+        unsigned w[4] = {row.x, row.y, 0u, 0u};
+        if constexpr (KT > 4) { w[2] = row.z; w[3] = row.w; }
+        int best = -1;
+#pragma unroll
+        for (int k = 0; k < KT; ++k) best = max(best, free_s[(k & 1) ? w[k >> 1] >> 16 : w[k >> 1] & 0xFFFFu]);
+        return best >= m;
     };
     auto first_fit = [&](const Row& row, int m, unsigned& kt, int& dt, int& fr_t) {
         unsigned w[4] = {row.x, row.y, 0u, 0u};
@@ -297,25 +299,26 @@ __global__ void __launch_bounds__(kPassThreads, 1) hx_conflict_kernel(HxTopkBufs
         for (int k = KT - 1; k >= 0; --k)
             if (fr[k] >= m) { kt = k; dt = (int)dk[k]; fr_t = fr[k]; }
     };
-    // rank scan + tid is in flight one staging step ahead of its use
-    uint4 nrow; float nm; unsigned ncall;
-    auto prefetch = [&](int from) {
+    // rank scan + tid is in flight two staging steps ahead of its use (a staging step without windows
+    // in between is shorter than a round trip to the L2)
+    uint4 nrow, nrow2; int nm, nm2; unsigned ncall, ncall2;
+    auto fetch = [&](int from, uint4& row, int& m, unsigned& call) {
         const int r = from + tid;
-        nrow = r < n ? __ldcg(tk.od + r) : make_uint4(~0u, ~0u, ~0u, ~0u);
-        nm = r < n ? __ldcg(tk.om + r) : 0.f;
-        ncall = r < n ? __ldcg(tk.ocall + r) : 0u;
+        row = r < n ? __ldcg(tk.od + r) : make_uint4(~0u, ~0u, ~0u, ~0u);
+        m = r < n ? __ldcg(tk.om + r) : 0;
+        call = r < n ? __ldcg(tk.ocall + r) : 0u;
     };
-    prefetch(0);
+    fetch(0, nrow, nm, ncall);
+    fetch(kPassThreads, nrow2, nm2, ncall2);
     unsigned n_acc = 0;                                         // kept by warp 0 (the same in its 32 lanes)
     unsigned count = 0;                                         // staged calls, the same in every thread
     for (int scan = 0; scan < n; scan += kPassThreads) {
-        const Row row = remap(nrow);
-        const int mm = __float2int_ru(nm);
+        const Row row = narrow(nrow);
+        const int mm = nm;
         const unsigned call = ncall;
-        prefetch(scan + kPassThreads);
-        unsigned kt0; int dt0, fr0;
-        first_fit(row, mm, kt0, dt0, fr0);
-        const bool live = scan + tid < n && dt0 >= 0;
+        nrow = nrow2; nm = nm2; ncall = ncall2;
+        fetch(scan + 2 * kPassThreads, nrow2, nm2, ncall2);
+        const bool live = scan + tid < n && any_fit(row, mm);
         const unsigned lm = __ballot_sync(0xffffffffu, live);   // ordered compaction behind the staged calls
         if (lane == 0) wsum[warp] = __popc(lm);
         __syncthreads();
@@ -458,13 +461,11 @@ cudaError_t hx_launch_conflict(const HxTables& t, const HxTopkBufs& tk, int n_ca
                                long long* launches) {
     (void)status;
     const int D = t.D, P = t.P;
-    const int staged = n_calls <= 16 * 1024;                       // every key held in registers, list fits shared memory
-    const size_t smB = staged ? (size_t)n_calls * 8 : 0;
-    static size_t allowed_bins[64];
-    cudaError_t e = hx_opt_in_smem(hx_order_bins_kernel, smB, allowed_bins, 24 * 1024);
-    if (e != cudaSuccess) return e;
-    hx_order_bins_kernel<<<1, 1024, smB, stream>>>(tk, n_calls, staged);
-    hx_order_rank_kernel<<<(n_calls + 127) / 128, 128, 0, stream>>>(tk, n_calls);
+    const int nb = (n_calls + kOrdThreads - 1) / kOrdThreads;
+    hx_order_hist_kernel<<<nb, kOrdThreads, 0, stream>>>(tk, n_calls);
+    hx_order_scatter_kernel<<<nb, kOrdThreads, 0, stream>>>(tk, n_calls);
+    hx_order_rank_kernel<<<(n_calls + 127) / 128, 128, 0, stream>>>(tk, n_calls, (unsigned)D);
+    cudaError_t e;
     const int fused = P <= kTailMaxP;                               // pairs published and queues summed inside the pass
     const size_t smRing = (size_t)kRing * 24 + (size_t)(D + 1) * 4;
     const size_t smTail = fused ? (size_t)kTailLen * 10 + (size_t)(4 + kPassThreads / 32) * P * 4 : 0;
@@ -475,7 +476,7 @@ cudaError_t hx_launch_conflict(const HxTables& t, const HxTopkBufs& tk, int n_ca
     e = hx_opt_in_smem(pass, smC, allowed_pass[tk.K <= 1 ? 0 : tk.K <= 2 ? 1 : tk.K <= 4 ? 2 : 3], 40 * 1024);
     if (e != cudaSuccess) return e;
     pass<<<1, kPassThreads, smC, stream>>>(tk, t, n_calls, commit, fused, out_assign);
-    *launches += 3;
+    *launches += 4;
     if (!fused) {
         hx_finish_kernel<<<(n_calls + 255) / 256, 256, 0, stream>>>(tk, D, out_assign);
         *launches += 1;

@@ -197,8 +197,11 @@ int ensure_topk(hx_cluster* h, int n_calls, int K) {
     HX_TRY(dev_alloc(h->tk_allocs, &b.dsel, cap), "alloc top-K");
     HX_TRY(dev_alloc(h->tk_allocs, &b.prio, cap), "alloc top-K");
     HX_TRY(dev_alloc(h->tk_allocs, &b.mtok, cap), "alloc top-K");
+    HX_TRY(dev_alloc(h->tk_allocs, &b.blk_lohi, (size_t)2 * HX_ORDER_MAXBLK), "alloc order");
+    HX_TRY(dev_alloc(h->tk_allocs, &b.ghist, (size_t)HX_ORDER_BINS), "alloc order");
+    HX_TRY(dev_alloc(h->tk_allocs, &b.oslot, cap), "alloc order");
     HX_TRY(dev_alloc(h->tk_allocs, &b.okey, cap), "alloc order");
-    HX_TRY(dev_alloc(h->tk_allocs, &b.obase, (size_t)2048 + 3), "alloc order");
+    HX_TRY(dev_alloc(h->tk_allocs, &b.obase, (size_t)HX_ORDER_BINS + 3), "alloc order");
     HX_TRY(dev_alloc(h->tk_allocs, &b.ocall, cap), "alloc order");
     HX_TRY(dev_alloc(h->tk_allocs, &b.om, cap), "alloc order");
     HX_TRY(dev_alloc(h->tk_allocs, &b.od, cap), "alloc order");
@@ -1126,7 +1129,10 @@ constexpr size_t kStaticBytes =
     2 * static_round(kSC * 16) +          // dsel, od
     4 * static_round(kSC * 4) +           // prio, mtok, ocall, om
     static_round(kSC * 8) +               // okey
-    static_round((2048 + 3) * 4) +        // obase
+    static_round((HX_ORDER_BINS + 3) * 4) +   // obase
+    static_round(2 * HX_ORDER_MAXBLK * 4) +   // blk_lohi
+    static_round(HX_ORDER_BINS * 4) +         // ghist
+    static_round(kSC * 4) +               // oslot
     static_round(4) +                     // n_acc
     3 * static_round(kSC * 4);            // acc_rk, acc_p, acc_t
 
@@ -1180,9 +1186,12 @@ int hx_schedule_batch_static(hx_cluster* h, const hx_call* calls, int n_calls, i
     b.prio = reinterpret_cast<float*>(carve(kSC * 4));
     b.mtok = reinterpret_cast<float*>(carve(kSC * 4));
     b.ocall = reinterpret_cast<unsigned int*>(carve(kSC * 4));
-    b.om = reinterpret_cast<float*>(carve(kSC * 4));
+    b.om = reinterpret_cast<int*>(carve(kSC * 4));
     b.okey = reinterpret_cast<unsigned long long*>(carve(kSC * 8));
-    b.obase = reinterpret_cast<unsigned int*>(carve((2048 + 3) * 4));
+    b.obase = reinterpret_cast<unsigned int*>(carve((HX_ORDER_BINS + 3) * 4));
+    b.blk_lohi = reinterpret_cast<unsigned int*>(carve(2 * HX_ORDER_MAXBLK * 4));
+    b.ghist = reinterpret_cast<unsigned int*>(carve(HX_ORDER_BINS * 4));
+    b.oslot = reinterpret_cast<unsigned int*>(carve(kSC * 4));
     b.n_acc = reinterpret_cast<unsigned int*>(carve(4));
     b.acc_rk = reinterpret_cast<unsigned int*>(carve(kSC * 4));
     b.acc_p = reinterpret_cast<int*>(carve(kSC * 4));

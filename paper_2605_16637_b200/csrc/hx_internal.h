@@ -72,17 +72,31 @@ struct HxTopkBufs {
     float* prio;               // [cap]
     float* mtok;               // [cap]
     // visiting order
+    unsigned int* blk_lohi;    // [2 * HX_ORDER_MAXBLK] smallest / largest finite key seen by each block of the scoring kernel
+    unsigned int* ghist;       // [HX_ORDER_BINS] keys per bin (zeroed by the scoring kernel)
+    unsigned int* oslot;       // [cap] bin << 16 | arrival number inside the bin, per call
     unsigned long long* okey;  // [cap] keys grouped by bin
-    unsigned int* obase;       // [2048 + 3] bin bounds, smallest key, key-to-bin shift
+    unsigned int* obase;       // [HX_ORDER_BINS + 3] bin bounds, smallest key, key-to-bin shift
     unsigned int* ocall;       // [cap] call of each rank
-    float* om;                 // [cap] demand of each rank
-    uint4* od;                 // [cap] same rows in visiting order
+    int* om;                   // [cap] demand of each rank, tokens
+    uint4* od;                 // [cap] same rows in visiting order, unused slots pointing at instance D
     // outcome: calls that obtained a pair, in visiting order
     unsigned int* n_acc;       // [1]
     unsigned int* acc_rk;      // [cap] call | k << 24
     int* acc_p;                // [cap] prefill instance obtained
     float* acc_t;              // [cap] prefill time added to that instance
 };
+
+// Visiting order of the capacity pass: key = bit pattern of the priority, inverted (larger priority =
+// smaller key); a priority of +inf, or one that is not a number or negative, gets HX_FIRST_KEY and is
+// visited first.  Bin 0 holds those keys; bins 1 .. HX_ORDER_BINS - 1 are linear in the key between the
+// smallest and the largest finite key of the batch.
+#define HX_ORDER_BINS 2048
+#define HX_ORDER_MAXBLK 1024
+#define HX_FIRST_KEY 0x807FFFFFu
+__host__ __device__ inline unsigned hx_order_key(unsigned prio_bits) {
+    return prio_bits >= 0x7F800000u ? HX_FIRST_KEY : ~prio_bits;
+}
 
 struct ScoreLaunch {
     const hx_call* calls;

@@ -227,6 +227,14 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
     float* capDs = qDs + Dpad;                                    // [Dpad]
     int* typeDs = reinterpret_cast<int*>(capDs + Dpad);           // [Dpad]
 
+    // visiting order of the capacity pass: this kernel clears the bin counters and leaves the smallest and
+    // the largest finite priority key of every block's calls behind (no state survives from earlier batches)
+    unsigned key_lo = 0xFFFFFFFFu, key_hi = 0u;
+    __shared__ unsigned key_lohi[2];
+    if (prm.s.K > 0) {
+        for (int i = blockIdx.x * nthr + tid; i < HX_ORDER_BINS; i += gridDim.x * nthr) prm.tk.ghist[i] = 0u;
+        if (tid == 0) { key_lohi[0] = 0xFFFFFFFFu; key_lohi[1] = 0u; }
+    }
     // the call records of the first tile come from DRAM: request them before anything else
     const bool with_dag = !(prm.s.flags & HX_FLAG_NO_DAG);
     uint4 pre[2];
@@ -551,7 +559,10 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
                     prm.s.out_assign[gc] = (jbest == HX_NONE) ? -1 : jbest;
                 } else {
                     prm.s.out_assign[gc] = -1;            // filled in by the capacity-conflict pass
-                    prm.tk.prio[gc] = __fdiv_rn(__fadd_rn(elapsed, v0), H);   // Eq. 2
+                    const float prio = __fdiv_rn(__fadd_rn(elapsed, v0), H);  // Eq. 2
+                    prm.tk.prio[gc] = prio;
+                    const unsigned key = hx_order_key(__float_as_uint(prio));
+                    if (key != HX_FIRST_KEY) { key_lo = min(key_lo, key); key_hi = max(key_hi, key); }
                     prm.tk.mtok[gc] = m;
                     unsigned dw[4] = {~0u, ~0u, ~0u, ~0u};          // decode instances of the slots, 8 x 16 bits
 #pragma unroll
@@ -568,6 +579,16 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
             }
         }
         __syncthreads();
+    }
+    if (prm.s.K > 0) {
+        key_lo = __reduce_min_sync(0xffffffffu, key_lo); key_hi = __reduce_max_sync(0xffffffffu, key_hi);
+        if (lane == 0) { atomicMin(&key_lohi[0], key_lo); atomicMax(&key_lohi[1], key_hi); }
+        __syncthreads();
+        // every slot of the table gets some block's values: the reader need not know the grid size
+        for (int b = blockIdx.x + tid * gridDim.x; b < HX_ORDER_MAXBLK; b += nthr * gridDim.x) {
+            prm.tk.blk_lohi[b] = key_lohi[0];
+            prm.tk.blk_lohi[HX_ORDER_MAXBLK + b] = key_lohi[1];
+        }
     }
 }
 
