@@ -546,6 +546,24 @@ def replay_leg():
             w = hr.replay(orc, oc, wl.row_ptr, wl.col, wl.node_wf, wl.n_workflows, wl.node_calls, arrival, dag)
             out["oracle_wall_ms_1_core_middle_load"] = 1e3 * (time.perf_counter() - t0)
             out["identical_to_oracle"] = bool(np.array_equal(r["fin"], w["fin"]) and r["req99"] == w["req99"])
+    # the stages of a call kept apart, the decode stage scheduled, estimation error on what the schedulers see
+    # (Section 7.6): Req95 / Req99 at four error levels on the heaviest of the loads above
+    arrival = u * float(cost.sum()) / (wl.P * LOADS[-1])
+    life = {}
+    for eps in (0.0, 0.1, 0.2, 0.3):
+        t0 = time.perf_counter()
+        r = gc.replay_lifecycle(wl.node_calls, arrival, est_error=eps)
+        dt = time.perf_counter() - t0
+        life["%.1f" % eps] = {"req95": r["req95"], "req99": r["req99"], "prefill_planner_runs": r["runs"],
+                              "decode_planner_runs": r["decode_runs"], "unplanned": r["stuck"], "wall_ms": 1e3 * dt,
+                              "us_per_planner_run": 1e6 * dt / max(r["runs"] + r["decode_runs"], 1)}
+    orc, oc = ho.Oracle(), ho.Cluster.from_workload(wl)
+    dag = orc.longest_path(wl.row_ptr, wl.col, cost, wl.node_wf, wl.n_workflows)
+    t0 = time.perf_counter()
+    w = hr.replay_lifecycle(orc, oc, wl.row_ptr, wl.col, wl.node_wf, wl.n_workflows, wl.node_calls, arrival, dag, est_error=0.2)
+    out["lifecycle"] = {"load": LOADS[-1], "est_error": life, "oracle_wall_ms_1_core_error_0.2": 1e3 * (time.perf_counter() - t0),
+                        "identical_to_oracle_error_0.2": bool(np.array_equal(
+                            gc.replay_lifecycle(wl.node_calls, arrival, est_error=0.2)["fin"], w["fin"]))}
     out["device_status"] = gc.status()
     gc.close()
     return out

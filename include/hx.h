@@ -383,14 +383,76 @@ int hx_schedule_greedy_plan(hx_cluster* h, const hx_call* calls, int n_calls,
  * left unplanned.  The call overwrites the cluster's loads and elapsed times,
  * uses `stream`, synchronises it once per planner run, allocates and frees its
  * device scratch, and restores hx_options on return.  Errors:
- * HX_ERR_INVALID_ARG (NULL array, qmax outside 1 .. HX_GREEDY_MAX_CALLS, sizes
- * that differ from the upload, node_calls[v].node != v, a negative or non-finite
- * arrival), HX_ERR_NOT_READY without horizons, and those of the calls it makes. */
+ * HX_ERR_INVALID_ARG (NULL array, qmax outside 1 .. HX_GREEDY_MAX_CALLS, a graph
+ * that differs from the uploaded one in size, row bounds, successors or workflow
+ * of a node, node_calls[v].node != v, a negative or non-finite arrival),
+ * HX_ERR_NOT_READY without horizons, and those of the calls it makes. */
 int hx_replay(hx_cluster* h, const uint32_t* row_ptr, const uint32_t* col_idx,
               const uint32_t* node_workflow, uint32_t n_nodes, uint32_t n_workflows,
               const hx_call* node_calls, const double* arrival_s, int qmax,
               double* out_fin, double* out_ratio, double* out_req, int* out_stats,
               void* stream);
+
+/* The same replay with the stages of a call's life kept apart, the decode stage
+ * scheduled, and scheduler-visible estimates that may be wrong (Section 6: the
+ * simulator follows every call through waiting for prefill, prefill, KV transfer,
+ * waiting for decode, decode and completion and keeps decode token-capacity
+ * intervals; Section 5.2: the schedulers run when work enters a stage; Section 5.4:
+ * decode scheduling with the planned instance as a lock; Section 7.6: a
+ * deterministic multiplicative error on the prefill and decode estimates the
+ * scheduler sees, the service durations unchanged).
+ *   What happens: prefill instance p serves the calls planned onto it one at a
+ * time in the order they were planned, each for its prefill time on p's class;
+ * the KV cache then travels for kv_bytes / link(p, d); at its decode instance d
+ * the call waits until d admits it: whenever a plan, an arrival or a completion
+ * changed d's state, the waiting calls are taken in the order of the latest
+ * decode plan (node number among calls of equal rank) and every one whose tokens
+ * (Eq. 3) fit the tokens really free starts decoding and holds them for its
+ * decode time on d's class; a call completes with its decode.
+ *   What the schedulers see: all service times from the same latency model with
+ * the constants of the call's model scaled by the binary32 factor 1 + est_error
+ * or 1 - est_error (the sign is a fixed function of the node number); prefill
+ * queue = estimated time left of the call in service (at least 0) plus the
+ * estimated prefill times queued behind it; free KV tokens = Cap(d) minus the
+ * tokens of every call planned onto d and not complete; decode hint 0; elapsed
+ * time t - a_w; decode snapshot = every call decoding on d until its estimated
+ * end (at least 1e-6 s from now).
+ *   Scheduler runs: hx_schedule_greedy_plan at every event time at which calls are
+ * ready (increasing node number, at most qmax per run, run after run; a call
+ * passed over stays ready); hx_schedule_decode, without commit, at every event
+ * time at which a KV transfer completed, over the calls waiting for decode
+ * (increasing node number, the first HX_DECODE_MAX_CALLS of them).  Events with
+ * equal time stamps are taken together.  Time is binary64 on the host, service
+ * times are the binary32 values of hx_estimate_calls.  The paper prints no
+ * pseudo-code of its simulator: these rules are this library's reading.
+ *   The replay runs on the uploaded forest (including appended nodes) with
+ * hx_critical_path enqueued; node_calls[v] (host) describes node v; arrival_s
+ * (host) has one entry per workflow.  Outputs (host): out_fin[n_nodes],
+ * out_ratio[n_workflows], out_req[2] = Req95, Req99 (Section 7.3), out_stats[3] =
+ * prefill planner runs, decode planner runs, calls never planned.  The call
+ * overwrites the cluster's loads, elapsed times and decode snapshot, uses
+ * `stream` and synchronises it once per planner run, allocates and frees its
+ * scratch, needs three times the cluster's models to fit HX_MAX_MODELS, and
+ * restores hx_options on return.  Errors: HX_ERR_INVALID_ARG (NULL array, qmax
+ * outside 1 .. HX_GREEDY_MAX_CALLS, est_error outside [0, 1), node_calls[v].node
+ * != v, a model id out of range, a bad arrival time, too many models),
+ * HX_ERR_NOT_READY without forest or horizons, and those of the calls it makes. */
+int hx_replay_lifecycle(hx_cluster* h, const hx_call* node_calls, const double* arrival_s,
+                        double est_error, int qmax, double* out_fin, double* out_ratio,
+                        double* out_req, int* out_stats, void* stream);
+
+/* Service-time estimates of n_calls call records (the Estimator of Section 4.2,
+ * "Scheduler internals": prefill time, decode time, KV-transfer volume and decode
+ * memory demand from input and output length with a roofline-style model), the
+ * terms the scoring and planning kernels build their projections from.  calls:
+ * device, 16-byte aligned.  Outputs, device: out_tpre and out_tdec
+ * float[n_calls][n_types] (seconds on each GPU class), out_kv_bytes
+ * float[n_calls] (bytes of the prompt's KV cache: the transfer takes this over the
+ * link bandwidth), out_tokens float[n_calls] (m of Eq. 3).  A record with a model id
+ * out of range gets +inf times and raises HX_ERR_INVALID_ARG in the status word.
+ * Enqueues one kernel on `stream`. */
+int hx_estimate_calls(hx_cluster* h, const hx_call* calls, int n_calls, float* out_tpre,
+                      float* out_tdec, float* out_kv_bytes, float* out_tokens, void* stream);
 
 /* Decode-stage scheduler (Section 5.4, "Decode scheduling with instance locks",
  * "Decode KV-capacity feasibility check", "Adaptive greedy decode assignment").

@@ -68,6 +68,8 @@ def _load():
         "hx_schedule_greedy": [vp, vp, ci, vp, vp, vp, vp],
         "hx_schedule_greedy_plan": [vp, vp, ci, vp, vp, vp, vp, vp],
         "hx_replay": [vp, vp, vp, vp, C.c_uint32, C.c_uint32, vp, vp, ci, vp, vp, vp, vp, vp],
+        "hx_replay_lifecycle": [vp, vp, vp, C.c_double, ci, vp, vp, vp, vp, vp],
+        "hx_estimate_calls": [vp, vp, ci, vp, vp, vp, vp, vp],
         "hx_decode_set_running": [vp, vp, vp, vp],
         "hx_schedule_decode": [vp, vp, vp, vp, ci, vp, vp, vp, vp, vp],
         "hx_get_topk": [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp)],
@@ -236,6 +238,26 @@ def hx_replay(h, row_ptr, col_idx, node_workflow, n_workflows, node_calls, arriv
                 stuck=int(stats[1]))
 
 
+def hx_replay_lifecycle(h, n_workflows, node_calls, arrival_s, est_error=0.0, qmax=4096, stream=0):
+    """Replay with separate stages, a scheduled decode stage and estimation error; host arrays in,
+    dict(fin, ratio, req95, req99, runs, decode_runs, stuck) out."""
+    calls, arr = _np(node_calls, CALL_DTYPE), _np(arrival_s, np.float64)
+    n, w = calls.shape[0], int(n_workflows)
+    if arr.shape[0] != w:
+        raise HxError(-1, "array lengths differ")
+    fin, ratio = np.zeros(n, np.float64), np.zeros(w, np.float64)
+    req, stats = np.zeros(2, np.float64), np.zeros(3, np.int32)
+    _check(_lib.hx_replay_lifecycle(h, _p(calls), _p(arr), float(est_error), int(qmax), _p(fin), _p(ratio), _p(req),
+                                    _p(stats), stream), h)
+    return dict(fin=fin, ratio=ratio, req95=float(req[0]), req99=float(req[1]), runs=int(stats[0]),
+                decode_runs=int(stats[1]), stuck=int(stats[2]))
+
+
+def hx_estimate_calls(h, calls_ptr, n_calls, out_tpre_ptr, out_tdec_ptr, out_kv_ptr, out_tokens_ptr, stream=0):
+    _check(_lib.hx_estimate_calls(h, calls_ptr, int(n_calls), out_tpre_ptr, out_tdec_ptr, out_kv_ptr, out_tokens_ptr,
+                                  stream), h)
+
+
 KV_INTERVAL_DTYPE = np.dtype([("end_s", "<f4"), ("tokens", "<f4")])
 
 
@@ -350,6 +372,7 @@ class Cluster:
         self.P = int((inst["role"] == 0).sum())
         self.D = int(inst.shape[0] - self.P)
         self.M = int(_np(models, np.float32).reshape(-1, 3).shape[0])
+        self.G = int(_np(gpu_types, np.float32).reshape(-1, 2).shape[0])
         self.n_nodes = 0
         self.n_workflows = 0
         self.topk = 0
@@ -457,6 +480,22 @@ class Cluster:
     def replay(self, row_ptr, col_idx, node_workflow, node_calls, arrival_s, qmax=4096):
         return hx_replay(self.h, row_ptr, col_idx, node_workflow, self.n_workflows, node_calls, arrival_s, qmax,
                          self._stream())
+
+    def replay_lifecycle(self, node_calls, arrival_s, est_error=0.0, qmax=4096):
+        return hx_replay_lifecycle(self.h, len(arrival_s), node_calls, arrival_s, est_error, qmax, self._stream())
+
+    def estimate_calls(self, calls):
+        """Service-time terms of the given calls: (tpre[n, G], tdec[n, G], kv_bytes[n], tokens[n]) device tensors."""
+        import torch
+        calls = _np(calls, CALL_DTYPE)
+        n = calls.shape[0]
+        dev = torch.from_numpy(calls.view(np.uint8).reshape(-1, 16).copy()).cuda()
+        tp = torch.empty((n, self.G), dtype=torch.float32, device="cuda"); td = torch.empty_like(tp)
+        kv = torch.empty(n, dtype=torch.float32, device="cuda"); tok = torch.empty_like(kv)
+        hx_estimate_calls(self.h, dev.data_ptr(), n, tp.data_ptr(), td.data_ptr(), kv.data_ptr(), tok.data_ptr(),
+                          self._stream())
+        torch.cuda.current_stream().synchronize()
+        return tp, td, kv, tok
 
     def decode_set_running(self, inst_ptr, end_s, tokens):
         run = np.zeros(len(end_s), KV_INTERVAL_DTYPE)

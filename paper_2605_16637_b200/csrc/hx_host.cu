@@ -106,6 +106,7 @@ struct hx_cluster {
     // copy streams and events of hx_schedule_sweep_host, created on first use
     cudaStream_t sw_in = nullptr, sw_out = nullptr;
     std::vector<cudaEvent_t> sw_ev;
+    int M_base = 0;                     // models before hx_push_scaled_models (0 = nothing pushed)
     hx_options opts{HX_MODE_COMPLETION, 0, 0, 0, 1.5f};
     std::string err;
     long long launches = 0;
@@ -383,6 +384,47 @@ void hx_cluster_shape(const hx_cluster* h, int* P, int* D, const float** capD_de
     *n_nodes = h->dag_uploaded ? h->N : 0; *n_workflows = h->dag_uploaded ? h->W : 0;
 }
 hx_options hx_current_options(const hx_cluster* h) { return h->opts; }
+
+int hx_cluster_tables_host(hx_cluster* h, std::vector<int>* typeP, std::vector<int>* typeD, std::vector<float>* invLT,
+                           int* Ppad, int* G, int* M, cudaStream_t s) {
+    typeP->resize(h->Ppad); typeD->resize(h->D); invLT->resize((size_t)h->D * h->Ppad);
+    *Ppad = h->Ppad; *G = h->G; *M = h->M;
+    HX_TRY(cudaMemcpyAsync(typeP->data(), h->tab.typeP, typeP->size() * sizeof(int), cudaMemcpyDeviceToHost, s), "reading the cluster tables");
+    HX_TRY(cudaMemcpyAsync(typeD->data(), h->tab.typeD, typeD->size() * sizeof(int), cudaMemcpyDeviceToHost, s), "reading the cluster tables");
+    HX_TRY(cudaMemcpyAsync(invLT->data(), h->tab.invLT, invLT->size() * sizeof(float), cudaMemcpyDeviceToHost, s), "reading the cluster tables");
+    HX_TRY(cudaStreamSynchronize(s), "cudaStreamSynchronize");
+    return HX_OK;
+}
+
+void hx_forest_host(const hx_cluster* h, std::vector<uint32_t>* row, std::vector<uint32_t>* col, std::vector<uint32_t>* node_wf) {
+    const uint32_t N = h->N;
+    row->assign((size_t)N + 1, 0); col->clear(); col->reserve(h->E);
+    for (uint32_t v = 0; v < N; ++v) {
+        for_each_successor(h, v, [&](uint32_t u) { col->push_back(u); });
+        (*row)[v + 1] = (uint32_t)col->size();
+    }
+    *node_wf = h->h_node_wf;
+}
+
+int hx_push_scaled_models(hx_cluster* h, float up, float down) {
+    if (h->M_base) return fail(h, HX_ERR_INVALID_ARG, "scaled models are already in place");
+    const int M = h->M;
+    if (3 * M > HX_MAX_MODELS) return fail(h, HX_ERR_INVALID_ARG, "three times the models do not fit the model table");
+    const float f[2] = {up, down};
+    for (int k = 0; k < 2; ++k)
+        for (int m = 0; m < M; ++m) {
+            const int o = (k + 1) * M + m;
+            h->ctab.phi[o] = h->ctab.phi[m] * f[k]; h->ctab.omega[o] = h->ctab.omega[m] * f[k];
+            h->ctab.kappa[o] = h->ctab.kappa[m] * f[k]; h->ctab.psi[o] = h->ctab.psi[m] * f[k];
+        }
+    h->M_base = M; h->M = 3 * M; h->tab.M = 3 * M;
+    return HX_OK;
+}
+
+void hx_pop_scaled_models(hx_cluster* h) {
+    if (!h->M_base) return;
+    h->M = h->M_base; h->tab.M = h->M_base; h->M_base = 0;
+}
 
 extern "C" {
 
@@ -1354,6 +1396,19 @@ int hx_schedule_decode(hx_cluster* h, const hx_call* calls, const int32_t* lock,
                "decode scheduler kernel");
     }
     if (o.commit) { h->dec_k_bound += 2 * n_calls; h->dec_k_total += 2LL * n_calls; }
+    return HX_OK;
+}
+
+int hx_estimate_calls(hx_cluster* h, const hx_call* calls, int n_calls, float* out_tpre, float* out_tdec,
+                      float* out_kv_bytes, float* out_tokens, void* stream) {
+    if (!h) return HX_ERR_INVALID_ARG;
+    if (n_calls < 0) return fail(h, HX_ERR_INVALID_ARG, "negative n_calls");
+    if (n_calls == 0) return HX_OK;
+    if (!calls || !out_tpre || !out_tdec || !out_kv_bytes || !out_tokens) return fail(h, HX_ERR_INVALID_ARG, "NULL buffer");
+    if (reinterpret_cast<uintptr_t>(calls) % 16) return fail(h, HX_ERR_INVALID_ARG, "calls must be 16-byte aligned");
+    DeviceGuard guard(h->device);
+    HX_TRY(hx_launch_estimate(h->ctab, h->G, h->M, calls, n_calls, out_tpre, out_tdec, out_kv_bytes, out_tokens, h->status,
+                              static_cast<cudaStream_t>(stream), &h->launches), "estimate kernel");
     return HX_OK;
 }
 

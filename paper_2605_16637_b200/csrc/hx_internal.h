@@ -134,6 +134,10 @@ cudaError_t hx_launch_conflict(const HxTables& t, const HxTopkBufs& tk, int n_ca
                                int32_t* out_assign, int* status, cudaStream_t stream,
                                long long* launches);
 
+cudaError_t hx_launch_estimate(const HxConstTables& ct, int G, int M, const hx_call* calls, int n_calls,
+                               float* tpre, float* tdec, float* kvB, float* m, int* status, cudaStream_t stream,
+                               long long* launches);
+
 size_t hx_greedy_smem_bytes(const HxTables& t, int n_calls);
 cudaError_t hx_launch_greedy(const HxTables& t, const HxConstTables& ct, const HxDagView& dag,
                              const hx_call* calls, int n_calls, int flags, int commit,
@@ -205,6 +209,15 @@ cudaError_t hx_launch_cost_update(const HxForestDev& f, const uint32_t* idx, con
 int hx_fail(hx_cluster* h, int code, const char* msg);            // records msg as the last error, returns code
 void hx_cluster_shape(const hx_cluster* h, int* P, int* D, const float** capD_dev, uint32_t* n_nodes, uint32_t* n_workflows);
 hx_options hx_current_options(const hx_cluster* h);
+// Classes of the instances (prefill first, then decode) and the reciprocal link table, read back from the device.
+int hx_cluster_tables_host(hx_cluster* h, std::vector<int>* typeP, std::vector<int>* typeD, std::vector<float>* invLT,
+                           int* Ppad, int* G, int* M, cudaStream_t s);
+// Successor lists of the forest as it stands (upload plus appended nodes and edges) and the workflow of every node.
+void hx_forest_host(const hx_cluster* h, std::vector<uint32_t>* row, std::vector<uint32_t>* col, std::vector<uint32_t>* node_wf);
+// Every model once more with its constants scaled by up and by down (models M .. 2M - 1 and 2M .. 3M - 1), until
+// hx_pop_scaled_models; HX_ERR_INVALID_ARG when three times the models do not fit the table.
+int hx_push_scaled_models(hx_cluster* h, float up, float down);
+void hx_pop_scaled_models(hx_cluster* h);
 
 // Opt a kernel in to `bytes` of dynamic shared memory, once per device and size: the attribute
 // call is too slow to repeat on every launch.  `allowed` is a per-kernel table of 64 entries
