@@ -501,6 +501,14 @@ def refine_leg():
         new = np.arange(wl.n_nodes + i * k, wl.n_nodes + (i + 1) * k, dtype=np.uint32)
         batches.append((rng.lognormal(0, 1, k).astype(np.float32), wfs, first_of[wfs], new))
     out["append_1000_nodes_ms"] = wall(lambda: gc.dag_append(*batches.pop(0)))
+    # 1,000 arriving workflows (Section 5.2, first trigger): registered, then their two source calls each handed in
+    state = {"n": wl.n_nodes + 5 * k, "w": wl.n_workflows}
+    def arrive():
+        gc.dag_append_workflows(np.zeros(k, np.float32))
+        wfs = np.repeat(np.arange(state["w"], state["w"] + k, dtype=np.uint32), 2)
+        gc.dag_append(rng.lognormal(0, 1, 2 * k).astype(np.float32), wfs, [], [])
+        state["n"] += 2 * k; state["w"] += k
+    out["arrival_1000_workflows_ms"] = wall(arrive)
     orc = ho.Oracle()
     t0 = time.perf_counter()
     orc.longest_path(wl.row_ptr, wl.col, cost, wl.node_wf, wl.n_workflows)

@@ -180,7 +180,8 @@ int hx_get_dag_results(hx_cluster* h, const float** cp, const float** tail, cons
  * the horizon is refined as the workflow reveals more of its DAG).  The new
  * nodes take the numbers n_nodes .. n_nodes + n_new_nodes - 1 (n_nodes = the
  * count before the call); new_costs[i] and new_node_workflow[i] (an existing
- * workflow) describe node n_nodes + i.  Edge e runs from edge_src[e] to
+ * workflow, possibly one registered by hx_dag_append_workflows) describe node
+ * n_nodes + i.  Edge e runs from edge_src[e] to
  * edge_dst[e]; either end may be an old or a new node of the same workflow.
  * All arrays are host arrays, read before the call returns.  The workflows
  * touched are levelised again as a group of their own and, once horizons
@@ -198,6 +199,24 @@ int hx_get_dag_results(hx_cluster* h, const float** cp, const float** tail, cons
 int hx_dag_append(hx_cluster* h, uint32_t n_new_nodes, const float* new_costs,
                   const uint32_t* new_node_workflow, uint32_t n_new_edges,
                   const uint32_t* edge_src, const uint32_t* edge_dst, void* stream);
+
+/* Arrival of workflows (Section 5.2: the scheduler runs "when a workflow arrives
+ * and reveals source calls"; Section 4.3: only the source calls are revealed on
+ * arrival).  Registers n_new_workflows workflows numbered n_workflows ..
+ * n_workflows + n_new_workflows - 1 (n_workflows = the count before the call)
+ * with the elapsed times new_elapsed_s (host, or NULL = all 0) and no node yet:
+ * their horizon is 0 until hx_dag_append hands in their first (source) calls,
+ * which then costs what any append costs and leaves every other workflow
+ * untouched.  The result equals a fresh upload of the grown forest bit for bit.
+ * The horizon and elapsed-time arrays keep a reserve (a quarter of the uploaded
+ * count, at least 4,096); beyond it they are reallocated, which synchronises the
+ * device and moves them: fetch hx_get_dag_results again.  The forward results
+ * are dropped; call hx_earliest_start again.  Later hx_dag_update_elapsed calls
+ * pass one value per workflow of the grown count.  Errors (nothing changed):
+ * HX_ERR_NOT_READY without an upload, HX_ERR_INVALID_ARG for an elapsed time
+ * that is negative or not finite. */
+int hx_dag_append_workflows(hx_cluster* h, uint32_t n_new_workflows, const float* new_elapsed_s,
+                            void* stream);
 
 /* Forward pass over the same forest (Section 4.1: a node becomes ready when
  * all its predecessors have completed): for every node v

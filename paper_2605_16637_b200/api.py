@@ -56,6 +56,7 @@ def _load():
         "hx_dag_update_elapsed": [vp, vp, vp],
         "hx_get_dag_results": [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp)],
         "hx_dag_append": [vp, C.c_uint32, vp, vp, C.c_uint32, vp, vp, vp],
+        "hx_dag_append_workflows": [vp, C.c_uint32, vp, vp],
         "hx_earliest_start": [vp, vp],
         "hx_get_earliest_results": [vp, C.POINTER(vp), C.POINTER(vp)],
         "hx_set_options": [vp, C.POINTER(_Options)],
@@ -176,6 +177,12 @@ def hx_dag_append(h, new_costs, new_node_workflow, edge_src, edge_dst, stream=0)
     if c.shape[0] != w.shape[0] or es.shape[0] != ed.shape[0]:
         raise HxError(-1, "array lengths differ")
     _check(_lib.hx_dag_append(h, c.shape[0], _p(c), _p(w), es.shape[0], _p(es), _p(ed), stream), h)
+
+
+def hx_dag_append_workflows(h, new_elapsed_s, stream=0):
+    """Registers len(new_elapsed_s) arriving workflows (numbered on from the old count, no nodes yet)."""
+    el = _np(new_elapsed_s, np.float32)
+    _check(_lib.hx_dag_append_workflows(h, el.shape[0], _p(el), stream), h)
 
 
 def hx_earliest_start(h, stream=0):
@@ -426,6 +433,10 @@ class Cluster:
     def dag_append(self, new_costs, new_node_workflow, edge_src, edge_dst):
         hx_dag_append(self.h, new_costs, new_node_workflow, edge_src, edge_dst, self._stream())
         self.n_nodes += int(np.asarray(new_costs).shape[0])
+
+    def dag_append_workflows(self, new_elapsed_s):
+        hx_dag_append_workflows(self.h, new_elapsed_s, self._stream())
+        self.n_workflows += int(np.asarray(new_elapsed_s).shape[0])
 
     def earliest_start(self):
         hx_earliest_start(self.h, self._stream())

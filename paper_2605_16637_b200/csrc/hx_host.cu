@@ -73,6 +73,8 @@ struct hx_cluster {
     std::vector<ForestPart> parts;      // part 0: the upload; later ones: workflows rebuilt by hx_dag_append
     uint32_t N = 0, E = 0, W = 0;       // current size of the forest
     size_t capN = 0;                    // room in cp, tail and node_wf
+    size_t capW = 0;                    // room in H and the elapsed times
+    std::vector<void*> wf_allocs;       // H, elapsed: regrown when arriving workflows outgrow them
     std::vector<void*> node_allocs;     // cp, tail, node_wf: regrown when appended nodes outgrow them
     float *g_cp = nullptr, *g_tail = nullptr, *g_H = nullptr;
     uint32_t* d_node_wf = nullptr;
@@ -564,7 +566,7 @@ int hx_cluster_destroy(hx_cluster* h) {
     DeviceGuard guard(h->device);
     cudaDeviceSynchronize();
     for (auto& p : h->parts) free_pool(p.allocs);
-    free_pool(h->node_allocs);
+    free_pool(h->node_allocs); free_pool(h->wf_allocs);
     free_pool(h->allocs); free_pool(h->dag_allocs); free_pool(h->fwd_allocs); free_pool(h->tk_allocs); free_pool(h->upd_allocs); free_pool(h->dec_allocs);
     if (h->st_calls) cudaFree(h->st_calls);
     if (h->st_assign) cudaFree(h->st_assign);
@@ -617,16 +619,19 @@ int hx_dag_upload(hx_cluster* h, const uint32_t* row_ptr, const uint32_t* col_id
     free_pool(h->fwd_allocs);
     h->dag_uploaded = false; h->cp_ready = false;
     h->fwd_built = false; h->est_ready = false; h->fwd_classes.clear();
-    h->N = h->E = h->W = 0; h->capN = 0;
+    free_pool(h->wf_allocs);
+    h->N = h->E = h->W = 0; h->capN = 0; h->capW = 0;
     // results and the node -> workflow map keep room for nodes appended later
     const size_t cap = (size_t)N + std::max<size_t>(N / 4, 4096);
     HX_TRY(dev_alloc(h->node_allocs, &h->g_cp, cap), "alloc cp");
     HX_TRY(dev_alloc(h->node_allocs, &h->g_tail, cap), "alloc tail");
     HX_TRY(dev_alloc(h->node_allocs, &h->d_node_wf, cap), "alloc node_workflow");
-    HX_TRY(dev_alloc(h->dag_allocs, &h->g_H, W), "alloc H");
+    const size_t capW = (size_t)W + std::max<size_t>(W / 4, 4096);   // room for workflows that arrive later
+    HX_TRY(dev_alloc(h->wf_allocs, &h->g_H, capW), "alloc H");
     HX_TRY(cudaMemcpy(h->d_node_wf, node_workflow, (size_t)N * sizeof(uint32_t), cudaMemcpyHostToDevice), "upload node_workflow");
     std::vector<float> el(workflow_elapsed_s, workflow_elapsed_s + W);
-    HX_TRY(dev_upload(h->dag_allocs, &h->d_elapsed, el), "upload elapsed");
+    HX_TRY(dev_alloc(h->wf_allocs, &h->d_elapsed, capW), "alloc elapsed");
+    HX_TRY(cudaMemcpy(h->d_elapsed, el.data(), (size_t)W * sizeof(float), cudaMemcpyHostToDevice), "upload elapsed");
     h->parts.emplace_back();
     ForestPart& base = h->parts.back();
     base.f.cp = h->g_cp; base.f.tail = h->g_tail; base.f.H = h->g_H;
@@ -639,7 +644,7 @@ int hx_dag_upload(hx_cluster* h, const uint32_t* row_ptr, const uint32_t* col_id
         if (!ok) return fail(h, HX_ERR_CUDA, "creating the side streams of the horizon pass");
         h->fj.ready = 1;
     }
-    h->N = N; h->E = E; h->W = W; h->capN = cap;
+    h->N = N; h->E = E; h->W = W; h->capN = cap; h->capW = capW;
     h->h_inv = std::move(hf.inv);
     h->h_node_wf.assign(node_workflow, node_workflow + N);
     h->h_wf_part.assign(W, 0);
@@ -973,7 +978,7 @@ int hx_dag_append(hx_cluster* h, uint32_t n_new_nodes, const float* new_costs, c
     for (uint32_t i = 0; i < n; ++i) h->h_inv[gid[i]] = hf.inv[i];
     for (size_t j = 0; j < touched.size(); ++j) {
         const uint32_t w = touched[j];
-        h->parts[h->h_wf_part[w]].drop(h->h_wf_local[w]);
+        if (h->h_wf_part[w] != ~0u) h->parts[h->h_wf_part[w]].drop(h->h_wf_local[w]);   // ~0u: arrived without nodes so far
         h->h_wf_part[w] = (uint32_t)q; h->h_wf_local[w] = (uint32_t)j;
         if (!fresh[j].empty()) {
             auto& v = h->extra_nodes[w];
@@ -997,6 +1002,45 @@ int hx_dag_append(hx_cluster* h, uint32_t n_new_nodes, const float* new_costs, c
         h->parts[q].classes(&cls);
         HX_TRY(hx_launch_cpath(h->parts[q].f, cls.data(), (int)cls.size(), s, &h->launches, &h->fj), "horizon kernels");
     }
+    return HX_OK;
+}
+
+int hx_dag_append_workflows(hx_cluster* h, uint32_t n_new_workflows, const float* new_elapsed_s, void* stream) {
+    if (!h) return HX_ERR_INVALID_ARG;
+    if (!h->dag_uploaded) return fail(h, HX_ERR_NOT_READY, "no forest uploaded");
+    if (n_new_workflows == 0) return HX_OK;
+    if ((uint64_t)h->W + n_new_workflows > 0xFFFFFFF0ull) return fail(h, HX_ERR_INVALID_ARG, "more than 2^32 workflows");
+    if (new_elapsed_s)
+        for (uint32_t i = 0; i < n_new_workflows; ++i)
+            if (!good_load(new_elapsed_s[i])) return fail(h, HX_ERR_INVALID_ARG, "elapsed times must be finite and >= 0");
+    DeviceGuard guard(h->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const uint32_t W0 = h->W, W1 = W0 + n_new_workflows;
+    if (W1 > h->capW) {                                   // H and the elapsed times move to larger arrays
+        const size_t cap = std::max<size_t>(W1, 2 * h->capW);
+        std::vector<void*> fresh;
+        float *H, *el;
+        cudaError_t e = dev_alloc(fresh, &H, cap);
+        if (e == cudaSuccess) e = dev_alloc(fresh, &el, cap);
+        if (e == cudaSuccess) e = cudaDeviceSynchronize();
+        if (e == cudaSuccess) e = cudaMemcpy(H, h->g_H, (size_t)W0 * sizeof(float), cudaMemcpyDeviceToDevice);
+        if (e == cudaSuccess) e = cudaMemcpy(el, h->d_elapsed, (size_t)W0 * sizeof(float), cudaMemcpyDeviceToDevice);
+        if (e != cudaSuccess) { free_pool(fresh); return fail_cuda(h, e, "growing the workflow arrays"); }
+        free_pool(h->wf_allocs);
+        h->wf_allocs = fresh;
+        h->g_H = H; h->d_elapsed = el; h->capW = cap;
+        for (auto& p : h->parts) p.f.H = H;
+    }
+    std::vector<float> el(n_new_workflows, 0.0f);
+    if (new_elapsed_s) el.assign(new_elapsed_s, new_elapsed_s + n_new_workflows);
+    HX_TRY(cudaMemsetAsync(h->g_H + W0, 0, (size_t)n_new_workflows * sizeof(float), s), "clearing the new horizons");
+    HX_TRY(cudaMemcpyAsync(h->d_elapsed + W0, el.data(), el.size() * sizeof(float), cudaMemcpyHostToDevice, s), "copy elapsed");
+    h->h_elapsed.insert(h->h_elapsed.end(), el.begin(), el.end());
+    h->h_wf_part.resize(W1, ~0u);                          // no part owns them until their first nodes arrive
+    h->h_wf_local.resize(W1, 0u);
+    h->h_base_wns.resize((size_t)W1 + 1, h->h_base_wns.back());   // no node of the upload belongs to them
+    h->W = W1;
+    h->fwd_built = false; h->est_ready = false;            // the transposed forest is rebuilt at the next forward pass
     return HX_OK;
 }
 

@@ -206,3 +206,103 @@ def test_rejected_appends_change_nothing(hx, oracle):
     after = gc.dag_results()
     assert all(np.array_equal(x, y) for x, y in zip(before, after))
     gc.close()
+
+
+@pytest.mark.parametrize("name, scale, base_frac, rounds", [("tiny", 1.0, 0.5, 3), ("medium", 1.0, 0.4, 5),
+                                                            ("large", 1 / 16, 0.7, 4)])
+def test_arriving_workflows_equal_a_fresh_upload(hx, oracle, name, scale, base_frac, rounds):
+    """Workflows that arrive after the upload (Section 5.2, first trigger of the scheduling loop): only a share
+    of the generated workflows is uploaded; the others arrive in rounds, each round registering its workflows,
+    handing in their source calls and, interleaved, later calls of workflows that arrived earlier plus a few
+    cost updates.  After every round cp, tail and H equal the oracle's pass over the forest as it stands."""
+    wl = make_workload(name, scale=scale)
+    rng = np.random.default_rng(41)
+    N, W = wl.n_nodes, wl.n_workflows
+    cost = rng.lognormal(0, 1, N).astype(np.float32)
+    src = np.repeat(np.arange(N, dtype=np.int64), np.diff(wl.row_ptr.astype(np.int64)))
+    dst = wl.col.astype(np.int64)
+    # arrival round of every workflow (0 = uploaded); workflows are renumbered in arrival order
+    w_round = np.where(rng.random(W) < base_frac, 0, rng.integers(1, rounds + 1, W))
+    w_round[0] = 0
+    w_order = np.argsort(w_round, kind="stable"); w_new = np.empty(W, np.int64); w_new[w_order] = np.arange(W)
+    indeg = np.bincount(dst, minlength=N)
+    # a node is revealed with its workflow if it is a source, else one or two rounds later
+    n_round = w_round[wl.node_wf] + np.where(indeg == 0, 0, rng.integers(0, 3, N))
+    n_round = np.minimum(n_round, rounds)
+    n_round[(w_round[wl.node_wf] == 0) & (rng.random(N) < 0.5)] = 0
+    n_order = np.argsort(n_round, kind="stable"); n_new = np.empty(N, np.int64); n_new[n_order] = np.arange(N)
+    cost_r, wf_r = cost[n_order], w_new[wl.node_wf[n_order]].astype(np.uint32)
+    s, d = n_new[src], n_new[dst]
+    e_round = np.maximum(n_round[src], n_round[dst])
+    n_at = [int(np.count_nonzero(n_round <= r)) for r in range(rounds + 1)]
+    w_at = [int(np.count_nonzero(w_round <= r)) for r in range(rounds + 1)]
+    elapsed = rng.uniform(0, 2, W).astype(np.float32)
+
+    def want(r, c):
+        m = e_round <= r
+        row, col = _csr(n_at[r], s[m], d[m])
+        return oracle.longest_path(row, col, c[:n_at[r]], wf_r[:n_at[r]], w_at[r]), row, col
+
+    gc = hh.gpu_cluster(wl)
+    m0 = e_round == 0
+    row, col = _csr(n_at[0], s[m0], d[m0])
+    gc.dag_upload(row, col, cost_r[:n_at[0]], wf_r[:n_at[0]], elapsed[:w_at[0]])
+    gc.critical_path()
+    cost_now = cost_r.copy()
+    for r in range(1, rounds + 1):
+        gc.dag_append_workflows(elapsed[w_at[r - 1]:w_at[r]])
+        cp, tail, H = gc.dag_results()
+        assert H.shape[0] == w_at[r] and np.all(H[w_at[r - 1]:] == 0)         # arrived, nothing revealed yet
+        m = e_round == r
+        gc.dag_append(cost_now[n_at[r - 1]:n_at[r]], wf_r[n_at[r - 1]:n_at[r]], s[m], d[m])
+        ids = rng.integers(0, n_at[r], max(1, n_at[r] // 100)).astype(np.uint32)
+        new = (cost_now[ids] * 1.25).astype(np.float32)
+        gc.update_costs(ids, new)
+        for i, v in zip(ids, new):
+            cost_now[i] = v
+        w, row, col = want(r, cost_now)
+        cp, tail, H = gc.dag_results()
+        assert np.array_equal(cp, w.cp) and np.array_equal(tail, w.tail) and np.array_equal(H, w.H), "round %d" % r
+    # the grown forest behaves like an uploaded one: elapsed times of the grown count, forward pass, full pass, scoring
+    gc.update_elapsed(elapsed[:w_at[rounds]])
+    gc.earliest_start()
+    est, eft = gc.earliest_results()
+    w_est, w_eft = oracle.earliest_start(row, col, cost_now)
+    assert np.array_equal(est, w_est) and np.array_equal(eft, w_eft)
+    gc.critical_path()
+    cp, tail, H = gc.dag_results()
+    assert np.array_equal(cp, w.cp) and np.array_equal(H, w.H)
+    oc = hh.oracle_cluster(wl)
+    calls = wl.node_calls[n_order][-min(N, 300):].copy()
+    calls["node"] = np.arange(N - len(calls), N)
+    gc.set_options(score_mode=hx.HX_MODE_RATIO)
+    a, c = gc.schedule_batch(calls)
+    oa, ocst, _ = oracle.schedule(oc, calls, mode=ho.MODE_RATIO, dag=w, node_wf=wf_r, elapsed=elapsed[:w_at[rounds]])
+    assert np.array_equal(a.cpu().numpy(), oa) and np.array_equal(c.cpu().numpy(), ocst)
+    assert gc.status() == 0
+    gc.close()
+
+
+def test_arriving_workflows_beyond_the_reserve_and_bad_arguments(hx, oracle):
+    wl = make_workload("tiny")
+    gc = hh.gpu_cluster(wl)
+    with pytest.raises(hx.HxError) as e:
+        gc.dag_append_workflows([0.0])
+    assert e.value.code == -4                                 # nothing uploaded yet
+    cost = np.ones(wl.n_nodes, np.float32)
+    gc.dag_upload(wl.row_ptr, wl.col, cost, wl.node_wf, wl.elapsed)
+    gc.critical_path()
+    with pytest.raises(hx.HxError):
+        gc.dag_append_workflows([-1.0])
+    with pytest.raises(hx.HxError):                           # a node of a workflow that has not arrived
+        gc.dag_append([1.0], [wl.n_workflows], [], [])
+    W0, N0 = wl.n_workflows, wl.n_nodes
+    k = 6000                                                  # more than the reserve of 4,096: the arrays move
+    gc.dag_append_workflows(np.zeros(k, np.float32))
+    new_cost = np.arange(1, k + 1, dtype=np.float32)
+    gc.dag_append(new_cost, np.arange(W0, W0 + k, dtype=np.uint32), [], [])
+    cp, tail, H = gc.dag_results()
+    base = oracle.longest_path(wl.row_ptr, wl.col, cost, wl.node_wf, W0)
+    assert np.array_equal(H[:W0], base.H) and np.array_equal(H[W0:], new_cost) and np.array_equal(cp[N0:], new_cost)
+    assert gc.status() == 0
+    gc.close()
