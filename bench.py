@@ -88,6 +88,31 @@ class ClockSampler:
 # CPU oracle legs (reference arm and cpu_baseline)
 # ----------------------------------------------------------------------------------------------
 
+def pin_to_one_core():
+    """The oracle is single-threaded: keep it on one core of the host for the whole measurement.  Returns the
+    core, or None where the platform has no affinity call."""
+    try:
+        core = sorted(os.sched_getaffinity(0))[0]
+        os.sched_setaffinity(0, {core})
+        return core
+    except (AttributeError, OSError):
+        return None
+
+
+def unpin(cores):
+    try:
+        os.sched_setaffinity(0, cores)
+    except (AttributeError, OSError):
+        pass
+
+
+def host_cores():
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count()
+
+
 def oracle_chunks(wl, n_chunks, with_dag):
     """Runs the oracle, as it stands, on the first n_chunks scheduler invocations of the
     workload; returns (candidates, seconds)."""
@@ -125,6 +150,8 @@ def run_reference(args):
         return
     wl = make_workload("sweep")
     n_chunks = 1                      # bounded sample per step: 1 of the 16 invocations
+    n_host = host_cores()
+    core = pin_to_one_core()
     times = []
     for i in range(args.warmup + args.steps):
         cand, dt = oracle_chunks(wl, n_chunks, with_dag=False)
@@ -140,7 +167,8 @@ def run_reference(args):
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": "sweep: 128x128 instances, 262,144 ready calls in chunks of 16,384, top-4 + commit",
                    "sample": sample},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "host_cores": n_host, "pinned_to_core": core,
+                         "kind": "oracle", "sample": sample, "omits": "horizons (the scores use elapsed = 0, tail = 0, H = 1)"},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0}))
 
@@ -283,6 +311,7 @@ def run_cuda(args):
     launches = launches_per_step * args.steps
     step_ms = np.array([a.elapsed_time(b) for a, b in ev])
     status = gc.status()
+    placed = (out_assign >= 0).view(n_chunks, chunk).sum(dim=1).cpu().numpy() / float(chunk)
     replay_ok = None
     if graph is not None:                               # a replayed step leaves the same placements as one enqueued call by call
         got_a, got_c = out_assign.clone(), out_cost.clone()
@@ -343,7 +372,16 @@ def run_cuda(args):
     lane_rate = chunk * P * D / (score_avg_ms * 1e-3)              # candidates per second of one launch
     peak = 2.0 * n_sm * FP32_LANES_PER_SM * sm_max_mhz * 1e6 / 1e12
     achieved = 2.0 * ALGO_LANE_OPS_PER_CANDIDATE * lane_rate / 1e12
+    rates, rate_ms = hx.hx_measure_fp32_rates(h, sptr)             # register-only loops, each longer than a millisecond
+    peak_measured = 2.0 * rates["fma"] / 1e12                      # every lane-instruction counted as 2 flop, like `peak`
+    loop_ceiling = rates["mix"]                                    # the loop issues one instruction of the mix per candidate and lane
     roofline = {"bound": "alu", "kernel": "hx_score_kernel", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                "peak_measured": peak_measured, "frac_of_peak_measured": achieved / peak_measured,
+                "loop_ceiling_measured": loop_ceiling, "loop_ceiling_unit": "candidates/s",
+                "frac_of_loop_ceiling": lane_rate / loop_ceiling,
+                "lane_instr_per_s_measured": rates, "micro_kernel_ms": rate_ms,
+                "measured_with": "hx_measure_fp32_rates: fma.rn.f32, fma.rn.f32x2, three-input min.f32 and their one-to-one "
+                                 "mix in registers, CUDA events, during the clock sampling of this run",
                 "frac": achieved / peak, "traffic": SCORE_DRAM_BYTES_PER_LAUNCH,
                 "peak_source": "%d SMs x %d FP32 lanes x %.0f MHz x 2 flop (%s sm_max_mhz)" % (
                     n_sm, FP32_LANES_PER_SM, sm_max_mhz, which),
@@ -352,18 +390,23 @@ def run_cuda(args):
                 "frac_executed": 2.0 * EXEC_LANE_OPS_PER_CANDIDATE * lane_rate / 1e12 / peak,
                 "lane_ops_executed_per_candidate": EXEC_LANE_OPS_PER_CANDIDATE,
                 "candidates_per_s_kernel": lane_rate,
-                "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch on this "
-                                  "workload (profiles/hx_score_kernel_sweep_chunk.md)",
+                "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum, one launch, same workload",
                 "time_share": {k: v[0] / max(inst_ms, 1e-9) for k, v in kt.items()},
                 "timed_with": "%d steps enqueued call by call with event pairs around every kernel family" % n_inst}
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
         n_b = 8
+        n_host, all_cores = host_cores(), (os.sched_getaffinity(0) if hasattr(os, "sched_getaffinity") else None)
+        core = pin_to_one_core()
         cand, dt = oracle_chunks(make_workload("sweep"), n_b, with_dag=False)
-        cpu = {"value": cand / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+        if all_cores is not None:
+            unpin(all_cores)
+        cpu = {"value": cand / dt, "unit": UNIT, "cores": 1, "host_cores": n_host, "pinned_to_core": core, "kind": "oracle",
                "sample": "%d of 16 invocations (%d calls x 16384 pairs, top-4 + conflict pass), %.1f s" % (
-                   n_b, n_b * chunk, dt)}
+                   n_b, n_b * chunk, dt),
+               "omits": "horizons (the scores use elapsed = 0, tail = 0, H = 1; the oracle's pass over the whole "
+                        "forest is timed in horizon_refinement.oracle_full_pass_ms_1_core)"}
 
     # side legs (oracle sample, greedy planner) are skipped together, e.g. under a profiler
     greedy = greedy_leg(with_cpu=True) if world == 1 and not args.no_cpu_baseline else None
@@ -377,7 +420,12 @@ def run_cuda(args):
                                "capacity-conflict pass with commit, horizons over %d nodes / %d workflows" % (
                                    P, D, n_calls, n_chunks, chunk, wl.topk, wl.n_nodes, wl.n_workflows),
                    "candidates_per_step": cand_per_step, "l2": "flushed between timed steps (256 MB write)",
-                   "seed": wl.seed, "score_mode": "ratio"},
+                   "seed": wl.seed, "score_mode": "ratio",
+                   "forest": "%d workflows of 8-24 nodes (chains, fan-out/join stages, random layered DAGs), %d nodes, "
+                             "%d edges" % (wl.n_workflows, wl.n_nodes, wl.n_edges)},
+        "placed_fraction": {"per_invocation": [float(x) for x in placed], "mean": float(placed.mean()),
+                            "what": "share of the 16,384 calls of each scheduler invocation that obtained a pair; the others "
+                                    "found none of their four candidate decode instances with room"},
         "schedule_latency": {"batch_calls": chunk, "p50_us": float(np.percentile(chunk_us, 50)),
                              "p95_us": float(np.percentile(chunk_us, 95)),
                              "what": "load refresh + hx_schedule_batch (scoring, top-4, conflict pass, commit) per "

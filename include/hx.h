@@ -540,6 +540,16 @@ int hx_get_status(hx_cluster* h, int* status, void* stream);
 int hx_enable_kernel_timing(hx_cluster* h, int enable);
 int hx_read_kernel_timing(hx_cluster* h, float* ms, int* launches);
 
+/* Measurement aid for the roofline of the scoring kernel, whose bound is the issue
+ * rate of the FP32 pipes (one fused multiply-add and one minimum per candidate,
+ * Algorithm 1, inner loop): runs four register-only loops of at least a
+ * millisecond each on `stream` and reports, in lane-instructions per second (32
+ * per warp instruction), what the device sustains for [0] fma.rn.f32, [1]
+ * fma.rn.f32x2, [2] three-input min.f32, [3] the one-to-one mix of [1] and [2]
+ * that the candidate loop issues; ms[4] receives the device time of each timed
+ * launch.  Synchronises.  Errors: HX_ERR_INVALID_ARG for NULL arguments. */
+int hx_measure_fp32_rates(hx_cluster* h, double* lane_instr_per_s, float* ms, void* stream);
+
 /* Message of the last error on this handle ("" if none); with h = NULL, the
  * message of the last failed hx_cluster_create of the calling thread. */
 const char* hx_last_error(const hx_cluster* h);

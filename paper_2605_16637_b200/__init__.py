@@ -12,7 +12,7 @@ from .api import (CALL_DTYPE, INSTANCE_DTYPE, HX_FLAG_NO_DAG, HX_FLAG_NO_TAIL, H
                   hx_read_kernel_timing, hx_dag_upload, hx_dag_update_costs, hx_dag_update_elapsed, hx_get_dag_results,
                   hx_dag_append, hx_earliest_start, hx_get_earliest_results,
                   hx_get_status, hx_get_topk, hx_last_error, hx_launch_count, hx_schedule_batch,
-                  hx_schedule_batch_host, hx_schedule_batch_host_async, hx_schedule_sweep_host, hx_set_attention_flops, hx_schedule_batch_static, hx_schedule_greedy, hx_schedule_greedy_plan, hx_replay, hx_replay_lifecycle, hx_dag_append_workflows, hx_estimate_calls,
+                  hx_schedule_batch_host, hx_schedule_batch_host_async, hx_schedule_sweep_host, hx_set_attention_flops, hx_schedule_batch_static, hx_schedule_greedy, hx_schedule_greedy_plan, hx_replay, hx_replay_lifecycle, hx_measure_fp32_rates, hx_dag_append_workflows, hx_estimate_calls,
                   hx_decode_set_running, hx_schedule_decode, KV_INTERVAL_DTYPE, hx_set_options, lib_path)
 
 __all__ = [n for n in dir() if n.startswith(("hx_", "HX_", "Hx")) or n in

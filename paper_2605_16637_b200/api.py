@@ -75,6 +75,7 @@ def _load():
         "hx_schedule_decode": [vp, vp, vp, vp, ci, vp, vp, vp, vp, vp],
         "hx_get_topk": [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp)],
         "hx_get_status": [vp, C.POINTER(ci), vp],
+        "hx_measure_fp32_rates": [vp, vp, vp, vp],
         "hx_enable_kernel_timing": [vp, ci],
         "hx_read_kernel_timing": [vp, C.POINTER(C.c_float), C.POINTER(ci)],
     }
@@ -329,6 +330,13 @@ def hx_get_status(h, stream=0):
     s = C.c_int(0)
     _check(_lib.hx_get_status(h, C.byref(s), stream), h)
     return s.value
+
+
+def hx_measure_fp32_rates(h, stream=0):
+    """Lane-instructions per second of fma.f32, fma.f32x2, three-input min and their mix; ms of each launch."""
+    rates, ms = np.zeros(4, np.float64), np.zeros(4, np.float32)
+    _check(_lib.hx_measure_fp32_rates(h, _p(rates), _p(ms), stream), h)
+    return dict(zip(("fma", "fma2", "min3", "mix"), (float(x) for x in rates))), ms.tolist()
 
 
 def hx_enable_kernel_timing(h, enable=True):

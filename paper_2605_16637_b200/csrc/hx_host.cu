@@ -520,8 +520,8 @@ int hx_cluster_create(const hx_gpu_type* gpu_types, int n_types, const hx_instan
     up(dev_upload(h->allocs, &d_phi, phi));
     up(dev_upload(h->allocs, &d_omega, omega)); up(dev_upload(h->allocs, &d_kappa, kappa));
     up(dev_upload(h->allocs, &d_typeP, typeP)); up(dev_upload(h->allocs, &d_typeD, typeD));
-    up(dev_alloc(h->allocs, &h->status, 1));
-    if (ok) up(cudaMemset(h->status, 0, sizeof(int)));
+    up(dev_alloc(h->allocs, &h->status, 2));                // status word, and a sink for the issue-rate kernels
+    if (ok) up(cudaMemset(h->status, 0, 2 * sizeof(int)));
     if (!ok) return bail(fail_cuda(h, first, "uploading cluster tables"));
     h->tab = HxTables{n_types, P, D, n_models, h->Ppad, d_invF, d_invB, d_typeP, d_typeD, d_qP, d_qD,
                       d_capD, d_freeD, d_invLT, d_invLTt, dpadT, d_phi, d_omega, d_kappa};
@@ -1472,6 +1472,15 @@ int hx_get_status(hx_cluster* h, int* status, void* stream) {
     HX_TRY(cudaMemcpyAsync(status, h->status, sizeof(int), cudaMemcpyDeviceToHost, s), "read status");
     HX_TRY(cudaMemsetAsync(h->status, 0, sizeof(int), s), "clear status");      // read and clear: the next read covers later work only
     HX_TRY(cudaStreamSynchronize(s), "cudaStreamSynchronize");
+    return HX_OK;
+}
+
+int hx_measure_fp32_rates(hx_cluster* h, double* lane_instr_per_s, float* ms, void* stream) {
+    if (!h || !lane_instr_per_s || !ms) return HX_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    // the status word doubles as the never-written sink of the loops (they store only if a sum hits one exact value)
+    HX_TRY(hx_run_micro(h->n_sm, reinterpret_cast<float*>(h->status + 1), static_cast<cudaStream_t>(stream), lane_instr_per_s, ms,
+                        &h->launches), "issue-rate kernels");
     return HX_OK;
 }
 

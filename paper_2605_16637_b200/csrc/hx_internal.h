@@ -138,6 +138,10 @@ cudaError_t hx_launch_estimate(const HxConstTables& ct, int G, int M, const hx_c
                                float* tpre, float* tdec, float* kvB, float* m, int* status, cudaStream_t stream,
                                long long* launches);
 
+// Issue rates of the instruction kinds of the candidate loop: lane-instructions per second of fma.rn.f32,
+// fma.rn.f32x2, three-input min.f32 and their one-to-one mix; device time of each timed launch in ms.
+cudaError_t hx_run_micro(int n_sm, float* sink, cudaStream_t stream, double* lane_instr_per_s, float* ms, long long* launches);
+
 size_t hx_greedy_smem_bytes(const HxTables& t, int n_calls);
 cudaError_t hx_launch_greedy(const HxTables& t, const HxConstTables& ct, const HxDagView& dag,
                              const hx_call* calls, int n_calls, int flags, int commit,
