@@ -319,7 +319,7 @@ int hx_schedule_sweep_host(hx_cluster* h, const hx_call* calls, int n_calls, int
  * synchronisation of an allocation is a stall; code running where the CUDA
  * allocator may not be entered at all.  This variant computes the same
  * results but keeps the top-K lists, the visiting order and the bookkeeping of
- * the capacity pass in one fixed array of about 1.9 MB that is part of the
+ * the capacity pass in one fixed array of about 2.0 MB that is part of the
  * library image; every device that loads the library holds that array until
  * the process exits.  It calls no allocating routine.
  *   Limits: n_calls <= HX_STATIC_MAX_CALLS when topk > 0, topk <=
@@ -329,8 +329,12 @@ int hx_schedule_sweep_host(hx_cluster* h, const hx_call* calls, int n_calls, int
  * error codes are those of hx_schedule_batch; hx_get_topk does not see this
  * call's lists.
  *   Set-up: the first call on a device looks up the array's device address
- * (once per device, under a lock).  Make that first call before starting any
- * stream capture.
+ * (once per device, under a lock); the first call with a given option set also
+ * makes the CUDA runtime load the kernels it launches and raise their
+ * shared-memory limit, which may allocate inside the driver.  Make one warm-up
+ * call per option set before the phase in which nothing may allocate, and
+ * before starting any stream capture.  (With kernel timing enabled the call
+ * also creates CUDA events the first few times; leave timing off there.)
  *   Sharing: all handles and all calls on a device use the same array, which
  * keeps whatever the previous call left; every call rewrites all it reads, so
  * nothing needs clearing, but two calls that overlap on the GPU (different

@@ -1287,9 +1287,14 @@ int hx_schedule_batch_static(hx_cluster* h, const hx_call* calls, int n_calls, i
     if (!(o.flags & HX_FLAG_NO_DAG))
         dag = HxDagView{h->d_node_wf, h->g_tail, h->g_H, h->d_elapsed, h->N, h->W};
     ScoreLaunch sl{calls, n_calls, out_assign, out_cost, o.score_mode, o.flags, o.topk, o.alpha};
-    HX_TRY(hx_launch_score(h->tab, h->ctab, dag, b, sl, h->n_sm, h->max_smem, h->status, s, &h->launches), "scoring kernel");
-    if (o.topk > 0)
+    {
+        SpanGuard span(h, 0, s);
+        HX_TRY(hx_launch_score(h->tab, h->ctab, dag, b, sl, h->n_sm, h->max_smem, h->status, s, &h->launches), "scoring kernel");
+    }
+    if (o.topk > 0) {
+        SpanGuard span(h, 1, s);
         HX_TRY(hx_launch_conflict(h->tab, b, n_calls, o.commit, out_assign, h->status, s, &h->launches), "conflict pass");
+    }
     return HX_OK;
 }
 

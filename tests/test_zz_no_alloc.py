@@ -68,6 +68,38 @@ def test_static_entry_point_matches_regular_one_twice_in_a_row(hx):
     gc.close()
 
 
+def test_static_entry_point_leaves_device_memory_as_it_is(hx):
+    """A handle that has never run the regular entry point (so none of its buffers exist): after the one documented
+    warm-up call, further calls through the allocation-free entry point leave the amount of free device memory
+    exactly as it was, and match the regular entry point run afterwards on the same inputs."""
+    import torch
+    wl = make_workload("sweep", scale=1 / 32)
+    gc = hh.gpu_cluster(wl)
+    gc.set_options(score_mode=hx.HX_MODE_COMPLETION, topk=4, commit=1, flags=hx.HX_FLAG_NO_DAG)
+    loads = (wl.load_s[:wl.P], wl.load_s[wl.P:], wl.kv_free[wl.P:])
+    n = len(wl.calls)
+    dev = torch.from_numpy(wl.calls.view(np.uint8).copy()).cuda()
+    a = torch.empty(n, dtype=torch.int32, device="cuda")
+    c = torch.empty(n, dtype=torch.float32, device="cuda")
+    sp = torch.cuda.current_stream().cuda_stream
+    gc.update_loads(*loads)
+    hx.hx_schedule_batch_static(gc.h, dev.data_ptr(), n, a.data_ptr(), c.data_ptr(), sp)     # warm-up: loads the kernels
+    torch.cuda.synchronize()
+    before = torch.cuda.mem_get_info()[0]
+    for rep in range(3):
+        gc.update_loads(*loads)
+        hx.hx_schedule_batch_static(gc.h, dev.data_ptr(), n, a.data_ptr(), c.data_ptr(), sp)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == before, "the allocation-free entry point changed the free device memory"
+    sa, sc = a.cpu().numpy(), c.cpu().numpy()
+    sq, _, sf = gc.read_loads()
+    ra, rc, rq, rf = _run(hx, gc, hx.hx_schedule_batch, dev, n, loads)
+    assert np.array_equal(sa, ra) and np.array_equal(sf, rf) and np.array_equal(sq, rq)
+    hh.assert_costs_close(sc, rc, "scores")
+    assert gc.status() == 0
+    gc.close()
+
+
 def test_static_entry_point_rejects_sizes_beyond_its_array(hx):
     import torch
     wl = make_workload("sweep", scale=1 / 15)             # a few calls more than the maximum
