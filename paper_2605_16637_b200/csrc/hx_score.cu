@@ -41,6 +41,7 @@ struct ScoreParams {
     int FS;              // row stride of the per-call finish times (Dpad + 4)
     int AS, LS;          // strides, in 16-byte units, between consecutive p / 4 of the A and link tiles
     int offA, offF, offCall, offInst;   // byte offsets into dynamic shared memory (LT at 0)
+    int offItem;         // selected (call, slot) entries waiting for their prefill index, 0 = recovery inside the selection loop
     int resident;        // whole link table and the A tile stay in shared memory for the index recovery
 };
 
@@ -226,6 +227,9 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
     float* qDs = reinterpret_cast<float*>(typePs + Ppad);         // [Dpad]
     float* capDs = qDs + Dpad;                                    // [Dpad]
     int* typeDs = reinterpret_cast<int*>(capDs + Dpad);           // [Dpad]
+    int* itemD = reinterpret_cast<int*>(smem + prm.offItem);      // [TCB * K] decode column of the entry, -1 = unused slot
+    float* itemV = reinterpret_cast<float*>(itemD + TCB * HX_MAX_TOPK);   // [TCB * K] its finish time
+    const bool deferred = prm.offItem != 0;                       // top-K lists with the operands resident: see below
 
     // visiting order of the capacity pass: this kernel clears the bin counters and leaves the smallest and
     // the largest finite priority key of every block's calls behind (no state survives from earlier batches)
@@ -519,7 +523,7 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
                 if (nsel > 0) v0 = sel_cost[0];
 #pragma unroll
                 for (int k0 = 0; k0 < HX_MAX_TOPK; k0 += 4) {
-                    if (k0 < nsel) {                          // uniform inside the group
+                    if (k0 < nsel && !deferred) {             // uniform inside the group
                         int pk[4];
                         recover(Four{}, &sel_d[k0], &sel_cost[k0], min(4, nsel - k0), pk);
 #pragma unroll
@@ -568,14 +572,60 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
 #pragma unroll
                     for (int k = 0; k < HX_MAX_TOPK; ++k) {
                         if (k >= K) break;
-                        const int pr = bad ? -1 : sel_pair[k];
-                        prm.tk.pair[(size_t)gc * K + k] = pr;
+                        const bool used = !bad && (deferred ? sel_cost[k] < HX_INF : sel_pair[k] >= 0);
+                        if (deferred) {                       // pair and prefill time follow once the prefill index is known
+                            itemD[c * K + k] = used ? sel_d[k] : -1;
+                            itemV[c * K + k] = sel_cost[k];
+                        } else {
+                            prm.tk.pair[(size_t)gc * K + k] = used ? sel_pair[k] : -1;
+                            prm.tk.tpre[(size_t)gc * K + k] = sel_tpre[k];
+                        }
                         prm.tk.cost[(size_t)gc * K + k] = bad ? HX_INF : sel_cost[k];
-                        prm.tk.tpre[(size_t)gc * K + k] = sel_tpre[k];
-                        dw[k >> 1] = (dw[k >> 1] & ~(0xFFFFu << ((k & 1) * 16))) | ((pr >= 0 ? (unsigned)sel_d[k] : 0xFFFFu) << ((k & 1) * 16));
+                        dw[k >> 1] = (dw[k >> 1] & ~(0xFFFFu << ((k & 1) * 16))) | ((used ? (unsigned)sel_d[k] : 0xFFFFu) << ((k & 1) * 16));
                     }
                     prm.tk.dsel[gc] = make_uint4(dw[0], dw[1], dw[2], dw[3]);
                 }
+            }
+        }
+        if (deferred) {
+            // Prefill index of every selected entry, one thread per entry (call c, column d, finish time v): the thread
+            // walks the call's prefill-finish row against the link-table row of d in 16-byte units (one packed FMA pair,
+            // two minima and a compare per unit; exact evaluation only where the ready time can reach v - Dd within the
+            // rounding slack of the last addition) and stops at the first unit that holds a match.
+            __syncthreads();
+            const int nItems = nvalid * K, nq = Ppad >> 2;
+            for (int item = tid; item < nItems; item += nthr) {
+                const int d = itemD[item];
+                const int c = item / K;
+                int best = HX_NONE;
+                if (d >= 0) {
+                    const float v = itemV[item], kvB = kvBs[c], qd = qDs[d];
+                    const float Dd = (mtoks[c] <= capDs[d]) ? tdecs[typeDs[d] * TCB + c] : HX_INF;
+                    const float thr = __fadd_rn(__fsub_rn(v, Dd), __fmul_rn(v, 4.76837158203125e-07f));
+                    const u64 kk2 = pack2(kvB, kvB);
+                    const ulonglong2* ap = reinterpret_cast<const ulonglong2*>(As) + c;
+                    const ulonglong2* lp = reinterpret_cast<const ulonglong2*>(LTs) + d;
+                    for (int q0 = 0; q0 < nq && best == HX_NONE; q0 += 4) {
+#pragma unroll
+                        for (int u4 = 3; u4 >= 0; --u4) {
+                            const int q = q0 + u4;
+                            if (q >= nq) continue;
+                            const ulonglong2 a = ap[(size_t)q * AS], l = lp[(size_t)q * LS];
+                            float r[4];
+                            unpack2(fma2(kk2, l.x, a.x), r[0], r[1]);
+                            unpack2(fma2(kk2, l.y, a.y), r[2], r[3]);
+                            if (fminf(min3(r[0], r[1], r[2]), r[3]) <= thr) {
+#pragma unroll
+                                for (int u = 3; u >= 0; --u)
+                                    if (__fadd_rn(fmaxf(r[u], qd), Dd) == v) best = 4 * q + u;
+                            }
+                        }
+                    }
+                }
+                const size_t o = (size_t)(c0 + c) * K + (item - c * K);
+                const bool ok = best != HX_NONE;
+                prm.tk.pair[o] = ok ? best * D + d : -1;
+                prm.tk.tpre[o] = ok ? tpres[typePs[best] * TCB + c] : 0.f;
             }
         }
         __syncthreads();
@@ -671,7 +721,10 @@ cudaError_t hx_launch_score(const HxTables& t, const HxConstTables& ct, const Hx
     if (prm.resident) { prm.offF = prm.offA + (int)aB; prm.offCall = prm.offF + round_up((int)f_rows, 16); }
     else { prm.offF = prm.offA; prm.offCall = prm.offA + (int)(aB > f_rows ? aB : round_up((int)f_rows, 16)); }
     prm.offInst = prm.offCall + (int)callB;
-    const size_t smem = prm.offInst + instB;
+    size_t smem = prm.offInst + instB;
+    prm.offItem = 0;
+    const size_t itemB = (size_t)prm.TCB * HX_MAX_TOPK * 8;
+    if (prm.resident && s.K > 0 && smem + itemB <= max_smem) { prm.offItem = (int)smem; smem += itemB; }
     if (smem > max_smem) return cudaErrorInvalidConfiguration;
     const int threads = 32 * prm.WDn * prm.WCn;
     const int grid = prm.nTiles < n_sm ? prm.nTiles : n_sm;
