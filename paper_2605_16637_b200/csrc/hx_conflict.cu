@@ -86,8 +86,10 @@ __device__ __forceinline__ unsigned bin_of(unsigned key, unsigned lo, unsigned s
 __global__ void __launch_bounds__(kOrdThreads) hx_order_hist_kernel(HxTopkBufs tk, int n) {
     __shared__ unsigned lohi[2];
     const int tid = threadIdx.x;
+    hx_release_dependents();
     if (tid == 0) { lohi[0] = 0xFFFFFFFFu; lohi[1] = 0u; }
     __syncthreads();
+    hx_wait_for_primary();                                        // the scoring kernel's key ranges, priorities and cleared counters
     unsigned lo = 0xFFFFFFFFu, hi = 0u;
     for (int b = tid; b < HX_ORDER_MAXBLK; b += kOrdThreads) {
         lo = min(lo, __ldcg(tk.blk_lohi + b)); hi = max(hi, __ldcg(tk.blk_lohi + HX_ORDER_MAXBLK + b));
@@ -111,6 +113,8 @@ __global__ void __launch_bounds__(kOrdThreads) hx_order_hist_kernel(HxTopkBufs t
 __global__ void __launch_bounds__(kOrdThreads) hx_order_scatter_kernel(HxTopkBufs tk, int n) {
     __shared__ unsigned hist[kBins], base[kBins + 1], tmp[33];
     const int tid = threadIdx.x;
+    hx_release_dependents();
+    hx_wait_for_primary();                                        // the complete bin counters
     for (int i = tid; i < kBins; i += kOrdThreads) hist[i] = __ldcg(tk.ghist + i);
     __syncthreads();
     block_exclusive_scan(hist, kBins, base, tmp);
@@ -125,13 +129,15 @@ __global__ void __launch_bounds__(kOrdThreads) hx_order_scatter_kernel(HxTopkBuf
 // 1c. Rank inside the bins and gather the per-call data in visiting order.
 __global__ void hx_order_rank_kernel(HxTopkBufs tk, int n, unsigned D) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    hx_release_dependents();
+    hx_wait_for_primary();                                        // every key is in its bin
     if (i >= n) return;
     const unsigned lo = tk.obase[kBins + 1], shift = tk.obase[kBins + 2];
     const u64 key = tk.okey[i];
     const unsigned bin = bin_of((unsigned)(key >> 32), lo, shift);
     const unsigned b0 = tk.obase[bin], b1 = tk.obase[bin + 1];
     unsigned rank = b0;
-    for (unsigned j = b0; j < b1; ++j) rank += __ldg(tk.okey + j) < key;
+    for (unsigned j = b0; j < b1; ++j) rank += __ldcg(tk.okey + j) < key;
     const unsigned c = (unsigned)key;
     tk.ocall[rank] = c;
     tk.om[rank] = __float2int_ru(tk.mtok[c]);                   // token counts are whole numbers below 2^24
@@ -270,6 +276,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) hx_conflict_kernel(HxTopkBufs
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const unsigned lt = (1u << lane) - 1u;
     for (int d = tid; d <= D; d += kPassThreads) free_s[d] = d < D ? __float2int_rd(t.freeD[d]) : -1;
+    hx_wait_for_primary();                                      // the visiting order
     __syncthreads();
     auto narrow = [&](const uint4& r) {                         // the slots this instantiation examines
         Row out;
@@ -462,10 +469,12 @@ cudaError_t hx_launch_conflict(const HxTables& t, const HxTopkBufs& tk, int n_ca
     (void)status;
     const int D = t.D, P = t.P;
     const int nb = (n_calls + kOrdThreads - 1) / kOrdThreads;
-    hx_order_hist_kernel<<<nb, kOrdThreads, 0, stream>>>(tk, n_calls);
-    hx_order_scatter_kernel<<<nb, kOrdThreads, 0, stream>>>(tk, n_calls);
-    hx_order_rank_kernel<<<(n_calls + 127) / 128, 128, 0, stream>>>(tk, n_calls, (unsigned)D);
-    cudaError_t e;
+    // every kernel of the pass may become resident while the one before it drains; each waits for its
+    // predecessor before reading what that one wrote
+    cudaError_t e = hx_launch_dependent(hx_order_hist_kernel, dim3(nb), dim3(kOrdThreads), 0, stream, tk, n_calls);
+    if (e == cudaSuccess) e = hx_launch_dependent(hx_order_scatter_kernel, dim3(nb), dim3(kOrdThreads), 0, stream, tk, n_calls);
+    if (e == cudaSuccess) e = hx_launch_dependent(hx_order_rank_kernel, dim3((n_calls + 127) / 128), dim3(128), 0, stream, tk, n_calls, (unsigned)D);
+    if (e != cudaSuccess) return e;
     const int fused = P <= kTailMaxP;                               // pairs published and queues summed inside the pass
     const size_t smRing = (size_t)kRing * 24 + (size_t)(D + 1) * 4;
     const size_t smTail = fused ? (size_t)kTailLen * 10 + (size_t)(4 + kPassThreads / 32) * P * 4 : 0;
@@ -475,7 +484,8 @@ cudaError_t hx_launch_conflict(const HxTables& t, const HxTopkBufs& tk, int n_ca
     static size_t allowed_pass[4][64];
     e = hx_opt_in_smem(pass, smC, allowed_pass[tk.K <= 1 ? 0 : tk.K <= 2 ? 1 : tk.K <= 4 ? 2 : 3], 40 * 1024);
     if (e != cudaSuccess) return e;
-    pass<<<1, kPassThreads, smC, stream>>>(tk, t, n_calls, commit, fused, out_assign);
+    e = hx_launch_dependent(pass, dim3(1), dim3(kPassThreads), smC, stream, tk, t, n_calls, commit, fused, out_assign);
+    if (e != cudaSuccess) return e;
     *launches += 4;
     if (!fused) {
         hx_finish_kernel<<<(n_calls + 255) / 256, 256, 0, stream>>>(tk, D, out_assign);

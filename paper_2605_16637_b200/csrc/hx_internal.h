@@ -223,6 +223,29 @@ void hx_forest_host(const hx_cluster* h, std::vector<uint32_t>* row, std::vector
 int hx_push_scaled_models(hx_cluster* h, float up, float down);
 void hx_pop_scaled_models(hx_cluster* h);
 
+// Programmatic dependent launch: a kernel launched with hx_launch_dependent may be made resident while the
+// kernel before it on the stream is still running (that kernel calls hx_release_dependents() early); it must
+// call hx_wait_for_primary() before it touches anything the earlier kernel writes.  The wait returns once the
+// earlier grid has completed and its writes are visible; launched the ordinary way both calls do nothing.
+__device__ __forceinline__ void hx_wait_for_primary() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void hx_release_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
+template <class... KArgs, class... Args>
+inline cudaError_t hx_launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                       Args... args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    // inside a stream capture the ordinary dependency is kept: replayed graphs of this chain measured slower
+    // with programmatic edges (1.88 against 1.78 ms per sweep step), enqueued launches faster (122 against 129 us
+    // per ready batch)
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(stream, &cap) != cudaSuccess) cap = cudaStreamCaptureStatusNone;
+    cfg.attrs = &attr; cfg.numAttrs = cap == cudaStreamCaptureStatusNone ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // Opt a kernel in to `bytes` of dynamic shared memory, once per device and size: the attribute
 // call is too slow to repeat on every launch.  `allowed` is a per-kernel table of 64 entries
 // that starts at the size the kernel may use without opting in.

@@ -235,6 +235,7 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
     // the largest finite priority key of every block's calls behind (no state survives from earlier batches)
     unsigned key_lo = 0xFFFFFFFFu, key_hi = 0u;
     __shared__ unsigned key_lohi[2];
+    hx_release_dependents();                                      // the first kernel of the capacity pass may get ready behind this one
     if (prm.s.K > 0) {
         for (int i = blockIdx.x * nthr + tid; i < HX_ORDER_BINS; i += gridDim.x * nthr) prm.tk.ghist[i] = 0u;
         if (tid == 0) { key_lohi[0] = 0xFFFFFFFFu; key_lohi[1] = 0u; }
