@@ -28,7 +28,7 @@ UNIT = "candidates/s"
 FP32_LANES_PER_SM = 128
 ALGO_LANE_OPS_PER_CANDIDATE = 4      # fma, max, add, min of the per-candidate cost definition
 EXEC_LANE_OPS_PER_CANDIDATE = 2      # what the candidate loop executes: fma and min
-SCORE_DRAM_BYTES_PER_LAUNCH = 3260672   # ncu, one launch of 16,384 calls x 128 x 128 pairs with top-4 lists
+SCORE_DRAM_BYTES_PER_LAUNCH = 3262208   # ncu, one launch of 16,384 calls x 128 x 128 pairs with top-4 lists
 
 
 def _peaks():
