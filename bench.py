@@ -441,6 +441,7 @@ def run_cuda(args):
         "decode_scheduler": decode_leg() if world == 1 and not args.no_cpu_baseline else None,
         "horizon_refinement": refine_leg() if world == 1 and not args.no_cpu_baseline else None,
         "replay": replay_leg() if world == 1 and not args.no_cpu_baseline else None,
+        "batch_robustness": robustness_leg() if world == 1 and not args.no_cpu_baseline else None,
     }
     print(json.dumps(out))
     if dist is not None:
@@ -561,6 +562,42 @@ def refine_leg():
     t0 = time.perf_counter()
     orc.longest_path(wl.row_ptr, wl.col, cost, wl.node_wf, wl.n_workflows)
     out["oracle_full_pass_ms_1_core"] = 1e3 * (time.perf_counter() - t0)
+    out["device_status"] = gc.status()
+    gc.close()
+    return out
+
+
+def robustness_leg():
+    """Side measurement, outside the timed region: one ready batch of the sweep (16,384 calls, top-4, capacity pass)
+    as generated, with a tenth of the calls fitting no decode instance (priority +inf), and with a fifth of the calls
+    exact duplicates of one another (equal priorities share a bin of the visiting order and are ranked against each
+    other there).  CUDA events around hx_schedule_batch, median of 20."""
+    import torch
+    import paper_2605_16637_b200 as hx
+    from hx_synth import make_workload
+    wl = make_workload("sweep")
+    gc = hx.Cluster.from_workload(wl)
+    gc.set_options(score_mode=hx.HX_MODE_RATIO, topk=wl.topk, commit=0, flags=hx.HX_FLAG_NO_DAG)
+    rng = np.random.default_rng(8)
+    base = wl.calls[:wl.chunk].copy()
+    infeasible = base.copy(); infeasible["prompt_tokens"][rng.random(wl.chunk) < 0.1] = 2.0e6
+    dup = base.copy(); m = rng.random(wl.chunk) < 0.2
+    dup["model"][m] = 0; dup["prompt_tokens"][m] = 777; dup["output_tokens"][m] = 33
+    out = {}
+    stream = torch.cuda.current_stream()
+    for label, calls in (("as_generated", base), ("tenth_infeasible", infeasible), ("fifth_duplicates", dup)):
+        dev = torch.from_numpy(calls.view(np.uint8).reshape(-1, 16).copy()).cuda()
+        a = torch.empty(wl.chunk, dtype=torch.int32, device="cuda"); c = torch.empty(wl.chunk, dtype=torch.float32, device="cuda")
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(20)]
+        for _ in range(3):
+            hx.hx_schedule_batch(gc.h, dev.data_ptr(), wl.chunk, a.data_ptr(), c.data_ptr(), stream.cuda_stream)
+        for e0, e1 in ev:
+            e0.record(stream)
+            hx.hx_schedule_batch(gc.h, dev.data_ptr(), wl.chunk, a.data_ptr(), c.data_ptr(), stream.cuda_stream)
+            e1.record(stream)
+        torch.cuda.synchronize()
+        out[label] = {"batch_us": 1e3 * float(np.median([e0.elapsed_time(e1) for e0, e1 in ev])),
+                      "placed": int((a >= 0).sum().item())}
     out["device_status"] = gc.status()
     gc.close()
     return out

@@ -47,6 +47,7 @@ extern "C" {
 #define HX_FLAG_NO_DAG       1     /* ignore the DAG: elapsed = 0, tail = 0, H = 1 */
 #define HX_FLAG_NO_TAIL      2     /* drop the remaining-critical-path term from the score */
 #define HX_FLAG_UNLOADED     4     /* score against an idle cluster (all queue loads zero) */
+#define HX_FLAG_ONE_PASS     8     /* hx_schedule_decode only: rank the queue once instead of after every assignment */
 
 #define HX_MAX_TYPES        32     /* GPU classes */
 #define HX_MAX_MODELS       32
@@ -507,7 +508,14 @@ int hx_estimate_calls(hx_cluster* h, const hx_call* calls, int n_calls, float* o
  * out_ratio: R when taken (+inf if never).  out_order: out_order[i] = call
  * taken in iteration i, -1 after the last.  With hx_options.commit the simulated
  * intervals become the snapshot of the next call; otherwise the snapshot is
- * left as it was.  Uses HX_FLAG_NO_DAG like hx_schedule_batch.  Errors:
+ * left as it was.  Uses HX_FLAG_NO_DAG like hx_schedule_batch.
+ *   HX_FLAG_ONE_PASS selects the lightweight ordering that Section 5.4 falls back
+ * to for large or special-case queues (Section 5.3, last sentence): every call
+ * is scored once, R with Delta_D projected against the snapshot alone, the calls
+ * are visited by decreasing score (lower index among equals), and a visited call
+ * takes the instance with the earliest finish in the state that the calls
+ * before it have left.  out_ratio is then the score the call was ordered by.
+ * The other entry points ignore the flag.  Errors:
  * HX_ERR_NOT_READY without a snapshot or horizons; HX_ERR_INVALID_ARG for sizes
  * out of range; a record with an id out of range, a lock >= n_decode or a
  * ready time that is negative or not finite is left unassigned and raises

@@ -410,6 +410,63 @@ int orc_decode_greedy(const OrcCluster* cl, const OrcDag* dag, const OrcCall* ca
     return placed;
 }
 
+// One-pass ordering for the decode stage (Section 5.4: queues that are large, or
+// a special case, fall back to the lightweight ordering of Section 5.3, last
+// sentence: one pass in the order of the risk score instead of re-planning after
+// every assignment).  Reading taken here: the score is the ratio of Eq. 2 with
+// Delta_D projected against the snapshot alone, as if no other queued call were
+// there; the calls are visited once by decreasing score (lower index first among
+// equals); a visited call is projected against the state that the calls before it
+// have left and takes the instance with the earliest finish, as in the greedy
+// form.  Arguments and outputs as orc_decode_greedy; ratio[c] is the score the
+// call was ordered by.
+int orc_decode_onepass(const OrcCluster* cl, const OrcDag* dag, const OrcCall* calls, int C, int flags,
+                       const uint32_t* run_ptr, const float* run_start, const float* run_end, const float* run_tok,
+                       const int32_t* lock, const float* ready,
+                       int32_t* inst, float* start, float* ratio, int32_t* order) {
+    const int D = cl->D;
+    std::vector<StepFn> fn(D);
+    for (int d = 0; d < D; ++d) {
+        fn[d].t.assign(1, 0.0f); fn[d].u.assign(1, 0.0f);
+        for (uint32_t i = run_ptr[d]; i < run_ptr[d + 1]; ++i)
+            add_interval(fn[d], run_start ? run_start[i] : 0.0f, run_end[i], run_tok[i]);
+    }
+    std::vector<Terms> terms(C);
+    for (int c = 0; c < C; ++c) { latency_terms(*cl, calls[c], terms[c]); inst[c] = -1; start[c] = INF; ratio[c] = INF; order[c] = -1; }
+    // earliest finish of call c over its legal instances in the current state
+    auto project = [&](int c, float* st, float* fin) {
+        const Terms& t = terms[c];
+        int arg = -1; *fin = INF; *st = 0.0f;
+        for (int d = 0; d < D; ++d) {
+            if (lock[c] >= 0 && lock[c] != d) continue;
+            if (!(t.m <= cl->capD[d])) continue;                    // Eq. 4
+            float f;
+            const float s = earliest_start(fn[d], cl->capD[d], t.m, t.tdec[cl->typeD[d]], ready[c], &f);
+            if (f < *fin) { *fin = f; *st = s; arg = d; }
+        }
+        return arg;
+    };
+    std::vector<int> visit;
+    std::vector<float> score(C, -INF);
+    for (int c = 0; c < C; ++c) {
+        float st, fin;
+        if (project(c, &st, &fin) < 0) continue;                    // fits no instance: never visited
+        const DagView v = dag_view(dag, calls[c], flags);
+        score[c] = (v.elapsed + fin) / v.H;                         // Eq. 2 against the snapshot
+        visit.push_back(c);
+    }
+    std::stable_sort(visit.begin(), visit.end(), [&](int a, int b) { return score[a] > score[b]; });
+    int placed = 0;
+    for (int c : visit) {
+        float st, fin;
+        const int d = project(c, &st, &fin);
+        if (d < 0) continue;
+        add_interval(fn[d], st, fin, terms[c].m);
+        inst[c] = d; start[c] = st; ratio[c] = score[c]; order[placed++] = c;
+    }
+    return placed;
+}
+
 // Longest node-weighted path to a sink, per node, over a successor-CSR DAG:
 //   tail[v] = max over successors u of cp[u]   (0 without successors)
 //   cp[v]   = cost[v] + tail[v]

@@ -245,3 +245,24 @@ class Oracle:
                                             _ptr(run_end), _ptr(run_tok), _ptr(lock),
                                             _ptr(ready), _ptr(inst), _ptr(start), _ptr(ratio), _ptr(order))
         return inst, start, ratio, order, int(placed)
+
+    def decode_onepass(self, cl: Cluster, calls, run_ptr, run_end, run_tok, lock, ready, flags=0,
+                       dag: DagResult | None = None, node_wf=None, elapsed=None, run_start=None):
+        """Decode stage with the one-pass ordering (Section 5.4 fallback, Section 5.3 last sentence):
+        ranked once against the snapshot, then placed in that order.  Returns as decode_greedy."""
+        calls, n = self._calls(calls)
+        run_ptr = _u32(run_ptr); run_end = _f32(run_end); run_tok = _f32(run_tok)
+        run_start = None if run_start is None else _f32(run_start)
+        lock = np.ascontiguousarray(lock, np.int32); ready = _f32(ready)
+        inst = np.zeros(n, np.int32); start = np.zeros(n, np.float32); ratio = np.zeros(n, np.float32)
+        order = np.zeros(n, np.int32)
+        c = cl._c()
+        d, keep = self._dag(dag, node_wf, elapsed)
+        if d is None:
+            flags |= FLAG_NO_DAG
+        self.lib.orc_decode_onepass.restype = C.c_int
+        placed = self.lib.orc_decode_onepass(C.byref(c), C.byref(d) if d is not None else None, _ptr(calls), n,
+                                             int(flags), _ptr(run_ptr), None if run_start is None else _ptr(run_start),
+                                             _ptr(run_end), _ptr(run_tok), _ptr(lock),
+                                             _ptr(ready), _ptr(inst), _ptr(start), _ptr(ratio), _ptr(order))
+        return inst, start, ratio, order, int(placed)

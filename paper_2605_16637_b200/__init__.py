@@ -5,7 +5,7 @@ The binding only marshals arguments; every step runs in the CUDA library.  It
 raises at import if the library has not been built (python -m
 paper_2605_16637_b200.build); there is no CPU fallback.
 """
-from .api import (CALL_DTYPE, INSTANCE_DTYPE, HX_FLAG_NO_DAG, HX_FLAG_NO_TAIL, HX_FLAG_UNLOADED,
+from .api import (CALL_DTYPE, INSTANCE_DTYPE, HX_FLAG_NO_DAG, HX_FLAG_NO_TAIL, HX_FLAG_UNLOADED, HX_FLAG_ONE_PASS,
                   HX_MODE_COMPLETION, HX_MODE_RATIO, HX_MODE_SLACK, HxError, Cluster,
                   hx_cluster_create, hx_cluster_destroy, hx_cluster_read_loads,
                   hx_cluster_update_loads, hx_critical_path, hx_enable_kernel_timing,

@@ -16,7 +16,7 @@ from .build import LIB_PATH
 
 HX_OK = 0
 HX_MODE_COMPLETION, HX_MODE_SLACK, HX_MODE_RATIO = 0, 1, 2
-HX_FLAG_NO_DAG, HX_FLAG_NO_TAIL, HX_FLAG_UNLOADED = 1, 2, 4
+HX_FLAG_NO_DAG, HX_FLAG_NO_TAIL, HX_FLAG_UNLOADED, HX_FLAG_ONE_PASS = 1, 2, 4, 8
 
 CALL_DTYPE = np.dtype([("node", "<u4"), ("model", "<u4"),
                        ("prompt_tokens", "<f4"), ("output_tokens", "<f4")])

@@ -13,9 +13,9 @@
 //     visiting order of the batch, three short grids.  Calls are binned by the
 //     leading bits of the priority key (bins linear in the key bits between the
 //     batch minimum and maximum, which the scoring kernel left behind per block;
-//     priorities of +inf have a bin of their own, so that calls that fit nowhere
-//     do not stretch the range); inside a bin every key counts the keys that
-//     precede it.  Keys (prio, call) are unique.
+//     priorities of +inf have a bin of their own, filled in call order, so that
+//     calls that fit nowhere neither stretch the range nor need ranking); inside
+//     every other bin a key counts the keys that precede it.  Keys (prio, call) are unique.
 //  2. hx_conflict_kernel - optimistic windows over the visiting order.  A warp
 //     takes the next W calls; every call picks the first candidate that fits the
 //     capacities committed so far, then checks it against the demand of the
@@ -84,7 +84,7 @@ __device__ __forceinline__ unsigned bin_of(unsigned key, unsigned lo, unsigned s
     return key == HX_FIRST_KEY ? 0u : 1u + ((key - lo) >> shift);
 }
 __global__ void __launch_bounds__(kOrdThreads) hx_order_hist_kernel(HxTopkBufs tk, int n) {
-    __shared__ unsigned lohi[2];
+    __shared__ unsigned lohi[2], wfirst[kOrdThreads / 32];
     const int tid = threadIdx.x;
     hx_release_dependents();
     if (tid == 0) { lohi[0] = 0xFFFFFFFFu; lohi[1] = 0u; }
@@ -102,9 +102,22 @@ __global__ void __launch_bounds__(kOrdThreads) hx_order_hist_kernel(HxTopkBufs t
     unsigned shift = 0;
     while ((span >> shift) >= (unsigned)(kBins - 1)) ++shift;
     if (blockIdx.x == 0 && tid == 0) { tk.obase[kBins + 1] = lo; tk.obase[kBins + 2] = shift; }
+    // Calls with the first key (all equal, so their order is the call order) take their place by counting: a
+    // stable number inside the block here, the blocks before this one in the scatter step.  Every other call
+    // draws an arrival number inside its bin.
     const int c = blockIdx.x * kOrdThreads + tid;
+    const unsigned key = c < n ? hx_order_key(__float_as_uint(__ldcg(tk.prio + c))) : 0u;
+    const bool first = c < n && key == HX_FIRST_KEY;
+    const unsigned vote = __ballot_sync(0xffffffffu, first);
+    if ((tid & 31) == 0) wfirst[tid >> 5] = __popc(vote);
+    __syncthreads();
+    unsigned before = 0, total = 0;
+#pragma unroll
+    for (int w = 0; w < kOrdThreads / 32; ++w) { before += w < (tid >> 5) ? wfirst[w] : 0u; total += wfirst[w]; }
+    if (tid == 0) { tk.ghist[kBins + blockIdx.x] = total; if (total) atomicAdd(tk.ghist, total); }
     if (c >= n) return;
-    const unsigned bin = bin_of(hx_order_key(__float_as_uint(__ldcg(tk.prio + c))), lo, shift);
+    if (first) { tk.oslot[c] = before + __popc(vote & ((1u << (tid & 31)) - 1u)); return; }
+    const unsigned bin = bin_of(key, lo, shift);
     tk.oslot[c] = (bin << 16) | atomicAdd(tk.ghist + bin, 1u);
 }
 
@@ -119,11 +132,20 @@ __global__ void __launch_bounds__(kOrdThreads) hx_order_scatter_kernel(HxTopkBuf
     __syncthreads();
     block_exclusive_scan(hist, kBins, base, tmp);
     if (blockIdx.x == 0) for (int i = tid; i <= kBins; i += kOrdThreads) tk.obase[i] = base[i];
+    // first-key calls of the blocks before this one (at most 256 blocks: one counter per thread)
+    unsigned mine = tid < (int)blockIdx.x ? __ldcg(tk.ghist + kBins + tid) : 0u;
+    mine = __reduce_add_sync(0xffffffffu, mine);
+    if ((tid & 31) == 0) tmp[tid >> 5] = mine;
+    __syncthreads();
+    unsigned first_before = 0;
+#pragma unroll
+    for (int w = 0; w < kOrdThreads / 32; ++w) first_before += tmp[w];
     const int c = blockIdx.x * kOrdThreads + tid;
     if (c >= n) return;
     const unsigned bs = __ldcg(tk.oslot + c);
     const unsigned key = hx_order_key(__float_as_uint(__ldcg(tk.prio + c)));
-    tk.okey[base[bs >> 16] + (bs & 0xFFFFu)] = ((u64)key << 32) | (unsigned)c;
+    const unsigned at = key == HX_FIRST_KEY ? first_before + bs : base[bs >> 16] + (bs & 0xFFFFu);
+    tk.okey[at] = ((u64)key << 32) | (unsigned)c;
 }
 
 // 1c. Rank inside the bins and gather the per-call data in visiting order.
@@ -136,8 +158,8 @@ __global__ void hx_order_rank_kernel(HxTopkBufs tk, int n, unsigned D) {
     const u64 key = tk.okey[i];
     const unsigned bin = bin_of((unsigned)(key >> 32), lo, shift);
     const unsigned b0 = tk.obase[bin], b1 = tk.obase[bin + 1];
-    unsigned rank = b0;
-    for (unsigned j = b0; j < b1; ++j) rank += __ldcg(tk.okey + j) < key;
+    unsigned rank = bin ? b0 : (unsigned)i;                       // the first bin arrived in call order
+    for (unsigned j = bin ? b0 : b1; j < b1; ++j) rank += __ldcg(tk.okey + j) < key;
     const unsigned c = (unsigned)key;
     tk.ocall[rank] = c;
     tk.om[rank] = __float2int_ru(tk.mtok[c]);                   // token counts are whole numbers below 2^24

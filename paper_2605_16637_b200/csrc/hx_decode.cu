@@ -9,6 +9,11 @@
 // its Delta_D is the earliest projected finish over those instances, its ratio
 // R = (elapsed + Delta_D) / H (Eq. 2); the call with the largest R (lower index
 // among equals) is assigned, its interval is added to the chosen instance.
+// With HX_FLAG_ONE_PASS (the lightweight ordering Section 5.4 falls back to,
+// Section 5.3 last sentence) R keeps the value of the first projection, against
+// the snapshot alone: the same loop then visits the calls in the order of that
+// score, each placed by its projection against the state left by the calls
+// before it.
 //
 // Tokens in use on an instance are a step function of time: breakpoints
 // t[0] = 0 < t[1] < ... and usage u[k] on [t[k], t[k+1]); the last segment runs
@@ -264,7 +269,8 @@ __global__ void __launch_bounds__(kThreads, 1) hx_decode_kernel(const __grid_con
             if (lane == 0) {
                 if (bd != 0x7fffffff) {
                     cbest[c] = bd; cstart[c] = bs; cfin[c] = best;
-                    cR[c] = __fdiv_rn(__fadd_rn(cel[c], best), cH[c]);
+                    // one-pass ordering: the score of the first projection (against the snapshot) stays
+                    if (it == 0 || !(prm.flags & HX_FLAG_ONE_PASS)) cR[c] = __fdiv_rn(__fadd_rn(cel[c], best), cH[c]);
                 } else { cbest[c] = kNoInst; cR[c] = HX_NEG_INF; }
             }
         }

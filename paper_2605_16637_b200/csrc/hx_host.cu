@@ -201,7 +201,7 @@ int ensure_topk(hx_cluster* h, int n_calls, int K) {
     HX_TRY(dev_alloc(h->tk_allocs, &b.prio, cap), "alloc top-K");
     HX_TRY(dev_alloc(h->tk_allocs, &b.mtok, cap), "alloc top-K");
     HX_TRY(dev_alloc(h->tk_allocs, &b.blk_lohi, (size_t)2 * HX_ORDER_MAXBLK), "alloc order");
-    HX_TRY(dev_alloc(h->tk_allocs, &b.ghist, (size_t)HX_ORDER_BINS), "alloc order");
+    HX_TRY(dev_alloc(h->tk_allocs, &b.ghist, (size_t)HX_ORDER_BINS + HX_ORDER_CALLBLK), "alloc order");
     HX_TRY(dev_alloc(h->tk_allocs, &b.oslot, cap), "alloc order");
     HX_TRY(dev_alloc(h->tk_allocs, &b.okey, cap), "alloc order");
     HX_TRY(dev_alloc(h->tk_allocs, &b.obase, (size_t)HX_ORDER_BINS + 3), "alloc order");
@@ -1057,7 +1057,7 @@ int hx_set_options(hx_cluster* h, const hx_options* o) {
     if (!h || !o) return HX_ERR_INVALID_ARG;
     if (o->score_mode < HX_MODE_COMPLETION || o->score_mode > HX_MODE_RATIO) return fail(h, HX_ERR_INVALID_ARG, "unknown score mode");
     if (o->topk < 0 || o->topk > HX_MAX_TOPK) return fail(h, HX_ERR_INVALID_ARG, "topk out of range");
-    if (o->flags & ~(HX_FLAG_NO_DAG | HX_FLAG_NO_TAIL | HX_FLAG_UNLOADED)) return fail(h, HX_ERR_INVALID_ARG, "unknown flag");
+    if (o->flags & ~(HX_FLAG_NO_DAG | HX_FLAG_NO_TAIL | HX_FLAG_UNLOADED | HX_FLAG_ONE_PASS)) return fail(h, HX_ERR_INVALID_ARG, "unknown flag");
     if (!std::isfinite(o->alpha) || o->alpha <= 0.f) return fail(h, HX_ERR_INVALID_ARG, "alpha must be finite and > 0");
     h->opts = *o;
     return HX_OK;
@@ -1217,7 +1217,7 @@ constexpr size_t kStaticBytes =
     static_round(kSC * 8) +               // okey
     static_round((HX_ORDER_BINS + 3) * 4) +   // obase
     static_round(2 * HX_ORDER_MAXBLK * 4) +   // blk_lohi
-    static_round(HX_ORDER_BINS * 4) +         // ghist
+    static_round((HX_ORDER_BINS + HX_ORDER_CALLBLK) * 4) +  // ghist
     static_round(kSC * 4) +               // oslot
     static_round(4) +                     // n_acc
     3 * static_round(kSC * 4);            // acc_rk, acc_p, acc_t
@@ -1276,7 +1276,7 @@ int hx_schedule_batch_static(hx_cluster* h, const hx_call* calls, int n_calls, i
     b.okey = reinterpret_cast<unsigned long long*>(carve(kSC * 8));
     b.obase = reinterpret_cast<unsigned int*>(carve((HX_ORDER_BINS + 3) * 4));
     b.blk_lohi = reinterpret_cast<unsigned int*>(carve(2 * HX_ORDER_MAXBLK * 4));
-    b.ghist = reinterpret_cast<unsigned int*>(carve(HX_ORDER_BINS * 4));
+    b.ghist = reinterpret_cast<unsigned int*>(carve((HX_ORDER_BINS + HX_ORDER_CALLBLK) * 4));
     b.oslot = reinterpret_cast<unsigned int*>(carve(kSC * 4));
     b.n_acc = reinterpret_cast<unsigned int*>(carve(4));
     b.acc_rk = reinterpret_cast<unsigned int*>(carve(kSC * 4));

@@ -73,7 +73,7 @@ struct HxTopkBufs {
     float* mtok;               // [cap]
     // visiting order
     unsigned int* blk_lohi;    // [2 * HX_ORDER_MAXBLK] smallest / largest finite key seen by each block of the scoring kernel
-    unsigned int* ghist;       // [HX_ORDER_BINS] keys per bin (zeroed by the scoring kernel)
+    unsigned int* ghist;       // [HX_ORDER_BINS] keys per bin (zeroed by the scoring kernel), then [HX_ORDER_CALLBLK] first-key calls per block of the binning kernel
     unsigned int* oslot;       // [cap] bin << 16 | arrival number inside the bin, per call
     unsigned long long* okey;  // [cap] keys grouped by bin
     unsigned int* obase;       // [HX_ORDER_BINS + 3] bin bounds, smallest key, key-to-bin shift
@@ -93,6 +93,7 @@ struct HxTopkBufs {
 // smallest and the largest finite key of the batch.
 #define HX_ORDER_BINS 2048
 #define HX_ORDER_MAXBLK 1024
+#define HX_ORDER_CALLBLK 256   /* blocks of 256 calls in the largest batch (HX_MAX_COMMIT_CALLS) */
 #define HX_FIRST_KEY 0x807FFFFFu
 __host__ __device__ inline unsigned hx_order_key(unsigned prio_bits) {
     return prio_bits >= 0x7F800000u ? HX_FIRST_KEY : ~prio_bits;

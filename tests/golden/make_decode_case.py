@@ -61,6 +61,44 @@ def clear(best, others):
     return all(abs(x - best) > MARGIN * abs(best) for x in others)
 
 
+def project(iv, c):
+    """(instance, start, finish) with the earliest finish over the legal instances, None if there is none."""
+    n, o, lock, ready, el, H = CALLS[c]
+    opts = {}
+    for d in range(2):
+        if (lock >= 0 and lock != d) or n + o > CAP[d]:
+            continue
+        tau = tdec(n, o, TYPE_D[d])
+        s = earliest(iv[d], CAP[d], n + o, tau, ready)
+        opts[d] = (s + tau, s)
+    if not opts:
+        return None
+    d = min(opts, key=lambda k: (opts[k][0], k))
+    assert clear(opts[d][0], [v[0] for k, v in opts.items() if k != d]), ("instance margin", c)
+    return d, opts[d][1], opts[d][0]
+
+
+def one_pass():
+    """The fallback ordering (Section 5.4 with Section 5.3, last sentence): ranked once by the ratio projected
+    against the running intervals alone, then placed in that order against the growing state."""
+    iv = [[(Fr(0), e, m) for e, m in RUNNING[d]] for d in range(2)]
+    score = {}
+    for c in range(len(CALLS)):
+        pr = project(iv, c)
+        if pr is not None:
+            score[c] = (CALLS[c][4] + pr[2]) / CALLS[c][5]
+    visit = sorted(score, key=lambda c: (-score[c], c))
+    for a, b in zip(visit, visit[1:]):
+        assert score[a] - score[b] > MARGIN * score[a], ("score margin", a, b)
+    inst = [-1] * len(CALLS); start = [None] * len(CALLS); ratio = [None] * len(CALLS)
+    for c in visit:
+        d, s, f = project(iv, c)
+        iv[d].append((s, f, CALLS[c][0] + CALLS[c][1]))
+        inst[c], start[c], ratio[c] = d, s, score[c]
+    return dict(order=visit, inst=inst, start=[None if s is None else float(s) for s in start],
+                ratio=[None if r is None else float(r) for r in ratio])
+
+
 def main():
     iv = [[(Fr(0), e, m) for e, m in RUNNING[d]] for d in range(2)]
     waiting = list(range(len(CALLS)))
@@ -103,13 +141,15 @@ def main():
                     calls=[dict(prompt_tokens=n, output_tokens=o, lock=lock, ready=float(r), elapsed=float(el),
                                 H=float(H)) for n, o, lock, r, el, H in CALLS]),
         expected=dict(order=order, inst=inst, start=[None if s is None else float(s) for s in start],
-                      ratio=[None if r is None else float(r) for r in ratio], trace=trace))
+                      ratio=[None if r is None else float(r) for r in ratio], trace=trace),
+        expected_one_pass=one_pass())
     path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "decode_hand.json")
     with open(path, "w") as f:
         json.dump(out, f, indent=1)
     print("wrote", path)
     for t in trace:
         print(t)
+    print("one pass:", out["expected_one_pass"])
     print("unplaced:", [c for c in range(len(CALLS)) if inst[c] < 0])
 
 

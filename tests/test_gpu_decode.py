@@ -61,10 +61,12 @@ def _running(rng, oc, per):
     return np.array(ptr, np.uint32), np.array(end, F32), np.array(tok, F32)
 
 
-def _check(hx, gc, oc, oracle, calls, lock, ready, ptr, end, tok, commit=0, run_start=None):
-    gc.set_options(score_mode=hx.HX_MODE_RATIO, commit=commit, flags=hx.HX_FLAG_NO_DAG)
+def _check(hx, gc, oc, oracle, calls, lock, ready, ptr, end, tok, commit=0, run_start=None, one_pass=False):
+    gc.set_options(score_mode=hx.HX_MODE_RATIO, commit=commit,
+                   flags=hx.HX_FLAG_NO_DAG | (hx.HX_FLAG_ONE_PASS if one_pass else 0))
     got = [t.cpu().numpy() for t in gc.schedule_decode(calls, lock, ready)]
-    want = oracle.decode_greedy(oc, calls, ptr, end, tok, lock, ready, run_start=run_start)
+    plan = oracle.decode_onepass if one_pass else oracle.decode_greedy
+    want = plan(oc, calls, ptr, end, tok, lock, ready, run_start=run_start)
     for g, w, name in zip(got, want[:4], ("instance", "start", "ratio", "order")):
         assert np.array_equal(g, w), name
     hh.assert_costs_close(got[2], want[2], "ratio")
@@ -86,6 +88,10 @@ def test_decode_scheduler_matches_oracle(hx, oracle, D, C, per, caps):
     assert placed == C and (start > ready).any()         # some calls wait for capacity
     # without commit the snapshot is untouched: the same queue gives the same plan again
     _check(hx, gc, oc, oracle, calls, lock, ready, ptr, end, tok)
+    # the one-pass ordering on the same queue: another plan (the order changes once calls wait for capacity)
+    o_inst, o_start, o_ratio, o_order, o_placed = _check(hx, gc, oc, oracle, calls, lock, ready, ptr, end, tok,
+                                                         one_pass=True)
+    assert o_placed == C and (C < 40 or not np.array_equal(o_order, order))
     gc.close()
 
 
@@ -106,6 +112,7 @@ def test_decode_scheduler_with_a_snapshot_too_long_for_shared_memory(hx, oracle,
     gc.decode_set_running(ptr, end, tok)
     inst, start, ratio, order, placed = _check(hx, gc, oc, oracle, calls, lock, ready, ptr, end, tok)
     assert placed == C and (start > ready).any()
+    _check(hx, gc, oc, oracle, calls, lock, ready, ptr, end, tok, one_pass=True)
     gc.close()
 
 
@@ -157,6 +164,14 @@ def test_decode_worked_run(hx):
     assert list(got[3]) == e["order"] and list(got[0]) == e["inst"]
     np.testing.assert_allclose(got[1], e["start"], rtol=2e-6, atol=1e-9)
     np.testing.assert_allclose(got[2], e["ratio"], rtol=2e-6)
+    # the one-pass ordering of the same queue, also worked out in exact arithmetic
+    e = g["expected_one_pass"]
+    gc.set_options(score_mode=hx.HX_MODE_RATIO, flags=hx.HX_FLAG_ONE_PASS)
+    got = [t.cpu().numpy() for t in gc.schedule_decode(calls, [r["lock"] for r in i["calls"]],
+                                                       [r["ready"] for r in i["calls"]])]
+    assert list(got[3]) == e["order"] and list(got[0]) == e["inst"]
+    np.testing.assert_allclose(got[1], e["start"], rtol=2e-6, atol=1e-9)
+    np.testing.assert_allclose(got[2], e["ratio"], rtol=2e-6)
     gc.close()
 
 
@@ -180,6 +195,15 @@ def test_decode_argument_checks_and_oversized_calls(hx, oracle):
     for g, w in zip(got, want[:4]):
         assert np.array_equal(g, w)
     assert gc.status() == 0
+    gc.set_options(flags=hx.HX_FLAG_NO_DAG | hx.HX_FLAG_ONE_PASS)   # the oversized call is never visited
+    got = [t.cpu().numpy() for t in gc.schedule_decode(calls, lock, ready)]
+    want = oracle.decode_onepass(oc, calls, [0, 0, 0, 0], [], [], lock, ready)
+    assert got[0][7] == -1 and np.isinf(got[2][7]) and want[4] == 19 and got[3][19] == -1
+    for g, w in zip(got, want[:4]):
+        assert np.array_equal(g, w)
+    with pytest.raises(hx.HxError):
+        gc.set_options(flags=16)                                # not a flag
+    gc.set_options(flags=hx.HX_FLAG_NO_DAG)
     bad = lock.copy(); bad[2] = 9                               # lock beyond the pool
     got = [t.cpu().numpy() for t in gc.schedule_decode(calls, bad, ready)]
     assert got[0][2] == -1 and gc.status() == -1
