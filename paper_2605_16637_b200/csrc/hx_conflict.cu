@@ -148,18 +148,39 @@ __global__ void __launch_bounds__(kOrdThreads) hx_order_scatter_kernel(HxTopkBuf
     tk.okey[at] = ((u64)key << 32) | (unsigned)c;
 }
 
-// 1c. Rank inside the bins and gather the per-call data in visiting order.
-__global__ void hx_order_rank_kernel(HxTopkBufs tk, int n, unsigned D) {
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+// 1c. Rank inside the bins and gather the per-call data in visiting order.  One key per thread; the block
+// brings the keys of all bins that its threads belong to (one contiguous stretch) through shared memory, a
+// tile at a time, and every thread counts the smaller keys of its own bin among them: a crowded bin (many
+// equal priorities) then costs one shared-memory load per comparison instead of a trip to L2.
+constexpr int kRankThreads = 128, kRankTile = 512;
+__global__ void __launch_bounds__(kRankThreads) hx_order_rank_kernel(HxTopkBufs tk, int n, unsigned D) {
+    __shared__ u64 tile[kRankTile];
+    __shared__ unsigned range[2];
+    const int tid = threadIdx.x;
+    const int i = blockIdx.x * kRankThreads + tid;
     hx_release_dependents();
     hx_wait_for_primary();                                        // every key is in its bin
-    if (i >= n) return;
+    const bool valid = i < n;
     const unsigned lo = tk.obase[kBins + 1], shift = tk.obase[kBins + 2];
-    const u64 key = tk.okey[i];
-    const unsigned bin = bin_of((unsigned)(key >> 32), lo, shift);
-    const unsigned b0 = tk.obase[bin], b1 = tk.obase[bin + 1];
-    unsigned rank = bin ? b0 : (unsigned)i;                       // the first bin arrived in call order
-    for (unsigned j = bin ? b0 : b1; j < b1; ++j) rank += __ldcg(tk.okey + j) < key;
+    const u64 key = valid ? tk.okey[i] : 0ull;
+    const unsigned bin = valid ? bin_of((unsigned)(key >> 32), lo, shift) : 0u;
+    // the first bin arrived in call order: nothing to count there
+    const unsigned b0 = bin ? tk.obase[bin] : (unsigned)i, b1 = bin ? tk.obase[bin + 1] : (unsigned)i;
+    if (tid == 0) range[0] = b0;                                  // bins ascend with the position: the first thread has the lowest
+    if (i == min(n, (int)(blockIdx.x + 1) * kRankThreads) - 1) range[1] = b1;   // ... and the last valid one the highest
+    __syncthreads();
+    const unsigned u0 = range[0], u1 = range[1];
+    unsigned rank = b0;
+    for (unsigned t0 = u0; t0 < u1; t0 += kRankTile) {
+        const unsigned len = min((unsigned)kRankTile, u1 - t0);
+        if (t0 != u0) __syncthreads();                            // the previous tile has been read
+        for (unsigned j = tid; j < len; j += kRankThreads) tile[j] = __ldcg(tk.okey + t0 + j);
+        __syncthreads();
+        const unsigned a = max(b0, t0), e = min(b1, t0 + len);
+#pragma unroll 4
+        for (unsigned j = a; j < e; ++j) rank += tile[j - t0] < key;
+    }
+    if (!valid) return;
     const unsigned c = (unsigned)key;
     tk.ocall[rank] = c;
     tk.om[rank] = __float2int_ru(tk.mtok[c]);                   // token counts are whole numbers below 2^24
@@ -495,7 +516,7 @@ cudaError_t hx_launch_conflict(const HxTables& t, const HxTopkBufs& tk, int n_ca
     // predecessor before reading what that one wrote
     cudaError_t e = hx_launch_dependent(hx_order_hist_kernel, dim3(nb), dim3(kOrdThreads), 0, stream, tk, n_calls);
     if (e == cudaSuccess) e = hx_launch_dependent(hx_order_scatter_kernel, dim3(nb), dim3(kOrdThreads), 0, stream, tk, n_calls);
-    if (e == cudaSuccess) e = hx_launch_dependent(hx_order_rank_kernel, dim3((n_calls + 127) / 128), dim3(128), 0, stream, tk, n_calls, (unsigned)D);
+    if (e == cudaSuccess) e = hx_launch_dependent(hx_order_rank_kernel, dim3((n_calls + kRankThreads - 1) / kRankThreads), dim3(kRankThreads), 0, stream, tk, n_calls, (unsigned)D);
     if (e != cudaSuccess) return e;
     const int fused = P <= kTailMaxP;                               // pairs published and queues summed inside the pass
     const size_t smRing = (size_t)kRing * 24 + (size_t)(D + 1) * 4;
