@@ -318,6 +318,9 @@ __global__ void __launch_bounds__(kPassThreads, 1) hx_conflict_kernel(HxTopkBufs
     __shared__ unsigned n_acc_s;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const unsigned lt = (1u << lane) - 1u;
+    // the scoring kernel of the next batch may take the other SMs and do the part of its set-up that reads
+    // nothing a kernel writes; it waits for this grid before it goes on, and releases its own dependents after
+    hx_release_dependents();
     for (int d = tid; d <= D; d += kPassThreads) free_s[d] = d < D ? __float2int_rd(t.freeD[d]) : -1;
     hx_wait_for_primary();                                      // the visiting order
     __syncthreads();

@@ -238,9 +238,9 @@ inline cudaError_t hx_launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3
     cudaLaunchAttribute attr{};
     attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr.val.programmaticStreamSerializationAllowed = 1;
-    // inside a stream capture the ordinary dependency is kept: replayed graphs of this chain measured slower
-    // with programmatic edges (1.88 against 1.78 ms per sweep step), enqueued launches faster (122 against 129 us
-    // per ready batch)
+    // inside a stream capture the ordinary dependency is kept: replayed graphs measured slower with programmatic
+    // edges (all edges of the capacity pass's chain: 1.88 against 1.78 ms per sweep step; the edge into the
+    // scoring kernel alone: 1.78 against 1.77), enqueued launches faster (122 against 129 us per ready batch)
     cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
     if (cudaStreamIsCapturing(stream, &cap) != cudaSuccess) cap = cudaStreamCaptureStatusNone;
     cfg.attrs = &attr; cfg.numAttrs = cap == cudaStreamCaptureStatusNone ? 1 : 0;

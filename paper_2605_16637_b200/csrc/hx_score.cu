@@ -235,11 +235,23 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
     // the largest finite priority key of every block's calls behind (no state survives from earlier batches)
     unsigned key_lo = 0xFFFFFFFFu, key_hi = 0u;
     __shared__ unsigned key_lohi[2];
-    hx_release_dependents();                                      // the first kernel of the capacity pass may get ready behind this one
-    if (prm.s.K > 0) {
-        for (int i = blockIdx.x * nthr + tid; i < HX_ORDER_BINS; i += gridDim.x * nthr) prm.tk.ghist[i] = 0u;
-        if (tid == 0) { key_lohi[0] = 0xFFFFFFFFu; key_lohi[1] = 0u; }
-    }
+    if (tid == 0) { key_lohi[0] = 0xFFFFFFFFu; key_lohi[1] = 0u; }
+    // Launched as a programmatic dependent, this kernel may become resident while the kernel before it on the
+    // stream (the capacity pass of the previous batch) still runs.  Everything up to sync_with_stream() reads
+    // only what no kernel writes (call records, instance classes and capacities, link table, model constants)
+    // and writes only shared memory; the prefill queues, the free KV tokens and every buffer of the top-K
+    // lists are touched after it.  The kernels behind this one are released after the wait, so that none of
+    // them can overtake the previous batch either.
+    bool synced = false;
+    auto sync_with_stream = [&] {
+        if (synced) return;
+        synced = true;
+        hx_wait_for_primary();
+        hx_release_dependents();                                  // the first kernel of the capacity pass may get ready behind this one
+        if (prm.s.K > 0)
+            for (int i = blockIdx.x * nthr + tid; i < HX_ORDER_BINS; i += gridDim.x * nthr) prm.tk.ghist[i] = 0u;
+        for (int p = tid; p < Ppad; p += nthr) qPs[p] = p < P ? (unloaded ? 0.0f : T.qP[p]) : HX_INF;
+    };
     // the call records of the first tile come from DRAM: request them before anything else
     const bool with_dag = !(prm.s.flags & HX_FLAG_NO_DAG);
     uint4 pre[2];
@@ -251,10 +263,7 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
         if (idx < TCB * G && gc < prm.s.n_calls) pre[k] = __ldg(reinterpret_cast<const uint4*>(prm.s.calls) + gc);
     }
     // instance tables; padded prefill slots can never win, padded decode columns are infeasible
-    for (int p = tid; p < Ppad; p += nthr) {
-        qPs[p] = p < P ? (unloaded ? 0.0f : T.qP[p]) : HX_INF;
-        typePs[p] = p < P ? T.typeP[p] : 0;
-    }
+    for (int p = tid; p < Ppad; p += nthr) typePs[p] = p < P ? T.typeP[p] : 0;
     for (int d = tid; d < Dpad; d += nthr) {
         qDs[d] = d < D ? (unloaded ? 0.0f : T.qD[d]) : 0.0f;
         capDs[d] = d < D ? T.capD[d] : -1.0f;
@@ -308,6 +317,7 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
             tdecs[g * TCB + c] = __fmul_rn(__fmul_rn(o, step), iB);
             if (g == 0) { kvBs[c] = kvB; mtoks[c] = __fadd_rn(n, o); }
         }
+        sync_with_stream();
         lt_wait();
         __syncthreads();
 
@@ -631,6 +641,7 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
         }
         __syncthreads();
     }
+    sync_with_stream();                                           // a block without a tile
     if (prm.s.K > 0) {
         key_lo = __reduce_min_sync(0xffffffffu, key_lo); key_hi = __reduce_max_sync(0xffffffffu, key_hi);
         if (lane == 0) { atomicMin(&key_lohi[0], key_lo); atomicMax(&key_lohi[1], key_hi); }
@@ -648,8 +659,7 @@ cudaError_t launch_one(const ScoreParams& prm, int grid, int threads, size_t sme
     static size_t allowed[64];
     cudaError_t e = hx_opt_in_smem(hx_score_kernel<TC, TD, LD>, smem, allowed, 0);
     if (e != cudaSuccess) return e;
-    hx_score_kernel<TC, TD, LD><<<grid, threads, smem, stream>>>(prm);
-    return cudaGetLastError();
+    return hx_launch_dependent(hx_score_kernel<TC, TD, LD>, dim3(grid), dim3(threads), smem, stream, prm);
 }
 
 inline int round_up(int a, int b) { return (a + b - 1) / b * b; }
