@@ -57,6 +57,7 @@ def test_greedy_on_generated_queues(hx, oracle, name, scale):
 
 @pytest.mark.parametrize("P, D, n, frac", [(1, 1, 9, 0.5), (2, 2, 64, 0.5), (3, 5, 200, 0.3), (16, 16, 700, 0.6),
                                            (33, 7, 333, 0.4), (64, 64, 256, 0.5),
+                                           (128, 64, 300, 0.5),     # per-class times cached, no room for the row minima
                                            (200, 200, 500, 0.4)])   # the last: no room for the cached per-class times
 def test_greedy_with_binding_capacity(hx, oracle, P, D, n, frac):
     rng = np.random.default_rng(100 + P + D)
