@@ -99,10 +99,10 @@ __global__ void __launch_bounds__(kThreads, 1) hx_decode_kernel(const __grid_con
     extern __shared__ __align__(16) unsigned char smem[];
     __shared__ float red_v[kWarps];
     __shared__ int red_c[kWarps];
-    __shared__ int s_call, s_d, s_ndirty, s_cur;
-    __shared__ float x_v[NC];                  // most urgent call of every block (written by its owner block)
-    __shared__ int x_c[NC];
-    __shared__ float x_commit[4];              // instance (int bits), start, finish, demand of the committed call
+    __shared__ int s_ndirty, s_cur, s_full;
+    // most urgent call of every block with its interval: ratio, call, instance (int bits), start, finish, demand;
+    // written by the owner block into every block, two sets used in turn by the iterations
+    __shared__ float x_cand[2][NC][6];
     const HxTables& T = prm.t;
     const int D = T.D;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -143,7 +143,7 @@ __global__ void __launch_bounds__(kThreads, 1) hx_decode_kernel(const __grid_con
         capDs[d] = T.capD[d]; typeDs[d] = T.typeD[d];
         Ks[d] = prm.base.K[d];
     }
-    if (tid == 0) s_cur = 0;
+    if (tid == 0) { s_cur = 0; s_full = 0; }
     __syncthreads();
     if (POOL && tid == 0) {                                     // every instance its breakpoints plus an equal share of the rest
         int sum = 0;
@@ -275,7 +275,7 @@ __global__ void __launch_bounds__(kThreads, 1) hx_decode_kernel(const __grid_con
             }
         }
         __syncthreads();
-        // (2) most urgent waiting call
+        // (2) most urgent waiting call of this block
         float rv = HX_NEG_INF; int rc = 0x7fffffff;
         for (int c = tid; c < n; c += kThreads) {
             const float r = cR[c];
@@ -289,6 +289,7 @@ __global__ void __launch_bounds__(kThreads, 1) hx_decode_kernel(const __grid_con
         }
         if (lane == 0) { red_v[warp] = rv; red_c[warp] = rc; }
         __syncthreads();
+        float (*xc)[6] = x_cand[it & 1];
         if (warp == 0) {
             rv = red_v[lane]; rc = red_c[lane];
 #pragma unroll
@@ -298,111 +299,109 @@ __global__ void __launch_bounds__(kThreads, 1) hx_decode_kernel(const __grid_con
                 if (ov > rv || (ov == rv && oc < rc)) { rv = ov; rc = oc; }
             }
             if (lane == 0) {
-                if (NC > 1) {                                  // publish the block's candidate in every block
-                    cg::cluster_group cl = cg::this_cluster();
-                    for (int r = 0; r < NC; ++r) {
-                        *cl.map_shared_rank(&x_v[rank], r) = rv;
-                        *cl.map_shared_rank(&x_c[rank], r) = rc;
-                    }
-                } else {
-                    x_v[0] = rv; x_c[0] = rc;
+                // the block's candidate with its interval (instance, start, finish, demand), published in every block
+                float cand[6] = {rv, __int_as_float(rc), 0.f, 0.f, 0.f, 0.f};
+                if (rc != 0x7fffffff) {
+                    const int li = rc / NC;
+                    cand[2] = __int_as_float(cbest[li]); cand[3] = cstart[li]; cand[4] = cfin[li];
+                    cand[5] = __fadd_rn(cn[li], co[li]);
                 }
-            }
-        }
-        if (NC > 1) cg::this_cluster().sync(); else __syncthreads();      // every thread of every block
-        if (warp == 0) {
-            rv = lane < NC ? x_v[lane] : HX_NEG_INF;           // all blocks reduce the same list
-            rc = lane < NC ? x_c[lane] : 0x7fffffff;
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) {
-                const float ov = __shfl_xor_sync(0xffffffffu, rv, off);
-                const int oc = __shfl_xor_sync(0xffffffffu, rc, off);
-                if (ov > rv || (ov == rv && oc < rc)) { rv = ov; rc = oc; }
-            }
-            if (lane == 0) s_call = rc == 0x7fffffff ? -1 : rc;
-            if (lane == 0 && rc != 0x7fffffff && rc % NC == rank) {
-                // the block that owns the call publishes its interval and records the result
-                const int li = rc / NC;
-                const int d = cbest[li];
-                const float st = cstart[li], en = cfin[li], m = __fadd_rn(cn[li], co[li]);
-                prm.out_inst[rc] = d; prm.out_start[rc] = st; prm.out_ratio[rc] = rv; prm.out_order[it] = rc;
-                cbest[li] = kDead; cR[li] = HX_NEG_INF;
                 if (NC > 1) {
                     cg::cluster_group cl = cg::this_cluster();
                     for (int r = 0; r < NC; ++r) {
-                        float* xc = cl.map_shared_rank(x_commit, r);
-                        xc[0] = __int_as_float(d); xc[1] = st; xc[2] = en; xc[3] = m;
+                        float* dst = cl.map_shared_rank(&xc[rank][0], r);
+#pragma unroll
+                        for (int k = 0; k < 6; ++k) dst[k] = cand[k];
                     }
                 } else {
-                    x_commit[0] = __int_as_float(d); x_commit[1] = st; x_commit[2] = en; x_commit[3] = m;
+#pragma unroll
+                    for (int k = 0; k < 6; ++k) xc[0][k] = cand[k];
                 }
+                s_ndirty = 0;                                  // the list of this iteration has been read by everybody
             }
         }
-        if (NC > 1) cg::this_cluster().sync(); else __syncthreads();      // the interval has reached every block
+        // one barrier per iteration: a block that runs ahead writes the other set of candidates, and cannot get
+        // past the next barrier before every block has read this one
+        if (NC > 1) cg::this_cluster().sync(); else __syncthreads();      // every thread of every block
+        // every warp of every block reduces the same list: nothing to hand round inside the block
+        rv = lane < NC ? xc[lane][0] : HX_NEG_INF;
+        rc = lane < NC ? __float_as_int(xc[lane][1]) : 0x7fffffff;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, rv, off);
+            const int oc = __shfl_xor_sync(0xffffffffu, rc, off);
+            if (ov > rv || (ov == rv && oc < rc)) { rv = ov; rc = oc; }
+        }
+        if (rc == 0x7fffffff) break;                            // nobody left that fits anywhere: all blocks leave
+        const float* win = xc[rc % NC];
+        const int ds = __float_as_int(win[2]);
         if (warp == 0) {
             // (3) commit (warp 0 of every block): add the interval [start, finish) with m tokens to the block's copy
-            if (s_call >= 0) {
-                const int d = __float_as_int(x_commit[0]);
-                const float st = x_commit[1], en = x_commit[2], m = x_commit[3];
-                int K = Ks[d];
-                bool room = POOL ? K + 2 <= roff[d + 1] - roff[d] : K + 2 <= cap;
-                if (POOL && !room) {
-                    // lay the regions out again in the other half, after two entries set aside for this commit
-                    if (lane == 0) {
-                        int sum = 0;
-                        for (int e = 0; e < D; ++e) sum += Ks[e];
-                        const int free_now = PT - sum - 2;
-                        if (free_now >= 0) {
-                            // half of what is free goes to the instance that ran full (it is the popular one and
-                            // would be back soon with an equal share), the rest is split evenly
-                            const int mine = free_now / 2, share = (free_now - mine) / D;
-                            int o = 0;
-                            for (int e = 0; e < D; ++e) { roff2[e] = o; o += Ks[e] + share + (e == d ? 2 + mine : 0); }
-                            roff2[D] = o;
-                        } else {
-                            roff2[D] = -1;                       // the pool itself is full: the host sized it too small
-                        }
+            const int d = ds;
+            const float st = win[3], en = win[4], m = win[5];
+            if (lane == 0 && rc % NC == rank) {                 // the block that owns the call records the result
+                const int li = rc / NC;
+                prm.out_inst[rc] = d; prm.out_start[rc] = st; prm.out_ratio[rc] = rv; prm.out_order[it] = rc;
+                cbest[li] = kDead; cR[li] = HX_NEG_INF;
+            }
+            int K = Ks[d];
+            bool room = POOL ? K + 2 <= roff[d + 1] - roff[d] : K + 2 <= cap;
+            if (POOL && !room) {
+                // lay the regions out again in the other half, after two entries set aside for this commit
+                if (lane == 0) {
+                    int sum = 0;
+                    for (int e = 0; e < D; ++e) sum += Ks[e];
+                    const int free_now = PT - sum - 2;
+                    if (free_now >= 0) {
+                        // half of what is free goes to the instance that ran full (it is the popular one and
+                        // would be back soon with an equal share), the rest is split evenly
+                        const int mine = free_now / 2, share = (free_now - mine) / D;
+                        int o = 0;
+                        for (int e = 0; e < D; ++e) { roff2[e] = o; o += Ks[e] + share + (e == d ? 2 + mine : 0); }
+                        roff2[D] = o;
+                    } else {
+                        roff2[D] = -1;                       // the pool itself is full: the host sized it too small
+                    }
+                }
+                __syncwarp();
+                if (roff2[D] >= 0) {
+                    const int cur = s_cur;
+                    for (int e = 0; e < D; ++e) {
+                        const float* ot = pool_t + (size_t)cur * PT + roff[e];
+                        const float* ou = pool_u + (size_t)cur * PT + roff[e];
+                        float* nt2 = pool_t + (size_t)(cur ^ 1) * PT + roff2[e];
+                        float* nu2 = pool_u + (size_t)(cur ^ 1) * PT + roff2[e];
+                        for (int i = lane; i < Ks[e]; i += 32) { nt2[i] = ot[i]; nu2[i] = ou[i]; }
                     }
                     __syncwarp();
-                    if (roff2[D] >= 0) {
-                        const int cur = s_cur;
-                        for (int e = 0; e < D; ++e) {
-                            const float* ot = pool_t + (size_t)cur * PT + roff[e];
-                            const float* ou = pool_u + (size_t)cur * PT + roff[e];
-                            float* nt2 = pool_t + (size_t)(cur ^ 1) * PT + roff2[e];
-                            float* nu2 = pool_u + (size_t)(cur ^ 1) * PT + roff2[e];
-                            for (int i = lane; i < Ks[e]; i += 32) { nt2[i] = ot[i]; nu2[i] = ou[i]; }
-                        }
-                        __syncwarp();
-                        for (int e = lane; e <= D; e += 32) roff[e] = roff2[e];
-                        if (lane == 0) s_cur = cur ^ 1;
-                        __syncwarp();
-                        room = true;
-                    }
-                }
-                float* tt = seg_t(d);
-                float* uu = seg_u(d);
-                __syncwarp();
-                if (!room) {                                    // cannot happen with the capacity the host sizes
-                    if (lane == 0) { atomicExch(prm.status, HX_ERR_INVALID_ARG); s_call = -1; }
-                } else {
-                    const int a = warp_cut(tt, uu, K, st, lane);
-                    const int b = warp_cut(tt, uu, K, en, lane);
-                    float mx = 0.f;
-                    for (int k = a + lane; k < b; k += 32) { const float uv = __fadd_rn(uu[k], m); uu[k] = uv; mx = fmaxf(mx, uv); }
-#pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-                    if (lane == 0) { Ks[d] = K; s_d = d; umax[d] = fmaxf(umax[d], mx); }
+                    for (int e = lane; e <= D; e += 32) roff[e] = roff2[e];
+                    if (lane == 0) s_cur = cur ^ 1;
+                    __syncwarp();
+                    room = true;
                 }
             }
-            if (lane == 0) s_ndirty = 0;
+            float* tt = seg_t(d);
+            float* uu = seg_u(d);
+            __syncwarp();
+            if (!room) {                                    // cannot happen with the capacity the host sizes
+                if (lane == 0) { atomicExch(prm.status, HX_ERR_INVALID_ARG); s_full = 1; }
+            } else {
+                const int a = warp_cut(tt, uu, K, st, lane);
+                const int b = warp_cut(tt, uu, K, en, lane);
+                float mx = 0.f;
+                for (int k = a + lane; k < b; k += 32) { const float uv = __fadd_rn(uu[k], m); uu[k] = uv; mx = fmaxf(mx, uv); }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+                if (lane == 0) { Ks[d] = K; umax[d] = fmaxf(umax[d], mx); }
+            }
+        } else {
+            // meanwhile the other warps list the calls whose best instance gets the interval (a call that is being
+            // taken right now may be listed: the projection skips it)
+            for (int c = tid - 32; c < n; c += kThreads - 32)
+                if (cbest[c] == ds) dirty[atomicAdd(&s_ndirty, 1)] = (unsigned short)c;
         }
         __syncthreads();
-        if (s_call < 0) break;
-        const int ds = s_d;
-        for (int c = tid; c < n; c += kThreads)
-            if (cbest[c] == ds) dirty[atomicAdd(&s_ndirty, 1)] = (unsigned short)c;
-        __syncthreads();
+        if (s_full) break;                                      // an instance's region ran full (same in every block)
     }
     if (prm.commit && rank == 0) {                              // the simulated state becomes the snapshot
         __syncthreads();
