@@ -7,6 +7,7 @@
 #include <cstring>
 #include <mutex>
 #include <new>
+#include <thread>
 #include <unordered_map>
 
 #include "hx_internal.h"
@@ -229,11 +230,131 @@ struct HostForest {
     std::vector<uint8_t> wf_class;
 };
 
+// Classes of the horizon pass by staging footprint; largest workflows first inside a class, so that the long
+// ones do not start last.
+void classify_workflows(HostForest* out) {
+    HostForest& hf = *out;
+    const uint32_t W = hf.W;
+    const auto& wf_node_start = hf.wf_node_start;
+    hf.wf_class.assign(W, 0);
+    for (auto& v : hf.ids) v.clear();
+    for (uint32_t w = 0; w < W; ++w) {
+        const size_t n = wf_node_start[w + 1] - wf_node_start[w], e = hf.wf_edge_start[w + 1] - hf.wf_edge_start[w];
+        const size_t nlev = hf.wf_seg_start[w + 1] - hf.wf_seg_start[w] - 1;
+        const size_t need = 4 * (3 * n + 1) + 4 * (nlev + 1) + 2 * e + 16;
+        const int k = hx_cpath_class_of(need, n);
+        hf.ids[k].push_back(w);
+        hf.wf_class[w] = (uint8_t)k;
+    }
+    for (auto& v : hf.ids)
+        std::stable_sort(v.begin(), v.end(), [&](uint32_t a, uint32_t b) {
+            return wf_node_start[a + 1] - wf_node_start[a] > wf_node_start[b + 1] - wf_node_start[b]; });
+}
+
+// The regrouping of prepare_forest for a forest whose nodes are listed workflow by workflow: every workflow is a
+// contiguous range of nodes with all its edges inside (the caller checked that no edge crosses workflows), so
+// the topological order, the heights and the ordering by (height, node number) are taken range by range on
+// arrays that stay in the cache.  Same result as the general path; false when a workflow has a cycle.
+bool regroup_workflow_by_workflow(const uint32_t* row_ptr, const uint32_t* col_idx, const float* node_costs,
+                                  const uint32_t* node_workflow, uint32_t N, uint32_t E, uint32_t W, HostForest* out) {
+    HostForest& hf = *out;
+    auto& wns = hf.wf_node_start;
+    wns.assign((size_t)W + 1, 0);
+    for (uint32_t v = 0; v < N; ++v) ++wns[node_workflow[v] + 1];
+    for (uint32_t w = 0; w < W; ++w) wns[w + 1] += wns[w];
+    hf.perm.resize(N); hf.inv.resize(N);
+    hf.irow.resize((size_t)N + 1); hf.icol32.resize(E); hf.icol16.assign((size_t)E + 2, 0);   // two spare entries: slices are copied as 32-bit words
+    hf.icost.resize(N);
+    hf.wf_seg_start.assign((size_t)W + 1, 0); hf.wf_edge_start.assign((size_t)W + 1, 0);
+    // Workflows are independent and every output position is known from the node and edge ranges, except the
+    // level boundaries, which each worker collects for its stretch of workflows and which are joined afterwards.
+    const unsigned hw = std::thread::hardware_concurrency();
+    const uint32_t n_workers = N < 65536 ? 1u : std::max(1u, std::min({hw ? hw : 1u, 8u, W}));
+    std::vector<std::vector<uint32_t>> seg_part(n_workers), seg_count(n_workers);
+    std::vector<char> failed(n_workers, 0);
+    auto work = [&](uint32_t k) {
+        const uint32_t w0 = (uint32_t)((uint64_t)W * k / n_workers), w1 = (uint32_t)((uint64_t)W * (k + 1) / n_workers);
+        std::vector<uint32_t> indeg, topo, hgt, order, cnt;
+        auto& segs = seg_part[k]; auto& nseg = seg_count[k];
+        segs.reserve((size_t)(wns[w1] - wns[w0]) + (w1 - w0)); nseg.reserve(w1 - w0);
+        for (uint32_t w = w0; w < w1; ++w) {
+            const uint32_t ns = wns[w], n = wns[w + 1] - ns;
+            if (indeg.size() < n) { indeg.resize(n); topo.resize(n); hgt.resize(n); order.resize(n); }
+            std::fill(indeg.begin(), indeg.begin() + n, 0u);
+            for (uint32_t e = row_ptr[ns]; e < row_ptr[ns + n]; ++e) ++indeg[col_idx[e] - ns];
+            uint32_t nt = 0;
+            for (uint32_t i = 0; i < n; ++i) if (indeg[i] == 0) topo[nt++] = i;
+            for (uint32_t i = 0; i < nt; ++i) {
+                const uint32_t v = ns + topo[i];
+                for (uint32_t e = row_ptr[v]; e < row_ptr[v + 1]; ++e) if (--indeg[col_idx[e] - ns] == 0) topo[nt++] = col_idx[e] - ns;
+            }
+            if (nt != n) { failed[k] = 1; return; }
+            uint32_t max_h = 0;
+            for (uint32_t i = n; i-- > 0;) {
+                const uint32_t l = topo[i], v = ns + l;
+                uint32_t hh = 0;
+                for (uint32_t e = row_ptr[v]; e < row_ptr[v + 1]; ++e) hh = std::max(hh, hgt[col_idx[e] - ns] + 1);
+                hgt[l] = hh; max_h = std::max(max_h, hh);
+            }
+            cnt.assign((size_t)max_h + 2, 0);          // stable counting sort by height: node number decides among equals
+            for (uint32_t i = 0; i < n; ++i) ++cnt[hgt[i] + 1];
+            for (size_t i = 1; i < cnt.size(); ++i) cnt[i] += cnt[i - 1];
+            for (uint32_t i = 0; i < n; ++i) order[cnt[hgt[i]]++] = i;
+            const size_t seg0 = segs.size();
+            segs.push_back(0);
+            for (uint32_t j = 0; j < n; ++j) {
+                hf.perm[ns + j] = ns + order[j]; hf.inv[ns + order[j]] = ns + j;
+                if (j + 1 == n || hgt[order[j + 1]] != hgt[order[j]]) segs.push_back(j + 1);
+            }
+            nseg.push_back((uint32_t)(segs.size() - seg0));
+            uint32_t o = row_ptr[ns];                  // the edges of a workflow keep their stretch of the edge array
+            hf.wf_edge_start[w] = o;
+            for (uint32_t j = 0; j < n; ++j) {
+                const uint32_t v = ns + order[j];
+                hf.icost[ns + j] = node_costs[v];
+                hf.irow[ns + j] = o;
+                for (uint32_t e = row_ptr[v]; e < row_ptr[v + 1]; ++e, ++o) {
+                    const uint32_t local = hf.inv[col_idx[e]] - ns;
+                    hf.icol32[o] = local; hf.icol16[o] = (uint16_t)local;
+                }
+            }
+        }
+    };
+    if (n_workers == 1) {
+        work(0);
+    } else {
+        std::vector<std::thread> pool;
+        for (uint32_t k = 1; k < n_workers; ++k) pool.emplace_back(work, k);
+        work(0);
+        for (auto& th : pool) th.join();
+    }
+    for (char f : failed) if (f) return false;
+    size_t off = 0;
+    uint32_t w = 0;
+    for (uint32_t k = 0; k < n_workers; ++k)
+        for (uint32_t c : seg_count[k]) { hf.wf_seg_start[w++] = (uint32_t)off; off += c; }
+    hf.seg_off.resize(off);
+    off = 0;
+    for (uint32_t k = 0; k < n_workers; ++k) { std::copy(seg_part[k].begin(), seg_part[k].end(), hf.seg_off.begin() + off); off += seg_part[k].size(); }
+    const uint32_t o = E;
+    hf.irow[N] = o;
+    hf.wf_seg_start[W] = (uint32_t)hf.seg_off.size();
+    hf.wf_edge_start[W] = o;
+    return true;
+}
+
 // Host part of an upload; false when the graph has a cycle.  The arrays were validated by the caller.
 bool prepare_forest(const uint32_t* row_ptr, const uint32_t* col_idx, const float* node_costs,
                     const uint32_t* node_workflow, uint32_t N, uint32_t E, uint32_t W, HostForest* out) {
     HostForest& hf = *out;
     hf.N = N; hf.E = E; hf.W = W;
+    bool grouped = true;                               // nodes listed workflow by workflow (the usual case)?
+    for (uint32_t v = 1; v < N && grouped; ++v) grouped = node_workflow[v] >= node_workflow[v - 1];
+    if (grouped) {
+        if (!regroup_workflow_by_workflow(row_ptr, col_idx, node_costs, node_workflow, N, E, W, &hf)) return false;
+        classify_workflows(&hf);
+        return true;
+    }
     std::vector<uint32_t> indeg(N, 0);
     for (uint32_t e = 0; e < E; ++e) ++indeg[col_idx[e]];
     // topological order (cycle check), then height above the sinks
@@ -299,22 +420,7 @@ bool prepare_forest(const uint32_t* row_ptr, const uint32_t* col_idx, const floa
     }
     for (uint32_t w = 0; w <= W; ++w) wf_edge_start[w] = irow[wf_node_start[w]];
 
-    // classes of the horizon pass by staging footprint
-    auto& ids = hf.ids; auto& wf_class = hf.wf_class;
-    wf_class.assign(W, 0);
-    for (uint32_t w = 0; w < W; ++w) {
-        const size_t n = wf_node_start[w + 1] - wf_node_start[w], e = wf_edge_start[w + 1] - wf_edge_start[w];
-        const size_t nlev = wf_seg_start[w + 1] - wf_seg_start[w] - 1;
-        const size_t need = 4 * (3 * n + 1) + 4 * (nlev + 1) + 2 * e + 16;
-        const int k = hx_cpath_class_of(need, n);
-        ids[k].push_back(w);
-        wf_class[w] = (uint8_t)k;
-    }
-    // largest workflows first inside a class, so that the long ones do not start last
-    for (auto& v : ids)
-        std::stable_sort(v.begin(), v.end(), [&](uint32_t a, uint32_t b) {
-            return wf_node_start[a + 1] - wf_node_start[a] > wf_node_start[b + 1] - wf_node_start[b]; });
-
+    classify_workflows(&hf);
     return true;
 }
 
@@ -326,6 +432,12 @@ int upload_forest(hx_cluster* h, const HostForest& hf, ForestPart* part,
     f->n_nodes = hf.N; f->n_edges = hf.E; f->n_workflows = hf.W;
     // one allocation and one copy for the whole part: sections packed on 256-byte boundaries
     std::vector<unsigned char> blob;
+    {   // room for every section at once: growing section by section would copy the blob again and again
+        size_t words = hf.wf_node_start.size() + hf.wf_edge_start.size() + hf.wf_seg_start.size() + hf.seg_off.size() +
+                       hf.irow.size() + hf.icol32.size() + hf.icost.size() + hf.perm.size() + (wf_gid ? wf_gid->size() : 0);
+        for (int k = 0; k < HX_CP_CLASSES; ++k) words += hf.ids[k].size();
+        blob.reserve(words * 4 + hf.icol16.size() * 2 + 256 * (10 + HX_CP_CLASSES));
+    }
     auto put = [&](const void* src, size_t bytes) {
         const size_t off = (blob.size() + 255) & ~size_t(255);
         blob.resize(off + bytes);
