@@ -300,6 +300,37 @@ def test_horizon_workflow_classes(hx, oracle, kind):
     gc.close()
 
 
+def test_horizons_of_a_forest_whose_workflows_are_interleaved(hx, oracle):
+    """Node numbers in random order (no workflow is a contiguous range): the upload regroups such a forest along
+    another path than one listed workflow by workflow; both must give the oracle's horizons, and the same values
+    node for node as the ordered listing."""
+    wl = make_workload("medium", scale=0.25)
+    rng = np.random.default_rng(12)
+    N = wl.n_nodes
+    cost = rng.lognormal(0, 1, N).astype(np.float32)
+    new_id = rng.permutation(N).astype(np.uint32)                 # old node v becomes new_id[v]
+    old_of = np.argsort(new_id)
+    rows, cols = [0], []
+    for v_new in range(N):
+        v = old_of[v_new]
+        cols += [int(new_id[u]) for u in wl.col[wl.row_ptr[v]:wl.row_ptr[v + 1]]]
+        rows.append(len(cols))
+    wf_new, cost_new = wl.node_wf[old_of], cost[old_of]
+    assert (np.diff(wf_new.astype(np.int64)) < 0).any()           # really interleaved
+    gc = hh.gpu_cluster(wl)
+    gc.dag_upload(rows, cols, cost_new, wf_new, wl.elapsed)
+    gc.critical_path()
+    cp, tail, H = gc.dag_results()
+    r = oracle.longest_path(rows, cols, cost_new, wf_new, wl.n_workflows)
+    assert np.array_equal(cp, r.cp) and np.array_equal(tail, r.tail) and np.array_equal(H, r.H)
+    gc.dag_upload(wl.row_ptr, wl.col, cost, wl.node_wf, wl.elapsed)
+    gc.critical_path()
+    cp0, tail0, H0 = gc.dag_results()
+    assert np.array_equal(cp0, cp[new_id]) and np.array_equal(tail0, tail[new_id]) and np.array_equal(H0, H)
+    assert gc.status() == 0
+    gc.close()
+
+
 @pytest.mark.parametrize("name, scale, K", [("tiny", 1.0, 2), ("medium", 1.0, 4), ("large", 1 / 32, 4),
                                             ("cp_stress", 1 / 50, 1), ("sweep", 1 / 64, 4), ("sweep", 1 / 64, 8)])
 def test_topk_and_capacity_pass(hx, oracle, name, scale, K):
