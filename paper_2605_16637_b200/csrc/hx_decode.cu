@@ -60,14 +60,23 @@ struct DecodeParams {
     int* status;
 };
 
-// Segment index holding x in t[0..K): the largest k with t[k] <= x.  Executed by one warp.
+// Segment index holding x in t[0..K): the largest k with t[k] <= x.  Executed by one warp: up to 1,024
+// breakpoints in two rounds (every lane samples the start of one stretch, then the lanes share the stretch that
+// holds x), longer arrays 32 breakpoints at a time.
 __device__ __forceinline__ int warp_find_segment(const float* t, int K, float x, int lane) {
+    if (K <= 1024) {
+        const int stride = (K + 31) >> 5;
+        const int s = lane * stride;
+        const int b = __popc(__ballot_sync(0xffffffffu, s < K && t[s] <= x)) - 1;     // t[0] = 0 <= x always
+        const int i = b * stride + lane;
+        return b * stride + __popc(__ballot_sync(0xffffffffu, lane < stride && i < K && t[i] <= x)) - 1;
+    }
     int cnt = 0;
     for (int i0 = 0; i0 < K; i0 += 32) {
         const int i = i0 + lane;
         cnt += __popc(__ballot_sync(0xffffffffu, i < K && t[i] <= x));
     }
-    return cnt - 1;                                     // t[0] = 0 <= x always
+    return cnt - 1;
 }
 
 // Make x a breakpoint of instance arrays (t, u, K); returns its index.  One warp.
