@@ -626,8 +626,15 @@ int hx_cluster_create(const hx_gpu_type* gpu_types, int n_types, const hx_instan
     bool ok = true; cudaError_t first = cudaSuccess;
     auto up = [&](cudaError_t r) { if (r != cudaSuccess && ok) { ok = false; first = r; } };
     up(dev_upload(h->allocs, &d_invF, invF)); up(dev_upload(h->allocs, &d_invB, invB));
-    up(dev_upload(h->allocs, &d_qP, qP)); up(dev_upload(h->allocs, &d_qD, qD));
-    up(dev_upload(h->allocs, &d_capD, capD)); up(dev_upload(h->allocs, &d_freeD, freeD));
+    {   // prefill queues, decode hints and free KV tokens side by side: a refresh of all three is one copy
+        std::vector<float> loads;
+        loads.insert(loads.end(), qP.begin(), qP.begin() + P);
+        loads.insert(loads.end(), qD.begin(), qD.begin() + D);
+        loads.insert(loads.end(), freeD.begin(), freeD.begin() + D);
+        up(dev_upload(h->allocs, &d_qP, loads));
+        d_qD = d_qP + P; d_freeD = d_qD + D;
+    }
+    up(dev_upload(h->allocs, &d_capD, capD));
     up(dev_upload(h->allocs, &d_invLT, invLT)); up(dev_upload(h->allocs, &d_invLTt, invLTt));
     up(dev_upload(h->allocs, &d_phi, phi));
     up(dev_upload(h->allocs, &d_omega, omega)); up(dev_upload(h->allocs, &d_kappa, kappa));
@@ -655,6 +662,10 @@ int hx_cluster_update_loads(hx_cluster* h, const float* qP, const float* qD, con
             if (k == 2 && !good_tokens(src[k][i]))
                 return fail(h, HX_ERR_INVALID_ARG, "free KV tokens must be whole numbers in [0, 2^24)");
         }
+    }
+    if (qP && qD == qP + h->P && kv_free == qD + h->D) {         // laid out like the device tables: one copy
+        HX_TRY(cudaMemcpyAsync(h->tab.qP, qP, ((size_t)h->P + 2 * (size_t)h->D) * sizeof(float), cudaMemcpyHostToDevice, s), "cudaMemcpyAsync(loads)");
+        return HX_OK;
     }
     for (int k = 0; k < 3; ++k)
         if (src[k])

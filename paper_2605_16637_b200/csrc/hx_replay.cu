@@ -24,7 +24,7 @@ struct Buffers {                               // device scratch and page-locked
     float* delta = nullptr;
     unsigned char* pinned = nullptr;
     ~Buffers() {
-        cudaFree(calls); cudaFree(assign); cudaFree(ratio); cudaFree(order); cudaFree(delta);
+        cudaFree(calls); cudaFree(assign); cudaFree(ratio); cudaFree(order);   // delta lies behind assign
         cudaFreeHost(pinned);
     }
 };
@@ -82,10 +82,11 @@ extern "C" int hx_replay(hx_cluster* h, const uint32_t* row_ptr, const uint32_t*
         cudaStreamSynchronize(s) != cudaSuccess)
         return hx_fail(h, HX_ERR_CUDA, "reading capacities and horizons");
     Buffers b;
-    if (cudaMalloc(&b.calls, (size_t)qmax * sizeof(hx_call)) != cudaSuccess || cudaMalloc(&b.assign, (size_t)qmax * 4) != cudaSuccess ||
-        cudaMalloc(&b.ratio, (size_t)qmax * 4) != cudaSuccess || cudaMalloc(&b.order, (size_t)qmax * 4) != cudaSuccess ||
-        cudaMalloc(&b.delta, (size_t)qmax * 4) != cudaSuccess)
+    // pairs and projected completions side by side: one copy brings a plan back
+    if (cudaMalloc(&b.calls, (size_t)qmax * sizeof(hx_call)) != cudaSuccess || cudaMalloc(&b.assign, (size_t)qmax * 8) != cudaSuccess ||
+        cudaMalloc(&b.ratio, (size_t)qmax * 4) != cudaSuccess || cudaMalloc(&b.order, (size_t)qmax * 4) != cudaSuccess)
         return hx_fail(h, HX_ERR_OOM, "replay scratch");
+    b.delta = reinterpret_cast<float*>(b.assign + qmax);
 
     std::vector<uint32_t> left(N, 0);
     for (uint32_t e = 0; e < row_ptr[N]; ++e) ++left[col_idx[e]];
@@ -101,9 +102,12 @@ extern "C" int hx_replay(hx_cluster* h, const uint32_t* row_ptr, const uint32_t*
     if (cudaHostAlloc(&b.pinned, (size_t)qmax * sizeof(hx_call) + n_f32 * 4 + (size_t)qmax * 4, cudaHostAllocDefault) != cudaSuccess)
         return hx_fail(h, HX_ERR_OOM, "replay staging");
     hx_call* chunk = reinterpret_cast<hx_call*>(b.pinned);
+    // queue loads, decode hints and free tokens in the order of the device tables (one copy refreshes all three),
+    // pairs and completions in the order of the device results
     float* qP = reinterpret_cast<float*>(chunk + qmax);
-    float *qP2 = qP + P, *qD = qP2 + P, *kv_free = qD + D, *elapsed = kv_free + D, *delta = elapsed + W;
-    int32_t* assign = reinterpret_cast<int32_t*>(delta + qmax);
+    float *qD = qP + P, *kv_free = qD + D, *qP2 = kv_free + D, *elapsed = qP2 + P;
+    int32_t* assign = reinterpret_cast<int32_t*>(elapsed + W);
+    float* delta = reinterpret_cast<float*>(assign + qmax);
     for (int d = 0; d < D; ++d) qD[d] = 0.0f;
     std::vector<uint32_t> offered;
     std::vector<char> touched(P);
@@ -142,8 +146,7 @@ extern "C" int hx_replay(hx_cluster* h, const uint32_t* row_ptr, const uint32_t*
             if (cudaMemcpyAsync(b.calls, chunk, (size_t)n * sizeof(hx_call), cudaMemcpyHostToDevice, s) != cudaSuccess)
                 return leave(hx_fail(h, HX_ERR_CUDA, "copying the ready calls"));
             if ((rc = hx_schedule_greedy_plan(h, b.calls, n, b.assign, b.ratio, b.order, b.delta, stream)) != HX_OK) return leave(rc);
-            if (cudaMemcpyAsync(assign, b.assign, (size_t)n * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
-                cudaMemcpyAsync(delta, b.delta, (size_t)n * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+            if (cudaMemcpyAsync(assign, b.assign, (size_t)qmax * 8, cudaMemcpyDeviceToHost, s) != cudaSuccess)
                 return leave(hx_fail(h, HX_ERR_CUDA, "reading the plan"));
             if ((rc = hx_cluster_read_loads(h, qP2, nullptr, nullptr, stream)) != HX_OK) return leave(rc);   // synchronises
             ++runs;
@@ -241,10 +244,11 @@ extern "C" int hx_replay_lifecycle(hx_cluster* h, const hx_call* node_calls, con
     float *d_tp = nullptr, *d_td = nullptr, *d_kv = nullptr, *d_m = nullptr, *d_ratio = nullptr, *d_dstart = nullptr, *d_dratio = nullptr;
     int32_t *d_assign = nullptr, *d_order = nullptr, *d_lock = nullptr, *d_dinst = nullptr, *d_dorder = nullptr;
     if (!b.alloc(&d_all, N) || !b.alloc(&d_tp, (size_t)N * G) || !b.alloc(&d_td, (size_t)N * G) || !b.alloc(&d_kv, N) || !b.alloc(&d_m, N) ||
-        !b.alloc(&d_calls, qmax) || !b.alloc(&d_assign, qmax) || !b.alloc(&d_ratio, qmax) || !b.alloc(&d_order, qmax) ||
+        !b.alloc(&d_calls, qmax) || !b.alloc(&d_assign, 2 * (size_t)qmax) || !b.alloc(&d_ratio, qmax) ||
         !b.alloc(&d_dcalls, dmax) || !b.alloc(&d_lock, dmax) || !b.alloc(&d_dinst, dmax) || !b.alloc(&d_dstart, dmax) ||
         !b.alloc(&d_dratio, dmax) || !b.alloc(&d_dorder, dmax))
         return hx_fail(h, HX_ERR_OOM, "replay scratch");
+    d_order = d_assign + qmax;                 // pairs and order side by side: one copy brings a plan back
     // service times from the library's own estimator: the real ones and the ones the schedulers believe
     std::vector<float> tpre((size_t)N * G), tdec((size_t)N * G), tpre_s((size_t)N * G), tdec_s((size_t)N * G), kvB(N), m_tok(N);
     for (int pass = 0; pass < 2; ++pass) {
@@ -341,8 +345,7 @@ extern "C" int hx_replay_lifecycle(hx_cluster* h, const hx_call* node_calls, con
             if (cudaMemcpyAsync(d_calls, chunk, (size_t)n * sizeof(hx_call), cudaMemcpyHostToDevice, s) != cudaSuccess)
                 return leave(hx_fail(h, HX_ERR_CUDA, "copying the ready calls"));
             if ((rc = hx_schedule_greedy_plan(h, d_calls, n, d_assign, d_ratio, d_order, nullptr, stream)) != HX_OK) return leave(rc);
-            if (cudaMemcpyAsync(assign, d_assign, (size_t)n * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
-                cudaMemcpyAsync(order, d_order, (size_t)n * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+            if (cudaMemcpyAsync(assign, d_assign, (size_t)qmax * 8, cudaMemcpyDeviceToHost, s) != cudaSuccess ||   // pairs and order, side by side
                 cudaStreamSynchronize(s) != cudaSuccess)
                 return leave(hx_fail(h, HX_ERR_CUDA, "reading the plan"));
             ++runs;
