@@ -109,6 +109,8 @@ __global__ void __launch_bounds__(kThreads, 1) hx_decode_kernel(const __grid_con
     __shared__ float red_v[kWarps];
     __shared__ int red_c[kWarps];
     __shared__ int s_ndirty, s_cur, s_full;
+    __shared__ float part_v[kWarps], part_s[kWarps];   // partial projections of warps that share a call
+    __shared__ int part_d[kWarps];
     // most urgent call of every block with its interval: ratio, call, instance (int bits), start, finish, demand;
     // written by the owner block into every block, two sets used in turn by the iterations
     __shared__ float x_cand[2][NC][6];
@@ -199,10 +201,23 @@ __global__ void __launch_bounds__(kThreads, 1) hx_decode_kernel(const __grid_con
     if (tid == 0) s_ndirty = n;
     __syncthreads();
 
-    for (int it = 0; it < n_all; ++it) {
+    int it = 0;
+    // result of a projection: instance, start, finish and ratio of call c (no instance: it can never be taken)
+    auto record = [&](int c, float best, float bs, int bd) {
+        if (bd != 0x7fffffff) {
+            cbest[c] = bd; cstart[c] = bs; cfin[c] = best;
+            // one-pass ordering: the score of the first projection (against the snapshot) stays
+            if (it == 0 || !(prm.flags & HX_FLAG_ONE_PASS)) cR[c] = __fdiv_rn(__fadd_rn(cel[c], best), cH[c]);
+        } else { cbest[c] = kNoInst; cR[c] = HX_NEG_INF; }
+    };
+    for (; it < n_all; ++it) {
         // (1) project the listed calls: one warp per call, lanes over the decode instances
         const int nd = s_ndirty;
-        for (int i = warp; i < nd; i += kWarps) {
+        // few listed calls: two or four warps share a call, each walking a part of its instances; the parts are
+        // put together after the barrier
+        const int split = nd * 4 <= kWarps ? 4 : nd * 2 <= kWarps ? 2 : 1;
+        for (int w = warp; w < nd * split; w += kWarps) {
+            const int i = w / split, part = w - i * split;
             const int c = dirty[i];
             if (cbest[c] == kDead) continue;
             const float nt = cn[c], ot = co[c];
@@ -223,7 +238,7 @@ __global__ void __launch_bounds__(kThreads, 1) hx_decode_kernel(const __grid_con
                         // room in every segment (token counts are whole numbers, so the sum is exact): the walk
                         // would accept the ready time itself
                         const float fin = __fadd_rn(rd, tau);
-                        if (fin < best) { best = fin; bs = rd; bd = d; }
+                        if (part == 0 && fin < best) { best = fin; bs = rd; bd = d; }
                     } else {
                         walk = true;
                     }
@@ -232,9 +247,10 @@ __global__ void __launch_bounds__(kThreads, 1) hx_decode_kernel(const __grid_con
                 // the sequential walk stops at the first segment that either has no room (the candidate start moves
                 // to the end of the run of such segments) or ends at or after candidate + duration (accepted)
                 unsigned todo = __ballot_sync(0xffffffffu, walk);
-                while (todo) {
+                for (int turn = 0; todo; ++turn) {
                     const int src = __ffs(todo) - 1;
                     todo &= todo - 1;
+                    if (turn % split != part) continue;           // another warp's instance
                     const int dd = d0 + src;
                     const float tau_d = __shfl_sync(0xffffffffu, tau, src);
                     const float* tt = seg_t(dd);
@@ -276,14 +292,22 @@ __global__ void __launch_bounds__(kThreads, 1) hx_decode_kernel(const __grid_con
                 if (ov < best || (ov == best && od < bd)) { best = ov; bs = os; bd = od; }
             }
             if (lane == 0) {
-                if (bd != 0x7fffffff) {
-                    cbest[c] = bd; cstart[c] = bs; cfin[c] = best;
-                    // one-pass ordering: the score of the first projection (against the snapshot) stays
-                    if (it == 0 || !(prm.flags & HX_FLAG_ONE_PASS)) cR[c] = __fdiv_rn(__fadd_rn(cel[c], best), cH[c]);
-                } else { cbest[c] = kNoInst; cR[c] = HX_NEG_INF; }
+                if (split > 1) { part_v[w] = best; part_s[w] = bs; part_d[w] = bd; }
+                else record(c, best, bs, bd);
             }
         }
         __syncthreads();
+        if (split > 1) {
+            if (tid < nd && cbest[dirty[tid]] != kDead) {
+                float best = HX_INF, bs = 0.f; int bd = 0x7fffffff;
+                for (int k = 0; k < split; ++k) {
+                    const float ov = part_v[tid * split + k]; const int od = part_d[tid * split + k];
+                    if (ov < best || (ov == best && od < bd)) { best = ov; bs = part_s[tid * split + k]; bd = od; }
+                }
+                record(dirty[tid], best, bs, bd);
+            }
+            __syncthreads();
+        }
         // (2) most urgent waiting call of this block
         float rv = HX_NEG_INF; int rc = 0x7fffffff;
         for (int c = tid; c < n; c += kThreads) {
