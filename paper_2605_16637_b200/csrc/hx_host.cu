@@ -499,6 +499,18 @@ void hx_cluster_shape(const hx_cluster* h, int* P, int* D, const float** capD_de
 }
 hx_options hx_current_options(const hx_cluster* h) { return h->opts; }
 
+int hx_update_loads_packed(hx_cluster* h, const float* packed, cudaStream_t s) {
+    const size_t n = (size_t)h->P + 2 * (size_t)h->D;
+    for (size_t i = 0; i < n; ++i) {
+        if (!good_load(packed[i])) return fail(h, HX_ERR_INVALID_ARG, "loads must be finite and >= 0");
+        if (i >= (size_t)h->P + h->D && !good_tokens(packed[i]))
+            return fail(h, HX_ERR_INVALID_ARG, "free KV tokens must be whole numbers in [0, 2^24)");
+    }
+    DeviceGuard guard(h->device);
+    HX_TRY(cudaMemcpyAsync(h->tab.qP, packed, n * sizeof(float), cudaMemcpyHostToDevice, s), "cudaMemcpyAsync(loads)");
+    return HX_OK;
+}
+
 int hx_cluster_tables_host(hx_cluster* h, std::vector<int>* typeP, std::vector<int>* typeD, std::vector<float>* invLT,
                            int* Ppad, int* G, int* M, cudaStream_t s) {
     typeP->resize(h->Ppad); typeD->resize(h->D); invLT->resize((size_t)h->D * h->Ppad);
@@ -662,10 +674,6 @@ int hx_cluster_update_loads(hx_cluster* h, const float* qP, const float* qD, con
             if (k == 2 && !good_tokens(src[k][i]))
                 return fail(h, HX_ERR_INVALID_ARG, "free KV tokens must be whole numbers in [0, 2^24)");
         }
-    }
-    if (qP && qD == qP + h->P && kv_free == qD + h->D) {         // laid out like the device tables: one copy
-        HX_TRY(cudaMemcpyAsync(h->tab.qP, qP, ((size_t)h->P + 2 * (size_t)h->D) * sizeof(float), cudaMemcpyHostToDevice, s), "cudaMemcpyAsync(loads)");
-        return HX_OK;
     }
     for (int k = 0; k < 3; ++k)
         if (src[k])

@@ -221,6 +221,9 @@ int hx_cluster_tables_host(hx_cluster* h, std::vector<int>* typeP, std::vector<i
 void hx_forest_host(const hx_cluster* h, std::vector<uint32_t>* row, std::vector<uint32_t>* col, std::vector<uint32_t>* node_wf);
 // Every model once more with its constants scaled by up and by down (models M .. 2M - 1 and 2M .. 3M - 1), until
 // hx_pop_scaled_models; HX_ERR_INVALID_ARG when three times the models do not fit the table.
+// hx_cluster_update_loads from ONE host array laid out like the device tables (prefill queues, decode hints, free KV
+// tokens: P + 2 D values of one allocation): a single copy.
+int hx_update_loads_packed(hx_cluster* h, const float* packed, cudaStream_t s);
 int hx_push_scaled_models(hx_cluster* h, float up, float down);
 void hx_pop_scaled_models(hx_cluster* h);
 

@@ -141,7 +141,7 @@ extern "C" int hx_replay(hx_cluster* h, const uint32_t* row_ptr, const uint32_t*
             for (int d = 0; d < D; ++d) kv_free[d] = (float)((double)cap[d] - used[d]);
             for (uint32_t w = 0; w < W; ++w) elapsed[w] = (float)std::max(0.0, t - arrival_s[w]);
             for (int i = 0; i < n; ++i) chunk[i] = node_calls[offered[o + i]];
-            if ((rc = hx_cluster_update_loads(h, qP, qD, kv_free, stream)) != HX_OK) return leave(rc);
+            if ((rc = hx_update_loads_packed(h, qP, s)) != HX_OK) return leave(rc);
             if ((rc = hx_dag_update_elapsed(h, elapsed, stream)) != HX_OK) return leave(rc);
             if (cudaMemcpyAsync(b.calls, chunk, (size_t)n * sizeof(hx_call), cudaMemcpyHostToDevice, s) != cudaSuccess)
                 return leave(hx_fail(h, HX_ERR_CUDA, "copying the ready calls"));
@@ -340,7 +340,7 @@ extern "C" int hx_replay_lifecycle(hx_cluster* h, const hx_call* node_calls, con
             }
             for (int d = 0; d < D; ++d) kv_free[d] = (float)((double)cap[d] - reserved[d]);
             for (int i = 0; i < n; ++i) chunk[i] = seen[offered[o + i]];
-            if ((rc = hx_cluster_update_loads(h, qP, qD, kv_free, stream)) != HX_OK) return leave(rc);
+            if ((rc = hx_update_loads_packed(h, qP, s)) != HX_OK) return leave(rc);
             if (!elapsed_sent) { if ((rc = hx_dag_update_elapsed(h, elapsed, stream)) != HX_OK) return leave(rc); elapsed_sent = true; }
             if (cudaMemcpyAsync(d_calls, chunk, (size_t)n * sizeof(hx_call), cudaMemcpyHostToDevice, s) != cudaSuccess)
                 return leave(hx_fail(h, HX_ERR_CUDA, "copying the ready calls"));
