@@ -21,13 +21,14 @@
 // time: a segment without room moves the candidate start to its end, and the
 // candidate is accepted once a segment ends at or after candidate + duration.
 // One persistent block; one warp projects one call with the lanes over the
-// instances; adding an interval only delays starts on that instance, so only
+// instances (two or four warps share a call when few calls are listed); adding
+// an interval only delays starts on that instance, so only
 // calls whose best instance it was are projected again.
 //
 // Long queues run on a thread-block cluster: call c belongs to block c mod kCluster, every block
-// keeps its own copy of the step functions, and per iteration the blocks exchange their most urgent
-// call and the winner's interval through distributed shared memory with two cluster barriers; all
-// blocks reduce the same candidates and insert the same interval, so the copies stay identical and
+// keeps its own copy of the step functions, and per iteration every block writes its most urgent call
+// with its interval into all blocks through distributed shared memory, behind one cluster barrier (two
+// sets of slots used in turn); all blocks reduce the same candidates and insert the same interval, so the copies stay identical and
 // every exit is taken by all blocks.
 #include <cooperative_groups.h>
 

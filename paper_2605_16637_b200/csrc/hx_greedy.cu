@@ -24,13 +24,15 @@
 // tells) or its decode instance no longer has room for the call (room only
 // shrinks, so the test at the time of use is exact); a re-projection recomputes
 // the rows that are not, D candidates each, and takes the minimum over the rows
-// instead of walking all P x D pairs.
+// instead of walking all P x D pairs: three block-wide passes over the listed
+// calls (find the rows, recompute them with four lanes each, reduce).
 //
 // Long queues run on a thread-block cluster of kCluster blocks (one SM each): call c belongs to
 // block c mod kCluster, every block keeps its own copy of the small simulated state, and per
-// iteration the blocks exchange their most urgent call and the winner's commit through
-// distributed shared memory with two cluster barriers.  All blocks reduce the same candidates and
-// apply the same commit, so their copies stay identical and every exit is taken by all of them.
+// iteration every block writes its most urgent call, with what its commit would change, into all
+// blocks through distributed shared memory, behind one cluster barrier (two sets of slots used in
+// turn).  All blocks reduce the same candidates and apply the same commit, so their copies stay
+// identical and every exit is taken by all of them.
 #include <cooperative_groups.h>
 
 #include "hx_internal.h"
