@@ -37,6 +37,18 @@ def test_binding_mirrors_the_header(hx):
         assert hasattr(hx, n), "binding lacks " + n
 
 
+def test_binding_constants_equal_the_header_macros(hx):
+    text = open(os.path.join(ROOT, "include", "hx.h")).read()
+    macros = {k: int(v, 0) for k, v in re.findall(r"#define\s+(HX_[A-Z_0-9]+)\s+(-?(?:0x[0-9A-Fa-f]+|\d+))\b", text)}
+    assert macros["HX_FLAG_ONE_PASS"] == 8 and macros["HX_OK"] == 0
+    checked = 0
+    for name, value in macros.items():
+        if hasattr(hx, name):
+            assert getattr(hx, name) == value, name
+            checked += 1
+    assert checked >= 6                                          # the flags and score modes at least
+
+
 def test_built_for_sm_100a():
     import importlib.util
     spec = importlib.util.spec_from_file_location("_b", os.path.join(ROOT, "paper_2605_16637_b200", "build.py"))
