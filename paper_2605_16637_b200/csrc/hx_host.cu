@@ -7,6 +7,7 @@
 #include <cstring>
 #include <mutex>
 #include <new>
+#include <system_error>
 #include <thread>
 #include <unordered_map>
 
@@ -324,8 +325,12 @@ bool regroup_workflow_by_workflow(const uint32_t* row_ptr, const uint32_t* col_i
         work(0);
     } else {
         std::vector<std::thread> pool;
-        for (uint32_t k = 1; k < n_workers; ++k) pool.emplace_back(work, k);
+        uint32_t started = 1;                          // stretches that have a thread of their own (0 runs here)
+        try {
+            for (; started < n_workers; ++started) pool.emplace_back(work, started);
+        } catch (const std::system_error&) {}          // no more threads to be had: this one takes the rest
         work(0);
+        for (uint32_t k = started; k < n_workers; ++k) work(k);
         for (auto& th : pool) th.join();
     }
     for (char f : failed) if (f) return false;
