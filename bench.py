@@ -244,10 +244,11 @@ def run_cuda(args):
     def step_device(sp, strm=None, chunk_events=None):
         hx.hx_critical_path(h, sp)
         hx.hx_cluster_update_loads(h, qP0, qD0, free0, sp)
+        # decode completions between two scheduler invocations: every capacity pass starts from free0 again
+        hx.hx_set_kv_free_restore(h, free0, sp)
         for i in range(n_chunks):
             if chunk_events is not None:
                 chunk_events[i][0].record(strm)
-            hx.hx_cluster_update_loads(h, None, None, free0, sp)
             hx.hx_schedule_batch(h, ptrs[i][0], chunk, ptrs[i][1], ptrs[i][2], sp)
             if chunk_events is not None:
                 chunk_events[i][1].record(strm)

@@ -123,6 +123,19 @@ int hx_cluster_create(const hx_gpu_type* gpu_types, int n_types,
 int hx_cluster_update_loads(hx_cluster* h, const float* qP, const float* qD,
                             const float* kv_free, void* stream);
 
+/* Capacity restored between scheduler invocations (decode completions free KV
+ * tokens while the scheduler is not looking): with kv_free != NULL (host,
+ * n_decode whole numbers below 2^24) every capacity-conflict pass from now on
+ * starts from these free KV tokens instead of the table's, exactly as if
+ * hx_cluster_update_loads(h, NULL, NULL, kv_free) had been enqueued ahead of
+ * every batch, but without a copy between the kernels of successive batches;
+ * the table is set to the same values at once, and a committing pass still
+ * writes what it leaves into the table.  NULL switches this off (enqueues
+ * nothing).  Only batches with topk > 0 read free KV tokens.  The copies are
+ * enqueued on `stream`; the host array may be reused when the call returns.
+ * HX_ERR_INVALID_ARG for a bad value, nothing changed. */
+int hx_set_kv_free_restore(hx_cluster* h, const float* kv_free, void* stream);
+
 /* Read the current loads back (after commits).  Synchronises `stream`. */
 int hx_cluster_read_loads(hx_cluster* h, float* qP, float* qD, float* kv_free, void* stream);
 
@@ -295,7 +308,8 @@ int hx_schedule_batch_host_async(hx_cluster* h, const hx_call* calls, int n_call
  * (the commits of a chunk are the snapshot of the next).  When kv_free_reset is
  * not NULL (host, n_decode values) the free KV tokens of the decode instances
  * are set to it ahead of every chunk (decode completions between two scheduler
- * invocations), as hx_cluster_update_loads(h, NULL, NULL, kv_free_reset) would.
+ * invocations), as hx_cluster_update_loads(h, NULL, NULL, kv_free_reset) would
+ * (done through hx_set_kv_free_restore, which is switched off again on return).
  * Unlike a loop over the per-chunk call, the records of all chunks go up on a
  * copy stream of the handle ahead of the kernels, and the results of a chunk
  * come down on a second copy stream while the next chunk is being scored; the

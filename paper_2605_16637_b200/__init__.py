@@ -7,7 +7,7 @@ paper_2605_16637_b200.build); there is no CPU fallback.
 """
 from .api import (CALL_DTYPE, INSTANCE_DTYPE, HX_FLAG_NO_DAG, HX_FLAG_NO_TAIL, HX_FLAG_UNLOADED, HX_FLAG_ONE_PASS,
                   HX_MODE_COMPLETION, HX_MODE_RATIO, HX_MODE_SLACK, HxError, Cluster,
-                  hx_cluster_create, hx_cluster_destroy, hx_cluster_read_loads,
+                  hx_cluster_create, hx_cluster_destroy, hx_cluster_read_loads, hx_set_kv_free_restore,
                   hx_cluster_update_loads, hx_critical_path, hx_enable_kernel_timing,
                   hx_read_kernel_timing, hx_dag_upload, hx_dag_update_costs, hx_dag_update_elapsed, hx_get_dag_results,
                   hx_dag_append, hx_earliest_start, hx_get_earliest_results,

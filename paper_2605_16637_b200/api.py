@@ -49,6 +49,7 @@ def _load():
         "hx_cluster_create": [vp, ci, vp, ci, vp, vp, ci, C.POINTER(vp)],
         "hx_cluster_update_loads": [vp, vp, vp, vp, vp],
         "hx_cluster_read_loads": [vp, vp, vp, vp, vp],
+        "hx_set_kv_free_restore": [vp, vp, vp],
         "hx_cluster_destroy": [vp],
         "hx_dag_upload": [vp, vp, vp, vp, vp, vp, u32, u32, u32],
         "hx_critical_path": [vp, vp],
@@ -123,6 +124,11 @@ def hx_cluster_create(gpu_types, instances, link_bw_gbps, models):
 def hx_cluster_update_loads(h, qP=None, qD=None, kv_free=None, stream=0):
     arrs = [None if a is None else _np(a, np.float32) for a in (qP, qD, kv_free)]
     _check(_lib.hx_cluster_update_loads(h, _p(arrs[0]), _p(arrs[1]), _p(arrs[2]), stream), h)
+
+
+def hx_set_kv_free_restore(h, kv_free=None, stream=0):
+    a = None if kv_free is None else _np(kv_free, np.float32)
+    _check(_lib.hx_set_kv_free_restore(h, _p(a), stream), h)
 
 
 def hx_cluster_read_loads(h, n_prefill, n_decode, stream=0):
@@ -411,6 +417,11 @@ class Cluster:
 
     def update_loads(self, qP=None, qD=None, kv_free=None):
         hx_cluster_update_loads(self.h, qP, qD, kv_free, self._stream())
+
+    def set_kv_free_restore(self, kv_free=None):
+        if kv_free is not None and np.asarray(kv_free).shape[0] != self.D:
+            raise HxError(-1, "one value per decode instance is needed")
+        hx_set_kv_free_restore(self.h, kv_free, self._stream())
 
     def read_loads(self):
         return hx_cluster_read_loads(self.h, self.P, self.D, self._stream())

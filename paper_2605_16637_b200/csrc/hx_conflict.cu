@@ -303,7 +303,8 @@ constexpr int kRing = 2048;        // staged calls waiting for the window warp (
 constexpr int kDrain = 96;         // the windows run once this many calls are staged (or the order is exhausted)
 template <int KT>   // candidate slots examined per call: K rounded up to 1, 2, 4 or 8
 __global__ void __launch_bounds__(kPassThreads, 1) hx_conflict_kernel(HxTopkBufs tk, HxTables t, int n, int commit,
-                                                                      int fused_tail, int32_t* out_assign) {
+                                                                      int fused_tail, int32_t* out_assign,
+                                                                      const float* free_reset) {
     extern __shared__ __align__(16) unsigned sm[];
     constexpr int NW = kPassThreads / 32;
     static_assert(NW == 32, "the staging step keeps one warp total per lane");
@@ -321,7 +322,10 @@ __global__ void __launch_bounds__(kPassThreads, 1) hx_conflict_kernel(HxTopkBufs
     // the scoring kernel of the next batch may take the other SMs and do the part of its set-up that reads
     // nothing a kernel writes; it waits for this grid before it goes on, and releases its own dependents after
     hx_release_dependents();
-    for (int d = tid; d <= D; d += kPassThreads) free_s[d] = d < D ? __float2int_rd(t.freeD[d]) : -1;
+    // free KV tokens the pass starts from: the table's, or the values the capacity is restored to ahead of every
+    // batch (neither is written by a kernel that may still run: the same grid of the batch before wrote the table)
+    const float* free0 = free_reset ? free_reset : t.freeD;
+    for (int d = tid; d <= D; d += kPassThreads) free_s[d] = d < D ? __float2int_rd(free0[d]) : -1;
     hx_wait_for_primary();                                      // the visiting order
     __syncthreads();
     auto narrow = [&](const uint4& r) {                         // the slots this instantiation examines
@@ -511,7 +515,7 @@ __global__ void __launch_bounds__(32 * kQWarps) hx_qsum_kernel(HxTopkBufs tk, Hx
 
 cudaError_t hx_launch_conflict(const HxTables& t, const HxTopkBufs& tk, int n_calls, int commit,
                                int32_t* out_assign, int* status, cudaStream_t stream,
-                               long long* launches) {
+                               long long* launches, const float* free_reset) {
     (void)status;
     const int D = t.D, P = t.P;
     const int nb = (n_calls + kOrdThreads - 1) / kOrdThreads;
@@ -530,7 +534,7 @@ cudaError_t hx_launch_conflict(const HxTables& t, const HxTopkBufs& tk, int n_ca
     static size_t allowed_pass[4][64];
     e = hx_opt_in_smem(pass, smC, allowed_pass[tk.K <= 1 ? 0 : tk.K <= 2 ? 1 : tk.K <= 4 ? 2 : 3], 40 * 1024);
     if (e != cudaSuccess) return e;
-    e = hx_launch_dependent(pass, dim3(1), dim3(kPassThreads), smC, stream, tk, t, n_calls, commit, fused, out_assign);
+    e = hx_launch_dependent(pass, dim3(1), dim3(kPassThreads), smC, stream, tk, t, n_calls, commit, fused, out_assign, free_reset);
     if (e != cudaSuccess) return e;
     *launches += 4;
     if (!fused) {

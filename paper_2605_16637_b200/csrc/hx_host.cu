@@ -107,6 +107,8 @@ struct hx_cluster {
     HxTopkBufs tk{};
     // staging for the host-buffer entry point
     hx_call* st_calls = nullptr; int32_t* st_assign = nullptr; float* st_cost = nullptr; int st_cap = 0;
+    float* d_free_reset = nullptr;      // [D] free KV tokens every capacity pass starts from while free_reset_on
+    bool free_reset_on = false;
     // copy streams and events of hx_schedule_sweep_host, created on first use
     cudaStream_t sw_in = nullptr, sw_out = nullptr;
     std::vector<cudaEvent_t> sw_ev;
@@ -657,6 +659,7 @@ int hx_cluster_create(const hx_gpu_type* gpu_types, int n_types, const hx_instan
     up(dev_upload(h->allocs, &d_omega, omega)); up(dev_upload(h->allocs, &d_kappa, kappa));
     up(dev_upload(h->allocs, &d_typeP, typeP)); up(dev_upload(h->allocs, &d_typeD, typeD));
     up(dev_alloc(h->allocs, &h->status, 2));                // status word, and a sink for the issue-rate kernels
+    up(dev_alloc(h->allocs, &h->d_free_reset, (size_t)D));
     if (ok) up(cudaMemset(h->status, 0, 2 * sizeof(int)));
     if (!ok) return bail(fail_cuda(h, first, "uploading cluster tables"));
     h->tab = HxTables{n_types, P, D, n_models, h->Ppad, d_invF, d_invB, d_typeP, d_typeD, d_qP, d_qD,
@@ -683,6 +686,20 @@ int hx_cluster_update_loads(hx_cluster* h, const float* qP, const float* qD, con
     for (int k = 0; k < 3; ++k)
         if (src[k])
             HX_TRY(cudaMemcpyAsync(dst[k], src[k], n[k] * sizeof(float), cudaMemcpyHostToDevice, s), "cudaMemcpyAsync(loads)");
+    return HX_OK;
+}
+
+int hx_set_kv_free_restore(hx_cluster* h, const float* kv_free, void* stream) {
+    if (!h) return HX_ERR_INVALID_ARG;
+    if (!kv_free) { h->free_reset_on = false; return HX_OK; }
+    for (int d = 0; d < h->D; ++d)
+        if (!good_tokens(kv_free[d])) return fail(h, HX_ERR_INVALID_ARG, "free KV tokens must be whole numbers in [0, 2^24)");
+    DeviceGuard guard(h->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    HX_TRY(cudaMemcpyAsync(h->d_free_reset, kv_free, h->D * sizeof(float), cudaMemcpyHostToDevice, s), "cudaMemcpyAsync(kv_free)");
+    // the table holds the same values until a pass commits: what a read-back shows without a commit
+    HX_TRY(cudaMemcpyAsync(h->tab.freeD, h->d_free_reset, h->D * sizeof(float), cudaMemcpyDeviceToDevice, s), "cudaMemcpyAsync(kv_free)");
+    h->free_reset_on = true;
     return HX_OK;
 }
 
@@ -1229,7 +1246,8 @@ int hx_schedule_batch(hx_cluster* h, const hx_call* calls, int n_calls, int32_t*
     }
     if (o.topk > 0) {
         SpanGuard span(h, 1, s);
-        HX_TRY(hx_launch_conflict(h->tab, tk, n_calls, o.commit, out_assign, h->status, s, &h->launches), "conflict pass");
+        HX_TRY(hx_launch_conflict(h->tab, tk, n_calls, o.commit, out_assign, h->status, s, &h->launches,
+                                  h->free_reset_on ? h->d_free_reset : nullptr), "conflict pass");
     }
     return HX_OK;
 }
@@ -1308,6 +1326,14 @@ int hx_schedule_sweep_host(hx_cluster* h, const hx_call* calls, int n_calls, int
     HX_TRY(cudaEventRecord(ev_start, s), "event");
     HX_TRY(cudaStreamWaitEvent(h->sw_in, ev_start, 0), "event");
     HX_TRY(cudaStreamWaitEvent(h->sw_out, ev_start, 0), "event");
+    // the free KV tokens every chunk starts from: one copy, then every capacity pass reads them itself (a copy ahead
+    // of every chunk would sit between the pass of one chunk and the scoring kernel of the next)
+    if (kv_free_reset)
+        if (int rc = hx_set_kv_free_restore(h, kv_free_reset, stream)) return rc;
+    struct RestoreOff {                                  // the values given here hold for this sweep only
+        hx_cluster* h; bool mine;
+        ~RestoreOff() { if (mine) h->free_reset_on = false; }
+    } restore_off{h, kv_free_reset != nullptr};
     // every chunk's records go up on their own stream, ahead of the kernels that need them
     for (int c = 0; c < n_chunks; ++c) {
         const size_t o = (size_t)c * chunk_calls, n = std::min<size_t>(chunk_calls, (size_t)n_calls - o);
@@ -1317,8 +1343,6 @@ int hx_schedule_sweep_host(hx_cluster* h, const hx_call* calls, int n_calls, int
     for (int c = 0; c < n_chunks; ++c) {
         const size_t o = (size_t)c * chunk_calls, n = std::min<size_t>(chunk_calls, (size_t)n_calls - o);
         HX_TRY(cudaStreamWaitEvent(s, h->sw_ev[2 + c], 0), "event");
-        if (kv_free_reset)
-            HX_TRY(cudaMemcpyAsync(h->tab.freeD, kv_free_reset, h->D * sizeof(float), cudaMemcpyHostToDevice, s), "cudaMemcpyAsync(loads)");
         const int rc = hx_schedule_batch(h, h->st_calls + o, (int)n, h->st_assign + o, h->st_cost + o, stream);
         if (rc != HX_OK) {                               // leave no stream waiting on work that will never come
             cudaEventRecord(ev_done, h->sw_out); cudaStreamWaitEvent(s, ev_done, 0);
@@ -1429,7 +1453,8 @@ int hx_schedule_batch_static(hx_cluster* h, const hx_call* calls, int n_calls, i
     }
     if (o.topk > 0) {
         SpanGuard span(h, 1, s);
-        HX_TRY(hx_launch_conflict(h->tab, b, n_calls, o.commit, out_assign, h->status, s, &h->launches), "conflict pass");
+        HX_TRY(hx_launch_conflict(h->tab, b, n_calls, o.commit, out_assign, h->status, s, &h->launches,
+                                  h->free_reset_on ? h->d_free_reset : nullptr), "conflict pass");
     }
     return HX_OK;
 }

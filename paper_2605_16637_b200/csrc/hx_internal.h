@@ -133,7 +133,7 @@ cudaError_t hx_launch_score(const HxTables& t, const HxConstTables& ct, const Hx
 
 cudaError_t hx_launch_conflict(const HxTables& t, const HxTopkBufs& tk, int n_calls, int commit,
                                int32_t* out_assign, int* status, cudaStream_t stream,
-                               long long* launches);
+                               long long* launches, const float* free_reset = nullptr);
 
 cudaError_t hx_launch_estimate(const HxConstTables& ct, int G, int M, const hx_call* calls, int n_calls,
                                float* tpre, float* tdec, float* kvB, float* m, int* status, cudaStream_t stream,

@@ -518,6 +518,42 @@ def test_sweep_entry_point_equals_the_batches_one_by_one(hx, oracle, reset):
     gc.close()
 
 
+@pytest.mark.parametrize("commit", [1, 0])
+def test_restored_capacity_equals_a_load_refresh_ahead_of_every_batch(hx, oracle, commit):
+    """hx_set_kv_free_restore once against hx_cluster_update_loads(kv_free) ahead of every batch: same pairs, costs
+    and loads after every batch; switched off, the committed capacities carry over again; a bad value changes nothing."""
+    wl = make_workload("sweep", scale=1 / 32)
+    oc, gc, dag = _prepare(hx, oracle, wl)
+    gc.set_options(score_mode=hx.HX_MODE_RATIO, topk=4, commit=commit, alpha=wl.alpha)
+    qP0, free0 = wl.load_s[:wl.P].copy(), wl.kv_free[wl.P:].copy()
+    n, chunks = 2000, 4
+    want = []
+    gc.update_loads(qP=qP0, kv_free=free0)
+    for i in range(chunks):
+        gc.update_loads(kv_free=free0)
+        a, c = gc.schedule_batch(wl.calls[i * n:(i + 1) * n])
+        want.append((a.cpu().numpy(), c.cpu().numpy(), gc.read_loads()))
+    gc.update_loads(qP=qP0, kv_free=np.zeros_like(free0))    # the table itself says "nothing free": the restore must win
+    gc.set_kv_free_restore(free0)
+    for i in range(chunks):
+        a, c = gc.schedule_batch(wl.calls[i * n:(i + 1) * n])
+        assert np.array_equal(a.cpu().numpy(), want[i][0]) and np.array_equal(c.cpu().numpy(), want[i][1])
+        for x, y in zip(gc.read_loads(), want[i][2]):
+            assert np.array_equal(x, y)
+    assert (want[0][0] >= 0).any() and gc.status() == 0
+    bad = free0.copy(); bad[0] = 10.5
+    with pytest.raises(hx.HxError):
+        gc.set_kv_free_restore(bad)
+    a, c = gc.schedule_batch(wl.calls[:n])                    # still restored to free0
+    if commit == 0:
+        assert np.array_equal(a.cpu().numpy(), want[0][0])
+    gc.set_kv_free_restore(None)                              # off: the table's values count again
+    gc.update_loads(qP=qP0, kv_free=np.zeros_like(free0))
+    a, c = gc.schedule_batch(wl.calls[:n])
+    assert (a.cpu().numpy() == -1).all()
+    gc.close()
+
+
 @pytest.mark.parametrize("P, D, n", [(4, 9, 300), (70, 130, 700)])
 def test_quadratic_prefill_variant(hx, oracle, P, D, n):
     """Attention FLOPs per token pair set on both sides: scoring, top-K lists and the greedy planner agree
