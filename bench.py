@@ -3,8 +3,8 @@
 
 One step = one pass of the whole path over the sweep configuration: horizon
 kernels over the workflow forest, then 16 scheduler invocations of 16,384 ready
-calls each against 128 x 128 instance pairs (load refresh, scoring with top-4
-lists, capacity-conflict pass with commit).  Prints one JSON line.
+calls each against 128 x 128 instance pairs (scoring with top-4 lists,
+capacity-conflict pass that starts from the restored free KV tokens, commit).  Prints one JSON line.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
 """
@@ -429,8 +429,8 @@ def run_cuda(args):
                                     "found none of their four candidate decode instances with room"},
         "schedule_latency": {"batch_calls": chunk, "p50_us": float(np.percentile(chunk_us, 50)),
                              "p95_us": float(np.percentile(chunk_us, 95)),
-                             "what": "load refresh + hx_schedule_batch (scoring, top-4, conflict pass, commit) per "
-                                     "ready batch, CUDA events"},
+                             "what": "hx_schedule_batch (scoring, top-4, conflict pass starting from the restored free KV "
+                                     "tokens, commit) per ready batch, CUDA events"},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "what": "hx_schedule_sweep_host (all 16 chunks, copies on their own streams) from pinned host memory into "
                         "pinned host memory, one synchronisation per step, wall clock"},

@@ -86,7 +86,6 @@ __device__ __forceinline__ unsigned bin_of(unsigned key, unsigned lo, unsigned s
 __global__ void __launch_bounds__(kOrdThreads) hx_order_hist_kernel(HxTopkBufs tk, int n) {
     __shared__ unsigned lohi[2], wfirst[kOrdThreads / 32];
     const int tid = threadIdx.x;
-    hx_release_dependents();
     if (tid == 0) { lohi[0] = 0xFFFFFFFFu; lohi[1] = 0u; }
     __syncthreads();
     hx_wait_for_primary();                                        // the scoring kernel's key ranges, priorities and cleared counters
@@ -126,7 +125,6 @@ __global__ void __launch_bounds__(kOrdThreads) hx_order_hist_kernel(HxTopkBufs t
 __global__ void __launch_bounds__(kOrdThreads) hx_order_scatter_kernel(HxTopkBufs tk, int n) {
     __shared__ unsigned hist[kBins], base[kBins + 1], tmp[33];
     const int tid = threadIdx.x;
-    hx_release_dependents();
     hx_wait_for_primary();                                        // the complete bin counters
     for (int i = tid; i < kBins; i += kOrdThreads) hist[i] = __ldcg(tk.ghist + i);
     __syncthreads();
@@ -158,7 +156,6 @@ __global__ void __launch_bounds__(kRankThreads) hx_order_rank_kernel(HxTopkBufs 
     __shared__ unsigned range[2];
     const int tid = threadIdx.x;
     const int i = blockIdx.x * kRankThreads + tid;
-    hx_release_dependents();
     hx_wait_for_primary();                                        // every key is in its bin
     const bool valid = i < n;
     const unsigned lo = tk.obase[kBins + 1], shift = tk.obase[kBins + 2];
@@ -519,8 +516,8 @@ cudaError_t hx_launch_conflict(const HxTables& t, const HxTopkBufs& tk, int n_ca
     (void)status;
     const int D = t.D, P = t.P;
     const int nb = (n_calls + kOrdThreads - 1) / kOrdThreads;
-    // every kernel of the pass may become resident while the one before it drains; each waits for its
-    // predecessor before reading what that one wrote
+    // every kernel of the pass is made ready while the one before it drains (released when its blocks exit);
+    // each waits for its predecessor before reading what that one wrote
     cudaError_t e = hx_launch_dependent(hx_order_hist_kernel, dim3(nb), dim3(kOrdThreads), 0, stream, tk, n_calls);
     if (e == cudaSuccess) e = hx_launch_dependent(hx_order_scatter_kernel, dim3(nb), dim3(kOrdThreads), 0, stream, tk, n_calls);
     if (e == cudaSuccess) e = hx_launch_dependent(hx_order_rank_kernel, dim3((n_calls + kRankThreads - 1) / kRankThreads), dim3(kRankThreads), 0, stream, tk, n_calls, (unsigned)D);

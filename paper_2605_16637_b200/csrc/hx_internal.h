@@ -228,9 +228,14 @@ int hx_push_scaled_models(hx_cluster* h, float up, float down);
 void hx_pop_scaled_models(hx_cluster* h);
 
 // Programmatic dependent launch: a kernel launched with hx_launch_dependent may be made resident while the
-// kernel before it on the stream is still running (that kernel calls hx_release_dependents() early); it must
-// call hx_wait_for_primary() before it touches anything the earlier kernel writes.  The wait returns once the
-// earlier grid has completed and its writes are visible; launched the ordinary way both calls do nothing.
+// kernel before it on the stream is still running, once every block of that kernel has called
+// hx_release_dependents() or exited; it must call hx_wait_for_primary() before it touches anything the earlier
+// kernel writes.  The wait returns once the earlier grid has completed and its writes are visible; launched the
+// ordinary way both calls do nothing.  The attribute is kept inside a stream capture (the replayed graph gets
+// programmatic edges).  Measured on the sweep step: a kernel that releases its dependents long before it ends
+// slows the step down unless the dependent has real work to do ahead of its wait (the scoring kernel behind the
+// capacity pass has, the binning kernel behind the scoring kernel has not: 1.72 against 1.64 ms per step), so
+// only the pass releases early.
 __device__ __forceinline__ void hx_wait_for_primary() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void hx_release_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
 template <class... KArgs, class... Args>
@@ -241,12 +246,7 @@ inline cudaError_t hx_launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3
     cudaLaunchAttribute attr{};
     attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr.val.programmaticStreamSerializationAllowed = 1;
-    // inside a stream capture the ordinary dependency is kept: replayed graphs measured slower with programmatic
-    // edges (all edges of the capacity pass's chain: 1.88 against 1.78 ms per sweep step; the edge into the
-    // scoring kernel alone: 1.78 against 1.77), enqueued launches faster (122 against 129 us per ready batch)
-    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
-    if (cudaStreamIsCapturing(stream, &cap) != cudaSuccess) cap = cudaStreamCaptureStatusNone;
-    cfg.attrs = &attr; cfg.numAttrs = cap == cudaStreamCaptureStatusNone ? 1 : 0;
+    cfg.attrs = &attr; cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 

@@ -240,14 +240,14 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
     // stream (the capacity pass of the previous batch) still runs.  Everything up to sync_with_stream() reads
     // only what no kernel writes (call records, instance classes and capacities, link table, model constants)
     // and writes only shared memory; the prefill queues, the free KV tokens and every buffer of the top-K
-    // lists are touched after it.  The kernels behind this one are released after the wait, so that none of
-    // them can overtake the previous batch either.
+    // lists are touched after it.  The kernels behind this one are released when a block is through (not
+    // earlier: blocks of the binning kernel that become resident beside this one have nothing to do before their
+    // wait and measurably slow the step down), so none of them can overtake the previous batch either.
     bool synced = false;
     auto sync_with_stream = [&] {
         if (synced) return;
         synced = true;
         hx_wait_for_primary();
-        hx_release_dependents();                                  // the first kernel of the capacity pass may get ready behind this one
         if (prm.s.K > 0)
             for (int i = blockIdx.x * nthr + tid; i < HX_ORDER_BINS; i += gridDim.x * nthr) prm.tk.ghist[i] = 0u;
         for (int p = tid; p < Ppad; p += nthr) qPs[p] = p < P ? (unloaded ? 0.0f : T.qP[p]) : HX_INF;
@@ -642,6 +642,7 @@ __global__ void __launch_bounds__(TD == 4 ? 512 : 256, 1) hx_score_kernel(const 
         __syncthreads();
     }
     sync_with_stream();                                           // a block without a tile
+    hx_release_dependents();                                      // the first kernel of the capacity pass may get ready now
     if (prm.s.K > 0) {
         key_lo = __reduce_min_sync(0xffffffffu, key_lo); key_hi = __reduce_max_sync(0xffffffffu, key_hi);
         if (lane == 0) { atomicMin(&key_lohi[0], key_lo); atomicMax(&key_lohi[1], key_hi); }
